@@ -1,0 +1,347 @@
+/*
+ * CPU oracle for the CoRun hot path: the per-request decoder forward pass
+ * (isolated prefill and one decode token), the request-bound random variate
+ * R(seed, t) and the deterministic sampling function S.
+ *
+ * THIS IS TEST INFRASTRUCTURE.  It is deliberately plain and slow, shares no
+ * code with the CUDA path, and must never be reached from the product path.
+ *
+ * What it computes (paper: Background "LLM Inference and Continuous Batching",
+ * Design "Determinism Contract", "Isolated Prefill", "Fixed-Shape Batched
+ * Decode", "Shape-Aligned Sampling", "Determinism Argument"):
+ *   a request's logits are those of the decoder forward pass of that request
+ *   alone (request isolation), so the oracle is the textbook definition of a
+ *   pre-norm GQA decoder with RoPE and a SwiGLU FFN, evaluated per request with
+ *   no batching, paging, graph or split logic.
+ *
+ * Precision: weights are bf16 bit patterns widened exactly; activations and
+ * the KV cache are stored in fp32; every reduction (dot product, mean of
+ * squares, softmax sum, weighted value sum) accumulates in fp64 in plain index
+ * order.  The only loop liberty taken: a matrix product evaluates several
+ * independent rows of activations per weight row at once (each output element
+ * is still one index-ordered fp64 sum), and OpenMP distributes independent
+ * output elements over cores.  No reduction is blocked, split or reordered.
+ *
+ * Pins (tests/test_oracle_*.py): brute-force attention and closed forms, RoPE
+ * norm and relative-position invariants, RMSNorm/SiLU closed forms, fp64 triple
+ * loop GEMM, prefill/decode cache consistency, row independence, degenerate
+ * network closed form, a library decoder on the tiny shape, Philox known
+ * answers, sampler limits and frequencies.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef struct {
+  int32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
+  float rms_eps, rope_theta;
+} orc_shape;
+
+typedef struct {
+  const uint16_t *embed;      /* [vocab, hidden]                      */
+  const uint16_t *lm_head;    /* [vocab, hidden]                      */
+  const uint16_t *final_norm; /* [hidden]                             */
+  const uint16_t *const *attn_norm; /* L x [hidden]                   */
+  const uint16_t *const *wqkv;      /* L x [(nq+2nkv)*hd, hidden]     */
+  const uint16_t *const *wo;        /* L x [hidden, nq*hd]            */
+  const uint16_t *const *mlp_norm;  /* L x [hidden]                   */
+  const uint16_t *const *wgate_up;  /* L x [2*ffn, hidden]            */
+  const uint16_t *const *wdown;     /* L x [hidden, ffn]              */
+} orc_weights;
+
+static inline double bf16_to_f64(uint16_t b) {
+  uint32_t u = ((uint32_t)b) << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return (double)f;
+}
+
+/* ---- elementary operators (exported so the pins can reach each one) ---- */
+
+/* out[r,n] = sum_k W[n,k] * X[r,k], k ascending, fp64 accumulator. */
+void orc_matmul_bf16(const uint16_t *W, int64_t N, int64_t K, const float *X, int64_t R, float *out) {
+  enum { RB = 8 };
+#pragma omp parallel for schedule(static)
+  for (int64_t n = 0; n < N; ++n) {
+    const uint16_t *w = W + n * K;
+    for (int64_t r0 = 0; r0 < R; r0 += RB) {
+      int64_t rb = R - r0 < RB ? R - r0 : RB;
+      double acc[RB];
+      for (int j = 0; j < RB; ++j) acc[j] = 0.0;
+      if (rb == RB) {
+        for (int64_t k = 0; k < K; ++k) {
+          double wk = bf16_to_f64(w[k]);
+          for (int j = 0; j < RB; ++j) acc[j] += wk * (double)X[(r0 + j) * K + k];
+        }
+      } else {
+        for (int64_t k = 0; k < K; ++k) {
+          double wk = bf16_to_f64(w[k]);
+          for (int64_t j = 0; j < rb; ++j) acc[j] += wk * (double)X[(r0 + j) * K + k];
+        }
+      }
+      for (int64_t j = 0; j < rb; ++j) out[(r0 + j) * N + n] = (float)acc[j];
+    }
+  }
+}
+
+/* out_i = x_i * g_i / sqrt(mean_j x_j^2 + eps) */
+void orc_rmsnorm(const float *x, const uint16_t *g, int64_t H, float eps, float *out) {
+  double ss = 0.0;
+  for (int64_t i = 0; i < H; ++i) ss += (double)x[i] * (double)x[i];
+  double inv = 1.0 / sqrt(ss / (double)H + (double)eps);
+  for (int64_t i = 0; i < H; ++i) out[i] = (float)((double)x[i] * inv * bf16_to_f64(g[i]));
+}
+
+/* Half-split rotary embedding of one head vector at position pos:
+ * pair (i, i+hd/2) is rotated by the angle pos * theta^(-2i/hd). */
+void orc_rope(float *v, int32_t head_dim, int64_t pos, float theta) {
+  int32_t half = head_dim / 2;
+  for (int32_t i = 0; i < half; ++i) {
+    double freq = pow((double)theta, -2.0 * (double)i / (double)head_dim);
+    double ang = (double)pos * freq;
+    double c = cos(ang), s = sin(ang);
+    double a = v[i], b = v[i + half];
+    v[i] = (float)(a * c - b * s);
+    v[i + half] = (float)(a * s + b * c);
+  }
+}
+
+double orc_silu(double z) { return z / (1.0 + exp(-z)); }
+
+/* Causal softmax attention of one query token at position p over cached
+ * positions 0..p (its own key included).  q: [nq, hd]; K, V: rows of
+ * nkv*hd floats with stride `stride` floats between positions. */
+void orc_attention(const float *q, const float *K, const float *V, int64_t stride, int64_t p,
+                   int32_t nq, int32_t nkv, int32_t hd, float *out) {
+  int32_t group = nq / nkv;
+  double scale = 1.0 / sqrt((double)hd);
+#pragma omp parallel for schedule(static)
+  for (int32_t j = 0; j < nq; ++j) {
+    int32_t g = j / group;
+    double *s = (double *)malloc(sizeof(double) * (size_t)(p + 1));
+    double m = -INFINITY;
+    for (int64_t t = 0; t <= p; ++t) {
+      const float *k = K + t * stride + (int64_t)g * hd;
+      double d = 0.0;
+      for (int32_t i = 0; i < hd; ++i) d += (double)q[j * hd + i] * (double)k[i];
+      s[t] = d * scale;
+      if (s[t] > m) m = s[t];
+    }
+    double z = 0.0;
+    for (int64_t t = 0; t <= p; ++t) {
+      s[t] = exp(s[t] - m);
+      z += s[t];
+    }
+    for (int32_t i = 0; i < hd; ++i) {
+      double o = 0.0;
+      for (int64_t t = 0; t <= p; ++t) o += s[t] * (double)V[t * stride + (int64_t)g * hd + i];
+      out[j * hd + i] = (float)(o / z);
+    }
+    free(s);
+  }
+}
+
+/* ---- the forward pass ---- */
+
+/*
+ * Runs tokens[0..T) of ONE request at positions pos0..pos0+T-1 through the
+ * decoder.  Kc/Vc: the request's cache, [L][max_T][nkv*hd] fp32; positions
+ * below pos0 must already be filled, positions pos0.. are written.
+ * logits: [T, vocab] if all_logits, else [vocab] for the last token; may be
+ * NULL to skip the LM head.  Returns 0, or -1 on a bad argument.
+ * Prefill is T = prompt length at pos0 = 0; a decode step is T = 1.
+ */
+int orc_forward(const orc_shape *sh, const orc_weights *w, const int32_t *tokens, int64_t T, int64_t pos0,
+                float *Kc, float *Vc, int64_t max_T, float *logits, int all_logits) {
+  const int64_t H = sh->hidden, nq = sh->n_q_heads, nkv = sh->n_kv_heads, hd = sh->head_dim;
+  const int64_t F = sh->ffn, Vn = sh->vocab, L = sh->n_layers;
+  const int64_t QD = nq * hd, KD = nkv * hd, QKV = QD + 2 * KD;
+  if (T <= 0 || pos0 < 0 || pos0 + T > max_T || nq % nkv || hd % 2) return -1;
+  for (int64_t t = 0; t < T; ++t)
+    if (tokens[t] < 0 || tokens[t] >= Vn) return -1;
+
+  float *h = (float *)malloc(sizeof(float) * T * H);
+  float *a = (float *)malloc(sizeof(float) * T * (H > F ? H : F));
+  float *qkv = (float *)malloc(sizeof(float) * T * QKV);
+  float *o = (float *)malloc(sizeof(float) * T * QD);
+  float *y = (float *)malloc(sizeof(float) * T * H);
+  float *gu = (float *)malloc(sizeof(float) * T * 2 * F);
+
+  for (int64_t t = 0; t < T; ++t)
+    for (int64_t i = 0; i < H; ++i) h[t * H + i] = (float)bf16_to_f64(w->embed[(int64_t)tokens[t] * H + i]);
+
+  for (int64_t l = 0; l < L; ++l) {
+    float *Kl = Kc + l * max_T * KD, *Vl = Vc + l * max_T * KD;
+    for (int64_t t = 0; t < T; ++t) orc_rmsnorm(h + t * H, w->attn_norm[l], H, sh->rms_eps, a + t * H);
+    orc_matmul_bf16(w->wqkv[l], QKV, H, a, T, qkv);
+    for (int64_t t = 0; t < T; ++t) {
+      float *row = qkv + t * QKV;
+      int64_t p = pos0 + t;
+      for (int64_t j = 0; j < nq; ++j) orc_rope(row + j * hd, (int32_t)hd, p, sh->rope_theta);
+      for (int64_t g = 0; g < nkv; ++g) orc_rope(row + QD + g * hd, (int32_t)hd, p, sh->rope_theta);
+      memcpy(Kl + p * KD, row + QD, sizeof(float) * KD);
+      memcpy(Vl + p * KD, row + QD + KD, sizeof(float) * KD);
+    }
+    for (int64_t t = 0; t < T; ++t)
+      orc_attention(qkv + t * QKV, Kl, Vl, KD, pos0 + t, (int32_t)nq, (int32_t)nkv, (int32_t)hd, o + t * QD);
+    orc_matmul_bf16(w->wo[l], H, QD, o, T, y);
+    for (int64_t i = 0; i < T * H; ++i) h[i] = h[i] + y[i];
+    for (int64_t t = 0; t < T; ++t) orc_rmsnorm(h + t * H, w->mlp_norm[l], H, sh->rms_eps, a + t * H);
+    orc_matmul_bf16(w->wgate_up[l], 2 * F, H, a, T, gu);
+    for (int64_t t = 0; t < T; ++t)
+      for (int64_t i = 0; i < F; ++i) {
+        double g = gu[t * 2 * F + i], u = gu[t * 2 * F + F + i];
+        a[t * F + i] = (float)(orc_silu(g) * u);
+      }
+    orc_matmul_bf16(w->wdown[l], H, F, a, T, y);
+    for (int64_t i = 0; i < T * H; ++i) h[i] = h[i] + y[i];
+  }
+
+  if (logits) {
+    if (all_logits) {
+      for (int64_t t = 0; t < T; ++t) orc_rmsnorm(h + t * H, w->final_norm, H, sh->rms_eps, a + t * H);
+      orc_matmul_bf16(w->lm_head, Vn, H, a, T, logits);
+    } else {
+      orc_rmsnorm(h + (T - 1) * H, w->final_norm, H, sh->rms_eps, a);
+      orc_matmul_bf16(w->lm_head, Vn, H, a, 1, logits);
+    }
+  }
+  free(h); free(a); free(qkv); free(o); free(y); free(gu);
+  return 0;
+}
+
+/* ---- request-bound random variate R(seed, t) ---- */
+
+/* Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw: "Parallel random
+ * numbers: as easy as 1, 2, 3", SC'11): multipliers 0xD2511F53 / 0xCD9E8D57,
+ * key schedule increments 0x9E3779B9 / 0xBB67AE85. */
+void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+  uint32_t k0 = key[0], k1 = key[1];
+  for (int r = 0; r < 10; ++r) {
+    uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+    uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+    uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+    uint32_t n1 = (uint32_t)p1;
+    uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+    uint32_t n3 = (uint32_t)p0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* R(seed, t): the top 24 bits of the first Philox word with key = seed and
+ * counter = (t, 0, 0, 0); the variate is u24 / 2^24 in [0, 1).  Stateless, so
+ * padding cannot consume it and moving slots cannot shift it. */
+uint32_t orc_variate_u24(uint64_t seed, uint64_t t) {
+  uint32_t ctr[4] = {(uint32_t)t, (uint32_t)(t >> 32), 0u, 0u};
+  uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  uint32_t out[4];
+  orc_philox4x32_10(ctr, key, out);
+  return out[0] >> 8;
+}
+
+/* ---- sampling function S ---- */
+
+typedef struct {
+  int64_t idx;
+  float logit;
+} orc_item;
+
+static int orc_item_desc(const void *pa, const void *pb) {
+  const orc_item *a = (const orc_item *)pa, *b = (const orc_item *)pb;
+  if (a->logit > b->logit) return -1;
+  if (a->logit < b->logit) return 1;
+  return a->idx < b->idx ? -1 : (a->idx > b->idx ? 1 : 0);
+}
+
+/*
+ * S(logits, u24).  temperature == 0: argmax, lowest id on ties.  Otherwise:
+ *   weight_i = floor(2^40 * exp((logit_i - max) / temperature))   (integer)
+ *   total    = sum_i weight_i ;  cut = floor(top_p * total)
+ *   nucleus  = tokens in descending logit order (ties: lower id first) up to
+ *              and including the first whose running weight sum >= cut
+ *   Z = nucleus weight ;  r = floor(u24 * Z / 2^24)
+ *   token    = first nucleus member, in ascending id order, whose running
+ *              weight sum exceeds r.
+ * The integer weights make every later decision exact.  `margin` (optional)
+ * receives how close, relative to `total`, the decision came to flipping
+ * (min of: distance of r to the nearest running-sum boundary, distance of the
+ * cut to the running sums adjacent to the nucleus edge).
+ */
+int32_t orc_sample(const float *logits, int64_t V, float temperature, float top_p, uint32_t u24, double *margin) {
+  int64_t best = 0;
+  for (int64_t i = 1; i < V; ++i)
+    if (logits[i] > logits[best]) best = i;
+  if (margin) *margin = 1.0;
+  if (temperature <= 0.0f) return (int32_t)best;
+
+  double mx = (double)logits[best];
+  uint64_t *wgt = (uint64_t *)malloc(sizeof(uint64_t) * (size_t)V);
+  orc_item *it = (orc_item *)malloc(sizeof(orc_item) * (size_t)V);
+  uint64_t total = 0;
+  for (int64_t i = 0; i < V; ++i) {
+    double e = exp(((double)logits[i] - mx) / (double)temperature);
+    wgt[i] = (uint64_t)floor(ldexp(e, 40));
+    total += wgt[i];
+    it[i].idx = i;
+    it[i].logit = logits[i];
+  }
+  qsort(it, (size_t)V, sizeof(orc_item), orc_item_desc);
+  uint64_t cut = (uint64_t)floor((double)top_p * (double)total);
+  if (cut > total) cut = total;
+  char *in = (char *)calloc((size_t)V, 1);
+  uint64_t run = 0, Z = 0;
+  double mg = 1.0;
+  for (int64_t r = 0; r < V; ++r) {
+    uint64_t before = run;
+    run += wgt[it[r].idx];
+    in[it[r].idx] = 1;
+    if (run >= cut) {
+      Z = run;
+      double d1 = (double)(run - cut) / (double)total;          /* cut just reached        */
+      double d0 = (double)(cut - before) / (double)total;       /* cut not reached before  */
+      mg = d1 < d0 ? d1 : d0;
+      if (cut >= total) mg = 1.0;  /* everything is kept: no edge to flip */
+      break;
+    }
+  }
+  unsigned __int128 prod = (unsigned __int128)u24 * (unsigned __int128)Z;
+  uint64_t rdraw = (uint64_t)(prod >> 24);
+  int32_t tok = -1;
+  run = 0;
+  for (int64_t i = 0; i < V; ++i) {
+    if (!in[i]) continue;
+    uint64_t before = run;
+    run += wgt[i];
+    if (run > rdraw) {
+      tok = (int32_t)i;
+      double d0 = (double)(rdraw - before) / (double)total;
+      double d1 = (double)(run - rdraw) / (double)total;
+      if (d0 < mg) mg = d0;
+      if (d1 < mg) mg = d1;
+      break;
+    }
+  }
+  if (margin) *margin = mg;
+  free(wgt); free(it); free(in);
+  return tok;
+}
+
+int orc_num_threads(void) {
+  int n = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+  {
+#pragma omp master
+    n = omp_get_num_threads();
+  }
+#endif
+  return n;
+}

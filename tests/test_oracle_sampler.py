@@ -1,0 +1,126 @@
+"""Pins for R(seed, t) and the sampling function S of the oracle."""
+import math
+import os
+
+import numpy as np
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_kat.txt")
+
+
+def test_philox_known_answers(orc):
+    n = 0
+    for line in open(GOLD):
+        if line.startswith("#") or not line.strip():
+            continue
+        w = [int(x, 16) for x in line.split()]
+        out = orc.philox4x32_10(w[0:4], w[4:6])
+        assert [int(x) for x in out] == w[6:10]
+        n += 1
+    assert n == 3
+
+
+def test_variate_is_first_word_top_24_bits(orc):
+    for seed, t in [(0, 0), (1042, 7), (2**40 + 5, 3)]:
+        w = orc.philox4x32_10([t, 0, 0, 0], [seed & 0xFFFFFFFF, seed >> 32])
+        assert orc.variate_u24(seed, t) == int(w[0]) >> 8
+
+
+def test_variate_uniformity_over_steps_and_seeds(orc):
+    for gen in (lambda i: orc.variate_u24(1042, i), lambda i: orc.variate_u24(i, 5)):
+        u = np.array([gen(i) for i in range(1 << 16)], dtype=np.float64) / 2**24
+        hist, _ = np.histogram(u, bins=64, range=(0, 1))
+        chi2 = float(((hist - 1024.0) ** 2 / 1024.0).sum())
+        assert chi2 < 120.0            # 63 dof: P(chi2 > 120) ~ 2e-5
+        assert abs(np.corrcoef(u[:-1], u[1:])[0, 1]) < 0.02
+
+
+def test_greedy_is_argmax_lowest_id_on_ties(orc):
+    lg = np.array([0.1, 2.0, -1.0, 2.0, 0.5], np.float32)
+    assert orc.sample(lg, 0.0, 1.0, 12345)[0] == 1
+    assert orc.sample(lg[::-1].copy(), 0.0, 1.0, 0)[0] == 1
+
+
+def test_small_temperature_and_small_top_p_give_argmax(orc):
+    rng = np.random.default_rng(0)
+    lg = rng.standard_normal(500).astype(np.float32)
+    am = int(np.argmax(lg))
+    for u in (0, 1 << 23, (1 << 24) - 1):
+        assert orc.sample(lg, 1e-3, 1.0, u)[0] == am
+        assert orc.sample(lg, 1.0, 1e-6, u)[0] == am
+
+
+def _flip_point(orc, lg, T, top_p, lo_tok):
+    """smallest u24 for which S no longer returns lo_tok (bisection; S is monotone in u)."""
+    lo, hi = 0, 1 << 24
+    while lo < hi:
+        mid = (lo + hi) // 2
+        if orc.sample(lg, T, top_p, mid)[0] == lo_tok:
+            lo = mid + 1
+        else:
+            hi = mid
+    return lo
+
+
+def test_two_logits_closed_form(orc):
+    for (l0, l1, T) in [(0.3, -0.4, 0.7), (1.0, 1.0, 1.0), (-2.0, 1.5, 0.6)]:
+        lg = np.array([l0, l1], np.float32)
+        u = _flip_point(orc, lg, T, 1.0, 0)
+        want = 1.0 / (1.0 + math.exp(-(float(lg[0]) - float(lg[1])) / T))
+        assert abs(u / 2**24 - want) < 2e-7
+
+
+def test_top_p_nucleus_and_id_ordered_inverse_cdf(orc):
+    # probabilities .05 .5 .15 .3 at ids 0..3 ; top_p .9 -> nucleus = ids {1,3,2}
+    # (descending p: .5, .3, .15 -> cumulative .95 >= .9), id 0 is cut.
+    p = np.array([0.05, 0.5, 0.15, 0.3])
+    lg = np.log(p).astype(np.float32)
+    Z = 0.95
+    # inverse CDF walks ids ascending: id1 [0,.5), id2 [.5,.65), id3 [.65,.95) of Z
+    edges = {1: 0.5 / Z, 2: 0.65 / Z}
+    assert orc.sample(lg, 1.0, 0.9, 0)[0] == 1
+    assert abs(_flip_point(orc, lg, 1.0, 0.9, 1) / 2**24 - edges[1]) < 1e-6
+    u12 = _flip_point(orc, lg, 1.0, 0.9, 1)
+    assert orc.sample(lg, 1.0, 0.9, u12)[0] == 2
+    # after id 2 comes id 3, never id 0
+    seen = {orc.sample(lg, 1.0, 0.9, u)[0] for u in range(0, 1 << 24, 4099)}
+    assert seen == {1, 2, 3}
+    # the crossing token is included: top_p .8 -> {1,3} exactly reaches .8
+    seen = {orc.sample(lg, 1.0, 0.79, u)[0] for u in range(0, 1 << 24, 4099)}
+    assert seen == {1, 3}
+    seen = {orc.sample(lg, 1.0, 0.45, u)[0] for u in range(0, 1 << 24, 4099)}
+    assert seen == {1}
+    # top_p = 1 keeps everything and reduces to the plain inverse CDF
+    assert abs(_flip_point(orc, lg, 1.0, 1.0, 0) / 2**24 - 0.05) < 1e-6
+
+
+def test_temperature_divides_logits(orc):
+    lg = np.array([0.0, 1.0], np.float32)
+    u = _flip_point(orc, lg, 0.5, 1.0, 0)
+    assert abs(u / 2**24 - 1.0 / (1.0 + math.exp(2.0))) < 2e-7
+
+
+def test_ties_enter_nucleus_lower_id_first(orc):
+    lg = np.zeros(4, np.float32)     # four equal tokens, top_p .5 -> ids {0,1}
+    seen = {orc.sample(lg, 1.0, 0.5, u)[0] for u in range(0, 1 << 24, 65537)}
+    assert seen == {0, 1}
+
+
+def test_frequencies_match_probabilities(orc):
+    rng = np.random.default_rng(1)
+    lg = rng.standard_normal(12).astype(np.float32)
+    T = 0.7
+    p = np.exp(lg.astype(np.float64) / T); p /= p.sum()
+    n = 100000
+    cnt = np.zeros(12)
+    for i in range(n):
+        cnt[orc.sample(lg, T, 1.0, orc.variate_u24(1000 + i, 3))[0]] += 1
+    chi2 = float(((cnt - n * p) ** 2 / (n * p)).sum())
+    assert chi2 < 45.0                 # 11 dof: P(chi2 > 45) ~ 5e-6
+
+
+def test_margin_reports_closeness_to_a_boundary(orc):
+    lg = np.array([0.0, 0.0], np.float32)
+    tok, m = orc.sample(lg, 1.0, 1.0, 1 << 23)          # exactly on the edge between the two
+    assert tok == 1 and m < 1e-6
+    tok, m = orc.sample(lg, 1.0, 1.0, 1 << 22)
+    assert tok == 0 and abs(m - 0.25) < 1e-6
