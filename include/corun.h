@@ -1,0 +1,190 @@
+/*
+ * corun.h -- C ABI of the CoRun hot path for NVIDIA B200 (sm_100a).
+ *
+ * One engine = one GPU, one model, ONE fixed padded decode shape (B slots,
+ * max_context).  A request lives in a slot: corun_prefill runs its prompt alone
+ * (batch of one, natural length, fixed-size chunks) and fills the slot's paged
+ * KV cache; corun_decode_step runs one fixed-shape decode iteration over all B
+ * slots, with padding in the unused ones, as a single CUDA-graph replay.
+ *
+ * Guarantee (paper, Design, "Determinism Contract" and "Determinism Argument"):
+ * within one engine the logits and tokens of a request are bitwise identical
+ * whatever slot it occupies, whatever requests or padding occupy the other
+ * slots, and across repeated runs.  Nothing is promised across different B,
+ * max_context, GPUs or library builds (same section, non-claims).
+ *
+ * Conventions
+ *   - every function returns 0 (CORUN_OK) or a negative corun_status; nothing
+ *     aborts, throws or traps;
+ *   - "device" pointers are CUDA device memory of the current device, "host"
+ *     pointers ordinary host memory;
+ *   - weight memory is BORROWED: allocated by the caller, never written, and it
+ *     must outlive the engine.  Everything else (KV pool, block tables,
+ *     workspaces, logits, the graph) is owned by the engine;
+ *   - host arrays are read/written only during the call; calls are synchronous
+ *     unless stated otherwise; an engine is not thread-safe;
+ *   - all kernels run on the stream given to corun_init.
+ */
+#ifndef CORUN_H_
+#define CORUN_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  CORUN_OK = 0,
+  CORUN_EINVAL = -1,   /* NULL pointer, bad shape, bad argument                         */
+  CORUN_ESLOT = -2,    /* slot out of range; busy on prefill; empty on decode / release */
+  CORUN_ENOSPACE = -3, /* the KV pool cannot hold the request's full reserved sequence  */
+  CORUN_ECTX = -4,     /* an active slot would exceed its reserved length               */
+  CORUN_ECUDA = -5,    /* a CUDA call failed (corun_last_cuda_error has the code)       */
+  CORUN_ETIMEOUT = -6, /* a bounded device-side wait expired (device status word)       */
+  CORUN_ENOMEM = -7    /* device or host allocation failed                              */
+} corun_status;
+
+typedef struct corun_engine corun_engine; /* opaque, owned by the library */
+
+/* Decoder shape.  arch 0 = dense GQA decoder: pre-norm RMSNorm, half-split
+ * RoPE on q and k, causal softmax attention, SwiGLU FFN, untied LM head, no
+ * biases.  Requirements: hidden, ffn and n_q_heads*head_dim multiples of 64;
+ * head_dim 64 or 128; n_q_heads / n_kv_heads in {1,2,4,8}. */
+typedef struct {
+  int32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
+  float rms_eps, rope_theta;
+  int32_t arch;
+} corun_shape;
+
+/* Device pointers to bf16 weights, row-major [out_features, in_features].
+ *   embed [vocab, hidden]; lm_head [vocab, hidden]; final_norm [hidden];
+ *   per layer (arrays of n_layers device pointers, the arrays themselves on the host):
+ *   attn_norm [hidden]; wqkv [(nq+2nkv)*hd, hidden] (q rows, then k, then v);
+ *   wo [hidden, nq*hd]; mlp_norm [hidden]; wgate_up [2*ffn, hidden] (gate rows,
+ *   then up rows); wdown [hidden, ffn].
+ * Matrix base addresses must be 16-byte aligned. */
+typedef struct {
+  const void *embed, *lm_head, *final_norm;
+  const void *const *attn_norm, *const *wqkv, *const *wo;
+  const void *const *mlp_norm, *const *wgate_up, *const *wdown;
+} corun_weights;
+
+/* temperature <= 0 selects greedy argmax (lowest id on ties); otherwise
+ * temperature -> softmax -> top-p nucleus -> inverse CDF (see corun_decode_step). */
+typedef struct {
+  float temperature, top_p;
+} corun_sampling;
+
+/*
+ * Creates an engine for the fixed decode shape (B, max_context) and captures
+ * its decode graph (paper, Design, "Fixed-Shape Batched Decode": one captured
+ * shape equal to the maximum concurrency, replayed for every decode iteration).
+ *   B               1..256 slots.
+ *   max_context     largest prompt + generated length of any request.
+ *   kv_block        tokens per KV page; must be 16.
+ *   kv_pool_blocks  pages in the pool; 0 = B * ceil(max_context / kv_block).
+ *   cuda_stream     a cudaStream_t (NULL = the legacy default stream).
+ * Errors: EINVAL, ENOMEM, ECUDA.  On success *out owns device memory until
+ * corun_destroy.
+ */
+int corun_init(const corun_shape *shape, const corun_weights *weights, int32_t B, int32_t max_context,
+               int32_t kv_block, int64_t kv_pool_blocks, void *cuda_stream, corun_engine **out);
+
+/*
+ * Isolated prefill (paper, Design, "Isolated Prefill"; Algorithm 1's admission
+ * rule): runs the n prompt tokens of one request alone, in fixed-size chunks
+ * whose sequence depends on n only, writes its KV cache, samples the first
+ * token with R(seed, 0) from the last position's logits ("Shape-Aligned
+ * Sampling": prefill presents one sampling row) and leaves that token pending
+ * for the slot's first decode step.
+ *   tokens       host, n ids in [0, vocab).
+ *   reserve_len  prompt + maximum new tokens, <= max_context; pages for the
+ *                whole reserved sequence are taken now, so a later decode step
+ *                can never run out (no preemption, no recompute).
+ *   out_first_token  host, may be NULL.
+ * Errors: EINVAL; ESLOT (slot busy / out of range); ENOSPACE (reservation does
+ * not fit; the engine is unchanged); ECUDA; ETIMEOUT.
+ */
+int corun_prefill(corun_engine *e, int32_t slot, const int32_t *tokens, int32_t n, int32_t reserve_len,
+                  const corun_sampling *sampling, uint64_t seed, int32_t *out_first_token);
+
+/*
+ * One fixed-shape decode iteration (paper, Design, "Fixed-Shape Batched
+ * Decode", "Shape-Aligned Sampling", "Determinism Argument"): every slot with
+ * active[s] != 0 feeds its pending token at position = its context length,
+ * appends K/V, attends over its own pages with a split count and combine order
+ * that depend on its own length only, and samples token = S(logits, R(seeds[s], t_s))
+ * where t_s counts the tokens this request has sampled so far (prefill used
+ * t = 0).  Inactive and empty slots are padding: they run through the same
+ * launch shape, consume no random variate, change no state and report -1.
+ *   active      host, B bytes.       seeds  host, B values (read where active).
+ *   out_tokens  host, B ints.
+ * Sampling: weight_i = floor(2^40 * exp((logit_i - max)/T)); nucleus = tokens
+ * by descending logit (ties: lower id first) up to and including the first
+ * whose running weight reaches floor(top_p * total); draw r = floor(u24 * Z / 2^24)
+ * with u24 the top 24 bits of Philox4x32-10(key = seed, counter = (t,0,0,0));
+ * the token is the first nucleus member in ascending id order whose running
+ * weight exceeds r.
+ * Errors: EINVAL; ESLOT (an active slot is empty); ECTX (an active slot is at
+ * its reserved length: the whole step is refused and nothing changes); ECUDA;
+ * ETIMEOUT.
+ */
+int corun_decode_step(corun_engine *e, const uint8_t *active, const uint64_t *seeds, int32_t *out_tokens);
+
+/* Asynchronous form for back-to-back replays: stages active/seeds and enqueues
+ * one decode iteration on the engine's stream without waiting.  Results of the
+ * last enqueued step are fetched by corun_decode_wait (out_tokens host, B ints,
+ * may be NULL).  Same semantics and errors as corun_decode_step. */
+int corun_decode_enqueue(corun_engine *e, const uint8_t *active, const uint64_t *seeds);
+int corun_decode_wait(corun_engine *e, int32_t *out_tokens);
+
+/* Frees the slot's pages and clears its state (host only).  ESLOT if empty. */
+int corun_release(corun_engine *e, int32_t slot);
+
+/* Destroys the engine and frees what it owns.  NULL is allowed. */
+void corun_destroy(corun_engine *e);
+
+/* ---- accessors used by tests and reports ---- */
+
+/* Logits row (vocab floats, host) of the slot's latest forward pass. */
+int corun_get_logits(corun_engine *e, int32_t slot, float *out);
+/* Replaces the slot's pending token (teacher forcing). */
+int corun_force_token(corun_engine *e, int32_t slot, int32_t token);
+/* Cached tokens of the slot, or a negative status. */
+int corun_context_len(corun_engine *e, int32_t slot);
+/* Free pages left in the pool, or a negative status. */
+int64_t corun_free_blocks(corun_engine *e);
+/* Reads / writes n cached positions [pos0, pos0+n) of one layer as fp32 rows of
+ * n_kv_heads*head_dim (host).  Writing beyond the current context length
+ * extends it (up to reserve_len); values are rounded to the cache's fp16. */
+int corun_debug_kv_read(corun_engine *e, int32_t slot, int32_t layer, int32_t pos0, int32_t n, float *k, float *v);
+int corun_debug_kv_write(corun_engine *e, int32_t slot, int32_t layer, int32_t pos0, int32_t n, const float *k,
+                         const float *v);
+/* Occupies an empty slot without running a prefill: reserves pages, sets the
+ * context length to n_ctx (cache contents undefined until written with
+ * corun_debug_kv_write), the pending token and the sampling state. */
+int corun_debug_adopt(corun_engine *e, int32_t slot, int32_t n_ctx, int32_t reserve_len, int32_t pending_token,
+                      const corun_sampling *sampling, int32_t step);
+/* eager != 0: launch the decode kernels one by one instead of replaying the graph. */
+int corun_debug_set_eager(corun_engine *e, int32_t eager);
+/* Number of kernel launches in one decode iteration. */
+int corun_decode_launches(corun_engine *e);
+/* Stand-alone run of the decode GEMM: out[r, n] = sum_k W[n, k] * X[r, k] with X
+ * fp32 [R, K] (device), W bf16 [N, K] (device), out fp32 [R, N] (device); R <= 256,
+ * K % 64 == 0.  Uses the engine-independent kernel path (split activations,
+ * tcgen05 MMA, fixed K order). */
+int corun_debug_gemm(const void *W, int32_t N, int32_t K, const float *X, int32_t R, float *out, void *cuda_stream);
+/* R(seed, t) as the engine computes it (top 24 bits of the first Philox word), on the device. */
+int corun_debug_variate(uint64_t seed, uint64_t t, uint32_t *out_u24 /* host */);
+/* Runs the engine's sampler on host logits rows [n_rows, vocab] (copied to the device). */
+int corun_debug_sample(const float *logits, int32_t n_rows, int32_t vocab, const corun_sampling *sampling,
+                       const uint32_t *u24, int32_t *out_tokens);
+
+const char *corun_strerror(int status);
+int corun_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CORUN_H_ */

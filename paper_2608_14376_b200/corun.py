@@ -1,0 +1,251 @@
+"""ctypes binding of the C ABI in ``include/corun.h`` (argument marshalling only).
+
+Every step of the hot path runs in the CUDA kernels of ``libcorun.so``; there
+is no CPU or PyTorch fallback: if the library is missing or the call fails, an
+exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcorun.so")
+
+OK, EINVAL, ESLOT, ENOSPACE, ECTX, ECUDA, ETIMEOUT, ENOMEM = 0, -1, -2, -3, -4, -5, -6, -7
+
+EXPORTS = [
+    "corun_init", "corun_prefill", "corun_decode_step", "corun_decode_enqueue", "corun_decode_wait",
+    "corun_release", "corun_destroy", "corun_get_logits", "corun_force_token", "corun_context_len",
+    "corun_free_blocks", "corun_debug_kv_read", "corun_debug_kv_write", "corun_debug_adopt",
+    "corun_debug_set_eager", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
+    "corun_debug_sample", "corun_strerror", "corun_last_cuda_error",
+]
+
+
+class CorunError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().corun_strerror(status).decode()
+        extra = f" (cuda error {lib().corun_last_cuda_error()})" if status == ECUDA else ""
+        super().__init__(f"{where}: {msg}{extra} [{status}]")
+
+
+class Shape(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in
+                ("n_layers", "hidden", "n_q_heads", "n_kv_heads", "head_dim", "ffn", "vocab")] + [
+        ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("arch", C.c_int32)]
+
+
+_PP = C.POINTER(C.c_void_p)
+
+
+class Weights(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p),
+                ("attn_norm", _PP), ("wqkv", _PP), ("wo", _PP), ("mlp_norm", _PP), ("wgate_up", _PP), ("wdown", _PP)]
+
+
+class Sampling(C.Structure):
+    _fields_ = [("temperature", C.c_float), ("top_p", C.c_float)]
+
+
+_lib = None
+
+
+def lib():
+    """Loads libcorun.so (built in-tree by ``paper_2608_14376_b200.build``); fails loudly if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2608_14376_b200.build` "
+                               "(there is no fallback path)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, u64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64
+        L.corun_init.argtypes = [C.POINTER(Shape), C.POINTER(Weights), i32, i32, i32, i64, vp, C.POINTER(vp)]
+        L.corun_prefill.argtypes = [vp, i32, vp, i32, i32, C.POINTER(Sampling), u64, C.POINTER(i32)]
+        L.corun_decode_step.argtypes = [vp, vp, vp, vp]
+        L.corun_decode_enqueue.argtypes = [vp, vp, vp]
+        L.corun_decode_wait.argtypes = [vp, vp]
+        L.corun_release.argtypes = [vp, i32]
+        L.corun_destroy.argtypes = [vp]
+        L.corun_destroy.restype = None
+        L.corun_get_logits.argtypes = [vp, i32, vp]
+        L.corun_force_token.argtypes = [vp, i32, i32]
+        L.corun_context_len.argtypes = [vp, i32]
+        L.corun_free_blocks.argtypes = [vp]
+        L.corun_free_blocks.restype = i64
+        L.corun_debug_kv_read.argtypes = [vp, i32, i32, i32, i32, vp, vp]
+        L.corun_debug_kv_write.argtypes = [vp, i32, i32, i32, i32, vp, vp]
+        L.corun_debug_adopt.argtypes = [vp, i32, i32, i32, i32, C.POINTER(Sampling), i32]
+        L.corun_debug_set_eager.argtypes = [vp, i32]
+        L.corun_decode_launches.argtypes = [vp]
+        L.corun_debug_gemm.argtypes = [vp, i32, i32, vp, i32, vp, vp]
+        L.corun_debug_variate.argtypes = [u64, u64, C.POINTER(C.c_uint32)]
+        L.corun_debug_sample.argtypes = [vp, i32, i32, C.POINTER(Sampling), vp, vp]
+        L.corun_strerror.argtypes = [C.c_int]
+        L.corun_strerror.restype = C.c_char_p
+        L.corun_last_cuda_error.argtypes = []
+        for n in EXPORTS:
+            getattr(L, n)
+        _lib = L
+    return _lib
+
+
+def _check(rc: int, where: str):
+    if rc != OK:
+        raise CorunError(rc, where)
+
+
+class Engine:
+    """One engine = one fixed decode shape (B, max_context) on the current CUDA device.
+
+    ``weights``: dict of torch bf16 CUDA tensors laid out as ``corun_weights``
+    describes (see ``synth.make_weights_*``); they are borrowed, keep them alive.
+    """
+
+    def __init__(self, shape, weights: dict, B: int, max_context: int, kv_pool_blocks: int = 0, stream=None):
+        import torch
+
+        self._torch = torch
+        self.shape, self.B, self.max_context = shape, B, max_context
+        self._weights = weights
+        d = shape.dict() if hasattr(shape, "dict") else dict(shape)
+        self._cs = Shape(d["n_layers"], d["hidden"], d["n_q_heads"], d["n_kv_heads"], d["head_dim"], d["ffn"],
+                         d["vocab"], d["rms_eps"], d["rope_theta"], 0)
+        cw = Weights()
+        self._arrs = {}
+        for k in ("embed", "lm_head", "final_norm"):
+            t = weights[k]
+            assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+            setattr(cw, k, t.data_ptr())
+        for k in ("attn_norm", "wqkv", "wo", "mlp_norm", "wgate_up", "wdown"):
+            ts = weights[k]
+            assert len(ts) == d["n_layers"]
+            for t in ts:
+                assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+            arr = (C.c_void_p * len(ts))(*[t.data_ptr() for t in ts])
+            self._arrs[k] = arr
+            setattr(cw, k, C.cast(arr, _PP))
+        self._cw = cw
+        torch.cuda.synchronize()
+        h = C.c_void_p()
+        _check(lib().corun_init(C.byref(self._cs), C.byref(cw), B, max_context, 16, kv_pool_blocks,
+                                C.c_void_p(stream) if stream else None, C.byref(h)), "corun_init")
+        self._h = h
+        self.vocab = d["vocab"]
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().corun_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the four calls of the boundary
+    def prefill(self, slot: int, tokens, reserve_len: int, temperature: float = 0.0, top_p: float = 1.0,
+                seed: int = 0) -> int:
+        t = np.ascontiguousarray(tokens, dtype=np.int32)
+        s = Sampling(temperature, top_p)
+        first = C.c_int32(-1)
+        _check(lib().corun_prefill(self._h, slot, t.ctypes.data, t.shape[0], reserve_len, C.byref(s),
+                                   seed & (2**64 - 1), C.byref(first)), "corun_prefill")
+        return int(first.value)
+
+    def decode_step(self, active, seeds) -> np.ndarray:
+        a = np.ascontiguousarray(active, dtype=np.uint8)
+        s = np.ascontiguousarray(seeds, dtype=np.uint64)
+        assert a.shape == (self.B,) and s.shape == (self.B,)
+        out = np.empty(self.B, np.int32)
+        _check(lib().corun_decode_step(self._h, a.ctypes.data, s.ctypes.data, out.ctypes.data), "corun_decode_step")
+        return out
+
+    def decode_enqueue(self, active, seeds):
+        a = np.ascontiguousarray(active, dtype=np.uint8)
+        s = np.ascontiguousarray(seeds, dtype=np.uint64)
+        _check(lib().corun_decode_enqueue(self._h, a.ctypes.data, s.ctypes.data), "corun_decode_enqueue")
+
+    def decode_wait(self) -> np.ndarray:
+        out = np.empty(self.B, np.int32)
+        _check(lib().corun_decode_wait(self._h, out.ctypes.data), "corun_decode_wait")
+        return out
+
+    def release(self, slot: int):
+        _check(lib().corun_release(self._h, slot), "corun_release")
+
+    # -- accessors
+    def logits(self, slot: int) -> np.ndarray:
+        out = np.empty(self.vocab, np.float32)
+        _check(lib().corun_get_logits(self._h, slot, out.ctypes.data), "corun_get_logits")
+        return out
+
+    def force_token(self, slot: int, token: int):
+        _check(lib().corun_force_token(self._h, slot, int(token)), "corun_force_token")
+
+    def context_len(self, slot: int) -> int:
+        rc = lib().corun_context_len(self._h, slot)
+        if rc < 0:
+            raise CorunError(rc, "corun_context_len")
+        return rc
+
+    def free_blocks(self) -> int:
+        return int(lib().corun_free_blocks(self._h))
+
+    def kv_read(self, slot: int, layer: int, pos0: int, n: int):
+        kd = self._cs.n_kv_heads * self._cs.head_dim
+        k = np.empty((n, kd), np.float32)
+        v = np.empty((n, kd), np.float32)
+        _check(lib().corun_debug_kv_read(self._h, slot, layer, pos0, n, k.ctypes.data, v.ctypes.data), "kv_read")
+        return k, v
+
+    def kv_write(self, slot: int, layer: int, pos0: int, k, v):
+        k = np.ascontiguousarray(k, dtype=np.float32)
+        v = np.ascontiguousarray(v, dtype=np.float32)
+        _check(lib().corun_debug_kv_write(self._h, slot, layer, pos0, k.shape[0], k.ctypes.data, v.ctypes.data),
+               "kv_write")
+
+    def adopt(self, slot: int, n_ctx: int, reserve_len: int, pending: int, temperature=0.0, top_p=1.0, step=1):
+        s = Sampling(temperature, top_p)
+        _check(lib().corun_debug_adopt(self._h, slot, n_ctx, reserve_len, pending, C.byref(s), step), "adopt")
+
+    def set_eager(self, eager: bool):
+        _check(lib().corun_debug_set_eager(self._h, 1 if eager else 0), "set_eager")
+
+    def decode_launches(self) -> int:
+        return int(lib().corun_decode_launches(self._h))
+
+
+def debug_gemm(W, X):
+    """out[r, n] = sum_k W[n, k] X[r, k]; W torch bf16 [N, K] cuda, X torch fp32 [R, K] cuda."""
+    import torch
+
+    N, K = W.shape
+    R = X.shape[0]
+    out = torch.empty((R, N), dtype=torch.float32, device=X.device)
+    torch.cuda.synchronize()
+    _check(lib().corun_debug_gemm(W.data_ptr(), N, K, X.data_ptr(), R, out.data_ptr(), None), "corun_debug_gemm")
+    return out
+
+
+def debug_variate(seed: int, t: int) -> int:
+    o = C.c_uint32(0)
+    _check(lib().corun_debug_variate(seed & (2**64 - 1), t, C.byref(o)), "corun_debug_variate")
+    return int(o.value)
+
+
+def debug_sample(logits, temperature: float, top_p: float, u24) -> np.ndarray:
+    lg = np.ascontiguousarray(logits, dtype=np.float32)
+    if lg.ndim == 1:
+        lg = lg[None]
+    u = np.ascontiguousarray(u24, dtype=np.uint32).reshape(-1)
+    assert u.shape[0] == lg.shape[0]
+    out = np.empty(lg.shape[0], np.int32)
+    s = Sampling(temperature, top_p)
+    _check(lib().corun_debug_sample(lg.ctypes.data, lg.shape[0], lg.shape[1], C.byref(s), u.ctypes.data,
+                                    out.ctypes.data), "corun_debug_sample")
+    return out

@@ -1,0 +1,727 @@
+// Host side of the C ABI: engine state, paged KV pool, the row program
+// (decode graph / eager prefill) and the debug accessors.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/corun.h"
+#include "gemm.cuh"
+#include "ops.cuh"
+
+using namespace corun;
+
+static int g_last_cuda_error = 0;
+
+#define CK(call)                                   \
+  do {                                             \
+    cudaError_t _e = (call);                       \
+    if (_e != cudaSuccess) {                       \
+      g_last_cuda_error = (int)_e;                 \
+      return CORUN_ECUDA;                          \
+    }                                              \
+  } while (0)
+#define RC(call)                  \
+  do {                            \
+    int _r = (call);              \
+    if (_r != CORUN_OK) return _r; \
+  } while (0)
+
+namespace {
+
+typedef __nv_bfloat16 bf16;
+
+// Buffers and GEMM plans of the row program at one fixed row count.
+struct Program {
+  int R = 0, BN = 0;
+  float *h = nullptr, *q = nullptr, *part_acc = nullptr, *part_ml = nullptr;
+  float *qkv_out = nullptr, *o_out = nullptr, *gu_out = nullptr, *down_out = nullptr, *logits = nullptr, *ws = nullptr;
+  bf16 *xn_hi = nullptr, *xn_lo = nullptr, *ao_hi = nullptr, *ao_lo = nullptr, *ff_hi = nullptr, *ff_lo = nullptr;
+  int *row_token = nullptr, *row_pos = nullptr, *row_active = nullptr, *row_slot = nullptr, *do_sample = nullptr;
+  int *sampled = nullptr;
+  GemmPlan p_qkv, p_o, p_gu, p_down, p_lm;
+  bool has_layers = false, has_lm = false;
+  std::vector<void *> allocs;
+};
+
+}  // namespace
+
+struct corun_engine {
+  corun_shape sh{};
+  int B = 0, max_ctx = 0, max_blocks = 0, max_splits = 0, chunk = 0, num_sms = 0;
+  int64_t pool_blocks = 0;
+  cudaStream_t st = nullptr;
+  bool own_stream = false;
+  const void *w0_qkv = nullptr, *w0_o = nullptr, *w0_gu = nullptr, *w0_down = nullptr;
+  // borrowed weights
+  const bf16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
+  std::vector<const bf16 *> attn_norm, mlp_norm;
+  std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_down;
+  // KV
+  __half *kv_pool = nullptr;
+  size_t layer_stride = 0;
+  int *d_block_table = nullptr;
+  std::vector<int> free_blocks;
+  std::vector<std::vector<int>> slot_blocks;
+  float2 *d_rope = nullptr;
+  // slot state: device
+  int *d_in_use = nullptr, *d_ctx = nullptr, *d_step = nullptr, *d_pending = nullptr;
+  float *d_temp = nullptr, *d_top_p = nullptr;
+  uint64_t *d_seeds = nullptr;
+  uint8_t *d_active = nullptr;
+  int *d_out_tokens = nullptr, *d_status = nullptr;
+  // slot state: host mirrors
+  std::vector<int> in_use, ctx, reserve, step;
+  // pinned staging
+  uint8_t *h_active = nullptr;
+  uint64_t *h_seeds = nullptr;
+  int *h_out_tokens = nullptr, *h_status = nullptr;
+  int *h_rows = nullptr;          // prefill row metadata staging [5][chunk]
+  bool staged_valid = false, in_flight = false;
+  Program dec, pre, lm1;
+  // prefill-only per-row sampling arrays (length 1)
+  float *d_pf_temp = nullptr, *d_pf_top_p = nullptr;
+  uint64_t *d_pf_seed = nullptr;
+  int *d_pf_step = nullptr, *d_pf_one = nullptr, *d_pf_tok = nullptr;
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t graph_exec = nullptr;
+  bool eager = false;
+  int decode_launches = 0;
+  std::vector<void *> allocs;
+};
+
+namespace {
+
+template <typename T>
+int dmalloc(std::vector<void *> &keep, T **p, size_t n, bool zero = true) {
+  void *q = nullptr;
+  if (n == 0) n = 1;
+  cudaError_t e = cudaMalloc(&q, n * sizeof(T));
+  if (e != cudaSuccess) {
+    g_last_cuda_error = (int)e;
+    return CORUN_ENOMEM;
+  }
+  keep.push_back(q);
+  if (zero && cudaMemset(q, 0, n * sizeof(T)) != cudaSuccess) return CORUN_ECUDA;
+  *p = (T *)q;
+  return CORUN_OK;
+}
+
+int pad16(int x) { return (x + 15) / 16 * 16; }
+
+int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm) {
+  const corun_shape &s = e->sh;
+  const int H = s.hidden, QD = s.n_q_heads * s.head_dim, KD = s.n_kv_heads * s.head_dim, F = s.ffn, V = s.vocab;
+  P.R = R;
+  P.BN = pad16(R);
+  P.has_layers = layers;
+  P.has_lm = lm;
+  auto &A = P.allocs;
+  RC(dmalloc(A, &P.xn_hi, (size_t)P.BN * H));
+  RC(dmalloc(A, &P.xn_lo, (size_t)P.BN * H));
+  RC(dmalloc(A, &P.ws, gemm_ws_floats(e->num_sms, P.BN)));
+  RC(dmalloc(A, &P.row_token, R));
+  RC(dmalloc(A, &P.row_pos, R));
+  RC(dmalloc(A, &P.row_active, R));
+  RC(dmalloc(A, &P.row_slot, R));
+  RC(dmalloc(A, &P.do_sample, R));
+  RC(dmalloc(A, &P.sampled, R));
+  if (layers) {
+    RC(dmalloc(A, &P.h, (size_t)R * H));
+    RC(dmalloc(A, &P.q, (size_t)R * QD));
+    RC(dmalloc(A, &P.part_acc, (size_t)R * s.n_q_heads * e->max_splits * s.head_dim));
+    RC(dmalloc(A, &P.part_ml, (size_t)R * s.n_q_heads * e->max_splits * 2));
+    RC(dmalloc(A, &P.qkv_out, (size_t)R * (QD + 2 * KD)));
+    RC(dmalloc(A, &P.o_out, (size_t)R * H));
+    RC(dmalloc(A, &P.gu_out, (size_t)R * 2 * F));
+    RC(dmalloc(A, &P.down_out, (size_t)R * H));
+    RC(dmalloc(A, &P.ao_hi, (size_t)P.BN * QD));
+    RC(dmalloc(A, &P.ao_lo, (size_t)P.BN * QD));
+    RC(dmalloc(A, &P.ff_hi, (size_t)P.BN * F));
+    RC(dmalloc(A, &P.ff_lo, (size_t)P.BN * F));
+    // the plans carry layer 0's weights; the per-layer tensor maps override them at launch
+    RC(gemm_plan_create(&P.p_qkv, e->w0_qkv, QD + 2 * KD, H, P.xn_hi, P.xn_lo, R, P.BN, P.qkv_out, P.ws, e->num_sms));
+    RC(gemm_plan_create(&P.p_o, e->w0_o, H, QD, P.ao_hi, P.ao_lo, R, P.BN, P.o_out, P.ws, e->num_sms));
+    RC(gemm_plan_create(&P.p_gu, e->w0_gu, 2 * F, H, P.xn_hi, P.xn_lo, R, P.BN, P.gu_out, P.ws, e->num_sms));
+    RC(gemm_plan_create(&P.p_down, e->w0_down, H, F, P.ff_hi, P.ff_lo, R, P.BN, P.down_out, P.ws, e->num_sms));
+  }
+  if (lm) {
+    RC(dmalloc(A, &P.logits, (size_t)R * V));
+    RC(gemm_plan_create(&P.p_lm, e->lm_head, V, H, P.xn_hi, P.xn_lo, R, P.BN, P.logits, P.ws, e->num_sms));
+  }
+  return CORUN_OK;
+}
+
+void program_destroy(Program &P) {
+  gemm_plan_destroy(&P.p_qkv);
+  gemm_plan_destroy(&P.p_o);
+  gemm_plan_destroy(&P.p_gu);
+  gemm_plan_destroy(&P.p_down);
+  gemm_plan_destroy(&P.p_lm);
+  for (void *p : P.allocs) cudaFree(p);
+  P.allocs.clear();
+}
+
+KvLayout kv_layout(const corun_engine *e) {
+  return KvLayout{e->kv_pool, e->d_block_table, e->max_blocks, e->sh.n_kv_heads, e->sh.head_dim, e->layer_stride};
+}
+
+// Enqueues embed -> all layers (ends with the last down GEMM).  Counts launches.
+int run_layers(corun_engine *e, Program &P, int *launches) {
+  const corun_shape &s = e->sh;
+  const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
+  const KvLayout kv = kv_layout(e);
+  int n = 0;
+  for (int l = 0; l < s.n_layers; ++l) {
+    GemmOut prev = P.p_down.out();
+    CK(launch_resid_norm(P.h, s.hidden, e->embed, rows, l == 0 ? nullptr : &prev, e->attn_norm[l], s.rms_eps, P.xn_hi,
+                         P.xn_lo, e->st));
+    CK(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st));
+    CK(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st));
+    CK(launch_attention(P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo, e->st));
+    CK(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st));
+    GemmOut o = P.p_o.out();
+    CK(launch_resid_norm(P.h, s.hidden, nullptr, rows, &o, e->mlp_norm[l], s.rms_eps, P.xn_hi, P.xn_lo, e->st));
+    CK(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st));
+    CK(launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st));
+    CK(gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st));
+    n += 10;
+  }
+  if (launches) *launches += n;
+  return CORUN_OK;
+}
+
+// One decode iteration on the stream (what the graph captures).
+int enqueue_decode_body(corun_engine *e, int *launches) {
+  Program &P = e->dec;
+  const corun_shape &s = e->sh;
+  int n = 0;
+  CK(cudaMemcpyAsync(e->d_active, e->h_active, e->B, cudaMemcpyHostToDevice, e->st));
+  CK(cudaMemcpyAsync(e->d_seeds, e->h_seeds, e->B * sizeof(uint64_t), cudaMemcpyHostToDevice, e->st));
+  CK(launch_prepare_rows(e->d_active, e->d_in_use, e->d_ctx, e->d_pending, e->B, P.row_token, P.row_pos, P.row_active,
+                         P.row_slot, P.do_sample, e->st));
+  n += 1;
+  RC(run_layers(e, P, &n));
+  const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
+  GemmOut prev = P.p_down.out();
+  CK(launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->final_norm, s.rms_eps, P.xn_hi, P.xn_lo, e->st));
+  CK(gemm_launch(P.p_lm, nullptr, e->d_status, e->st));
+  CK(gemm_fixup_launch(P.p_lm, e->st));
+  SampleArgs sa{P.logits, s.vocab, P.do_sample, e->d_temp, e->d_top_p, e->d_seeds, e->d_step, nullptr, P.sampled};
+  CK(launch_sampler(sa, P.R, e->st));
+  CK(launch_advance(P.row_active, P.sampled, e->B, e->d_ctx, e->d_step, e->d_pending, e->d_out_tokens, e->st));
+  n += 4 + (P.p_lm.n_split_tiles ? 1 : 0);
+  CK(cudaMemcpyAsync(e->h_out_tokens, e->d_out_tokens, e->B * sizeof(int), cudaMemcpyDeviceToHost, e->st));
+  CK(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, e->st));
+  if (launches) *launches = n;
+  return CORUN_OK;
+}
+
+int check_status(corun_engine *e) {
+  if (*e->h_status != 0) return CORUN_ETIMEOUT;
+  return CORUN_OK;
+}
+
+int sync_stream(corun_engine *e) {
+  CK(cudaStreamSynchronize(e->st));
+  e->in_flight = false;
+  return CORUN_OK;
+}
+
+int reserve_blocks(corun_engine *e, int slot, int reserve_len) {
+  const int need = (reserve_len + KV_BLOCK - 1) / KV_BLOCK;
+  if ((size_t)need > e->free_blocks.size()) return CORUN_ENOSPACE;
+  std::vector<int> &mine = e->slot_blocks[slot];
+  mine.clear();
+  std::vector<int> row(e->max_blocks, 0);
+  for (int i = 0; i < need; ++i) {
+    mine.push_back(e->free_blocks.back());
+    e->free_blocks.pop_back();
+    row[i] = mine.back();
+  }
+  CK(cudaMemcpyAsync(e->d_block_table + (size_t)slot * e->max_blocks, row.data(), e->max_blocks * sizeof(int),
+                     cudaMemcpyHostToDevice, e->st));
+  CK(cudaStreamSynchronize(e->st));   // `row` is pageable and local
+  return CORUN_OK;
+}
+
+int set_slot_state(corun_engine *e, int slot, int in_use, int ctx, int step, int pending, float temp, float top_p) {
+  CK(cudaMemcpyAsync(e->d_in_use + slot, &in_use, sizeof(int), cudaMemcpyHostToDevice, e->st));
+  CK(cudaMemcpyAsync(e->d_ctx + slot, &ctx, sizeof(int), cudaMemcpyHostToDevice, e->st));
+  CK(cudaMemcpyAsync(e->d_step + slot, &step, sizeof(int), cudaMemcpyHostToDevice, e->st));
+  CK(cudaMemcpyAsync(e->d_pending + slot, &pending, sizeof(int), cudaMemcpyHostToDevice, e->st));
+  CK(cudaMemcpyAsync(e->d_temp + slot, &temp, sizeof(float), cudaMemcpyHostToDevice, e->st));
+  CK(cudaMemcpyAsync(e->d_top_p + slot, &top_p, sizeof(float), cudaMemcpyHostToDevice, e->st));
+  CK(cudaStreamSynchronize(e->st));
+  return CORUN_OK;
+}
+
+bool slot_ok(const corun_engine *e, int slot) { return slot >= 0 && slot < e->B; }
+
+}  // namespace
+
+extern "C" {
+
+int corun_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char *corun_strerror(int st) {
+  switch (st) {
+    case CORUN_OK: return "ok";
+    case CORUN_EINVAL: return "invalid argument";
+    case CORUN_ESLOT: return "bad slot (out of range, busy, or empty)";
+    case CORUN_ENOSPACE: return "KV pool cannot hold the reserved sequence";
+    case CORUN_ECTX: return "an active slot is at its reserved length";
+    case CORUN_ECUDA: return "CUDA error";
+    case CORUN_ETIMEOUT: return "a bounded device-side wait expired";
+    case CORUN_ENOMEM: return "out of memory";
+    default: return "unknown status";
+  }
+}
+
+int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int32_t max_context, int32_t kv_block,
+               int64_t kv_pool_blocks, void *cuda_stream, corun_engine **out) {
+  if (!shape || !w || !out) return CORUN_EINVAL;
+  *out = nullptr;
+  const corun_shape &s = *shape;
+  if (s.arch != 0 || s.n_layers < 1 || s.hidden < 64 || s.hidden % 64 || s.ffn < 64 || s.ffn % 64 || s.vocab < 1)
+    return CORUN_EINVAL;
+  if (s.head_dim != 64 && s.head_dim != 128) return CORUN_EINVAL;
+  if (s.n_q_heads < 1 || s.n_kv_heads < 1 || s.n_q_heads % s.n_kv_heads) return CORUN_EINVAL;
+  const int group = s.n_q_heads / s.n_kv_heads;
+  if (group != 1 && group != 2 && group != 4 && group != 8) return CORUN_EINVAL;
+  if ((s.n_q_heads * s.head_dim) % 64) return CORUN_EINVAL;
+  if (!(s.rms_eps >= 0.f) || !(s.rope_theta > 0.f)) return CORUN_EINVAL;
+  if (B < 1 || B > 256 || max_context < 1 || kv_block != KV_BLOCK || kv_pool_blocks < 0) return CORUN_EINVAL;
+  if (!w->embed || !w->lm_head || !w->final_norm || !w->attn_norm || !w->wqkv || !w->wo || !w->mlp_norm ||
+      !w->wgate_up || !w->wdown)
+    return CORUN_EINVAL;
+  for (int l = 0; l < s.n_layers; ++l)
+    if (!w->attn_norm[l] || !w->wqkv[l] || !w->wo[l] || !w->mlp_norm[l] || !w->wgate_up[l] || !w->wdown[l])
+      return CORUN_EINVAL;
+
+  int dev = 0;
+  CK(cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  CK(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) return CORUN_ECUDA;   // tcgen05 / TMEM kernels: sm_100a only
+
+  corun_engine *e = new (std::nothrow) corun_engine();
+  if (!e) return CORUN_ENOMEM;
+  auto fail = [&](int rc) {
+    corun_destroy(e);
+    return rc;
+  };
+  e->sh = s;
+  e->B = B;
+  e->max_ctx = max_context;
+  e->max_blocks = (max_context + KV_BLOCK - 1) / KV_BLOCK;
+  e->max_splits = (max_context + ATT_SPLIT - 1) / ATT_SPLIT;
+  e->num_sms = prop.multiProcessorCount;
+  e->st = (cudaStream_t)cuda_stream;
+  if (!e->st) {   // the legacy default stream cannot be captured: use a private one
+    if (cudaStreamCreateWithFlags(&e->st, cudaStreamNonBlocking) != cudaSuccess) return fail(CORUN_ECUDA);
+    e->own_stream = true;
+  }
+  e->w0_qkv = w->wqkv[0];
+  e->w0_o = w->wo[0];
+  e->w0_gu = w->wgate_up[0];
+  e->w0_down = w->wdown[0];
+  e->pool_blocks = kv_pool_blocks ? kv_pool_blocks : (int64_t)B * e->max_blocks;
+  e->chunk = 256;
+  if (const char *c = getenv("CORUN_PREFILL_CHUNK")) {
+    const int v = atoi(c);
+    if (v >= 16 && v <= 256 && v % 16 == 0) e->chunk = v;
+  }
+  e->embed = (const bf16 *)w->embed;
+  e->lm_head = (const bf16 *)w->lm_head;
+  e->final_norm = (const bf16 *)w->final_norm;
+  const int H = s.hidden, QD = s.n_q_heads * s.head_dim, KD = s.n_kv_heads * s.head_dim, F = s.ffn;
+  e->tm_qkv.resize(s.n_layers);
+  e->tm_o.resize(s.n_layers);
+  e->tm_gu.resize(s.n_layers);
+  e->tm_down.resize(s.n_layers);
+  for (int l = 0; l < s.n_layers; ++l) {
+    e->attn_norm.push_back((const bf16 *)w->attn_norm[l]);
+    e->mlp_norm.push_back((const bf16 *)w->mlp_norm[l]);
+    int rc;
+    if ((rc = gemm_encode_map(&e->tm_qkv[l], w->wqkv[l], QD + 2 * KD, H, GEMM_TILE_M))) return fail(rc);
+    if ((rc = gemm_encode_map(&e->tm_o[l], w->wo[l], H, QD, GEMM_TILE_M))) return fail(rc);
+    if ((rc = gemm_encode_map(&e->tm_gu[l], w->wgate_up[l], 2 * F, H, GEMM_TILE_M))) return fail(rc);
+    if ((rc = gemm_encode_map(&e->tm_down[l], w->wdown[l], H, F, GEMM_TILE_M))) return fail(rc);
+  }
+
+  auto &A = e->allocs;
+  int rc;
+  e->layer_stride = (size_t)e->pool_blocks * 2 * s.n_kv_heads * KV_BLOCK * s.head_dim;
+  if ((rc = dmalloc(A, &e->kv_pool, e->layer_stride * s.n_layers, false))) return fail(rc);
+  if ((rc = dmalloc(A, &e->d_block_table, (size_t)B * e->max_blocks))) return fail(rc);
+  if ((rc = dmalloc(A, &e->d_in_use, B)) || (rc = dmalloc(A, &e->d_ctx, B)) || (rc = dmalloc(A, &e->d_step, B)) ||
+      (rc = dmalloc(A, &e->d_pending, B)) || (rc = dmalloc(A, &e->d_temp, B)) || (rc = dmalloc(A, &e->d_top_p, B)) ||
+      (rc = dmalloc(A, &e->d_seeds, B)) || (rc = dmalloc(A, &e->d_active, B)) || (rc = dmalloc(A, &e->d_out_tokens, B)) ||
+      (rc = dmalloc(A, &e->d_status, 1)) || (rc = dmalloc(A, &e->d_pf_temp, 1)) || (rc = dmalloc(A, &e->d_pf_top_p, 1)) ||
+      (rc = dmalloc(A, &e->d_pf_seed, 1)) || (rc = dmalloc(A, &e->d_pf_step, 1)) || (rc = dmalloc(A, &e->d_pf_one, 1)) ||
+      (rc = dmalloc(A, &e->d_pf_tok, 1)))
+    return fail(rc);
+  {
+    // cos/sin of pos * theta^(-2i/hd), evaluated in fp64 on the host
+    const int half = s.head_dim / 2;
+    std::vector<float2> tab((size_t)max_context * half);
+    for (int p = 0; p < max_context; ++p)
+      for (int i = 0; i < half; ++i) {
+        const double ang = (double)p * std::pow((double)s.rope_theta, -2.0 * (double)i / (double)s.head_dim);
+        tab[(size_t)p * half + i] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+      }
+    if ((rc = dmalloc(A, &e->d_rope, tab.size(), false))) return fail(rc);
+    if (cudaMemcpy(e->d_rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice) != cudaSuccess)
+      return fail(CORUN_ECUDA);
+    const int one = 1;
+    if (cudaMemcpy(e->d_pf_one, &one, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return fail(CORUN_ECUDA);
+  }
+  e->free_blocks.resize((size_t)e->pool_blocks);
+  for (int64_t i = 0; i < e->pool_blocks; ++i) e->free_blocks[(size_t)i] = (int)(e->pool_blocks - 1 - i);
+  e->slot_blocks.resize(B);
+  e->in_use.assign(B, 0);
+  e->ctx.assign(B, 0);
+  e->reserve.assign(B, 0);
+  e->step.assign(B, 0);
+  if (cudaMallocHost(&e->h_active, B) != cudaSuccess || cudaMallocHost(&e->h_seeds, B * sizeof(uint64_t)) != cudaSuccess ||
+      cudaMallocHost(&e->h_out_tokens, B * sizeof(int)) != cudaSuccess ||
+      cudaMallocHost(&e->h_status, sizeof(int)) != cudaSuccess ||
+      cudaMallocHost(&e->h_rows, (size_t)5 * e->chunk * sizeof(int)) != cudaSuccess)
+    return fail(CORUN_ENOMEM);
+  memset(e->h_active, 0, B);
+  memset(e->h_seeds, 0, B * sizeof(uint64_t));
+  *e->h_status = 0;
+
+  if ((rc = program_create(e, e->dec, B, true, true))) return fail(rc);
+  if ((rc = program_create(e, e->pre, e->chunk, true, false))) return fail(rc);
+  if ((rc = program_create(e, e->lm1, 1, false, true))) return fail(rc);
+
+  // eager warm-up on an all-padding batch (also validates every launch), then capture
+  if ((rc = enqueue_decode_body(e, &e->decode_launches))) return fail(rc);
+  if (cudaStreamSynchronize(e->st) != cudaSuccess) return fail(CORUN_ECUDA);
+  if ((rc = check_status(e))) return fail(rc);
+  if (cudaStreamBeginCapture(e->st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return fail(CORUN_ECUDA);
+  rc = enqueue_decode_body(e, nullptr);
+  cudaError_t ce = cudaStreamEndCapture(e->st, &e->graph);
+  if (rc) return fail(rc);
+  if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return fail(CORUN_ECUDA); }
+  ce = cudaGraphInstantiate(&e->graph_exec, e->graph, 0);
+  if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return fail(CORUN_ECUDA); }
+  *out = e;
+  return CORUN_OK;
+}
+
+void corun_destroy(corun_engine *e) {
+  if (!e) return;
+  cudaStreamSynchronize(e->st);
+  if (e->graph_exec) cudaGraphExecDestroy(e->graph_exec);
+  if (e->graph) cudaGraphDestroy(e->graph);
+  program_destroy(e->dec);
+  program_destroy(e->pre);
+  program_destroy(e->lm1);
+  for (void *p : e->allocs) cudaFree(p);
+  if (e->h_active) cudaFreeHost(e->h_active);
+  if (e->h_seeds) cudaFreeHost(e->h_seeds);
+  if (e->h_out_tokens) cudaFreeHost(e->h_out_tokens);
+  if (e->h_status) cudaFreeHost(e->h_status);
+  if (e->h_rows) cudaFreeHost(e->h_rows);
+  if (e->own_stream) cudaStreamDestroy(e->st);
+  delete e;
+}
+
+int corun_prefill(corun_engine *e, int32_t slot, const int32_t *tokens, int32_t n, int32_t reserve_len,
+                  const corun_sampling *sampling, uint64_t seed, int32_t *out_first_token) {
+  if (!e || !tokens || !sampling || n < 1 || reserve_len < n || reserve_len > e->max_ctx) return CORUN_EINVAL;
+  if (!slot_ok(e, slot) || e->in_use[slot]) return CORUN_ESLOT;
+  for (int i = 0; i < n; ++i)
+    if (tokens[i] < 0 || tokens[i] >= e->sh.vocab) return CORUN_EINVAL;
+  RC(sync_stream(e));
+  RC(reserve_blocks(e, slot, reserve_len));
+  Program &P = e->pre;
+  const corun_shape &s = e->sh;
+  const int CH = e->chunk;
+  int last_row = 0;
+  for (int pos0 = 0; pos0 < n; pos0 += CH) {
+    const int rows_here = (n - pos0 < CH) ? n - pos0 : CH;
+    int *tok = e->h_rows, *pos = tok + CH, *act = pos + CH, *slt = act + CH;
+    for (int i = 0; i < CH; ++i) {
+      const bool on = i < rows_here;
+      tok[i] = on ? tokens[pos0 + i] : 0;
+      pos[i] = on ? pos0 + i : 0;
+      act[i] = on ? 1 : 0;
+      slt[i] = slot;
+    }
+    CK(cudaMemcpyAsync(P.row_token, tok, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
+    CK(cudaMemcpyAsync(P.row_pos, pos, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
+    CK(cudaMemcpyAsync(P.row_active, act, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
+    CK(cudaMemcpyAsync(P.row_slot, slt, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
+    RC(run_layers(e, P, nullptr));
+    CK(cudaStreamSynchronize(e->st));   // the staging arrays are reused by the next chunk
+    last_row = rows_here - 1;
+  }
+  // last position only: final norm -> LM head (one row) -> sample with R(seed, 0)
+  {
+    Program &L = e->lm1;
+    GemmOut prev = P.p_down.out();
+    prev.direct += (size_t)last_row * prev.N;
+    prev.ws += (size_t)last_row * 128;
+    const Rows one{P.row_token + last_row, P.row_pos + last_row, P.row_active + last_row, P.row_slot + last_row, 1};
+    CK(launch_resid_norm(P.h + (size_t)last_row * s.hidden, s.hidden, nullptr, one, &prev, e->final_norm, s.rms_eps,
+                         L.xn_hi, L.xn_lo, e->st));
+    CK(gemm_launch(L.p_lm, nullptr, e->d_status, e->st));
+    CK(gemm_fixup_launch(L.p_lm, e->st));
+    const int zero = 0;
+    CK(cudaMemcpyAsync(e->d_pf_temp, &sampling->temperature, sizeof(float), cudaMemcpyHostToDevice, e->st));
+    CK(cudaMemcpyAsync(e->d_pf_top_p, &sampling->top_p, sizeof(float), cudaMemcpyHostToDevice, e->st));
+    CK(cudaMemcpyAsync(e->d_pf_seed, &seed, sizeof(uint64_t), cudaMemcpyHostToDevice, e->st));
+    CK(cudaMemcpyAsync(e->d_pf_step, &zero, sizeof(int), cudaMemcpyHostToDevice, e->st));
+    SampleArgs sa{L.logits, s.vocab, e->d_pf_one, e->d_pf_temp, e->d_pf_top_p, e->d_pf_seed, e->d_pf_step, nullptr,
+                  e->d_pf_tok};
+    CK(launch_sampler(sa, 1, e->st));
+    CK(cudaMemcpyAsync(e->dec.logits + (size_t)slot * s.vocab, L.logits, (size_t)s.vocab * sizeof(float),
+                       cudaMemcpyDeviceToDevice, e->st));
+    CK(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, e->st));
+    CK(cudaStreamSynchronize(e->st));
+  }
+  int first = -1;
+  CK(cudaMemcpy(&first, e->d_pf_tok, sizeof(int), cudaMemcpyDeviceToHost));
+  RC(check_status(e));
+  RC(set_slot_state(e, slot, 1, n, 1, first, sampling->temperature, sampling->top_p));
+  e->in_use[slot] = 1;
+  e->ctx[slot] = n;
+  e->reserve[slot] = reserve_len;
+  e->step[slot] = 1;
+  if (out_first_token) *out_first_token = first;
+  return CORUN_OK;
+}
+
+int corun_decode_enqueue(corun_engine *e, const uint8_t *active, const uint64_t *seeds) {
+  if (!e || !active || !seeds) return CORUN_EINVAL;
+  for (int s = 0; s < e->B; ++s) {
+    if (!active[s]) continue;
+    if (!e->in_use[s]) return CORUN_ESLOT;
+    if (e->ctx[s] + 1 > e->reserve[s]) return CORUN_ECTX;
+  }
+  bool same = e->staged_valid;
+  for (int s = 0; s < e->B && same; ++s) {
+    const uint8_t a = active[s] ? 1 : 0;
+    if (e->h_active[s] != a || (a && e->h_seeds[s] != seeds[s])) same = false;
+  }
+  if (!same) {
+    if (e->in_flight) RC(sync_stream(e));   // an earlier replay may still read the staging buffers
+    for (int s = 0; s < e->B; ++s) {
+      e->h_active[s] = active[s] ? 1 : 0;
+      e->h_seeds[s] = active[s] ? seeds[s] : 0;
+    }
+    e->staged_valid = true;
+  }
+  if (e->eager) {
+    RC(enqueue_decode_body(e, nullptr));
+  } else {
+    CK(cudaGraphLaunch(e->graph_exec, e->st));
+  }
+  e->in_flight = true;
+  for (int s = 0; s < e->B; ++s)
+    if (active[s]) {
+      e->ctx[s] += 1;
+      e->step[s] += 1;
+    }
+  return CORUN_OK;
+}
+
+int corun_decode_wait(corun_engine *e, int32_t *out_tokens) {
+  if (!e) return CORUN_EINVAL;
+  RC(sync_stream(e));
+  if (out_tokens) memcpy(out_tokens, e->h_out_tokens, e->B * sizeof(int));
+  return check_status(e);
+}
+
+int corun_decode_step(corun_engine *e, const uint8_t *active, const uint64_t *seeds, int32_t *out_tokens) {
+  if (!out_tokens) return CORUN_EINVAL;
+  RC(corun_decode_enqueue(e, active, seeds));
+  return corun_decode_wait(e, out_tokens);
+}
+
+int corun_release(corun_engine *e, int32_t slot) {
+  if (!e) return CORUN_EINVAL;
+  if (!slot_ok(e, slot) || !e->in_use[slot]) return CORUN_ESLOT;
+  RC(sync_stream(e));
+  for (int b : e->slot_blocks[slot]) e->free_blocks.push_back(b);
+  e->slot_blocks[slot].clear();
+  RC(set_slot_state(e, slot, 0, 0, 0, 0, 0.f, 1.f));
+  e->in_use[slot] = 0;
+  e->ctx[slot] = 0;
+  e->reserve[slot] = 0;
+  e->step[slot] = 0;
+  return CORUN_OK;
+}
+
+int corun_get_logits(corun_engine *e, int32_t slot, float *out) {
+  if (!e || !out) return CORUN_EINVAL;
+  if (!slot_ok(e, slot) || !e->in_use[slot]) return CORUN_ESLOT;
+  RC(sync_stream(e));
+  CK(cudaMemcpy(out, e->dec.logits + (size_t)slot * e->sh.vocab, (size_t)e->sh.vocab * sizeof(float),
+                cudaMemcpyDeviceToHost));
+  return CORUN_OK;
+}
+
+int corun_force_token(corun_engine *e, int32_t slot, int32_t token) {
+  if (!e || token < 0 || token >= e->sh.vocab) return CORUN_EINVAL;
+  if (!slot_ok(e, slot) || !e->in_use[slot]) return CORUN_ESLOT;
+  RC(sync_stream(e));
+  CK(cudaMemcpy(e->d_pending + slot, &token, sizeof(int), cudaMemcpyHostToDevice));
+  return CORUN_OK;
+}
+
+int corun_context_len(corun_engine *e, int32_t slot) {
+  if (!e) return CORUN_EINVAL;
+  if (!slot_ok(e, slot) || !e->in_use[slot]) return CORUN_ESLOT;
+  return e->ctx[slot];
+}
+
+int64_t corun_free_blocks(corun_engine *e) { return e ? (int64_t)e->free_blocks.size() : (int64_t)CORUN_EINVAL; }
+
+static int kv_io(corun_engine *e, int slot, int layer, int pos0, int n, float *k, float *v, int write) {
+  if (!e || !k || !v || n < 0 || pos0 < 0 || layer < 0 || layer >= e->sh.n_layers) return CORUN_EINVAL;
+  if (!slot_ok(e, slot) || !e->in_use[slot]) return CORUN_ESLOT;
+  const int limit = write ? e->reserve[slot] : e->ctx[slot];
+  if (pos0 + n > limit) return CORUN_EINVAL;
+  if (n == 0) return CORUN_OK;
+  RC(sync_stream(e));
+  const size_t elems = (size_t)n * e->sh.n_kv_heads * e->sh.head_dim;
+  float *dk = nullptr, *dv = nullptr;
+  if (cudaMalloc(&dk, elems * sizeof(float)) != cudaSuccess) return CORUN_ENOMEM;
+  if (cudaMalloc(&dv, elems * sizeof(float)) != cudaSuccess) { cudaFree(dk); return CORUN_ENOMEM; }
+  int rc = CORUN_OK;
+  cudaError_t ce = cudaSuccess;
+  if (write) {
+    ce = cudaMemcpy(dk, k, elems * sizeof(float), cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess) ce = cudaMemcpy(dv, v, elems * sizeof(float), cudaMemcpyHostToDevice);
+  }
+  if (ce == cudaSuccess) ce = launch_kv_copy(kv_layout(e), layer, slot, pos0, n, dk, dv, write, e->st);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(e->st);
+  if (ce == cudaSuccess && !write) {
+    ce = cudaMemcpy(k, dk, elems * sizeof(float), cudaMemcpyDeviceToHost);
+    if (ce == cudaSuccess) ce = cudaMemcpy(v, dv, elems * sizeof(float), cudaMemcpyDeviceToHost);
+  }
+  if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; rc = CORUN_ECUDA; }
+  cudaFree(dk);
+  cudaFree(dv);
+  if (rc == CORUN_OK && write && pos0 + n > e->ctx[slot]) {
+    e->ctx[slot] = pos0 + n;
+    const int c = e->ctx[slot];
+    CK(cudaMemcpy(e->d_ctx + slot, &c, sizeof(int), cudaMemcpyHostToDevice));
+  }
+  return rc;
+}
+
+int corun_debug_kv_read(corun_engine *e, int32_t slot, int32_t layer, int32_t pos0, int32_t n, float *k, float *v) {
+  return kv_io(e, slot, layer, pos0, n, k, v, 0);
+}
+int corun_debug_kv_write(corun_engine *e, int32_t slot, int32_t layer, int32_t pos0, int32_t n, const float *k,
+                         const float *v) {
+  return kv_io(e, slot, layer, pos0, n, const_cast<float *>(k), const_cast<float *>(v), 1);
+}
+
+int corun_debug_adopt(corun_engine *e, int32_t slot, int32_t n_ctx, int32_t reserve_len, int32_t pending_token,
+                      const corun_sampling *sampling, int32_t step) {
+  if (!e || !sampling || n_ctx < 0 || reserve_len < n_ctx || reserve_len < 1 || reserve_len > e->max_ctx ||
+      pending_token < 0 || pending_token >= e->sh.vocab || step < 0)
+    return CORUN_EINVAL;
+  if (!slot_ok(e, slot) || e->in_use[slot]) return CORUN_ESLOT;
+  RC(sync_stream(e));
+  RC(reserve_blocks(e, slot, reserve_len));
+  RC(set_slot_state(e, slot, 1, n_ctx, step, pending_token, sampling->temperature, sampling->top_p));
+  e->in_use[slot] = 1;
+  e->ctx[slot] = n_ctx;
+  e->reserve[slot] = reserve_len;
+  e->step[slot] = step;
+  return CORUN_OK;
+}
+
+int corun_debug_set_eager(corun_engine *e, int32_t eager) {
+  if (!e) return CORUN_EINVAL;
+  RC(sync_stream(e));
+  e->eager = eager != 0;
+  return CORUN_OK;
+}
+
+int corun_decode_launches(corun_engine *e) { return e ? e->decode_launches : CORUN_EINVAL; }
+
+int corun_debug_gemm(const void *W, int32_t N, int32_t K, const float *X, int32_t R, float *out, void *cuda_stream) {
+  if (!W || !X || !out || N < 1 || K < 64 || K % 64 || R < 1 || R > 256) return CORUN_EINVAL;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int dev = 0, sms = 0;
+  CK(cudaGetDevice(&dev));
+  CK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const int BN = pad16(R);
+  std::vector<void *> keep;
+  bf16 *hi = nullptr, *lo = nullptr;
+  float *ws = nullptr;
+  int *status = nullptr;
+  int rc = CORUN_OK;
+  GemmPlan p;
+  if ((rc = dmalloc(keep, &hi, (size_t)BN * K)) == 0 && (rc = dmalloc(keep, &lo, (size_t)BN * K)) == 0 &&
+      (rc = dmalloc(keep, &ws, gemm_ws_floats(sms, BN))) == 0 && (rc = dmalloc(keep, &status, 1)) == 0 &&
+      (rc = gemm_plan_create(&p, W, N, K, hi, lo, R, BN, out, ws, sms)) == 0) {
+    cudaError_t ce = launch_split(X, R, K, hi, lo, st);
+    if (ce == cudaSuccess) ce = gemm_launch(p, nullptr, status, st);
+    if (ce == cudaSuccess) ce = gemm_fixup_launch(p, st);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+    int hs = 0;
+    if (ce == cudaSuccess) ce = cudaMemcpy(&hs, status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; rc = CORUN_ECUDA; }
+    else if (hs != 0) rc = CORUN_ETIMEOUT;
+  }
+  gemm_plan_destroy(&p);
+  for (void *q : keep) cudaFree(q);
+  return rc;
+}
+
+int corun_debug_variate(uint64_t seed, uint64_t t, uint32_t *out_u24) {
+  if (!out_u24) return CORUN_EINVAL;
+  uint32_t *d = nullptr;
+  if (cudaMalloc(&d, sizeof(uint32_t)) != cudaSuccess) return CORUN_ENOMEM;
+  cudaError_t ce = launch_variate(seed, t, d, nullptr);
+  if (ce == cudaSuccess) ce = cudaMemcpy(out_u24, d, sizeof(uint32_t), cudaMemcpyDeviceToHost);
+  cudaFree(d);
+  if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
+  return CORUN_OK;
+}
+
+int corun_debug_sample(const float *logits, int32_t n_rows, int32_t vocab, const corun_sampling *sampling,
+                       const uint32_t *u24, int32_t *out_tokens) {
+  if (!logits || !sampling || !u24 || !out_tokens || n_rows < 1 || vocab < 1) return CORUN_EINVAL;
+  std::vector<void *> keep;
+  float *dl = nullptr, *dt = nullptr, *dp = nullptr;
+  int *dflag = nullptr, *dstep = nullptr, *dtok = nullptr;
+  uint32_t *du = nullptr;
+  uint64_t *dseed = nullptr;
+  int rc;
+  if ((rc = dmalloc(keep, &dl, (size_t)n_rows * vocab, false)) == 0 && (rc = dmalloc(keep, &dt, n_rows)) == 0 &&
+      (rc = dmalloc(keep, &dp, n_rows)) == 0 && (rc = dmalloc(keep, &dflag, n_rows)) == 0 &&
+      (rc = dmalloc(keep, &dstep, n_rows)) == 0 && (rc = dmalloc(keep, &dtok, n_rows)) == 0 &&
+      (rc = dmalloc(keep, &du, n_rows)) == 0 && (rc = dmalloc(keep, &dseed, n_rows)) == 0) {
+    std::vector<float> t(n_rows, sampling->temperature), p(n_rows, sampling->top_p);
+    std::vector<int> ones(n_rows, 1);
+    cudaError_t ce = cudaMemcpy(dl, logits, (size_t)n_rows * vocab * sizeof(float), cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess) ce = cudaMemcpy(dt, t.data(), n_rows * sizeof(float), cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess) ce = cudaMemcpy(dp, p.data(), n_rows * sizeof(float), cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess) ce = cudaMemcpy(dflag, ones.data(), n_rows * sizeof(int), cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess) ce = cudaMemcpy(du, u24, n_rows * sizeof(uint32_t), cudaMemcpyHostToDevice);
+    SampleArgs sa{dl, vocab, dflag, dt, dp, dseed, dstep, du, dtok};
+    if (ce == cudaSuccess) ce = launch_sampler(sa, n_rows, nullptr);
+    if (ce == cudaSuccess) ce = cudaMemcpy(out_tokens, dtok, n_rows * sizeof(int), cudaMemcpyDeviceToHost);
+    if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; rc = CORUN_ECUDA; }
+  }
+  for (void *q : keep) cudaFree(q);
+  return rc;
+}
+
+}  // extern "C"

@@ -1,0 +1,281 @@
+// tcgen05 / TMEM / TMA GEMM for sm_100a with a static, shape-keyed work partition.
+#include "gemm.cuh"
+
+#include <cudaTypedefs.h>
+
+#include <vector>
+
+#include "../../include/corun.h"
+#include "ptx.cuh"
+
+namespace corun {
+
+namespace {
+
+constexpr int MAX_STAGES = 8;
+
+// Role loops walk the CTA's flat k-block range [k0, k1) segment by segment; a
+// segment is the part of the range that falls into one weight tile.
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmHi,
+                    const __grid_constant__ CUtensorMap tmLo, float *__restrict__ direct, float *__restrict__ ws,
+                    const int *__restrict__ cta_start, int N, int KB, int BN, int R, int stages, int tmem_cols,
+                    uint32_t idesc, int *status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
+  __shared__ __align__(8) uint64_t tmem_full_bar;
+  __shared__ __align__(8) uint64_t tmem_empty_bar;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int cta = blockIdx.x;
+  const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t w_bytes = GEMM_TILE_M * GEMM_BLOCK_K * 2;          // 16 KiB
+  const uint32_t x_bytes = (uint32_t)BN * GEMM_BLOCK_K * 2;         // BN * 128 B
+  const uint32_t stage_bytes = w_bytes + 2 * x_bytes;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    mbar_init(smem_u32(&tmem_full_bar), 1);
+    mbar_init(smem_u32(&tmem_empty_bar), 128);
+    fence_mbar_init();
+    fence_proxy_async();
+    prefetch_tensormap(&tmW);
+    prefetch_tensormap(&tmHi);
+    prefetch_tensormap(&tmLo);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_base_s), (uint32_t)tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+  volatile int *abort_p = &abort_flag;
+
+  const int k0 = cta_start[cta], k1 = cta_start[cta + 1];
+  int fail = 0;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---------------- TMA producer ----------------
+      const uint64_t pol_w = l2_policy_evict_first();   // weights are streamed once per step
+      const uint64_t pol_x = l2_policy_evict_last();    // activations are re-read by every CTA
+      int it = 0;
+      for (int g = k0; g < k1; ++g, ++it) {
+        const int tile = g / KB, kb = g - tile * KB;
+        const int s = it % stages;
+        const uint32_t ph = (uint32_t)(it / stages) & 1u;
+        if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_p)) { fail = DEV_TIMEOUT_PRODUCER; break; }
+        const uint32_t fb = smem_u32(&full_bar[s]);
+        const uint32_t dst = tiles_base + (uint32_t)s * stage_bytes;
+        mbar_arrive_expect_tx(fb, stage_bytes);
+        tma_load_2d(dst, &tmW, kb * GEMM_BLOCK_K, tile * GEMM_TILE_M, fb, pol_w);
+        tma_load_2d(dst + w_bytes, &tmHi, kb * GEMM_BLOCK_K, 0, fb, pol_x);
+        tma_load_2d(dst + w_bytes + x_bytes, &tmLo, kb * GEMM_BLOCK_K, 0, fb, pol_x);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ---------------- MMA issuer ----------------
+      int it = 0, seg = 0;
+      for (int g = k0; g < k1 && !fail; ++seg) {
+        const int tile = g / KB, kb_begin = g - tile * KB;
+        const int kb_end = min(KB, kb_begin + (k1 - g));
+        if (!mbar_wait(smem_u32(&tmem_empty_bar), ((uint32_t)seg & 1u) ^ 1u, abort_p)) { fail = DEV_TIMEOUT_MMA; break; }
+        tc_fence_after();
+        for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
+          const int s = it % stages;
+          const uint32_t ph = (uint32_t)(it / stages) & 1u;
+          if (!mbar_wait(smem_u32(&full_bar[s]), ph, abort_p)) { fail = DEV_TIMEOUT_MMA; break; }
+          tc_fence_after();
+          const uint32_t a_addr = tiles_base + (uint32_t)s * stage_bytes;
+          const uint64_t a_desc = umma_desc_sw128(a_addr);
+          const uint64_t hi_desc = umma_desc_sw128(a_addr + w_bytes);
+          const uint64_t lo_desc = umma_desc_sw128(a_addr + w_bytes + x_bytes);
+#pragma unroll
+          for (int k = 0; k < GEMM_BLOCK_K / 16; ++k) {
+            // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in 16-byte units
+            const uint64_t adv = (uint64_t)(k * 2);
+            umma_bf16(tmem_base, a_desc + adv, hi_desc + adv, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
+            umma_bf16(tmem_base, a_desc + adv, lo_desc + adv, idesc, 1u);
+          }
+          umma_commit(smem_u32(&empty_bar[s]));   // frees the stage once these MMAs have read it
+        }
+        if (fail) break;
+        umma_commit(smem_u32(&tmem_full_bar));    // accumulator of this segment is complete
+        g += kb_end - kb_begin;
+      }
+    }
+  } else {
+    // ---------------- epilogue: TMEM -> registers -> global ----------------
+    const int lane_base = (warp & 3) * 32;          // the TMEM lanes this warp may read
+    const int row = lane_base + lane;               // row of the weight tile = output feature
+    int seg = 0;
+    for (int g = k0; g < k1; ++seg) {
+      const int tile = g / KB, kb_begin = g - tile * KB;
+      const int kb_end = min(KB, kb_begin + (k1 - g));
+      const bool whole = (kb_begin == 0 && kb_end == KB);
+      bool ok = mbar_wait(smem_u32(&tmem_full_bar), (uint32_t)seg & 1u, abort_p);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { fail = DEV_TIMEOUT_EPILOGUE; break; }
+      tc_fence_after();
+      const int n = tile * GEMM_TILE_M + row;
+      float *dst;
+      size_t stride;
+      int rows_out;
+      bool row_ok;
+      if (whole) {
+        dst = direct + n;
+        stride = (size_t)N;
+        rows_out = R;
+        row_ok = n < N;
+      } else {
+        dst = ws + ((size_t)(cta * 2 + (seg == 0 ? 0 : 1)) * BN) * 128 + row;
+        stride = 128;
+        rows_out = BN;
+        row_ok = true;
+      }
+      for (int c0 = 0; c0 < BN; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld16(tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)c0, v);
+        tmem_ld_wait();
+        if (row_ok) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (c0 + j < rows_out) dst[(size_t)(c0 + j) * stride] = __uint_as_float(v[j]);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(smem_u32(&tmem_empty_bar));
+      g += kb_end - kb_begin;
+    }
+  }
+
+  if (fail) {
+    atomicCAS(status, 0, fail);
+    // let copies that are still in flight land before the shared memory is given back
+    for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, (uint32_t)tmem_cols);
+}
+
+__global__ void gemm_fixup_kernel(GemmOut g, float *direct, const int *split_tiles, int R) {
+  const int t = split_tiles[blockIdx.x];
+  const int n = t * 128 + threadIdx.x;
+  if (n >= g.N) return;
+  for (int r = 0; r < R; ++r) direct[(size_t)r * g.N + n] = gemm_load(g, r, n);
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+  if (!fn) {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (PFN_cuTensorMapEncodeTiled_v12000)p;
+  }
+  return fn;
+}
+
+}  // namespace
+
+int gemm_encode_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows) {
+  auto enc = get_encode();
+  if (!enc) return CORUN_ECUDA;
+  if (((uintptr_t)base & 15u) || (K % GEMM_BLOCK_K) || box_rows > 256 || box_rows < 1) return CORUN_EINVAL;
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {(cuuint32_t)GEMM_BLOCK_K, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? CORUN_OK : CORUN_ECUDA;
+}
+
+int gemm_plan_create(GemmPlan *p, const void *W, int N, int K, const void *Xhi, const void *Xlo, int R, int BN,
+                     float *direct, float *ws, int num_sms) {
+  if (N <= 0 || K <= 0 || K % GEMM_BLOCK_K || BN % 16 || BN < 16 || BN > 256 || R < 1 || R > BN) return CORUN_EINVAL;
+  p->N = N; p->K = K; p->R = R; p->BN = BN;
+  p->n_tiles = (N + GEMM_TILE_M - 1) / GEMM_TILE_M;
+  p->KB = K / GEMM_BLOCK_K;
+  const long long total = (long long)p->n_tiles * p->KB;
+  p->grid = (int)(total < num_sms ? total : num_sms);
+  if (total * (long long)p->grid >= (1ll << 31)) return CORUN_EINVAL;
+  const size_t stage = (size_t)GEMM_TILE_M * GEMM_BLOCK_K * 2 + 2 * (size_t)BN * GEMM_BLOCK_K * 2;
+  int stages = (int)((220 * 1024 - 1024) / stage);
+  if (stages > MAX_STAGES) stages = MAX_STAGES;
+  if (stages < 2) return CORUN_EINVAL;
+  p->stages = stages;
+  p->smem_bytes = stage * stages + 1024;
+  p->tmem_cols = 32;
+  while (p->tmem_cols < BN) p->tmem_cols *= 2;
+  // kind::f16 instruction descriptor: D fp32 (bits 4-5 = 1), A and B bf16 (bits 7-9, 10-12 = 1),
+  // both K-major (bits 15, 16 = 0), N >> 3 at bits 17-22, M >> 4 at bits 24-28.
+  p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(GEMM_TILE_M >> 4) << 24);
+  p->direct = direct;
+  p->ws = ws;
+  int rc;
+  if ((rc = gemm_encode_map(&p->tmW, W, N, K, GEMM_TILE_M)) != 0) return rc;
+  if ((rc = gemm_encode_map(&p->tmHi, Xhi, BN, K, BN)) != 0) return rc;
+  if ((rc = gemm_encode_map(&p->tmLo, Xlo, BN, K, BN)) != 0) return rc;
+
+  std::vector<int> tab((size_t)p->grid + 1 + 3 * (size_t)p->n_tiles);
+  int *cs = tab.data(), *cb = cs + p->grid + 1, *ce = cb + p->n_tiles, *sp = ce + p->n_tiles;
+  for (int c = 0; c <= p->grid; ++c) cs[c] = (int)((long long)c * total / p->grid);
+  p->n_split_tiles = 0;
+  for (int t = 0, c = 0; t < p->n_tiles; ++t) {
+    const int first = t * p->KB, last = first + p->KB - 1;
+    while (cs[c + 1] <= first) ++c;
+    cb[t] = c;
+    int d = c;
+    while (cs[d + 1] <= last) ++d;
+    ce[t] = d;
+    if (cb[t] != ce[t]) sp[p->n_split_tiles++] = t;
+  }
+  if (cudaMalloc(&p->d_cta_start, tab.size() * sizeof(int)) != cudaSuccess) return CORUN_ENOMEM;
+  if (cudaMemcpy(p->d_cta_start, tab.data(), tab.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess)
+    return CORUN_ECUDA;
+  p->d_tile_cbeg = p->d_cta_start + p->grid + 1;
+  p->d_tile_cend = p->d_tile_cbeg + p->n_tiles;
+  p->d_split_tiles = p->d_tile_cend + p->n_tiles;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gemm_streamk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+      return CORUN_ECUDA;
+    attr_set = true;
+  }
+  return CORUN_OK;
+}
+
+void gemm_plan_destroy(GemmPlan *p) {
+  if (p->d_cta_start) cudaFree(p->d_cta_start);
+  p->d_cta_start = nullptr;
+}
+
+cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int *d_status, cudaStream_t st) {
+  gemm_streamk_kernel<<<p.grid, GEMM_THREADS, p.smem_bytes, st>>>(tmW_override ? *tmW_override : p.tmW, p.tmHi, p.tmLo,
+                                                                  p.direct, p.ws, p.d_cta_start, p.N, p.KB, p.BN, p.R,
+                                                                  p.stages, p.tmem_cols, p.idesc, d_status);
+  return cudaGetLastError();
+}
+
+cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st) {
+  if (p.n_split_tiles == 0) return cudaSuccess;
+  gemm_fixup_kernel<<<p.n_split_tiles, 128, 0, st>>>(p.out(), p.direct, p.d_split_tiles, p.R);
+  return cudaGetLastError();
+}
+
+}  // namespace corun

@@ -1,0 +1,72 @@
+// Launchers of the non-GEMM kernels of the decode / prefill row program.
+// A "row" is one query token: in decode row r is slot r, in prefill the rows
+// are consecutive prompt positions of one slot.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gemm.cuh"
+
+namespace corun {
+
+constexpr int KV_BLOCK = 16;      // tokens per page
+constexpr int ATT_SPLIT = 256;    // tokens per attention split (fixed; count = f(own context))
+
+// Per-row metadata (device arrays of length R).
+struct Rows {
+  const int *token;    // token fed to the row
+  const int *pos;      // position of that token = tokens cached before it
+  const int *active;   // 0 = padding row
+  const int *slot;     // whose block table the row uses
+  int R;
+};
+
+struct KvLayout {
+  __half *pool;            // [layer][block][k|v][n_kv][16][hd]
+  const int *block_table;  // [n_slots][max_blocks]
+  int max_blocks, n_kv, hd;
+  size_t layer_stride;     // halfs per layer
+};
+
+struct SampleArgs {
+  const float *logits;     // [R, V]
+  int V;
+  const int *do_sample;    // per row: 0 skip, 1 sample
+  const float *temperature, *top_p;  // per row
+  const uint64_t *seed;    // per row
+  const int *step;         // per row: t of R(seed, t)
+  const uint32_t *u24_override;  // optional per-row variate (debug); nullptr = Philox
+  int *out_token;          // per row (untouched when skipped)
+};
+
+// h = E[token] (first = 1) or h += GEMM result (first = 0); then RMSNorm with
+// gains g -> bf16 hi/lo pair.
+cudaError_t launch_resid_norm(float *h, int H, const __nv_bfloat16 *embed, const Rows &rows, const GemmOut *prev,
+                              const __nv_bfloat16 *gains, float eps, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
+                              cudaStream_t st);
+// RoPE on q and k, q -> q_out fp32 [R, nq*hd], k/v -> pages (fp16) at the row's position.
+cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *rope_tab, int nq, const KvLayout &kv,
+                            int layer, float *q_out, cudaStream_t st);
+// Split-KV paged attention partials and their fixed-order combine -> bf16 hi/lo [R, nq*hd].
+cudaError_t launch_attention(const float *q, const Rows &rows, int nq, const KvLayout &kv, int layer, int max_splits,
+                             float *part_acc, float *part_ml, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
+                             cudaStream_t st);
+// y = silu(gate) * up from the gate-up GEMM result -> bf16 hi/lo [R, F].
+cudaError_t launch_swiglu(const GemmOut &gu, int R, int F, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, cudaStream_t st);
+// x fp32 [R, K] -> bf16 hi/lo.
+cudaError_t launch_split(const float *x, int R, int K, __nv_bfloat16 *hi, __nv_bfloat16 *lo, cudaStream_t st);
+cudaError_t launch_sampler(const SampleArgs &a, int R, cudaStream_t st);
+// decode bookkeeping
+cudaError_t launch_prepare_rows(const uint8_t *active_mask, const int *in_use, const int *ctx_len, const int *pending,
+                                int B, int *row_token, int *row_pos, int *row_active, int *row_slot, int *do_sample,
+                                cudaStream_t st);
+cudaError_t launch_advance(const int *row_active, const int *sampled, int B, int *ctx_len, int *step, int *pending,
+                           int *out_tokens, cudaStream_t st);
+// debug cache access (fp32 rows of n_kv*hd)
+cudaError_t launch_kv_copy(const KvLayout &kv, int layer, int slot, int pos0, int n, float *k, float *v, int write,
+                           cudaStream_t st);
+cudaError_t launch_variate(uint64_t seed, uint64_t t, uint32_t *out, cudaStream_t st);
+
+}  // namespace corun

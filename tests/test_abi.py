@@ -1,0 +1,70 @@
+"""The C-ABI library loads without a GPU and exports every symbol the header declares."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2608_14376_b200 import build, corun
+
+    build.build()
+    return corun.lib()
+
+
+def _declared():
+    src = open(os.path.join(ROOT, "include", "corun.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(corun_[a-z_0-9]+)\s*\(", src)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared()
+    assert "corun_init" in names and "corun_prefill" in names and "corun_decode_step" in names \
+        and "corun_release" in names
+    for n in names:
+        assert getattr(lib, n) is not None, n
+
+
+def test_binding_lists_the_same_symbols():
+    from paper_2608_14376_b200 import corun
+
+    assert sorted(corun.EXPORTS) == _declared()
+
+
+def test_argument_validation_needs_no_gpu(lib):
+    from paper_2608_14376_b200 import corun
+
+    h = C.c_void_p()
+    assert lib.corun_init(None, None, 1, 16, 16, 0, None, C.byref(h)) == corun.EINVAL
+    sh = corun.Shape(2, 250, 4, 2, 64, 768, 2048, 1e-6, 1e4, 0)     # hidden not a multiple of 64
+    w = corun.Weights()
+    assert lib.corun_init(C.byref(sh), C.byref(w), 1, 16, 16, 0, None, C.byref(h)) == corun.EINVAL
+    assert lib.corun_decode_step(None, None, None, None) == corun.EINVAL
+    assert lib.corun_release(None, 0) == corun.EINVAL
+    assert lib.corun_prefill(None, 0, None, 0, 0, None, 0, None) == corun.EINVAL
+    assert lib.corun_debug_gemm(None, 1, 64, None, 1, None, None) == corun.EINVAL
+    lib.corun_destroy(None)
+
+
+def test_strerror_covers_every_status(lib):
+    seen = set()
+    for st in range(0, -8, -1):
+        s = lib.corun_strerror(st)
+        assert s and s != b"unknown status"
+        seen.add(s)
+    assert len(seen) == 8
+    assert lib.corun_strerror(-99) == b"unknown status"
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    from paper_2608_14376_b200 import corun
+
+    monkeypatch.setattr(corun, "_lib", None)
+    monkeypatch.setattr(corun, "LIB_PATH", "/nonexistent/libcorun.so")
+    with pytest.raises(RuntimeError):
+        corun.lib()

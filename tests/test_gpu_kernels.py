@@ -1,0 +1,115 @@
+"""GPU parity of single kernels against the oracle, through the C ABI."""
+import numpy as np
+import pytest
+
+from paper_2608_14376_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def torch_cuda():
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    return torch
+
+
+def _gemm_case(orc, torch, R, N, K, seed):
+    from paper_2608_14376_b200 import corun
+
+    rng = np.random.default_rng(seed)
+    Wb = synth.f32_to_bf16_bits(rng.standard_normal((N, K)).astype(np.float32) * 0.02)
+    X = rng.standard_normal((R, K)).astype(np.float32)
+    Wt = torch.from_numpy(Wb.view(np.int16).copy()).view(torch.bfloat16).cuda()
+    Xt = torch.from_numpy(X).cuda()
+    out = corun.debug_gemm(Wt, Xt).cpu().numpy()
+    ref = orc.matmul_bf16(Wb, X)
+    return out, ref, Wt, Xt
+
+
+# rows x weight rows x K: single tile, ragged N, several tiles, more k-blocks than CTAs, all 256 rows
+@pytest.mark.parametrize("R,N,K", [(8, 128, 64), (8, 512, 256), (5, 384, 768), (1, 2048, 256), (40, 200, 128),
+                                   (64, 1536, 256), (64, 4096, 4096), (130, 1024, 1024), (256, 512, 512)])
+def test_gemm_matches_oracle(orc, torch_cuda, R, N, K):
+    out, ref, _, _ = _gemm_case(orc, torch_cuda, R, N, K, seed=R + N + K)
+    # split activations carry 16 significand bits: error << 1e-4 of the output scale (0.02 * sqrt(K))
+    tol = 2e-5 * 0.02 * np.sqrt(K) * 4 + 1e-6
+    assert np.abs(out - ref).max() <= tol, (np.abs(out - ref).max(), tol)
+
+
+def test_gemm_rows_are_position_invariant(orc, torch_cuda):
+    from paper_2608_14376_b200 import corun
+
+    torch = torch_cuda
+    out, _, Wt, Xt = _gemm_case(orc, torch, 64, 1024, 4096, seed=3)
+    perm = torch.randperm(64, generator=torch.Generator().manual_seed(1)).cuda()
+    out_p = corun.debug_gemm(Wt, Xt[perm].contiguous()).cpu().numpy()
+    np.testing.assert_array_equal(out_p, out[perm.cpu().numpy()])
+    # other rows' values cannot leak into a row
+    Y = Xt.clone()
+    Y[1:] = 1e30
+    out_y = corun.debug_gemm(Wt, Y).cpu().numpy()
+    np.testing.assert_array_equal(out_y[0], out[0])
+    # repeated runs
+    np.testing.assert_array_equal(corun.debug_gemm(Wt, Xt).cpu().numpy(), out)
+
+
+def test_variate_matches_oracle(orc, torch_cuda):
+    from paper_2608_14376_b200 import corun
+
+    rng = np.random.default_rng(0)
+    pairs = [(0, 0), (1042, 7), (2**63 + 11, 2**33 + 5)] + [
+        (int(rng.integers(0, 2**63)), int(rng.integers(0, 4096))) for _ in range(1500)]
+    for seed, t in pairs:
+        assert corun.debug_variate(seed, t) == orc.variate_u24(seed, t)
+
+
+def _check_sampler(orc, logits, T, top_p, us):
+    from paper_2608_14376_b200 import corun
+
+    rows = np.repeat(logits[None], len(us), axis=0)
+    got = corun.debug_sample(rows, T, top_p, np.array(us, np.uint32))
+    n_checked = 0
+    for u, g in zip(us, got):
+        want, margin = orc.sample(logits, T, top_p, int(u))
+        if margin < 1e-5:          # decision within fp32-vs-fp64 weight rounding of a boundary
+            continue
+        assert g == want, (u, g, want, margin)
+        n_checked += 1
+    return n_checked
+
+
+@pytest.mark.parametrize("V", [2048, 151936])
+def test_sampler_matches_oracle(orc, torch_cuda, V):
+    rng = np.random.default_rng(V)
+    us = [0, 1, (1 << 24) - 1, 1 << 23] + [int(x) for x in rng.integers(0, 1 << 24, 28)]
+    logits = (rng.standard_normal(V) * 1.28).astype(np.float32)
+    n = 0
+    for T, top_p in [(0.7, 0.95), (1.0, 1.0), (0.6, 0.5), (0.7, 1e-6), (2.0, 0.999)]:
+        n += _check_sampler(orc, logits, T, top_p, us)
+    assert n > 100
+    # greedy
+    from paper_2608_14376_b200 import corun
+
+    assert corun.debug_sample(logits, 0.0, 1.0, [5])[0] == int(np.argmax(logits))
+
+
+def test_sampler_ties_and_degenerate_rows(orc, torch_cuda):
+    from paper_2608_14376_b200 import corun
+
+    rng = np.random.default_rng(5)
+    us = [int(x) for x in rng.integers(0, 1 << 24, 32)]
+    # heavily tied logits (quantised to 1/4): the nucleus edge falls inside a tie group
+    tied = (np.round(rng.standard_normal(4096) * 4) / 4).astype(np.float32)
+    assert _check_sampler(orc, tied, 0.7, 0.9, us) > 20
+    assert _check_sampler(orc, tied, 1.0, 0.3, us) > 20
+    # all equal
+    flat = np.zeros(1000, np.float32)
+    assert _check_sampler(orc, flat, 1.0, 0.5, us) > 20
+    # one dominant token, very wide range
+    wide = (rng.standard_normal(3000) * 30).astype(np.float32)
+    assert _check_sampler(orc, wide, 0.7, 0.95, us) > 20
+    # argmax picks the lowest id among equal maxima
+    two = np.zeros(777, np.float32); two[[5, 300]] = 3.0
+    assert corun.debug_sample(two, 0.0, 1.0, [0])[0] == 5
