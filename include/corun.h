@@ -120,7 +120,11 @@ int corun_prefill(corun_engine *e, int32_t slot, const int32_t *tokens, int32_t 
  * launch shape, consume no random variate, change no state and report -1.
  *   active      host, B bytes.       seeds  host, B values (read where active).
  *   out_tokens  host, B ints.
- * Sampling: weight_i = floor(2^40 * exp((logit_i - max)/T)); nucleus = tokens
+ * Sampling: weight_i = floor(2^40 * exp2(fl32(fl32(logit_i - max) * fl32(log2(e)/T))))
+ * where exp2 is evaluated in fp32 as: n = rint(x), f = x - n, degree-7 Taylor
+ * polynomial of 2^f (coefficients ln(2)^k/k! rounded to fp32) in Horner form with
+ * separately rounded multiply and add, scaled exactly by 2^n -- an integer that is
+ * identical on every IEEE-754 implementation; nucleus = tokens
  * by descending logit (ties: lower id first) up to and including the first
  * whose running weight reaches floor(top_p * total); draw r = floor(u24 * Z / 2^24)
  * with u24 the top 24 bits of Philox4x32-10(key = seed, counter = (t,0,0,0));

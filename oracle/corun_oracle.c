@@ -262,18 +262,55 @@ static int orc_item_desc(const void *pa, const void *pb) {
 }
 
 /*
+ * exp2 as S defines it: fp32, round-to-nearest-even split x = n + f with
+ * |f| <= 1/2, then the degree-7 Taylor polynomial of 2^f (coefficients
+ * ln(2)^k / k! rounded to fp32) in Horner form with separately rounded
+ * multiplies and adds (no fused multiply-add), then the exact scaling by 2^n.
+ * Spelling the arithmetic out makes the integer weights below reproducible bit
+ * for bit on any IEEE-754 machine, so that the sampling decision (an integer) is
+ * taken in one stated precision by every implementation.  Relative error < 1e-7.
+ */
+static float orc_pexp2_mantissa(float x, int *n_out) {
+  static const float c[8] = {1.0f, 0x1.62e430p-1f, 0x1.ebfbe0p-3f, 0x1.c6b08ep-5f, 0x1.3b2ab6p-7f,
+                             0x1.5d87fep-10f, 0x1.430912p-13f, 0x1.ffcbfcp-17f};
+  float n = rintf(x);
+  float f = x - n;
+  float p = c[7];
+  for (int k = 6; k >= 0; --k) {
+    float t = p * f;
+    p = t + c[k];
+  }
+  *n_out = (int)n;
+  return p;
+}
+
+/* weight = floor(2^40 * 2^x) for x <= 0, x in fp32 */
+uint64_t orc_weight(float logit, float max_logit, float inv_t_log2e) {
+  float d = logit - max_logit;
+  float x = d * inv_t_log2e;
+  if (!(x > -64.0f)) return 0;
+  int n;
+  float p = orc_pexp2_mantissa(x, &n);
+  if (n < -41) return 0;
+  return (uint64_t)ldexpf(p, n + 40);      /* exact scaling, then truncation */
+}
+
+/*
  * S(logits, u24).  temperature == 0: argmax, lowest id on ties.  Otherwise:
- *   weight_i = floor(2^40 * exp((logit_i - max) / temperature))   (integer)
- *   total    = sum_i weight_i ;  cut = floor(top_p * total)
+ *   weight_i = floor(2^40 * exp2(fl32(fl32(logit_i - max) * fl32(log2(e) / temperature))))
+ *              with exp2 as defined above (integer; equals floor(2^40 * exp((logit_i - max)/T))
+ *              up to a relative 2e-7)
+ *   total    = sum_i weight_i ;  cut = floor(top_p * total)   (fp64 product)
  *   nucleus  = tokens in descending logit order (ties: lower id first) up to
  *              and including the first whose running weight sum >= cut
  *   Z = nucleus weight ;  r = floor(u24 * Z / 2^24)
  *   token    = first nucleus member, in ascending id order, whose running
  *              weight sum exceeds r.
- * The integer weights make every later decision exact.  `margin` (optional)
- * receives how close, relative to `total`, the decision came to flipping
- * (min of: distance of r to the nearest running-sum boundary, distance of the
- * cut to the running sums adjacent to the nucleus edge).
+ * The weights are integers in a stated fp32 arithmetic, so every decision is
+ * exact and any implementation must return the same token.  `margin`
+ * (optional) receives how close, relative to `total`, the decision came to
+ * flipping (min of: distance of r to the nearest running-sum boundary,
+ * distance of the cut to the running sums adjacent to the nucleus edge).
  */
 int32_t orc_sample(const float *logits, int64_t V, float temperature, float top_p, uint32_t u24, double *margin) {
   int64_t best = 0;
@@ -282,13 +319,13 @@ int32_t orc_sample(const float *logits, int64_t V, float temperature, float top_
   if (margin) *margin = 1.0;
   if (temperature <= 0.0f) return (int32_t)best;
 
-  double mx = (double)logits[best];
+  const float mx = logits[best];
+  const float inv_t_log2e = 0x1.715476p+0f / temperature;
   uint64_t *wgt = (uint64_t *)malloc(sizeof(uint64_t) * (size_t)V);
   orc_item *it = (orc_item *)malloc(sizeof(orc_item) * (size_t)V);
   uint64_t total = 0;
   for (int64_t i = 0; i < V; ++i) {
-    double e = exp(((double)logits[i] - mx) / (double)temperature);
-    wgt[i] = (uint64_t)floor(ldexp(e, 40));
+    wgt[i] = orc_weight(logits[i], mx, inv_t_log2e);
     total += wgt[i];
     it[i].idx = i;
     it[i].logit = logits[i];

@@ -28,7 +28,7 @@ def build(force: bool = False) -> str:
     """Compile the oracle with gcc (-O2, OpenMP, no fast-math) and return the path."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         subprocess.check_call(
-            ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=gnu11", "-o", _LIB, _SRC, "-lm"]
+            ["gcc", "-O2", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared", "-std=gnu11", "-o", _LIB, _SRC, "-lm"]
         )
     return _LIB
 
@@ -73,6 +73,8 @@ def lib():
         L.orc_sample.restype = C.c_int32
         L.orc_sample.argtypes = [C.c_void_p, C.c_int64, C.c_float, C.c_float, C.c_uint32, C.POINTER(C.c_double)]
         L.orc_num_threads.restype = C.c_int
+        L.orc_weight.restype = C.c_uint64
+        L.orc_weight.argtypes = [C.c_float, C.c_float, C.c_float]
         _lib = L
     return _lib
 
@@ -248,6 +250,11 @@ def sample(logits, temperature: float, top_p: float, u24: int):
     m = C.c_double(0.0)
     tok = lib().orc_sample(_ptr(lg), lg.shape[0], temperature, top_p, u24, C.byref(m))
     return int(tok), float(m.value)
+
+
+def weight(logit: float, max_logit: float, inv_t_log2e: float) -> int:
+    """Integer sampling weight floor(2^40 * exp2(...)) of one token (see corun_oracle.c)."""
+    return int(lib().orc_weight(logit, max_logit, inv_t_log2e))
 
 
 def num_threads() -> int:

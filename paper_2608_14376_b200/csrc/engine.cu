@@ -16,7 +16,6 @@
 
 using namespace corun;
 
-static int g_last_cuda_error = 0;
 
 #define CK(call)                                   \
   do {                                             \

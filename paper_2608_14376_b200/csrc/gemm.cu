@@ -10,6 +10,8 @@
 
 namespace corun {
 
+int g_last_cuda_error = 0;
+
 namespace {
 
 constexpr int MAX_STAGES = 8;
@@ -193,7 +195,7 @@ PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
 
 int gemm_encode_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows) {
   auto enc = get_encode();
-  if (!enc) return CORUN_ECUDA;
+  if (!enc) { g_last_cuda_error = 99999; return CORUN_ECUDA; }
   if (((uintptr_t)base & 15u) || (K % GEMM_BLOCK_K) || box_rows > 256 || box_rows < 1) return CORUN_EINVAL;
   cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)K * 2};
@@ -202,6 +204,7 @@ int gemm_encode_map(CUtensorMap *m, const void *base, int rows, int K, int box_r
   CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) g_last_cuda_error = 100000 + (int)r;
   return r == CUDA_SUCCESS ? CORUN_OK : CORUN_ECUDA;
 }
 
@@ -246,15 +249,15 @@ int gemm_plan_create(GemmPlan *p, const void *W, int N, int K, const void *Xhi, 
     if (cb[t] != ce[t]) sp[p->n_split_tiles++] = t;
   }
   if (cudaMalloc(&p->d_cta_start, tab.size() * sizeof(int)) != cudaSuccess) return CORUN_ENOMEM;
-  if (cudaMemcpy(p->d_cta_start, tab.data(), tab.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess)
-    return CORUN_ECUDA;
+  cudaError_t me = cudaMemcpy(p->d_cta_start, tab.data(), tab.size() * sizeof(int), cudaMemcpyHostToDevice);
+  if (me != cudaSuccess) { g_last_cuda_error = (int)me; return CORUN_ECUDA; }
   p->d_tile_cbeg = p->d_cta_start + p->grid + 1;
   p->d_tile_cend = p->d_tile_cbeg + p->n_tiles;
   p->d_split_tiles = p->d_tile_cend + p->n_tiles;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_streamk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
-      return CORUN_ECUDA;
+    cudaError_t ae = cudaFuncSetAttribute(gemm_streamk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 221 * 1024);
+    if (ae != cudaSuccess) { g_last_cuda_error = (int)ae; return CORUN_ECUDA; }
     attr_set = true;
   }
   return CORUN_OK;

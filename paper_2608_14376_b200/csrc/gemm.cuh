@@ -15,6 +15,9 @@
 
 namespace corun {
 
+// Last CUDA runtime error (cudaError_t), or 100000 + CUresult for driver calls.
+extern int g_last_cuda_error;
+
 constexpr int GEMM_TILE_M = 128;   // weight rows per tile
 constexpr int GEMM_BLOCK_K = 64;   // bf16 elements per k-block (= one 128-byte swizzle row)
 constexpr int GEMM_THREADS = 192;  // warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 epilogue

@@ -397,10 +397,27 @@ struct SmpShared {
   int sel_bin, winner;
 };
 
-// Integer weight of a token: floor(2^40 * exp((l - max)/T)), evaluated in fp32.
+// Integer weight of a token: floor(2^40 * exp2(x)), x = fl32(fl32(l - max) * inv_t_log2e).
+// exp2 is spelled out so that the integer is the same on every IEEE-754 machine:
+// x = n + f with n = rint(x); degree-7 Taylor polynomial of 2^f (ln(2)^k / k! in fp32),
+// Horner form, separately rounded multiplies and adds; exact scaling by 2^(n+40).
 __device__ __forceinline__ unsigned long long smp_weight(float l, float mx, float inv_t_log2e) {
-  const float e = exp2f((l - mx) * inv_t_log2e);
-  return (unsigned long long)(e * 1099511627776.0f);
+  const float x = __fmul_rn(__fsub_rn(l, mx), inv_t_log2e);
+  if (!(x > -64.0f)) return 0ull;
+  const float n = rintf(x);
+  const float f = __fsub_rn(x, n);
+  float p = 0x1.ffcbfcp-17f;
+  p = __fadd_rn(__fmul_rn(p, f), 0x1.430912p-13f);
+  p = __fadd_rn(__fmul_rn(p, f), 0x1.5d87fep-10f);
+  p = __fadd_rn(__fmul_rn(p, f), 0x1.3b2ab6p-7f);
+  p = __fadd_rn(__fmul_rn(p, f), 0x1.c6b08ep-5f);
+  p = __fadd_rn(__fmul_rn(p, f), 0x1.ebfbe0p-3f);
+  p = __fadd_rn(__fmul_rn(p, f), 0x1.62e430p-1f);
+  p = __fadd_rn(__fmul_rn(p, f), 1.0f);
+  const int ni = (int)n;
+  if (ni < -41) return 0ull;
+  const float scale = __int_as_float((ni + 40 + 127) << 23);   // 2^(n+40), exact
+  return (unsigned long long)__fmul_rn(p, scale);              // truncation = floor
 }
 
 // After a histogram pass: finds the first bin (ascending index = descending
@@ -461,7 +478,7 @@ __global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
     return;
   }
   const float mx = bv;
-  const float inv_t_log2e = 1.4426950408889634f / temperature;
+  const float inv_t_log2e = __fdiv_rn(0x1.715476p+0f, temperature);
   const uint32_t u24 = a.u24_override ? a.u24_override[r] : philox_u24(a.seed[r], (uint64_t)a.step[r]);
 
   // ---- pass A: bins linear in (max - logit); bin 0 holds the largest logits

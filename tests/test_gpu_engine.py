@@ -136,11 +136,10 @@ def test_sampled_decoding_is_invariant_and_matches_S_on_gpu_logits(orc, tiny, en
     checked = 0
     for t, (row, tok) in enumerate(zip(rows, toks)):
         lg = np.frombuffer(row, np.float32)
-        want, margin = orc.sample(lg, T, P, orc.variate_u24(seed, t))
-        if margin >= 1e-5:
-            assert tok == want, t
-            checked += 1
-    assert checked >= 10
+        want, _ = orc.sample(lg, T, P, orc.variate_u24(seed, t))
+        assert tok == want, t
+        checked += 1
+    assert checked == 13
     # a different seed draws different variates
     _, toks3 = _run_request(engine, 2, prompts[0], seed + 1, {}, 12, T, P)
     assert toks3 != toks
@@ -191,7 +190,7 @@ def test_error_paths(tiny, engine):
     engine.decode_step(active, np.zeros(B, np.uint64))                            # ctx 16 -> 17 = reserve
     assert status(lambda: engine.decode_step(active, np.zeros(B, np.uint64))) == corun.ECTX
     assert engine.context_len(0) == 17                                            # refused step changed nothing
-    active[3] = 1
+    active[0] = 0; active[3] = 1                                                  # slot 3 is empty
     assert status(lambda: engine.decode_step(active, np.zeros(B, np.uint64))) == corun.ESLOT
     engine.release(0)
 

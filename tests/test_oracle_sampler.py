@@ -124,3 +124,20 @@ def test_margin_reports_closeness_to_a_boundary(orc):
     assert tok == 1 and m < 1e-6
     tok, m = orc.sample(lg, 1.0, 1.0, 1 << 22)
     assert tok == 0 and abs(m - 0.25) < 1e-6
+
+
+def test_integer_weight_follows_the_exponential(orc):
+    """floor(2^40 * exp2(x)) in the stated fp32 arithmetic stays within 2e-7 of the exact exponential."""
+    rng = np.random.default_rng(3)
+    c = float(np.float32(1.4426950408889634) / np.float32(0.7))
+    worst = 0.0
+    for d in np.concatenate([rng.uniform(-25, 0, 4000), [0.0, -1e-7, -0.5, -19.999]]):
+        l = np.float32(d)
+        x = float(np.float32(np.float32(l - np.float32(0.0)) * np.float32(c)))
+        w = orc.weight(float(l), 0.0, c)
+        exact = 2.0 ** (40 + x)
+        assert abs(w - exact) <= 2e-7 * exact + 1.0
+        worst = max(worst, abs(w - exact) / exact)
+    assert orc.weight(0.0, 0.0, c) == 1 << 40
+    assert orc.weight(-100.0, 0.0, c) == 0
+    assert orc.weight(-19.4, 0.0, c) > 0          # 2^40 * 2^-39.98: the last non-zero weights
