@@ -1,0 +1,331 @@
+#!/usr/bin/env python
+"""Decode benchmark of the CoRun hot path (one JSON line on stdout).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl corun|reference] [--workload NAME]
+
+A step is one fixed-shape decode iteration (one graph replay) over the whole
+padded batch.  Workload ``qwen3_8b_b64`` is the Qwen3-8B-shaped configuration:
+B = 64 slots, 40 active, per-slot context uniform in 512..4096, KV block 16,
+seeded top-p 0.95 / temperature 0.7 sampling, random bf16 weights N(0, 0.02).
+The cache is filled with seeded synthetic values on the device before timing.
+
+N > 1 runs N independent replicas (the path does not shard; no collectives on
+the data path); the value is the sum over replicas divided by the slowest one.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_14376_b200 import synth  # noqa: E402
+
+WORKLOADS = {
+    # name: (shape, B, n_active, ctx_lo, ctx_hi, temperature, top_p, kv std)
+    "qwen3_8b_b64": (synth.QWEN3_8B, 64, 40, 512, 4096, 0.7, 0.95, 1.28),
+    "tiny_b8": (synth.TINY, 8, 5, 16, 64, 0.7, 0.95, 0.3),
+}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), float(d.get("bf16_tflops", 1590.0)), "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.t.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def workload_inputs(name: str):
+    sh, B, n_active, lo, hi, T, P, kv_std = WORKLOADS[name]
+    slots = synth.pick_slots(B, n_active, seed=7)
+    ctx = synth.uniform_lengths(lo, hi, n_active, seed=2)
+    return sh, B, slots, ctx, T, P, kv_std
+
+
+def oracle_decode_sample(sh, w_np, ctxs, kv_std, n_steps, warmup, T, P):
+    """Times the oracle, as it stands, on one decode step per listed context (independent requests)."""
+    from oracle import oracle
+
+    model = oracle.Model(oracle.Shape(**sh.dict()), w_np)
+    reqs = []
+    for i, c in enumerate(ctxs):
+        cache = model.new_cache(int(c) + n_steps + warmup + 1)
+        for layer in range(sh.n_layers):
+            k, v = synth.synthetic_kv(int(c), sh.kv_dim, kv_std, seed=100 * i + layer)
+            cache[0][layer, :int(c)] = k
+            cache[1][layer, :int(c)] = v
+        reqs.append([cache, int(c), 1 + i, synth.request_seed(i)])
+    times = []
+    for step in range(warmup + n_steps):
+        t0 = time.perf_counter()
+        for rq in reqs:
+            cache, c, tok, seed = rq
+            lg = model.forward([tok], c, cache)
+            rq[2], _ = oracle.sample(lg, T, P, oracle.variate_u24(seed, step + 1))
+            rq[1] = c + 1
+        if step >= warmup:
+            times.append(time.perf_counter() - t0)
+    return times, oracle.num_threads()
+
+
+def make_weights(sh, device):
+    import torch
+
+    if device == "cuda" and torch.cuda.is_available():
+        return synth.make_weights_torch(sh, seed=0, device="cuda")
+    return synth.make_weights_torch(sh, seed=0, device="cpu")
+
+
+def run_reference(args, rank, world):
+    """Reference arm = the CPU oracle on the host cores, rank 0 only."""
+    if rank != 0:
+        return
+    import torch
+
+    sh, B, slots, ctx, T, P, kv_std = workload_inputs(args.workload)
+    w_t = make_weights(sh, "cuda" if torch.cuda.is_available() else "cpu")
+    w_np = synth.weights_torch_to_numpy(w_t)
+    del w_t
+    sample = [int(ctx[0])]
+    times, cores = oracle_decode_sample(sh, w_np, sample, kv_std, args.steps, args.warmup, T, P)
+    ms = 1e3 * sum(times) / len(times)
+    val = len(sample) / (ms / 1e3)
+    desc = f"{len(sample)} of {len(slots)} active requests (context {sample[0]}), one decode token each per step"
+    print(json.dumps({
+        "impl": "reference", "metric": "decode_tok_per_s", "value": val, "unit": "tok/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64 accumulate / f32 storage", "data": "synthetic",
+        "config": {"workload": args.workload, "B": B, "active": len(slots), "sample": desc},
+        "cpu_baseline": {"value": val, "unit": "tok/s", "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": "tok/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_corun(args, rank, world):
+    import torch
+
+    from paper_2608_14376_b200 import build as cbuild, corun
+
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        cbuild.build()
+    if dist:
+        dist.barrier()
+    sh, B, slots, ctx, T, P, kv_std = workload_inputs(args.workload)
+    K, W = args.steps, args.warmup
+    total_steps = 2 * (K + W) + 8
+    max_ctx = -(-(int(ctx.max()) + total_steps + 16) // 256) * 256
+    w_t = make_weights(sh, "cuda")
+    stream = torch.cuda.Stream()
+    eng = corun.Engine(sh, w_t, B, max_ctx, stream=stream.cuda_stream)
+    for i, (s, c) in enumerate(zip(slots, ctx)):
+        eng.adopt(int(s), 0, int(c) + total_steps, pending=1 + i, temperature=T, top_p=P, step=1)
+        eng.kv_fill(int(s), int(c), kv_std, seed=100 + i)
+    active = np.zeros(B, np.uint8); active[slots] = 1
+    seeds = np.zeros(B, np.uint64)
+    for i, s in enumerate(slots):
+        seeds[s] = synth.request_seed(i)
+    n_active = int(active.sum())
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident timing: K graph replays back to back, CUDA events on the engine's stream
+    for _ in range(W):
+        eng.decode_enqueue(active, seeds)
+    eng.decode_wait()
+    sync_all()
+    clocks = ClockSampler(local)
+    clocks.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+    ev[0].record(stream)
+    for i in range(K):
+        eng.decode_enqueue(active, seeds)
+        ev[i + 1].record(stream)
+    toks = eng.decode_wait()
+    sync_all()
+    clk = clocks.stop()
+    assert all(toks[s] >= 0 for s in slots) and all(toks[s] == -1 for s in range(B) if not active[s])
+    step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(K)]
+    total_ms = ev[0].elapsed_time(ev[K])
+    if dist:
+        t = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / K
+    value = world * n_active / (ms_per_step / 1e3)
+
+    # ---- end to end through the C ABI with host buffers: mask + seeds in, tokens out, every step
+    for _ in range(W):
+        eng.decode_step(active, seeds)
+    sync_all()
+    t0 = time.perf_counter()
+    for _ in range(K):
+        toks = eng.decode_step(active, seeds)
+    e2e_s = time.perf_counter() - t0
+    if dist:
+        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_val = world * n_active * K / e2e_s
+
+    # ---- per-kernel durations (isolated launches rotating over the layers' weights, CUDA events)
+    L = sh.n_layers
+    reps = max(10, min(72, 2 * L))
+    kt = {name: eng.time_kernel(i, reps if i != 4 and i != 9 else 10) for i, name in enumerate(eng.KERNEL_KINDS)}
+    gemm_ms = L * (kt["gemm_qkv"] + kt["gemm_o"] + kt["gemm_gate_up"] + kt["gemm_down"]) + kt["gemm_lm_head"]
+    n_gemm = 4 * L + 1
+    w_bytes = sh.weight_bytes_per_step()
+    cur_ctx = [eng.context_len(int(s)) for s in slots]
+    kv_bytes = sum(c * sh.kv_bytes_per_token(2) for c in cur_ctx)
+    kv_bytes_mid = sum((int(c) + W + K // 2) * sh.kv_bytes_per_token(2) for c in ctx)
+    hbm, tf, which = measured_peaks()
+    flops = 2 * B * (w_bytes // 2) + 4 * sh.n_q_heads * sh.head_dim * sh.n_layers * sum(int(c) for c in ctx)
+    t_roof_ms = max((w_bytes + kv_bytes_mid) / (hbm * 1e9), flops / (tf * 1e12)) * 1e3
+    traffic = None
+    tp = os.path.join(ROOT, "profiles", "gemm_dram_traffic.json")
+    if os.path.exists(tp) and args.workload == "qwen3_8b_b64":
+        traffic = json.load(open(tp)).get("dram_bytes_per_launch_avg")
+    roofline = {
+        "kernel": "gemm_streamk_kernel (all %d launches of a step)" % n_gemm, "bound": "hbm",
+        "achieved": (w_bytes / n_gemm) / (gemm_ms / n_gemm * 1e-3) / 1e9, "peak": hbm, "unit": "GB/s",
+        "peak_source": which + " (MEASURED_PEAKS.json hbm_gbs)" if which == "measured" else "fallback 6650",
+        "traffic": traffic, "bytes_per_launch_avg": w_bytes / n_gemm, "ms_per_launch_avg": gemm_ms / n_gemm,
+    }
+    roofline["frac"] = roofline["achieved"] / hbm
+    att_bytes = kv_bytes / L
+    step_roof = {"bytes": w_bytes + kv_bytes_mid, "flops": flops, "t_roofline_ms": t_roof_ms,
+                 "frac_of_" + which: t_roof_ms / ms_per_step,
+                 "frac_of_nominal_8TBs": max((w_bytes + kv_bytes_mid) / 8e12, flops / 2.25e15) * 1e3 / ms_per_step}
+    kernels = {k: {"ms_per_launch": v} for k, v in kt.items()}
+    for k, n in (("gemm_qkv", sh.qkv_dim * sh.hidden), ("gemm_o", sh.hidden * sh.q_dim),
+                 ("gemm_gate_up", 2 * sh.ffn * sh.hidden), ("gemm_down", sh.hidden * sh.ffn),
+                 ("gemm_lm_head", sh.vocab * sh.hidden)):
+        kernels[k]["GBs"] = 2 * n / (kt[k] * 1e-3) / 1e9
+    kernels["attention"]["GBs"] = att_bytes / (kt["attention"] * 1e-3) / 1e9
+    launches = eng.decode_launches()
+
+    cpu = None
+    if rank == 0 and not args.no_cpu_baseline:
+        w_np = synth.weights_torch_to_numpy(w_t)
+        n_s = 2 if sh.n_layers > 8 else len(slots)
+        sample = [int(c) for c in ctx[:n_s]]
+        times, cores = oracle_decode_sample(sh, w_np, sample, kv_std, 2, 1, T, P)
+        v = n_s / (sum(times) / len(times))
+        cpu = {"value": v, "unit": "tok/s", "cores": cores, "kind": "oracle",
+               "sample": f"{n_s} of {len(slots)} active requests (contexts {sample}), one decode token each, "
+                         f"2 timed steps after 1 warm-up"}
+    eng.close()
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    srt = sorted(step_ms)
+    print(json.dumps({
+        "metric": "decode_tok_per_s", "value": value, "unit": "tok/s", "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 weights x split-bf16 activations, fp32 accumulate; fp16 KV; fp32 attention and residual",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "B": B, "active": n_active, "context": f"uniform {ctx.min()}..{ctx.max()}",
+                   "mean_context": float(np.mean(ctx)), "max_context": max_ctx, "kv_block": 16,
+                   "sampling": {"temperature": T, "top_p": P}, "parallelism": "replicas only" if world > 1 else "1 GPU",
+                   "l2": "each step streams %.1f GB (weights + KV), far more than the 126 MB L2: no flush needed"
+                         % ((w_bytes + kv_bytes_mid) / 1e9)},
+        "tpot_ms": {"p50": srt[len(srt) // 2], "p99": srt[min(len(srt) - 1, int(0.99 * len(srt)))],
+                    "mean": ms_per_step},
+        "clocks": clk, "gpu_launches": launches * K,
+        "e2e": {"value": e2e_val, "unit": "tok/s", "ms_per_step": 1e3 * e2e_s / K,
+                "h2d_bytes_per_step": B * 9, "d2h_bytes_per_step": B * 4 + 4},
+        "roofline": roofline, "step_roofline": step_roof, "kernels": kernels, "cpu_baseline": cpu,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="corun", choices=["corun", "reference"])
+    ap.add_argument("--workload", default="qwen3_8b_b64", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_corun(args, rank, world)
+
+
+if __name__ == "__main__":
+    main()

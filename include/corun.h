@@ -170,6 +170,17 @@ int corun_debug_kv_write(corun_engine *e, int32_t slot, int32_t layer, int32_t p
  * corun_debug_kv_write), the pending token and the sampling state. */
 int corun_debug_adopt(corun_engine *e, int32_t slot, int32_t n_ctx, int32_t reserve_len, int32_t pending_token,
                       const corun_sampling *sampling, int32_t step);
+/* Bench set-up: fills cached positions [0, n_ctx) of every layer of an occupied slot
+ * with seeded N(0, std^2) values generated on the device and sets its context length. */
+int corun_debug_kv_fill(corun_engine *e, int32_t slot, int32_t n_ctx, float std, uint64_t seed);
+/* Times one kernel kind of the decode program in isolation, on the engine's stream,
+ * with CUDA events: `reps` launches rotating over the layers' weights (so that L2
+ * cannot hold them), after a short warm-up; *avg_ms = mean duration of one launch.
+ * kind: 0 QKV GEMM, 1 O GEMM, 2 gate-up GEMM, 3 down GEMM, 4 LM-head GEMM (+ partial
+ * fix-up), 5 attention (split + combine), 6 residual + RMSNorm, 7 RoPE + KV append,
+ * 8 SwiGLU, 9 sampler.  Uses the rows of the last decode step; overwrites
+ * intermediate buffers (not the cache beyond each active slot's next position). */
+int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *avg_ms);
 /* eager != 0: launch the decode kernels one by one instead of replaying the graph. */
 int corun_debug_set_eager(corun_engine *e, int32_t eager);
 /* Number of kernel launches in one decode iteration. */

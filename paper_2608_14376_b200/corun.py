@@ -20,7 +20,7 @@ EXPORTS = [
     "corun_init", "corun_prefill", "corun_decode_step", "corun_decode_enqueue", "corun_decode_wait",
     "corun_release", "corun_destroy", "corun_get_logits", "corun_force_token", "corun_context_len",
     "corun_free_blocks", "corun_debug_kv_read", "corun_debug_kv_write", "corun_debug_adopt",
-    "corun_debug_set_eager", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
+    "corun_debug_set_eager", "corun_debug_kv_fill", "corun_debug_time_kernel", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
     "corun_debug_sample", "corun_strerror", "corun_last_cuda_error",
 ]
 
@@ -80,6 +80,8 @@ def lib():
         L.corun_debug_kv_write.argtypes = [vp, i32, i32, i32, i32, vp, vp]
         L.corun_debug_adopt.argtypes = [vp, i32, i32, i32, i32, C.POINTER(Sampling), i32]
         L.corun_debug_set_eager.argtypes = [vp, i32]
+        L.corun_debug_kv_fill.argtypes = [vp, i32, i32, C.c_float, u64]
+        L.corun_debug_time_kernel.argtypes = [vp, i32, i32, C.POINTER(C.c_float)]
         L.corun_decode_launches.argtypes = [vp]
         L.corun_debug_gemm.argtypes = [vp, i32, i32, vp, i32, vp, vp]
         L.corun_debug_variate.argtypes = [u64, u64, C.POINTER(C.c_uint32)]
@@ -212,6 +214,17 @@ class Engine:
     def adopt(self, slot: int, n_ctx: int, reserve_len: int, pending: int, temperature=0.0, top_p=1.0, step=1):
         s = Sampling(temperature, top_p)
         _check(lib().corun_debug_adopt(self._h, slot, n_ctx, reserve_len, pending, C.byref(s), step), "adopt")
+
+    def kv_fill(self, slot: int, n_ctx: int, std: float, seed: int):
+        _check(lib().corun_debug_kv_fill(self._h, slot, n_ctx, std, seed & (2**64 - 1)), "kv_fill")
+
+    KERNEL_KINDS = ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head", "attention",
+                    "resid_norm", "rope_kv_append", "swiglu", "sampler")
+
+    def time_kernel(self, kind: int, reps: int) -> float:
+        ms = C.c_float(0.0)
+        _check(lib().corun_debug_time_kernel(self._h, kind, reps, C.byref(ms)), "time_kernel")
+        return float(ms.value)
 
     def set_eager(self, eager: bool):
         _check(lib().corun_debug_set_eager(self._h, 1 if eager else 0), "set_eager")

@@ -644,6 +644,68 @@ int corun_debug_adopt(corun_engine *e, int32_t slot, int32_t n_ctx, int32_t rese
   return CORUN_OK;
 }
 
+int corun_debug_kv_fill(corun_engine *e, int32_t slot, int32_t n_ctx, float std, uint64_t seed) {
+  if (!e || n_ctx < 0 || !(std >= 0.f)) return CORUN_EINVAL;
+  if (!slot_ok(e, slot) || !e->in_use[slot]) return CORUN_ESLOT;
+  if (n_ctx > e->reserve[slot]) return CORUN_EINVAL;
+  RC(sync_stream(e));
+  CK(launch_kv_fill(kv_layout(e), e->sh.n_layers, slot, n_ctx, std, seed, e->st));
+  CK(cudaMemcpyAsync(e->d_ctx + slot, &n_ctx, sizeof(int), cudaMemcpyHostToDevice, e->st));
+  CK(cudaStreamSynchronize(e->st));
+  e->ctx[slot] = n_ctx;
+  return CORUN_OK;
+}
+
+int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *avg_ms) {
+  if (!e || !avg_ms || reps < 1 || kind < 0 || kind > 9) return CORUN_EINVAL;
+  RC(sync_stream(e));
+  Program &P = e->dec;
+  const corun_shape &s = e->sh;
+  const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
+  const KvLayout kv = kv_layout(e);
+  cudaEvent_t a, b;
+  CK(cudaEventCreate(&a));
+  CK(cudaEventCreate(&b));
+  int rc = CORUN_OK;
+  for (int pass = 0; pass < 2 && rc == CORUN_OK; ++pass) {   // pass 0 warms up
+    const int n = pass == 0 ? (reps < 3 ? reps : 3) : reps;
+    cudaError_t ce = cudaEventRecord(a, e->st);
+    for (int i = 0; i < n && ce == cudaSuccess; ++i) {
+      const int l = i % s.n_layers;   // rotate over the layers so that L2 cannot hold the weights
+      GemmOut prev = P.p_down.out();
+      switch (kind) {
+        case 0: ce = gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st); break;
+        case 1: ce = gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st); break;
+        case 2: ce = gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st); break;
+        case 3: ce = gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st); break;
+        case 4: ce = gemm_launch(P.p_lm, nullptr, e->d_status, e->st);
+                if (ce == cudaSuccess) ce = gemm_fixup_launch(P.p_lm, e->st);
+                break;
+        case 5: ce = launch_attention(P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.part_acc, P.part_ml, P.ao_hi,
+                                      P.ao_lo, e->st); break;
+        case 6: ce = launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->attn_norm[l], s.rms_eps, P.xn_hi,
+                                       P.xn_lo, e->st); break;
+        case 7: ce = launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st); break;
+        case 8: ce = launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st); break;
+        case 9: {
+          SampleArgs sa{P.logits, s.vocab, P.do_sample, e->d_temp, e->d_top_p, e->d_seeds, e->d_step, nullptr, P.sampled};
+          ce = launch_sampler(sa, P.R, e->st);
+          break;
+        }
+      }
+    }
+    if (ce == cudaSuccess) ce = cudaEventRecord(b, e->st);
+    if (ce == cudaSuccess) ce = cudaEventSynchronize(b);
+    float ms = 0.f;
+    if (ce == cudaSuccess) ce = cudaEventElapsedTime(&ms, a, b);
+    if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; rc = CORUN_ECUDA; }
+    *avg_ms = ms / (float)n;
+  }
+  cudaEventDestroy(a);
+  cudaEventDestroy(b);
+  return rc;
+}
+
 int corun_debug_set_eager(corun_engine *e, int32_t eager) {
   if (!e) return CORUN_EINVAL;
   RC(sync_stream(e));

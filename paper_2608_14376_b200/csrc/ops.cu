@@ -632,6 +632,34 @@ __global__ void kv_copy_kernel(KvLayout kv, int layer, int slot, int pos0, int n
   }
 }
 
+__device__ __forceinline__ uint64_t mix64(uint64_t z) {
+  z += 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+// Synthetic cache contents for timing runs: position-hashed normals, one thread per (layer, token, pair).
+__global__ void kv_fill_kernel(KvLayout kv, int n_layers, int slot, int n, float std, uint64_t seed) {
+  const int KD = kv.n_kv * kv.hd;
+  const size_t per_layer = (size_t)n * KD;
+  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= per_layer * n_layers) return;
+  const int layer = (int)(idx / per_layer);
+  const size_t rem = idx - (size_t)layer * per_layer;
+  const int t = (int)(rem / KD), e = (int)(rem - (size_t)t * KD);
+  const int g = e / kv.hd, i = e - g * kv.hd;
+  const uint64_t h = mix64(seed ^ mix64(((uint64_t)slot << 48) ^ ((uint64_t)layer << 40) ^ ((uint64_t)t << 16) ^ (uint64_t)e));
+  const float u1 = ((float)(uint32_t)(h >> 40) + 1.0f) * (1.0f / 16777217.0f);
+  const float u2 = (float)(uint32_t)((h >> 8) & 0xFFFFFFu) * (1.0f / 16777216.0f);
+  const float rad = sqrtf(-2.0f * logf(u1)) * std;
+  const int blk = kv.block_table[(size_t)slot * kv.max_blocks + t / KV_BLOCK];
+  __half *base = kv.pool + (size_t)layer * kv.layer_stride + (size_t)blk * 2 * kv.n_kv * KV_BLOCK * kv.hd;
+  __half *kp = base + ((size_t)g * KV_BLOCK + t % KV_BLOCK) * kv.hd + i;
+  *kp = __float2half_rn(rad * cospif(2.0f * u2));
+  *(kp + (size_t)kv.n_kv * KV_BLOCK * kv.hd) = __float2half_rn(rad * sinpif(2.0f * u2));
+}
+
 template <int HD>
 cudaError_t launch_attn_hd(int group, dim3 grid, cudaStream_t st, const float *q, const Rows &rows, int nq,
                            const KvLayout &kv, int layer, int max_splits, float *pa, float *pm) {
@@ -711,6 +739,13 @@ cudaError_t launch_kv_copy(const KvLayout &kv, int layer, int slot, int pos0, in
   const size_t tot = (size_t)n * kv.n_kv * kv.hd;
   if (tot == 0) return cudaSuccess;
   kv_copy_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(kv, layer, slot, pos0, n, k, v, write);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_kv_fill(const KvLayout &kv, int n_layers, int slot, int n, float std, uint64_t seed, cudaStream_t st) {
+  const size_t tot = (size_t)n * kv.n_kv * kv.hd * n_layers;
+  if (tot == 0) return cudaSuccess;
+  kv_fill_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(kv, n_layers, slot, n, std, seed);
   return cudaGetLastError();
 }
 

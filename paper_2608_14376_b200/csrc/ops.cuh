@@ -67,6 +67,8 @@ cudaError_t launch_advance(const int *row_active, const int *sampled, int B, int
 // debug cache access (fp32 rows of n_kv*hd)
 cudaError_t launch_kv_copy(const KvLayout &kv, int layer, int slot, int pos0, int n, float *k, float *v, int write,
                            cudaStream_t st);
+// fills cached positions [0, n) of every layer of a slot with seeded N(0, std^2) values (bench set-up)
+cudaError_t launch_kv_fill(const KvLayout &kv, int n_layers, int slot, int n, float std, uint64_t seed, cudaStream_t st);
 cudaError_t launch_variate(uint64_t seed, uint64_t t, uint32_t *out, cudaStream_t st);
 
 }  // namespace corun
