@@ -42,7 +42,8 @@ typedef enum {
   CORUN_ECTX = -4,     /* an active slot would exceed its reserved length               */
   CORUN_ECUDA = -5,    /* a CUDA call failed (corun_last_cuda_error has the code)       */
   CORUN_ETIMEOUT = -6, /* a bounded device-side wait expired (device status word)       */
-  CORUN_ENOMEM = -7    /* device or host allocation failed                              */
+  CORUN_ENOMEM = -7,   /* device or host allocation failed                              */
+  CORUN_ELIMIT = -8    /* a size exceeds the fixed capacity of corun_gemm_static        */
 } corun_status;
 
 typedef struct corun_engine corun_engine; /* opaque, owned by the library */
@@ -195,6 +196,38 @@ int corun_debug_variate(uint64_t seed, uint64_t t, uint32_t *out_u24 /* host */)
 /* Runs the engine's sampler on host logits rows [n_rows, vocab] (copied to the device). */
 int corun_debug_sample(const float *logits, int32_t n_rows, int32_t vocab, const corun_sampling *sampling,
                        const uint32_t *u24, int32_t *out_tokens);
+
+/*
+ * corun_gemm_static -- corun_debug_gemm for callers that cannot allocate.
+ * (The paper has no counterpart; this is a service entry point of the library.)
+ *
+ * Same operation and argument meaning as corun_debug_gemm:
+ *   out[r, n] = sum_k W[n, k] * X[r, k],  W bf16 [N, K], X fp32 [R, K], out fp32 [R, N],
+ * all three in device memory owned by the caller.  It is meant for hosts that
+ * may not call cudaMalloc where they need the product: code running inside an
+ * arena that took all device memory at start-up, loops that cannot afford the
+ * device-wide synchronisation an allocation or a free implies, processes with
+ * a fixed memory budget.  Everything the kernel needs besides its inputs and
+ * output (split activations, per-CTA partial sums, partition tables, status
+ * word) lives in one array of about 3.3 MiB that is part of the library image:
+ * every GPU that loads the library holds it until the process exits.
+ *
+ * Limits (fixed by that array): R <= CORUN_STATIC_MAX_ROWS, K <= CORUN_STATIC_MAX_K
+ * (and K % 64 == 0), N <= CORUN_STATIC_MAX_N, at most 192 SMs.  Beyond them the
+ * call returns CORUN_ELIMIT and does nothing.  The call makes no cudaMalloc,
+ * cudaFree or any other allocating call.
+ *
+ * The first call on each device resolves the array's device address and sets a
+ * kernel attribute; make that first call outside any stream capture.  All calls
+ * share the one array, which keeps the previous call's contents (the call clears
+ * the parts that must start at zero): two calls that overlap on the GPU -- from
+ * two threads, or on two streams -- race on it.  The call is synchronous on
+ * `cuda_stream`.  Errors: EINVAL, ELIMIT, ECUDA, ETIMEOUT.
+ */
+#define CORUN_STATIC_MAX_ROWS 16
+#define CORUN_STATIC_MAX_K 4096
+#define CORUN_STATIC_MAX_N 8192
+int corun_gemm_static(const void *W, int32_t N, int32_t K, const float *X, int32_t R, float *out, void *cuda_stream);
 
 const char *corun_strerror(int status);
 int corun_last_cuda_error(void);

@@ -14,14 +14,14 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libcorun.so")
 
-OK, EINVAL, ESLOT, ENOSPACE, ECTX, ECUDA, ETIMEOUT, ENOMEM = 0, -1, -2, -3, -4, -5, -6, -7
+OK, EINVAL, ESLOT, ENOSPACE, ECTX, ECUDA, ETIMEOUT, ENOMEM, ELIMIT = 0, -1, -2, -3, -4, -5, -6, -7, -8
 
 EXPORTS = [
     "corun_init", "corun_prefill", "corun_decode_step", "corun_decode_enqueue", "corun_decode_wait",
     "corun_release", "corun_destroy", "corun_get_logits", "corun_force_token", "corun_context_len",
     "corun_free_blocks", "corun_debug_kv_read", "corun_debug_kv_write", "corun_debug_adopt",
     "corun_debug_set_eager", "corun_debug_kv_fill", "corun_debug_time_kernel", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
-    "corun_debug_sample", "corun_strerror", "corun_last_cuda_error",
+    "corun_debug_sample", "corun_gemm_static", "corun_strerror", "corun_last_cuda_error",
 ]
 
 
@@ -86,6 +86,7 @@ def lib():
         L.corun_debug_gemm.argtypes = [vp, i32, i32, vp, i32, vp, vp]
         L.corun_debug_variate.argtypes = [u64, u64, C.POINTER(C.c_uint32)]
         L.corun_debug_sample.argtypes = [vp, i32, i32, C.POINTER(Sampling), vp, vp]
+        L.corun_gemm_static.argtypes = [vp, i32, i32, vp, i32, vp, vp]
         L.corun_strerror.argtypes = [C.c_int]
         L.corun_strerror.restype = C.c_char_p
         L.corun_last_cuda_error.argtypes = []
@@ -242,6 +243,20 @@ def debug_gemm(W, X):
     out = torch.empty((R, N), dtype=torch.float32, device=X.device)
     torch.cuda.synchronize()
     _check(lib().corun_debug_gemm(W.data_ptr(), N, K, X.data_ptr(), R, out.data_ptr(), None), "corun_debug_gemm")
+    return out
+
+
+def gemm_static(W, X):
+    """Same product as ``debug_gemm`` through ``corun_gemm_static``: the library's own fixed scratch
+    array is used instead of fresh allocations (for callers that must not allocate device memory).
+    The output tensor is the caller's; rows <= 16, K <= 4096, N <= 8192."""
+    import torch
+
+    N, K = W.shape
+    R = X.shape[0]
+    out = torch.empty((R, N), dtype=torch.float32, device=X.device)
+    torch.cuda.synchronize()
+    _check(lib().corun_gemm_static(W.data_ptr(), N, K, X.data_ptr(), R, out.data_ptr(), None), "corun_gemm_static")
     return out
 
 

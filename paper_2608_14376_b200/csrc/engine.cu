@@ -278,6 +278,7 @@ const char *corun_strerror(int st) {
     case CORUN_ECUDA: return "CUDA error";
     case CORUN_ETIMEOUT: return "a bounded device-side wait expired";
     case CORUN_ENOMEM: return "out of memory";
+    case CORUN_ELIMIT: return "size exceeds the fixed capacity of corun_gemm_static";
     default: return "unknown status";
   }
 }

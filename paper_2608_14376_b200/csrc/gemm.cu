@@ -263,6 +263,10 @@ int gemm_plan_create(GemmPlan *p, const void *W, int N, int K, const void *Xhi, 
   return CORUN_OK;
 }
 
+cudaError_t gemm_prepare_kernel() {
+  return cudaFuncSetAttribute(gemm_streamk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 221 * 1024);
+}
+
 void gemm_plan_destroy(GemmPlan *p) {
   if (p->d_cta_start) cudaFree(p->d_cta_start);
   p->d_cta_start = nullptr;

@@ -75,6 +75,8 @@ void gemm_plan_destroy(GemmPlan *p);
 cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int *d_status, cudaStream_t st);
 // Encodes a tensor map for a bf16 [rows, K] row-major matrix with a [box_rows, 64] box, 128-byte swizzle.
 int gemm_encode_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows);
+// Opts the GEMM kernel into its dynamic shared-memory size (idempotent, allocates nothing).
+cudaError_t gemm_prepare_kernel();
 // direct[r, n] = gemm_load(r, n) for every tile that has partials (makes `direct` a plain matrix).
 cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st);
 

@@ -53,11 +53,11 @@ def test_argument_validation_needs_no_gpu(lib):
 
 def test_strerror_covers_every_status(lib):
     seen = set()
-    for st in range(0, -8, -1):
+    for st in range(0, -9, -1):
         s = lib.corun_strerror(st)
         assert s and s != b"unknown status"
         seen.add(s)
-    assert len(seen) == 8
+    assert len(seen) == 9
     assert lib.corun_strerror(-99) == b"unknown status"
 
 
