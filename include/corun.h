@@ -182,6 +182,12 @@ int corun_debug_kv_fill(corun_engine *e, int32_t slot, int32_t n_ctx, float std,
  * 8 SwiGLU, 9 sampler.  Uses the rows of the last decode step; overwrites
  * intermediate buffers (not the cache beyond each active slot's next position). */
 int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *avg_ms);
+/* Copies the first n floats of an intermediate buffer of the decode program to the host, as left by
+ * the last decode step: which = 0 rotated queries [B, nq*hd]; 1 attention split partials
+ * [B][nq][max_splits][hd]; 2 their (max, sum) pairs [B][nq][max_splits][2] (base-2 domain);
+ * 3 the residual stream [B, hidden]; 4 / 5 the attention output's bf16 hi / lo halves [BN, nq*hd] as raw
+ * memory (two bf16 per float); 6 the O-projection's direct output [B, hidden]; 7 the GEMM partial workspace. */
+int corun_debug_read(corun_engine *e, int32_t which, float *out, int64_t n);
 /* eager != 0: launch the decode kernels one by one instead of replaying the graph. */
 int corun_debug_set_eager(corun_engine *e, int32_t eager);
 /* Number of kernel launches in one decode iteration. */

@@ -20,7 +20,7 @@ EXPORTS = [
     "corun_init", "corun_prefill", "corun_decode_step", "corun_decode_enqueue", "corun_decode_wait",
     "corun_release", "corun_destroy", "corun_get_logits", "corun_force_token", "corun_context_len",
     "corun_free_blocks", "corun_debug_kv_read", "corun_debug_kv_write", "corun_debug_adopt",
-    "corun_debug_set_eager", "corun_debug_kv_fill", "corun_debug_time_kernel", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
+    "corun_debug_set_eager", "corun_debug_read", "corun_debug_kv_fill", "corun_debug_time_kernel", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
     "corun_debug_sample", "corun_gemm_static", "corun_strerror", "corun_last_cuda_error",
 ]
 
@@ -80,6 +80,7 @@ def lib():
         L.corun_debug_kv_write.argtypes = [vp, i32, i32, i32, i32, vp, vp]
         L.corun_debug_adopt.argtypes = [vp, i32, i32, i32, i32, C.POINTER(Sampling), i32]
         L.corun_debug_set_eager.argtypes = [vp, i32]
+        L.corun_debug_read.argtypes = [vp, i32, vp, i64]
         L.corun_debug_kv_fill.argtypes = [vp, i32, i32, C.c_float, u64]
         L.corun_debug_time_kernel.argtypes = [vp, i32, i32, C.POINTER(C.c_float)]
         L.corun_decode_launches.argtypes = [vp]
@@ -227,8 +228,13 @@ class Engine:
         _check(lib().corun_debug_time_kernel(self._h, kind, reps, C.byref(ms)), "time_kernel")
         return float(ms.value)
 
+    def debug_read(self, which: int, n: int) -> np.ndarray:
+        out = np.empty(n, np.float32)
+        _check(lib().corun_debug_read(self._h, which, out.ctypes.data, n), "corun_debug_read")
+        return out
+
     def set_eager(self, eager: bool):
-        _check(lib().corun_debug_set_eager(self._h, 1 if eager else 0), "set_eager")
+        _check(lib().corun_debug_set_eager(self._h, int(eager)), "set_eager")
 
     def decode_launches(self) -> int:
         return int(lib().corun_decode_launches(self._h))

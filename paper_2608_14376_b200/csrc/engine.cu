@@ -90,6 +90,7 @@ struct corun_engine {
   cudaGraph_t graph = nullptr;
   cudaGraphExec_t graph_exec = nullptr;
   bool eager = false;
+  int stop_after = -1;            // debug: eager decode stops after this many stages of layer 0
   int decode_launches = 0;
   std::vector<void *> allocs;
 };
@@ -176,21 +177,31 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
   const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
   const KvLayout kv = kv_layout(e);
   int n = 0;
+  int stage = 0;
+  const int stop = (e->eager && &P == &e->dec) ? e->stop_after : -1;
+#define STAGE(call)                                   \
+  do {                                                \
+    if (stop >= 0 && stage >= stop) return CORUN_OK;  \
+    CK(call);                                         \
+    ++stage;                                          \
+  } while (0)
   for (int l = 0; l < s.n_layers; ++l) {
     GemmOut prev = P.p_down.out();
-    CK(launch_resid_norm(P.h, s.hidden, e->embed, rows, l == 0 ? nullptr : &prev, e->attn_norm[l], s.rms_eps, P.xn_hi,
-                         P.xn_lo, e->st));
-    CK(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st));
-    CK(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st));
-    CK(launch_attention(P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo, e->st));
-    CK(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st));
+    STAGE(launch_resid_norm(P.h, s.hidden, e->embed, rows, l == 0 ? nullptr : &prev, e->attn_norm[l], s.rms_eps,
+                            P.xn_hi, P.xn_lo, e->st));
+    STAGE(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st));
+    STAGE(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st));
+    STAGE(launch_attention(P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo,
+                           e->st));
+    STAGE(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st));
     GemmOut o = P.p_o.out();
-    CK(launch_resid_norm(P.h, s.hidden, nullptr, rows, &o, e->mlp_norm[l], s.rms_eps, P.xn_hi, P.xn_lo, e->st));
-    CK(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st));
-    CK(launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st));
-    CK(gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st));
+    STAGE(launch_resid_norm(P.h, s.hidden, nullptr, rows, &o, e->mlp_norm[l], s.rms_eps, P.xn_hi, P.xn_lo, e->st));
+    STAGE(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st));
+    STAGE(launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st));
+    STAGE(gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st));
     n += 10;
   }
+#undef STAGE
   if (launches) *launches += n;
   return CORUN_OK;
 }
@@ -206,15 +217,17 @@ int enqueue_decode_body(corun_engine *e, int *launches) {
                          P.row_slot, P.do_sample, e->st));
   n += 1;
   RC(run_layers(e, P, &n));
-  const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
-  GemmOut prev = P.p_down.out();
-  CK(launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->final_norm, s.rms_eps, P.xn_hi, P.xn_lo, e->st));
-  CK(gemm_launch(P.p_lm, nullptr, e->d_status, e->st));
-  CK(gemm_fixup_launch(P.p_lm, e->st));
-  SampleArgs sa{P.logits, s.vocab, P.do_sample, e->d_temp, e->d_top_p, e->d_seeds, e->d_step, nullptr, P.sampled};
-  CK(launch_sampler(sa, P.R, e->st));
-  CK(launch_advance(P.row_active, P.sampled, e->B, e->d_ctx, e->d_step, e->d_pending, e->d_out_tokens, e->st));
-  n += 4 + (P.p_lm.n_split_tiles ? 1 : 0);
+  if (!(e->eager && e->stop_after >= 0)) {   // (debug) a truncated layer stack skips the tail too
+    const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
+    GemmOut prev = P.p_down.out();
+    CK(launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->final_norm, s.rms_eps, P.xn_hi, P.xn_lo, e->st));
+    CK(gemm_launch(P.p_lm, nullptr, e->d_status, e->st));
+    CK(gemm_fixup_launch(P.p_lm, e->st));
+    SampleArgs sa{P.logits, s.vocab, P.do_sample, e->d_temp, e->d_top_p, e->d_seeds, e->d_step, nullptr, P.sampled};
+    CK(launch_sampler(sa, P.R, e->st));
+    CK(launch_advance(P.row_active, P.sampled, e->B, e->d_ctx, e->d_step, e->d_pending, e->d_out_tokens, e->st));
+    n += 4 + (P.p_lm.n_split_tiles ? 1 : 0);
+  }
   CK(cudaMemcpyAsync(e->h_out_tokens, e->d_out_tokens, e->B * sizeof(int), cudaMemcpyDeviceToHost, e->st));
   CK(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, e->st));
   if (launches) *launches = n;
@@ -402,6 +415,9 @@ int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int3
   if ((rc = program_create(e, e->pre, e->chunk, true, false))) return fail(rc);
   if ((rc = program_create(e, e->lm1, 1, false, true))) return fail(rc);
 
+  // the allocations above were cleared and filled through the legacy stream, which the engine's
+  // stream does not wait for: drain the device once before the first launch
+  if (cudaDeviceSynchronize() != cudaSuccess) return fail(CORUN_ECUDA);
   // eager warm-up on an all-padding batch (also validates every launch), then capture
   if ((rc = enqueue_decode_body(e, &e->decode_launches))) return fail(rc);
   if (cudaStreamSynchronize(e->st) != cudaSuccess) return fail(CORUN_ECUDA);
@@ -490,7 +506,8 @@ int corun_prefill(corun_engine *e, int32_t slot, const int32_t *tokens, int32_t 
     CK(cudaStreamSynchronize(e->st));
   }
   int first = -1;
-  CK(cudaMemcpy(&first, e->d_pf_tok, sizeof(int), cudaMemcpyDeviceToHost));
+  CK(cudaMemcpyAsync(&first, e->d_pf_tok, sizeof(int), cudaMemcpyDeviceToHost, e->st));
+  CK(cudaStreamSynchronize(e->st));
   RC(check_status(e));
   RC(set_slot_state(e, slot, 1, n, 1, first, sampling->temperature, sampling->top_p));
   e->in_use[slot] = 1;
@@ -566,8 +583,9 @@ int corun_get_logits(corun_engine *e, int32_t slot, float *out) {
   if (!e || !out) return CORUN_EINVAL;
   if (!slot_ok(e, slot) || !e->in_use[slot]) return CORUN_ESLOT;
   RC(sync_stream(e));
-  CK(cudaMemcpy(out, e->dec.logits + (size_t)slot * e->sh.vocab, (size_t)e->sh.vocab * sizeof(float),
-                cudaMemcpyDeviceToHost));
+  CK(cudaMemcpyAsync(out, e->dec.logits + (size_t)slot * e->sh.vocab, (size_t)e->sh.vocab * sizeof(float),
+                     cudaMemcpyDeviceToHost, e->st));
+  CK(cudaStreamSynchronize(e->st));
   return CORUN_OK;
 }
 
@@ -575,7 +593,8 @@ int corun_force_token(corun_engine *e, int32_t slot, int32_t token) {
   if (!e || token < 0 || token >= e->sh.vocab) return CORUN_EINVAL;
   if (!slot_ok(e, slot) || !e->in_use[slot]) return CORUN_ESLOT;
   RC(sync_stream(e));
-  CK(cudaMemcpy(e->d_pending + slot, &token, sizeof(int), cudaMemcpyHostToDevice));
+  CK(cudaMemcpyAsync(e->d_pending + slot, &token, sizeof(int), cudaMemcpyHostToDevice, e->st));
+  CK(cudaStreamSynchronize(e->st));
   return CORUN_OK;
 }
 
@@ -600,23 +619,27 @@ static int kv_io(corun_engine *e, int slot, int layer, int pos0, int n, float *k
   if (cudaMalloc(&dv, elems * sizeof(float)) != cudaSuccess) { cudaFree(dk); return CORUN_ENOMEM; }
   int rc = CORUN_OK;
   cudaError_t ce = cudaSuccess;
+  // every copy is ordered on the engine's own stream: a host-synchronous cudaMemcpy from pageable
+  // memory may return before its DMA has landed, and the engine's stream does not wait for the
+  // legacy stream
   if (write) {
-    ce = cudaMemcpy(dk, k, elems * sizeof(float), cudaMemcpyHostToDevice);
-    if (ce == cudaSuccess) ce = cudaMemcpy(dv, v, elems * sizeof(float), cudaMemcpyHostToDevice);
+    ce = cudaMemcpyAsync(dk, k, elems * sizeof(float), cudaMemcpyHostToDevice, e->st);
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(dv, v, elems * sizeof(float), cudaMemcpyHostToDevice, e->st);
   }
   if (ce == cudaSuccess) ce = launch_kv_copy(kv_layout(e), layer, slot, pos0, n, dk, dv, write, e->st);
-  if (ce == cudaSuccess) ce = cudaStreamSynchronize(e->st);
   if (ce == cudaSuccess && !write) {
-    ce = cudaMemcpy(k, dk, elems * sizeof(float), cudaMemcpyDeviceToHost);
-    if (ce == cudaSuccess) ce = cudaMemcpy(v, dv, elems * sizeof(float), cudaMemcpyDeviceToHost);
+    ce = cudaMemcpyAsync(k, dk, elems * sizeof(float), cudaMemcpyDeviceToHost, e->st);
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(v, dv, elems * sizeof(float), cudaMemcpyDeviceToHost, e->st);
   }
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(e->st);
   if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; rc = CORUN_ECUDA; }
   cudaFree(dk);
   cudaFree(dv);
   if (rc == CORUN_OK && write && pos0 + n > e->ctx[slot]) {
     e->ctx[slot] = pos0 + n;
     const int c = e->ctx[slot];
-    CK(cudaMemcpy(e->d_ctx + slot, &c, sizeof(int), cudaMemcpyHostToDevice));
+    CK(cudaMemcpyAsync(e->d_ctx + slot, &c, sizeof(int), cudaMemcpyHostToDevice, e->st));
+    CK(cudaStreamSynchronize(e->st));
   }
   return rc;
 }
@@ -707,10 +730,36 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
   return rc;
 }
 
+int corun_debug_read(corun_engine *e, int32_t which, float *out, int64_t n) {
+  if (!e || !out || n < 0) return CORUN_EINVAL;
+  RC(sync_stream(e));
+  Program &P = e->dec;
+  const corun_shape &s = e->sh;
+  const size_t QD = (size_t)s.n_q_heads * s.head_dim;
+  const float *src = nullptr;
+  size_t have = 0;
+  switch (which) {
+    case 0: src = P.q; have = (size_t)P.R * QD; break;
+    case 1: src = P.part_acc; have = (size_t)P.R * s.n_q_heads * e->max_splits * s.head_dim; break;
+    case 2: src = P.part_ml; have = (size_t)P.R * s.n_q_heads * e->max_splits * 2; break;
+    case 3: src = P.h; have = (size_t)P.R * s.hidden; break;
+    case 4: src = (const float *)P.ao_hi; have = (size_t)P.BN * QD / 2; break;
+    case 5: src = (const float *)P.ao_lo; have = (size_t)P.BN * QD / 2; break;
+    case 6: src = P.o_out; have = (size_t)P.R * s.hidden; break;
+    case 7: src = P.ws; have = gemm_ws_floats(e->num_sms, P.BN); break;
+    default: return CORUN_EINVAL;
+  }
+  if ((size_t)n > have) return CORUN_EINVAL;
+  CK(cudaMemcpyAsync(out, src, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, e->st));
+  CK(cudaStreamSynchronize(e->st));
+  return CORUN_OK;
+}
+
 int corun_debug_set_eager(corun_engine *e, int32_t eager) {
   if (!e) return CORUN_EINVAL;
   RC(sync_stream(e));
   e->eager = eager != 0;
+  e->stop_after = eager > 1 ? eager - 2 : -1;   // eager = 2 + k: stop the layer stack after k stages
   return CORUN_OK;
 }
 
@@ -732,7 +781,8 @@ int corun_debug_gemm(const void *W, int32_t N, int32_t K, const float *X, int32_
   if ((rc = dmalloc(keep, &hi, (size_t)BN * K)) == 0 && (rc = dmalloc(keep, &lo, (size_t)BN * K)) == 0 &&
       (rc = dmalloc(keep, &ws, gemm_ws_floats(sms, BN))) == 0 && (rc = dmalloc(keep, &status, 1)) == 0 &&
       (rc = gemm_plan_create(&p, W, N, K, hi, lo, R, BN, out, ws, sms)) == 0) {
-    cudaError_t ce = launch_split(X, R, K, hi, lo, st);
+    cudaError_t ce = cudaDeviceSynchronize();   // allocations were cleared through the legacy stream
+    if (ce == cudaSuccess) ce = launch_split(X, R, K, hi, lo, st);
     if (ce == cudaSuccess) ce = gemm_launch(p, nullptr, status, st);
     if (ce == cudaSuccess) ce = gemm_fixup_launch(p, st);
     if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);

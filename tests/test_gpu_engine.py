@@ -256,3 +256,27 @@ def test_adopted_slot_with_written_cache_matches_oracle(orc, tiny, engine):
     active = np.zeros(B, np.uint8); active[6] = 1
     engine.decode_step(active, np.zeros(B, np.uint64))
     assert np.abs(engine.logits(6) - want).max() <= TOL
+
+
+@pytest.mark.parametrize("n_ctx", [255, 256, 257, 700, 1023])
+def test_multi_split_attention_matches_oracle(orc, tiny, n_ctx):
+    """Contexts spanning several 256-token splits and ragged tails (synthetic cache rows)."""
+    from paper_2608_14376_b200 import corun
+
+    sh = tiny.sh
+    e = corun.Engine(sh, tiny.w_t, B, 1040)
+    cache = tiny.oracle.new_cache(n_ctx + 2)
+    e.adopt(2, 0, n_ctx + 2, pending=33)
+    for layer in range(sh.n_layers):
+        k, v = synth.synthetic_kv(n_ctx, sh.kv_dim, 0.5, seed=7 * n_ctx + layer)
+        cache[0][layer, :n_ctx] = k
+        cache[1][layer, :n_ctx] = v
+        e.kv_write(2, layer, 0, k, v)
+    want = tiny.oracle.forward([33], n_ctx, cache)
+    active = np.zeros(B, np.uint8); active[2] = 1
+    e.decode_step(active, np.zeros(B, np.uint64))
+    err = float(np.abs(e.logits(2) - want).max())
+    k_back, v_back = e.kv_read(2, 1, 0, n_ctx)
+    np.testing.assert_array_equal(k_back, cache[0][1, :n_ctx])
+    e.close()
+    assert err <= TOL, err

@@ -1,0 +1,126 @@
+"""Full-size parity at the Qwen3-8B shape (36 layers, hidden 4096, 32 q / 8 kv heads, head_dim 128,
+FFN 12288, vocab 151936; B = 64), in the launch configuration bench.py times: sampled outputs the
+oracle can compute one by one.  (i) real isolated prefill + teacher-forced decode steps for two
+requests; (ii) long contexts via seeded synthetic cache rows (the oracle cannot afford to prefill
+them), one decode step, run among co-tenants; (iii) bitwise slot / co-tenant invariance."""
+import numpy as np
+import pytest
+
+from paper_2608_14376_b200 import synth
+from tests.helpers import oracle_model, top2_gap
+
+pytestmark = pytest.mark.gpu
+
+B, MAX_CTX = 64, 4352
+TOL, GAP = 3e-2, 0.1
+T, P = 0.7, 0.95
+
+
+@pytest.fixture(scope="module")
+def qwen(orc):
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    if torch.cuda.get_device_properties(0).total_memory < 100e9:
+        pytest.skip("needs a large-memory GPU")
+    from paper_2608_14376_b200 import corun
+
+    sh = synth.QWEN3_8B
+    w_t = synth.make_weights_torch(sh, seed=0, device="cuda")
+    w_np = synth.weights_torch_to_numpy(w_t)
+    model = oracle_model(orc, sh, w_np)
+    eng = corun.Engine(sh, w_t, B, MAX_CTX, kv_pool_blocks=6000)
+    yield sh, model, eng
+    eng.close()
+
+
+def _compare(eng, slot, ref_logits, stats):
+    lg = eng.logits(slot)
+    stats["worst"] = max(stats["worst"], float(np.abs(lg - ref_logits).max()))
+    return lg
+
+
+def test_prefill_and_decode_parity_with_sampling(orc, qwen):
+    sh, model, eng = qwen
+    prompts = synth.make_prompts(sh.vocab, [48, 150], seed=5)
+    slots = [9, 41]
+    stats = {"worst": 0.0}
+    reqs = []
+    for i, (s, p) in enumerate(zip(slots, prompts)):
+        seed = synth.request_seed(i)
+        r = orc.Request(model, p, seed, T, P, max_T=len(p) + 8)
+        want = r.prefill()
+        got = eng.prefill(s, p, len(p) + 8, T, P, seed)
+        lg = _compare(eng, s, r.logits, stats)
+        # the engine's sample is S applied to its own logits with the same variate
+        assert got == orc.sample(lg, T, P, orc.variate_u24(seed, 0))[0]
+        if top2_gap(r.logits) > GAP:
+            assert int(np.argmax(lg)) == int(np.argmax(r.logits))
+        eng.force_token(s, want)
+        reqs.append(r)
+    active = np.zeros(B, np.uint8); active[slots] = 1
+    seeds = np.zeros(B, np.uint64)
+    for i, s in enumerate(slots):
+        seeds[s] = synth.request_seed(i)
+    for step in range(3):
+        toks = eng.decode_step(active, seeds)
+        for i, s in enumerate(slots):
+            r = reqs[i]
+            want = r.decode()
+            lg = _compare(eng, s, r.logits, stats)
+            assert toks[s] == orc.sample(lg, T, P, orc.variate_u24(int(seeds[s]), step + 1))[0]
+            if top2_gap(r.logits) > GAP:
+                assert int(np.argmax(lg)) == int(np.argmax(r.logits))
+            eng.force_token(s, want)
+    for s in slots:
+        eng.release(s)
+    print("qwen prefill+decode: max |delta logit| = %.4g" % stats["worst"])
+    assert stats["worst"] <= TOL, stats["worst"]
+
+
+def _adopt_with_cache(eng, model, sh, slot, n_ctx, seed, pending):
+    cache = model.new_cache(n_ctx + 2)
+    eng.adopt(slot, 0, n_ctx + 2, pending=pending, temperature=T, top_p=P, step=1)
+    for layer in range(sh.n_layers):
+        k, v = synth.synthetic_kv(n_ctx, sh.kv_dim, 1.28, seed=seed * 100 + layer)
+        cache[0][layer, :n_ctx] = k
+        cache[1][layer, :n_ctx] = v
+        eng.kv_write(slot, layer, 0, k, v)
+    return cache
+
+
+def test_long_context_decode_parity_and_invariance(orc, qwen):
+    sh, model, eng = qwen
+    # contexts spanning 1..16 splits with ragged tails, run together in one padded batch
+    cases = [(3, 3001, 11), (20, 700, 12), (57, 255, 13), (33, 4000, 14)]
+    caches = {}
+    for slot, n_ctx, seed in cases:
+        caches[slot] = _adopt_with_cache(eng, model, sh, slot, n_ctx, seed, pending=1000 + slot)
+    active = np.zeros(B, np.uint8)
+    seeds = np.zeros(B, np.uint64)
+    for slot, _, seed in cases:
+        active[slot] = 1; seeds[slot] = seed
+    toks = eng.decode_step(active, seeds)
+    worst = 0.0
+    rows = {}
+    for slot, n_ctx, seed in cases:
+        ref = model.forward([1000 + slot], n_ctx, caches[slot])
+        lg = eng.logits(slot)
+        rows[slot] = lg.tobytes()
+        worst = max(worst, float(np.abs(lg - ref).max()))
+        assert toks[slot] == orc.sample(lg, T, P, orc.variate_u24(seed, 1))[0]
+        if top2_gap(ref) > GAP:
+            assert int(np.argmax(lg)) == int(np.argmax(ref))
+    print("qwen long-context decode: max |delta logit| = %.4g" % worst)
+    assert worst <= TOL, worst
+    for slot, _, _ in cases:
+        eng.release(slot)
+    # invariance: the 700-token request alone in another slot gives the same logit bytes
+    slot2 = 62
+    _adopt_with_cache(eng, model, sh, slot2, 700, 12, pending=1000 + 20)
+    active[:] = 0; active[slot2] = 1
+    seeds[:] = 0; seeds[slot2] = 12
+    toks2 = eng.decode_step(active, seeds)
+    assert eng.logits(slot2).tobytes() == rows[20]
+    assert toks2[slot2] == toks[20]
+    eng.release(slot2)
