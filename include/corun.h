@@ -215,7 +215,7 @@ int corun_debug_sample(const float *logits, int32_t n_rows, int32_t vocab, const
  * device-wide synchronisation an allocation or a free implies, processes with
  * a fixed memory budget.  Everything the kernel needs besides its inputs and
  * output (split activations, per-CTA partial sums, partition tables, status
- * word) lives in one array of about 3.3 MiB that is part of the library image:
+ * word) lives in one array of about 6.3 MiB that is part of the library image:
  * every GPU that loads the library holds it until the process exits.
  *
  * Limits (fixed by that array): R <= CORUN_STATIC_MAX_ROWS, K <= CORUN_STATIC_MAX_K

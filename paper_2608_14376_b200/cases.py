@@ -1,0 +1,107 @@
+"""Small single-kernel cases for profiling (a few GB on the device, inputs larger than L2).
+
+    python -m paper_2608_14376_b200.cases gemm      [--N 24576 --K 4096 --R 64 --reps 3]
+    python -m paper_2608_14376_b200.cases kernels   [--layers 4 --B 64 --active-frac 0.625 --vocab 32768]
+    python -m paper_2608_14376_b200.cases attention [--layers 2 --B 64 --active 40 --ctx-lo 512 --ctx-hi 4096 --reps 2]
+
+``gemm`` runs the stand-alone decode GEMM on seeded inputs; ``attention`` builds a Qwen3-8B-shaped
+engine with few layers, fills the cache of the active slots on the device and runs decode steps.
+Each prints the CUDA-event time per launch, for comparison with what a profiler reports.
+"""
+from __future__ import annotations
+
+import argparse
+
+import numpy as np
+
+
+def case_gemm(a):
+    import torch
+
+    from . import corun
+
+    g = torch.Generator(device="cuda").manual_seed(0)
+    W = (torch.randn((a.N, a.K), generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+    X = torch.randn((a.R, a.K), generator=g, device="cuda")
+    out = None
+    for _ in range(a.reps):
+        out = corun.debug_gemm(W, X)
+    ref = (X[:4].double() @ W.double().T).float()
+    print("gemm N=%d K=%d R=%d: max |err| on 4 rows = %.3g" % (a.N, a.K, a.R, (out[:4] - ref).abs().max().item()))
+
+
+def case_attention(a):
+    import torch
+
+    from . import corun, synth
+
+    sh = synth.ModelShape(a.layers, 4096, 32, 8, 128, 12288, 4096, 1e-6, 1e6)
+    w = synth.make_weights_torch(sh, seed=0, device="cuda")
+    ctx = synth.uniform_lengths(a.ctx_lo, a.ctx_hi, a.active, seed=2)
+    slots = synth.pick_slots(a.B, a.active, seed=7)
+    max_ctx = -(-(int(ctx.max()) + a.reps + 32) // 256) * 256
+    eng = corun.Engine(sh, w, a.B, max_ctx)
+    for i, (s, c) in enumerate(zip(slots, ctx)):
+        eng.adopt(int(s), 0, int(c) + a.reps + 16, pending=1 + i, temperature=0.7, top_p=0.95)
+        eng.kv_fill(int(s), int(c), 1.28, seed=100 + i)
+    active = np.zeros(a.B, np.uint8); active[slots] = 1
+    seeds = np.arange(a.B, dtype=np.uint64) + 1000
+    for _ in range(a.reps):
+        eng.decode_step(active, seeds)
+    kv_bytes = sum((int(c) + a.reps) * 4096 for c in ctx)
+    ms = eng.time_kernel(5, 2 * a.layers)
+    print("attention: %d active, mean ctx %.0f, %.1f MB of KV per layer, %.1f us per launch pair (%.0f GB/s)"
+          % (a.active, float(np.mean(ctx)), kv_bytes / 1e6, ms * 1e3, kv_bytes / ms / 1e6))
+    eng.close()
+
+
+def case_kernels(a):
+    """Per-kernel CUDA-event times of the decode program at the Qwen3-8B layer shape (few layers)."""
+    import torch
+
+    from . import corun, synth
+
+    sh = synth.ModelShape(a.layers, 4096, 32, 8, 128, 12288, a.vocab, 1e-6, 1e6)
+    w = synth.make_weights_torch(sh, seed=0, device="cuda")
+    n_act = max(1, int(round(a.B * a.active_frac)))
+    ctx = synth.uniform_lengths(a.ctx_lo, a.ctx_hi, n_act, seed=2)
+    slots = synth.pick_slots(a.B, n_act, seed=7)
+    max_ctx = -(-(int(ctx.max()) + 64) // 256) * 256
+    eng = corun.Engine(sh, w, a.B, max_ctx)
+    for i, (s, c) in enumerate(zip(slots, ctx)):
+        eng.adopt(int(s), 0, int(c) + 32, pending=1 + i, temperature=0.7, top_p=0.95)
+        eng.kv_fill(int(s), int(c), 1.28, seed=100 + i)
+    active = np.zeros(a.B, np.uint8); active[slots] = 1
+    seeds = np.arange(a.B, dtype=np.uint64) + 1000
+    for _ in range(2):
+        eng.decode_step(active, seeds)
+    nbytes = {"gemm_qkv": 2 * sh.qkv_dim * sh.hidden, "gemm_o": 2 * sh.hidden * sh.q_dim,
+              "gemm_gate_up": 4 * sh.ffn * sh.hidden, "gemm_down": 2 * sh.hidden * sh.ffn,
+              "gemm_lm_head": 2 * sh.vocab * sh.hidden, "attention": sum((int(c) + 3) * 4096 for c in ctx)}
+    for i, name in enumerate(eng.KERNEL_KINDS):
+        ms = eng.time_kernel(i, 4 * a.layers if i not in (4, 9) else 6)
+        extra = "  %7.0f GB/s" % (nbytes[name] / ms / 1e6) if name in nbytes else ""
+        print("%-16s %8.2f us%s" % (name, ms * 1e3, extra))
+    eng.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    sub = ap.add_subparsers(dest="case", required=True)
+    g = sub.add_parser("gemm")
+    g.add_argument("--N", type=int, default=24576); g.add_argument("--K", type=int, default=4096)
+    g.add_argument("--R", type=int, default=64); g.add_argument("--reps", type=int, default=3)
+    t = sub.add_parser("attention")
+    t.add_argument("--layers", type=int, default=2); t.add_argument("--B", type=int, default=64)
+    t.add_argument("--active", type=int, default=40); t.add_argument("--ctx-lo", type=int, default=512)
+    t.add_argument("--ctx-hi", type=int, default=4096); t.add_argument("--reps", type=int, default=2)
+    k = sub.add_parser("kernels")
+    k.add_argument("--layers", type=int, default=4); k.add_argument("--B", type=int, default=64)
+    k.add_argument("--active-frac", type=float, default=0.625); k.add_argument("--ctx-lo", type=int, default=512)
+    k.add_argument("--ctx-hi", type=int, default=4096); k.add_argument("--vocab", type=int, default=32768)
+    a = ap.parse_args()
+    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels}[a.case](a)
+
+
+if __name__ == "__main__":
+    main()

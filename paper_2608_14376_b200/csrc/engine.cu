@@ -61,6 +61,7 @@ struct corun_engine {
   const bf16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
   std::vector<const bf16 *> attn_norm, mlp_norm;
   std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_down;
+  CUtensorMap tm_kv;
   // KV
   __half *kv_pool = nullptr;
   size_t layer_stride = 0;
@@ -168,7 +169,8 @@ void program_destroy(Program &P) {
 }
 
 KvLayout kv_layout(const corun_engine *e) {
-  return KvLayout{e->kv_pool, e->d_block_table, e->max_blocks, e->sh.n_kv_heads, e->sh.head_dim, e->layer_stride};
+  return KvLayout{e->kv_pool, e->d_block_table, e->max_blocks, e->sh.n_kv_heads, e->sh.head_dim, e->layer_stride,
+                  (long long)e->pool_blocks};
 }
 
 // Enqueues embed -> all layers (ends with the last down GEMM).  Counts launches.
@@ -191,8 +193,8 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
                             P.xn_hi, P.xn_lo, e->st));
     STAGE(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st));
     STAGE(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st));
-    STAGE(launch_attention(P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo,
-                           e->st));
+    STAGE(launch_attention(e->tm_kv, P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.part_acc, P.part_ml, P.ao_hi,
+                           P.ao_lo, e->d_status, e->st));
     STAGE(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st));
     GemmOut o = P.p_o.out();
     STAGE(launch_resid_norm(P.h, s.hidden, nullptr, rows, &o, e->mlp_norm[l], s.rms_eps, P.xn_hi, P.xn_lo, e->st));
@@ -362,16 +364,23 @@ int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int3
     e->attn_norm.push_back((const bf16 *)w->attn_norm[l]);
     e->mlp_norm.push_back((const bf16 *)w->mlp_norm[l]);
     int rc;
-    if ((rc = gemm_encode_map(&e->tm_qkv[l], w->wqkv[l], QD + 2 * KD, H, GEMM_TILE_M))) return fail(rc);
-    if ((rc = gemm_encode_map(&e->tm_o[l], w->wo[l], H, QD, GEMM_TILE_M))) return fail(rc);
-    if ((rc = gemm_encode_map(&e->tm_gu[l], w->wgate_up[l], 2 * F, H, GEMM_TILE_M))) return fail(rc);
-    if ((rc = gemm_encode_map(&e->tm_down[l], w->wdown[l], H, F, GEMM_TILE_M))) return fail(rc);
+    if ((rc = gemm_encode_map(&e->tm_qkv[l], w->wqkv[l], QD + 2 * KD, H, GEMM_TILE_N))) return fail(rc);
+    if ((rc = gemm_encode_map(&e->tm_o[l], w->wo[l], H, QD, GEMM_TILE_N))) return fail(rc);
+    if ((rc = gemm_encode_map(&e->tm_gu[l], w->wgate_up[l], 2 * F, H, GEMM_TILE_N))) return fail(rc);
+    if ((rc = gemm_encode_map(&e->tm_down[l], w->wdown[l], H, F, GEMM_TILE_N))) return fail(rc);
   }
 
   auto &A = e->allocs;
   int rc;
   e->layer_stride = (size_t)e->pool_blocks * 2 * s.n_kv_heads * KV_BLOCK * s.head_dim;
-  if ((rc = dmalloc(A, &e->kv_pool, e->layer_stride * s.n_layers, false))) return fail(rc);
+  // zero-filled: masked positions of a page are multiplied by zero weights, so they must be finite
+  if ((rc = dmalloc(A, &e->kv_pool, e->layer_stride * s.n_layers, true))) return fail(rc);
+  {
+    const unsigned long long rows = (unsigned long long)s.n_layers * e->pool_blocks * 2 * s.n_kv_heads * KV_BLOCK;
+    if (rows >= (1ull << 31)) return fail(CORUN_EINVAL);
+    if ((rc = tma_encode_2d(&e->tm_kv, e->kv_pool, 1, rows, s.head_dim, KV_BLOCK, 64))) return fail(rc);
+    if (attention_prepare() != cudaSuccess) return fail(CORUN_ECUDA);
+  }
   if ((rc = dmalloc(A, &e->d_block_table, (size_t)B * e->max_blocks))) return fail(rc);
   if ((rc = dmalloc(A, &e->d_in_use, B)) || (rc = dmalloc(A, &e->d_ctx, B)) || (rc = dmalloc(A, &e->d_step, B)) ||
       (rc = dmalloc(A, &e->d_pending, B)) || (rc = dmalloc(A, &e->d_temp, B)) || (rc = dmalloc(A, &e->d_top_p, B)) ||
@@ -486,7 +495,7 @@ int corun_prefill(corun_engine *e, int32_t slot, const int32_t *tokens, int32_t 
     Program &L = e->lm1;
     GemmOut prev = P.p_down.out();
     prev.direct += (size_t)last_row * prev.N;
-    prev.ws += (size_t)last_row * 128;
+    prev.ws += (size_t)last_row * GEMM_TILE_N;
     const Rows one{P.row_token + last_row, P.row_pos + last_row, P.row_active + last_row, P.row_slot + last_row, 1};
     CK(launch_resid_norm(P.h + (size_t)last_row * s.hidden, s.hidden, nullptr, one, &prev, e->final_norm, s.rms_eps,
                          L.xn_hi, L.xn_lo, e->st));
@@ -705,8 +714,8 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
         case 4: ce = gemm_launch(P.p_lm, nullptr, e->d_status, e->st);
                 if (ce == cudaSuccess) ce = gemm_fixup_launch(P.p_lm, e->st);
                 break;
-        case 5: ce = launch_attention(P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.part_acc, P.part_ml, P.ao_hi,
-                                      P.ao_lo, e->st); break;
+        case 5: ce = launch_attention(e->tm_kv, P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.part_acc, P.part_ml,
+                                      P.ao_hi, P.ao_lo, e->d_status, e->st); break;
         case 6: ce = launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->attn_norm[l], s.rms_eps, P.xn_hi,
                                        P.xn_lo, e->st); break;
         case 7: ce = launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st); break;

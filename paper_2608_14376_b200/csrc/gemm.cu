@@ -3,6 +3,7 @@
 
 #include <cudaTypedefs.h>
 
+#include <cstdlib>
 #include <vector>
 
 #include "../../include/corun.h"
@@ -15,9 +16,18 @@ int g_last_cuda_error = 0;
 namespace {
 
 constexpr int MAX_STAGES = 8;
+constexpr uint32_t W_TILE_BYTES = GEMM_TILE_N * GEMM_BLOCK_K * 2;          // 32 KiB
+constexpr uint32_t A_BLOCK_BYTES = GEMM_ROW_BLOCK * GEMM_BLOCK_K * 2;      // 16 KiB: what one MMA reads of A
 
 // Role loops walk the CTA's flat k-block range [k0, k1) segment by segment; a
 // segment is the part of the range that falls into one weight tile.
+//
+// Operands: A = activations (hi or lo), 128 rows per MMA, K-major, 128-byte
+// swizzle; B = 256 weight rows, same layout; D = fp32 [128 rows x 256 weight
+// rows] in TMEM (lane = activation row, column = weight row), one accumulator
+// per block of 128 activation rows.  When fewer than 128 rows are loaded the
+// MMA still reads 128 rows of shared memory; the extra accumulator lanes hold
+// meaningless values that are never read back.
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmHi,
                     const __grid_constant__ CUtensorMap tmLo, float *__restrict__ direct, float *__restrict__ ws,
@@ -34,9 +44,9 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t w_bytes = GEMM_TILE_M * GEMM_BLOCK_K * 2;          // 16 KiB
   const uint32_t x_bytes = (uint32_t)BN * GEMM_BLOCK_K * 2;         // BN * 128 B
-  const uint32_t stage_bytes = w_bytes + 2 * x_bytes;
+  const uint32_t stage_bytes = W_TILE_BYTES + 2 * x_bytes;
+  const int n_rb = (BN + GEMM_ROW_BLOCK - 1) / GEMM_ROW_BLOCK;      // blocks of 128 activation rows
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -79,9 +89,9 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const uint32_t fb = smem_u32(&full_bar[s]);
         const uint32_t dst = tiles_base + (uint32_t)s * stage_bytes;
         mbar_arrive_expect_tx(fb, stage_bytes);
-        tma_load_2d(dst, &tmW, kb * GEMM_BLOCK_K, tile * GEMM_TILE_M, fb, pol_w);
-        tma_load_2d(dst + w_bytes, &tmHi, kb * GEMM_BLOCK_K, 0, fb, pol_x);
-        tma_load_2d(dst + w_bytes + x_bytes, &tmLo, kb * GEMM_BLOCK_K, 0, fb, pol_x);
+        tma_load_2d(dst, &tmW, kb * GEMM_BLOCK_K, tile * GEMM_TILE_N, fb, pol_w);
+        tma_load_2d(dst + W_TILE_BYTES, &tmHi, kb * GEMM_BLOCK_K, 0, fb, pol_x);
+        tma_load_2d(dst + W_TILE_BYTES + x_bytes, &tmLo, kb * GEMM_BLOCK_K, 0, fb, pol_x);
       }
     }
   } else if (warp == 1) {
@@ -98,28 +108,30 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           const uint32_t ph = (uint32_t)(it / stages) & 1u;
           if (!mbar_wait(smem_u32(&full_bar[s]), ph, abort_p)) { fail = DEV_TIMEOUT_MMA; break; }
           tc_fence_after();
-          const uint32_t a_addr = tiles_base + (uint32_t)s * stage_bytes;
-          const uint64_t a_desc = umma_desc_sw128(a_addr);
-          const uint64_t hi_desc = umma_desc_sw128(a_addr + w_bytes);
-          const uint64_t lo_desc = umma_desc_sw128(a_addr + w_bytes + x_bytes);
+          const uint32_t w_addr = tiles_base + (uint32_t)s * stage_bytes;
+          const uint64_t w_desc = umma_desc_sw128(w_addr);
+          for (int rb = 0; rb < n_rb; ++rb) {
+            const uint64_t hi_desc = umma_desc_sw128(w_addr + W_TILE_BYTES + (uint32_t)rb * A_BLOCK_BYTES);
+            const uint64_t lo_desc = umma_desc_sw128(w_addr + W_TILE_BYTES + x_bytes + (uint32_t)rb * A_BLOCK_BYTES);
+            const uint32_t d_tmem = tmem_base + (uint32_t)rb * GEMM_TILE_N;
 #pragma unroll
-          for (int k = 0; k < GEMM_BLOCK_K / 16; ++k) {
-            // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in 16-byte units
-            const uint64_t adv = (uint64_t)(k * 2);
-            umma_bf16(tmem_base, a_desc + adv, hi_desc + adv, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
-            umma_bf16(tmem_base, a_desc + adv, lo_desc + adv, idesc, 1u);
+            for (int k = 0; k < GEMM_BLOCK_K / 16; ++k) {
+              // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in 16-byte units
+              const uint64_t adv = (uint64_t)(k * 2);
+              umma_bf16(d_tmem, hi_desc + adv, w_desc + adv, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
+              umma_bf16(d_tmem, lo_desc + adv, w_desc + adv, idesc, 1u);
+            }
           }
           umma_commit(smem_u32(&empty_bar[s]));   // frees the stage once these MMAs have read it
         }
         if (fail) break;
-        umma_commit(smem_u32(&tmem_full_bar));    // accumulator of this segment is complete
+        umma_commit(smem_u32(&tmem_full_bar));    // accumulators of this segment are complete
         g += kb_end - kb_begin;
       }
     }
   } else {
     // ---------------- epilogue: TMEM -> registers -> global ----------------
     const int lane_base = (warp & 3) * 32;          // the TMEM lanes this warp may read
-    const int row = lane_base + lane;               // row of the weight tile = output feature
     int seg = 0;
     for (int g = k0; g < k1; ++seg) {
       const int tile = g / KB, kb_begin = g - tile * KB;
@@ -129,30 +141,33 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) { fail = DEV_TIMEOUT_EPILOGUE; break; }
       tc_fence_after();
-      const int n = tile * GEMM_TILE_M + row;
-      float *dst;
-      size_t stride;
-      int rows_out;
-      bool row_ok;
-      if (whole) {
-        dst = direct + n;
-        stride = (size_t)N;
-        rows_out = R;
-        row_ok = n < N;
-      } else {
-        dst = ws + ((size_t)(cta * 2 + (seg == 0 ? 0 : 1)) * BN) * 128 + row;
-        stride = 128;
-        rows_out = BN;
-        row_ok = true;
-      }
-      for (int c0 = 0; c0 < BN; c0 += 16) {
-        uint32_t v[16];
-        tmem_ld16(tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)c0, v);
-        tmem_ld_wait();
-        if (row_ok) {
+      const int n0 = tile * GEMM_TILE_N;
+      for (int rb = 0; rb < n_rb; ++rb) {
+        const int row_base = rb * GEMM_ROW_BLOCK + lane_base;
+        const int rows_valid = whole ? R : BN;      // partials keep the padded row count
+        if (row_base >= rows_valid) continue;        // warp-uniform: nothing of this warp's lanes is needed
+        const int row = row_base + lane;
+        const bool row_ok = row < rows_valid;
+        float *dst = whole ? direct + (size_t)row * N + n0
+                           : ws + ((size_t)(cta * 2 + (seg == 0 ? 0 : 1)) * BN + row) * GEMM_TILE_N;
+        const bool vec_ok = whole ? ((N & 3) == 0) : true;
+        for (int c0 = 0; c0 < GEMM_TILE_N; c0 += 16) {
+          if (whole && n0 + c0 >= N) break;          // columns beyond the matrix (last tile)
+          uint32_t v[16];
+          tmem_ld16(tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)(rb * GEMM_TILE_N + c0), v);
+          tmem_ld_wait();
+          if (!row_ok) continue;
+          if (vec_ok && (!whole || n0 + c0 + 16 <= N)) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j)
-            if (c0 + j < rows_out) dst[(size_t)(c0 + j) * stride] = __uint_as_float(v[j]);
+            for (int j = 0; j < 16; j += 4)
+              *reinterpret_cast<float4 *>(dst + c0 + j) =
+                  make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
+                              __uint_as_float(v[j + 3]));
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              if (n0 + c0 + j < N) dst[c0 + j] = __uint_as_float(v[j]);
+          }
         }
       }
       tc_fence_before();
@@ -172,11 +187,10 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   if (warp == 1) tmem_dealloc(tmem_base, (uint32_t)tmem_cols);
 }
 
-__global__ void gemm_fixup_kernel(GemmOut g, float *direct, const int *split_tiles, int R) {
-  const int t = split_tiles[blockIdx.x];
-  const int n = t * 128 + threadIdx.x;
-  if (n >= g.N) return;
-  for (int r = 0; r < R; ++r) direct[(size_t)r * g.N + n] = gemm_load(g, r, n);
+__global__ void __launch_bounds__(GEMM_TILE_N) gemm_fixup_kernel(GemmOut g, float *direct, const int *split_tiles) {
+  const int t = split_tiles[blockIdx.x], r = blockIdx.y;
+  const int n = t * GEMM_TILE_N + threadIdx.x;
+  if (n < g.N) direct[(size_t)r * g.N + n] = gemm_load(g, r, n);
 }
 
 PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
@@ -193,73 +207,99 @@ PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
 
 }  // namespace
 
-int gemm_encode_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows) {
+int tma_encode_2d(CUtensorMap *m, const void *base, int is_fp16, unsigned long long rows, int cols, int box_rows,
+                  int box_cols) {
   auto enc = get_encode();
   if (!enc) { g_last_cuda_error = 99999; return CORUN_ECUDA; }
-  if (((uintptr_t)base & 15u) || (K % GEMM_BLOCK_K) || box_rows > 256 || box_rows < 1) return CORUN_EINVAL;
-  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-  cuuint32_t box[2] = {(cuuint32_t)GEMM_BLOCK_K, (cuuint32_t)box_rows};
+  if (((uintptr_t)base & 15u) || (cols % 8) || box_cols * 2 != 128 || box_rows > 256 || box_rows < 1) return CORUN_EINVAL;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = enc(m, is_fp16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                   const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) g_last_cuda_error = 100000 + (int)r;
   return r == CUDA_SUCCESS ? CORUN_OK : CORUN_ECUDA;
 }
 
-int gemm_plan_create(GemmPlan *p, const void *W, int N, int K, const void *Xhi, const void *Xlo, int R, int BN,
-                     float *direct, float *ws, int num_sms) {
+int gemm_encode_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows) {
+  if (K % GEMM_BLOCK_K) return CORUN_EINVAL;
+  return tma_encode_2d(m, base, 0, (unsigned long long)rows, K, box_rows, GEMM_BLOCK_K);
+}
+
+int gemm_plan_fill(GemmPlan *p, const void *W, int N, int K, const void *Xhi, const void *Xlo, int R, int BN,
+                   float *direct, float *ws, int num_sms, int *tab, int tab_cap, int *tab_ints) {
   if (N <= 0 || K <= 0 || K % GEMM_BLOCK_K || BN % 16 || BN < 16 || BN > 256 || R < 1 || R > BN) return CORUN_EINVAL;
   p->N = N; p->K = K; p->R = R; p->BN = BN;
-  p->n_tiles = (N + GEMM_TILE_M - 1) / GEMM_TILE_M;
+  p->n_tiles = (N + GEMM_TILE_N - 1) / GEMM_TILE_N;
   p->KB = K / GEMM_BLOCK_K;
   const long long total = (long long)p->n_tiles * p->KB;
   p->grid = (int)(total < num_sms ? total : num_sms);
   if (total * (long long)p->grid >= (1ll << 31)) return CORUN_EINVAL;
-  const size_t stage = (size_t)GEMM_TILE_M * GEMM_BLOCK_K * 2 + 2 * (size_t)BN * GEMM_BLOCK_K * 2;
-  int stages = (int)((220 * 1024 - 1024) / stage);
+  const size_t stage = (size_t)W_TILE_BYTES + 2 * (size_t)BN * GEMM_BLOCK_K * 2;
+  // the MMA always reads 128 activation rows: leave that much readable behind the last stage
+  int stages = (int)((220 * 1024 - 1024 - A_BLOCK_BYTES) / stage);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
+  if (const char *ev = getenv("CORUN_GEMM_STAGES")) {   // experiments only: shallower ring
+    const int v = atoi(ev);
+    if (v >= 2 && v < stages) stages = v;
+  }
   if (stages < 2) return CORUN_EINVAL;
   p->stages = stages;
-  p->smem_bytes = stage * stages + 1024;
-  p->tmem_cols = 32;
-  while (p->tmem_cols < BN) p->tmem_cols *= 2;
+  p->smem_bytes = stage * stages + A_BLOCK_BYTES + 1024;
+  p->tmem_cols = BN > GEMM_ROW_BLOCK ? 512 : 256;
   // kind::f16 instruction descriptor: D fp32 (bits 4-5 = 1), A and B bf16 (bits 7-9, 10-12 = 1),
   // both K-major (bits 15, 16 = 0), N >> 3 at bits 17-22, M >> 4 at bits 24-28.
-  p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(GEMM_TILE_M >> 4) << 24);
+  p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GEMM_TILE_N >> 3) << 17) |
+             ((uint32_t)(GEMM_ROW_BLOCK >> 4) << 24);
   p->direct = direct;
   p->ws = ws;
   int rc;
-  if ((rc = gemm_encode_map(&p->tmW, W, N, K, GEMM_TILE_M)) != 0) return rc;
+  if ((rc = gemm_encode_map(&p->tmW, W, N, K, GEMM_TILE_N)) != 0) return rc;
   if ((rc = gemm_encode_map(&p->tmHi, Xhi, BN, K, BN)) != 0) return rc;
   if ((rc = gemm_encode_map(&p->tmLo, Xlo, BN, K, BN)) != 0) return rc;
 
-  std::vector<int> tab((size_t)p->grid + 1 + 3 * (size_t)p->n_tiles);
-  int *cs = tab.data(), *cb = cs + p->grid + 1, *ce = cb + p->n_tiles, *sp = ce + p->n_tiles;
+  const int n_ints = p->grid + 1 + 3 * p->n_tiles;
+  if (n_ints > tab_cap) return CORUN_ELIMIT;
+  int *cs = tab, *cb = cs + p->grid + 1, *ce = cb + p->n_tiles, *sp = ce + p->n_tiles;
   for (int c = 0; c <= p->grid; ++c) cs[c] = (int)((long long)c * total / p->grid);
   p->n_split_tiles = 0;
   for (int t = 0, c = 0; t < p->n_tiles; ++t) {
     const int first = t * p->KB, last = first + p->KB - 1;
     while (cs[c + 1] <= first) ++c;
-    cb[t] = c;
+    cb[t] = 2 * c + (cs[c] < first ? 1 : 0);   // a CTA that began before the tile wrote its second slot
     int d = c;
     while (cs[d + 1] <= last) ++d;
     ce[t] = d;
-    if (cb[t] != ce[t]) sp[p->n_split_tiles++] = t;
+    if (c != d) sp[p->n_split_tiles++] = t;
   }
-  if (cudaMalloc(&p->d_cta_start, tab.size() * sizeof(int)) != cudaSuccess) return CORUN_ENOMEM;
-  cudaError_t me = cudaMemcpy(p->d_cta_start, tab.data(), tab.size() * sizeof(int), cudaMemcpyHostToDevice);
-  if (me != cudaSuccess) { g_last_cuda_error = (int)me; return CORUN_ECUDA; }
-  p->d_tile_cbeg = p->d_cta_start + p->grid + 1;
-  p->d_tile_cend = p->d_tile_cbeg + p->n_tiles;
+  *tab_ints = n_ints;
+  return CORUN_OK;
+}
+
+void gemm_plan_bind_tables(GemmPlan *p, int *d_tab) {
+  p->d_cta_start = d_tab;
+  p->d_tile_first = d_tab + p->grid + 1;
+  p->d_tile_cend = p->d_tile_first + p->n_tiles;
   p->d_split_tiles = p->d_tile_cend + p->n_tiles;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t ae = cudaFuncSetAttribute(gemm_streamk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 221 * 1024);
-    if (ae != cudaSuccess) { g_last_cuda_error = (int)ae; return CORUN_ECUDA; }
-    attr_set = true;
-  }
+}
+
+int gemm_plan_create(GemmPlan *p, const void *W, int N, int K, const void *Xhi, const void *Xlo, int R, int BN,
+                     float *direct, float *ws, int num_sms) {
+  if (N <= 0 || K <= 0 || K % GEMM_BLOCK_K) return CORUN_EINVAL;
+  const int n_tiles = (N + GEMM_TILE_N - 1) / GEMM_TILE_N;
+  std::vector<int> tab((size_t)num_sms + 1 + 3 * (size_t)n_tiles);
+  int n_ints = 0;
+  int rc = gemm_plan_fill(p, W, N, K, Xhi, Xlo, R, BN, direct, ws, num_sms, tab.data(), (int)tab.size(), &n_ints);
+  if (rc != CORUN_OK) return rc;
+  int *d_tab = nullptr;
+  if (cudaMalloc(&d_tab, (size_t)n_ints * sizeof(int)) != cudaSuccess) return CORUN_ENOMEM;
+  cudaError_t me = cudaMemcpy(d_tab, tab.data(), (size_t)n_ints * sizeof(int), cudaMemcpyHostToDevice);
+  if (me != cudaSuccess) { g_last_cuda_error = (int)me; cudaFree(d_tab); return CORUN_ECUDA; }
+  gemm_plan_bind_tables(p, d_tab);
+  cudaError_t ae = gemm_prepare_kernel();
+  if (ae != cudaSuccess) { g_last_cuda_error = (int)ae; return CORUN_ECUDA; }
   return CORUN_OK;
 }
 
@@ -281,7 +321,7 @@ cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int 
 
 cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st) {
   if (p.n_split_tiles == 0) return cudaSuccess;
-  gemm_fixup_kernel<<<p.n_split_tiles, 128, 0, st>>>(p.out(), p.direct, p.d_split_tiles, p.R);
+  gemm_fixup_kernel<<<dim3(p.n_split_tiles, p.R), GEMM_TILE_N, 0, st>>>(p.out(), p.direct, p.d_split_tiles);
   return cudaGetLastError();
 }
 

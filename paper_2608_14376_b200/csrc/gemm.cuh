@@ -1,8 +1,9 @@
 // Decode / prefill-chunk GEMM  out[r, n] = sum_k W[n, k] * (Xhi[r, k] + Xlo[r, k]).
 //
-// The weight matrix is the 128-row MMA operand, the (padded) rows of
-// activations are the N operand, so one fixed tiling serves every row count
-// up to 256.  The flat space of (weight tile, 64-wide k-block) pairs is cut
+// The rows of activations (up to 256, in blocks of 128) are the M operand of
+// the MMA and a tile of 256 weight rows is its N operand, so every tcgen05.mma
+// is a full-size 128 x 256 x 16 instruction whatever the row count; one fixed
+// tiling serves every row count.  The flat space of (weight tile, 64-wide k-block) pairs is cut
 // into one contiguous, equally sized range per CTA; the cut depends on the
 // shape (N, K) and the grid only, never on which rows are occupied.  A tile
 // whose k-blocks all belong to one CTA is written straight to `direct`;
@@ -18,30 +19,53 @@ namespace corun {
 // Last CUDA runtime error (cudaError_t), or 100000 + CUresult for driver calls.
 extern int g_last_cuda_error;
 
-constexpr int GEMM_TILE_M = 128;   // weight rows per tile
+constexpr int GEMM_TILE_N = 256;   // weight rows per tile (the MMA's N)
+constexpr int GEMM_ROW_BLOCK = 128; // activation rows per MMA (the MMA's M)
 constexpr int GEMM_BLOCK_K = 64;   // bf16 elements per k-block (= one 128-byte swizzle row)
 constexpr int GEMM_THREADS = 192;  // warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 epilogue
 
 // What a consumer kernel needs to read a GEMM result.
 struct GemmOut {
   const float *direct;   // [rows, N]; valid for tiles owned by one CTA
-  const float *ws;       // [(cta*2 + slot), BN, 128] partials
-  const int *cta_start;  // [grid + 1] first flat k-block of each CTA
-  const int *tile_cbeg;  // [n_tiles] first CTA touching the tile
-  const int *tile_cend;  // [n_tiles] last CTA touching the tile
+  const float *ws;       // [(cta*2 + slot), BN, 256] partials
+  const int *tile_first; // [n_tiles] 2 * (first CTA touching the tile) + (the slot that CTA used for it)
+  const int *tile_cend;  // [n_tiles] last CTA touching the tile (every later CTA used slot 0)
   int N, KB, BN;
 };
 
 // Value (r, n) of a GEMM result, partials added in ascending CTA order.
 __device__ __forceinline__ float gemm_load(const GemmOut &g, int r, int n) {
-  const int t = n >> 7, row = n & 127;
-  const int c0 = g.tile_cbeg[t], c1 = g.tile_cend[t];
+  const int t = n >> 8, col = n & 255;
+  const int f = g.tile_first[t], c0 = f >> 1, c1 = g.tile_cend[t];
   if (c0 == c1) return g.direct[(size_t)r * g.N + n];
+  const float *p = g.ws + ((size_t)r) * GEMM_TILE_N + col;
+  const size_t cta_stride = (size_t)2 * g.BN * GEMM_TILE_N;
   float acc = 0.f;
-  const int first_kb = t * g.KB;
-  for (int c = c0; c <= c1; ++c) {
-    const int slot = (g.cta_start[c] >= first_kb) ? 0 : 1;
-    acc += g.ws[((size_t)(c * 2 + slot) * g.BN + r) * 128 + row];
+  acc += p[(size_t)f * g.BN * GEMM_TILE_N];
+  for (int c = c0 + 1; c <= c1; ++c) acc += p[(size_t)c * cta_stride];
+  return acc;
+}
+
+// Four consecutive values (n % 4 == 0, N % 4 == 0) with the same summation order as gemm_load.
+// Loads are issued four partials at a time; an absent partial contributes +0.0f.
+__device__ __forceinline__ float4 gemm_load4(const GemmOut &g, int r, int n) {
+  const int t = n >> 8, col = n & 255;
+  const int f = g.tile_first[t], c0 = f >> 1, c1 = g.tile_cend[t];
+  if (c0 == c1) return *reinterpret_cast<const float4 *>(g.direct + (size_t)r * g.N + n);
+  const float *p = g.ws + ((size_t)r) * GEMM_TILE_N + col;
+  const size_t cta_stride = (size_t)2 * g.BN * GEMM_TILE_N;
+  float4 acc = *reinterpret_cast<const float4 *>(p + (size_t)f * g.BN * GEMM_TILE_N);
+  acc.x += 0.f; acc.y += 0.f; acc.z += 0.f; acc.w += 0.f;   // same rounding path as 0 + first partial
+  for (int c = c0 + 1; c <= c1; c += 4) {
+    float4 v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      v[j] = (c + j <= c1) ? *reinterpret_cast<const float4 *>(p + (size_t)(c + j) * cta_stride)
+                           : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      acc.x += v[j].x; acc.y += v[j].y; acc.z += v[j].z; acc.w += v[j].w;
+    }
   }
   return acc;
 }
@@ -55,14 +79,14 @@ struct GemmPlan {
   size_t smem_bytes = 0;
   float *direct = nullptr;           // not owned
   float *ws = nullptr;               // not owned
-  int *d_cta_start = nullptr, *d_tile_cbeg = nullptr, *d_tile_cend = nullptr;  // owned (one allocation)
+  int *d_cta_start = nullptr, *d_tile_first = nullptr, *d_tile_cend = nullptr;  // owned (one allocation)
   int *d_split_tiles = nullptr;      // tiles with partials (same allocation)
   int n_split_tiles = 0;
-  GemmOut out() const { return GemmOut{direct, ws, d_cta_start, d_tile_cbeg, d_tile_cend, N, KB, BN}; }
+  GemmOut out() const { return GemmOut{direct, ws, d_tile_first, d_tile_cend, N, KB, BN}; }
 };
 
 // Workspace floats needed by any plan with this grid and BN.
-inline size_t gemm_ws_floats(int grid, int BN) { return (size_t)grid * 2 * BN * 128; }
+inline size_t gemm_ws_floats(int grid, int BN) { return (size_t)grid * 2 * BN * GEMM_TILE_N; }
 
 // Builds the plan: tensor maps for W [N, K] bf16 and the split activations
 // Xhi / Xlo [BN, K] bf16 (row pitch K), the CTA partition and its tables.
@@ -70,6 +94,13 @@ inline size_t gemm_ws_floats(int grid, int BN) { return (size_t)grid * 2 * BN * 
 int gemm_plan_create(GemmPlan *p, const void *W, int N, int K, const void *Xhi, const void *Xlo, int R, int BN,
                      float *direct, float *ws, int num_sms);
 void gemm_plan_destroy(GemmPlan *p);
+// The allocation-free half of gemm_plan_create: fills every host-side field and tensor map of the
+// plan and writes the partition tables (cta_start, tile_first, tile_cend, split_tiles) to `tab`
+// (capacity tab_cap ints; *tab_ints = ints used).  gemm_plan_bind_tables points the plan at a device
+// copy of those tables.
+int gemm_plan_fill(GemmPlan *p, const void *W, int N, int K, const void *Xhi, const void *Xlo, int R, int BN,
+                   float *direct, float *ws, int num_sms, int *tab, int tab_cap, int *tab_ints);
+void gemm_plan_bind_tables(GemmPlan *p, int *d_tab);
 // Enqueues the GEMM.  `W` may override the weight matrix of the plan (same
 // shape) by passing a different tensor map.
 cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int *d_status, cudaStream_t st);
@@ -77,6 +108,9 @@ cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int 
 int gemm_encode_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows);
 // Opts the GEMM kernel into its dynamic shared-memory size (idempotent, allocates nothing).
 cudaError_t gemm_prepare_kernel();
+// Tensor map for a 16-bit [rows, cols] row-major matrix with a [box_rows, 64] box (128 bytes wide), 128-byte swizzle.
+int tma_encode_2d(CUtensorMap *m, const void *base, int is_fp16, unsigned long long rows, int cols, int box_rows,
+                  int box_cols);
 // direct[r, n] = gemm_load(r, n) for every tile that has partials (makes `direct` a plain matrix).
 cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st);
 

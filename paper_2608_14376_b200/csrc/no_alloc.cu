@@ -24,20 +24,20 @@ constexpr int NA_MAX_K = CORUN_STATIC_MAX_K;
 constexpr int NA_MAX_N = CORUN_STATIC_MAX_N;
 constexpr int NA_MAX_GRID = 192;                 // CTAs (= SMs) the partial-sum area is sized for
 constexpr int NA_BN = 16;                        // padded row count of the MMA's N operand
-constexpr int NA_MAX_TILES = NA_MAX_N / GEMM_TILE_M;
+constexpr int NA_MAX_TILES = NA_MAX_N / GEMM_TILE_N;
 
 constexpr size_t NA_OFF_HI = 0;
 constexpr size_t NA_HILO_BYTES = (size_t)NA_BN * NA_MAX_K * sizeof(__nv_bfloat16);
 constexpr size_t NA_OFF_LO = NA_OFF_HI + NA_HILO_BYTES;
 constexpr size_t NA_OFF_WS = NA_OFF_LO + NA_HILO_BYTES;
-constexpr size_t NA_WS_BYTES = (size_t)NA_MAX_GRID * 2 * NA_BN * 128 * sizeof(float);
+constexpr size_t NA_WS_BYTES = (size_t)NA_MAX_GRID * 2 * NA_BN * GEMM_TILE_N * sizeof(float);
 constexpr size_t NA_OFF_TAB = NA_OFF_WS + NA_WS_BYTES;
 constexpr int NA_TAB_INTS = NA_MAX_GRID + 1 + 3 * NA_MAX_TILES;
 constexpr size_t NA_TAB_BYTES = ((size_t)NA_TAB_INTS * sizeof(int) + 255) / 256 * 256;
 constexpr size_t NA_OFF_STATUS = NA_OFF_TAB + NA_TAB_BYTES;
 constexpr size_t NA_BYTES = NA_OFF_STATUS + 256;
 
-// The scratch itself (about 3.3 MiB per GPU).  In host code this name is only
+// The scratch itself (about 6.3 MiB per GPU).  In host code this name is only
 // a handle for cudaGetSymbolAddress; kernels get the address obtained there.
 static __device__ __align__(256) unsigned char g_static_scratch[NA_BYTES];
 
@@ -87,41 +87,12 @@ extern "C" int corun_gemm_static(const void *W, int32_t N, int32_t K, const floa
   int *tab = (int *)(base + NA_OFF_TAB);
   int *status = (int *)(base + NA_OFF_STATUS);
 
-  // the same static partition as the allocating path: equal contiguous k-block ranges per CTA
+  // the same static partition as the allocating path, with its tables built on the stack
   GemmPlan p;
-  p.N = N; p.K = K; p.R = R; p.BN = NA_BN;
-  p.n_tiles = (N + GEMM_TILE_M - 1) / GEMM_TILE_M;
-  p.KB = K / GEMM_BLOCK_K;
-  const long long total = (long long)p.n_tiles * p.KB;
-  p.grid = (int)(total < sms ? total : sms);
-  const size_t stage = (size_t)GEMM_TILE_M * GEMM_BLOCK_K * 2 + 2 * (size_t)NA_BN * GEMM_BLOCK_K * 2;
-  p.stages = 8;
-  p.smem_bytes = stage * p.stages + 1024;
-  p.tmem_cols = 32;
-  p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NA_BN >> 3) << 17) | ((uint32_t)(GEMM_TILE_M >> 4) << 24);
-  p.direct = out;
-  p.ws = ws;
   int host_tab[NA_TAB_INTS];
-  int *cs = host_tab, *cb = cs + p.grid + 1, *cend = cb + p.n_tiles, *sp = cend + p.n_tiles;
-  for (int c = 0; c <= p.grid; ++c) cs[c] = (int)((long long)c * total / p.grid);
-  p.n_split_tiles = 0;
-  for (int t = 0, c = 0; t < p.n_tiles; ++t) {
-    const int first = t * p.KB, last = first + p.KB - 1;
-    while (cs[c + 1] <= first) ++c;
-    cb[t] = c;
-    int d = c;
-    while (cs[d + 1] <= last) ++d;
-    cend[t] = d;
-    if (cb[t] != cend[t]) sp[p.n_split_tiles++] = t;
-  }
-  const int n_ints = p.grid + 1 + 3 * p.n_tiles;
-  p.d_cta_start = tab;
-  p.d_tile_cbeg = tab + p.grid + 1;
-  p.d_tile_cend = p.d_tile_cbeg + p.n_tiles;
-  p.d_split_tiles = p.d_tile_cend + p.n_tiles;
-  if ((rc = gemm_encode_map(&p.tmW, W, N, K, GEMM_TILE_M)) != 0) return rc;
-  if ((rc = gemm_encode_map(&p.tmHi, hi, NA_BN, K, NA_BN)) != 0) return rc;
-  if ((rc = gemm_encode_map(&p.tmLo, lo, NA_BN, K, NA_BN)) != 0) return rc;
+  int n_ints = 0;
+  if ((rc = gemm_plan_fill(&p, W, N, K, hi, lo, R, NA_BN, out, ws, sms, host_tab, NA_TAB_INTS, &n_ints)) != 0) return rc;
+  gemm_plan_bind_tables(&p, tab);
 
   // The array keeps whatever the previous call left: clear what must start at
   // zero (padding rows of the split activations, the status word).

@@ -15,293 +15,97 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &hi, __nv_bflo
   lo = __float2bfloat16_rn(x - __bfloat162float(hi));
 }
 
-// Sum over the block in a fixed order: xor-butterfly inside each warp, then
-// the warp totals added in ascending warp order by every thread.
-template <int NWARPS>
-__device__ __forceinline__ float block_sum_fixed(float v, float *scratch /*[NWARPS]*/) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  __syncthreads();
-  if (lane == 0) scratch[warp] = v;
-  __syncthreads();
-  float t = 0.f;
-#pragma unroll
-  for (int w = 0; w < NWARPS; ++w) t += scratch[w];
-  return t;
+// ---------------------------------------------------------------- residual + RMSNorm
+constexpr int NORM_MAX_THREADS = 1024;
+
+__device__ __forceinline__ void store_split4(float4 y, __nv_bfloat16 *hi, __nv_bfloat16 *lo) {
+  __nv_bfloat16 a[4], b[4];
+  split_bf16(y.x, a[0], b[0]);
+  split_bf16(y.y, a[1], b[1]);
+  split_bf16(y.z, a[2], b[2]);
+  split_bf16(y.w, a[3], b[3]);
+  *reinterpret_cast<uint2 *>(hi) = *reinterpret_cast<const uint2 *>(a);
+  *reinterpret_cast<uint2 *>(lo) = *reinterpret_cast<const uint2 *>(b);
 }
 
-// ---------------------------------------------------------------- residual + RMSNorm
-constexpr int NORM_THREADS = 256;
-
-__global__ void __launch_bounds__(NORM_THREADS)
+// One CTA per row, one float4 per thread and pass (H % 4 == 0).  Sum of squares: thread-serial over
+// the thread's elements (ascending), xor-butterfly in the warp, warp totals in ascending order.
+__global__ void __launch_bounds__(NORM_MAX_THREADS)
 resid_norm_kernel(float *__restrict__ h, int H, const __nv_bfloat16 *__restrict__ embed, Rows rows, GemmOut prev,
                   int first, const __nv_bfloat16 *__restrict__ gains, float eps, __nv_bfloat16 *__restrict__ out_hi,
                   __nv_bfloat16 *__restrict__ out_lo) {
-  __shared__ float scratch[NORM_THREADS / 32];
+  __shared__ float scratch[NORM_MAX_THREADS / 32];
   const int r = blockIdx.x;
   float *hr = h + (size_t)r * H;
   float ss = 0.f;
   if (first) {
     const __nv_bfloat16 *e = embed + (size_t)rows.token[r] * H;
-    for (int i = threadIdx.x; i < H; i += NORM_THREADS) {
-      const float x = __bfloat162float(e[i]);
-      hr[i] = x;
-      ss = fmaf(x, x, ss);
+    for (int i = threadIdx.x * 4; i < H; i += blockDim.x * 4) {
+      const uint2 raw = *reinterpret_cast<const uint2 *>(e + i);
+      const __nv_bfloat162 *b2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+      const float2 lo2 = __bfloat1622float2(b2[0]), hi2 = __bfloat1622float2(b2[1]);
+      const float4 x = make_float4(lo2.x, lo2.y, hi2.x, hi2.y);
+      *reinterpret_cast<float4 *>(hr + i) = x;
+      ss = fmaf(x.x, x.x, ss); ss = fmaf(x.y, x.y, ss); ss = fmaf(x.z, x.z, ss); ss = fmaf(x.w, x.w, ss);
     }
   } else {
-    for (int i = threadIdx.x; i < H; i += NORM_THREADS) {
-      const float x = hr[i] + gemm_load(prev, r, i);
-      hr[i] = x;
-      ss = fmaf(x, x, ss);
+    for (int i = threadIdx.x * 4; i < H; i += blockDim.x * 4) {
+      const float4 d = gemm_load4(prev, r, i);
+      float4 x = *reinterpret_cast<const float4 *>(hr + i);
+      x.x += d.x; x.y += d.y; x.z += d.z; x.w += d.w;
+      *reinterpret_cast<float4 *>(hr + i) = x;
+      ss = fmaf(x.x, x.x, ss); ss = fmaf(x.y, x.y, ss); ss = fmaf(x.z, x.z, ss); ss = fmaf(x.w, x.w, ss);
     }
   }
-  const float tot = block_sum_fixed<NORM_THREADS / 32>(ss, scratch);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  if (lane == 0) scratch[warp] = ss;
+  __syncthreads();
+  float tot = 0.f;
+  for (int w = 0; w < nwarps; ++w) tot += scratch[w];
   const float inv = rsqrtf(tot / (float)H + eps);
-  for (int i = threadIdx.x; i < H; i += NORM_THREADS) {
-    const float y = hr[i] * inv * __bfloat162float(gains[i]);
-    __nv_bfloat16 a, b;
-    split_bf16(y, a, b);
-    out_hi[(size_t)r * H + i] = a;
-    out_lo[(size_t)r * H + i] = b;
+  for (int i = threadIdx.x * 4; i < H; i += blockDim.x * 4) {
+    const float4 x = *reinterpret_cast<const float4 *>(hr + i);   // written by this same thread above
+    const uint2 raw = *reinterpret_cast<const uint2 *>(gains + i);
+    const __nv_bfloat162 *g2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+    const float2 ga = __bfloat1622float2(g2[0]), gb = __bfloat1622float2(g2[1]);
+    const float4 y = make_float4(x.x * inv * ga.x, x.y * inv * ga.y, x.z * inv * gb.x, x.w * inv * gb.y);
+    store_split4(y, out_hi + (size_t)r * H + i, out_lo + (size_t)r * H + i);
   }
 }
 
 // ---------------------------------------------------------------- RoPE + KV append
-__global__ void __launch_bounds__(256)
+// One CTA per (head, row): heads 0..nq-1 are q, nq..nq+nkv-1 are k, the rest are v; hd/2 threads.
+__global__ void __launch_bounds__(64)
 qkv_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, int nq, KvLayout kv, int layer,
                 float *__restrict__ q_out) {
-  const int r = blockIdx.x;
+  const int head = blockIdx.x, r = blockIdx.y, i = threadIdx.x;
   const int hd = kv.hd, half = hd >> 1, nkv = kv.n_kv;
   const int pos = rows.pos[r];
-  const int active = rows.active[r];
-  const float2 *cs = rope_tab + (size_t)pos * half;
-  const int QD = nq * hd, KD = nkv * hd;
-  __half *kdst = nullptr, *vdst = nullptr;
-  if (active) {
-    const int blk = kv.block_table[(size_t)rows.slot[r] * kv.max_blocks + pos / KV_BLOCK];
-    __half *base = kv.pool + (size_t)layer * kv.layer_stride + (size_t)blk * 2 * nkv * KV_BLOCK * hd;
-    kdst = base + (size_t)(pos % KV_BLOCK) * hd;                       // + g * 16 * hd per head
-    vdst = base + (size_t)nkv * KV_BLOCK * hd + (size_t)(pos % KV_BLOCK) * hd;
-  }
-  // rotated pairs of q and k
-  const int n_pairs = (nq + nkv) * half;
-  for (int idx = threadIdx.x; idx < n_pairs; idx += blockDim.x) {
-    const int head = idx / half, i = idx - head * half;
-    const int col = head * hd + i;                 // q heads then k heads are contiguous in the GEMM output
-    const float a = gemm_load(qkv, r, col), b = gemm_load(qkv, r, col + half);
-    const float2 t = cs[i];                        // (cos, sin)
-    const float ra = a * t.x - b * t.y, rb = a * t.y + b * t.x;
-    if (head < nq) {
-      q_out[(size_t)r * QD + col] = ra;
-      q_out[(size_t)r * QD + col + half] = rb;
-    } else if (active) {
-      const int g = head - nq;
-      kdst[(size_t)g * KV_BLOCK * hd + i] = __float2half_rn(ra);
-      kdst[(size_t)g * KV_BLOCK * hd + i + half] = __float2half_rn(rb);
-    }
-  }
-  if (active) {
-    for (int idx = threadIdx.x; idx < KD; idx += blockDim.x) {
-      const int g = idx / hd, i = idx - g * hd;
-      vdst[(size_t)g * KV_BLOCK * hd + i] = __float2half_rn(gemm_load(qkv, r, QD + KD + idx));
-    }
-  }
-}
-
-// ---------------------------------------------------------------- split-KV paged attention
-constexpr int ATT_THREADS = 128;
-
-template <int HD, int GROUP>
-__global__ void __launch_bounds__(ATT_THREADS)
-attn_split_kernel(const float *__restrict__ q, Rows rows, int nq, KvLayout kv, int layer, int max_splits,
-                  float *__restrict__ part_acc, float *__restrict__ part_ml) {
-  constexpr int CH = HD / 8;                 // 16-byte chunks per cached row
-  constexpr int NTG = ATT_THREADS / CH;      // token groups in the value pass
-  const int split = blockIdx.x, g = blockIdx.y, r = blockIdx.z;
-  if (!rows.active[r]) return;
-  const int ctx = rows.pos[r] + 1;           // the new token attends to itself too
-  const int t0 = split * ATT_SPLIT;
-  if (t0 >= ctx) return;
-  const int ntok = min(ATT_SPLIT, ctx - t0);
-
-  __shared__ __align__(16) float q_s[GROUP][HD];
-  __shared__ __align__(16) float p_s[ATT_SPLIT * GROUP];
-  __shared__ __align__(16) float red_s[NTG][GROUP][HD];
-  __shared__ float wred_s[ATT_THREADS / 32][GROUP];
-  __shared__ int blk_s[ATT_SPLIT / KV_BLOCK];
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int nkv = kv.n_kv;
-  const __half *pool = kv.pool + (size_t)layer * kv.layer_stride;
-  const size_t blk_halfs = (size_t)2 * nkv * KV_BLOCK * HD;
-  // 1/sqrt(hd) * log2(e): scores live in the base-2 domain
-  const float qscale = (HD == 128 ? 0.08838834764831845f : 0.125f) * 1.4426950408889634f;
-  for (int i = tid; i < GROUP * HD; i += ATT_THREADS)
-    q_s[i / HD][i % HD] = q[(size_t)r * nq * HD + (size_t)(g * GROUP) * HD + i] * qscale;
-  if (tid < ATT_SPLIT / KV_BLOCK) {
-    const int b = t0 / KV_BLOCK + tid;
-    blk_s[tid] = (b * KV_BLOCK < ctx) ? kv.block_table[(size_t)rows.slot[r] * kv.max_blocks + b] : 0;
-  }
-  __syncthreads();
-
-  // ---- scores: one thread per cached token, dot product in ascending dim order
-  float lmax[GROUP];
-#pragma unroll
-  for (int h = 0; h < GROUP; ++h) lmax[h] = -CUDART_INF_F;
-#pragma unroll
-  for (int rep = 0; rep < ATT_SPLIT / ATT_THREADS; ++rep) {
-    const int tt = tid + rep * ATT_THREADS;
-    float s[GROUP];
-#pragma unroll
-    for (int h = 0; h < GROUP; ++h) s[h] = 0.f;
-    if (tt < ntok) {
-      const uint4 *kp = reinterpret_cast<const uint4 *>(pool + (size_t)blk_s[tt / KV_BLOCK] * blk_halfs +
-                                                        (size_t)g * KV_BLOCK * HD + (size_t)(tt % KV_BLOCK) * HD);
-#pragma unroll 4
-      for (int c = 0; c < CH; ++c) {
-        const uint4 kk = __ldg(kp + c);
-        const __half2 *k2 = reinterpret_cast<const __half2 *>(&kk);
-        float kf[8];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const float2 f = __half22float2(k2[j]);
-          kf[2 * j] = f.x;
-          kf[2 * j + 1] = f.y;
-        }
-#pragma unroll
-        for (int h = 0; h < GROUP; ++h) {
-          const float4 qa = *reinterpret_cast<const float4 *>(&q_s[h][c * 8]);
-          const float4 qb = *reinterpret_cast<const float4 *>(&q_s[h][c * 8 + 4]);
-          float a = s[h];
-          a = fmaf(qa.x, kf[0], a); a = fmaf(qa.y, kf[1], a); a = fmaf(qa.z, kf[2], a); a = fmaf(qa.w, kf[3], a);
-          a = fmaf(qb.x, kf[4], a); a = fmaf(qb.y, kf[5], a); a = fmaf(qb.z, kf[6], a); a = fmaf(qb.w, kf[7], a);
-          s[h] = a;
-        }
-      }
-#pragma unroll
-      for (int h = 0; h < GROUP; ++h) lmax[h] = fmaxf(lmax[h], s[h]);
-    } else {
-#pragma unroll
-      for (int h = 0; h < GROUP; ++h) s[h] = -CUDART_INF_F;
-    }
-#pragma unroll
-    for (int h = 0; h < GROUP; ++h) p_s[tt * GROUP + h] = s[h];
-  }
-  // ---- split maximum (exact, order-free)
-#pragma unroll
-  for (int h = 0; h < GROUP; ++h) {
-    float v = lmax[h];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    if (lane == 0) wred_s[warp][h] = v;
-  }
-  __syncthreads();
-  float m[GROUP], lsum[GROUP];
-#pragma unroll
-  for (int h = 0; h < GROUP; ++h) {
-    float v = wred_s[0][h];
-#pragma unroll
-    for (int w = 1; w < ATT_THREADS / 32; ++w) v = fmaxf(v, wred_s[w][h]);
-    m[h] = v;
-    lsum[h] = 0.f;
-  }
-  __syncthreads();
-  // ---- probabilities and their sum (fixed tree)
-#pragma unroll
-  for (int rep = 0; rep < ATT_SPLIT / ATT_THREADS; ++rep) {
-    const int tt = tid + rep * ATT_THREADS;
-#pragma unroll
-    for (int h = 0; h < GROUP; ++h) {
-      const float p = exp2f(p_s[tt * GROUP + h] - m[h]);   // -inf -> 0 for the tail
-      p_s[tt * GROUP + h] = p;
-      lsum[h] += p;
-    }
-  }
-#pragma unroll
-  for (int h = 0; h < GROUP; ++h) {
-    float v = lsum[h];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    if (lane == 0) wred_s[warp][h] = v;
-  }
-  __syncthreads();
-  if (tid < GROUP) {
-    float v = 0.f;
-    for (int w = 0; w < ATT_THREADS / 32; ++w) v += wred_s[w][tid];
-    float *ml = part_ml + (((size_t)r * nq + g * GROUP + tid) * max_splits + split) * 2;
-    ml[0] = m[tid];
-    ml[1] = v;
-  }
-  // ---- weighted values: thread = (8-dim chunk, token group), tokens ascending inside a group
-  const int dc = tid % CH, tg = tid / CH;
-  float acc[GROUP][8];
-#pragma unroll
-  for (int h = 0; h < GROUP; ++h)
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[h][j] = 0.f;
-  for (int tt = tg; tt < ntok; tt += NTG) {
-    const uint4 *vp = reinterpret_cast<const uint4 *>(pool + (size_t)blk_s[tt / KV_BLOCK] * blk_halfs +
-                                                      (size_t)(nkv + g) * KV_BLOCK * HD + (size_t)(tt % KV_BLOCK) * HD);
-    const uint4 vv = __ldg(vp + dc);
-    const __half2 *v2 = reinterpret_cast<const __half2 *>(&vv);
-    float vf[8];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float2 f = __half22float2(v2[j]);
-      vf[2 * j] = f.x;
-      vf[2 * j + 1] = f.y;
-    }
-#pragma unroll
-    for (int h = 0; h < GROUP; ++h) {
-      const float p = p_s[tt * GROUP + h];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) acc[h][j] = fmaf(p, vf[j], acc[h][j]);
-    }
-  }
-#pragma unroll
-  for (int h = 0; h < GROUP; ++h)
-#pragma unroll
-    for (int j = 0; j < 8; ++j) red_s[tg][h][dc * 8 + j] = acc[h][j];
-  __syncthreads();
-  for (int idx = tid; idx < GROUP * HD; idx += ATT_THREADS) {
-    const int h = idx / HD, d = idx - h * HD;
-    float o = 0.f;
-#pragma unroll
-    for (int t = 0; t < NTG; ++t) o += red_s[t][h][d];
-    part_acc[(((size_t)r * nq + g * GROUP + h) * max_splits + split) * HD + d] = o;
-  }
-}
-
-// Combines the splits of each (row, head) in ascending split order.
-__global__ void __launch_bounds__(256)
-attn_combine_kernel(Rows rows, int nq, int hd, int max_splits, const float *__restrict__ part_acc,
-                    const float *__restrict__ part_ml, __nv_bfloat16 *__restrict__ out_hi,
-                    __nv_bfloat16 *__restrict__ out_lo) {
-  const int r = blockIdx.x;
-  const int QD = nq * hd;
   const bool active = rows.active[r] != 0;
-  const int nsplit = active ? (rows.pos[r] + 1 + ATT_SPLIT - 1) / ATT_SPLIT : 0;
-  for (int idx = threadIdx.x; idx < QD; idx += blockDim.x) {
-    float o = 0.f;
-    if (active) {
-      const int j = idx / hd, d = idx - j * hd;
-      const float *ml = part_ml + ((size_t)r * nq + j) * max_splits * 2;
-      const float *pa = part_acc + ((size_t)r * nq + j) * max_splits * hd + d;
-      float M = ml[0];
-      for (int s = 1; s < nsplit; ++s) M = fmaxf(M, ml[2 * s]);
-      float num = 0.f, den = 0.f;
-      for (int s = 0; s < nsplit; ++s) {
-        const float w = exp2f(ml[2 * s] - M);
-        num = fmaf(pa[(size_t)s * hd], w, num);
-        den = fmaf(ml[2 * s + 1], w, den);
-      }
-      o = num / den;
-    }
-    __nv_bfloat16 a, b;
-    split_bf16(o, a, b);
-    out_hi[(size_t)r * QD + idx] = a;
-    out_lo[(size_t)r * QD + idx] = b;
+  if (head >= nq && !active) return;               // padding rows write no cache
+  const int col = head * hd + i;                   // q, k and v heads are contiguous in the GEMM output
+  const float a = gemm_load(qkv, r, col), b = gemm_load(qkv, r, col + half);
+  if (head < nq) {
+    const float2 t = rope_tab[(size_t)pos * half + i];   // (cos, sin)
+    float *q = q_out + (size_t)r * nq * hd + col;
+    q[0] = a * t.x - b * t.y;
+    q[half] = a * t.y + b * t.x;
+    return;
+  }
+  const int blk = kv.block_table[(size_t)rows.slot[r] * kv.max_blocks + pos / KV_BLOCK];
+  __half *base = kv.pool + (size_t)layer * kv.layer_stride + (size_t)blk * 2 * nkv * KV_BLOCK * hd +
+                 (size_t)(pos % KV_BLOCK) * hd + i;
+  // a page holds the nkv key tiles followed by the nkv value tiles, in the order of the GEMM's heads
+  __half *dst = base + (size_t)(head - nq) * KV_BLOCK * hd;
+  if (head < nq + nkv) {
+    const float2 t = rope_tab[(size_t)pos * half + i];
+    dst[0] = __float2half_rn(a * t.x - b * t.y);
+    dst[half] = __float2half_rn(a * t.y + b * t.x);
+  } else {
+    dst[0] = __float2half_rn(a);
+    dst[half] = __float2half_rn(b);
   }
 }
 
@@ -309,14 +113,12 @@ attn_combine_kernel(Rows rows, int nq, int hd, int max_splits, const float *__re
 __global__ void __launch_bounds__(256)
 swiglu_kernel(GemmOut gu, int F, __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo) {
   const int r = blockIdx.y;
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  const int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i >= F) return;
-  const float g = gemm_load(gu, r, i), u = gemm_load(gu, r, F + i);
-  const float y = g / (1.f + expf(-g)) * u;
-  __nv_bfloat16 a, b;
-  split_bf16(y, a, b);
-  out_hi[(size_t)r * F + i] = a;
-  out_lo[(size_t)r * F + i] = b;
+  const float4 g = gemm_load4(gu, r, i), u = gemm_load4(gu, r, F + i);
+  const float4 y = make_float4(g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
+                               g.z / (1.f + expf(-g.z)) * u.z, g.w / (1.f + expf(-g.w)) * u.w);
+  store_split4(y, out_hi + (size_t)r * F + i, out_lo + (size_t)r * F + i);
 }
 
 __global__ void split_kernel(const float *__restrict__ x, size_t n, __nv_bfloat16 *__restrict__ hi,
@@ -660,19 +462,6 @@ __global__ void kv_fill_kernel(KvLayout kv, int n_layers, int slot, int n, float
   *(kp + (size_t)kv.n_kv * KV_BLOCK * kv.hd) = __float2half_rn(rad * sinpif(2.0f * u2));
 }
 
-template <int HD>
-cudaError_t launch_attn_hd(int group, dim3 grid, cudaStream_t st, const float *q, const Rows &rows, int nq,
-                           const KvLayout &kv, int layer, int max_splits, float *pa, float *pm) {
-  switch (group) {
-    case 1: attn_split_kernel<HD, 1><<<grid, ATT_THREADS, 0, st>>>(q, rows, nq, kv, layer, max_splits, pa, pm); break;
-    case 2: attn_split_kernel<HD, 2><<<grid, ATT_THREADS, 0, st>>>(q, rows, nq, kv, layer, max_splits, pa, pm); break;
-    case 4: attn_split_kernel<HD, 4><<<grid, ATT_THREADS, 0, st>>>(q, rows, nq, kv, layer, max_splits, pa, pm); break;
-    case 8: attn_split_kernel<HD, 8><<<grid, ATT_THREADS, 0, st>>>(q, rows, nq, kv, layer, max_splits, pa, pm); break;
-    default: return cudaErrorInvalidValue;
-  }
-  return cudaGetLastError();
-}
-
 }  // namespace
 
 cudaError_t launch_resid_norm(float *h, int H, const __nv_bfloat16 *embed, const Rows &rows, const GemmOut *prev,
@@ -680,32 +469,21 @@ cudaError_t launch_resid_norm(float *h, int H, const __nv_bfloat16 *embed, const
                               cudaStream_t st) {
   GemmOut g{};
   if (prev) g = *prev;
-  resid_norm_kernel<<<rows.R, NORM_THREADS, 0, st>>>(h, H, embed, rows, g, prev ? 0 : 1, gains, eps, out_hi, out_lo);
+  int threads = H / 4;
+  if (threads > NORM_MAX_THREADS) threads = NORM_MAX_THREADS;
+  threads = (threads + 31) / 32 * 32;
+  resid_norm_kernel<<<rows.R, threads, 0, st>>>(h, H, embed, rows, g, prev ? 0 : 1, gains, eps, out_hi, out_lo);
   return cudaGetLastError();
 }
 
 cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *rope_tab, int nq, const KvLayout &kv,
                             int layer, float *q_out, cudaStream_t st) {
-  qkv_post_kernel<<<rows.R, 256, 0, st>>>(qkv, rows, rope_tab, nq, kv, layer, q_out);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_attention(const float *q, const Rows &rows, int nq, const KvLayout &kv, int layer, int max_splits,
-                             float *part_acc, float *part_ml, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
-                             cudaStream_t st) {
-  const dim3 grid(max_splits, kv.n_kv, rows.R);
-  const int group = nq / kv.n_kv;
-  cudaError_t e;
-  if (kv.hd == 128) e = launch_attn_hd<128>(group, grid, st, q, rows, nq, kv, layer, max_splits, part_acc, part_ml);
-  else if (kv.hd == 64) e = launch_attn_hd<64>(group, grid, st, q, rows, nq, kv, layer, max_splits, part_acc, part_ml);
-  else return cudaErrorInvalidValue;
-  if (e != cudaSuccess) return e;
-  attn_combine_kernel<<<rows.R, 256, 0, st>>>(rows, nq, kv.hd, max_splits, part_acc, part_ml, out_hi, out_lo);
+  qkv_post_kernel<<<dim3(nq + 2 * kv.n_kv, rows.R), kv.hd / 2, 0, st>>>(qkv, rows, rope_tab, nq, kv, layer, q_out);
   return cudaGetLastError();
 }
 
 cudaError_t launch_swiglu(const GemmOut &gu, int R, int F, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, cudaStream_t st) {
-  swiglu_kernel<<<dim3((F + 255) / 256, R), 256, 0, st>>>(gu, F, out_hi, out_lo);
+  swiglu_kernel<<<dim3((F / 4 + 255) / 256, R), 256, 0, st>>>(gu, F, out_hi, out_lo);
   return cudaGetLastError();
 }
 

@@ -12,7 +12,7 @@
 namespace corun {
 
 constexpr int KV_BLOCK = 16;      // tokens per page
-constexpr int ATT_SPLIT = 256;    // tokens per attention split (fixed; count = f(own context))
+constexpr int ATT_SPLIT = 128;    // tokens per attention split (fixed; count = f(own context))
 
 // Per-row metadata (device arrays of length R).
 struct Rows {
@@ -28,6 +28,7 @@ struct KvLayout {
   const int *block_table;  // [n_slots][max_blocks]
   int max_blocks, n_kv, hd;
   size_t layer_stride;     // halfs per layer
+  long long pool_blocks;   // pages per layer
 };
 
 struct SampleArgs {
@@ -50,9 +51,11 @@ cudaError_t launch_resid_norm(float *h, int H, const __nv_bfloat16 *embed, const
 cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *rope_tab, int nq, const KvLayout &kv,
                             int layer, float *q_out, cudaStream_t st);
 // Split-KV paged attention partials and their fixed-order combine -> bf16 hi/lo [R, nq*hd].
-cudaError_t launch_attention(const float *q, const Rows &rows, int nq, const KvLayout &kv, int layer, int max_splits,
-                             float *part_acc, float *part_ml, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
-                             cudaStream_t st);
+// tmKV: tensor map over the whole pool as [all cached rows, hd] fp16 with a [16, 64] box (see attention.cu).
+cudaError_t launch_attention(const CUtensorMap &tmKV, const float *q, const Rows &rows, int nq, const KvLayout &kv,
+                             int layer, int max_splits, float *part_acc, float *part_ml, __nv_bfloat16 *out_hi,
+                             __nv_bfloat16 *out_lo, int *d_status, cudaStream_t st);
+cudaError_t attention_prepare();   // opts the kernels into their shared-memory size (idempotent)
 // y = silu(gate) * up from the gate-up GEMM result -> bf16 hi/lo [R, F].
 cudaError_t launch_swiglu(const GemmOut &gu, int R, int F, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, cudaStream_t st);
 // x fp32 [R, K] -> bf16 hi/lo.
