@@ -182,6 +182,11 @@ int corun_debug_kv_fill(corun_engine *e, int32_t slot, int32_t n_ctx, float std,
  * 8 SwiGLU, 9 sampler.  Uses the rows of the last decode step; overwrites
  * intermediate buffers (not the cache beyond each active slot's next position). */
 int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *avg_ms);
+/* Runs GEMM `kind` (0 QKV, 1 O, 2 gate-up, 3 down, 4 LM head) of the decode program on one layer's
+ * weights three times and returns the last launch's per-CTA timeline: stamps[cta*8 + i] (host, room for
+ * 8 * 256 values) are globaltimer nanoseconds at: 0 kernel entry, 1 set-up done, 2 first TMA issued,
+ * 3 last TMA issued, 4 first stage landed, 5 last MMA issued, 6 last accumulator complete, 7 epilogue done. */
+int corun_debug_gemm_trace(corun_engine *e, int32_t kind, int32_t layer, uint64_t *stamps, int32_t *n_ctas);
 /* Copies the first n floats of an intermediate buffer of the decode program to the host, as left by
  * the last decode step: which = 0 rotated queries [B, nq*hd]; 1 attention split partials
  * [B][nq][max_splits][hd]; 2 their (max, sum) pairs [B][nq][max_splits][2] (base-2 domain);

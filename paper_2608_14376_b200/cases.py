@@ -82,6 +82,12 @@ def case_kernels(a):
         ms = eng.time_kernel(i, 4 * a.layers if i not in (4, 9) else 6)
         extra = "  %7.0f GB/s" % (nbytes[name] / ms / 1e6) if name in nbytes else ""
         print("%-16s %8.2f us%s" % (name, ms * 1e3, extra))
+    if a.trace:
+        for kind in (1, 2):
+            t = eng.gemm_trace(kind, 1)
+            names = ["entry", "setup", "tma0", "tmaN", "land0", "mmaN", "accN", "done"]
+            print(eng.KERNEL_KINDS[kind], "timeline (us, median / max over CTAs):",
+                  "  ".join("%s %.2f/%.2f" % (n, np.median(t[:, i]) / 1e3, t[:, i].max() / 1e3) for i, n in enumerate(names)))
     eng.close()
 
 
@@ -99,6 +105,7 @@ def main():
     k.add_argument("--layers", type=int, default=4); k.add_argument("--B", type=int, default=64)
     k.add_argument("--active-frac", type=float, default=0.625); k.add_argument("--ctx-lo", type=int, default=512)
     k.add_argument("--ctx-hi", type=int, default=4096); k.add_argument("--vocab", type=int, default=32768)
+    k.add_argument("--trace", action="store_true")
     a = ap.parse_args()
     {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels}[a.case](a)
 

@@ -18,6 +18,7 @@
 #include <cuda_fp16.h>
 #include <math_constants.h>
 
+#include "launch.cuh"
 #include "ops.cuh"
 #include "ptx.cuh"
 
@@ -60,18 +61,18 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(
 template <int HD>
 __global__ void __launch_bounds__(ATT_THREADS)
 attn_split_kernel(const __grid_constant__ CUtensorMap tmKV, const float *__restrict__ q, Rows rows, int nq, int group,
-                  KvLayout kv, int layer, int max_splits, float *__restrict__ part_acc, float *__restrict__ part_ml,
-                  int *status) {
+                  KvLayout kv, int layer, int max_splits, const int *__restrict__ work, const int *__restrict__ n_work,
+                  float *__restrict__ part_acc, float *__restrict__ part_ml, int *status) {
   constexpr int NBOX = HD / 64;                  // boxes per (page, head) tile
   constexpr int TILE_BYTES = NBOX * BOX_BYTES;   // K (or V) of one page and head
   constexpr int KSTEPS = HD / 16;                // k-steps of the score MMA
   constexpr int NT = HD / 8;                     // n-tiles of the value MMA
-  const int split = blockIdx.x, g = blockIdx.y, r = blockIdx.z;
-  if (!rows.active[r]) return;
-  const int ctx = rows.pos[r] + 1;               // the new token attends to itself too
-  const int t0 = split * ATT_SPLIT;
-  if (t0 >= ctx) return;
-  const int n_pages = min(ATT_PAGES, (ctx - t0 + KV_BLOCK - 1) / KV_BLOCK);
+  griddep_launch_dependents();
+  griddep_wait();                                // the item list and q come from earlier kernels
+  // persistent CTAs walk the step's list of (row, split) items x kv heads with a fixed stride; the
+  // list only decides which CTA computes an item, never how it is computed
+  const int n_items = *n_work * kv.n_kv;
+  if ((int)blockIdx.x >= n_items) return;
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar[4];
@@ -80,15 +81,23 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmKV, const float *__restr
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;     // K tiles, then V tiles
   const uint32_t v_tiles = tiles + ATT_PAGES * TILE_BYTES;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-
-  if (tid < ATT_PAGES)
-    page_s[tid] = tid < n_pages ? kv.block_table[(size_t)rows.slot[r] * kv.max_blocks + t0 / KV_BLOCK + tid] : 0;
   if (tid == 0) {
     abort_flag = 0;
     for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bar[w]), 1);
     fence_mbar_init();
     fence_proxy_async();
   }
+  bool failed = false;
+  uint32_t parity = 0;                           // phase of this warp's barrier: flips each time it is armed
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+  const int wi = work[item / kv.n_kv], g = item % kv.n_kv;
+  const int r = wi >> 8, split = wi & 255;
+  const int ctx = rows.pos[r] + 1;               // the new token attends to itself too
+  const int t0 = split * ATT_SPLIT;
+  const int n_pages = min(ATT_PAGES, (ctx - t0 + KV_BLOCK - 1) / KV_BLOCK);
+  __syncthreads();                               // the previous item's merge buffers (tile memory) are free
+  if (tid < ATT_PAGES)
+    page_s[tid] = tid < n_pages ? kv.block_table[(size_t)rows.slot[r] * kv.max_blocks + t0 / KV_BLOCK + tid] : 0;
   __syncthreads();
   if (tid == 0) {
     const uint64_t pol = l2_policy_evict_first();       // the cache is streamed once per step
@@ -141,10 +150,10 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmKV, const float *__restr
   float m_run = -CUDART_INF_F, l_run = 0.f;
 
   const int warp_t0 = t0 + warp * 32;
-  bool failed = false;
   if (warp_t0 < ctx) {
-    bool ok = mbar_wait(smem_u32(&bar[warp]), 0u, &abort_flag);
+    bool ok = mbar_wait(smem_u32(&bar[warp]), parity, &abort_flag);
     ok = __all_sync(0xffffffffu, ok);
+    parity ^= 1u;                                // armed exactly when this warp has tokens (warp_t0 < ctx)
     if (!ok) {
       failed = true;
     } else {
@@ -253,6 +262,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmKV, const float *__restr
       part_ml[slot * 2 + 1] = den;
     }
   }
+  }   // items
   if (failed || abort_flag) {
     if (tid == 0) atomicCAS(status, 0, DEV_TIMEOUT_EPILOGUE);
     for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let copies in flight land before the CTA retires
@@ -265,6 +275,8 @@ __global__ void __launch_bounds__(128)
 attn_combine_kernel(Rows rows, int nq, int hd, int max_splits, const float *__restrict__ part_acc,
                     const float *__restrict__ part_ml, __nv_bfloat16 *__restrict__ out_hi,
                     __nv_bfloat16 *__restrict__ out_lo) {
+  griddep_launch_dependents();
+  griddep_wait();
   const int j = blockIdx.x, r = blockIdx.y, d = threadIdx.x;
   float o = 0.f;
   if (rows.active[r]) {
@@ -288,6 +300,22 @@ attn_combine_kernel(Rows rows, int nq, int hd, int max_splits, const float *__re
   out_lo[idx] = b;
 }
 
+// Lists the (row, split) items of the step: active rows in ascending order, splits ascending.
+// One CTA; rows <= 256.  Entry = row << 8 | split.
+__global__ void __launch_bounds__(256) attn_worklist_kernel(Rows rows, int *__restrict__ work, int *__restrict__ n_work) {
+  griddep_launch_dependents();
+  griddep_wait();
+  __shared__ int cnt[256];
+  const int r = threadIdx.x;
+  const int mine = (r < rows.R && rows.active[r]) ? (rows.pos[r] + 1 + ATT_SPLIT - 1) / ATT_SPLIT : 0;
+  cnt[r] = mine;
+  __syncthreads();
+  int before = 0;
+  for (int i = 0; i < r; ++i) before += cnt[i];
+  for (int s = 0; s < mine; ++s) work[before + s] = (r << 8) | s;
+  if (r == 255) *n_work = before + mine;
+}
+
 template <int HD>
 constexpr size_t att_smem_bytes() {
   return (size_t)2 * ATT_PAGES * (HD / 64) * BOX_BYTES + 1024;
@@ -303,24 +331,31 @@ cudaError_t attention_prepare() {
                               (int)att_smem_bytes<64>());
 }
 
+cudaError_t launch_attn_worklist(const Rows &rows, int *work, int *n_work, cudaStream_t st) {
+  if (rows.R > 256) return cudaErrorInvalidValue;
+  return launch_k(attn_worklist_kernel, dim3(1), dim3(256), 0, st, true, rows, work, n_work);
+}
+
 cudaError_t launch_attention(const CUtensorMap &tmKV, const float *q, const Rows &rows, int nq, const KvLayout &kv,
-                             int layer, int max_splits, float *part_acc, float *part_ml, __nv_bfloat16 *out_hi,
-                             __nv_bfloat16 *out_lo, int *d_status, cudaStream_t st) {
-  const dim3 grid(max_splits, kv.n_kv, rows.R);
+                             int layer, int max_splits, const int *work, const int *n_work, int grid_ctas,
+                             float *part_acc, float *part_ml, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
+                             int *d_status, cudaStream_t st) {
   const int group = nq / kv.n_kv;
-  if (group < 1 || group > 8) return cudaErrorInvalidValue;
+  if (group < 1 || group > 8 || max_splits > 256) return cudaErrorInvalidValue;
+  const long long most = (long long)rows.R * max_splits * kv.n_kv;
+  const int grid = (int)(most < grid_ctas ? most : grid_ctas);
+  cudaError_t e;
   if (kv.hd == 128)
-    attn_split_kernel<128><<<grid, ATT_THREADS, att_smem_bytes<128>(), st>>>(tmKV, q, rows, nq, group, kv, layer,
-                                                                              max_splits, part_acc, part_ml, d_status);
+    e = launch_k(attn_split_kernel<128>, dim3(grid), dim3(ATT_THREADS), att_smem_bytes<128>(), st, true, tmKV, q, rows, nq,
+                 group, kv, layer, max_splits, work, n_work, part_acc, part_ml, d_status);
   else if (kv.hd == 64)
-    attn_split_kernel<64><<<grid, ATT_THREADS, att_smem_bytes<64>(), st>>>(tmKV, q, rows, nq, group, kv, layer,
-                                                                            max_splits, part_acc, part_ml, d_status);
+    e = launch_k(attn_split_kernel<64>, dim3(grid), dim3(ATT_THREADS), att_smem_bytes<64>(), st, true, tmKV, q, rows, nq,
+                 group, kv, layer, max_splits, work, n_work, part_acc, part_ml, d_status);
   else
     return cudaErrorInvalidValue;
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  attn_combine_kernel<<<dim3(nq, rows.R), kv.hd, 0, st>>>(rows, nq, kv.hd, max_splits, part_acc, part_ml, out_hi, out_lo);
-  return cudaGetLastError();
+  return launch_k(attn_combine_kernel, dim3(nq, rows.R), dim3(kv.hd), 0, st, true, rows, nq, kv.hd, max_splits, part_acc,
+                  part_ml, out_hi, out_lo);
 }
 
 }  // namespace corun

@@ -42,7 +42,7 @@ struct Program {
   float *qkv_out = nullptr, *o_out = nullptr, *gu_out = nullptr, *down_out = nullptr, *logits = nullptr, *ws = nullptr;
   bf16 *xn_hi = nullptr, *xn_lo = nullptr, *ao_hi = nullptr, *ao_lo = nullptr, *ff_hi = nullptr, *ff_lo = nullptr;
   int *row_token = nullptr, *row_pos = nullptr, *row_active = nullptr, *row_slot = nullptr, *do_sample = nullptr;
-  int *sampled = nullptr;
+  int *sampled = nullptr, *att_work = nullptr, *att_n_work = nullptr;
   GemmPlan p_qkv, p_o, p_gu, p_down, p_lm;
   bool has_layers = false, has_lm = false;
   std::vector<void *> allocs;
@@ -137,6 +137,8 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm) {
     RC(dmalloc(A, &P.q, (size_t)R * QD));
     RC(dmalloc(A, &P.part_acc, (size_t)R * s.n_q_heads * e->max_splits * s.head_dim));
     RC(dmalloc(A, &P.part_ml, (size_t)R * s.n_q_heads * e->max_splits * 2));
+    RC(dmalloc(A, &P.att_work, (size_t)R * e->max_splits));
+    RC(dmalloc(A, &P.att_n_work, 1));
     RC(dmalloc(A, &P.qkv_out, (size_t)R * (QD + 2 * KD)));
     RC(dmalloc(A, &P.o_out, (size_t)R * H));
     RC(dmalloc(A, &P.gu_out, (size_t)R * 2 * F));
@@ -179,6 +181,8 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
   const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
   const KvLayout kv = kv_layout(e);
   int n = 0;
+  CK(launch_attn_worklist(rows, P.att_work, P.att_n_work, e->st));   // the same items serve every layer
+  n += 1;
   int stage = 0;
   const int stop = (e->eager && &P == &e->dec) ? e->stop_after : -1;
 #define STAGE(call)                                   \
@@ -191,16 +195,16 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
     GemmOut prev = P.p_down.out();
     STAGE(launch_resid_norm(P.h, s.hidden, e->embed, rows, l == 0 ? nullptr : &prev, e->attn_norm[l], s.rms_eps,
                             P.xn_hi, P.xn_lo, e->st));
-    STAGE(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st));
+    STAGE(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, nullptr, true));
     STAGE(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st));
-    STAGE(launch_attention(e->tm_kv, P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.part_acc, P.part_ml, P.ao_hi,
-                           P.ao_lo, e->d_status, e->st));
-    STAGE(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st));
+    STAGE(launch_attention(e->tm_kv, P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work, P.att_n_work,
+                           3 * e->num_sms, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo, e->d_status, e->st));
+    STAGE(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st, nullptr, true));
     GemmOut o = P.p_o.out();
     STAGE(launch_resid_norm(P.h, s.hidden, nullptr, rows, &o, e->mlp_norm[l], s.rms_eps, P.xn_hi, P.xn_lo, e->st));
-    STAGE(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st));
+    STAGE(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st, nullptr, true));
     STAGE(launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st));
-    STAGE(gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st));
+    STAGE(gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st, nullptr, true));
     n += 10;
   }
 #undef STAGE
@@ -223,10 +227,10 @@ int enqueue_decode_body(corun_engine *e, int *launches) {
     const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
     GemmOut prev = P.p_down.out();
     CK(launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->final_norm, s.rms_eps, P.xn_hi, P.xn_lo, e->st));
-    CK(gemm_launch(P.p_lm, nullptr, e->d_status, e->st));
-    CK(gemm_fixup_launch(P.p_lm, e->st));
+    CK(gemm_launch(P.p_lm, nullptr, e->d_status, e->st, nullptr, true));
+    CK(gemm_fixup_launch(P.p_lm, e->st, true));
     SampleArgs sa{P.logits, s.vocab, P.do_sample, e->d_temp, e->d_top_p, e->d_seeds, e->d_step, nullptr, P.sampled};
-    CK(launch_sampler(sa, P.R, e->st));
+    CK(launch_sampler(sa, P.R, e->st, true));
     CK(launch_advance(P.row_active, P.sampled, e->B, e->d_ctx, e->d_step, e->d_pending, e->d_out_tokens, e->st));
     n += 4 + (P.p_lm.n_split_tiles ? 1 : 0);
   }
@@ -311,7 +315,7 @@ int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int3
   if (group != 1 && group != 2 && group != 4 && group != 8) return CORUN_EINVAL;
   if ((s.n_q_heads * s.head_dim) % 64) return CORUN_EINVAL;
   if (!(s.rms_eps >= 0.f) || !(s.rope_theta > 0.f)) return CORUN_EINVAL;
-  if (B < 1 || B > 256 || max_context < 1 || kv_block != KV_BLOCK || kv_pool_blocks < 0) return CORUN_EINVAL;
+  if (B < 1 || B > 256 || max_context < 1 || max_context > 256 * ATT_SPLIT || kv_block != KV_BLOCK || kv_pool_blocks < 0) return CORUN_EINVAL;
   if (!w->embed || !w->lm_head || !w->final_norm || !w->attn_norm || !w->wqkv || !w->wo || !w->mlp_norm ||
       !w->wgate_up || !w->wdown)
     return CORUN_EINVAL;
@@ -714,8 +718,9 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
         case 4: ce = gemm_launch(P.p_lm, nullptr, e->d_status, e->st);
                 if (ce == cudaSuccess) ce = gemm_fixup_launch(P.p_lm, e->st);
                 break;
-        case 5: ce = launch_attention(e->tm_kv, P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.part_acc, P.part_ml,
-                                      P.ao_hi, P.ao_lo, e->d_status, e->st); break;
+        case 5: ce = launch_attention(e->tm_kv, P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work,
+                                      P.att_n_work, 3 * e->num_sms, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo,
+                                      e->d_status, e->st); break;
         case 6: ce = launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->attn_norm[l], s.rms_eps, P.xn_hi,
                                        P.xn_lo, e->st); break;
         case 7: ce = launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st); break;
@@ -737,6 +742,26 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
   cudaEventDestroy(a);
   cudaEventDestroy(b);
   return rc;
+}
+
+int corun_debug_gemm_trace(corun_engine *e, int32_t kind, int32_t layer, uint64_t *stamps, int32_t *n_ctas) {
+  if (!e || !stamps || !n_ctas || kind < 0 || kind > 4 || layer < 0 || layer >= e->sh.n_layers) return CORUN_EINVAL;
+  RC(sync_stream(e));
+  Program &P = e->dec;
+  const GemmPlan *pl[5] = {&P.p_qkv, &P.p_o, &P.p_gu, &P.p_down, &P.p_lm};
+  const CUtensorMap *tm[5] = {&e->tm_qkv[layer], &e->tm_o[layer], &e->tm_gu[layer], &e->tm_down[layer], nullptr};
+  const GemmPlan &p = *pl[kind];
+  unsigned long long *d = nullptr;
+  if (cudaMalloc(&d, (size_t)p.grid * 8 * sizeof(unsigned long long)) != cudaSuccess) return CORUN_ENOMEM;
+  cudaError_t ce = cudaMemsetAsync(d, 0, (size_t)p.grid * 8 * sizeof(unsigned long long), e->st);
+  for (int i = 0; i < 3 && ce == cudaSuccess; ++i) ce = gemm_launch(p, tm[kind], e->d_status, e->st, d);   // last one counts
+  if (ce == cudaSuccess)
+    ce = cudaMemcpyAsync(stamps, d, (size_t)p.grid * 8 * sizeof(unsigned long long), cudaMemcpyDeviceToHost, e->st);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(e->st);
+  cudaFree(d);
+  if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
+  *n_ctas = p.grid;
+  return CORUN_OK;
 }
 
 int corun_debug_read(corun_engine *e, int32_t which, float *out, int64_t n) {

@@ -7,11 +7,13 @@
 #include <vector>
 
 #include "../../include/corun.h"
+#include "launch.cuh"
 #include "ptx.cuh"
 
 namespace corun {
 
 int g_last_cuda_error = 0;
+bool g_use_pdl = !(getenv("CORUN_NO_PDL") && atoi(getenv("CORUN_NO_PDL")) != 0);
 
 namespace {
 
@@ -32,21 +34,35 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmHi,
                     const __grid_constant__ CUtensorMap tmLo, float *__restrict__ direct, float *__restrict__ ws,
                     const int *__restrict__ cta_start, int N, int KB, int BN, int R, int stages, int tmem_cols,
-                    uint32_t idesc, int *status) {
+                    uint32_t idesc, int *status, unsigned long long *trace) {
   extern __shared__ uint8_t smem_raw[];
+  // optional per-CTA timeline (debug): 8 globaltimer stamps
+#define TRACE(i) do { if (trace) trace[(size_t)blockIdx.x * 8 + (i)] = globaltimer_ns(); } while (0)
+  if (threadIdx.x == 0) TRACE(0);
+  griddep_launch_dependents();   // the next kernel may start its prologue
   __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
   __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
-  __shared__ __align__(8) uint64_t tmem_full_bar;
-  __shared__ __align__(8) uint64_t tmem_empty_bar;
+  __shared__ __align__(8) uint64_t tmem_full_bar[2];    // one pair per accumulator buffer
+  __shared__ __align__(8) uint64_t tmem_empty_bar[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
+  __shared__ float xch[64 * 33];   // hi/lo hand-over of the stacked epilogue (row pitch 33: no bank conflicts)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t x_bytes = (uint32_t)BN * GEMM_BLOCK_K * 2;         // BN * 128 B
-  const uint32_t stage_bytes = W_TILE_BYTES + 2 * x_bytes;
+  // Up to 64 rows: hi and lo share one 128-row A tile (hi in rows 0.., lo in rows 64..), so one MMA
+  // per k-slice yields W*hi in accumulator lanes 0-63 and W*lo in lanes 64-127; the epilogue adds them.
+  const bool stacked = BN <= 64;
+  const uint32_t lo_off = stacked ? (uint32_t)(64 * GEMM_BLOCK_K * 2) : x_bytes;
+  const uint32_t stage_bytes = W_TILE_BYTES + (stacked ? A_BLOCK_BYTES : 2 * x_bytes);
+  const uint32_t tx_bytes = W_TILE_BYTES + 2 * x_bytes;
   const int n_rb = (BN + GEMM_ROW_BLOCK - 1) / GEMM_ROW_BLOCK;      // blocks of 128 activation rows
+  // up to 128 rows need 256 TMEM columns: two accumulator buffers fit, so the epilogue of one
+  // segment overlaps the MMAs of the next
+  const int n_acc = (n_rb == 1) ? 2 : 1;
+  const uint32_t acc_cols = (uint32_t)n_rb * GEMM_TILE_N;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -54,8 +70,10 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       mbar_init(smem_u32(&full_bar[s]), 1);
       mbar_init(smem_u32(&empty_bar[s]), 1);
     }
-    mbar_init(smem_u32(&tmem_full_bar), 1);
-    mbar_init(smem_u32(&tmem_empty_bar), 128);
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(smem_u32(&tmem_full_bar[a]), 1);
+      mbar_init(smem_u32(&tmem_empty_bar[a]), 128);
+    }
     fence_mbar_init();
     fence_proxy_async();
     prefetch_tensormap(&tmW);
@@ -71,6 +89,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
   volatile int *abort_p = &abort_flag;
+  if (threadIdx.x == 0) TRACE(1);
 
   const int k0 = cta_start[cta], k1 = cta_start[cta + 1];
   int fail = 0;
@@ -80,19 +99,39 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       // ---------------- TMA producer ----------------
       const uint64_t pol_w = l2_policy_evict_first();   // weights are streamed once per step
       const uint64_t pol_x = l2_policy_evict_last();    // activations are re-read by every CTA
-      int it = 0;
-      for (int g = k0; g < k1; ++g, ++it) {
+      // The weights depend on no earlier kernel: fill the ring with weight tiles first, then wait for
+      // the predecessor (which produces the activations) and add the activation tiles to the same
+      // barriers.
+      const int n_pre = min(stages, k1 - k0);
+      for (int it = 0; it < n_pre; ++it) {
+        const int g = k0 + it, tile = g / KB, kb = g - tile * KB;
+        const uint32_t fb = smem_u32(&full_bar[it]);
+        mbar_arrive_expect_tx(fb, tx_bytes);
+        tma_load_2d(tiles_base + (uint32_t)it * stage_bytes, &tmW, kb * GEMM_BLOCK_K, tile * GEMM_TILE_N, fb, pol_w);
+        if (it == 0) TRACE(2);
+      }
+      griddep_wait();
+      for (int it = 0; it < n_pre; ++it) {
+        const int g = k0 + it, tile = g / KB, kb = g - tile * KB;
+        const uint32_t fb = smem_u32(&full_bar[it]);
+        const uint32_t dst = tiles_base + (uint32_t)it * stage_bytes;
+        tma_load_2d(dst + W_TILE_BYTES, &tmHi, kb * GEMM_BLOCK_K, 0, fb, pol_x);
+        tma_load_2d(dst + W_TILE_BYTES + lo_off, &tmLo, kb * GEMM_BLOCK_K, 0, fb, pol_x);
+      }
+      int it = n_pre;
+      for (int g = k0 + n_pre; g < k1; ++g, ++it) {
         const int tile = g / KB, kb = g - tile * KB;
         const int s = it % stages;
         const uint32_t ph = (uint32_t)(it / stages) & 1u;
         if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_p)) { fail = DEV_TIMEOUT_PRODUCER; break; }
         const uint32_t fb = smem_u32(&full_bar[s]);
         const uint32_t dst = tiles_base + (uint32_t)s * stage_bytes;
-        mbar_arrive_expect_tx(fb, stage_bytes);
+        mbar_arrive_expect_tx(fb, tx_bytes);
         tma_load_2d(dst, &tmW, kb * GEMM_BLOCK_K, tile * GEMM_TILE_N, fb, pol_w);
         tma_load_2d(dst + W_TILE_BYTES, &tmHi, kb * GEMM_BLOCK_K, 0, fb, pol_x);
-        tma_load_2d(dst + W_TILE_BYTES + x_bytes, &tmLo, kb * GEMM_BLOCK_K, 0, fb, pol_x);
+        tma_load_2d(dst + W_TILE_BYTES + lo_off, &tmLo, kb * GEMM_BLOCK_K, 0, fb, pol_x);
       }
+      TRACE(3);
     }
   } else if (warp == 1) {
     if (lane == 0) {
@@ -101,33 +140,47 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       for (int g = k0; g < k1 && !fail; ++seg) {
         const int tile = g / KB, kb_begin = g - tile * KB;
         const int kb_end = min(KB, kb_begin + (k1 - g));
-        if (!mbar_wait(smem_u32(&tmem_empty_bar), ((uint32_t)seg & 1u) ^ 1u, abort_p)) { fail = DEV_TIMEOUT_MMA; break; }
+        const int acc = seg % n_acc;
+        const uint32_t use = (uint32_t)(seg / n_acc);     // how often this buffer has been used before
+        if (!mbar_wait(smem_u32(&tmem_empty_bar[acc]), (use & 1u) ^ 1u, abort_p)) { fail = DEV_TIMEOUT_MMA; break; }
         tc_fence_after();
         for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
           const int s = it % stages;
           const uint32_t ph = (uint32_t)(it / stages) & 1u;
           if (!mbar_wait(smem_u32(&full_bar[s]), ph, abort_p)) { fail = DEV_TIMEOUT_MMA; break; }
+          if (it == 0) TRACE(4);
           tc_fence_after();
           const uint32_t w_addr = tiles_base + (uint32_t)s * stage_bytes;
           const uint64_t w_desc = umma_desc_sw128(w_addr);
-          for (int rb = 0; rb < n_rb; ++rb) {
-            const uint64_t hi_desc = umma_desc_sw128(w_addr + W_TILE_BYTES + (uint32_t)rb * A_BLOCK_BYTES);
-            const uint64_t lo_desc = umma_desc_sw128(w_addr + W_TILE_BYTES + x_bytes + (uint32_t)rb * A_BLOCK_BYTES);
-            const uint32_t d_tmem = tmem_base + (uint32_t)rb * GEMM_TILE_N;
+          if (stacked) {
+            const uint64_t a_desc = umma_desc_sw128(w_addr + W_TILE_BYTES);
+            const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_cols;
 #pragma unroll
             for (int k = 0; k < GEMM_BLOCK_K / 16; ++k) {
-              // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in 16-byte units
               const uint64_t adv = (uint64_t)(k * 2);
-              umma_bf16(d_tmem, hi_desc + adv, w_desc + adv, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
-              umma_bf16(d_tmem, lo_desc + adv, w_desc + adv, idesc, 1u);
+              umma_bf16(d_tmem, a_desc + adv, w_desc + adv, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
+            }
+          } else {
+            for (int rb = 0; rb < n_rb; ++rb) {
+              const uint64_t hi_desc = umma_desc_sw128(w_addr + W_TILE_BYTES + (uint32_t)rb * A_BLOCK_BYTES);
+              const uint64_t lo_desc = umma_desc_sw128(w_addr + W_TILE_BYTES + x_bytes + (uint32_t)rb * A_BLOCK_BYTES);
+              const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_cols + (uint32_t)rb * GEMM_TILE_N;
+#pragma unroll
+              for (int k = 0; k < GEMM_BLOCK_K / 16; ++k) {
+                // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in 16-byte units
+                const uint64_t adv = (uint64_t)(k * 2);
+                umma_bf16(d_tmem, hi_desc + adv, w_desc + adv, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
+                umma_bf16(d_tmem, lo_desc + adv, w_desc + adv, idesc, 1u);
+              }
             }
           }
           umma_commit(smem_u32(&empty_bar[s]));   // frees the stage once these MMAs have read it
         }
         if (fail) break;
-        umma_commit(smem_u32(&tmem_full_bar));    // accumulators of this segment are complete
+        umma_commit(smem_u32(&tmem_full_bar[acc]));    // accumulators of this segment are complete
         g += kb_end - kb_begin;
       }
+      TRACE(5);
     }
   } else {
     // ---------------- epilogue: TMEM -> registers -> global ----------------
@@ -137,11 +190,56 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       const int tile = g / KB, kb_begin = g - tile * KB;
       const int kb_end = min(KB, kb_begin + (k1 - g));
       const bool whole = (kb_begin == 0 && kb_end == KB);
-      bool ok = mbar_wait(smem_u32(&tmem_full_bar), (uint32_t)seg & 1u, abort_p);
+      const int acc = seg % n_acc;
+      const uint32_t use = (uint32_t)(seg / n_acc);
+      bool ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), use & 1u, abort_p);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) { fail = DEV_TIMEOUT_EPILOGUE; break; }
       tc_fence_after();
+      if (g + (kb_end - kb_begin) >= k1 && threadIdx.x == 64) TRACE(6);   // last accumulator is ready
       const int n0 = tile * GEMM_TILE_N;
+      if (stacked) {
+        // lanes 0-63 (warps with lane_base 0, 32) hold W*hi of rows 0-63, lanes 64-127 hold W*lo of the
+        // same rows: the lo warps hand their values over through shared memory, 32 columns at a time
+        const bool lo_warp = lane_base >= 64;
+        const int row = (lane_base & 63) + lane;
+        const int rows_valid = whole ? R : BN;
+        const bool warp_needed = (lane_base & 63) < rows_valid;   // warp-uniform
+        const bool row_ok = row < rows_valid;
+        float *dst = whole ? direct + (size_t)row * N + n0
+                           : ws + ((size_t)(cta * 2 + (seg == 0 ? 0 : 1)) * BN + row) * GEMM_TILE_N;
+        const bool vec_ok = whole ? ((N & 3) == 0) : true;
+        for (int c0 = 0; c0 < GEMM_TILE_N; c0 += 32) {
+          if (whole && n0 + c0 >= N) break;          // columns beyond the matrix (last tile); uniform
+          uint32_t v[32];
+          if (warp_needed) {
+            const uint32_t ta = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)acc * acc_cols + (uint32_t)c0;
+            tmem_ld16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+            tmem_ld16(ta + 16, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
+            tmem_ld_wait();
+            if (lo_warp) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) xch[row * 33 + j] = __uint_as_float(v[j]);
+            }
+          }
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          if (warp_needed && !lo_warp && row_ok) {
+            float f[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]) + xch[row * 33 + j];
+            if (vec_ok && (!whole || n0 + c0 + 32 <= N)) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4 *>(dst + c0 + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (n0 + c0 + j < N) dst[c0 + j] = f[j];
+            }
+          }
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+      } else
       for (int rb = 0; rb < n_rb; ++rb) {
         const int row_base = rb * GEMM_ROW_BLOCK + lane_base;
         const int rows_valid = whole ? R : BN;      // partials keep the padded row count
@@ -154,7 +252,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         for (int c0 = 0; c0 < GEMM_TILE_N; c0 += 16) {
           if (whole && n0 + c0 >= N) break;          // columns beyond the matrix (last tile)
           uint32_t v[16];
-          tmem_ld16(tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)(rb * GEMM_TILE_N + c0), v);
+          tmem_ld16(tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)acc * acc_cols + (uint32_t)(rb * GEMM_TILE_N + c0), v);
           tmem_ld_wait();
           if (!row_ok) continue;
           if (vec_ok && (!whole || n0 + c0 + 16 <= N)) {
@@ -171,9 +269,10 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         }
       }
       tc_fence_before();
-      mbar_arrive(smem_u32(&tmem_empty_bar));
+      mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
       g += kb_end - kb_begin;
     }
+    if (threadIdx.x == 64) TRACE(7);
   }
 
   if (fail) {
@@ -188,6 +287,8 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 }
 
 __global__ void __launch_bounds__(GEMM_TILE_N) gemm_fixup_kernel(GemmOut g, float *direct, const int *split_tiles) {
+  griddep_launch_dependents();
+  griddep_wait();
   const int t = split_tiles[blockIdx.x], r = blockIdx.y;
   const int n = t * GEMM_TILE_N + threadIdx.x;
   if (n < g.N) direct[(size_t)r * g.N + n] = gemm_load(g, r, n);
@@ -237,9 +338,9 @@ int gemm_plan_fill(GemmPlan *p, const void *W, int N, int K, const void *Xhi, co
   const long long total = (long long)p->n_tiles * p->KB;
   p->grid = (int)(total < num_sms ? total : num_sms);
   if (total * (long long)p->grid >= (1ll << 31)) return CORUN_EINVAL;
-  const size_t stage = (size_t)W_TILE_BYTES + 2 * (size_t)BN * GEMM_BLOCK_K * 2;
+  const size_t stage = (size_t)W_TILE_BYTES + (BN <= 64 ? (size_t)A_BLOCK_BYTES : 2 * (size_t)BN * GEMM_BLOCK_K * 2);
   // the MMA always reads 128 activation rows: leave that much readable behind the last stage
-  int stages = (int)((220 * 1024 - 1024 - A_BLOCK_BYTES) / stage);
+  int stages = (int)((216 * 1024 - 1024 - A_BLOCK_BYTES) / stage);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (const char *ev = getenv("CORUN_GEMM_STAGES")) {   // experiments only: shallower ring
     const int v = atoi(ev);
@@ -248,7 +349,7 @@ int gemm_plan_fill(GemmPlan *p, const void *W, int N, int K, const void *Xhi, co
   if (stages < 2) return CORUN_EINVAL;
   p->stages = stages;
   p->smem_bytes = stage * stages + A_BLOCK_BYTES + 1024;
-  p->tmem_cols = BN > GEMM_ROW_BLOCK ? 512 : 256;
+  p->tmem_cols = 512;   // two accumulator buffers (<= 128 rows) or two row blocks
   // kind::f16 instruction descriptor: D fp32 (bits 4-5 = 1), A and B bf16 (bits 7-9, 10-12 = 1),
   // both K-major (bits 15, 16 = 0), N >> 3 at bits 17-22, M >> 4 at bits 24-28.
   p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GEMM_TILE_N >> 3) << 17) |
@@ -304,7 +405,7 @@ int gemm_plan_create(GemmPlan *p, const void *W, int N, int K, const void *Xhi, 
 }
 
 cudaError_t gemm_prepare_kernel() {
-  return cudaFuncSetAttribute(gemm_streamk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 221 * 1024);
+  return cudaFuncSetAttribute(gemm_streamk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 216 * 1024);
 }
 
 void gemm_plan_destroy(GemmPlan *p) {
@@ -312,17 +413,17 @@ void gemm_plan_destroy(GemmPlan *p) {
   p->d_cta_start = nullptr;
 }
 
-cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int *d_status, cudaStream_t st) {
-  gemm_streamk_kernel<<<p.grid, GEMM_THREADS, p.smem_bytes, st>>>(tmW_override ? *tmW_override : p.tmW, p.tmHi, p.tmLo,
-                                                                  p.direct, p.ws, p.d_cta_start, p.N, p.KB, p.BN, p.R,
-                                                                  p.stages, p.tmem_cols, p.idesc, d_status);
-  return cudaGetLastError();
+cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int *d_status, cudaStream_t st,
+                        unsigned long long *trace, bool pdl) {
+  return launch_k(gemm_streamk_kernel, dim3(p.grid), dim3(GEMM_THREADS), p.smem_bytes, st, pdl,
+                  tmW_override ? *tmW_override : p.tmW, p.tmHi, p.tmLo, p.direct, p.ws, p.d_cta_start, p.N, p.KB, p.BN,
+                  p.R, p.stages, p.tmem_cols, p.idesc, d_status, trace);
 }
 
-cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st) {
+cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st, bool pdl) {
   if (p.n_split_tiles == 0) return cudaSuccess;
-  gemm_fixup_kernel<<<dim3(p.n_split_tiles, p.R), GEMM_TILE_N, 0, st>>>(p.out(), p.direct, p.d_split_tiles);
-  return cudaGetLastError();
+  return launch_k(gemm_fixup_kernel, dim3(p.n_split_tiles, p.R), dim3(GEMM_TILE_N), 0, st, pdl, p.out(), p.direct,
+                  p.d_split_tiles);
 }
 
 }  // namespace corun

@@ -103,7 +103,9 @@ int gemm_plan_fill(GemmPlan *p, const void *W, int N, int K, const void *Xhi, co
 void gemm_plan_bind_tables(GemmPlan *p, int *d_tab);
 // Enqueues the GEMM.  `W` may override the weight matrix of the plan (same
 // shape) by passing a different tensor map.
-cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int *d_status, cudaStream_t st);
+cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int *d_status, cudaStream_t st,
+                        unsigned long long *trace = nullptr,   // optional [grid][8] globaltimer stamps (debug)
+                        bool pdl = false);                     // programmatic dependent launch (row program)
 // Encodes a tensor map for a bf16 [rows, K] row-major matrix with a [box_rows, 64] box, 128-byte swizzle.
 int gemm_encode_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows);
 // Opts the GEMM kernel into its dynamic shared-memory size (idempotent, allocates nothing).
@@ -112,6 +114,6 @@ cudaError_t gemm_prepare_kernel();
 int tma_encode_2d(CUtensorMap *m, const void *base, int is_fp16, unsigned long long rows, int cols, int box_rows,
                   int box_cols);
 // direct[r, n] = gemm_load(r, n) for every tile that has partials (makes `direct` a plain matrix).
-cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st);
+cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st, bool pdl = false);
 
 }  // namespace corun

@@ -4,6 +4,9 @@
 // that depends on the row's own data and the model shape only; no float atomics.
 #include "ops.cuh"
 
+#include "launch.cuh"
+#include "ptx.cuh"
+
 #include <math_constants.h>
 
 namespace corun {
@@ -34,6 +37,8 @@ __global__ void __launch_bounds__(NORM_MAX_THREADS)
 resid_norm_kernel(float *__restrict__ h, int H, const __nv_bfloat16 *__restrict__ embed, Rows rows, GemmOut prev,
                   int first, const __nv_bfloat16 *__restrict__ gains, float eps, __nv_bfloat16 *__restrict__ out_hi,
                   __nv_bfloat16 *__restrict__ out_lo) {
+  griddep_launch_dependents();
+  griddep_wait();
   __shared__ float scratch[NORM_MAX_THREADS / 32];
   const int r = blockIdx.x;
   float *hr = h + (size_t)r * H;
@@ -80,6 +85,8 @@ resid_norm_kernel(float *__restrict__ h, int H, const __nv_bfloat16 *__restrict_
 __global__ void __launch_bounds__(64)
 qkv_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, int nq, KvLayout kv, int layer,
                 float *__restrict__ q_out) {
+  griddep_launch_dependents();
+  griddep_wait();
   const int head = blockIdx.x, r = blockIdx.y, i = threadIdx.x;
   const int hd = kv.hd, half = hd >> 1, nkv = kv.n_kv;
   const int pos = rows.pos[r];
@@ -112,6 +119,8 @@ qkv_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, int
 // ---------------------------------------------------------------- SwiGLU
 __global__ void __launch_bounds__(256)
 swiglu_kernel(GemmOut gu, int F, __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo) {
+  griddep_launch_dependents();
+  griddep_wait();
   const int r = blockIdx.y;
   const int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i >= F) return;
@@ -246,6 +255,8 @@ __device__ void smp_select_bin(SmpShared &sh, unsigned long long cut) {
 }
 
 __global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
+  griddep_launch_dependents();
+  griddep_wait();
   const int r = blockIdx.x;
   if (!a.do_sample[r]) return;
   __shared__ SmpShared sh;
@@ -389,6 +400,8 @@ __global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
 __global__ void prepare_rows_kernel(const uint8_t *active_mask, const int *in_use, const int *ctx_len,
                                     const int *pending, int B, int *row_token, int *row_pos, int *row_active,
                                     int *row_slot, int *do_sample) {
+  griddep_launch_dependents();
+  griddep_wait();
   const int s = blockIdx.x * blockDim.x + threadIdx.x;
   if (s >= B) return;
   const int act = (active_mask[s] != 0 && in_use[s] != 0) ? 1 : 0;
@@ -401,6 +414,8 @@ __global__ void prepare_rows_kernel(const uint8_t *active_mask, const int *in_us
 
 __global__ void advance_kernel(const int *row_active, const int *sampled, int B, int *ctx_len, int *step, int *pending,
                                int *out_tokens) {
+  griddep_launch_dependents();
+  griddep_wait();
   const int s = blockIdx.x * blockDim.x + threadIdx.x;
   if (s >= B) return;
   if (row_active[s]) {
@@ -472,19 +487,18 @@ cudaError_t launch_resid_norm(float *h, int H, const __nv_bfloat16 *embed, const
   int threads = H / 4;
   if (threads > NORM_MAX_THREADS) threads = NORM_MAX_THREADS;
   threads = (threads + 31) / 32 * 32;
-  resid_norm_kernel<<<rows.R, threads, 0, st>>>(h, H, embed, rows, g, prev ? 0 : 1, gains, eps, out_hi, out_lo);
-  return cudaGetLastError();
+  return launch_k(resid_norm_kernel, dim3(rows.R), dim3(threads), 0, st, true, h, H, embed, rows, g, prev ? 0 : 1, gains,
+                  eps, out_hi, out_lo);
 }
 
 cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *rope_tab, int nq, const KvLayout &kv,
                             int layer, float *q_out, cudaStream_t st) {
-  qkv_post_kernel<<<dim3(nq + 2 * kv.n_kv, rows.R), kv.hd / 2, 0, st>>>(qkv, rows, rope_tab, nq, kv, layer, q_out);
-  return cudaGetLastError();
+  return launch_k(qkv_post_kernel, dim3(nq + 2 * kv.n_kv, rows.R), dim3(kv.hd / 2), 0, st, true, qkv, rows, rope_tab, nq,
+                  kv, layer, q_out);
 }
 
 cudaError_t launch_swiglu(const GemmOut &gu, int R, int F, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, cudaStream_t st) {
-  swiglu_kernel<<<dim3((F / 4 + 255) / 256, R), 256, 0, st>>>(gu, F, out_hi, out_lo);
-  return cudaGetLastError();
+  return launch_k(swiglu_kernel, dim3((F / 4 + 255) / 256, R), dim3(256), 0, st, true, gu, F, out_hi, out_lo);
 }
 
 cudaError_t launch_split(const float *x, int R, int K, __nv_bfloat16 *hi, __nv_bfloat16 *lo, cudaStream_t st) {
@@ -493,9 +507,8 @@ cudaError_t launch_split(const float *x, int R, int K, __nv_bfloat16 *hi, __nv_b
   return cudaGetLastError();
 }
 
-cudaError_t launch_sampler(const SampleArgs &a, int R, cudaStream_t st) {
-  sampler_kernel<<<R, SMP_THREADS, 0, st>>>(a);
-  return cudaGetLastError();
+cudaError_t launch_sampler(const SampleArgs &a, int R, cudaStream_t st, bool pdl) {
+  return launch_k(sampler_kernel, dim3(R), dim3(SMP_THREADS), 0, st, pdl, a);
 }
 
 cudaError_t launch_prepare_rows(const uint8_t *active_mask, const int *in_use, const int *ctx_len, const int *pending,
@@ -508,8 +521,8 @@ cudaError_t launch_prepare_rows(const uint8_t *active_mask, const int *in_use, c
 
 cudaError_t launch_advance(const int *row_active, const int *sampled, int B, int *ctx_len, int *step, int *pending,
                            int *out_tokens, cudaStream_t st) {
-  advance_kernel<<<(B + 127) / 128, 128, 0, st>>>(row_active, sampled, B, ctx_len, step, pending, out_tokens);
-  return cudaGetLastError();
+  return launch_k(advance_kernel, dim3((B + 127) / 128), dim3(128), 0, st, true, row_active, sampled, B, ctx_len, step,
+                  pending, out_tokens);
 }
 
 cudaError_t launch_kv_copy(const KvLayout &kv, int layer, int slot, int pos0, int n, float *k, float *v, int write,

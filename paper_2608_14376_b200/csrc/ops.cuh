@@ -52,15 +52,19 @@ cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *
                             int layer, float *q_out, cudaStream_t st);
 // Split-KV paged attention partials and their fixed-order combine -> bf16 hi/lo [R, nq*hd].
 // tmKV: tensor map over the whole pool as [all cached rows, hd] fp16 with a [16, 64] box (see attention.cu).
+// work / n_work: the step's (row, split) items from launch_attn_worklist (the same for every layer);
+// grid_ctas: persistent CTAs to launch (3 per SM).
 cudaError_t launch_attention(const CUtensorMap &tmKV, const float *q, const Rows &rows, int nq, const KvLayout &kv,
-                             int layer, int max_splits, float *part_acc, float *part_ml, __nv_bfloat16 *out_hi,
-                             __nv_bfloat16 *out_lo, int *d_status, cudaStream_t st);
+                             int layer, int max_splits, const int *work, const int *n_work, int grid_ctas,
+                             float *part_acc, float *part_ml, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
+                             int *d_status, cudaStream_t st);
+cudaError_t launch_attn_worklist(const Rows &rows, int *work, int *n_work, cudaStream_t st);
 cudaError_t attention_prepare();   // opts the kernels into their shared-memory size (idempotent)
 // y = silu(gate) * up from the gate-up GEMM result -> bf16 hi/lo [R, F].
 cudaError_t launch_swiglu(const GemmOut &gu, int R, int F, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, cudaStream_t st);
 // x fp32 [R, K] -> bf16 hi/lo.
 cudaError_t launch_split(const float *x, int R, int K, __nv_bfloat16 *hi, __nv_bfloat16 *lo, cudaStream_t st);
-cudaError_t launch_sampler(const SampleArgs &a, int R, cudaStream_t st);
+cudaError_t launch_sampler(const SampleArgs &a, int R, cudaStream_t st, bool pdl = false);
 // decode bookkeeping
 cudaError_t launch_prepare_rows(const uint8_t *active_mask, const int *in_use, const int *ctx_len, const int *pending,
                                 int B, int *row_token, int *row_pos, int *row_active, int *row_slot, int *do_sample,
