@@ -88,6 +88,17 @@ def case_kernels(a):
             names = ["entry", "setup", "tma0", "tmaN", "land0", "mmaN", "accN", "done"]
             print(eng.KERNEL_KINDS[kind], "timeline (us, median / max over CTAs):",
                   "  ".join("%s %.2f/%.2f" % (n, np.median(t[:, i]) / 1e3, t[:, i].max() / 1e3) for i, n in enumerate(names)))
+        t = eng.attn_trace(1)
+        ok = t[:, :, 3] > 0
+        t0 = t[:, :, 0][ok].min()
+        load = (t[:, :, 1] - t[:, :, 0])[ok] / 1e3
+        wait = (t[:, :, 2] - t[:, :, 0])[ok] / 1e3
+        hold = (t[:, :, 3] - t[:, :, 2])[ok] / 1e3
+        stall = (t[:, :, 1] - t[:, :, 2])[ok] / 1e3
+        print("attention items: %d; load issue->landed median %.2f us (p90 %.2f); group start->release median %.2f us "
+              "(p90 %.2f); of which waiting for the data median %.2f us; issue->group start median %.2f; span %.1f us"
+              % (ok.sum(), np.median(load), np.percentile(load, 90), np.median(hold), np.percentile(hold, 90),
+                 np.median(np.maximum(stall, 0)), np.median(wait), (t[:, :, 3][ok].max() - t0) / 1e3))
     eng.close()
 
 

@@ -1,20 +1,23 @@
-// Request-local split-KV paged attention for one query token per row.
+// Request-local split-KV paged attention for one query token per row, on tcgen05.
 //
-// A CTA owns (row, kv head, split of 128 cached tokens = 8 pages).  One thread
-// issues TMA tile loads for the split's K and V pages ([16 tokens x 64 dims]
-// boxes, 128-byte swizzle, straight from the page pool through one tensor map)
-// and each of the 4 warps consumes its own quarter (2 pages) as soon as its
-// mbarrier completes.  Scores and weighted values run on the tensor cores
-// (mma.sync m16n8k16, fp16 inputs, fp32 accumulate): the cached K/V are fp16
-// exactly; the query rows and the softmax weights enter as an fp16 hi/lo pair
-// (x = hi + lo, 22 significand bits) stacked in the 16 rows of the A operand:
-// rows 0..G-1 hold hi of the G query heads of this kv head, rows 8..8+G-1
-// their lo parts, so both halves land in the same thread and are added there.
+// An item is (row, split of 128 cached tokens = 8 pages, kv head).  One persistent CTA per SM:
+//   warp 0        streams items with TMA into a ring of 3 item buffers (keys: [16 tokens x 64 dims]
+//                 boxes, 128-byte swizzle; values, cached transposed: [hd dims x 16 tokens] boxes,
+//                 32-byte swizzle), straight from the page pool through two tensor maps per layer;
+//   2 groups of 4 warps take the items alternately.  Per item a group
+//     1. writes the query rows as fp16 hi/lo pairs into a [16 x hd] operand tile (rows 0..G-1 hi of
+//        the G query heads of this kv head, rows 8..8+G-1 their lo parts; q = hi + lo, 22 bits),
+//     2. S^T[128 tokens x 16] = K[128 x hd] * Q^T       (tcgen05.mma, M = 128, N = 16, K = 16 per step)
+//        -> TMEM lane = token, so each of the 128 threads owns one cached token,
+//     3. softmax over the item: exact max and a fixed-order sum over the 128 tokens,
+//        weights written as fp16 hi/lo rows of a [16 x 128 tokens] operand tile,
+//     4. O^T[hd dims x 16] = V^T[hd x 128 tokens] * P^T  (one MMA per page), TMEM lane = dim,
+//     5. adds the hi and lo columns and writes the split's partial (max, sum, O) to global memory.
+// The cached K / V are fp16 exactly, accumulation is fp32.
 //
-// Invariance: the split size is fixed, the split count is a function of the
-// row's own context length, each warp walks its pages in ascending order with
-// an online softmax, the 4 warps are merged in ascending order and the splits
-// are combined in ascending order by one owner.  Nothing depends on other rows.
+// Invariance: the split size is fixed, the split count is a function of the row's own context
+// length, every reduction inside an item has one fixed order, and the splits are combined in
+// ascending order by one owner.  The work list only decides which CTA computes an item.
 #include <cuda_fp16.h>
 #include <math_constants.h>
 
@@ -26,247 +29,316 @@ namespace corun {
 
 namespace {
 
-constexpr int ATT_THREADS = 128;
-constexpr int ATT_PAGES = ATT_SPLIT / KV_BLOCK;   // 8 pages per split
-constexpr int BOX_BYTES = KV_BLOCK * 128;         // one [16 x 64] fp16 box
+constexpr int ATT_NBUF = 3;                        // item buffers in the ring
+constexpr int ATT_GROUPS = 2;                      // consumer groups of 4 warps
+constexpr int ATT_SLOTS = 6;                       // barrier slots: a multiple of both
+constexpr int ATT_THREADS = 32 + ATT_GROUPS * 128; // producer warp + consumers
+constexpr int ATT_PAGES = ATT_SPLIT / KV_BLOCK;    // 8 pages per split
+constexpr int KBOX_BYTES = KV_BLOCK * 128;         // one [16 tokens x 64 dims] fp16 key box
+constexpr int OPND_BYTES = 16 * 128;               // one [16 rows x 64 cols] fp16 half of a q / p operand tile
+constexpr uint32_t ATT_TMEM_COLS = 64;             // per group: 16 columns of S^T and 16 of O^T
 
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-               : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-               : "r"(addr));
-}
-// D += A(16x16, row) * B(16x8, col), fp16 inputs, fp32 accumulate
-__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack_half2(__half a, __half b) {
-  return (uint32_t)__half_as_ushort(a) | ((uint32_t)__half_as_ushort(b) << 16);
-}
+// byte offset of 16-byte chunk `chunk` of row `row` inside a 128-byte-swizzled tile of 128-byte rows
+__device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
+
 // x = hi + lo with hi, lo fp16
 __device__ __forceinline__ void split_half(float x, __half &hi, __half &lo) {
   hi = __float2half_rn(x);
   lo = __float2half_rn(x - __half2float(hi));
 }
-// byte offset of 16-byte chunk `chunk` of row `row` inside a 128-byte-swizzled [16 x 128 B] box
-__device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
 
 template <int HD>
-__global__ void __launch_bounds__(ATT_THREADS)
-attn_split_kernel(const __grid_constant__ CUtensorMap tmKV, const float *__restrict__ q, Rows rows, int nq, int group,
-                  KvLayout kv, int layer, int max_splits, const int *__restrict__ work, const int *__restrict__ n_work,
-                  float *__restrict__ part_acc, float *__restrict__ part_ml, int *status) {
-  constexpr int NBOX = HD / 64;                  // boxes per (page, head) tile
-  constexpr int TILE_BYTES = NBOX * BOX_BYTES;   // K (or V) of one page and head
-  constexpr int KSTEPS = HD / 16;                // k-steps of the score MMA
-  constexpr int NT = HD / 8;                     // n-tiles of the value MMA
+struct AttLayout {
+  static constexpr int NHALF = HD / 64;                          // 64-dim halves of a key row
+  static constexpr int K_BYTES = NHALF * ATT_PAGES * KBOX_BYTES; // keys of an item: [half][page][16 x 128 B]
+  static constexpr int VT_BYTES = HD * KV_BLOCK * 2;             // one page's V^T tile: [hd x 32 B]
+  static constexpr int ITEM_BYTES = K_BYTES + ATT_PAGES * VT_BYTES;
+  static constexpr int Q_BYTES = NHALF * OPND_BYTES;             // [half][16 x 128 B]
+  static constexpr int P_BYTES = 2 * OPND_BYTES;                 // 128 tokens = 2 halves of 64
+  static constexpr int GROUP_BYTES = Q_BYTES + P_BYTES;
+  // the value MMA always reads 128 rows of V^T (M = 128): with hd = 64 that runs into what follows
+  static constexpr int PAD_BYTES = (HD < 128) ? 128 * KV_BLOCK * 2 : 0;
+  static constexpr size_t SMEM = (size_t)ATT_NBUF * ITEM_BYTES + ATT_GROUPS * GROUP_BYTES + PAD_BYTES + 1024;
+};
+
+template <int HD>
+__global__ void __launch_bounds__(ATT_THREADS, 1)
+attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                  const float *__restrict__ q, Rows rows, int nq, int group, KvLayout kv, int max_splits,
+                  const int *__restrict__ work, const int *__restrict__ n_work, float *__restrict__ part_acc,
+                  float *__restrict__ part_ml, int *status, unsigned long long *trace) {
+  using L = AttLayout<HD>;
+  // optional timeline (debug): per CTA and item (first 64): [load issued, item landed, group starts, released]
+#define ATRACE(k, i) do { if (trace && (k) < 64) trace[((size_t)blockIdx.x * 64 + (k)) * 4 + (i)] = globaltimer_ns(); } while (0)
+  constexpr int KSTEPS = HD / 16;
   griddep_launch_dependents();
   griddep_wait();                                // the item list and q come from earlier kernels
-  // persistent CTAs walk the step's list of (row, split) items x kv heads with a fixed stride; the
-  // list only decides which CTA computes an item, never how it is computed
   const int n_items = *n_work * kv.n_kv;
   if ((int)blockIdx.x >= n_items) return;
 
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bar[4];
-  __shared__ int page_s[ATT_PAGES];
+  __shared__ __align__(8) uint64_t full_bar[ATT_SLOTS];
+  __shared__ __align__(8) uint64_t empty_bar[ATT_NBUF];
+  __shared__ __align__(8) uint64_t mma_bar[ATT_GROUPS];
+  __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
-  const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;     // K tiles, then V tiles
-  const uint32_t v_tiles = tiles + ATT_PAGES * TILE_BYTES;
+  __shared__ int stop_s[ATT_GROUPS];             // group-uniform copy of abort_flag, refreshed once per item
+  __shared__ float red_s[ATT_GROUPS][4][8];      // cross-warp softmax reductions
+  const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *ring_ptr = smem_raw + (ring - smem_u32(smem_raw));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     abort_flag = 0;
-    for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bar[w]), 1);
+    for (int g = 0; g < ATT_GROUPS; ++g) { stop_s[g] = 0; mbar_init(smem_u32(&mma_bar[g]), 1); }
+    for (int s = 0; s < ATT_SLOTS; ++s) mbar_init(smem_u32(&full_bar[s]), 1);
+    for (int b = 0; b < ATT_NBUF; ++b) mbar_init(smem_u32(&empty_bar[b]), 1);
     fence_mbar_init();
     fence_proxy_async();
   }
+  if (warp == 0) {
+    tmem_alloc(smem_u32(&tmem_base_s), ATT_TMEM_COLS);
+    tmem_relinquish();
+  } else {
+    // operand tiles start out as zeros: rows of unused heads are never written and must stay finite
+    uint4 *z = reinterpret_cast<uint4 *>(ring_ptr + (size_t)ATT_NBUF * L::ITEM_BYTES);
+    for (int i = tid - 32; i < ATT_GROUPS * L::GROUP_BYTES / 16; i += ATT_THREADS - 32) z[i] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
   bool failed = false;
-  uint32_t parity = 0;                           // phase of this warp's barrier: flips each time it is armed
-  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-  const int wi = work[item / kv.n_kv], g = item % kv.n_kv;
-  const int r = wi >> 8, split = wi & 255;
-  const int ctx = rows.pos[r] + 1;               // the new token attends to itself too
-  const int t0 = split * ATT_SPLIT;
-  const int n_pages = min(ATT_PAGES, (ctx - t0 + KV_BLOCK - 1) / KV_BLOCK);
-  __syncthreads();                               // the previous item's merge buffers (tile memory) are free
-  if (tid < ATT_PAGES)
-    page_s[tid] = tid < n_pages ? kv.block_table[(size_t)rows.slot[r] * kv.max_blocks + t0 / KV_BLOCK + tid] : 0;
-  __syncthreads();
-  if (tid == 0) {
+  // instruction descriptor: D fp32 (bits 4-5 = 1), A and B fp16 (0), K-major, N = 16 (N >> 3 at bit 17),
+  // M = 128 (M >> 4 at bit 24)
+  const uint32_t idesc = (1u << 4) | ((uint32_t)(16 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+
+  if (warp == 0) {
+    // ---------------- producer: one lane per page ----------------
     const uint64_t pol = l2_policy_evict_first();       // the cache is streamed once per step
-    for (int w = 0; w < 4; ++w) {
-      const int np = min(2, n_pages - 2 * w);
-      if (np <= 0) break;
-      const uint32_t b = smem_u32(&bar[w]);
-      mbar_arrive_expect_tx(b, (uint32_t)(np * 2 * TILE_BYTES));
-      for (int p = 2 * w; p < 2 * w + np; ++p) {
-        // pool rows: (((layer * pool_blocks + page) * 2 + k|v) * n_kv + head) * 16 + token
-        const long long base = ((long long)layer * kv.pool_blocks + page_s[p]) * 2;
-        const int row_k = (int)(((base + 0) * kv.n_kv + g) * KV_BLOCK);
-        const int row_v = (int)(((base + 1) * kv.n_kv + g) * KV_BLOCK);
+    int k = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++k) {
+      const int buf = k % ATT_NBUF, slot = k % ATT_SLOTS;
+      if (k >= ATT_NBUF) {                               // the buffer's previous item must have been released
+        bool ok = mbar_wait(smem_u32(&empty_bar[buf]), (uint32_t)(k / ATT_NBUF - 1) & 1u, &abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { failed = true; break; }
+      }
+      const int wi = work[item / kv.n_kv], g = item % kv.n_kv;
+      const int r = wi >> 8, split = wi & 255;
+      const int ctx = rows.pos[r] + 1;
+      const int t0 = split * ATT_SPLIT;
+      const int n_pages = min(ATT_PAGES, (ctx - t0 + KV_BLOCK - 1) / KV_BLOCK);
+      const uint32_t fb = smem_u32(&full_bar[slot]);
+      if (lane == 0) { ATRACE(k, 0); mbar_arrive_expect_tx(fb, (uint32_t)(n_pages * (L::NHALF * KBOX_BYTES + L::VT_BYTES))); }
+      __syncwarp();
+      if (lane < n_pages) {
+        const int page = kv.block_table[(size_t)rows.slot[r] * kv.max_blocks + t0 / KV_BLOCK + lane];
+        // this layer's pages as rows of hd halfs: the key tile of (page, head) starts at row
+        //   page * 2 * n_kv * 16 + head * 16;
+        // as rows of 16 halfs: the transposed value tile starts at row page * 2 * n_kv * hd + (n_kv + head) * hd
+        const int row_k = (page * 2 * kv.n_kv + g) * KV_BLOCK;
+        const int row_v = (page * 2 * kv.n_kv + kv.n_kv + g) * HD;
+        const uint32_t item_base = ring + (uint32_t)buf * L::ITEM_BYTES;
 #pragma unroll
-        for (int x = 0; x < NBOX; ++x) {
-          tma_load_2d(tiles + p * TILE_BYTES + x * BOX_BYTES, &tmKV, x * 64, row_k, b, pol);
-          tma_load_2d(v_tiles + p * TILE_BYTES + x * BOX_BYTES, &tmKV, x * 64, row_v, b, pol);
-        }
+        for (int x = 0; x < L::NHALF; ++x)
+          tma_load_2d(item_base + (uint32_t)(x * ATT_PAGES + lane) * KBOX_BYTES, &tmK, x * 64, row_k, fb, pol);
+        tma_load_2d(item_base + L::K_BYTES + (uint32_t)lane * L::VT_BYTES, &tmV, 0, row_v, fb, pol);
       }
     }
-  }
-
-  // ---- query rows as A fragments: rows 0..G-1 hi, rows 8..8+G-1 lo (raw q; the scale goes on the scores)
-  const int qrow = lane >> 2;                    // fragment row of this lane (and of its +8 partner)
-  const bool row_used = qrow < group;
-  uint32_t qa[KSTEPS][4];
-  {
-    const float *qp = q + (size_t)r * nq * HD + (size_t)(g * group + (row_used ? qrow : 0)) * HD + (lane & 3) * 2;
+  } else {
+    // ---------------- consumers ----------------
+    const int gi = (warp - 1) >> 2, gtid = (tid - 32) & 127;
+    const int quad = warp & 3;                     // the TMEM lane quarter this warp may read
+    const int tl = quad * 32 + lane;               // TMEM lane of this thread: token (scores) / dim (values)
+    const float sscale = (HD == 128 ? 0.08838834764831845f : 0.125f) * 1.4426950408889634f;   // log2(e)/sqrt(hd)
+    const uint32_t q_tile = ring + ATT_NBUF * L::ITEM_BYTES + (uint32_t)gi * L::GROUP_BYTES;
+    const uint32_t p_tile = q_tile + L::Q_BYTES;
+    uint8_t *q_ptr = ring_ptr + (size_t)ATT_NBUF * L::ITEM_BYTES + (size_t)gi * L::GROUP_BYTES;
+    uint8_t *p_ptr = q_ptr + L::Q_BYTES;
+    const uint32_t s_tmem = tmem_base + (uint32_t)gi * 32;       // S^T: 16 columns
+    const uint32_t o_tmem = s_tmem + 16;                          // O^T: 16 columns
+    const uint32_t mbar = smem_u32(&mma_bar[gi]);
+    uint32_t mma_phase = 0, full_bits = 0;         // bit j: phase of the full barrier of this group's j-th slot
+    constexpr int QPT = (8 * (HD / 2) + 127) / 128;   // float2 query values per thread (up to 8 heads)
+    float2 qreg[QPT];
+    auto load_q = [&](int r_, int g_) {
 #pragma unroll
-    for (int ks = 0; ks < KSTEPS; ++ks) {
-      float2 x0 = make_float2(0.f, 0.f), x1 = make_float2(0.f, 0.f);
-      if (row_used) {
-        x0 = *reinterpret_cast<const float2 *>(qp + ks * 16);
-        x1 = *reinterpret_cast<const float2 *>(qp + ks * 16 + 8);
-      }
-      __half h0, l0, h1, l1, h2, l2, h3, l3;
-      split_half(x0.x, h0, l0); split_half(x0.y, h1, l1);
-      split_half(x1.x, h2, l2); split_half(x1.y, h3, l3);
-      qa[ks][0] = pack_half2(h0, h1);   // (row, k..k+1)      hi
-      qa[ks][1] = pack_half2(l0, l1);   // (row + 8, k..k+1)  lo
-      qa[ks][2] = pack_half2(h2, h3);   // (row, k+8..k+9)    hi
-      qa[ks][3] = pack_half2(l2, l3);   // (row + 8, ...)     lo
-    }
-  }
-  const float sscale = (HD == 128 ? 0.08838834764831845f : 0.125f) * 1.4426950408889634f;   // log2(e)/sqrt(hd)
-
-  float o[NT][4];
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
-  float m_run = -CUDART_INF_F, l_run = 0.f;
-
-  const int warp_t0 = t0 + warp * 32;
-  if (warp_t0 < ctx) {
-    bool ok = mbar_wait(smem_u32(&bar[warp]), parity, &abort_flag);
-    ok = __all_sync(0xffffffffu, ok);
-    parity ^= 1u;                                // armed exactly when this warp has tokens (warp_t0 < ctx)
-    if (!ok) {
-      failed = true;
-    } else {
-      // ldmatrix lane roles: matrix mi = lane / 8, row inside it = lane % 8
-      const int mi = lane >> 3, mr = lane & 7;
-      for (int step = 0; step < 2; ++step) {
-        const int p = warp * 2 + step;
-        const int tok0 = t0 + p * KV_BLOCK;
-        if (tok0 >= ctx) break;                                   // warp-uniform
-        const uint32_t kt = tiles + p * TILE_BYTES, vt = v_tiles + p * TILE_BYTES;
-        // ---- scores S[16 x 16 tokens]: two n-tiles of 8 tokens
-        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int ks = 0; ks < KSTEPS; ++ks) {
-          // matrices: (tokens 0-7, dims lo), (tokens 0-7, dims hi), (tokens 8-15, dims lo), (tokens 8-15, dims hi)
-          const int row = (mi >> 1) * 8 + mr;
-          const int chunk = (ks & 3) * 2 + (mi & 1);
-          uint32_t b0, b1, b2, b3;
-          ldsm_x4(kt + (ks >> 2) * BOX_BYTES + swz(row, chunk), b0, b1, b2, b3);
-          mma16816(s0, qa[ks], b0, b1);
-          mma16816(s1, qa[ks], b2, b3);
-        }
-        // this lane: head `qrow`, tokens tok0 + (lane&3)*2 + {0,1} (n-tile 0) and + 8 (n-tile 1); hi + lo rows
-        float sc[4];
-        sc[0] = (s0[0] + s0[2]) * sscale; sc[1] = (s0[1] + s0[3]) * sscale;
-        sc[2] = (s1[0] + s1[2]) * sscale; sc[3] = (s1[1] + s1[3]) * sscale;
-        const int tk = tok0 + (lane & 3) * 2;
-        if (tk >= ctx) sc[0] = -CUDART_INF_F;
-        if (tk + 1 >= ctx) sc[1] = -CUDART_INF_F;
-        if (tk + 8 >= ctx) sc[2] = -CUDART_INF_F;
-        if (tk + 9 >= ctx) sc[3] = -CUDART_INF_F;
-        float mx = fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3]));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));      // max over the 16 tokens of this row
-        const float m_new = fmaxf(m_run, mx);                      // finite: token tok0 is valid
-        const float alpha = exp2f(m_run - m_new);                  // 0 on the first step
-        float pr[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) pr[i] = exp2f(sc[i] - m_new);
-        l_run = l_run * alpha + ((pr[0] + pr[1]) + (pr[2] + pr[3]));   // this lane's tokens; lanes are added at the end
-        m_run = m_new;
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          o[nt][0] *= alpha; o[nt][1] *= alpha; o[nt][2] *= alpha; o[nt][3] *= alpha;
-        }
-        __half ph[4], pl[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) split_half(pr[i], ph[i], pl[i]);
-        uint32_t pa[4];
-        pa[0] = pack_half2(ph[0], ph[1]);   // (row, tokens 0-7 pair)      hi
-        pa[1] = pack_half2(pl[0], pl[1]);   // (row + 8, ...)              lo
-        pa[2] = pack_half2(ph[2], ph[3]);   // (row, tokens 8-15 pair)     hi
-        pa[3] = pack_half2(pl[2], pl[3]);   // (row + 8, ...)              lo
-        // ---- weighted values O[16 x HD] += P[16 x 16 tokens] * V[16 tokens x HD]
-#pragma unroll
-        for (int np = 0; np < NT / 2; ++np) {
-          // matrices: (tokens 0-7, dims d0..d0+7), (tokens 8-15, same dims), (tokens 0-7, d0+8..), (tokens 8-15, d0+8..)
-          const int row = (mi & 1) * 8 + mr;
-          const int chunk = ((np * 2) & 7) + (mi >> 1);
-          uint32_t b0, b1, b2, b3;
-          ldsm_x4_trans(vt + ((np * 16) >> 6) * BOX_BYTES + swz(row, chunk), b0, b1, b2, b3);
-          mma16816(o[2 * np], pa, b0, b1);
-          mma16816(o[2 * np + 1], pa, b2, b3);
+      for (int i = 0; i < QPT; ++i) {
+        const int idx = gtid + i * 128;
+        if (idx < group * (HD / 2)) {
+          const int h = idx / (HD / 2), d = (idx - h * (HD / 2)) * 2;
+          qreg[i] = *reinterpret_cast<const float2 *>(q + (size_t)r_ * nq * HD + (size_t)(g_ * group + h) * HD + d);
         }
       }
+    };
+    if ((int)blockIdx.x + gi * (int)gridDim.x < n_items) {
+      const int it0 = blockIdx.x + gi * gridDim.x;
+      load_q(work[it0 / kv.n_kv] >> 8, it0 % kv.n_kv);
     }
-  }
-  // row sums: add the 4 lanes that share a fragment row (fixed order)
-  l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-  l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    int k = gi;
+    for (int item = blockIdx.x + gi * gridDim.x; item < n_items; item += ATT_GROUPS * gridDim.x, k += ATT_GROUPS) {
+      const int buf = k % ATT_NBUF, slot = k % ATT_SLOTS, j = slot / ATT_GROUPS;
+      const int wi = work[item / kv.n_kv], g = item % kv.n_kv;
+      const int r = wi >> 8, split = wi & 255;
+      const int ctx = rows.pos[r] + 1;               // the new token attends to itself too
+      const int t0 = split * ATT_SPLIT;
+      const int n_pages = min(ATT_PAGES, (ctx - t0 + KV_BLOCK - 1) / KV_BLOCK);
+      const uint32_t k_tiles = ring + (uint32_t)buf * L::ITEM_BYTES;
+      const uint32_t v_tiles = k_tiles + L::K_BYTES;
 
-  // ---- merge the 4 warps in ascending order (the tile memory is free once every warp is here)
-  __syncthreads();
-  float *o_s = reinterpret_cast<float *>(smem_raw + (tiles - smem_u32(smem_raw)));   // [4][8][HD]
-  float *m_s = o_s + 4 * 8 * HD;                                                     // [4][8]
-  float *l_s = m_s + 32;                                                             // [4][8]
-  if (row_used) {
+      if (gtid == 0) ATRACE(k, 2);
+      // ---- 1. query operand tile: rows h (hi) and 8 + h (lo) of head g * group + h; the scale goes on the
+      //         scores.  The values were fetched one item ahead (qreg), so no global latency sits here.
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      const int d = nt * 8 + (lane & 3) * 2;
-      float2 v = make_float2(o[nt][0] + o[nt][2], o[nt][1] + o[nt][3]);   // hi rows + lo rows
-      *reinterpret_cast<float2 *>(&o_s[(warp * 8 + qrow) * HD + d]) = v;
-    }
-    if ((lane & 3) == 0) {
-      m_s[warp * 8 + qrow] = m_run;
-      l_s[warp * 8 + qrow] = l_run;
+      for (int i = 0; i < QPT; ++i) {
+        const int idx = gtid + i * 128;
+        if (idx < group * (HD / 2)) {
+          const int h = idx / (HD / 2), d = (idx - h * (HD / 2)) * 2;
+          __half h0, l0, h1, l1;
+          split_half(qreg[i].x, h0, l0);
+          split_half(qreg[i].y, h1, l1);
+          const uint32_t off = (uint32_t)(d >> 6) * OPND_BYTES + (uint32_t)((d & 7) * 2);
+          const int chunk = (d & 63) >> 3;
+          *reinterpret_cast<__half2 *>(q_ptr + off + swz(h, chunk)) = __halves2half2(h0, h1);
+          *reinterpret_cast<__half2 *>(q_ptr + off + swz(8 + h, chunk)) = __halves2half2(l0, l1);
+        }
+      }
+      {   // fetch the next item's query values now; they are consumed at the top of the next iteration
+        const int nxt = item + ATT_GROUPS * (int)gridDim.x;
+        if (nxt < n_items) {
+          const int nwi = work[nxt / kv.n_kv], ng = nxt % kv.n_kv, nr = nwi >> 8;
+          load_q(nr, ng);
+        }
+      }
+      fence_proxy_async();                           // the MMA reads this tile through the async proxy
+      if (gtid == 0) stop_s[gi] = abort_flag;
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + gi) : "memory");
+      if (stop_s[gi]) break;                         // the same decision in all 4 warps of the group
+
+      // ---- 2. S^T = K * Q^T, issued by one thread once the item has landed
+      if (gtid == 0) {
+        const bool ok = mbar_wait(smem_u32(&full_bar[slot]), (full_bits >> j) & 1u, &abort_flag);
+        ATRACE(k, 1);
+        if (ok) {
+          tc_fence_after();
+#pragma unroll
+          for (int ks = 0; ks < KSTEPS; ++ks) {
+            const uint64_t adv = (uint64_t)((ks & 3) * 2);      // 16 dims = 32 bytes inside the swizzled row
+            const uint64_t a = umma_desc_sw128(k_tiles + (uint32_t)(ks >> 2) * (ATT_PAGES * KBOX_BYTES)) + adv;
+            const uint64_t b = umma_desc_sw128(q_tile + (uint32_t)(ks >> 2) * OPND_BYTES) + adv;
+            umma_bf16(s_tmem, a, b, idesc, ks > 0 ? 1u : 0u);   // operand format (fp16) is in idesc
+          }
+        }
+        umma_commit(mbar);                           // also arrives if the wait gave up: nobody may hang here
+      }
+      full_bits ^= 1u << j;
+      {
+        bool ok = mbar_wait(mbar, mma_phase, &abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        mma_phase ^= 1u;
+        if (!ok) failed = true;
+      }
+      tc_fence_after();
+
+      // ---- 3. softmax over the item; this thread owns token t0 + tl
+      uint32_t sv[16];
+      tmem_ld16(s_tmem + ((uint32_t)(quad * 32) << 16), sv);
+      tmem_ld_wait();
+      const bool tok_ok = t0 + tl < ctx;
+      float sc[8];
+#pragma unroll
+      for (int h = 0; h < 8; ++h) {
+        sc[h] = tok_ok ? (__uint_as_float(sv[h]) + __uint_as_float(sv[8 + h])) * sscale : -CUDART_INF_F;
+        float m = sc[h];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (lane == h) red_s[gi][quad][h] = m;
+      }
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + gi) : "memory");
+      float pr[8], mx[8];
+      float my_sum = 0.f;                            // lane h keeps the warp's sum of head h
+#pragma unroll
+      for (int h = 0; h < 8; ++h) {
+        // exact maximum over the 128 tokens (token t0 is always valid, so it is finite for used heads)
+        mx[h] = fmaxf(fmaxf(red_s[gi][0][h], red_s[gi][1][h]), fmaxf(red_s[gi][2][h], red_s[gi][3][h]));
+        pr[h] = exp2f(sc[h] - mx[h]);                // 0 for masked tokens
+        float s = pr[h];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);   // fixed butterfly
+        if (lane == h) my_sum = s;
+      }
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + gi) : "memory");   // everyone has read the maxima
+      if (lane < 8) red_s[gi][quad][lane] = my_sum;
+      // weights as fp16 hi/lo into the [16 x 128 tokens] operand tile: rows h and 8 + h, column = token
+      {
+        const uint32_t off = (uint32_t)(tl >> 6) * OPND_BYTES + (uint32_t)((tl & 7) * 2);
+        const int chunk = (tl & 63) >> 3;
+#pragma unroll
+        for (int h = 0; h < 8; ++h) {
+          if (h < group) {
+            __half ph, pl;
+            split_half(pr[h], ph, pl);
+            *reinterpret_cast<__half *>(p_ptr + off + swz(h, chunk)) = ph;
+            *reinterpret_cast<__half *>(p_ptr + off + swz(8 + h, chunk)) = pl;
+          }
+        }
+      }
+      fence_proxy_async();
+      tc_fence_before();
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + gi) : "memory");
+
+      // ---- 4. O^T = V^T * P^T, one MMA per loaded page (16 tokens)
+      if (gtid == 0) {
+        tc_fence_after();
+        for (int p = 0; p < n_pages; ++p) {
+          const uint64_t a = umma_desc_sw32(v_tiles + (uint32_t)p * L::VT_BYTES);
+          const uint64_t b = umma_desc_sw128(p_tile + (uint32_t)(p >> 2) * OPND_BYTES) + (uint64_t)((p & 3) * 2);
+          umma_bf16(o_tmem, a, b, idesc, p > 0 ? 1u : 0u);
+        }
+        umma_commit(mbar);
+      }
+      {
+        bool ok = mbar_wait(mbar, mma_phase, &abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        mma_phase ^= 1u;
+        if (!ok) failed = true;
+      }
+      tc_fence_after();
+
+      // ---- 5. this thread owns output dim tl: add the hi and lo columns, write the partial
+      if (quad * 32 < HD) {                          // warp-uniform: with hd = 64 only lanes 0-63 hold dims
+        uint32_t ov[16];
+        tmem_ld16(o_tmem + ((uint32_t)(quad * 32) << 16), ov);
+        tmem_ld_wait();
+#pragma unroll
+        for (int h = 0; h < 8; ++h) {
+          if (h < group) {
+            const size_t pslot = ((size_t)r * nq + g * group + h) * max_splits + split;
+            part_acc[pslot * HD + tl] = __uint_as_float(ov[h]) + __uint_as_float(ov[8 + h]);
+          }
+        }
+      }
+#pragma unroll
+      for (int h = 0; h < 8; ++h) {
+        if (h < group && gtid == h) {              // red_s holds the four warps' sums by now
+          const size_t pslot = ((size_t)r * nq + g * group + h) * max_splits + split;
+          part_ml[pslot * 2] = mx[h];
+          part_ml[pslot * 2 + 1] = ((red_s[gi][0][h] + red_s[gi][1][h]) + red_s[gi][2][h]) + red_s[gi][3][h];
+        }
+      }
+      tc_fence_before();
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + gi) : "memory");   // the item's buffers and TMEM are free
+      if (gtid == 0) { mbar_arrive(smem_u32(&empty_bar[buf])); ATRACE(k, 3); }
     }
   }
-  __syncthreads();
-  for (int idx = tid; idx < group * HD; idx += ATT_THREADS) {
-    const int h = idx / HD, d = idx - h * HD;
-    float M = m_s[h];
-#pragma unroll
-    for (int w = 1; w < 4; ++w) M = fmaxf(M, m_s[w * 8 + h]);     // warp 0 always holds a valid token
-    float num = 0.f, den = 0.f;
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      const float wgt = exp2f(m_s[w * 8 + h] - M);                 // 0 for a warp without tokens
-      num = fmaf(o_s[(w * 8 + h) * HD + d], wgt, num);
-      den = fmaf(l_s[w * 8 + h], wgt, den);
-    }
-    const size_t slot = ((size_t)r * nq + g * group + h) * max_splits + split;
-    part_acc[slot * HD + d] = num;
-    if (d == 0) {
-      part_ml[slot * 2] = M;
-      part_ml[slot * 2 + 1] = den;
-    }
-  }
-  }   // items
   if (failed || abort_flag) {
-    if (tid == 0) atomicCAS(status, 0, DEV_TIMEOUT_EPILOGUE);
+    if (lane == 0) atomicCAS(status, 0, DEV_TIMEOUT_EPILOGUE);
     for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let copies in flight land before the CTA retires
   }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 0) tmem_dealloc(tmem_base, ATT_TMEM_COLS);
 }
 
 // Combines the splits of each (row, head) in ascending split order: one CTA per (head, row),
@@ -316,19 +388,14 @@ __global__ void __launch_bounds__(256) attn_worklist_kernel(Rows rows, int *__re
   if (r == 255) *n_work = before + mine;
 }
 
-template <int HD>
-constexpr size_t att_smem_bytes() {
-  return (size_t)2 * ATT_PAGES * (HD / 64) * BOX_BYTES + 1024;
-}
-
 }  // namespace
 
 cudaError_t attention_prepare() {
   cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)att_smem_bytes<128>());
+                                       (int)AttLayout<128>::SMEM);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(attn_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)att_smem_bytes<64>());
+                              (int)AttLayout<64>::SMEM);
 }
 
 cudaError_t launch_attn_worklist(const Rows &rows, int *work, int *n_work, cudaStream_t st) {
@@ -336,21 +403,22 @@ cudaError_t launch_attn_worklist(const Rows &rows, int *work, int *n_work, cudaS
   return launch_k(attn_worklist_kernel, dim3(1), dim3(256), 0, st, true, rows, work, n_work);
 }
 
-cudaError_t launch_attention(const CUtensorMap &tmKV, const float *q, const Rows &rows, int nq, const KvLayout &kv,
-                             int layer, int max_splits, const int *work, const int *n_work, int grid_ctas,
-                             float *part_acc, float *part_ml, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
-                             int *d_status, cudaStream_t st) {
+cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, const float *q, const Rows &rows, int nq,
+                             const KvLayout &kv, int layer, int max_splits, const int *work, const int *n_work,
+                             int grid_ctas, float *part_acc, float *part_ml, __nv_bfloat16 *out_hi,
+                             __nv_bfloat16 *out_lo, int *d_status, cudaStream_t st, unsigned long long *trace) {
+  (void)layer;   // the tensor maps are the layer's
   const int group = nq / kv.n_kv;
   if (group < 1 || group > 8 || max_splits > 256) return cudaErrorInvalidValue;
   const long long most = (long long)rows.R * max_splits * kv.n_kv;
   const int grid = (int)(most < grid_ctas ? most : grid_ctas);
   cudaError_t e;
   if (kv.hd == 128)
-    e = launch_k(attn_split_kernel<128>, dim3(grid), dim3(ATT_THREADS), att_smem_bytes<128>(), st, true, tmKV, q, rows, nq,
-                 group, kv, layer, max_splits, work, n_work, part_acc, part_ml, d_status);
+    e = launch_k(attn_split_kernel<128>, dim3(grid), dim3(ATT_THREADS), AttLayout<128>::SMEM, st, true, tmK, tmV, q, rows,
+                 nq, group, kv, max_splits, work, n_work, part_acc, part_ml, d_status, trace);
   else if (kv.hd == 64)
-    e = launch_k(attn_split_kernel<64>, dim3(grid), dim3(ATT_THREADS), att_smem_bytes<64>(), st, true, tmKV, q, rows, nq,
-                 group, kv, layer, max_splits, work, n_work, part_acc, part_ml, d_status);
+    e = launch_k(attn_split_kernel<64>, dim3(grid), dim3(ATT_THREADS), AttLayout<64>::SMEM, st, true, tmK, tmV, q, rows,
+                 nq, group, kv, max_splits, work, n_work, part_acc, part_ml, d_status, trace);
   else
     return cudaErrorInvalidValue;
   if (e != cudaSuccess) return e;

@@ -61,7 +61,7 @@ struct corun_engine {
   const bf16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
   std::vector<const bf16 *> attn_norm, mlp_norm;
   std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_down;
-  CUtensorMap tm_kv;
+  std::vector<CUtensorMap> tm_k, tm_v;   // per layer: key view and transposed-value view of the pages
   // KV
   __half *kv_pool = nullptr;
   size_t layer_stride = 0;
@@ -197,8 +197,8 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
                             P.xn_hi, P.xn_lo, e->st));
     STAGE(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, nullptr, true));
     STAGE(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st));
-    STAGE(launch_attention(e->tm_kv, P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work, P.att_n_work,
-                           3 * e->num_sms, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo, e->d_status, e->st));
+    STAGE(launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work, P.att_n_work,
+                           e->num_sms, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo, e->d_status, e->st));
     STAGE(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st, nullptr, true));
     GemmOut o = P.p_o.out();
     STAGE(launch_resid_norm(P.h, s.hidden, nullptr, rows, &o, e->mlp_norm[l], s.rms_eps, P.xn_hi, P.xn_lo, e->st));
@@ -380,9 +380,16 @@ int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int3
   // zero-filled: masked positions of a page are multiplied by zero weights, so they must be finite
   if ((rc = dmalloc(A, &e->kv_pool, e->layer_stride * s.n_layers, true))) return fail(rc);
   {
-    const unsigned long long rows = (unsigned long long)s.n_layers * e->pool_blocks * 2 * s.n_kv_heads * KV_BLOCK;
-    if (rows >= (1ull << 31)) return fail(CORUN_EINVAL);
-    if ((rc = tma_encode_2d(&e->tm_kv, e->kv_pool, 1, rows, s.head_dim, KV_BLOCK, 64))) return fail(rc);
+    // one layer's pages seen as rows of hd halfs (keys) and as rows of 16 halfs (transposed values)
+    const unsigned long long halfs = (unsigned long long)e->layer_stride;
+    if (halfs / KV_BLOCK >= (1ull << 31)) return fail(CORUN_EINVAL);
+    e->tm_k.resize(s.n_layers);
+    e->tm_v.resize(s.n_layers);
+    for (int l = 0; l < s.n_layers; ++l) {
+      const __half *base = e->kv_pool + (size_t)l * e->layer_stride;
+      if ((rc = tma_encode_2d(&e->tm_k[l], base, 1, halfs / s.head_dim, s.head_dim, KV_BLOCK, 64))) return fail(rc);
+      if ((rc = tma_encode_2d(&e->tm_v[l], base, 1, halfs / KV_BLOCK, KV_BLOCK, s.head_dim, KV_BLOCK))) return fail(rc);
+    }
     if (attention_prepare() != cudaSuccess) return fail(CORUN_ECUDA);
   }
   if ((rc = dmalloc(A, &e->d_block_table, (size_t)B * e->max_blocks))) return fail(rc);
@@ -718,8 +725,8 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
         case 4: ce = gemm_launch(P.p_lm, nullptr, e->d_status, e->st);
                 if (ce == cudaSuccess) ce = gemm_fixup_launch(P.p_lm, e->st);
                 break;
-        case 5: ce = launch_attention(e->tm_kv, P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work,
-                                      P.att_n_work, 3 * e->num_sms, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo,
+        case 5: ce = launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work,
+                                      P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo,
                                       e->d_status, e->st); break;
         case 6: ce = launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->attn_norm[l], s.rms_eps, P.xn_hi,
                                        P.xn_lo, e->st); break;
@@ -761,6 +768,28 @@ int corun_debug_gemm_trace(corun_engine *e, int32_t kind, int32_t layer, uint64_
   cudaFree(d);
   if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
   *n_ctas = p.grid;
+  return CORUN_OK;
+}
+
+int corun_debug_attn_trace(corun_engine *e, int32_t layer, uint64_t *stamps, int32_t *n_ctas) {
+  if (!e || !stamps || !n_ctas || layer < 0 || layer >= e->sh.n_layers) return CORUN_EINVAL;
+  RC(sync_stream(e));
+  Program &P = e->dec;
+  const corun_shape &s = e->sh;
+  const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
+  const size_t n = (size_t)e->num_sms * 64 * 4;
+  unsigned long long *d = nullptr;
+  if (cudaMalloc(&d, n * sizeof(unsigned long long)) != cudaSuccess) return CORUN_ENOMEM;
+  cudaError_t ce = cudaMemsetAsync(d, 0, n * sizeof(unsigned long long), e->st);
+  for (int i = 0; i < 2 && ce == cudaSuccess; ++i)
+    ce = launch_attention(e->tm_k[layer], e->tm_v[layer], P.q, rows, s.n_q_heads, kv_layout(e), layer, e->max_splits,
+                          P.att_work, P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo, e->d_status,
+                          e->st, d);
+  if (ce == cudaSuccess) ce = cudaMemcpyAsync(stamps, d, n * sizeof(unsigned long long), cudaMemcpyDeviceToHost, e->st);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(e->st);
+  cudaFree(d);
+  if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
+  *n_ctas = e->num_sms;
   return CORUN_OK;
 }
 

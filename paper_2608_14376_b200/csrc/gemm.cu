@@ -312,14 +312,16 @@ int tma_encode_2d(CUtensorMap *m, const void *base, int is_fp16, unsigned long l
                   int box_cols) {
   auto enc = get_encode();
   if (!enc) { g_last_cuda_error = 99999; return CORUN_ECUDA; }
-  if (((uintptr_t)base & 15u) || (cols % 8) || box_cols * 2 != 128 || box_rows > 256 || box_rows < 1) return CORUN_EINVAL;
+  if (((uintptr_t)base & 15u) || (cols % 8) || (box_cols * 2 != 128 && box_cols * 2 != 32) || box_rows > 256 || box_rows < 1)
+    return CORUN_EINVAL;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
   cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = enc(m, is_fp16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
                    const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                   box_cols * 2 == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_32B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) g_last_cuda_error = 100000 + (int)r;
   return r == CUDA_SUCCESS ? CORUN_OK : CORUN_ECUDA;
 }

@@ -110,7 +110,8 @@ cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int 
 int gemm_encode_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows);
 // Opts the GEMM kernel into its dynamic shared-memory size (idempotent, allocates nothing).
 cudaError_t gemm_prepare_kernel();
-// Tensor map for a 16-bit [rows, cols] row-major matrix with a [box_rows, 64] box (128 bytes wide), 128-byte swizzle.
+// Tensor map for a 16-bit [rows, cols] row-major matrix with a [box_rows, box_cols] box: 64 columns
+// (128 bytes, 128-byte swizzle) or 16 columns (32 bytes, 32-byte swizzle).
 int tma_encode_2d(CUtensorMap *m, const void *base, int is_fp16, unsigned long long rows, int cols, int box_rows,
                   int box_cols);
 // direct[r, n] = gemm_load(r, n) for every tile that has partials (makes `direct` a plain matrix).

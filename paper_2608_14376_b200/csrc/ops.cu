@@ -102,17 +102,17 @@ qkv_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, int
     return;
   }
   const int blk = kv.block_table[(size_t)rows.slot[r] * kv.max_blocks + pos / KV_BLOCK];
-  __half *base = kv.pool + (size_t)layer * kv.layer_stride + (size_t)blk * 2 * nkv * KV_BLOCK * hd +
-                 (size_t)(pos % KV_BLOCK) * hd + i;
-  // a page holds the nkv key tiles followed by the nkv value tiles, in the order of the GEMM's heads
-  __half *dst = base + (size_t)(head - nq) * KV_BLOCK * hd;
+  __half *page = kv.pool + (size_t)layer * kv.layer_stride + (size_t)blk * 2 * nkv * KV_BLOCK * hd;
+  const int tok = pos % KV_BLOCK;
   if (head < nq + nkv) {
     const float2 t = rope_tab[(size_t)pos * half + i];
-    dst[0] = __float2half_rn(a * t.x - b * t.y);
-    dst[half] = __float2half_rn(a * t.y + b * t.x);
+    const int g = head - nq;
+    page[kv_k_off(hd, g, tok, i)] = __float2half_rn(a * t.x - b * t.y);
+    page[kv_k_off(hd, g, tok, i + half)] = __float2half_rn(a * t.y + b * t.x);
   } else {
-    dst[0] = __float2half_rn(a);
-    dst[half] = __float2half_rn(b);
+    const int g = head - nq - nkv;
+    page[kv_v_off(nkv, hd, g, tok, i)] = __float2half_rn(a);
+    page[kv_v_off(nkv, hd, g, tok, i + half)] = __float2half_rn(b);
   }
 }
 
@@ -438,8 +438,8 @@ __global__ void kv_copy_kernel(KvLayout kv, int layer, int slot, int pos0, int n
   const int pos = pos0 + t;
   const int blk = kv.block_table[(size_t)slot * kv.max_blocks + pos / KV_BLOCK];
   __half *base = kv.pool + (size_t)layer * kv.layer_stride + (size_t)blk * 2 * kv.n_kv * KV_BLOCK * kv.hd;
-  __half *kp = base + ((size_t)g * KV_BLOCK + pos % KV_BLOCK) * kv.hd + i;
-  __half *vp = kp + (size_t)kv.n_kv * KV_BLOCK * kv.hd;
+  __half *kp = base + kv_k_off(kv.hd, g, pos % KV_BLOCK, i);
+  __half *vp = base + kv_v_off(kv.n_kv, kv.hd, g, pos % KV_BLOCK, i);
   if (write) {
     *kp = __float2half_rn(k[idx]);
     *vp = __float2half_rn(v[idx]);
@@ -472,9 +472,8 @@ __global__ void kv_fill_kernel(KvLayout kv, int n_layers, int slot, int n, float
   const float rad = sqrtf(-2.0f * logf(u1)) * std;
   const int blk = kv.block_table[(size_t)slot * kv.max_blocks + t / KV_BLOCK];
   __half *base = kv.pool + (size_t)layer * kv.layer_stride + (size_t)blk * 2 * kv.n_kv * KV_BLOCK * kv.hd;
-  __half *kp = base + ((size_t)g * KV_BLOCK + t % KV_BLOCK) * kv.hd + i;
-  *kp = __float2half_rn(rad * cospif(2.0f * u2));
-  *(kp + (size_t)kv.n_kv * KV_BLOCK * kv.hd) = __float2half_rn(rad * sinpif(2.0f * u2));
+  base[kv_k_off(kv.hd, g, t % KV_BLOCK, i)] = __float2half_rn(rad * cospif(2.0f * u2));
+  base[kv_v_off(kv.n_kv, kv.hd, g, t % KV_BLOCK, i)] = __float2half_rn(rad * sinpif(2.0f * u2));
 }
 
 }  // namespace

@@ -23,8 +23,18 @@ struct Rows {
   int R;
 };
 
+// Offsets (in halfs) inside one page: keys as [head][token][dim], then values TRANSPOSED as
+// [head][dim][token], so that both are K-major operands of the attention MMAs (scores contract over
+// dims, weighted values contract over tokens).
+__host__ __device__ inline size_t kv_k_off(int hd, int g, int tok, int dim) {
+  return ((size_t)g * KV_BLOCK + tok) * hd + dim;
+}
+__host__ __device__ inline size_t kv_v_off(int n_kv, int hd, int g, int tok, int dim) {
+  return (size_t)n_kv * KV_BLOCK * hd + ((size_t)g * hd + dim) * KV_BLOCK + tok;
+}
+
 struct KvLayout {
-  __half *pool;            // [layer][block][k|v][n_kv][16][hd]
+  __half *pool;            // [layer][page][ K: [n_kv][16][hd] | V^T: [n_kv][hd][16] ]
   const int *block_table;  // [n_slots][max_blocks]
   int max_blocks, n_kv, hd;
   size_t layer_stride;     // halfs per layer
@@ -51,13 +61,15 @@ cudaError_t launch_resid_norm(float *h, int H, const __nv_bfloat16 *embed, const
 cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *rope_tab, int nq, const KvLayout &kv,
                             int layer, float *q_out, cudaStream_t st);
 // Split-KV paged attention partials and their fixed-order combine -> bf16 hi/lo [R, nq*hd].
-// tmKV: tensor map over the whole pool as [all cached rows, hd] fp16 with a [16, 64] box (see attention.cu).
+// tmK / tmV: tensor maps over this layer's pages: keys as rows of hd halfs with a [16, 64] box (128-byte
+// swizzle), values as rows of 16 halfs with an [hd, 16] box (32-byte swizzle); see attention.cu.
 // work / n_work: the step's (row, split) items from launch_attn_worklist (the same for every layer);
-// grid_ctas: persistent CTAs to launch (3 per SM).
-cudaError_t launch_attention(const CUtensorMap &tmKV, const float *q, const Rows &rows, int nq, const KvLayout &kv,
-                             int layer, int max_splits, const int *work, const int *n_work, int grid_ctas,
-                             float *part_acc, float *part_ml, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
-                             int *d_status, cudaStream_t st);
+// grid_ctas: persistent CTAs to launch (one per SM).
+cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, const float *q, const Rows &rows, int nq,
+                             const KvLayout &kv, int layer, int max_splits, const int *work, const int *n_work,
+                             int grid_ctas, float *part_acc, float *part_ml, __nv_bfloat16 *out_hi,
+                             __nv_bfloat16 *out_lo, int *d_status, cudaStream_t st,
+                             unsigned long long *trace = nullptr);   // optional [grid][64][4] stamps (debug)
 cudaError_t launch_attn_worklist(const Rows &rows, int *work, int *n_work, cudaStream_t st);
 cudaError_t attention_prepare();   // opts the kernels into their shared-memory size (idempotent)
 // y = silu(gate) * up from the gate-up GEMM result -> bf16 hi/lo [R, F].
