@@ -66,15 +66,27 @@ def case_kernels(a):
     n_act = max(1, int(round(a.B * a.active_frac)))
     ctx = synth.uniform_lengths(a.ctx_lo, a.ctx_hi, n_act, seed=2)
     slots = synth.pick_slots(a.B, n_act, seed=7)
-    max_ctx = -(-(int(ctx.max()) + 64) // 256) * 256
+    max_ctx = -(-(int(ctx.max()) + 128) // 256) * 256
     eng = corun.Engine(sh, w, a.B, max_ctx)
     for i, (s, c) in enumerate(zip(slots, ctx)):
-        eng.adopt(int(s), 0, int(c) + 32, pending=1 + i, temperature=0.7, top_p=0.95)
+        eng.adopt(int(s), 0, int(c) + 64, pending=1 + i, temperature=0.7, top_p=0.95)
         eng.kv_fill(int(s), int(c), 1.28, seed=100 + i)
     active = np.zeros(a.B, np.uint8); active[slots] = 1
     seeds = np.arange(a.B, dtype=np.uint64) + 1000
     for _ in range(2):
         eng.decode_step(active, seeds)
+    import time as _t
+    for label, mask in (("step, given rows active", active), ("step, all rows padding", np.zeros(a.B, np.uint8))):
+        for _ in range(3):
+            eng.decode_enqueue(mask, seeds)
+        eng.decode_wait()
+        t0 = _t.perf_counter()
+        for _ in range(20):
+            eng.decode_enqueue(mask, seeds)
+        eng.decode_wait()
+        dt = (_t.perf_counter() - t0) / 20
+        print("%-26s %8.1f us  (%.1f us per layer)" % (label, dt * 1e6, dt * 1e6 / a.layers))
+    eng.decode_step(active, seeds)
     nbytes = {"gemm_qkv": 2 * sh.qkv_dim * sh.hidden, "gemm_o": 2 * sh.hidden * sh.q_dim,
               "gemm_gate_up": 4 * sh.ffn * sh.hidden, "gemm_down": 2 * sh.hidden * sh.ffn,
               "gemm_lm_head": 2 * sh.vocab * sh.hidden, "attention": sum((int(c) + 3) * 4096 for c in ctx)}

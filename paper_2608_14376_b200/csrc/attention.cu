@@ -341,35 +341,68 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   if (warp == 0) tmem_dealloc(tmem_base, ATT_TMEM_COLS);
 }
 
-// Combines the splits of each (row, head) in ascending split order: one CTA per (head, row),
-// one thread per output dim.  Output: bf16 hi/lo pair for the O projection.
-__global__ void __launch_bounds__(128)
-attn_combine_kernel(Rows rows, int nq, int hd, int max_splits, const float *__restrict__ part_acc,
+// Combines the splits of each (row, head): one warp per (row, head).  Lanes first hold one split each
+// (max by butterfly, which is exact; the denominator by a fixed butterfly over at most 32 lanes, then
+// ascending chunks of 32), then every lane owns hd/32 output dims and adds the splits' weighted
+// partial outputs in ascending split order.  Output: bf16 hi/lo pair for the O projection.
+template <int HD>
+__global__ void __launch_bounds__(256)
+attn_combine_kernel(Rows rows, int nq, int max_splits, const float *__restrict__ part_acc,
                     const float *__restrict__ part_ml, __nv_bfloat16 *__restrict__ out_hi,
                     __nv_bfloat16 *__restrict__ out_lo) {
+  constexpr int DPL = HD / 32;                   // dims per lane (4 or 2)
   griddep_launch_dependents();
   griddep_wait();
-  const int j = blockIdx.x, r = blockIdx.y, d = threadIdx.x;
-  float o = 0.f;
+  const int lane = threadIdx.x & 31;
+  const int pair = blockIdx.x * 8 + (threadIdx.x >> 5);      // (row, head) index
+  if (pair >= rows.R * nq) return;
+  const int r = pair / nq, j = pair - r * nq;
+  float o[DPL];
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) o[i] = 0.f;
   if (rows.active[r]) {
     const int nsplit = (rows.pos[r] + 1 + ATT_SPLIT - 1) / ATT_SPLIT;
-    const float *ml = part_ml + ((size_t)r * nq + j) * max_splits * 2;
-    const float *pa = part_acc + ((size_t)r * nq + j) * max_splits * hd + d;
-    float M = ml[0];
-    for (int s = 1; s < nsplit; ++s) M = fmaxf(M, ml[2 * s]);
-    float num = 0.f, den = 0.f;
-    for (int s = 0; s < nsplit; ++s) {
-      const float w = exp2f(ml[2 * s] - M);
-      num = fmaf(pa[(size_t)s * hd], w, num);
-      den = fmaf(ml[2 * s + 1], w, den);
+    const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + ((size_t)r * nq + j) * max_splits;
+    const float *pa = part_acc + ((size_t)r * nq + j) * max_splits * HD + lane * DPL;
+    float M = -CUDART_INF_F;
+    for (int s0 = 0; s0 < nsplit; s0 += 32) {
+      float m = (s0 + lane < nsplit) ? ml[s0 + lane].x : -CUDART_INF_F;
+#pragma unroll
+      for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
+      M = fmaxf(M, m);
     }
-    o = num / den;
+    float den = 0.f;
+    for (int s0 = 0; s0 < nsplit; s0 += 32) {
+      float2 v = (s0 + lane < nsplit) ? ml[s0 + lane] : make_float2(-CUDART_INF_F, 0.f);
+      const float w = exp2f(v.x - M);              // this lane's split weight (0 beyond the last split)
+      float d = v.y * w;
+#pragma unroll
+      for (int k = 16; k > 0; k >>= 1) d += __shfl_xor_sync(0xffffffffu, d, k);
+      den += d;
+      const int cnt = min(32, nsplit - s0);
+      for (int s = 0; s < cnt; ++s) {
+        const float ws = __shfl_sync(0xffffffffu, w, s);
+        const float *p = pa + (size_t)(s0 + s) * HD;
+        if (DPL == 4) {
+          const float4 a = *reinterpret_cast<const float4 *>(p);
+          o[0] = fmaf(a.x, ws, o[0]); o[1] = fmaf(a.y, ws, o[1]);
+          o[DPL - 2] = fmaf(a.z, ws, o[DPL - 2]); o[DPL - 1] = fmaf(a.w, ws, o[DPL - 1]);
+        } else {
+          const float2 a = *reinterpret_cast<const float2 *>(p);
+          o[0] = fmaf(a.x, ws, o[0]); o[1] = fmaf(a.y, ws, o[1]);
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) o[i] = o[i] / den;
   }
-  const __nv_bfloat16 a = __float2bfloat16_rn(o);
-  const __nv_bfloat16 b = __float2bfloat16_rn(o - __bfloat162float(a));
-  const size_t idx = (size_t)r * nq * hd + (size_t)j * hd + d;
-  out_hi[idx] = a;
-  out_lo[idx] = b;
+  const size_t idx = (size_t)r * nq * HD + (size_t)j * HD + lane * DPL;
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) {
+    const __nv_bfloat16 a = __float2bfloat16_rn(o[i]);
+    out_hi[idx + i] = a;
+    out_lo[idx + i] = __float2bfloat16_rn(o[i] - __bfloat162float(a));
+  }
 }
 
 // Lists the (row, split) items of the step: active rows in ascending order, splits ascending.
@@ -422,8 +455,12 @@ cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, con
   else
     return cudaErrorInvalidValue;
   if (e != cudaSuccess) return e;
-  return launch_k(attn_combine_kernel, dim3(nq, rows.R), dim3(kv.hd), 0, st, true, rows, nq, kv.hd, max_splits, part_acc,
-                  part_ml, out_hi, out_lo);
+  const dim3 cgrid((rows.R * nq + 7) / 8);
+  if (kv.hd == 128)
+    return launch_k(attn_combine_kernel<128>, cgrid, dim3(256), 0, st, true, rows, nq, max_splits, part_acc, part_ml, out_hi,
+                    out_lo);
+  return launch_k(attn_combine_kernel<64>, cgrid, dim3(256), 0, st, true, rows, nq, max_splits, part_acc, part_ml, out_hi,
+                  out_lo);
 }
 
 }  // namespace corun
