@@ -93,6 +93,22 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(x: float, dist, device) -> float:
+    """Slowest rank's value (all-reduce MAX); `dist` is torch.distributed or None for a single process."""
+    if dist is None:
+        return float(x)
+    import torch
+
+    t = torch.tensor([float(x)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(units_per_step_per_replica: int, world: int, ms_per_step_max: float) -> float:
+    """Whole-job units/s of `world` independent replicas: all their units over the slowest one's time."""
+    return world * units_per_step_per_replica / (ms_per_step_max / 1e3)
+
+
 def workload_inputs(name: str):
     sh, B, n_active, lo, hi, T, P, kv_std = WORKLOADS[name]
     slots = synth.pick_slots(B, n_active, seed=7)
@@ -215,13 +231,9 @@ def run_corun(args, rank, world):
     clk = clocks.stop()
     assert all(toks[s] >= 0 for s in slots) and all(toks[s] == -1 for s in range(B) if not active[s])
     step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(K)]
-    total_ms = ev[0].elapsed_time(ev[K])
-    if dist:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(ev[0].elapsed_time(ev[K]), dist, "cuda")
     ms_per_step = total_ms / K
-    value = world * n_active / (ms_per_step / 1e3)
+    value = replica_throughput(n_active, world, ms_per_step)
 
     # ---- end to end through the C ABI with host buffers: mask + seeds in, tokens out, every step
     for _ in range(W):
@@ -230,12 +242,8 @@ def run_corun(args, rank, world):
     t0 = time.perf_counter()
     for _ in range(K):
         toks = eng.decode_step(active, seeds)
-    e2e_s = time.perf_counter() - t0
-    if dist:
-        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_val = world * n_active * K / e2e_s
+    e2e_s = max_over_ranks(time.perf_counter() - t0, dist, "cuda")
+    e2e_val = replica_throughput(n_active, world, 1e3 * e2e_s / K)
 
     # ---- per-kernel durations (isolated launches rotating over the layers' weights, CUDA events)
     L = sh.n_layers
