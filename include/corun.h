@@ -187,6 +187,10 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
  * 8 * 256 values) are globaltimer nanoseconds at: 0 kernel entry, 1 set-up done, 2 first TMA issued,
  * 3 last TMA issued, 4 first stage landed, 5 last MMA issued, 6 last accumulator complete, 7 epilogue done. */
 int corun_debug_gemm_trace(corun_engine *e, int32_t kind, int32_t layer, uint64_t *stamps, int32_t *n_ctas);
+/* With CORUN_TRACE_STEP=1 in the environment at corun_init, every layer GEMM of the decode program records
+ * its per-CTA timeline (the 8 stamps of corun_debug_gemm_trace) on every step; this copies the last step's
+ * stamps, [4 * n_layers][n_sms][8] values (n must equal that count), to the host. */
+int corun_debug_step_trace(corun_engine *e, uint64_t *stamps, int64_t n);
 /* Runs the attention of one layer twice on the rows of the last decode step and returns the second launch's
  * timeline: stamps[(cta*64 + k)*4 + i] (host, room for 256*64*4 values), globaltimer ns of the CTA's k-th item
  * (k < 64): 0 load issued, 1 item landed (seen by its consumer group), 2 the group starts on it, 3 released. */

@@ -20,7 +20,7 @@ EXPORTS = [
     "corun_init", "corun_prefill", "corun_decode_step", "corun_decode_enqueue", "corun_decode_wait",
     "corun_release", "corun_destroy", "corun_get_logits", "corun_force_token", "corun_context_len",
     "corun_free_blocks", "corun_debug_kv_read", "corun_debug_kv_write", "corun_debug_adopt",
-    "corun_debug_set_eager", "corun_debug_read", "corun_debug_gemm_trace", "corun_debug_attn_trace", "corun_debug_kv_fill", "corun_debug_time_kernel", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
+    "corun_debug_set_eager", "corun_debug_read", "corun_debug_gemm_trace", "corun_debug_attn_trace", "corun_debug_step_trace", "corun_debug_kv_fill", "corun_debug_time_kernel", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
     "corun_debug_sample", "corun_gemm_static", "corun_strerror", "corun_last_cuda_error",
 ]
 
@@ -83,6 +83,7 @@ def lib():
         L.corun_debug_read.argtypes = [vp, i32, vp, i64]
         L.corun_debug_gemm_trace.argtypes = [vp, i32, i32, vp, C.POINTER(i32)]
         L.corun_debug_attn_trace.argtypes = [vp, i32, vp, C.POINTER(i32)]
+        L.corun_debug_step_trace.argtypes = [vp, vp, i64]
         L.corun_debug_kv_fill.argtypes = [vp, i32, i32, C.c_float, u64]
         L.corun_debug_time_kernel.argtypes = [vp, i32, i32, C.POINTER(C.c_float)]
         L.corun_decode_launches.argtypes = [vp]
@@ -237,6 +238,13 @@ class Engine:
         _check(lib().corun_debug_gemm_trace(self._h, kind, layer, st.ctypes.data, C.byref(n)), "gemm_trace")
         t = st[:8 * n.value].reshape(n.value, 8).astype(np.int64)
         return t - t[:, 0].min()
+
+    def step_trace(self, n_sms: int = 148) -> np.ndarray:
+        """GEMM timelines of the last decode step, [4 * n_layers, n_sms, 8] ns (engine made with CORUN_TRACE_STEP=1)."""
+        n = 4 * self._cs.n_layers * n_sms * 8
+        st = np.zeros(n, np.uint64)
+        _check(lib().corun_debug_step_trace(self._h, st.ctypes.data, n), "step_trace")
+        return st.reshape(4 * self._cs.n_layers, n_sms, 8).astype(np.int64)
 
     def attn_trace(self, layer: int = 0) -> np.ndarray:
         """Per-CTA, per-item attention timeline [n_ctas, 64, 4] in ns (0 where an item does not exist)."""

@@ -380,16 +380,22 @@ attn_combine_kernel(Rows rows, int nq, int max_splits, const float *__restrict__
       for (int k = 16; k > 0; k >>= 1) d += __shfl_xor_sync(0xffffffffu, d, k);
       den += d;
       const int cnt = min(32, nsplit - s0);
-      for (int s = 0; s < cnt; ++s) {
-        const float ws = __shfl_sync(0xffffffffu, w, s);
-        const float *p = pa + (size_t)(s0 + s) * HD;
-        if (DPL == 4) {
-          const float4 a = *reinterpret_cast<const float4 *>(p);
-          o[0] = fmaf(a.x, ws, o[0]); o[1] = fmaf(a.y, ws, o[1]);
-          o[DPL - 2] = fmaf(a.z, ws, o[DPL - 2]); o[DPL - 1] = fmaf(a.w, ws, o[DPL - 1]);
-        } else {
-          const float2 a = *reinterpret_cast<const float2 *>(p);
-          o[0] = fmaf(a.x, ws, o[0]); o[1] = fmaf(a.y, ws, o[1]);
+      for (int sb = 0; sb < cnt; sb += 8) {          // eight splits' partial outputs are fetched together
+        float4 a[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          a[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (sb + u < cnt) {
+            const float *p = pa + (size_t)(s0 + sb + u) * HD;
+            if (DPL == 4) a[u] = *reinterpret_cast<const float4 *>(p);
+            else { const float2 t = *reinterpret_cast<const float2 *>(p); a[u].x = t.x; a[u].y = t.y; }
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const float ws = __shfl_sync(0xffffffffu, w, (sb + u) & 31);   // weight 0 beyond the last split
+          o[0] = fmaf(a[u].x, ws, o[0]); o[1] = fmaf(a[u].y, ws, o[1]);
+          if (DPL == 4) { o[DPL - 2] = fmaf(a[u].z, ws, o[DPL - 2]); o[DPL - 1] = fmaf(a[u].w, ws, o[DPL - 1]); }
         }
       }
     }

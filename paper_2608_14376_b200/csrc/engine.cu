@@ -91,6 +91,7 @@ struct corun_engine {
   cudaGraph_t graph = nullptr;
   cudaGraphExec_t graph_exec = nullptr;
   bool eager = false;
+  unsigned long long *step_trace = nullptr;   // debug (CORUN_TRACE_STEP=1): GEMM timelines of a whole step
   int stop_after = -1;            // debug: eager decode stops after this many stages of layer 0
   int decode_launches = 0;
   std::vector<void *> allocs;
@@ -183,6 +184,10 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
   int n = 0;
   CK(launch_attn_worklist(rows, P.att_work, P.att_n_work, e->st));   // the same items serve every layer
   n += 1;
+  // (debug) slice of the step trace for the idx-th GEMM of the decode program: [num_sms][8] stamps
+  auto tr = [&](int idx) -> unsigned long long * {
+    return (e->step_trace && &P == &e->dec) ? e->step_trace + (size_t)idx * e->num_sms * 8 : nullptr;
+  };
   int stage = 0;
   const int stop = (e->eager && &P == &e->dec) ? e->stop_after : -1;
 #define STAGE(call)                                   \
@@ -195,16 +200,16 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
     GemmOut prev = P.p_down.out();
     STAGE(launch_resid_norm(P.h, s.hidden, e->embed, rows, l == 0 ? nullptr : &prev, e->attn_norm[l], s.rms_eps,
                             P.xn_hi, P.xn_lo, e->st));
-    STAGE(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, nullptr, true));
+    STAGE(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, tr(4 * l + 0), true));
     STAGE(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st));
     STAGE(launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work, P.att_n_work,
                            e->num_sms, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo, e->d_status, e->st));
-    STAGE(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st, nullptr, true));
+    STAGE(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st, tr(4 * l + 1), true));
     GemmOut o = P.p_o.out();
     STAGE(launch_resid_norm(P.h, s.hidden, nullptr, rows, &o, e->mlp_norm[l], s.rms_eps, P.xn_hi, P.xn_lo, e->st));
-    STAGE(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st, nullptr, true));
+    STAGE(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st, tr(4 * l + 2), true));
     STAGE(launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st));
-    STAGE(gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st, nullptr, true));
+    STAGE(gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st, tr(4 * l + 3), true));
     n += 10;
   }
 #undef STAGE
@@ -431,6 +436,9 @@ int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int3
   memset(e->h_seeds, 0, B * sizeof(uint64_t));
   *e->h_status = 0;
 
+  if (const char *ts = getenv("CORUN_TRACE_STEP")) {
+    if (atoi(ts) != 0 && (rc = dmalloc(A, &e->step_trace, (size_t)4 * s.n_layers * e->num_sms * 8))) return fail(rc);
+  }
   if ((rc = program_create(e, e->dec, B, true, true))) return fail(rc);
   if ((rc = program_create(e, e->pre, e->chunk, true, false))) return fail(rc);
   if ((rc = program_create(e, e->lm1, 1, false, true))) return fail(rc);
@@ -790,6 +798,17 @@ int corun_debug_attn_trace(corun_engine *e, int32_t layer, uint64_t *stamps, int
   cudaFree(d);
   if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
   *n_ctas = e->num_sms;
+  return CORUN_OK;
+}
+
+int corun_debug_step_trace(corun_engine *e, uint64_t *stamps, int64_t n) {
+  if (!e || !stamps) return CORUN_EINVAL;
+  if (!e->step_trace) return CORUN_EINVAL;    // the engine was not created with CORUN_TRACE_STEP=1
+  const int64_t have = (int64_t)4 * e->sh.n_layers * e->num_sms * 8;
+  if (n != have) return CORUN_EINVAL;
+  RC(sync_stream(e));
+  CK(cudaMemcpyAsync(stamps, e->step_trace, (size_t)n * sizeof(uint64_t), cudaMemcpyDeviceToHost, e->st));
+  CK(cudaStreamSynchronize(e->st));
   return CORUN_OK;
 }
 
