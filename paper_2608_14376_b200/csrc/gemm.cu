@@ -18,6 +18,7 @@ bool g_use_pdl = !(getenv("CORUN_NO_PDL") && atoi(getenv("CORUN_NO_PDL")) != 0);
 namespace {
 
 constexpr int MAX_STAGES = 8;
+constexpr int GEMM_MAX_DYN_SMEM = 209 * 1024;   // leaves room for the static shared memory within the 227 KiB of a CTA
 constexpr uint32_t W_TILE_BYTES = GEMM_TILE_N * GEMM_BLOCK_K * 2;          // 32 KiB
 constexpr uint32_t A_BLOCK_BYTES = GEMM_ROW_BLOCK * GEMM_BLOCK_K * 2;      // 16 KiB: what one MMA reads of A
 
@@ -46,7 +47,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   __shared__ __align__(8) uint64_t tmem_empty_bar[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
-  __shared__ float xch[64 * 33];   // hi/lo hand-over of the stacked epilogue (row pitch 33: no bank conflicts)
+  __shared__ float xch[2][64 * 33];   // stacked epilogue: W*hi and W*lo of 64 rows x 32 columns (row pitch 33: no bank conflicts)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x;
@@ -200,41 +201,45 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       const int n0 = tile * GEMM_TILE_N;
       if (stacked) {
         // lanes 0-63 (warps with lane_base 0, 32) hold W*hi of rows 0-63, lanes 64-127 hold W*lo of the
-        // same rows: the lo warps hand their values over through shared memory, 32 columns at a time
+        // same rows: every warp parks 32 columns of its rows in shared memory, then the 128 threads add
+        // the two halves and store whole 128-byte row segments (four rows per warp instruction)
         const bool lo_warp = lane_base >= 64;
         const int row = (lane_base & 63) + lane;
         const int rows_valid = whole ? R : BN;
         const bool warp_needed = (lane_base & 63) < rows_valid;   // warp-uniform
-        const bool row_ok = row < rows_valid;
-        float *dst = whole ? direct + (size_t)row * N + n0
-                           : ws + ((size_t)(cta * 2 + (seg == 0 ? 0 : 1)) * BN + row) * GEMM_TILE_N;
+        float *xs = xch[lo_warp ? 1 : 0] + row * 33;
+        const int te = (int)threadIdx.x - 64, srow = te >> 3, scol = (te & 7) * 4;
+        float *dst0 = whole ? direct + n0 : ws + (size_t)(cta * 2 + (seg == 0 ? 0 : 1)) * BN * GEMM_TILE_N;
+        const size_t pitch = whole ? (size_t)N : (size_t)GEMM_TILE_N;
         const bool vec_ok = whole ? ((N & 3) == 0) : true;
         for (int c0 = 0; c0 < GEMM_TILE_N; c0 += 32) {
           if (whole && n0 + c0 >= N) break;          // columns beyond the matrix (last tile); uniform
-          uint32_t v[32];
           if (warp_needed) {
+            uint32_t v[32];
             const uint32_t ta = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)acc * acc_cols + (uint32_t)c0;
             tmem_ld16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
             tmem_ld16(ta + 16, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
             tmem_ld_wait();
-            if (lo_warp) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j) xch[row * 33 + j] = __uint_as_float(v[j]);
-            }
+            for (int j = 0; j < 32; ++j) xs[j] = __uint_as_float(v[j]);
           }
           asm volatile("bar.sync 1, 128;" ::: "memory");
-          if (warp_needed && !lo_warp && row_ok) {
-            float f[32];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]) + xch[row * 33 + j];
-            if (vec_ok && (!whole || n0 + c0 + 32 <= N)) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4 *>(dst + c0 + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (n0 + c0 + j < N) dst[c0 + j] = f[j];
+          for (int i = 0; i < 4; ++i) {
+            const int r = i * 16 + srow;
+            if (r < rows_valid) {
+              const float *h = xch[0] + r * 33 + scol, *l = xch[1] + r * 33 + scol;
+              const float4 f = make_float4(h[0] + l[0], h[1] + l[1], h[2] + l[2], h[3] + l[3]);
+              float *d = dst0 + (size_t)r * pitch + c0 + scol;
+              if (vec_ok && (!whole || n0 + c0 + scol + 4 <= N)) {
+                *reinterpret_cast<float4 *>(d) = f;
+              } else {
+                const int nn = n0 + c0 + scol;
+                if (nn < N) d[0] = f.x;
+                if (nn + 1 < N) d[1] = f.y;
+                if (nn + 2 < N) d[2] = f.z;
+                if (nn + 3 < N) d[3] = f.w;
+              }
             }
           }
           asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -342,7 +347,7 @@ int gemm_plan_fill(GemmPlan *p, const void *W, int N, int K, const void *Xhi, co
   if (total * (long long)p->grid >= (1ll << 31)) return CORUN_EINVAL;
   const size_t stage = (size_t)W_TILE_BYTES + (BN <= 64 ? (size_t)A_BLOCK_BYTES : 2 * (size_t)BN * GEMM_BLOCK_K * 2);
   // the MMA always reads 128 activation rows: leave that much readable behind the last stage
-  int stages = (int)((216 * 1024 - 1024 - A_BLOCK_BYTES) / stage);
+  int stages = (int)((GEMM_MAX_DYN_SMEM - 1024 - A_BLOCK_BYTES) / stage);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (const char *ev = getenv("CORUN_GEMM_STAGES")) {   // experiments only: shallower ring
     const int v = atoi(ev);
@@ -407,7 +412,7 @@ int gemm_plan_create(GemmPlan *p, const void *W, int N, int K, const void *Xhi, 
 }
 
 cudaError_t gemm_prepare_kernel() {
-  return cudaFuncSetAttribute(gemm_streamk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 216 * 1024);
+  return cudaFuncSetAttribute(gemm_streamk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
 }
 
 void gemm_plan_destroy(GemmPlan *p) {

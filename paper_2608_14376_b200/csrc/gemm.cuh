@@ -35,7 +35,7 @@ struct GemmOut {
 
 // Value (r, n) of a GEMM result, partials added in ascending CTA order.
 __device__ __forceinline__ float gemm_load(const GemmOut &g, int r, int n) {
-  const int t = n >> 8, col = n & 255;
+  const int t = n / GEMM_TILE_N, col = n % GEMM_TILE_N;
   const int f = g.tile_first[t], c0 = f >> 1, c1 = g.tile_cend[t];
   if (c0 == c1) return g.direct[(size_t)r * g.N + n];
   const float *p = g.ws + ((size_t)r) * GEMM_TILE_N + col;
@@ -49,7 +49,7 @@ __device__ __forceinline__ float gemm_load(const GemmOut &g, int r, int n) {
 // Four consecutive values (n % 4 == 0, N % 4 == 0) with the same summation order as gemm_load.
 // Loads are issued four partials at a time; an absent partial contributes +0.0f.
 __device__ __forceinline__ float4 gemm_load4(const GemmOut &g, int r, int n) {
-  const int t = n >> 8, col = n & 255;
+  const int t = n / GEMM_TILE_N, col = n % GEMM_TILE_N;
   const int f = g.tile_first[t], c0 = f >> 1, c1 = g.tile_cend[t];
   if (c0 == c1) return *reinterpret_cast<const float4 *>(g.direct + (size_t)r * g.N + n);
   const float *p = g.ws + ((size_t)r) * GEMM_TILE_N + col;

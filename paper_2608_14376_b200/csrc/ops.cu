@@ -197,6 +197,8 @@ __device__ __forceinline__ unsigned long long block_excl_scan_u64(unsigned long 
   return wtot[warp] + inc - v;
 }
 
+constexpr int SMP_CAND = 2048;   // tokens of the selected coarse bin that are kept in shared memory
+
 struct SmpShared {
   unsigned long long hist[SMP_BINS];
   unsigned int cnt[SMP_BINS];
@@ -204,8 +206,10 @@ struct SmpShared {
   unsigned long long total, carried, sel_sum;
   float red_val[32];
   int red_idx[32];
-  unsigned int kmin, kmax, sel_cnt;
-  int sel_bin, winner;
+  unsigned int kmin, kmax, sel_cnt, n_cand;
+  int sel_bin, sel_warp, tie_max_id;
+  float cand_x[SMP_CAND];
+  int cand_id[SMP_CAND];
 };
 
 // Integer weight of a token: floor(2^40 * exp2(x)), x = fl32(fl32(l - max) * inv_t_log2e).
@@ -233,8 +237,11 @@ __device__ __forceinline__ unsigned long long smp_weight(float l, float mx, floa
 
 // After a histogram pass: finds the first bin (ascending index = descending
 // logit) that is non-empty and whose running weight reaches the cut; adds the
-// weight of the bins before it to `carried`.
-__device__ void smp_select_bin(SmpShared &sh, unsigned long long cut) {
+// weight of the bins before it to `carried`.  With use_cnt = false a bin counts
+// as non-empty when its weight is positive (the coarse pass keeps no counts:
+// there the selected bin always has positive weight, because bin 0 holds the
+// maximum, whose weight is 2^40).
+__device__ void smp_select_bin(SmpShared &sh, unsigned long long cut, bool use_cnt) {
   const int tid = threadIdx.x;
   const unsigned long long a = sh.hist[2 * tid], b = sh.hist[2 * tid + 1];
   unsigned long long tot;
@@ -242,81 +249,63 @@ __device__ void smp_select_bin(SmpShared &sh, unsigned long long cut) {
   if (tid == 0) sh.sel_bin = SMP_BINS;
   __syncthreads();
   const unsigned long long base = sh.carried + before;
-  if (sh.cnt[2 * tid] && base + a >= cut) atomicMin(&sh.sel_bin, 2 * tid);
-  else if (sh.cnt[2 * tid + 1] && base + a + b >= cut) atomicMin(&sh.sel_bin, 2 * tid + 1);
+  const bool ne0 = use_cnt ? sh.cnt[2 * tid] != 0u : a != 0ull;
+  const bool ne1 = use_cnt ? sh.cnt[2 * tid + 1] != 0u : b != 0ull;
+  if (ne0 && base + a >= cut) atomicMin(&sh.sel_bin, 2 * tid);
+  else if (ne1 && base + a + b >= cut) atomicMin(&sh.sel_bin, 2 * tid + 1);
   __syncthreads();
   const int sel = sh.sel_bin;   // < SMP_BINS: total weight always reaches the cut
   if (sel < SMP_BINS && (sel >> 1) == tid) {
     sh.carried = base + ((sel & 1) ? a : 0ull);
     sh.sel_sum = (sel & 1) ? b : a;
-    sh.sel_cnt = sh.cnt[sel];
+    sh.sel_cnt = use_cnt ? sh.cnt[sel] : 0u;
   }
   __syncthreads();
 }
 
-__global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
-  griddep_launch_dependents();
-  griddep_wait();
-  const int r = blockIdx.x;
-  if (!a.do_sample[r]) return;
-  __shared__ SmpShared sh;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int V = a.V;
-  const float *lg = a.logits + (size_t)r * V;
+// One refinement step in key space: bins the keys of [kmin, kmax] into SMP_BINS
+// equal ranges (descending key = ascending bin), selects the bin where the
+// running weight reaches the cut and narrows [kmin, kmax] to it.
+struct KeyRange { uint32_t kmin, kmax; };
+__device__ __forceinline__ int smp_key_bin(uint32_t k, uint32_t kmin, unsigned long long width) {
+  return SMP_BINS - 1 - (int)(((unsigned long long)(k - kmin) * SMP_BINS) / width);
+}
+__device__ __forceinline__ KeyRange smp_narrow(const SmpShared &sh, uint32_t kmin, unsigned long long width) {
+  const unsigned long long j = (unsigned long long)(SMP_BINS - 1 - sh.sel_bin);
+  // keys k with floor((k - kmin) * BINS / width) == j
+  const unsigned long long lo = (j * width + SMP_BINS - 1) / SMP_BINS;
+  const unsigned long long hi = ((j + 1) * width + SMP_BINS - 1) / SMP_BINS - 1;
+  return KeyRange{kmin + (uint32_t)lo, kmin + (uint32_t)hi};
+}
 
-  // ---- argmax, lowest id on ties
-  float bv = -CUDART_INF_F;
-  int bi = 0x7fffffff;
-  for (int i = tid; i < V; i += SMP_THREADS) {
-    const float x = lg[i];
-    if (x > bv || (x == bv && i < bi)) { bv = x; bi = i; }
+// Every logit of the row in ascending id by float4 where the row allows it (V % 4 == 0), else one by one.
+#define SMP_FOREACH(BODY)                                                                  \
+  if (vec) {                                                                               \
+    _Pragma("unroll 2") for (int i4 = tid; i4 < n4; i4 += SMP_THREADS) {                   \
+      const float4 q4 = reinterpret_cast<const float4 *>(lg)[i4];                          \
+      const float xs4[4] = {q4.x, q4.y, q4.z, q4.w};                                       \
+      _Pragma("unroll") for (int j4 = 0; j4 < 4; ++j4) {                                   \
+        const int i = 4 * i4 + j4;                                                         \
+        const float x = xs4[j4];                                                           \
+        BODY                                                                               \
+      }                                                                                    \
+    }                                                                                      \
+  } else {                                                                                 \
+    for (int i = tid; i < V; i += SMP_THREADS) {                                           \
+      const float x = lg[i];                                                               \
+      BODY                                                                                 \
+    }                                                                                      \
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-  }
-  if (lane == 0) { sh.red_val[warp] = bv; sh.red_idx[warp] = bi; }
-  __syncthreads();
-  bv = sh.red_val[0]; bi = sh.red_idx[0];
-  for (int w = 1; w < SMP_THREADS / 32; ++w) {
-    const float ov = sh.red_val[w];
-    const int oi = sh.red_idx[w];
-    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-  }
-  const float temperature = a.temperature[r];
-  if (!(temperature > 0.f)) {
-    if (tid == 0) a.out_token[r] = bi;
-    return;
-  }
-  const float mx = bv;
-  const float inv_t_log2e = __fdiv_rn(0x1.715476p+0f, temperature);
-  const uint32_t u24 = a.u24_override ? a.u24_override[r] : philox_u24(a.seed[r], (uint64_t)a.step[r]);
 
-  // ---- pass A: bins linear in (max - logit); bin 0 holds the largest logits
-  // weights vanish beyond (max - l)/T > 27.73, so the bins cover 28 T logit units
-  const float scale_a = (float)SMP_BINS / (28.f * temperature);
-  for (int i = tid; i < SMP_BINS; i += SMP_THREADS) { sh.hist[i] = 0ull; sh.cnt[i] = 0u; }
-  if (tid == 0) { sh.carried = 0ull; sh.kmin = 0xffffffffu; sh.kmax = 0u; }
+// Slow tail, used when the selected coarse bin holds more tokens than the
+// candidate list (rows with very many equal or nearly equal logits): the
+// refinement and the final walk read the whole row every time.
+__device__ __noinline__ void smp_tail_full_row(SmpShared &sh, const SampleArgs &a, int r, const float *lg, float mx,
+                                               float inv_t_log2e, float scale_a, int bin_a, unsigned long long cut,
+                                               uint32_t u24) {
+  const int tid = threadIdx.x, V = a.V;
+  if (tid == 0) { sh.kmin = 0xffffffffu; sh.kmax = 0u; }
   __syncthreads();
-  unsigned long long mysum = 0ull;
-  for (int i = tid; i < V; i += SMP_THREADS) {
-    const float x = lg[i];
-    const unsigned long long w = smp_weight(x, mx, inv_t_log2e);
-    const int bin = min(SMP_BINS - 1, (int)((mx - x) * scale_a));
-    atomicAdd(&sh.hist[bin], w);
-    atomicAdd(&sh.cnt[bin], 1u);
-    mysum += w;
-  }
-  unsigned long long total;
-  block_excl_scan_u64(mysum, sh.wtot, &sh.total);
-  total = sh.total;
-  unsigned long long cut = __double2ull_rd((double)a.top_p[r] * (double)total);
-  if (cut > total) cut = total;
-  smp_select_bin(sh, cut);
-  const int bin_a = sh.sel_bin;
-  // key range of the selected bin
   for (int i = tid; i < V; i += SMP_THREADS) {
     const float x = lg[i];
     if (min(SMP_BINS - 1, (int)((mx - x) * scale_a)) == bin_a) {
@@ -327,7 +316,6 @@ __global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
   }
   __syncthreads();
   uint32_t kmin = sh.kmin, kmax = sh.kmax;
-  // ---- passes B: exact refinement in key space until one key remains
   for (int pass = 0; pass < 4 && kmax > kmin; ++pass) {
     const unsigned long long width = (unsigned long long)(kmax - kmin) + 1ull;
     __syncthreads();
@@ -337,20 +325,15 @@ __global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
       const float x = lg[i];
       const uint32_t k = ordered_key(x);
       if (k >= kmin && k <= kmax) {
-        const int j = (int)(((unsigned long long)(k - kmin) * SMP_BINS) / width);
-        const int bin = SMP_BINS - 1 - j;            // descending key = ascending bin
+        const int bin = smp_key_bin(k, kmin, width);
         atomicAdd(&sh.hist[bin], smp_weight(x, mx, inv_t_log2e));
         atomicAdd(&sh.cnt[bin], 1u);
       }
     }
     __syncthreads();
-    smp_select_bin(sh, cut);
-    const unsigned long long j = (unsigned long long)(SMP_BINS - 1 - sh.sel_bin);
-    // keys k with floor((k - kmin) * BINS / width) == j
-    const unsigned long long lo = (j * width + SMP_BINS - 1) / SMP_BINS;
-    const unsigned long long hi = ((j + 1) * width + SMP_BINS - 1) / SMP_BINS - 1;
-    kmax = kmin + (uint32_t)hi;
-    kmin = kmin + (uint32_t)lo;
+    smp_select_bin(sh, cut, true);
+    const KeyRange kr = smp_narrow(sh, kmin, width);
+    kmin = kr.kmin; kmax = kr.kmax;
   }
   // Now every token with key == kmin (== kmax) is tied at the nucleus edge.
   const uint32_t kstar = kmin;
@@ -363,7 +346,7 @@ __global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
   const unsigned long long Z = carried + m_ties * wstar;
   const unsigned long long rdraw = __umul64hi(Z, (unsigned long long)u24 << 40);   // floor(u24 * Z / 2^24)
 
-  // ---- inverse CDF over nucleus members in ascending id order; thread = contiguous id range
+  // inverse CDF over nucleus members in ascending id order; thread = contiguous id range
   const int per = (V + SMP_THREADS - 1) / SMP_THREADS;
   const int i0 = min(V, tid * per), i1 = min(V, i0 + per);
   unsigned long long nt = 0ull;
@@ -395,6 +378,230 @@ __global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
     a.out_token[r] = tok;
   }
 }
+
+// Sampling S (top-p nucleus + inverse CDF) of one row per CTA, all in integers
+// once the weights are formed, so the result does not depend on the order in
+// which threads meet the tokens.  Four coalesced passes over the row: maximum;
+// coarse histogram of the weights over (max - logit); collection of the tokens
+// of the bin where the running weight reaches the cut (the nucleus edge is
+// then found among those few tokens in shared memory); per-warp totals of the
+// nucleus weights in id order, after which one warp walks its range to the drawn token.
+__global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
+  griddep_launch_dependents();
+  griddep_wait();
+  const int r = blockIdx.x;
+  if (!a.do_sample[r]) return;
+  __shared__ SmpShared sh;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int V = a.V;
+  const float *lg = a.logits + (size_t)r * V;
+  const bool vec = (V & 3) == 0 && (((uintptr_t)lg) & 15u) == 0;
+  const int n4 = V >> 2;
+
+  // ---- argmax, lowest id on ties
+  float bv = -CUDART_INF_F;
+  int bi = 0x7fffffff;
+  SMP_FOREACH(if (x > bv || (x == bv && i < bi)) { bv = x; bi = i; })
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+  }
+  if (lane == 0) { sh.red_val[warp] = bv; sh.red_idx[warp] = bi; }
+  __syncthreads();
+  bv = sh.red_val[0]; bi = sh.red_idx[0];
+  for (int w = 1; w < SMP_THREADS / 32; ++w) {
+    const float ov = sh.red_val[w];
+    const int oi = sh.red_idx[w];
+    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+  }
+  const float temperature = a.temperature[r];
+  if (!(temperature > 0.f)) {
+    if (tid == 0) a.out_token[r] = bi;
+    return;
+  }
+  const float mx = bv;
+  const float inv_t_log2e = __fdiv_rn(0x1.715476p+0f, temperature);
+  const uint32_t u24 = a.u24_override ? a.u24_override[r] : philox_u24(a.seed[r], (uint64_t)a.step[r]);
+
+  // ---- pass A: bins linear in (max - logit); bin 0 holds the largest logits
+  // weights vanish beyond (max - l)/T > 27.73, so the bins cover 28 T logit units
+  const float scale_a = (float)SMP_BINS / (28.f * temperature);
+  for (int i = tid; i < SMP_BINS; i += SMP_THREADS) { sh.hist[i] = 0ull; sh.cnt[i] = 0u; }
+  if (tid == 0) { sh.carried = 0ull; sh.kmin = 0xffffffffu; sh.kmax = 0u; sh.n_cand = 0u; sh.tie_max_id = 0x7fffffff; }
+  __syncthreads();
+  unsigned long long mysum = 0ull;
+  SMP_FOREACH({
+    (void)i;
+    const unsigned long long w = smp_weight(x, mx, inv_t_log2e);
+    if (w) {
+      atomicAdd(&sh.hist[min(SMP_BINS - 1, (int)((mx - x) * scale_a))], w);
+      mysum += w;
+    }
+  })
+  block_excl_scan_u64(mysum, sh.wtot, &sh.total);
+  const unsigned long long total = sh.total;
+  unsigned long long cut = __double2ull_rd((double)a.top_p[r] * (double)total);
+  if (cut > total) cut = total;
+  smp_select_bin(sh, cut, false);
+  const int bin_a = sh.sel_bin;
+
+  // ---- the tokens of the selected bin, with their key range
+  SMP_FOREACH({
+    if (min(SMP_BINS - 1, (int)((mx - x) * scale_a)) == bin_a) {
+      const unsigned int c = atomicAdd(&sh.n_cand, 1u);
+      if (c < (unsigned)SMP_CAND) { sh.cand_x[c] = x; sh.cand_id[c] = i; }
+      const uint32_t k = ordered_key(x);
+      atomicMin(&sh.kmin, k);
+      atomicMax(&sh.kmax, k);
+    }
+  })
+  __syncthreads();
+  const int n_cand = (int)sh.n_cand;
+  if (tid == 0) sh.sel_cnt = (unsigned)n_cand;   // stands if no refinement is needed: all those tokens share one key
+  __syncthreads();
+  if (n_cand > SMP_CAND) {   // uniform in the block
+    smp_tail_full_row(sh, a, r, lg, mx, inv_t_log2e, scale_a, bin_a, cut, u24);
+    return;
+  }
+  uint32_t kmin = sh.kmin, kmax = sh.kmax;
+  // ---- exact refinement in key space, over the candidates only, until one key remains
+  for (int pass = 0; pass < 4 && kmax > kmin; ++pass) {
+    const unsigned long long width = (unsigned long long)(kmax - kmin) + 1ull;
+    __syncthreads();
+    for (int i = tid; i < SMP_BINS; i += SMP_THREADS) { sh.hist[i] = 0ull; sh.cnt[i] = 0u; }
+    __syncthreads();
+    for (int c = tid; c < n_cand; c += SMP_THREADS) {
+      const float x = sh.cand_x[c];
+      const uint32_t k = ordered_key(x);
+      if (k >= kmin && k <= kmax) {
+        const int bin = smp_key_bin(k, kmin, width);
+        atomicAdd(&sh.hist[bin], smp_weight(x, mx, inv_t_log2e));
+        atomicAdd(&sh.cnt[bin], 1u);
+      }
+    }
+    __syncthreads();
+    smp_select_bin(sh, cut, true);
+    const KeyRange kr = smp_narrow(sh, kmin, width);
+    kmin = kr.kmin; kmax = kr.kmax;
+  }
+  __syncthreads();
+  // Now every token with key == kmin (== kmax) is tied at the nucleus edge.
+  const uint32_t kstar = kmin;
+  const unsigned long long carried = sh.carried;     // weight of tokens with key > kstar
+  const unsigned int n_tied = sh.sel_cnt;
+  const unsigned long long wstar = n_tied ? sh.sel_sum / n_tied : 0ull;
+  unsigned long long m_ties = 1ull;
+  if (wstar > 0ull && cut > carried) m_ties = (cut - carried + wstar - 1ull) / wstar;
+  if (m_ties < 1ull) m_ties = 1ull;
+  if (m_ties > n_tied) m_ties = n_tied;
+  const unsigned long long Z = carried + m_ties * wstar;
+  const unsigned long long rdraw = __umul64hi(Z, (unsigned long long)u24 << 40);   // floor(u24 * Z / 2^24)
+  // the tied tokens that belong to the nucleus are the m_ties lowest ids: find the largest of them
+  if (m_ties < n_tied) {
+    for (int c = tid; c < n_cand; c += SMP_THREADS) {
+      if (ordered_key(sh.cand_x[c]) != kstar) continue;
+      const int id = sh.cand_id[c];
+      unsigned long long rank = 0ull;
+      for (int j = 0; j < n_cand; ++j)
+        rank += (ordered_key(sh.cand_x[j]) == kstar && sh.cand_id[j] < id) ? 1ull : 0ull;
+      if (rank == m_ties - 1ull) sh.tie_max_id = id;
+    }
+  }
+  __syncthreads();
+  const int tie_max_id = sh.tie_max_id;
+
+  // ---- inverse CDF over the nucleus in ascending id order.  Warp w owns a contiguous id range and its
+  // lanes take consecutive float4 groups (or single ids), so ids ascend with the lane in every step.
+  const int units = vec ? n4 : V;                       // float4 groups or single ids
+  const int per_warp = (units + 31) / 32;
+  const int u_begin = min(units, warp * per_warp), u_end = min(units, u_begin + per_warp);
+  const int n_it = (per_warp + 31) / 32;                // the same for every warp
+  auto unit_weights = [&](int u, unsigned long long (&w)[4]) {
+    float xs[4];
+    int cntu = 1;
+    if (vec) {
+      const float4 q = reinterpret_cast<const float4 *>(lg)[u];
+      xs[0] = q.x; xs[1] = q.y; xs[2] = q.z; xs[3] = q.w;
+      cntu = 4;
+    } else {
+      xs[0] = lg[u];
+    }
+    const int id0 = vec ? 4 * u : u;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      w[j] = 0ull;
+      if (j < cntu) {
+        const uint32_t k = ordered_key(xs[j]);
+        if (k > kstar) w[j] = smp_weight(xs[j], mx, inv_t_log2e);
+        else if (k == kstar && id0 + j <= tie_max_id) w[j] = wstar;
+      }
+    }
+  };
+  unsigned long long ws = 0ull;
+  for (int it = 0; it < n_it; ++it) {
+    const int u = u_begin + it * 32 + lane;
+    if (u < u_end) {
+      unsigned long long w[4];
+      unit_weights(u, w);
+      ws += w[0] + w[1] + w[2] + w[3];
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ws += __shfl_xor_sync(0xffffffffu, ws, o);
+  __syncthreads();
+  if (lane == 0) sh.wtot[warp] = ws;
+  if (tid == 0) sh.sel_warp = 31;
+  __syncthreads();
+  if (warp == 0) {
+    const unsigned long long w = sh.wtot[lane];
+    unsigned long long inc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long n = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += n;
+    }
+    sh.wtot[lane] = inc - w;   // weight before the warp's range
+    if (rdraw >= inc - w && rdraw < inc) sh.sel_warp = lane;
+  }
+  __syncthreads();
+  if (warp != sh.sel_warp) return;
+  unsigned long long run = sh.wtot[warp];
+  int tok = (vec ? 4 * u_end : u_end) - 1;
+  for (int it = 0; it < n_it; ++it) {
+    const int u = u_begin + it * 32 + lane;
+    unsigned long long w[4] = {0ull, 0ull, 0ull, 0ull};
+    if (u < u_end) unit_weights(u, w);
+    const unsigned long long s = w[0] + w[1] + w[2] + w[3];
+    unsigned long long inc = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long n = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += n;
+    }
+    const unsigned hit = __ballot_sync(0xffffffffu, run + inc > rdraw);
+    if (hit) {
+      const int L = __ffs(hit) - 1;
+      if (lane == L) {
+        unsigned long long c = run + inc - s;
+        const int id0 = vec ? 4 * u : u;
+        int t = id0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          c += w[j];
+          if (c > rdraw) { t = id0 + j; break; }
+        }
+        tok = t;
+      }
+      tok = __shfl_sync(0xffffffffu, tok, L);
+      break;
+    }
+    run += __shfl_sync(0xffffffffu, inc, 31);
+  }
+  if (lane == 0) a.out_token[r] = tok;
+}
+#undef SMP_FOREACH
 
 // ---------------------------------------------------------------- decode bookkeeping
 __global__ void prepare_rows_kernel(const uint8_t *active_mask, const int *in_use, const int *ctx_len,

@@ -106,6 +106,12 @@ def test_sampler_ties_and_degenerate_rows(orc, torch_cuda):
     # all equal
     flat = np.zeros(1000, np.float32)
     assert _check_sampler(orc, flat, 1.0, 0.5, us) > 20
+    # more equal, or nearly equal, logits at the nucleus edge than the kernel keeps in shared memory
+    assert _check_sampler(orc, np.zeros(8192, np.float32), 1.0, 0.5, us) > 20
+    dense = (1.0 + rng.integers(0, 50, 6000) * 1.2e-7).astype(np.float32)
+    assert _check_sampler(orc, dense, 0.7, 0.6, us) > 20
+    mixed = np.concatenate([dense, (rng.standard_normal(3000) * 1.28).astype(np.float32)])
+    assert _check_sampler(orc, mixed, 0.7, 0.9, us) > 20
     # one dominant token, very wide range
     wide = (rng.standard_normal(3000) * 30).astype(np.float32)
     assert _check_sampler(orc, wide, 0.7, 0.95, us) > 20
