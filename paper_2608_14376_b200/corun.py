@@ -247,11 +247,11 @@ class Engine:
         return st.reshape(4 * self._cs.n_layers, n_sms, 8).astype(np.int64)
 
     def attn_trace(self, layer: int = 0) -> np.ndarray:
-        """Per-CTA, per-item attention timeline [n_ctas, 64, 4] in ns (0 where an item does not exist)."""
-        st = np.zeros(256 * 64 * 4, np.uint64)
+        """Per-CTA, per-item attention timeline [n_ctas, 64, 8] in ns (0 where an item does not exist)."""
+        st = np.zeros(256 * 64 * 8, np.uint64)
         n = C.c_int32(0)
         _check(lib().corun_debug_attn_trace(self._h, layer, st.ctypes.data, C.byref(n)), "attn_trace")
-        return st[:n.value * 256].reshape(n.value, 64, 4).astype(np.int64)
+        return st[:n.value * 512].reshape(n.value, 64, 8).astype(np.int64)
 
     def debug_read(self, which: int, n: int) -> np.ndarray:
         out = np.empty(n, np.float32)

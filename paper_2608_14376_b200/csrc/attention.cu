@@ -1,9 +1,14 @@
 // Request-local split-KV paged attention for one query token per row, on tcgen05.
 //
-// An item is (row, split of 128 cached tokens = 8 pages, kv head).  One persistent CTA per SM:
-//   warp 0        streams items with TMA into a ring of 3 item buffers (keys: [16 tokens x 64 dims]
-//                 boxes, 128-byte swizzle; values, cached transposed: [hd dims x 16 tokens] boxes,
-//                 32-byte swizzle), straight from the page pool through two tensor maps per layer;
+// An item is (row, kv head, split of 128 cached tokens = 8 pages); the step's items are listed in that
+// order and every CTA takes one contiguous stretch of the list, so consecutive items of a CTA mostly
+// share their query rows.  One persistent CTA per SM:
+//   warp 0        streams the items' keys with TMA into a ring of 3 key buffers ([16 tokens x 64 dims]
+//                 boxes, 128-byte swizzle), warp 1 their values into a ring of 3 value buffers (cached
+//                 transposed: [hd dims x 16 tokens] boxes, 32-byte swizzle), straight from the page pool
+//                 through two tensor maps per layer.  A key buffer is free again as soon as the scores
+//                 exist, a value buffer at the end of the item, so the key loads run ahead of the value
+//                 loads and more bytes are in flight than with whole-item buffers;
 //   2 groups of 4 warps take the items alternately.  Per item a group
 //     1. writes the query rows as fp16 hi/lo pairs into a [16 x hd] operand tile (rows 0..G-1 hi of
 //        the G query heads of this kv head, rows 8..8+G-1 their lo parts; q = hi + lo, 22 bits),
@@ -32,7 +37,7 @@ namespace {
 constexpr int ATT_NBUF = 3;                        // item buffers in the ring
 constexpr int ATT_GROUPS = 2;                      // consumer groups of 4 warps
 constexpr int ATT_SLOTS = 6;                       // barrier slots: a multiple of both
-constexpr int ATT_THREADS = 32 + ATT_GROUPS * 128; // producer warp + consumers
+constexpr int ATT_THREADS = 64 + ATT_GROUPS * 128; // two producer warps + consumers
 constexpr int ATT_PAGES = ATT_SPLIT / KV_BLOCK;    // 8 pages per split
 constexpr int KBOX_BYTES = KV_BLOCK * 128;         // one [16 tokens x 64 dims] fp16 key box
 constexpr int OPND_BYTES = 16 * 128;               // one [16 rows x 64 cols] fp16 half of a q / p operand tile
@@ -52,7 +57,8 @@ struct AttLayout {
   static constexpr int NHALF = HD / 64;                          // 64-dim halves of a key row
   static constexpr int K_BYTES = NHALF * ATT_PAGES * KBOX_BYTES; // keys of an item: [half][page][16 x 128 B]
   static constexpr int VT_BYTES = HD * KV_BLOCK * 2;             // one page's V^T tile: [hd x 32 B]
-  static constexpr int ITEM_BYTES = K_BYTES + ATT_PAGES * VT_BYTES;
+  static constexpr int V_BYTES = ATT_PAGES * VT_BYTES;           // values of an item
+  static constexpr int ITEM_BYTES = K_BYTES + V_BYTES;
   static constexpr int Q_BYTES = NHALF * OPND_BYTES;             // [half][16 x 128 B]
   static constexpr int P_BYTES = 2 * OPND_BYTES;                 // 128 tokens = 2 halves of 64
   static constexpr int GROUP_BYTES = Q_BYTES + P_BYTES;
@@ -61,24 +67,28 @@ struct AttLayout {
   static constexpr size_t SMEM = (size_t)ATT_NBUF * ITEM_BYTES + ATT_GROUPS * GROUP_BYTES + PAD_BYTES + 1024;
 };
 
-template <int HD>
+template <int HD, int GROUP>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                  const float *__restrict__ q, Rows rows, int nq, int group, KvLayout kv, int max_splits,
+                  const float *__restrict__ q, Rows rows, int nq, KvLayout kv, int max_splits,
                   const int *__restrict__ work, const int *__restrict__ n_work, float *__restrict__ part_acc,
                   float *__restrict__ part_ml, int *status, unsigned long long *trace) {
   using L = AttLayout<HD>;
-  // optional timeline (debug): per CTA and item (first 64): [load issued, item landed, group starts, released]
-#define ATRACE(k, i) do { if (trace && (k) < 64) trace[((size_t)blockIdx.x * 64 + (k)) * 4 + (i)] = globaltimer_ns(); } while (0)
+  // optional timeline (debug): per CTA and item (first 64): [key load issued, keys landed, group starts, released, scores done, weights written, values landed, output done]
+#define ATRACE(k, i) do { if (trace && (k) < 64) trace[((size_t)blockIdx.x * 64 + (k)) * 8 + (i)] = globaltimer_ns(); } while (0)
   constexpr int KSTEPS = HD / 16;
   griddep_launch_dependents();
   griddep_wait();                                // the item list and q come from earlier kernels
-  const int n_items = *n_work * kv.n_kv;
-  if ((int)blockIdx.x >= n_items) return;
+  constexpr int group = GROUP;                   // query heads per kv head
+  const int n_total = *n_work;
+  // this CTA's stretch of the item list
+  const int item_lo = (int)(((long long)blockIdx.x * n_total) / gridDim.x);
+  const int n_items = (int)(((long long)(blockIdx.x + 1) * n_total) / gridDim.x) - item_lo;
+  if (n_items <= 0) return;
 
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_bar[ATT_SLOTS];
-  __shared__ __align__(8) uint64_t empty_bar[ATT_NBUF];
+  __shared__ __align__(8) uint64_t kfull_bar[ATT_SLOTS], vfull_bar[ATT_SLOTS];
+  __shared__ __align__(8) uint64_t kempty_bar[ATT_NBUF], vempty_bar[ATT_NBUF];
   __shared__ __align__(8) uint64_t mma_bar[ATT_GROUPS];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
@@ -90,18 +100,18 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   if (tid == 0) {
     abort_flag = 0;
     for (int g = 0; g < ATT_GROUPS; ++g) { stop_s[g] = 0; mbar_init(smem_u32(&mma_bar[g]), 1); }
-    for (int s = 0; s < ATT_SLOTS; ++s) mbar_init(smem_u32(&full_bar[s]), 1);
-    for (int b = 0; b < ATT_NBUF; ++b) mbar_init(smem_u32(&empty_bar[b]), 1);
+    for (int s = 0; s < ATT_SLOTS; ++s) { mbar_init(smem_u32(&kfull_bar[s]), 1); mbar_init(smem_u32(&vfull_bar[s]), 1); }
+    for (int b = 0; b < ATT_NBUF; ++b) { mbar_init(smem_u32(&kempty_bar[b]), 1); mbar_init(smem_u32(&vempty_bar[b]), 1); }
     fence_mbar_init();
     fence_proxy_async();
   }
   if (warp == 0) {
     tmem_alloc(smem_u32(&tmem_base_s), ATT_TMEM_COLS);
     tmem_relinquish();
-  } else {
+  } else if (warp >= 2) {
     // operand tiles start out as zeros: rows of unused heads are never written and must stay finite
     uint4 *z = reinterpret_cast<uint4 *>(ring_ptr + (size_t)ATT_NBUF * L::ITEM_BYTES);
-    for (int i = tid - 32; i < ATT_GROUPS * L::GROUP_BYTES / 16; i += ATT_THREADS - 32) z[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = tid - 64; i < ATT_GROUPS * L::GROUP_BYTES / 16; i += ATT_THREADS - 64) z[i] = make_uint4(0u, 0u, 0u, 0u);
   }
   tc_fence_before();
   __syncthreads();
@@ -112,42 +122,51 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   // M = 128 (M >> 4 at bit 24)
   const uint32_t idesc = (1u << 4) | ((uint32_t)(16 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
-  if (warp == 0) {
-    // ---------------- producer: one lane per page ----------------
+  // shared memory: [key ring][value ring][operand tiles of the groups]
+  const uint32_t vring = ring + (uint32_t)ATT_NBUF * L::K_BYTES;
+  if (warp < 2) {
+    // ---------------- producers: warp 0 keys, warp 1 values; one lane per page ----------------
+    const bool is_v = warp == 1;
     const uint64_t pol = l2_policy_evict_first();       // the cache is streamed once per step
-    int k = 0;
-    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++k) {
+    uint64_t *full = is_v ? vfull_bar : kfull_bar, *empty = is_v ? vempty_bar : kempty_bar;
+    for (int k = 0; k < n_items; ++k) {
       const int buf = k % ATT_NBUF, slot = k % ATT_SLOTS;
       if (k >= ATT_NBUF) {                               // the buffer's previous item must have been released
-        bool ok = mbar_wait(smem_u32(&empty_bar[buf]), (uint32_t)(k / ATT_NBUF - 1) & 1u, &abort_flag);
+        bool ok = mbar_wait(smem_u32(&empty[buf]), (uint32_t)(k / ATT_NBUF - 1) & 1u, &abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { failed = true; break; }
       }
-      const int wi = work[item / kv.n_kv], g = item % kv.n_kv;
-      const int r = wi >> 8, split = wi & 255;
+      const int wi = work[item_lo + k];
+      const int r = wi >> 16, g = (wi >> 8) & 255, split = wi & 255;
       const int ctx = rows.pos[r] + 1;
       const int t0 = split * ATT_SPLIT;
       const int n_pages = min(ATT_PAGES, (ctx - t0 + KV_BLOCK - 1) / KV_BLOCK);
-      const uint32_t fb = smem_u32(&full_bar[slot]);
-      if (lane == 0) { ATRACE(k, 0); mbar_arrive_expect_tx(fb, (uint32_t)(n_pages * (L::NHALF * KBOX_BYTES + L::VT_BYTES))); }
+      const uint32_t fb = smem_u32(&full[slot]);
+      if (lane == 0) {
+        if (!is_v) ATRACE(k, 0);
+        mbar_arrive_expect_tx(fb, (uint32_t)(n_pages * (is_v ? L::VT_BYTES : L::NHALF * KBOX_BYTES)));
+      }
       __syncwarp();
       if (lane < n_pages) {
         const int page = kv.block_table[(size_t)rows.slot[r] * kv.max_blocks + t0 / KV_BLOCK + lane];
         // this layer's pages as rows of hd halfs: the key tile of (page, head) starts at row
         //   page * 2 * n_kv * 16 + head * 16;
         // as rows of 16 halfs: the transposed value tile starts at row page * 2 * n_kv * hd + (n_kv + head) * hd
-        const int row_k = (page * 2 * kv.n_kv + g) * KV_BLOCK;
-        const int row_v = (page * 2 * kv.n_kv + kv.n_kv + g) * HD;
-        const uint32_t item_base = ring + (uint32_t)buf * L::ITEM_BYTES;
+        if (is_v) {
+          const int row_v = (page * 2 * kv.n_kv + kv.n_kv + g) * HD;
+          tma_load_2d(vring + (uint32_t)buf * L::V_BYTES + (uint32_t)lane * L::VT_BYTES, &tmV, 0, row_v, fb, pol);
+        } else {
+          const int row_k = (page * 2 * kv.n_kv + g) * KV_BLOCK;
+          const uint32_t kb = ring + (uint32_t)buf * L::K_BYTES;
 #pragma unroll
-        for (int x = 0; x < L::NHALF; ++x)
-          tma_load_2d(item_base + (uint32_t)(x * ATT_PAGES + lane) * KBOX_BYTES, &tmK, x * 64, row_k, fb, pol);
-        tma_load_2d(item_base + L::K_BYTES + (uint32_t)lane * L::VT_BYTES, &tmV, 0, row_v, fb, pol);
+          for (int x = 0; x < L::NHALF; ++x)
+            tma_load_2d(kb + (uint32_t)(x * ATT_PAGES + lane) * KBOX_BYTES, &tmK, x * 64, row_k, fb, pol);
+        }
       }
     }
   } else {
     // ---------------- consumers ----------------
-    const int gi = (warp - 1) >> 2, gtid = (tid - 32) & 127;
+    const int gi = (warp - 2) >> 2, gtid = (tid - 64) & 127;
     const int quad = warp & 3;                     // the TMEM lane quarter this warp may read
     const int tl = quad * 32 + lane;               // TMEM lane of this thread: token (scores) / dim (values)
     const float sscale = (HD == 128 ? 0.08838834764831845f : 0.125f) * 1.4426950408889634f;   // log2(e)/sqrt(hd)
@@ -158,8 +177,8 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     const uint32_t s_tmem = tmem_base + (uint32_t)gi * 32;       // S^T: 16 columns
     const uint32_t o_tmem = s_tmem + 16;                          // O^T: 16 columns
     const uint32_t mbar = smem_u32(&mma_bar[gi]);
-    uint32_t mma_phase = 0, full_bits = 0;         // bit j: phase of the full barrier of this group's j-th slot
-    constexpr int QPT = (8 * (HD / 2) + 127) / 128;   // float2 query values per thread (up to 8 heads)
+    uint32_t mma_phase = 0, full_bits = 0;         // bit j: phase of the full barriers of this group's j-th slot
+    constexpr int QPT = (GROUP * (HD / 2) + 127) / 128;   // float2 query values per thread
     float2 qreg[QPT];
     auto load_q = [&](int r_, int g_) {
 #pragma unroll
@@ -171,44 +190,42 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         }
       }
     };
-    if ((int)blockIdx.x + gi * (int)gridDim.x < n_items) {
-      const int it0 = blockIdx.x + gi * gridDim.x;
-      load_q(work[it0 / kv.n_kv] >> 8, it0 % kv.n_kv);
-    }
-    int k = gi;
-    for (int item = blockIdx.x + gi * gridDim.x; item < n_items; item += ATT_GROUPS * gridDim.x, k += ATT_GROUPS) {
+    int q_built = -1, q_loaded = -1;               // (row, kv head) keys of the operand tile / of qreg
+    for (int k = gi; k < n_items; k += ATT_GROUPS) {
       const int buf = k % ATT_NBUF, slot = k % ATT_SLOTS, j = slot / ATT_GROUPS;
-      const int wi = work[item / kv.n_kv], g = item % kv.n_kv;
-      const int r = wi >> 8, split = wi & 255;
+      const int wi = work[item_lo + k];
+      const int r = wi >> 16, g = (wi >> 8) & 255, split = wi & 255;
       const int ctx = rows.pos[r] + 1;               // the new token attends to itself too
       const int t0 = split * ATT_SPLIT;
       const int n_pages = min(ATT_PAGES, (ctx - t0 + KV_BLOCK - 1) / KV_BLOCK);
-      const uint32_t k_tiles = ring + (uint32_t)buf * L::ITEM_BYTES;
-      const uint32_t v_tiles = k_tiles + L::K_BYTES;
+      const uint32_t k_tiles = ring + (uint32_t)buf * L::K_BYTES;
+      const uint32_t v_tiles = vring + (uint32_t)buf * L::V_BYTES;
 
       if (gtid == 0) ATRACE(k, 2);
       // ---- 1. query operand tile: rows h (hi) and 8 + h (lo) of head g * group + h; the scale goes on the
-      //         scores.  The values were fetched one item ahead (qreg), so no global latency sits here.
+      //         scores.  Rebuilt only when (row, kv head) changes; the values were normally fetched one
+      //         item ahead (qreg), so no global latency sits here.
+      if ((wi >> 8) != q_built) {
+        if (q_loaded != (wi >> 8)) load_q(r, g);
 #pragma unroll
-      for (int i = 0; i < QPT; ++i) {
-        const int idx = gtid + i * 128;
-        if (idx < group * (HD / 2)) {
-          const int h = idx / (HD / 2), d = (idx - h * (HD / 2)) * 2;
-          __half h0, l0, h1, l1;
-          split_half(qreg[i].x, h0, l0);
-          split_half(qreg[i].y, h1, l1);
-          const uint32_t off = (uint32_t)(d >> 6) * OPND_BYTES + (uint32_t)((d & 7) * 2);
-          const int chunk = (d & 63) >> 3;
-          *reinterpret_cast<__half2 *>(q_ptr + off + swz(h, chunk)) = __halves2half2(h0, h1);
-          *reinterpret_cast<__half2 *>(q_ptr + off + swz(8 + h, chunk)) = __halves2half2(l0, l1);
+        for (int i = 0; i < QPT; ++i) {
+          const int idx = gtid + i * 128;
+          if (idx < group * (HD / 2)) {
+            const int h = idx / (HD / 2), d = (idx - h * (HD / 2)) * 2;
+            __half h0, l0, h1, l1;
+            split_half(qreg[i].x, h0, l0);
+            split_half(qreg[i].y, h1, l1);
+            const uint32_t off = (uint32_t)(d >> 6) * OPND_BYTES + (uint32_t)((d & 7) * 2);
+            const int chunk = (d & 63) >> 3;
+            *reinterpret_cast<__half2 *>(q_ptr + off + swz(h, chunk)) = __halves2half2(h0, h1);
+            *reinterpret_cast<__half2 *>(q_ptr + off + swz(8 + h, chunk)) = __halves2half2(l0, l1);
+          }
         }
+        q_built = q_loaded = wi >> 8;
       }
-      {   // fetch the next item's query values now; they are consumed at the top of the next iteration
-        const int nxt = item + ATT_GROUPS * (int)gridDim.x;
-        if (nxt < n_items) {
-          const int nwi = work[nxt / kv.n_kv], ng = nxt % kv.n_kv, nr = nwi >> 8;
-          load_q(nr, ng);
-        }
+      if (k + ATT_GROUPS < n_items) {   // fetch the next item's query values now if they differ
+        const int nwi = work[item_lo + k + ATT_GROUPS];
+        if ((nwi >> 8) != q_built) { load_q(nwi >> 16, (nwi >> 8) & 255); q_loaded = nwi >> 8; }
       }
       fence_proxy_async();                           // the MMA reads this tile through the async proxy
       if (gtid == 0) stop_s[gi] = abort_flag;
@@ -217,7 +234,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 
       // ---- 2. S^T = K * Q^T, issued by one thread once the item has landed
       if (gtid == 0) {
-        const bool ok = mbar_wait(smem_u32(&full_bar[slot]), (full_bits >> j) & 1u, &abort_flag);
+        const bool ok = mbar_wait(smem_u32(&kfull_bar[slot]), (full_bits >> j) & 1u, &abort_flag);
         ATRACE(k, 1);
         if (ok) {
           tc_fence_after();
@@ -231,7 +248,6 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         }
         umma_commit(mbar);                           // also arrives if the wait gave up: nobody may hang here
       }
-      full_bits ^= 1u << j;
       {
         bool ok = mbar_wait(mbar, mma_phase, &abort_flag);
         ok = __all_sync(0xffffffffu, ok);
@@ -239,15 +255,16 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         if (!ok) failed = true;
       }
       tc_fence_after();
+      if (gtid == 0) { mbar_arrive(smem_u32(&kempty_bar[buf])); ATRACE(k, 4); }   // the scores exist: the key buffer is free
 
       // ---- 3. softmax over the item; this thread owns token t0 + tl
       uint32_t sv[16];
       tmem_ld16(s_tmem + ((uint32_t)(quad * 32) << 16), sv);
       tmem_ld_wait();
       const bool tok_ok = t0 + tl < ctx;
-      float sc[8];
+      float sc[GROUP];
 #pragma unroll
-      for (int h = 0; h < 8; ++h) {
+      for (int h = 0; h < GROUP; ++h) {
         sc[h] = tok_ok ? (__uint_as_float(sv[h]) + __uint_as_float(sv[8 + h])) * sscale : -CUDART_INF_F;
         float m = sc[h];
 #pragma unroll
@@ -255,10 +272,10 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         if (lane == h) red_s[gi][quad][h] = m;
       }
       asm volatile("bar.sync %0, 128;" ::"r"(1 + gi) : "memory");
-      float pr[8], mx[8];
+      float pr[GROUP], mx[GROUP];
       float my_sum = 0.f;                            // lane h keeps the warp's sum of head h
 #pragma unroll
-      for (int h = 0; h < 8; ++h) {
+      for (int h = 0; h < GROUP; ++h) {
         // exact maximum over the 128 tokens (token t0 is always valid, so it is finite for used heads)
         mx[h] = fmaxf(fmaxf(red_s[gi][0][h], red_s[gi][1][h]), fmaxf(red_s[gi][2][h], red_s[gi][3][h]));
         pr[h] = exp2f(sc[h] - mx[h]);                // 0 for masked tokens
@@ -268,19 +285,17 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         if (lane == h) my_sum = s;
       }
       asm volatile("bar.sync %0, 128;" ::"r"(1 + gi) : "memory");   // everyone has read the maxima
-      if (lane < 8) red_s[gi][quad][lane] = my_sum;
+      if (lane < GROUP) red_s[gi][quad][lane] = my_sum;
       // weights as fp16 hi/lo into the [16 x 128 tokens] operand tile: rows h and 8 + h, column = token
       {
         const uint32_t off = (uint32_t)(tl >> 6) * OPND_BYTES + (uint32_t)((tl & 7) * 2);
         const int chunk = (tl & 63) >> 3;
 #pragma unroll
-        for (int h = 0; h < 8; ++h) {
-          if (h < group) {
-            __half ph, pl;
-            split_half(pr[h], ph, pl);
-            *reinterpret_cast<__half *>(p_ptr + off + swz(h, chunk)) = ph;
-            *reinterpret_cast<__half *>(p_ptr + off + swz(8 + h, chunk)) = pl;
-          }
+        for (int h = 0; h < GROUP; ++h) {
+          __half ph, pl;
+          split_half(pr[h], ph, pl);
+          *reinterpret_cast<__half *>(p_ptr + off + swz(h, chunk)) = ph;
+          *reinterpret_cast<__half *>(p_ptr + off + swz(8 + h, chunk)) = pl;
         }
       }
       fence_proxy_async();
@@ -289,14 +304,18 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 
       // ---- 4. O^T = V^T * P^T, one MMA per loaded page (16 tokens)
       if (gtid == 0) {
+        ATRACE(k, 5);
+        const bool ok = mbar_wait(smem_u32(&vfull_bar[slot]), (full_bits >> j) & 1u, &abort_flag);
+        ATRACE(k, 6);
         tc_fence_after();
-        for (int p = 0; p < n_pages; ++p) {
+        for (int p = 0; ok && p < n_pages; ++p) {
           const uint64_t a = umma_desc_sw32(v_tiles + (uint32_t)p * L::VT_BYTES);
           const uint64_t b = umma_desc_sw128(p_tile + (uint32_t)(p >> 2) * OPND_BYTES) + (uint64_t)((p & 3) * 2);
           umma_bf16(o_tmem, a, b, idesc, p > 0 ? 1u : 0u);
         }
-        umma_commit(mbar);
+        umma_commit(mbar);                           // also arrives if the wait gave up
       }
+      full_bits ^= 1u << j;
       {
         bool ok = mbar_wait(mbar, mma_phase, &abort_flag);
         ok = __all_sync(0xffffffffu, ok);
@@ -304,6 +323,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         if (!ok) failed = true;
       }
       tc_fence_after();
+      if (gtid == 0) { mbar_arrive(smem_u32(&vempty_bar[buf])); ATRACE(k, 7); }   // the value buffer is free
 
       // ---- 5. this thread owns output dim tl: add the hi and lo columns, write the partial
       if (quad * 32 < HD) {                          // warp-uniform: with hd = 64 only lanes 0-63 hold dims
@@ -311,24 +331,22 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         tmem_ld16(o_tmem + ((uint32_t)(quad * 32) << 16), ov);
         tmem_ld_wait();
 #pragma unroll
-        for (int h = 0; h < 8; ++h) {
-          if (h < group) {
-            const size_t pslot = ((size_t)r * nq + g * group + h) * max_splits + split;
-            part_acc[pslot * HD + tl] = __uint_as_float(ov[h]) + __uint_as_float(ov[8 + h]);
-          }
+        for (int h = 0; h < GROUP; ++h) {
+          const size_t pslot = ((size_t)r * nq + g * group + h) * max_splits + split;
+          part_acc[pslot * HD + tl] = __uint_as_float(ov[h]) + __uint_as_float(ov[8 + h]);
         }
       }
 #pragma unroll
-      for (int h = 0; h < 8; ++h) {
-        if (h < group && gtid == h) {              // red_s holds the four warps' sums by now
+      for (int h = 0; h < GROUP; ++h) {
+        if (gtid == h) {                           // red_s holds the four warps' sums by now
           const size_t pslot = ((size_t)r * nq + g * group + h) * max_splits + split;
           part_ml[pslot * 2] = mx[h];
           part_ml[pslot * 2 + 1] = ((red_s[gi][0][h] + red_s[gi][1][h]) + red_s[gi][2][h]) + red_s[gi][3][h];
         }
       }
       tc_fence_before();
-      asm volatile("bar.sync %0, 128;" ::"r"(1 + gi) : "memory");   // the item's buffers and TMEM are free
-      if (gtid == 0) { mbar_arrive(smem_u32(&empty_bar[buf])); ATRACE(k, 3); }
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + gi) : "memory");   // the group's TMEM and operand tiles are free
+      if (gtid == 0) ATRACE(k, 3);
     }
   }
   if (failed || abort_flag) {
@@ -411,9 +429,10 @@ attn_combine_kernel(Rows rows, int nq, int max_splits, const float *__restrict__
   }
 }
 
-// Lists the (row, split) items of the step: active rows in ascending order, splits ascending.
-// One CTA; rows <= 256.  Entry = row << 8 | split.
-__global__ void __launch_bounds__(256) attn_worklist_kernel(Rows rows, int *__restrict__ work, int *__restrict__ n_work) {
+// Lists the items of the step: active rows ascending, kv heads ascending, splits ascending.
+// One CTA; rows <= 256.  Entry = row << 16 | kv head << 8 | split.
+__global__ void __launch_bounds__(256) attn_worklist_kernel(Rows rows, int n_kv, int *__restrict__ work,
+                                                            int *__restrict__ n_work) {
   griddep_launch_dependents();
   griddep_wait();
   __shared__ int cnt[256];
@@ -421,25 +440,66 @@ __global__ void __launch_bounds__(256) attn_worklist_kernel(Rows rows, int *__re
   const int mine = (r < rows.R && rows.active[r]) ? (rows.pos[r] + 1 + ATT_SPLIT - 1) / ATT_SPLIT : 0;
   cnt[r] = mine;
   __syncthreads();
-  int before = 0;
-  for (int i = 0; i < r; ++i) before += cnt[i];
-  for (int s = 0; s < mine; ++s) work[before + s] = (r << 8) | s;
-  if (r == 255) *n_work = before + mine;
+  // every warp lists one row at a time
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int row = warp; row < rows.R; row += 8) {
+    int before = 0;
+    for (int i = lane; i < row; i += 32) before += cnt[i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+    const int ns = cnt[row];
+    for (int i = lane; i < ns * n_kv; i += 32) work[before * n_kv + i] = (row << 16) | ((i / ns) << 8) | (i % ns);
+  }
+  if (r == 255) {
+    int tot = 0;
+    for (int i = 0; i < 256; ++i) tot += cnt[i];
+    *n_work = tot * n_kv;
+  }
 }
 
 }  // namespace
 
+namespace {
+template <int HD, int GROUP>
+cudaError_t prepare_one() {
+  return cudaFuncSetAttribute(attn_split_kernel<HD, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)AttLayout<HD>::SMEM);
+}
+template <int HD>
+cudaError_t launch_attn_split(int group, int grid, cudaStream_t st, const CUtensorMap &tmK, const CUtensorMap &tmV,
+                         const float *q, const Rows &rows, int nq, const KvLayout &kv, int max_splits, const int *work,
+                         const int *n_work, float *part_acc, float *part_ml, int *d_status, unsigned long long *trace) {
+#define CORUN_ATT_CASE(G)                                                                                          \
+  case G:                                                                                                          \
+    return launch_k(attn_split_kernel<HD, G>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
+                    rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, d_status, trace);
+  switch (group) {
+    CORUN_ATT_CASE(1)
+    CORUN_ATT_CASE(2)
+    CORUN_ATT_CASE(4)
+    CORUN_ATT_CASE(8)
+    default: return cudaErrorInvalidValue;
+  }
+#undef CORUN_ATT_CASE
+}
+}  // namespace
+
 cudaError_t attention_prepare() {
-  cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)AttLayout<128>::SMEM);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(attn_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)AttLayout<64>::SMEM);
+  cudaError_t e = cudaSuccess;
+  if (e == cudaSuccess) e = prepare_one<128, 1>();
+  if (e == cudaSuccess) e = prepare_one<128, 2>();
+  if (e == cudaSuccess) e = prepare_one<128, 4>();
+  if (e == cudaSuccess) e = prepare_one<128, 8>();
+  if (e == cudaSuccess) e = prepare_one<64, 1>();
+  if (e == cudaSuccess) e = prepare_one<64, 2>();
+  if (e == cudaSuccess) e = prepare_one<64, 4>();
+  if (e == cudaSuccess) e = prepare_one<64, 8>();
+  return e;
 }
 
-cudaError_t launch_attn_worklist(const Rows &rows, int *work, int *n_work, cudaStream_t st) {
-  if (rows.R > 256) return cudaErrorInvalidValue;
-  return launch_k(attn_worklist_kernel, dim3(1), dim3(256), 0, st, true, rows, work, n_work);
+cudaError_t launch_attn_worklist(const Rows &rows, int n_kv, int *work, int *n_work, cudaStream_t st) {
+  if (rows.R > 256 || n_kv > 255) return cudaErrorInvalidValue;
+  return launch_k(attn_worklist_kernel, dim3(1), dim3(256), 0, st, true, rows, n_kv, work, n_work);
 }
 
 cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, const float *q, const Rows &rows, int nq,
@@ -448,16 +508,14 @@ cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, con
                              __nv_bfloat16 *out_lo, int *d_status, cudaStream_t st, unsigned long long *trace) {
   (void)layer;   // the tensor maps are the layer's
   const int group = nq / kv.n_kv;
-  if (group < 1 || group > 8 || max_splits > 256) return cudaErrorInvalidValue;
+  if (group * kv.n_kv != nq || max_splits > 256) return cudaErrorInvalidValue;
   const long long most = (long long)rows.R * max_splits * kv.n_kv;
   const int grid = (int)(most < grid_ctas ? most : grid_ctas);
   cudaError_t e;
   if (kv.hd == 128)
-    e = launch_k(attn_split_kernel<128>, dim3(grid), dim3(ATT_THREADS), AttLayout<128>::SMEM, st, true, tmK, tmV, q, rows,
-                 nq, group, kv, max_splits, work, n_work, part_acc, part_ml, d_status, trace);
+    e = launch_attn_split<128>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, d_status, trace);
   else if (kv.hd == 64)
-    e = launch_k(attn_split_kernel<64>, dim3(grid), dim3(ATT_THREADS), AttLayout<64>::SMEM, st, true, tmK, tmV, q, rows,
-                 nq, group, kv, max_splits, work, n_work, part_acc, part_ml, d_status, trace);
+    e = launch_attn_split<64>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, d_status, trace);
   else
     return cudaErrorInvalidValue;
   if (e != cudaSuccess) return e;

@@ -138,7 +138,7 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm) {
     RC(dmalloc(A, &P.q, (size_t)R * QD));
     RC(dmalloc(A, &P.part_acc, (size_t)R * s.n_q_heads * e->max_splits * s.head_dim));
     RC(dmalloc(A, &P.part_ml, (size_t)R * s.n_q_heads * e->max_splits * 2));
-    RC(dmalloc(A, &P.att_work, (size_t)R * e->max_splits));
+    RC(dmalloc(A, &P.att_work, (size_t)R * e->max_splits * e->sh.n_kv_heads));
     RC(dmalloc(A, &P.att_n_work, 1));
     RC(dmalloc(A, &P.qkv_out, (size_t)R * (QD + 2 * KD)));
     RC(dmalloc(A, &P.o_out, (size_t)R * H));
@@ -182,7 +182,7 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
   const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
   const KvLayout kv = kv_layout(e);
   int n = 0;
-  CK(launch_attn_worklist(rows, P.att_work, P.att_n_work, e->st));   // the same items serve every layer
+  CK(launch_attn_worklist(rows, e->sh.n_kv_heads, P.att_work, P.att_n_work, e->st));   // the same items serve every layer
   n += 1;
   // (debug) slice of the step trace for the idx-th GEMM of the decode program: [num_sms][8] stamps
   auto tr = [&](int idx) -> unsigned long long * {
@@ -785,7 +785,7 @@ int corun_debug_attn_trace(corun_engine *e, int32_t layer, uint64_t *stamps, int
   Program &P = e->dec;
   const corun_shape &s = e->sh;
   const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
-  const size_t n = (size_t)e->num_sms * 64 * 4;
+  const size_t n = (size_t)e->num_sms * 64 * 8;
   unsigned long long *d = nullptr;
   if (cudaMalloc(&d, n * sizeof(unsigned long long)) != cudaSuccess) return CORUN_ENOMEM;
   cudaError_t ce = cudaMemsetAsync(d, 0, n * sizeof(unsigned long long), e->st);

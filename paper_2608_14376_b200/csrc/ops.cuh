@@ -63,14 +63,14 @@ cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *
 // Split-KV paged attention partials and their fixed-order combine -> bf16 hi/lo [R, nq*hd].
 // tmK / tmV: tensor maps over this layer's pages: keys as rows of hd halfs with a [16, 64] box (128-byte
 // swizzle), values as rows of 16 halfs with an [hd, 16] box (32-byte swizzle); see attention.cu.
-// work / n_work: the step's (row, split) items from launch_attn_worklist (the same for every layer);
+// work / n_work: the step's (row, kv head, split) items from launch_attn_worklist (the same for every layer);
 // grid_ctas: persistent CTAs to launch (one per SM).
 cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, const float *q, const Rows &rows, int nq,
                              const KvLayout &kv, int layer, int max_splits, const int *work, const int *n_work,
                              int grid_ctas, float *part_acc, float *part_ml, __nv_bfloat16 *out_hi,
                              __nv_bfloat16 *out_lo, int *d_status, cudaStream_t st,
-                             unsigned long long *trace = nullptr);   // optional [grid][64][4] stamps (debug)
-cudaError_t launch_attn_worklist(const Rows &rows, int *work, int *n_work, cudaStream_t st);
+                             unsigned long long *trace = nullptr);   // optional [grid][64][8] stamps (debug)
+cudaError_t launch_attn_worklist(const Rows &rows, int n_kv, int *work, int *n_work, cudaStream_t st);
 cudaError_t attention_prepare();   // opts the kernels into their shared-memory size (idempotent)
 // y = silu(gate) * up from the gate-up GEMM result -> bf16 hi/lo [R, F].
 cudaError_t launch_swiglu(const GemmOut &gu, int R, int F, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, cudaStream_t st);
