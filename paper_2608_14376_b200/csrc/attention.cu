@@ -17,7 +17,10 @@
 //     3. softmax over the item: exact max and a fixed-order sum over the 128 tokens,
 //        weights written as fp16 hi/lo rows of a [16 x 128 tokens] operand tile,
 //     4. O^T[hd dims x 16] = V^T[hd x 128 tokens] * P^T  (one MMA per page), TMEM lane = dim,
-//     5. adds the hi and lo columns and writes the split's partial (max, sum, O) to global memory.
+//     5. adds the hi and lo columns and writes the split's partial (max, sum, O) to global memory;
+//   4 combiner warps: when a group leaves a (row, kv head) it reports how many of that pair's splits it
+//   wrote; the combiners add this to the pair's device-wide counter and, when the count is complete,
+//   combine the pair's splits (in ascending split order, so it does not matter who does it).
 // The cached K / V are fp16 exactly, accumulation is fp32.
 //
 // Invariance: the split size is fixed, the split count is a function of the row's own context
@@ -37,7 +40,8 @@ namespace {
 constexpr int ATT_NBUF = 3;                        // item buffers in the ring
 constexpr int ATT_GROUPS = 2;                      // consumer groups of 4 warps
 constexpr int ATT_SLOTS = 6;                       // barrier slots: a multiple of both
-constexpr int ATT_THREADS = 64 + ATT_GROUPS * 128; // two producer warps + consumers
+constexpr int ATT_THREADS = 64 + ATT_GROUPS * 128 + 128; // two producer warps + consumers + combiners
+constexpr int ATT_QDEPTH = 8;                      // reports a group may have outstanding
 constexpr int ATT_PAGES = ATT_SPLIT / KV_BLOCK;    // 8 pages per split
 constexpr int KBOX_BYTES = KV_BLOCK * 128;         // one [16 tokens x 64 dims] fp16 key box
 constexpr int OPND_BYTES = 16 * 128;               // one [16 rows x 64 cols] fp16 half of a q / p operand tile
@@ -50,6 +54,68 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) { return (uint32_t)(
 __device__ __forceinline__ void split_half(float x, __half &hi, __half &lo) {
   hi = __float2half_rn(x);
   lo = __float2half_rn(x - __half2float(hi));
+}
+
+// Combines the splits of one (row, head) by one warp.  Lanes first hold one split each (max by
+// butterfly, which is exact; the denominator by a fixed butterfly over at most 32 lanes, then
+// ascending chunks of 32), then every lane owns hd/32 output dims and adds the splits' weighted
+// partial outputs in ascending split order.  Output: bf16 hi/lo pair for the O projection.
+// The partials may come from other SMs: they are read past the L1 cache.
+template <int HD>
+__device__ __forceinline__ void attn_combine_pair(int r, int j, int nsplit, int nq, int max_splits,
+                                                  const float *__restrict__ part_acc, const float *__restrict__ part_ml,
+                                                  __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo,
+                                                  int lane) {
+  constexpr int DPL = HD / 32;                   // dims per lane (4 or 2)
+  float o[DPL];
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) o[i] = 0.f;
+  const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + ((size_t)r * nq + j) * max_splits;
+  const float *pa = part_acc + ((size_t)r * nq + j) * max_splits * HD + lane * DPL;
+  float M = -CUDART_INF_F;
+  for (int s0 = 0; s0 < nsplit; s0 += 32) {
+    float m = (s0 + lane < nsplit) ? __ldcg(ml + s0 + lane).x : -CUDART_INF_F;
+#pragma unroll
+    for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
+    M = fmaxf(M, m);
+  }
+  float den = 0.f;
+  for (int s0 = 0; s0 < nsplit; s0 += 32) {
+    float2 v = (s0 + lane < nsplit) ? __ldcg(ml + s0 + lane) : make_float2(-CUDART_INF_F, 0.f);
+    const float w = exp2f(v.x - M);              // this lane's split weight (0 beyond the last split)
+    float d = v.y * w;
+#pragma unroll
+    for (int k = 16; k > 0; k >>= 1) d += __shfl_xor_sync(0xffffffffu, d, k);
+    den += d;
+    const int cnt = min(32, nsplit - s0);
+    for (int sb = 0; sb < cnt; sb += 8) {          // eight splits' partial outputs are fetched together
+      float4 a[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        a[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (sb + u < cnt) {
+          const float *p = pa + (size_t)(s0 + sb + u) * HD;
+          if (DPL == 4) a[u] = __ldcg(reinterpret_cast<const float4 *>(p));
+          else { const float2 t = __ldcg(reinterpret_cast<const float2 *>(p)); a[u].x = t.x; a[u].y = t.y; }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const float ws = __shfl_sync(0xffffffffu, w, (sb + u) & 31);   // weight 0 beyond the last split
+        o[0] = fmaf(a[u].x, ws, o[0]); o[1] = fmaf(a[u].y, ws, o[1]);
+        if (DPL == 4) { o[DPL - 2] = fmaf(a[u].z, ws, o[DPL - 2]); o[DPL - 1] = fmaf(a[u].w, ws, o[DPL - 1]); }
+      }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) o[i] = o[i] / den;
+  const size_t idx = (size_t)r * nq * HD + (size_t)j * HD + lane * DPL;
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) {
+    const __nv_bfloat16 a = __float2bfloat16_rn(o[i]);
+    out_hi[idx + i] = a;
+    out_lo[idx + i] = __float2bfloat16_rn(o[i] - __bfloat162float(a));
+  }
 }
 
 template <int HD>
@@ -72,7 +138,8 @@ __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                   const float *__restrict__ q, Rows rows, int nq, KvLayout kv, int max_splits,
                   const int *__restrict__ work, const int *__restrict__ n_work, float *__restrict__ part_acc,
-                  float *__restrict__ part_ml, int *status, unsigned long long *trace) {
+                  float *__restrict__ part_ml, int *__restrict__ done_count, __nv_bfloat16 *__restrict__ out_hi,
+                  __nv_bfloat16 *__restrict__ out_lo, int *status, unsigned long long *trace) {
   using L = AttLayout<HD>;
   // optional timeline (debug): per CTA and item (first 64): [key load issued, keys landed, group starts, released, scores done, weights written, values landed, output done]
 #define ATRACE(k, i) do { if (trace && (k) < 64) trace[((size_t)blockIdx.x * 64 + (k)) * 8 + (i)] = globaltimer_ns(); } while (0)
@@ -94,12 +161,16 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   __shared__ int abort_flag;
   __shared__ int stop_s[ATT_GROUPS];             // group-uniform copy of abort_flag, refreshed once per item
   __shared__ float red_s[ATT_GROUPS][4][8];      // cross-warp softmax reductions
+  // reports of the consumer groups to the combiners: (row << 8 | kv head, splits written), -1 = group is done
+  __shared__ int rep_key[ATT_GROUPS][ATT_QDEPTH], rep_cnt[ATT_GROUPS][ATT_QDEPTH];
+  __shared__ unsigned rep_tail[ATT_GROUPS], rep_head[ATT_GROUPS];
+  __shared__ int cmb_s[3];                       // what the combiners do next: row, kv head, split count (0 none, -1 leave)
   const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *ring_ptr = smem_raw + (ring - smem_u32(smem_raw));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     abort_flag = 0;
-    for (int g = 0; g < ATT_GROUPS; ++g) { stop_s[g] = 0; mbar_init(smem_u32(&mma_bar[g]), 1); }
+    for (int g = 0; g < ATT_GROUPS; ++g) { stop_s[g] = 0; rep_tail[g] = 0u; rep_head[g] = 0u; mbar_init(smem_u32(&mma_bar[g]), 1); }
     for (int s = 0; s < ATT_SLOTS; ++s) { mbar_init(smem_u32(&kfull_bar[s]), 1); mbar_init(smem_u32(&vfull_bar[s]), 1); }
     for (int b = 0; b < ATT_NBUF; ++b) { mbar_init(smem_u32(&kempty_bar[b]), 1); mbar_init(smem_u32(&vempty_bar[b]), 1); }
     fence_mbar_init();
@@ -108,10 +179,10 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   if (warp == 0) {
     tmem_alloc(smem_u32(&tmem_base_s), ATT_TMEM_COLS);
     tmem_relinquish();
-  } else if (warp >= 2) {
+  } else if (warp >= 2 && warp < 2 + 4 * ATT_GROUPS) {
     // operand tiles start out as zeros: rows of unused heads are never written and must stay finite
     uint4 *z = reinterpret_cast<uint4 *>(ring_ptr + (size_t)ATT_NBUF * L::ITEM_BYTES);
-    for (int i = tid - 64; i < ATT_GROUPS * L::GROUP_BYTES / 16; i += ATT_THREADS - 64) z[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = tid - 64; i < ATT_GROUPS * L::GROUP_BYTES / 16; i += ATT_GROUPS * 128) z[i] = make_uint4(0u, 0u, 0u, 0u);
   }
   tc_fence_before();
   __syncthreads();
@@ -164,9 +235,25 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         }
       }
     }
-  } else {
+  } else if (warp < 2 + 4 * ATT_GROUPS) {
     // ---------------- consumers ----------------
     const int gi = (warp - 2) >> 2, gtid = (tid - 64) & 127;
+    // Report to the combiners (one thread, after a group barrier that follows the group's stores).
+    auto report = [&](int key, int cnt) {
+      const unsigned t = rep_tail[gi];               // written by this thread only
+      if (t - *(volatile unsigned *)&rep_head[gi] >= (unsigned)ATT_QDEPTH) {
+        const uint64_t t0 = globaltimer_ns();
+        while (t - *(volatile unsigned *)&rep_head[gi] >= (unsigned)ATT_QDEPTH) {
+          __nanosleep(64);
+          if (abort_flag || globaltimer_ns() - t0 > 2000000000ull) { abort_flag = 1; return; }
+        }
+      }
+      rep_key[gi][t % ATT_QDEPTH] = key;
+      rep_cnt[gi][t % ATT_QDEPTH] = cnt;
+      __threadfence_block();
+      *(volatile unsigned *)&rep_tail[gi] = t + 1u;
+    };
+    int run_cnt = 0;
     const int quad = warp & 3;                     // the TMEM lane quarter this warp may read
     const int tl = quad * 32 + lane;               // TMEM lane of this thread: token (scores) / dim (values)
     const float sscale = (HD == 128 ? 0.08838834764831845f : 0.125f) * 1.4426950408889634f;   // log2(e)/sqrt(hd)
@@ -223,9 +310,11 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         }
         q_built = q_loaded = wi >> 8;
       }
+      bool run_ends = true;                          // is this the group's last item of its (row, kv head)?
       if (k + ATT_GROUPS < n_items) {   // fetch the next item's query values now if they differ
         const int nwi = work[item_lo + k + ATT_GROUPS];
         if ((nwi >> 8) != q_built) { load_q(nwi >> 16, (nwi >> 8) & 255); q_loaded = nwi >> 8; }
+        run_ends = (nwi >> 8) != (wi >> 8);
       }
       fence_proxy_async();                           // the MMA reads this tile through the async proxy
       if (gtid == 0) stop_s[gi] = abort_flag;
@@ -347,6 +436,67 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       tc_fence_before();
       asm volatile("bar.sync %0, 128;" ::"r"(1 + gi) : "memory");   // the group's TMEM and operand tiles are free
       if (gtid == 0) ATRACE(k, 3);
+      ++run_cnt;
+      if (run_ends) {
+        if (gtid == 0) report(wi >> 8, run_cnt);
+        run_cnt = 0;
+      }
+    }
+    if (gtid == 0) report(-1, 0);                    // always: the combiners wait for every group
+  } else {
+    // ---------------- combiners ----------------
+    const int ctid = tid - 64 - ATT_GROUPS * 128, cw = ctid >> 5;
+    unsigned head[ATT_GROUPS];
+    int groups_done = 0;
+#pragma unroll
+    for (int g = 0; g < ATT_GROUPS; ++g) head[g] = 0u;
+    for (;;) {
+      if (ctid == 0) {
+        int key = 0, cnt = 0, got = -1;
+        const uint64_t t0 = globaltimer_ns();
+        for (uint32_t spin = 0; got < 0; ++spin) {
+#pragma unroll
+          for (int g = 0; g < ATT_GROUPS; ++g)
+            if (got < 0 && *(volatile unsigned *)&rep_tail[g] != head[g]) got = g;
+          if (got >= 0) break;
+          __nanosleep(100);
+          if ((spin & 255u) == 255u && (abort_flag || globaltimer_ns() - t0 > 4000000000ull)) { abort_flag = 1; break; }
+        }
+        if (got < 0) {
+          cmb_s[2] = -1;                             // gave up: leave
+        } else {
+          __threadfence_block();
+#pragma unroll
+          for (int g = 0; g < ATT_GROUPS; ++g)
+            if (g == got) {
+              key = rep_key[g][head[g] % ATT_QDEPTH];
+              cnt = rep_cnt[g][head[g] % ATT_QDEPTH];
+              head[g] += 1u;
+              *(volatile unsigned *)&rep_head[g] = head[g];
+            }
+          if (key < 0) {
+            ++groups_done;
+            cmb_s[2] = (groups_done == ATT_GROUPS) ? -1 : 0;
+          } else {
+            const int r_ = key >> 8, g_ = key & 255;
+            const int ns = (rows.pos[r_] + 1 + ATT_SPLIT - 1) / ATT_SPLIT;
+            __threadfence();                         // the group's partial results are visible device-wide ...
+            int *c = done_count + r_ * kv.n_kv + g_;
+            const int seen = atomicAdd(c, cnt) + cnt;   // ... before its splits are counted
+            if (seen == ns) *c = 0;                  // complete: nobody else touches the counter until the next launch
+            cmb_s[0] = r_; cmb_s[1] = g_; cmb_s[2] = (seen == ns) ? ns : 0;
+          }
+        }
+      }
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + ATT_GROUPS) : "memory");
+      const int r_ = cmb_s[0], g_ = cmb_s[1], ns = cmb_s[2];
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + ATT_GROUPS) : "memory");
+      if (ns < 0) break;
+      if (ns > 0) {
+        __threadfence();                             // the other contributors' partial results are visible here
+        for (int h = cw; h < GROUP; h += 4)
+          attn_combine_pair<HD>(r_, g_ * GROUP + h, ns, nq, max_splits, part_acc, part_ml, out_hi, out_lo, lane);
+      }
     }
   }
   if (failed || abort_flag) {
@@ -357,76 +507,6 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   __syncthreads();
   tc_fence_after();
   if (warp == 0) tmem_dealloc(tmem_base, ATT_TMEM_COLS);
-}
-
-// Combines the splits of each (row, head): one warp per (row, head).  Lanes first hold one split each
-// (max by butterfly, which is exact; the denominator by a fixed butterfly over at most 32 lanes, then
-// ascending chunks of 32), then every lane owns hd/32 output dims and adds the splits' weighted
-// partial outputs in ascending split order.  Output: bf16 hi/lo pair for the O projection.
-template <int HD>
-__global__ void __launch_bounds__(256)
-attn_combine_kernel(Rows rows, int nq, int max_splits, const float *__restrict__ part_acc,
-                    const float *__restrict__ part_ml, __nv_bfloat16 *__restrict__ out_hi,
-                    __nv_bfloat16 *__restrict__ out_lo) {
-  constexpr int DPL = HD / 32;                   // dims per lane (4 or 2)
-  griddep_launch_dependents();
-  griddep_wait();
-  const int lane = threadIdx.x & 31;
-  const int pair = blockIdx.x * 8 + (threadIdx.x >> 5);      // (row, head) index
-  if (pair >= rows.R * nq) return;
-  const int r = pair / nq, j = pair - r * nq;
-  float o[DPL];
-#pragma unroll
-  for (int i = 0; i < DPL; ++i) o[i] = 0.f;
-  if (rows.active[r]) {
-    const int nsplit = (rows.pos[r] + 1 + ATT_SPLIT - 1) / ATT_SPLIT;
-    const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + ((size_t)r * nq + j) * max_splits;
-    const float *pa = part_acc + ((size_t)r * nq + j) * max_splits * HD + lane * DPL;
-    float M = -CUDART_INF_F;
-    for (int s0 = 0; s0 < nsplit; s0 += 32) {
-      float m = (s0 + lane < nsplit) ? ml[s0 + lane].x : -CUDART_INF_F;
-#pragma unroll
-      for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
-      M = fmaxf(M, m);
-    }
-    float den = 0.f;
-    for (int s0 = 0; s0 < nsplit; s0 += 32) {
-      float2 v = (s0 + lane < nsplit) ? ml[s0 + lane] : make_float2(-CUDART_INF_F, 0.f);
-      const float w = exp2f(v.x - M);              // this lane's split weight (0 beyond the last split)
-      float d = v.y * w;
-#pragma unroll
-      for (int k = 16; k > 0; k >>= 1) d += __shfl_xor_sync(0xffffffffu, d, k);
-      den += d;
-      const int cnt = min(32, nsplit - s0);
-      for (int sb = 0; sb < cnt; sb += 8) {          // eight splits' partial outputs are fetched together
-        float4 a[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          a[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (sb + u < cnt) {
-            const float *p = pa + (size_t)(s0 + sb + u) * HD;
-            if (DPL == 4) a[u] = *reinterpret_cast<const float4 *>(p);
-            else { const float2 t = *reinterpret_cast<const float2 *>(p); a[u].x = t.x; a[u].y = t.y; }
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const float ws = __shfl_sync(0xffffffffu, w, (sb + u) & 31);   // weight 0 beyond the last split
-          o[0] = fmaf(a[u].x, ws, o[0]); o[1] = fmaf(a[u].y, ws, o[1]);
-          if (DPL == 4) { o[DPL - 2] = fmaf(a[u].z, ws, o[DPL - 2]); o[DPL - 1] = fmaf(a[u].w, ws, o[DPL - 1]); }
-        }
-      }
-    }
-#pragma unroll
-    for (int i = 0; i < DPL; ++i) o[i] = o[i] / den;
-  }
-  const size_t idx = (size_t)r * nq * HD + (size_t)j * HD + lane * DPL;
-#pragma unroll
-  for (int i = 0; i < DPL; ++i) {
-    const __nv_bfloat16 a = __float2bfloat16_rn(o[i]);
-    out_hi[idx + i] = a;
-    out_lo[idx + i] = __float2bfloat16_rn(o[i] - __bfloat162float(a));
-  }
 }
 
 // Lists the items of the step: active rows ascending, kv heads ascending, splits ascending.
@@ -468,11 +548,12 @@ cudaError_t prepare_one() {
 template <int HD>
 cudaError_t launch_attn_split(int group, int grid, cudaStream_t st, const CUtensorMap &tmK, const CUtensorMap &tmV,
                          const float *q, const Rows &rows, int nq, const KvLayout &kv, int max_splits, const int *work,
-                         const int *n_work, float *part_acc, float *part_ml, int *d_status, unsigned long long *trace) {
+                         const int *n_work, float *part_acc, float *part_ml, int *done_count, __nv_bfloat16 *out_hi,
+                         __nv_bfloat16 *out_lo, int *d_status, unsigned long long *trace) {
 #define CORUN_ATT_CASE(G)                                                                                          \
   case G:                                                                                                          \
     return launch_k(attn_split_kernel<HD, G>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
-                    rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, d_status, trace);
+                    rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, out_hi, out_lo, d_status, trace);
   switch (group) {
     CORUN_ATT_CASE(1)
     CORUN_ATT_CASE(2)
@@ -504,27 +585,20 @@ cudaError_t launch_attn_worklist(const Rows &rows, int n_kv, int *work, int *n_w
 
 cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, const float *q, const Rows &rows, int nq,
                              const KvLayout &kv, int layer, int max_splits, const int *work, const int *n_work,
-                             int grid_ctas, float *part_acc, float *part_ml, __nv_bfloat16 *out_hi,
+                             int grid_ctas, float *part_acc, float *part_ml, int *done_count, __nv_bfloat16 *out_hi,
                              __nv_bfloat16 *out_lo, int *d_status, cudaStream_t st, unsigned long long *trace) {
   (void)layer;   // the tensor maps are the layer's
   const int group = nq / kv.n_kv;
   if (group * kv.n_kv != nq || max_splits > 256) return cudaErrorInvalidValue;
   const long long most = (long long)rows.R * max_splits * kv.n_kv;
   const int grid = (int)(most < grid_ctas ? most : grid_ctas);
-  cudaError_t e;
   if (kv.hd == 128)
-    e = launch_attn_split<128>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, d_status, trace);
-  else if (kv.hd == 64)
-    e = launch_attn_split<64>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, d_status, trace);
-  else
-    return cudaErrorInvalidValue;
-  if (e != cudaSuccess) return e;
-  const dim3 cgrid((rows.R * nq + 7) / 8);
-  if (kv.hd == 128)
-    return launch_k(attn_combine_kernel<128>, cgrid, dim3(256), 0, st, true, rows, nq, max_splits, part_acc, part_ml, out_hi,
-                    out_lo);
-  return launch_k(attn_combine_kernel<64>, cgrid, dim3(256), 0, st, true, rows, nq, max_splits, part_acc, part_ml, out_hi,
-                  out_lo);
+    return launch_attn_split<128>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml,
+                                  done_count, out_hi, out_lo, d_status, trace);
+  if (kv.hd == 64)
+    return launch_attn_split<64>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml,
+                                 done_count, out_hi, out_lo, d_status, trace);
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace corun

@@ -42,7 +42,7 @@ struct Program {
   float *qkv_out = nullptr, *o_out = nullptr, *gu_out = nullptr, *down_out = nullptr, *logits = nullptr, *ws = nullptr;
   bf16 *xn_hi = nullptr, *xn_lo = nullptr, *ao_hi = nullptr, *ao_lo = nullptr, *ff_hi = nullptr, *ff_lo = nullptr;
   int *row_token = nullptr, *row_pos = nullptr, *row_active = nullptr, *row_slot = nullptr, *do_sample = nullptr;
-  int *sampled = nullptr, *att_work = nullptr, *att_n_work = nullptr;
+  int *sampled = nullptr, *att_work = nullptr, *att_n_work = nullptr, *att_done = nullptr;
   GemmPlan p_qkv, p_o, p_gu, p_down, p_lm;
   bool has_layers = false, has_lm = false;
   std::vector<void *> allocs;
@@ -140,6 +140,7 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm) {
     RC(dmalloc(A, &P.part_ml, (size_t)R * s.n_q_heads * e->max_splits * 2));
     RC(dmalloc(A, &P.att_work, (size_t)R * e->max_splits * e->sh.n_kv_heads));
     RC(dmalloc(A, &P.att_n_work, 1));
+    RC(dmalloc(A, &P.att_done, (size_t)R * e->sh.n_kv_heads));
     RC(dmalloc(A, &P.qkv_out, (size_t)R * (QD + 2 * KD)));
     RC(dmalloc(A, &P.o_out, (size_t)R * H));
     RC(dmalloc(A, &P.gu_out, (size_t)R * 2 * F));
@@ -203,14 +204,14 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
     STAGE(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, tr(4 * l + 0), true));
     STAGE(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st));
     STAGE(launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work, P.att_n_work,
-                           e->num_sms, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo, e->d_status, e->st));
+                           e->num_sms, P.part_acc, P.part_ml, P.att_done, P.ao_hi, P.ao_lo, e->d_status, e->st));
     STAGE(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st, tr(4 * l + 1), true));
     GemmOut o = P.p_o.out();
     STAGE(launch_resid_norm(P.h, s.hidden, nullptr, rows, &o, e->mlp_norm[l], s.rms_eps, P.xn_hi, P.xn_lo, e->st));
     STAGE(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st, tr(4 * l + 2), true));
     STAGE(launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st));
     STAGE(gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st, tr(4 * l + 3), true));
-    n += 10;
+    n += 9;
   }
 #undef STAGE
   if (launches) *launches += n;
@@ -734,7 +735,7 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
                 if (ce == cudaSuccess) ce = gemm_fixup_launch(P.p_lm, e->st);
                 break;
         case 5: ce = launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work,
-                                      P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo,
+                                      P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_done, P.ao_hi, P.ao_lo,
                                       e->d_status, e->st); break;
         case 6: ce = launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->attn_norm[l], s.rms_eps, P.xn_hi,
                                        P.xn_lo, e->st); break;
@@ -791,8 +792,8 @@ int corun_debug_attn_trace(corun_engine *e, int32_t layer, uint64_t *stamps, int
   cudaError_t ce = cudaMemsetAsync(d, 0, n * sizeof(unsigned long long), e->st);
   for (int i = 0; i < 2 && ce == cudaSuccess; ++i)
     ce = launch_attention(e->tm_k[layer], e->tm_v[layer], P.q, rows, s.n_q_heads, kv_layout(e), layer, e->max_splits,
-                          P.att_work, P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.ao_hi, P.ao_lo, e->d_status,
-                          e->st, d);
+                          P.att_work, P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_done, P.ao_hi, P.ao_lo, e->d_status,
+                          e->st, i == 1 ? d : nullptr);   // only the second launch is recorded
   if (ce == cudaSuccess) ce = cudaMemcpyAsync(stamps, d, n * sizeof(unsigned long long), cudaMemcpyDeviceToHost, e->st);
   if (ce == cudaSuccess) ce = cudaStreamSynchronize(e->st);
   cudaFree(d);

@@ -152,7 +152,7 @@ def test_eager_launches_equal_graph_replay(tiny, engine):
     rows_e, toks_e = _run_request(engine, 3, prompt, 5, {}, 6)
     engine.set_eager(False)
     assert rows_g == rows_e and toks_g == toks_e
-    assert engine.decode_launches() == 7 + 10 * tiny.sh.n_layers
+    assert engine.decode_launches() == 7 + 9 * tiny.sh.n_layers
 
 
 def test_padding_rows_change_nothing_and_report_minus_one(tiny, engine):
