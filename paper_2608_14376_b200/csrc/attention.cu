@@ -1,8 +1,10 @@
 // Request-local split-KV paged attention for one query token per row, on tcgen05.
 //
 // An item is (row, kv head, split of 128 cached tokens = 8 pages); the step's items are listed in that
-// order and every CTA takes one contiguous stretch of the list, so consecutive items of a CTA mostly
-// share their query rows.  One persistent CTA per SM:
+// order and every CTA takes one contiguous stretch of the list (its two consumer groups one half each),
+// so consecutive items of a group mostly share their query rows.  That covers the first 15/16 of the list; the rest is dealt out two items at a
+// time through a counter, so that CTAs that got through their stretch sooner take more of it (which CTA
+// computes an item has no influence on any value).  One persistent CTA per SM:
 //   warp 0        streams the items' keys with TMA into a ring of 3 key buffers ([16 tokens x 64 dims]
 //                 boxes, 128-byte swizzle), warp 1 their values into a ring of 3 value buffers (cached
 //                 transposed: [hd dims x 16 tokens] boxes, 32-byte swizzle), straight from the page pool
@@ -72,38 +74,74 @@ __device__ __forceinline__ void attn_combine_pair(int r, int j, int nsplit, int 
   for (int i = 0; i < DPL; ++i) o[i] = 0.f;
   const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + ((size_t)r * nq + j) * max_splits;
   const float *pa = part_acc + ((size_t)r * nq + j) * max_splits * HD + lane * DPL;
-  float M = -CUDART_INF_F;
-  for (int s0 = 0; s0 < nsplit; s0 += 32) {
-    float m = (s0 + lane < nsplit) ? __ldcg(ml + s0 + lane).x : -CUDART_INF_F;
-#pragma unroll
-    for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
-    M = fmaxf(M, m);
-  }
+  auto load_acc = [&](int s) -> float4 {
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (s < nsplit) {
+      const float *p = pa + (size_t)s * HD;
+      if (DPL == 4) a = __ldcg(reinterpret_cast<const float4 *>(p));
+      else { const float2 t = __ldcg(reinterpret_cast<const float2 *>(p)); a.x = t.x; a.y = t.y; }
+    }
+    return a;
+  };
+  auto add_acc = [&](const float4 &a, float ws) {
+    o[0] = fmaf(a.x, ws, o[0]); o[1] = fmaf(a.y, ws, o[1]);
+    if (DPL == 4) { o[DPL - 2] = fmaf(a.z, ws, o[DPL - 2]); o[DPL - 1] = fmaf(a.w, ws, o[DPL - 1]); }
+  };
   float den = 0.f;
-  for (int s0 = 0; s0 < nsplit; s0 += 32) {
-    float2 v = (s0 + lane < nsplit) ? __ldcg(ml + s0 + lane) : make_float2(-CUDART_INF_F, 0.f);
-    const float w = exp2f(v.x - M);              // this lane's split weight (0 beyond the last split)
-    float d = v.y * w;
+  if (nsplit <= 64) {
+    // usual case: the (max, sum) pairs of all splits sit in two registers per lane, and the first
+    // sixteen partial outputs are requested before anything depends on them
+    const float2 none = make_float2(-CUDART_INF_F, 0.f);
+    const float2 v0 = lane < nsplit ? __ldcg(ml + lane) : none;
+    const float2 v1 = 32 + lane < nsplit ? __ldcg(ml + 32 + lane) : none;
+    float4 a[16];
 #pragma unroll
-    for (int k = 16; k > 0; k >>= 1) d += __shfl_xor_sync(0xffffffffu, d, k);
-    den += d;
-    const int cnt = min(32, nsplit - s0);
-    for (int sb = 0; sb < cnt; sb += 8) {          // eight splits' partial outputs are fetched together
-      float4 a[8];
+    for (int u = 0; u < 16; ++u) a[u] = load_acc(u);
+    float M = fmaxf(v0.x, v1.x);
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        a[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (sb + u < cnt) {
-          const float *p = pa + (size_t)(s0 + sb + u) * HD;
-          if (DPL == 4) a[u] = __ldcg(reinterpret_cast<const float4 *>(p));
-          else { const float2 t = __ldcg(reinterpret_cast<const float2 *>(p)); a[u].x = t.x; a[u].y = t.y; }
-        }
+    for (int k = 16; k > 0; k >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, k));
+    const float w0 = exp2f(v0.x - M), w1 = exp2f(v1.x - M);   // 0 beyond the last split
+    float d0 = v0.y * w0, d1 = v1.y * w1;
+#pragma unroll
+    for (int k = 16; k > 0; k >>= 1) {
+      d0 += __shfl_xor_sync(0xffffffffu, d0, k);
+      d1 += __shfl_xor_sync(0xffffffffu, d1, k);
+    }
+    den = nsplit > 32 ? d0 + d1 : d0;
+    for (int sb = 0; sb < nsplit; sb += 16) {
+      if (sb > 0) {
+#pragma unroll
+        for (int u = 0; u < 16; ++u) a[u] = load_acc(sb + u);
       }
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const float ws = __shfl_sync(0xffffffffu, w, (sb + u) & 31);   // weight 0 beyond the last split
-        o[0] = fmaf(a[u].x, ws, o[0]); o[1] = fmaf(a[u].y, ws, o[1]);
-        if (DPL == 4) { o[DPL - 2] = fmaf(a[u].z, ws, o[DPL - 2]); o[DPL - 1] = fmaf(a[u].w, ws, o[DPL - 1]); }
+      for (int u = 0; u < 16; ++u) {
+        const int sidx = sb + u;
+        const float ws = __shfl_sync(0xffffffffu, sidx < 32 ? w0 : w1, sidx & 31);
+        add_acc(a[u], ws);                         // beyond the last split: 0 * 0
+      }
+    }
+  } else {
+    float M = -CUDART_INF_F;
+    for (int s0 = 0; s0 < nsplit; s0 += 32) {
+      float m = (s0 + lane < nsplit) ? __ldcg(ml + s0 + lane).x : -CUDART_INF_F;
+#pragma unroll
+      for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
+      M = fmaxf(M, m);
+    }
+    for (int s0 = 0; s0 < nsplit; s0 += 32) {
+      float2 v = (s0 + lane < nsplit) ? __ldcg(ml + s0 + lane) : make_float2(-CUDART_INF_F, 0.f);
+      const float w = exp2f(v.x - M);              // this lane's split weight (0 beyond the last split)
+      float d = v.y * w;
+#pragma unroll
+      for (int k = 16; k > 0; k >>= 1) d += __shfl_xor_sync(0xffffffffu, d, k);
+      den += d;
+      const int cnt = min(32, nsplit - s0);
+      for (int sb = 0; sb < cnt; sb += 8) {          // eight splits' partial outputs are fetched together
+        float4 a[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) a[u] = sb + u < cnt ? load_acc(s0 + sb + u) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) add_acc(a[u], __shfl_sync(0xffffffffu, w, (sb + u) & 31));
       }
     }
   }
@@ -138,8 +176,9 @@ __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                   const float *__restrict__ q, Rows rows, int nq, KvLayout kv, int max_splits,
                   const int *__restrict__ work, const int *__restrict__ n_work, float *__restrict__ part_acc,
-                  float *__restrict__ part_ml, int *__restrict__ done_count, __nv_bfloat16 *__restrict__ out_hi,
-                  __nv_bfloat16 *__restrict__ out_lo, int *status, unsigned long long *trace) {
+                  float *__restrict__ part_ml, int *__restrict__ done_count, int *__restrict__ pool_count,
+                  __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo, int *status,
+                  unsigned long long *trace) {
   using L = AttLayout<HD>;
   // optional timeline (debug): per CTA and item (first 64): [key load issued, keys landed, group starts, released, scores done, weights written, values landed, output done]
 #define ATRACE(k, i) do { if (trace && (k) < 64) trace[((size_t)blockIdx.x * 64 + (k)) * 8 + (i)] = globaltimer_ns(); } while (0)
@@ -148,10 +187,10 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   griddep_wait();                                // the item list and q come from earlier kernels
   constexpr int group = GROUP;                   // query heads per kv head
   const int n_total = *n_work;
-  // this CTA's stretch of the item list
-  const int item_lo = (int)(((long long)blockIdx.x * n_total) / gridDim.x);
-  const int n_items = (int)(((long long)(blockIdx.x + 1) * n_total) / gridDim.x) - item_lo;
-  if (n_items <= 0) return;
+  if (n_total <= 0) return;
+  // this CTA's stretch of the item list, and where the shared pool begins
+  const int n_fixed = (int)(((long long)n_total * 15 / 16) / gridDim.x);
+  const int item_lo = (int)blockIdx.x * n_fixed, pool_lo = (int)gridDim.x * n_fixed;
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t kfull_bar[ATT_SLOTS], vfull_bar[ATT_SLOTS];
@@ -164,7 +203,10 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   // reports of the consumer groups to the combiners: (row << 8 | kv head, splits written), -1 = group is done
   __shared__ int rep_key[ATT_GROUPS][ATT_QDEPTH], rep_cnt[ATT_GROUPS][ATT_QDEPTH];
   __shared__ unsigned rep_tail[ATT_GROUPS], rep_head[ATT_GROUPS];
-  __shared__ int cmb_s[3];                       // what the combiners do next: row, kv head, split count (0 none, -1 leave)
+  __shared__ int cmb_s[2], cmb_list[8][3];       // what the combiners do next: how many pairs, leave?; (row, kv head, split count)
+  // pairs of pool items drawn by the key producer for the whole CTA: ring of 4, one barrier each
+  __shared__ __align__(8) uint64_t pool_bar[4];
+  __shared__ int pool_pair[4];
   const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *ring_ptr = smem_raw + (ring - smem_u32(smem_raw));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -173,6 +215,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     for (int g = 0; g < ATT_GROUPS; ++g) { stop_s[g] = 0; rep_tail[g] = 0u; rep_head[g] = 0u; mbar_init(smem_u32(&mma_bar[g]), 1); }
     for (int s = 0; s < ATT_SLOTS; ++s) { mbar_init(smem_u32(&kfull_bar[s]), 1); mbar_init(smem_u32(&vfull_bar[s]), 1); }
     for (int b = 0; b < ATT_NBUF; ++b) { mbar_init(smem_u32(&kempty_bar[b]), 1); mbar_init(smem_u32(&vempty_bar[b]), 1); }
+    for (int b = 0; b < 4; ++b) mbar_init(smem_u32(&pool_bar[b]), 1);
     fence_mbar_init();
     fence_proxy_async();
   }
@@ -193,6 +236,33 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   // M = 128 (M >> 4 at bit 24)
   const uint32_t idesc = (1u << 4) | ((uint32_t)(16 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
+  // Item of this CTA's k-th slot (every role walks the slots 0, 1, 2, ... with the same ring indices):
+  // first the fixed stretch, then pairs drawn from the pool.  The key producer draws (draw = true, whole
+  // warp) and publishes the pair; the other roles wait for it.  -1: no more work; -2: nothing in this slot.
+  int pair_j = -1, pair_c = 0;
+  auto item_of = [&](int k, bool draw) -> int {
+    if (k < n_fixed)   // even slots walk the first half of the stretch (group 0), odd slots the second half (group 1)
+      return item_lo + ((k & 1) ? ((n_fixed + 1) >> 1) + (k >> 1) : (k >> 1));
+    const int j = (k - n_fixed) >> 1;
+    if (j != pair_j) {
+      if (draw) {
+        int c = 0;
+        if (lane == 0) {
+          c = atomicAdd(pool_count, 1);
+          pool_pair[j & 3] = c;
+          mbar_arrive(smem_u32(&pool_bar[j & 3]));
+        }
+        pair_c = __shfl_sync(0xffffffffu, c, 0);
+      } else {
+        if (!mbar_wait(smem_u32(&pool_bar[j & 3]), (uint32_t)(j >> 2) & 1u, &abort_flag)) return -1;
+        pair_c = pool_pair[j & 3];
+      }
+      pair_j = j;
+    }
+    if (pool_lo + pair_c * 2 >= n_total) return -1;
+    const int it = pool_lo + pair_c * 2 + ((k - n_fixed) & 1);
+    return it < n_total ? it : -2;
+  };
   // shared memory: [key ring][value ring][operand tiles of the groups]
   const uint32_t vring = ring + (uint32_t)ATT_NBUF * L::K_BYTES;
   if (warp < 2) {
@@ -200,14 +270,17 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     const bool is_v = warp == 1;
     const uint64_t pol = l2_policy_evict_first();       // the cache is streamed once per step
     uint64_t *full = is_v ? vfull_bar : kfull_bar, *empty = is_v ? vempty_bar : kempty_bar;
-    for (int k = 0; k < n_items; ++k) {
+    for (int k = 0;; ++k) {
+      const int item = item_of(k, !is_v);
+      if (item == -1) break;
+      if (item == -2) continue;
       const int buf = k % ATT_NBUF, slot = k % ATT_SLOTS;
       if (k >= ATT_NBUF) {                               // the buffer's previous item must have been released
         bool ok = mbar_wait(smem_u32(&empty[buf]), (uint32_t)(k / ATT_NBUF - 1) & 1u, &abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { failed = true; break; }
       }
-      const int wi = work[item_lo + k];
+      const int wi = work[item];
       const int r = wi >> 16, g = (wi >> 8) & 255, split = wi & 255;
       const int ctx = rows.pos[r] + 1;
       const int t0 = split * ATT_SPLIT;
@@ -278,9 +351,11 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       }
     };
     int q_built = -1, q_loaded = -1;               // (row, kv head) keys of the operand tile / of qreg
-    for (int k = gi; k < n_items; k += ATT_GROUPS) {
+    for (int k = gi;; k += ATT_GROUPS) {
+      const int item = item_of(k, false);
+      if (item < 0) break;
       const int buf = k % ATT_NBUF, slot = k % ATT_SLOTS, j = slot / ATT_GROUPS;
-      const int wi = work[item_lo + k];
+      const int wi = work[item];
       const int r = wi >> 16, g = (wi >> 8) & 255, split = wi & 255;
       const int ctx = rows.pos[r] + 1;               // the new token attends to itself too
       const int t0 = split * ATT_SPLIT;
@@ -311,8 +386,8 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         q_built = q_loaded = wi >> 8;
       }
       bool run_ends = true;                          // is this the group's last item of its (row, kv head)?
-      if (k + ATT_GROUPS < n_items) {   // fetch the next item's query values now if they differ
-        const int nwi = work[item_lo + k + ATT_GROUPS];
+      if (k + ATT_GROUPS < n_fixed) {   // fetch the next item's query values now if they differ
+        const int nwi = work[item + 1];
         if ((nwi >> 8) != q_built) { load_q(nwi >> 16, (nwi >> 8) & 255); q_loaded = nwi >> 8; }
         run_ends = (nwi >> 8) != (wi >> 8);
       }
@@ -438,11 +513,12 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       if (gtid == 0) ATRACE(k, 3);
       ++run_cnt;
       if (run_ends) {
-        if (gtid == 0) report(wi >> 8, run_cnt);
+        // a group that wrote every split of the pair itself says so: nothing has to be counted then
+        if (gtid == 0) report(wi >> 8, run_cnt | ((run_cnt * ATT_SPLIT >= ctx) ? 0x10000 : 0));
         run_cnt = 0;
       }
     }
-    if (gtid == 0) report(-1, 0);                    // always: the combiners wait for every group
+    if (gtid == 0) { ATRACE(63, gi); report(-1, 0); }   // always: the combiners wait for every group
   } else {
     // ---------------- combiners ----------------
     const int ctid = tid - 64 - ATT_GROUPS * 128, cw = ctid >> 5;
@@ -452,52 +528,72 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     for (int g = 0; g < ATT_GROUPS; ++g) head[g] = 0u;
     for (;;) {
       if (ctid == 0) {
-        int key = 0, cnt = 0, got = -1;
+        // take every hand-in that is waiting (up to 8), make the groups' partial results visible
+        // device-wide with one fence, then count them all
+        int key[8], cnt[8], n = 0;
         const uint64_t t0 = globaltimer_ns();
-        for (uint32_t spin = 0; got < 0; ++spin) {
+        bool gave_up = false;
+        for (uint32_t spin = 0;; ++spin) {
 #pragma unroll
-          for (int g = 0; g < ATT_GROUPS; ++g)
-            if (got < 0 && *(volatile unsigned *)&rep_tail[g] != head[g]) got = g;
-          if (got >= 0) break;
-          __nanosleep(100);
-          if ((spin & 255u) == 255u && (abort_flag || globaltimer_ns() - t0 > 4000000000ull)) { abort_flag = 1; break; }
-        }
-        if (got < 0) {
-          cmb_s[2] = -1;                             // gave up: leave
-        } else {
-          __threadfence_block();
-#pragma unroll
-          for (int g = 0; g < ATT_GROUPS; ++g)
-            if (g == got) {
-              key = rep_key[g][head[g] % ATT_QDEPTH];
-              cnt = rep_cnt[g][head[g] % ATT_QDEPTH];
+          for (int g = 0; g < ATT_GROUPS; ++g) {
+            const unsigned tl_ = *(volatile unsigned *)&rep_tail[g];
+            if (tl_ != head[g]) __threadfence_block();
+            while (head[g] != tl_ && n < 8) {
+              const int k_ = rep_key[g][head[g] % ATT_QDEPTH], c_ = rep_cnt[g][head[g] % ATT_QDEPTH];
               head[g] += 1u;
-              *(volatile unsigned *)&rep_head[g] = head[g];
+              if (k_ < 0) ++groups_done;
+              else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                  if (i == n) { key[i] = k_; cnt[i] = c_; }
+                ++n;
+              }
             }
-          if (key < 0) {
-            ++groups_done;
-            cmb_s[2] = (groups_done == ATT_GROUPS) ? -1 : 0;
-          } else {
-            const int r_ = key >> 8, g_ = key & 255;
-            const int ns = (rows.pos[r_] + 1 + ATT_SPLIT - 1) / ATT_SPLIT;
-            __threadfence();                         // the group's partial results are visible device-wide ...
-            int *c = done_count + r_ * kv.n_kv + g_;
-            const int seen = atomicAdd(c, cnt) + cnt;   // ... before its splits are counted
-            if (seen == ns) *c = 0;                  // complete: nobody else touches the counter until the next launch
-            cmb_s[0] = r_; cmb_s[1] = g_; cmb_s[2] = (seen == ns) ? ns : 0;
+            *(volatile unsigned *)&rep_head[g] = head[g];
           }
+          if (n > 0 || groups_done == ATT_GROUPS) break;
+          __nanosleep(100);
+          if ((spin & 255u) == 255u && (abort_flag || globaltimer_ns() - t0 > 4000000000ull)) { abort_flag = 1; gave_up = true; break; }
+        }
+        int n_out = 0;
+        if (n > 0) {
+          int ns[8], seen[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            if (i < n) ns[i] = (rows.pos[key[i] >> 8] + 1 + ATT_SPLIT - 1) / ATT_SPLIT;
+          __threadfence();                           // the partial results are visible device-wide ...
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            if (i < n)   // ... before they are counted
+              seen[i] = (cnt[i] & 0x10000) ? ns[i]
+                                           : atomicAdd(done_count + (key[i] >> 8) * kv.n_kv + (key[i] & 255), cnt[i]) + cnt[i];
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            if (i < n && seen[i] == ns[i]) {
+              if (!(cnt[i] & 0x10000))
+                done_count[(key[i] >> 8) * kv.n_kv + (key[i] & 255)] = 0;   // complete: nobody else touches it until the next launch
+              cmb_list[n_out][0] = key[i] >> 8; cmb_list[n_out][1] = key[i] & 255; cmb_list[n_out][2] = ns[i];
+              ++n_out;
+            }
+        }
+        cmb_s[0] = n_out;
+        cmb_s[1] = (gave_up || (groups_done == ATT_GROUPS && n == 0)) ? 1 : 0;   // leave once nothing is left
+      }
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + ATT_GROUPS) : "memory");
+      const int n_out = cmb_s[0], leave = cmb_s[1];
+      if (n_out > 0 && ctid == 0 && trace) atomicAdd(&trace[((size_t)blockIdx.x * 64 + 63) * 8 + 3], (unsigned long long)n_out);
+      if (n_out > 0) {
+        __threadfence();                             // the other contributors' partial results are visible here
+        for (int i = 0; i < n_out; ++i) {
+          const int r_ = cmb_list[i][0], g_ = cmb_list[i][1], ns = cmb_list[i][2];
+          for (int h = cw; h < GROUP; h += 4)
+            attn_combine_pair<HD>(r_, g_ * GROUP + h, ns, nq, max_splits, part_acc, part_ml, out_hi, out_lo, lane);
         }
       }
       asm volatile("bar.sync %0, 128;" ::"r"(1 + ATT_GROUPS) : "memory");
-      const int r_ = cmb_s[0], g_ = cmb_s[1], ns = cmb_s[2];
-      asm volatile("bar.sync %0, 128;" ::"r"(1 + ATT_GROUPS) : "memory");
-      if (ns < 0) break;
-      if (ns > 0) {
-        __threadfence();                             // the other contributors' partial results are visible here
-        for (int h = cw; h < GROUP; h += 4)
-          attn_combine_pair<HD>(r_, g_ * GROUP + h, ns, nq, max_splits, part_acc, part_ml, out_hi, out_lo, lane);
-      }
+      if (leave) break;
     }
+    if (ctid == 0) ATRACE(63, 2);
   }
   if (failed || abort_flag) {
     if (lane == 0) atomicCAS(status, 0, DEV_TIMEOUT_EPILOGUE);
@@ -512,9 +608,11 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 // Lists the items of the step: active rows ascending, kv heads ascending, splits ascending.
 // One CTA; rows <= 256.  Entry = row << 16 | kv head << 8 | split.
 __global__ void __launch_bounds__(256) attn_worklist_kernel(Rows rows, int n_kv, int *__restrict__ work,
-                                                            int *__restrict__ n_work) {
+                                                            int *__restrict__ n_work, int *__restrict__ pool_counts,
+                                                            int n_pool_counts) {
   griddep_launch_dependents();
   griddep_wait();
+  for (int i = threadIdx.x; i < n_pool_counts; i += 256) pool_counts[i] = 0;   // one pool counter per attention launch of the step
   __shared__ int cnt[256];
   const int r = threadIdx.x;
   const int mine = (r < rows.R && rows.active[r]) ? (rows.pos[r] + 1 + ATT_SPLIT - 1) / ATT_SPLIT : 0;
@@ -548,12 +646,12 @@ cudaError_t prepare_one() {
 template <int HD>
 cudaError_t launch_attn_split(int group, int grid, cudaStream_t st, const CUtensorMap &tmK, const CUtensorMap &tmV,
                          const float *q, const Rows &rows, int nq, const KvLayout &kv, int max_splits, const int *work,
-                         const int *n_work, float *part_acc, float *part_ml, int *done_count, __nv_bfloat16 *out_hi,
-                         __nv_bfloat16 *out_lo, int *d_status, unsigned long long *trace) {
+                         const int *n_work, float *part_acc, float *part_ml, int *done_count, int *pool_count,
+                         __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int *d_status, unsigned long long *trace) {
 #define CORUN_ATT_CASE(G)                                                                                          \
   case G:                                                                                                          \
     return launch_k(attn_split_kernel<HD, G>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
-                    rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, out_hi, out_lo, d_status, trace);
+                    rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, d_status, trace);
   switch (group) {
     CORUN_ATT_CASE(1)
     CORUN_ATT_CASE(2)
@@ -578,15 +676,18 @@ cudaError_t attention_prepare() {
   return e;
 }
 
-cudaError_t launch_attn_worklist(const Rows &rows, int n_kv, int *work, int *n_work, cudaStream_t st) {
+cudaError_t launch_attn_worklist(const Rows &rows, int n_kv, int *work, int *n_work, int *pool_counts,
+                                 int n_pool_counts, cudaStream_t st) {
   if (rows.R > 256 || n_kv > 255) return cudaErrorInvalidValue;
-  return launch_k(attn_worklist_kernel, dim3(1), dim3(256), 0, st, true, rows, n_kv, work, n_work);
+  return launch_k(attn_worklist_kernel, dim3(1), dim3(256), 0, st, true, rows, n_kv, work, n_work, pool_counts,
+                  n_pool_counts);
 }
 
 cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, const float *q, const Rows &rows, int nq,
                              const KvLayout &kv, int layer, int max_splits, const int *work, const int *n_work,
-                             int grid_ctas, float *part_acc, float *part_ml, int *done_count, __nv_bfloat16 *out_hi,
-                             __nv_bfloat16 *out_lo, int *d_status, cudaStream_t st, unsigned long long *trace) {
+                             int grid_ctas, float *part_acc, float *part_ml, int *done_count, int *pool_count,
+                             __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int *d_status, cudaStream_t st,
+                             unsigned long long *trace) {
   (void)layer;   // the tensor maps are the layer's
   const int group = nq / kv.n_kv;
   if (group * kv.n_kv != nq || max_splits > 256) return cudaErrorInvalidValue;
@@ -594,10 +695,10 @@ cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, con
   const int grid = (int)(most < grid_ctas ? most : grid_ctas);
   if (kv.hd == 128)
     return launch_attn_split<128>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml,
-                                  done_count, out_hi, out_lo, d_status, trace);
+                                  done_count, pool_count, out_hi, out_lo, d_status, trace);
   if (kv.hd == 64)
     return launch_attn_split<64>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml,
-                                 done_count, out_hi, out_lo, d_status, trace);
+                                 done_count, pool_count, out_hi, out_lo, d_status, trace);
   return cudaErrorInvalidValue;
 }
 

@@ -42,7 +42,7 @@ struct Program {
   float *qkv_out = nullptr, *o_out = nullptr, *gu_out = nullptr, *down_out = nullptr, *logits = nullptr, *ws = nullptr;
   bf16 *xn_hi = nullptr, *xn_lo = nullptr, *ao_hi = nullptr, *ao_lo = nullptr, *ff_hi = nullptr, *ff_lo = nullptr;
   int *row_token = nullptr, *row_pos = nullptr, *row_active = nullptr, *row_slot = nullptr, *do_sample = nullptr;
-  int *sampled = nullptr, *att_work = nullptr, *att_n_work = nullptr, *att_done = nullptr;
+  int *sampled = nullptr, *att_work = nullptr, *att_n_work = nullptr, *att_done = nullptr, *att_pool = nullptr;
   GemmPlan p_qkv, p_o, p_gu, p_down, p_lm;
   bool has_layers = false, has_lm = false;
   std::vector<void *> allocs;
@@ -141,6 +141,7 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm) {
     RC(dmalloc(A, &P.att_work, (size_t)R * e->max_splits * e->sh.n_kv_heads));
     RC(dmalloc(A, &P.att_n_work, 1));
     RC(dmalloc(A, &P.att_done, (size_t)R * e->sh.n_kv_heads));
+    RC(dmalloc(A, &P.att_pool, (size_t)s.n_layers));
     RC(dmalloc(A, &P.qkv_out, (size_t)R * (QD + 2 * KD)));
     RC(dmalloc(A, &P.o_out, (size_t)R * H));
     RC(dmalloc(A, &P.gu_out, (size_t)R * 2 * F));
@@ -183,7 +184,7 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
   const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
   const KvLayout kv = kv_layout(e);
   int n = 0;
-  CK(launch_attn_worklist(rows, e->sh.n_kv_heads, P.att_work, P.att_n_work, e->st));   // the same items serve every layer
+  CK(launch_attn_worklist(rows, e->sh.n_kv_heads, P.att_work, P.att_n_work, P.att_pool, s.n_layers, e->st));   // the same items serve every layer
   n += 1;
   // (debug) slice of the step trace for the idx-th GEMM of the decode program: [num_sms][8] stamps
   auto tr = [&](int idx) -> unsigned long long * {
@@ -204,7 +205,7 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
     STAGE(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, tr(4 * l + 0), true));
     STAGE(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st));
     STAGE(launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work, P.att_n_work,
-                           e->num_sms, P.part_acc, P.part_ml, P.att_done, P.ao_hi, P.ao_lo, e->d_status, e->st));
+                           e->num_sms, P.part_acc, P.part_ml, P.att_done, P.att_pool + l, P.ao_hi, P.ao_lo, e->d_status, e->st));
     STAGE(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st, tr(4 * l + 1), true));
     GemmOut o = P.p_o.out();
     STAGE(launch_resid_norm(P.h, s.hidden, nullptr, rows, &o, e->mlp_norm[l], s.rms_eps, P.xn_hi, P.xn_lo, e->st));
@@ -734,9 +735,12 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
         case 4: ce = gemm_launch(P.p_lm, nullptr, e->d_status, e->st);
                 if (ce == cudaSuccess) ce = gemm_fixup_launch(P.p_lm, e->st);
                 break;
-        case 5: ce = launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work,
-                                      P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_done, P.ao_hi, P.ao_lo,
-                                      e->d_status, e->st); break;
+        case 5: ce = cudaMemsetAsync(P.att_pool + l, 0, sizeof(int), e->st);   // the launch does not reset its pool counter
+                if (ce == cudaSuccess)
+                  ce = launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work,
+                                        P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_done, P.att_pool + l,
+                                        P.ao_hi, P.ao_lo, e->d_status, e->st);
+                break;
         case 6: ce = launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->attn_norm[l], s.rms_eps, P.xn_hi,
                                        P.xn_lo, e->st); break;
         case 7: ce = launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st); break;
@@ -790,10 +794,13 @@ int corun_debug_attn_trace(corun_engine *e, int32_t layer, uint64_t *stamps, int
   unsigned long long *d = nullptr;
   if (cudaMalloc(&d, n * sizeof(unsigned long long)) != cudaSuccess) return CORUN_ENOMEM;
   cudaError_t ce = cudaMemsetAsync(d, 0, n * sizeof(unsigned long long), e->st);
-  for (int i = 0; i < 2 && ce == cudaSuccess; ++i)
-    ce = launch_attention(e->tm_k[layer], e->tm_v[layer], P.q, rows, s.n_q_heads, kv_layout(e), layer, e->max_splits,
-                          P.att_work, P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_done, P.ao_hi, P.ao_lo, e->d_status,
-                          e->st, i == 1 ? d : nullptr);   // only the second launch is recorded
+  for (int i = 0; i < 2 && ce == cudaSuccess; ++i) {
+    ce = cudaMemsetAsync(P.att_pool + layer, 0, sizeof(int), e->st);   // the launch does not reset its pool counter
+    if (ce == cudaSuccess)
+      ce = launch_attention(e->tm_k[layer], e->tm_v[layer], P.q, rows, s.n_q_heads, kv_layout(e), layer, e->max_splits,
+                            P.att_work, P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_done, P.att_pool + layer,
+                            P.ao_hi, P.ao_lo, e->d_status, e->st, i == 1 ? d : nullptr);   // only the second launch is recorded
+  }
   if (ce == cudaSuccess) ce = cudaMemcpyAsync(stamps, d, n * sizeof(unsigned long long), cudaMemcpyDeviceToHost, e->st);
   if (ce == cudaSuccess) ce = cudaStreamSynchronize(e->st);
   cudaFree(d);

@@ -62,17 +62,19 @@ cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *
                             int layer, float *q_out, cudaStream_t st);
 // Split-KV paged attention partials and their fixed-order combine -> bf16 hi/lo [R, nq*hd] (rows that are
 // not active keep what they held).  done_count: [R * n_kv] ints, zero before the first launch (the kernel
-// leaves them zero).
+// leaves them zero).  pool_count: one int, zero before the launch (not reset by it): the items beyond the
+// CTAs' fixed stretches are drawn through it.
 // tmK / tmV: tensor maps over this layer's pages: keys as rows of hd halfs with a [16, 64] box (128-byte
 // swizzle), values as rows of 16 halfs with an [hd, 16] box (32-byte swizzle); see attention.cu.
 // work / n_work: the step's (row, kv head, split) items from launch_attn_worklist (the same for every layer);
 // grid_ctas: persistent CTAs to launch (one per SM).
 cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, const float *q, const Rows &rows, int nq,
                              const KvLayout &kv, int layer, int max_splits, const int *work, const int *n_work,
-                             int grid_ctas, float *part_acc, float *part_ml, int *done_count, __nv_bfloat16 *out_hi,
-                             __nv_bfloat16 *out_lo, int *d_status, cudaStream_t st,
+                             int grid_ctas, float *part_acc, float *part_ml, int *done_count, int *pool_count,
+                             __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int *d_status, cudaStream_t st,
                              unsigned long long *trace = nullptr);   // optional [grid][64][8] stamps (debug)
-cudaError_t launch_attn_worklist(const Rows &rows, int n_kv, int *work, int *n_work, cudaStream_t st);
+cudaError_t launch_attn_worklist(const Rows &rows, int n_kv, int *work, int *n_work, int *pool_counts,
+                                 int n_pool_counts, cudaStream_t st);   // also zeroes the launches' pool counters
 cudaError_t attention_prepare();   // opts the kernels into their shared-memory size (idempotent)
 // y = silu(gate) * up from the gate-up GEMM result -> bf16 hi/lo [R, F].
 cudaError_t launch_swiglu(const GemmOut &gu, int R, int F, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, cudaStream_t st);
