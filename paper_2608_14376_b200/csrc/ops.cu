@@ -7,6 +7,7 @@
 #include "launch.cuh"
 #include "ptx.cuh"
 
+#include <cooperative_groups.h>
 #include <math_constants.h>
 
 namespace corun {
@@ -210,6 +211,14 @@ struct SmpShared {
   int sel_bin, sel_warp, tie_max_id;
   float cand_x[SMP_CAND];
   int cand_id[SMP_CAND];
+  // per-CTA results that the other CTAs of the row's cluster read
+  float loc_val; int loc_idx;                     // slice maximum and its lowest id
+  unsigned long long loc_total;                   // slice sum of weights
+  unsigned long long loc_wtot[32];                // per-warp nucleus weight of the slice, in id order
+  // decisions of the cluster's first CTA, read by the others
+  int bc_bin, bc_overflow, bc_tie_max_id, bc_sel_rank, bc_sel_warp;
+  unsigned int bc_kstar;
+  unsigned long long bc_wstar, bc_rdraw, bc_before;
 };
 
 // Integer weight of a token: floor(2^40 * exp2(x)), x = fl32(fl32(l - max) * inv_t_log2e).
@@ -278,10 +287,11 @@ __device__ __forceinline__ KeyRange smp_narrow(const SmpShared &sh, uint32_t kmi
   return KeyRange{kmin + (uint32_t)lo, kmin + (uint32_t)hi};
 }
 
-// Every logit of the row in ascending id by float4 where the row allows it (V % 4 == 0), else one by one.
+// Every logit of this CTA's slice of the row, by float4 where the row allows it (V % 4 == 0), else one
+// by one.  Units are float4 groups or single ids; the slice is [u_lo, u_hi).
 #define SMP_FOREACH(BODY)                                                                  \
   if (vec) {                                                                               \
-    _Pragma("unroll 2") for (int i4 = tid; i4 < n4; i4 += SMP_THREADS) {                   \
+    _Pragma("unroll 2") for (int i4 = u_lo + tid; i4 < u_hi; i4 += SMP_THREADS) {          \
       const float4 q4 = reinterpret_cast<const float4 *>(lg)[i4];                          \
       const float xs4[4] = {q4.x, q4.y, q4.z, q4.w};                                       \
       _Pragma("unroll") for (int j4 = 0; j4 < 4; ++j4) {                                   \
@@ -291,7 +301,7 @@ __device__ __forceinline__ KeyRange smp_narrow(const SmpShared &sh, uint32_t kmi
       }                                                                                    \
     }                                                                                      \
   } else {                                                                                 \
-    for (int i = tid; i < V; i += SMP_THREADS) {                                           \
+    for (int i = u_lo + tid; i < u_hi; i += SMP_THREADS) {                                 \
       const float x = lg[i];                                                               \
       BODY                                                                                 \
     }                                                                                      \
@@ -379,24 +389,34 @@ __device__ __noinline__ void smp_tail_full_row(SmpShared &sh, const SampleArgs &
   }
 }
 
-// Sampling S (top-p nucleus + inverse CDF) of one row per CTA, all in integers
-// once the weights are formed, so the result does not depend on the order in
-// which threads meet the tokens.  Four coalesced passes over the row: maximum;
-// coarse histogram of the weights over (max - logit); collection of the tokens
-// of the bin where the running weight reaches the cut (the nucleus edge is
-// then found among those few tokens in shared memory); per-warp totals of the
-// nucleus weights in id order, after which one warp walks its range to the drawn token.
-__global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
+// Sampling S (top-p nucleus + inverse CDF) of one row per cluster of SMP_CLUSTER CTAs, all in integers
+// once the weights are formed, so the result does not depend on the order in which threads meet the
+// tokens.  Every CTA takes a contiguous slice of the row; the first CTA of the cluster merges what the
+// slices found (through distributed shared memory) and takes the decisions.  Four passes over the row:
+// maximum; coarse histogram of the weights over (max - logit); collection of the tokens of the bin where
+// the running weight reaches the cut (the nucleus edge is then found among those few tokens in shared
+// memory); per-warp totals of the nucleus weights in id order, after which one warp walks its range to
+// the drawn token.
+constexpr int SMP_CLUSTER = 4;
+
+__global__ void __cluster_dims__(SMP_CLUSTER, 1, 1) __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
+  namespace cg = cooperative_groups;
   griddep_launch_dependents();
   griddep_wait();
-  const int r = blockIdx.x;
-  if (!a.do_sample[r]) return;
+  const int r = blockIdx.x / SMP_CLUSTER;
+  if (!a.do_sample[r]) return;                     // the same for the whole cluster
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = (int)cluster.block_rank();
   __shared__ SmpShared sh;
+  SmpShared *peer[SMP_CLUSTER];
+#pragma unroll
+  for (int k = 0; k < SMP_CLUSTER; ++k) peer[k] = cluster.map_shared_rank(&sh, k);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int V = a.V;
   const float *lg = a.logits + (size_t)r * V;
   const bool vec = (V & 3) == 0 && (((uintptr_t)lg) & 15u) == 0;
-  const int n4 = V >> 2;
+  const int units = vec ? (V >> 2) : V;            // float4 groups or single ids
+  const int u_lo = (int)(((long long)units * rank) / SMP_CLUSTER), u_hi = (int)(((long long)units * (rank + 1)) / SMP_CLUSTER);
 
   // ---- argmax, lowest id on ties
   float bv = -CUDART_INF_F;
@@ -410,15 +430,27 @@ __global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
   }
   if (lane == 0) { sh.red_val[warp] = bv; sh.red_idx[warp] = bi; }
   __syncthreads();
-  bv = sh.red_val[0]; bi = sh.red_idx[0];
-  for (int w = 1; w < SMP_THREADS / 32; ++w) {
-    const float ov = sh.red_val[w];
-    const int oi = sh.red_idx[w];
+  if (tid == 0) {
+    bv = sh.red_val[0]; bi = sh.red_idx[0];
+    for (int w = 1; w < SMP_THREADS / 32; ++w) {
+      const float ov = sh.red_val[w];
+      const int oi = sh.red_idx[w];
+      if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+    }
+    sh.loc_val = bv; sh.loc_idx = bi;
+  }
+  cluster.sync();
+  bv = peer[0]->loc_val; bi = peer[0]->loc_idx;
+#pragma unroll
+  for (int k = 1; k < SMP_CLUSTER; ++k) {
+    const float ov = peer[k]->loc_val;
+    const int oi = peer[k]->loc_idx;
     if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
   }
   const float temperature = a.temperature[r];
   if (!(temperature > 0.f)) {
-    if (tid == 0) a.out_token[r] = bi;
+    if (rank == 0 && tid == 0) a.out_token[r] = bi;
+    cluster.sync();                                // nobody leaves while its shared memory may still be read
     return;
   }
   const float mx = bv;
@@ -440,14 +472,29 @@ __global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
       mysum += w;
     }
   })
-  block_excl_scan_u64(mysum, sh.wtot, &sh.total);
-  const unsigned long long total = sh.total;
-  unsigned long long cut = __double2ull_rd((double)a.top_p[r] * (double)total);
-  if (cut > total) cut = total;
-  smp_select_bin(sh, cut, false);
-  const int bin_a = sh.sel_bin;
+  block_excl_scan_u64(mysum, sh.wtot, &sh.loc_total);
+  cluster.sync();                                  // every slice's histogram and total are complete
+  unsigned long long cut = 0ull;
+  if (rank == 0) {
+    unsigned long long total = 0ull;
+#pragma unroll
+    for (int k = 0; k < SMP_CLUSTER; ++k) total += peer[k]->loc_total;
+    for (int i = tid; i < SMP_BINS; i += SMP_THREADS) {
+      unsigned long long h = sh.hist[i];
+#pragma unroll
+      for (int k = 1; k < SMP_CLUSTER; ++k) h += peer[k]->hist[i];
+      sh.hist[i] = h;
+    }
+    __syncthreads();
+    cut = __double2ull_rd((double)a.top_p[r] * (double)total);
+    if (cut > total) cut = total;
+    smp_select_bin(sh, cut, false);
+    if (tid == 0) sh.bc_bin = sh.sel_bin;
+  }
+  cluster.sync();
+  const int bin_a = peer[0]->bc_bin;
 
-  // ---- the tokens of the selected bin, with their key range
+  // ---- the tokens of the selected bin in this slice, with their key range
   SMP_FOREACH({
     if (min(SMP_BINS - 1, (int)((mx - x) * scale_a)) == bin_a) {
       const unsigned int c = atomicAdd(&sh.n_cand, 1u);
@@ -457,66 +504,101 @@ __global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
       atomicMax(&sh.kmax, k);
     }
   })
-  __syncthreads();
-  const int n_cand = (int)sh.n_cand;
-  if (tid == 0) sh.sel_cnt = (unsigned)n_cand;   // stands if no refinement is needed: all those tokens share one key
-  __syncthreads();
-  if (n_cand > SMP_CAND) {   // uniform in the block
-    smp_tail_full_row(sh, a, r, lg, mx, inv_t_log2e, scale_a, bin_a, cut, u24);
-    return;
-  }
-  uint32_t kmin = sh.kmin, kmax = sh.kmax;
-  // ---- exact refinement in key space, over the candidates only, until one key remains
-  for (int pass = 0; pass < 4 && kmax > kmin; ++pass) {
-    const unsigned long long width = (unsigned long long)(kmax - kmin) + 1ull;
-    __syncthreads();
-    for (int i = tid; i < SMP_BINS; i += SMP_THREADS) { sh.hist[i] = 0ull; sh.cnt[i] = 0u; }
-    __syncthreads();
-    for (int c = tid; c < n_cand; c += SMP_THREADS) {
-      const float x = sh.cand_x[c];
-      const uint32_t k = ordered_key(x);
-      if (k >= kmin && k <= kmax) {
-        const int bin = smp_key_bin(k, kmin, width);
-        atomicAdd(&sh.hist[bin], smp_weight(x, mx, inv_t_log2e));
-        atomicAdd(&sh.cnt[bin], 1u);
+  cluster.sync();                                  // every slice's candidates are listed
+  if (rank == 0) {
+    // gather the other slices' candidates behind this slice's
+    unsigned int n_all = sh.n_cand, kmin = sh.kmin, kmax = sh.kmax;
+    unsigned int off[SMP_CLUSTER];
+    off[0] = 0u;
+#pragma unroll
+    for (int k = 1; k < SMP_CLUSTER; ++k) {
+      off[k] = n_all;
+      n_all += peer[k]->n_cand;
+      kmin = min(kmin, peer[k]->kmin);
+      kmax = max(kmax, peer[k]->kmax);
+    }
+    __syncthreads();                               // everyone has read n_cand / kmin / kmax of this CTA
+    const int n_cand = (int)n_all;
+    if (tid == 0) { sh.sel_cnt = n_all; sh.bc_overflow = n_cand > SMP_CAND ? 1 : 0; }   // sel_cnt stands if no refinement is needed
+    if (n_cand <= SMP_CAND) {
+#pragma unroll
+      for (int k = 1; k < SMP_CLUSTER; ++k) {
+        const int nk = (int)(k + 1 < SMP_CLUSTER ? off[k + 1] : n_all) - (int)off[k];
+        for (int c = tid; c < nk; c += SMP_THREADS) {
+          sh.cand_x[off[k] + c] = peer[k]->cand_x[c];
+          sh.cand_id[off[k] + c] = peer[k]->cand_id[c];
+        }
       }
     }
     __syncthreads();
-    smp_select_bin(sh, cut, true);
-    const KeyRange kr = smp_narrow(sh, kmin, width);
-    kmin = kr.kmin; kmax = kr.kmax;
-  }
-  __syncthreads();
-  // Now every token with key == kmin (== kmax) is tied at the nucleus edge.
-  const uint32_t kstar = kmin;
-  const unsigned long long carried = sh.carried;     // weight of tokens with key > kstar
-  const unsigned int n_tied = sh.sel_cnt;
-  const unsigned long long wstar = n_tied ? sh.sel_sum / n_tied : 0ull;
-  unsigned long long m_ties = 1ull;
-  if (wstar > 0ull && cut > carried) m_ties = (cut - carried + wstar - 1ull) / wstar;
-  if (m_ties < 1ull) m_ties = 1ull;
-  if (m_ties > n_tied) m_ties = n_tied;
-  const unsigned long long Z = carried + m_ties * wstar;
-  const unsigned long long rdraw = __umul64hi(Z, (unsigned long long)u24 << 40);   // floor(u24 * Z / 2^24)
-  // the tied tokens that belong to the nucleus are the m_ties lowest ids: find the largest of them
-  if (m_ties < n_tied) {
-    for (int c = tid; c < n_cand; c += SMP_THREADS) {
-      if (ordered_key(sh.cand_x[c]) != kstar) continue;
-      const int id = sh.cand_id[c];
-      unsigned long long rank = 0ull;
-      for (int j = 0; j < n_cand; ++j)
-        rank += (ordered_key(sh.cand_x[j]) == kstar && sh.cand_id[j] < id) ? 1ull : 0ull;
-      if (rank == m_ties - 1ull) sh.tie_max_id = id;
+    if (n_cand > SMP_CAND) {
+      // rare: this CTA finishes the row alone, reading all of it
+      smp_tail_full_row(sh, a, r, lg, mx, inv_t_log2e, scale_a, bin_a, cut, u24);
+    } else {
+      // ---- exact refinement in key space, over the candidates only, until one key remains
+      for (int pass = 0; pass < 4 && kmax > kmin; ++pass) {
+        const unsigned long long width = (unsigned long long)(kmax - kmin) + 1ull;
+        __syncthreads();
+        for (int i = tid; i < SMP_BINS; i += SMP_THREADS) { sh.hist[i] = 0ull; sh.cnt[i] = 0u; }
+        __syncthreads();
+        for (int c = tid; c < n_cand; c += SMP_THREADS) {
+          const float x = sh.cand_x[c];
+          const uint32_t k = ordered_key(x);
+          if (k >= kmin && k <= kmax) {
+            const int bin = smp_key_bin(k, kmin, width);
+            atomicAdd(&sh.hist[bin], smp_weight(x, mx, inv_t_log2e));
+            atomicAdd(&sh.cnt[bin], 1u);
+          }
+        }
+        __syncthreads();
+        smp_select_bin(sh, cut, true);
+        const KeyRange kr = smp_narrow(sh, kmin, width);
+        kmin = kr.kmin; kmax = kr.kmax;
+      }
+      __syncthreads();
+      // Now every token with key == kmin (== kmax) is tied at the nucleus edge.
+      const uint32_t kstar = kmin;
+      const unsigned long long carried = sh.carried;     // weight of tokens with key > kstar
+      const unsigned int n_tied = sh.sel_cnt;
+      const unsigned long long wstar = n_tied ? sh.sel_sum / n_tied : 0ull;
+      unsigned long long m_ties = 1ull;
+      if (wstar > 0ull && cut > carried) m_ties = (cut - carried + wstar - 1ull) / wstar;
+      if (m_ties < 1ull) m_ties = 1ull;
+      if (m_ties > n_tied) m_ties = n_tied;
+      const unsigned long long Z = carried + m_ties * wstar;
+      // the tied tokens that belong to the nucleus are the m_ties lowest ids: find the largest of them
+      if (m_ties < n_tied) {
+        for (int c = tid; c < n_cand; c += SMP_THREADS) {
+          if (ordered_key(sh.cand_x[c]) != kstar) continue;
+          const int id = sh.cand_id[c];
+          unsigned long long rank_ = 0ull;
+          for (int j = 0; j < n_cand; ++j)
+            rank_ += (ordered_key(sh.cand_x[j]) == kstar && sh.cand_id[j] < id) ? 1ull : 0ull;
+          if (rank_ == m_ties - 1ull) sh.tie_max_id = id;
+        }
+      }
+      __syncthreads();
+      if (tid == 0) {
+        sh.bc_kstar = kstar;
+        sh.bc_wstar = wstar;
+        sh.bc_tie_max_id = sh.tie_max_id;
+        sh.bc_rdraw = __umul64hi(Z, (unsigned long long)u24 << 40);   // floor(u24 * Z / 2^24)
+      }
     }
   }
-  __syncthreads();
-  const int tie_max_id = sh.tie_max_id;
+  cluster.sync();
+  if (peer[0]->bc_overflow) {
+    cluster.sync();
+    return;
+  }
+  const uint32_t kstar = peer[0]->bc_kstar;
+  const unsigned long long wstar = peer[0]->bc_wstar, rdraw = peer[0]->bc_rdraw;
+  const int tie_max_id = peer[0]->bc_tie_max_id;
 
-  // ---- inverse CDF over the nucleus in ascending id order.  Warp w owns a contiguous id range and its
-  // lanes take consecutive float4 groups (or single ids), so ids ascend with the lane in every step.
-  const int units = vec ? n4 : V;                       // float4 groups or single ids
-  const int per_warp = (units + 31) / 32;
-  const int u_begin = min(units, warp * per_warp), u_end = min(units, u_begin + per_warp);
+  // ---- inverse CDF over the nucleus in ascending id order.  Inside the slice warp w owns a contiguous
+  // range of units and its lanes take consecutive units, so ids ascend with the lane in every step.
+  const int per_warp = (u_hi - u_lo + 31) / 32;
+  const int w_begin = min(u_hi, u_lo + warp * per_warp), w_end = min(u_hi, w_begin + per_warp);
   const int n_it = (per_warp + 31) / 32;                // the same for every warp
   auto unit_weights = [&](int u, unsigned long long (&w)[4]) {
     float xs[4];
@@ -541,8 +623,8 @@ __global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
   };
   unsigned long long ws = 0ull;
   for (int it = 0; it < n_it; ++it) {
-    const int u = u_begin + it * 32 + lane;
-    if (u < u_end) {
+    const int u = w_begin + it * 32 + lane;
+    if (u < w_end) {
       unsigned long long w[4];
       unit_weights(u, w);
       ws += w[0] + w[1] + w[2] + w[3];
@@ -550,56 +632,81 @@ __global__ void __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) ws += __shfl_xor_sync(0xffffffffu, ws, o);
-  __syncthreads();
-  if (lane == 0) sh.wtot[warp] = ws;
-  if (tid == 0) sh.sel_warp = 31;
-  __syncthreads();
-  if (warp == 0) {
-    const unsigned long long w = sh.wtot[lane];
+  if (lane == 0) sh.loc_wtot[warp] = ws;
+  cluster.sync();                                  // every slice's warp totals are in place
+  if (rank == 0 && warp < SMP_CLUSTER) {
+    // warp k scans the 32 warp totals of slice k; lane 0 of warp 0 then walks the four slice totals
+    const unsigned long long w = peer[warp]->loc_wtot[lane];
     unsigned long long inc = w;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const unsigned long long n = __shfl_up_sync(0xffffffffu, inc, o);
       if (lane >= o) inc += n;
     }
-    sh.wtot[lane] = inc - w;   // weight before the warp's range
-    if (rdraw >= inc - w && rdraw < inc) sh.sel_warp = lane;
+    sh.hist[warp * 32 + lane] = inc - w;           // weight before the warp inside its slice (hist is free by now)
+    if (lane == 31) sh.wtot[warp] = inc;           // slice total
   }
   __syncthreads();
-  if (warp != sh.sel_warp) return;
-  unsigned long long run = sh.wtot[warp];
-  int tok = (vec ? 4 * u_end : u_end) - 1;
-  for (int it = 0; it < n_it; ++it) {
-    const int u = u_begin + it * 32 + lane;
-    unsigned long long w[4] = {0ull, 0ull, 0ull, 0ull};
-    if (u < u_end) unit_weights(u, w);
-    const unsigned long long s = w[0] + w[1] + w[2] + w[3];
-    unsigned long long inc = s;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const unsigned long long n = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += n;
-    }
-    const unsigned hit = __ballot_sync(0xffffffffu, run + inc > rdraw);
-    if (hit) {
-      const int L = __ffs(hit) - 1;
-      if (lane == L) {
-        unsigned long long c = run + inc - s;
-        const int id0 = vec ? 4 * u : u;
-        int t = id0;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          c += w[j];
-          if (c > rdraw) { t = id0 + j; break; }
+  if (rank == 0 && tid == 0) {
+    unsigned long long before = 0ull;
+    int sr = SMP_CLUSTER - 1, sw = 31;
+    bool found = false;
+    for (int k = 0; k < SMP_CLUSTER && !found; ++k) {
+      if (rdraw < before + sh.wtot[k]) {
+        const unsigned long long inside = rdraw - before;
+        sr = k;
+        sw = 31;
+        for (int w = 0; w < 32; ++w) {
+          const unsigned long long b0 = sh.hist[k * 32 + w];
+          const unsigned long long b1 = w < 31 ? sh.hist[k * 32 + w + 1] : sh.wtot[k];
+          if (inside >= b0 && inside < b1) { sw = w; break; }
         }
-        tok = t;
+        before += sh.hist[k * 32 + sw];
+        found = true;
+      } else {
+        before += sh.wtot[k];
       }
-      tok = __shfl_sync(0xffffffffu, tok, L);
-      break;
     }
-    run += __shfl_sync(0xffffffffu, inc, 31);
+    sh.bc_sel_rank = sr; sh.bc_sel_warp = sw; sh.bc_before = before;
   }
-  if (lane == 0) a.out_token[r] = tok;
+  cluster.sync();
+  const int sel_rank = peer[0]->bc_sel_rank, sel_warp = peer[0]->bc_sel_warp;
+  unsigned long long run = peer[0]->bc_before;
+  if (rank == sel_rank && warp == sel_warp) {
+    int tok = (vec ? 4 * w_end : w_end) - 1;
+    for (int it = 0; it < n_it; ++it) {
+      const int u = w_begin + it * 32 + lane;
+      unsigned long long w[4] = {0ull, 0ull, 0ull, 0ull};
+      if (u < w_end) unit_weights(u, w);
+      const unsigned long long s_ = w[0] + w[1] + w[2] + w[3];
+      unsigned long long inc = s_;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+      }
+      const unsigned hit = __ballot_sync(0xffffffffu, run + inc > rdraw);
+      if (hit) {
+        const int Lh = __ffs(hit) - 1;
+        if (lane == Lh) {
+          unsigned long long c = run + inc - s_;
+          const int id0 = vec ? 4 * u : u;
+          int t = id0;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            c += w[j];
+            if (c > rdraw) { t = id0 + j; break; }
+          }
+          tok = t;
+        }
+        tok = __shfl_sync(0xffffffffu, tok, Lh);
+        break;
+      }
+      run += __shfl_sync(0xffffffffu, inc, 31);
+    }
+    if (lane == 0) a.out_token[r] = tok;
+  }
+  cluster.sync();                                  // nobody leaves while its shared memory may still be read
 }
 #undef SMP_FOREACH
 
@@ -714,7 +821,7 @@ cudaError_t launch_split(const float *x, int R, int K, __nv_bfloat16 *hi, __nv_b
 }
 
 cudaError_t launch_sampler(const SampleArgs &a, int R, cudaStream_t st, bool pdl) {
-  return launch_k(sampler_kernel, dim3(R), dim3(SMP_THREADS), 0, st, pdl, a);
+  return launch_k(sampler_kernel, dim3(R * SMP_CLUSTER), dim3(SMP_THREADS), 0, st, pdl, a);
 }
 
 cudaError_t launch_prepare_rows(const uint8_t *active_mask, const int *in_use, const int *ctx_len, const int *pending,
