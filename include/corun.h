@@ -84,7 +84,8 @@ typedef struct {
  *   B               1..256 slots.
  *   max_context     largest prompt + generated length of any request.
  *   kv_block        tokens per KV page; must be 16.
- *   kv_pool_blocks  pages in the pool; 0 = B * ceil(max_context / kv_block).
+ *   kv_pool_blocks  pages in the pool; 0 = B * ceil(max_context / kv_block), or as many as fit in the
+ *                   device memory that is free now less 6 GiB, whichever is less.
  *   cuda_stream     a cudaStream_t (NULL = the legacy default stream).
  * Errors: EINVAL, ENOMEM, ECUDA.  On success *out owns device memory until
  * corun_destroy.

@@ -3,10 +3,14 @@
     python -m paper_2608_14376_b200.cases gemm      [--N 24576 --K 4096 --R 64 --reps 3]
     python -m paper_2608_14376_b200.cases kernels   [--layers 4 --B 64 --active-frac 0.625 --vocab 32768]
     python -m paper_2608_14376_b200.cases attention [--layers 2 --B 64 --active 40 --ctx-lo 512 --ctx-hi 4096 --reps 2]
+    python -m paper_2608_14376_b200.cases sweep     [--Bs 1,8,32,128,256 --fractions 0.125,0.5,1 --steps 10]
 
 ``gemm`` runs the stand-alone decode GEMM on seeded inputs; ``attention`` builds a Qwen3-8B-shaped
 engine with few layers, fills the cache of the active slots on the device and runs decode steps.
 Each prints the CUDA-event time per launch, for comparison with what a profiler reports.
+``sweep`` is the occupancy sweep on the full Qwen3-8B shape: one engine per padded batch B, contexts
+uniform in 256..8192 (seed 3) filled on the device, requests admitted in seeded order until the KV
+pool is full; prints decode tok/s, time per output token and the fraction of the step roofline.
 """
 from __future__ import annotations
 
@@ -114,6 +118,62 @@ def case_kernels(a):
     eng.close()
 
 
+def case_sweep(a):
+    import json
+    import os
+    import time
+
+    import torch
+
+    from . import corun, synth
+
+    sh = synth.QWEN3_8B
+    w = synth.make_weights_torch(sh, seed=0, device="cuda")
+    hbm = 6650.0
+    peaks = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    if os.path.exists(peaks):
+        hbm = float(json.load(open(peaks)).get("hbm_gbs", hbm))
+    max_ctx = 8192 + 64
+    print("| B | fraction | active | mean ctx | ms per step | tok/s | step roofline ms (%.0f GB/s) | fraction of roofline |" % hbm)
+    print("|---|---|---|---|---|---|---|---|")
+    for B in [int(x) for x in a.Bs.split(",")]:
+        eng = corun.Engine(sh, w, B, max_ctx)
+        seeds = np.arange(B, dtype=np.uint64) + 1000
+        for f in [float(x) for x in a.fractions.split(",")]:
+            want = max(1, int(round(B * f)))
+            ctx = synth.uniform_lengths(256, 8192, want, seed=3)
+            slots = synth.pick_slots(B, want, seed=7)
+            got = []
+            for i, (s, c) in enumerate(zip(slots, ctx)):
+                try:
+                    eng.adopt(int(s), 0, int(c) + a.steps + 8, pending=1 + i, temperature=0.7, top_p=0.95)
+                except corun.CorunError as e:
+                    if e.status != corun.ENOSPACE:
+                        raise
+                    break                                    # the pool is full: the rest is not admitted
+                eng.kv_fill(int(s), int(c), 1.28, seed=100 + i)
+                got.append((int(s), int(c)))
+            active = np.zeros(B, np.uint8)
+            active[[s for s, _ in got]] = 1
+            for _ in range(3):
+                eng.decode_enqueue(active, seeds)
+            eng.decode_wait()
+            t0 = time.perf_counter()
+            for _ in range(a.steps):
+                eng.decode_enqueue(active, seeds)
+            eng.decode_wait()
+            ms = (time.perf_counter() - t0) / a.steps * 1e3
+            nbytes = sh.weight_bytes_per_step() + sum((c + 3 + a.steps // 2) * sh.kv_bytes_per_token(2) for _, c in got)
+            t_roof = nbytes / (hbm * 1e9) * 1e3
+            print("| %d | %.3f | %d | %.0f | %.3f | %.0f | %.3f | %.2f |" % (B, f, len(got), np.mean([c for _, c in got]), ms,
+                                                                       len(got) / ms * 1e3, t_roof, t_roof / ms))
+            for s, _ in got:
+                eng.release(s)
+        eng.close()
+        del eng
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     sub = ap.add_subparsers(dest="case", required=True)
@@ -129,8 +189,11 @@ def main():
     k.add_argument("--active-frac", type=float, default=0.625); k.add_argument("--ctx-lo", type=int, default=512)
     k.add_argument("--ctx-hi", type=int, default=4096); k.add_argument("--vocab", type=int, default=32768)
     k.add_argument("--trace", action="store_true")
+    w = sub.add_parser("sweep")
+    w.add_argument("--Bs", default="1,8,32,128,256"); w.add_argument("--fractions", default="0.125,0.5,1")
+    w.add_argument("--steps", type=int, default=10)
     a = ap.parse_args()
-    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels}[a.case](a)
+    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "sweep": case_sweep}[a.case](a)
 
 
 if __name__ == "__main__":

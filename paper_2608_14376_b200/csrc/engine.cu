@@ -358,6 +358,17 @@ int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int3
   e->w0_gu = w->wgate_up[0];
   e->w0_down = w->wdown[0];
   e->pool_blocks = kv_pool_blocks ? kv_pool_blocks : (int64_t)B * e->max_blocks;
+  if (!kv_pool_blocks) {
+    // default size: a full reservation for every slot, or as many pages as fit beside 6 GiB that are
+    // left for the programs' buffers, whichever is less (admission then refuses what does not fit)
+    size_t free_b = 0, total_b = 0;
+    if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess) return fail(CORUN_ECUDA);
+    const size_t page_b = (size_t)s.n_layers * 2 * s.n_kv_heads * KV_BLOCK * s.head_dim * sizeof(__half);
+    const size_t keep = (size_t)6 << 30;
+    const int64_t fit = free_b > keep ? (int64_t)((free_b - keep) / page_b) : 0;
+    if (fit < e->pool_blocks) e->pool_blocks = fit;
+    if (e->pool_blocks < 1) return fail(CORUN_ENOMEM);
+  }
   e->chunk = 256;
   if (const char *c = getenv("CORUN_PREFILL_CHUNK")) {
     const int v = atoi(c);
