@@ -161,6 +161,9 @@ int corun_force_token(corun_engine *e, int32_t slot, int32_t token);
 int corun_context_len(corun_engine *e, int32_t slot);
 /* Free pages left in the pool, or a negative status. */
 int64_t corun_free_blocks(corun_engine *e);
+/* The engine's fixed dimensions: slots, largest context, tokens per page, pages in the pool
+ * (any of the out pointers may be NULL). */
+int corun_engine_info(corun_engine *e, int32_t *B, int32_t *max_context, int32_t *kv_block, int64_t *pool_blocks);
 /* Reads / writes n cached positions [pos0, pos0+n) of one layer as fp32 rows of
  * n_kv_heads*head_dim (host).  Writing beyond the current context length
  * extends it (up to reserve_len); values are rounded to the cache's fp16. */

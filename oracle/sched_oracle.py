@@ -1,0 +1,157 @@
+"""Plain restatement of the paper's isolated-prefill scheduling (Design, "Isolated Prefill":
+Algorithm 1 "Finding the request for isolated prefill" and Algorithm 2 "Scheduling isolated prefill").
+
+TEST INFRASTRUCTURE ONLY: imported by ``tests/``.  It shares no code with the library's scheduler
+and never imports it.
+
+The algorithms wrap an existing scheduler (``schedule_origin``).  Here that scheduler is the
+smallest one that makes the wrapper meaningful, in the paper's vocabulary:
+
+* two queues, ``running`` (requests that have started execution) and ``waiting`` (requests that
+  have not started prefill);
+* ``schedule_origin()`` first continues the prefill of every running request that still has
+  prompt tokens to compute (one chunk of at most ``chunk`` tokens each), then admits waiting
+  requests in order (first chunk each) while the running limit allows and the head's whole
+  sequence fits -- the same two tests as Algorithm 1, so it never admits what Algorithm 1
+  declined (by the paper, an iteration for which Algorithm 1 finds no request is an ordinary
+  decode iteration; this is the reading of that statement) and it stops at the first request that
+  does not fit.  Such requests form the iteration's prefill batch; if the batch is empty it
+  schedules one decode token for every running request.  Left to itself it would batch several
+  prefills together; Algorithm 2 hides all but one request from it.
+
+Nothing here computes tokens: a request produces ``max_new`` tokens, the first at the end of its
+prefill, and then leaves.  KV capacity is counted in pages of ``kv_block`` tokens; a request's
+pages for its whole configured sequence (prompt + max_new) are taken when it is admitted
+(Algorithm 1, "can_fit_full_sequence") and returned when it leaves, so nothing is ever preempted.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+
+@dataclass
+class Request:
+    rid: int
+    num_prompt_tokens: int
+    max_new: int
+    num_computed_tokens: int = 0
+    num_output_tokens: int = 0
+    pages: int = 0
+
+
+@dataclass
+class Iteration:
+    kind: str                       # "prefill" | "decode" | "idle"
+    requests: list = field(default_factory=list)   # request ids taking part, in `running` order
+    tokens: int = 0                 # prompt tokens computed (prefill) or 0
+
+
+class Scheduler:
+    def __init__(self, max_num_reqs: int, pool_pages: int, kv_block: int = 16, chunk: int = 256):
+        self.max_num_reqs = max_num_reqs
+        self.free_pages = pool_pages
+        self.kv_block = kv_block
+        self.chunk = chunk
+        self.running: list[Request] = []
+        self.waiting: list[Request] = []
+        self.finished: list[int] = []
+        self._next = 0
+
+    # ------------------------------------------------------------------ requests
+    def add_request(self, num_prompt_tokens: int, max_new: int) -> int:
+        r = Request(self._next, num_prompt_tokens, max_new)
+        self._next += 1
+        self.waiting.append(r)
+        return r.rid
+
+    def can_fit_full_sequence(self, r: Request) -> bool:
+        need = -(-(r.num_prompt_tokens + r.max_new) // self.kv_block)
+        return need <= self.free_pages
+
+    # ------------------------------------------------------------------ Algorithm 1
+    def find_prefill_request(self):
+        if self.running:
+            head = self.running[0]
+            if head.num_computed_tokens < head.num_prompt_tokens:
+                return head                                   # continue chunked prefill
+        if self.waiting and len(self.running) < self.max_num_reqs:
+            head = self.waiting[0]                            # peek_request
+            if self.can_fit_full_sequence(head):
+                return head
+        return None
+
+    # ------------------------------------------------------------------ the wrapped scheduler
+    def schedule_origin(self) -> Iteration:
+        batch, tokens = [], 0
+        for r in self.running:
+            if r.num_computed_tokens < r.num_prompt_tokens:
+                n = min(self.chunk, r.num_prompt_tokens - r.num_computed_tokens)
+                r.num_computed_tokens += n
+                batch.append(r); tokens += n
+        while self.waiting and len(self.running) < self.max_num_reqs and self.can_fit_full_sequence(self.waiting[0]):
+            r = self.waiting.pop(0)
+            r.pages = -(-(r.num_prompt_tokens + r.max_new) // self.kv_block)
+            self.free_pages -= r.pages
+            n = min(self.chunk, r.num_prompt_tokens)
+            r.num_computed_tokens = n
+            self.running.append(r)
+            batch.append(r); tokens += n
+        if batch:
+            it = Iteration("prefill", [r.rid for r in batch], tokens)
+            for r in batch:
+                if r.num_computed_tokens == r.num_prompt_tokens:
+                    r.num_output_tokens = 1                   # the prefill's last position samples the first token
+            self._retire()
+            return it
+        if not self.running:
+            return Iteration("idle")
+        it = Iteration("decode", [r.rid for r in self.running])
+        for r in self.running:
+            r.num_output_tokens += 1
+        self._retire()
+        return it
+
+    def _retire(self):
+        for r in list(self.running):
+            if r.num_computed_tokens == r.num_prompt_tokens and r.num_output_tokens >= r.max_new:
+                self.running.remove(r)
+                self.free_pages += r.pages
+                self.finished.append(r.rid)
+
+    # ------------------------------------------------------------------ Algorithm 2
+    def schedule(self) -> Iteration:
+        det = self.find_prefill_request()
+        if det is None:
+            return self.schedule_origin()
+        stashed_running = list(self.running)
+        stashed_waiting = list(self.waiting)
+        self.waiting.clear()
+        if det in self.running:
+            self.running = [det]
+            stashed_running.remove(det)
+        else:
+            self.running = []
+            self.waiting.append(det)
+            stashed_waiting.remove(det)
+        output = self.schedule_origin()
+        self.running = self.running + stashed_running
+        for request in stashed_waiting:
+            self.waiting.append(request)
+        return output
+
+    # ------------------------------------------------------------------ one decision of the collapsed form
+    def decision(self) -> Iteration:
+        """``schedule()`` until the request it started prefilling has all its prompt computed: the
+        chunks of one prefill as one record (Algorithm 1 resumes a partial prefill before anything
+        else, so they are consecutive anyway)."""
+        it = self.schedule()
+        if it.kind != "prefill":
+            return it
+        rid = it.requests[0]
+        while True:
+            head = self.running[0] if self.running else None
+            if head is None or head.rid != rid or head.num_computed_tokens >= head.num_prompt_tokens:
+                return it
+            nxt = self.schedule()
+            assert nxt.kind == "prefill" and nxt.requests == [rid]
+            it.tokens += nxt.tokens

@@ -4,6 +4,7 @@
     python -m paper_2608_14376_b200.cases kernels   [--layers 4 --B 64 --active-frac 0.625 --vocab 32768]
     python -m paper_2608_14376_b200.cases attention [--layers 2 --B 64 --active 40 --ctx-lo 512 --ctx-hi 4096 --reps 2]
     python -m paper_2608_14376_b200.cases sweep     [--Bs 1,8,32,128,256 --fractions 0.125,0.5,1 --steps 10]
+    python -m paper_2608_14376_b200.cases trace     [--requests 200 --rate 4 --B 128 --replay 4]
 
 ``gemm`` runs the stand-alone decode GEMM on seeded inputs; ``attention`` builds a Qwen3-8B-shaped
 engine with few layers, fills the cache of the active slots on the device and runs decode steps.
@@ -11,6 +12,10 @@ Each prints the CUDA-event time per launch, for comparison with what a profiler 
 ``sweep`` is the occupancy sweep on the full Qwen3-8B shape: one engine per padded batch B, contexts
 uniform in 256..8192 (seed 3) filled on the device, requests admitted in seeded order until the KV
 pool is full; prints decode tok/s, time per output token and the fraction of the step roofline.
+``trace`` serves a synthetic request trace through the host scheduler on the Qwen3-8B shape (Poisson
+arrivals, log-normal prompt and output lengths, sigma 1): the clock is virtual -- it advances by the
+measured duration of every scheduling decision and jumps to the next arrival when the engine is idle
+-- and a few requests are replayed alone afterwards to check that their tokens are identical.
 """
 from __future__ import annotations
 
@@ -174,6 +179,75 @@ def case_sweep(a):
         torch.cuda.empty_cache()
 
 
+def case_trace(a):
+    import time
+
+    import torch
+
+    from . import corun, synth
+
+    sh = synth.QWEN3_8B
+    w = synth.make_weights_torch(sh, seed=0, device="cuda")
+    rng = np.random.default_rng(5)
+    n = a.requests
+    arrival = np.cumsum(rng.exponential(1.0 / a.rate, n))
+    plen = np.minimum(8192, np.maximum(1, np.round(np.exp(np.log(1024) + rng.standard_normal(n))))).astype(int)
+    olen = np.minimum(2048, np.maximum(2, np.round(np.exp(np.log(256) + rng.standard_normal(n))))).astype(int)
+    prompts = synth.make_prompts(sh.vocab, plen, seed=6)
+    eng = corun.Engine(sh, w, a.B, 10240)
+    sch = corun.Scheduler(engine=eng)
+    now, nxt = 0.0, 0
+    t_first, t_done, busy_s, n_dec, n_pre, act_sum = {}, {}, 0.0, 0, 0, 0
+    ids = []
+    while len(t_done) < n:
+        while nxt < n and arrival[nxt] <= now:
+            ids.append(sch.submit(prompts[nxt], int(olen[nxt]), 0.7, 0.95, synth.request_seed(nxt)))
+            nxt += 1
+        t0 = time.perf_counter()
+        action, rid, n_act = sch.step()
+        dt = time.perf_counter() - t0
+        if action == corun.SCHED_IDLE:
+            now = max(now, float(arrival[nxt]))            # nothing runs: jump to the next arrival
+            continue
+        now += dt
+        busy_s += dt
+        if action == corun.SCHED_PREFILL:
+            n_pre += 1
+            t_first[rid] = now
+        else:
+            n_dec += 1
+            act_sum += n_act
+        for i in list(t_first):                             # requests that just produced their last token
+            if i not in t_done and sch.slot_of(i) < 0:
+                t_done[i] = now
+    ttft = np.array([t_first[i] - arrival[i] for i in range(n)])
+    tpot = np.array([(t_done[i] - t_first[i]) / (olen[i] - 1) for i in range(n)])
+    total_out = int(olen.sum())
+    print("trace: %d requests, %.1f req/s, prompt median %d (mean %.0f), output median %d (mean %.0f); B = %d"
+          % (n, a.rate, int(np.median(plen)), plen.mean(), int(np.median(olen)), olen.mean(), a.B))
+    print("virtual makespan %.1f s (engine busy %.1f s); %d prefills, %d decode iterations, mean %.1f running per iteration"
+          % (now, busy_s, n_pre, n_dec, act_sum / max(1, n_dec)))
+    print("output tokens/s over the makespan %.0f; over busy time %.0f" % (total_out / now, total_out / busy_s))
+    print("TTFT  p50 %.3f s  p99 %.3f s;  TPOT  p50 %.2f ms  p99 %.2f ms"
+          % (np.percentile(ttft, 50), np.percentile(ttft, 99), np.percentile(tpot, 50) * 1e3, np.percentile(tpot, 99) * 1e3))
+    served = [sch.poll(i)[0] for i in ids]
+    sch.close()
+    # replay a seeded sample alone on the same engine: the tokens must be identical
+    pick = np.random.default_rng(9).permutation(n)[:a.replay]
+    same = 0
+    for i in pick:
+        one = corun.Scheduler(engine=eng)
+        rid = one.submit(prompts[i], int(olen[i]), 0.7, 0.95, synth.request_seed(int(i)))
+        while not one.poll(rid)[1]:
+            one.step()
+        same += int(np.array_equal(one.poll(rid)[0], served[i]))
+        one.close()
+    print("replayed alone: %d of %d sampled requests produce identical token sequences" % (same, len(pick)))
+    eng.close()
+    if same != len(pick):
+        raise SystemExit(1)
+
+
 def main():
     ap = argparse.ArgumentParser()
     sub = ap.add_subparsers(dest="case", required=True)
@@ -192,8 +266,12 @@ def main():
     w = sub.add_parser("sweep")
     w.add_argument("--Bs", default="1,8,32,128,256"); w.add_argument("--fractions", default="0.125,0.5,1")
     w.add_argument("--steps", type=int, default=10)
+    tr = sub.add_parser("trace")
+    tr.add_argument("--requests", type=int, default=200); tr.add_argument("--rate", type=float, default=4.0)
+    tr.add_argument("--B", type=int, default=128); tr.add_argument("--replay", type=int, default=4)
     a = ap.parse_args()
-    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "sweep": case_sweep}[a.case](a)
+    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "sweep": case_sweep,
+     "trace": case_trace}[a.case](a)
 
 
 if __name__ == "__main__":

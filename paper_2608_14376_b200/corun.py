@@ -21,7 +21,9 @@ EXPORTS = [
     "corun_release", "corun_destroy", "corun_get_logits", "corun_force_token", "corun_context_len",
     "corun_free_blocks", "corun_debug_kv_read", "corun_debug_kv_write", "corun_debug_adopt",
     "corun_debug_set_eager", "corun_debug_read", "corun_debug_gemm_trace", "corun_debug_attn_trace", "corun_debug_step_trace", "corun_debug_kv_fill", "corun_debug_time_kernel", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
-    "corun_debug_sample", "corun_gemm_static", "corun_strerror", "corun_last_cuda_error",
+    "corun_debug_sample", "corun_gemm_static", "corun_strerror", "corun_last_cuda_error", "corun_engine_info",
+    "corun_sched_create", "corun_sched_create_for_engine", "corun_sched_destroy", "corun_sched_submit",
+    "corun_sched_step", "corun_sched_poll", "corun_sched_slot_of", "corun_sched_counts",
 ]
 
 
@@ -49,6 +51,21 @@ class Weights(C.Structure):
 
 class Sampling(C.Structure):
     _fields_ = [("temperature", C.c_float), ("top_p", C.c_float)]
+
+
+PREFILL_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.c_int32, C.c_int32, C.POINTER(Sampling),
+                         C.c_uint64, C.POINTER(C.c_int32))
+DECODE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.POINTER(C.c_uint8), C.POINTER(C.c_uint64), C.POINTER(C.c_int32))
+RELEASE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32)
+FREE_BLOCKS_FN = C.CFUNCTYPE(C.c_int64, C.c_void_p)
+
+
+class SchedOps(C.Structure):
+    """``corun_sched_ops``: the four engine calls the scheduler makes."""
+    _fields_ = [("prefill", PREFILL_FN), ("decode_step", DECODE_FN), ("release", RELEASE_FN),
+                ("free_blocks", FREE_BLOCKS_FN)]
+
+SCHED_IDLE, SCHED_PREFILL, SCHED_DECODE = 0, 1, 2
 
 
 _lib = None
@@ -94,6 +111,16 @@ def lib():
         L.corun_strerror.argtypes = [C.c_int]
         L.corun_strerror.restype = C.c_char_p
         L.corun_last_cuda_error.argtypes = []
+        L.corun_engine_info.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32), C.POINTER(i64)]
+        L.corun_sched_create.argtypes = [C.POINTER(SchedOps), vp, i32, i32, i32, C.POINTER(vp)]
+        L.corun_sched_create_for_engine.argtypes = [vp, C.POINTER(vp)]
+        L.corun_sched_destroy.argtypes = [vp]
+        L.corun_sched_destroy.restype = None
+        L.corun_sched_submit.argtypes = [vp, vp, i32, i32, C.POINTER(Sampling), u64, C.POINTER(i64)]
+        L.corun_sched_step.argtypes = [vp, C.POINTER(i32), C.POINTER(i64), C.POINTER(i32)]
+        L.corun_sched_poll.argtypes = [vp, i64, vp, i32, C.POINTER(i32), C.POINTER(i32)]
+        L.corun_sched_slot_of.argtypes = [vp, i64, C.POINTER(i32)]
+        L.corun_sched_counts.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
         for n in EXPORTS:
             getattr(L, n)
         _lib = L
@@ -263,6 +290,58 @@ class Engine:
 
     def decode_launches(self) -> int:
         return int(lib().corun_decode_launches(self._h))
+
+
+class Scheduler:
+    """Host scheduler (isolated prefill in front of the padded decode iteration) around an
+    ``Engine``, or around a table of callbacks standing in for one (``ops``: a ``SchedOps`` whose
+    callbacks the caller keeps alive, with ``B``, ``kv_block`` and ``max_context``)."""
+
+    def __init__(self, engine: "Engine" = None, ops: SchedOps = None, B: int = 0, kv_block: int = 16,
+                 max_context: int = 0):
+        h = C.c_void_p()
+        if engine is not None:
+            _check(lib().corun_sched_create_for_engine(engine._h, C.byref(h)), "corun_sched_create_for_engine")
+        else:
+            _check(lib().corun_sched_create(C.byref(ops), None, B, kv_block, max_context, C.byref(h)), "corun_sched_create")
+        self._h, self._keep = h, (engine, ops)
+
+    def close(self):
+        if self._h:
+            lib().corun_sched_destroy(self._h)
+            self._h = None
+
+    def submit(self, prompt, max_new_tokens: int, temperature: float = 0.0, top_p: float = 1.0, seed: int = 0) -> int:
+        t = np.ascontiguousarray(prompt, dtype=np.int32)
+        s = Sampling(temperature, top_p)
+        rid = C.c_int64(-1)
+        _check(lib().corun_sched_submit(self._h, t.ctypes.data, t.shape[0], max_new_tokens, C.byref(s),
+                                        seed & (2**64 - 1), C.byref(rid)), "corun_sched_submit")
+        return int(rid.value)
+
+    def step(self):
+        """One scheduling decision -> (action, request id of a prefill or -1, requests that took part)."""
+        a, rid, n = C.c_int32(0), C.c_int64(-1), C.c_int32(0)
+        _check(lib().corun_sched_step(self._h, C.byref(a), C.byref(rid), C.byref(n)), "corun_sched_step")
+        return int(a.value), int(rid.value), int(n.value)
+
+    def poll(self, rid: int):
+        """-> (tokens produced so far, finished?)"""
+        n, fin = C.c_int32(0), C.c_int32(0)
+        _check(lib().corun_sched_poll(self._h, rid, None, 0, C.byref(n), C.byref(fin)), "corun_sched_poll")
+        out = np.empty(max(1, n.value), np.int32)
+        _check(lib().corun_sched_poll(self._h, rid, out.ctypes.data, n.value, C.byref(n), C.byref(fin)), "corun_sched_poll")
+        return out[:n.value].copy(), bool(fin.value)
+
+    def slot_of(self, rid: int) -> int:
+        s = C.c_int32(-1)
+        _check(lib().corun_sched_slot_of(self._h, rid, C.byref(s)), "corun_sched_slot_of")
+        return int(s.value)
+
+    def counts(self):
+        w, r = C.c_int32(0), C.c_int32(0)
+        _check(lib().corun_sched_counts(self._h, C.byref(w), C.byref(r)), "corun_sched_counts")
+        return int(w.value), int(r.value)
 
 
 def debug_gemm(W, X):

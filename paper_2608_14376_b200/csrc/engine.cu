@@ -647,6 +647,15 @@ int corun_context_len(corun_engine *e, int32_t slot) {
 
 int64_t corun_free_blocks(corun_engine *e) { return e ? (int64_t)e->free_blocks.size() : (int64_t)CORUN_EINVAL; }
 
+int corun_engine_info(corun_engine *e, int32_t *B, int32_t *max_context, int32_t *kv_block, int64_t *pool_blocks) {
+  if (!e) return CORUN_EINVAL;
+  if (B) *B = e->B;
+  if (max_context) *max_context = e->max_ctx;
+  if (kv_block) *kv_block = KV_BLOCK;
+  if (pool_blocks) *pool_blocks = e->pool_blocks;
+  return CORUN_OK;
+}
+
 static int kv_io(corun_engine *e, int slot, int layer, int pos0, int n, float *k, float *v, int write) {
   if (!e || !k || !v || n < 0 || pos0 < 0 || layer < 0 || layer >= e->sh.n_layers) return CORUN_EINVAL;
   if (!slot_ok(e, slot) || !e->in_use[slot]) return CORUN_ESLOT;

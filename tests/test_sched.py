@@ -1,0 +1,241 @@
+"""Host scheduling (isolated prefill in front of the padded decode iteration).
+
+The oracle (``oracle/sched_oracle.py``, Algorithms 1 and 2 written out) is pinned to hand-derived
+iteration sequences and to the properties the paper states; the library's scheduler is then driven
+against a stand-in engine (callbacks that only count pages) and must take the same decisions."""
+import ctypes as C
+import os
+
+import numpy as np
+import pytest
+
+from oracle import sched_oracle
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _golden_cases():
+    cases, cur = [], None
+    for line in open(os.path.join(ROOT, "tests", "golden", "sched_isolated_prefill_traces.txt")):
+        t = line.split()
+        if not t or t[0].startswith("#"):
+            continue
+        if t[0] == "case":
+            cur = dict(name=t[1], reqs=[], its=[], **{k: int(v) for k, v in (x.split("=") for x in t[2:])})
+            cases.append(cur)
+        elif t[0] == "req":
+            cur["reqs"].append((int(t[1]), int(t[2])))
+        elif t[0] == "P":
+            cur["its"].append(("prefill", [int(t[1])], int(t[2])))
+        elif t[0] == "D":
+            cur["its"].append(("decode", [int(x) for x in t[1:]], 0))
+        elif t[0] == "I":
+            cur["its"].append(("idle", [], 0))
+    return cases
+
+
+@pytest.mark.parametrize("case", _golden_cases(), ids=lambda c: c["name"])
+def test_oracle_reproduces_hand_derived_iterations(case):
+    s = sched_oracle.Scheduler(case["max_num_reqs"], case["pool_pages"], case["kv_block"], case["chunk"])
+    for p, m in case["reqs"]:
+        s.add_request(p, m)
+    got = []
+    for _ in case["its"]:
+        it = s.schedule()
+        got.append((it.kind, it.requests, it.tokens))
+    assert got == case["its"]
+    assert s.free_pages == case["pool_pages"] and not s.running and not s.waiting
+
+
+def _random_trace(seed, n_req=40):
+    rng = np.random.default_rng(seed)
+    B = int(rng.integers(1, 6))
+    kv_block = 16
+    reqs = [(int(rng.integers(1, 200)), int(rng.integers(1, 12))) for _ in range(n_req)]
+    biggest = max(-(-(p + m) // kv_block) for p, m in reqs)
+    pool = biggest + int(rng.integers(0, 3 * biggest))          # every request fits alone; often not together
+    # submissions interleaved with decisions: ("submit", k) / ("step", k)
+    script, left = [], n_req
+    while left:
+        k = int(min(left, rng.integers(1, 6)))
+        script.append(("submit", k)); left -= k
+        script.append(("step", int(rng.integers(0, 8))))
+    return B, kv_block, pool, reqs, script
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_oracle_keeps_the_papers_properties(seed):
+    B, kv_block, pool, reqs, script = _random_trace(seed)
+    s = sched_oracle.Scheduler(B, pool, kv_block, chunk=64)
+    its, nxt = [], 0
+    for op, k in script + [("step", 10 ** 6)]:
+        if op == "submit":
+            for p, m in reqs[nxt:nxt + k]:
+                s.add_request(p, m)
+            nxt += k
+            continue
+        for _ in range(k):
+            free_before, running_before = s.free_pages, [r.rid for r in s.running]
+            waiting_before = [r.rid for r in s.waiting]
+            it = s.schedule()
+            its.append(it)
+            if it.kind == "prefill":
+                assert len(it.requests) == 1                      # a prefill batch is one request
+                rid = it.requests[0]
+                if rid in waiting_before:                         # admission: FIFO head, room for a slot and for the whole sequence
+                    assert rid == waiting_before[0]
+                    assert len(running_before) < B
+                    assert -(-(sum(reqs[rid])) // kv_block) <= free_before
+                else:                                             # continuing a chunked prefill: it was the head of running
+                    assert rid == running_before[0]
+            elif it.kind == "decode":
+                assert it.requests == running_before              # everything that runs takes part: nothing is preempted
+                head = waiting_before[0] if waiting_before else None
+                assert head is None or len(running_before) >= B or -(-(sum(reqs[head])) // kv_block) > free_before
+            else:
+                assert not running_before
+                if nxt == len(reqs) and not waiting_before:
+                    break
+            assert 0 <= s.free_pages <= pool and len(s.running) <= B
+    # every request was prefilled exactly once over consecutive iterations, in submission order
+    order, seen = [], {}
+    for i, it in enumerate(its):
+        if it.kind == "prefill":
+            rid = it.requests[0]
+            if rid in seen:
+                assert seen[rid][-1] == i - 1                     # chunks of one prefill are not interrupted
+            else:
+                order.append(rid)
+            seen.setdefault(rid, []).append(i)
+    assert order == list(range(len(reqs)))
+    assert {r: sum(its[i].tokens for i in ix) for r, ix in seen.items()} == {r: reqs[r][0] for r in range(len(reqs))}
+    assert sorted(s.finished) == list(range(len(reqs))) and s.free_pages == pool
+    # tokens per request: one from the prefill plus one per decode iteration it took part in
+    for rid, (p, m) in enumerate(reqs):
+        assert 1 + sum(1 for it in its if it.kind == "decode" and rid in it.requests) == m
+
+
+class _StandInEngine:
+    """Counts pages like the engine's admission does and records every call."""
+
+    def __init__(self, B, pool, kv_block):
+        from paper_2608_14376_b200 import corun
+
+        self.corun, self.B, self.free, self.kv_block = corun, B, pool, kv_block
+        self.pages = {}
+        self.calls = []
+        self.step_of = {}
+        self.fail_next = None
+        self.ops = corun.SchedOps(corun.PREFILL_FN(self._prefill), corun.DECODE_FN(self._decode),
+                                  corun.RELEASE_FN(self._release), corun.FREE_BLOCKS_FN(lambda ctx: self.free))
+
+    def _prefill(self, ctx, slot, tokens, n, reserve, sampling, seed, first):
+        if self.fail_next == "prefill":
+            self.fail_next = None
+            return self.corun.ECUDA
+        need = -(-reserve // self.kv_block)
+        if slot in self.pages:
+            return self.corun.ESLOT
+        if need > self.free:
+            return self.corun.ENOSPACE
+        self.free -= need
+        self.pages[slot] = need
+        self.step_of[slot] = 1
+        self.calls.append(("prefill", slot, n, reserve, int(seed)))
+        first[0] = int(seed) % 1000
+        return 0
+
+    def _decode(self, ctx, active, seeds, out):
+        if self.fail_next == "decode":
+            self.fail_next = None
+            return self.corun.ETIMEOUT
+        act = [i for i in range(self.B) if active[i]]
+        assert all(s in self.pages for s in act)
+        for i in range(self.B):
+            out[i] = (int(seeds[i]) % 1000 + self.step_of[i]) if active[i] else -1
+            if active[i]:
+                self.step_of[i] += 1
+        self.calls.append(("decode", tuple(act), tuple(int(seeds[i]) for i in act)))
+        return 0
+
+    def _release(self, ctx, slot):
+        self.free += self.pages.pop(slot)
+        self.calls.append(("release", slot))
+        return 0
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_library_scheduler_takes_the_oracles_decisions(seed):
+    from paper_2608_14376_b200 import build, corun
+
+    build.build()
+    B, kv_block, pool, reqs, script = _random_trace(100 + seed)
+    eng = _StandInEngine(B, pool, kv_block)
+    sch = corun.Scheduler(ops=eng.ops, B=B, kv_block=kv_block, max_context=256)
+    ref = sched_oracle.Scheduler(B, pool, kv_block, chunk=64)
+    nxt, rid_of = 0, []
+    try:
+        for op, k in script + [("step", 10 ** 6)]:
+            if op == "submit":
+                for p, m in reqs[nxt:nxt + k]:
+                    rid_of.append(sch.submit(np.arange(p) % 97, m, 0.7, 0.9, seed=5000 + len(rid_of)))
+                    ref.add_request(p, m)
+                nxt += k
+                continue
+            for _ in range(k):
+                want = ref.decision()
+                action, rid, n = sch.step()
+                assert action == {"idle": corun.SCHED_IDLE, "prefill": corun.SCHED_PREFILL, "decode": corun.SCHED_DECODE}[want.kind]
+                if want.kind == "prefill":
+                    assert rid == want.requests[0] and n == 1
+                    kind, slot, n_tok, reserve, sd = eng.calls[-1] if eng.calls[-1][0] == "prefill" else eng.calls[-2]
+                    assert (kind, n_tok, reserve, sd) == ("prefill", reqs[rid][0], sum(reqs[rid]), 5000 + rid)
+                elif want.kind == "decode":
+                    assert n == len(want.requests)
+                    dec = [c for c in eng.calls if c[0] == "decode"][-1]
+                    assert sorted(dec[2]) == sorted(5000 + r for r in want.requests)   # exactly the running requests, with their own seeds
+                assert sch.counts() == (len(ref.waiting), len(ref.running))
+                assert eng.free == ref.free_pages
+                if want.kind == "idle" and nxt == len(reqs):
+                    break
+        assert rid_of == list(range(len(reqs)))
+        for rid, (p, m) in enumerate(reqs):
+            toks, fin = sch.poll(rid)
+            assert fin and len(toks) == m and sch.slot_of(rid) == -1
+            assert list(toks) == [(5000 + rid) % 1000 + t for t in range(m)]   # the stand-in's tokens count the request's own steps
+        assert eng.free == pool and not eng.pages
+    finally:
+        sch.close()
+
+
+def test_library_scheduler_argument_and_engine_errors():
+    from paper_2608_14376_b200 import build, corun
+
+    build.build()
+    L = corun.lib()
+    h = C.c_void_p()
+    assert L.corun_sched_create(None, None, 4, 16, 128, C.byref(h)) == corun.EINVAL
+    assert L.corun_sched_create_for_engine(None, C.byref(h)) == corun.EINVAL
+    assert L.corun_sched_step(None, None, None, None) == corun.EINVAL
+    eng = _StandInEngine(2, 8, 16)
+    sch = corun.Scheduler(ops=eng.ops, B=2, kv_block=16, max_context=64)
+    try:
+        with pytest.raises(corun.CorunError):
+            sch.submit(np.zeros(60, np.int32), 10)          # longer than max_context
+        with pytest.raises(corun.CorunError):
+            sch.submit(np.zeros(0, np.int32), 1)
+        with pytest.raises(corun.CorunError):
+            sch.poll(0)
+        a = sch.submit(np.zeros(10, np.int32), 3, seed=1)
+        eng.fail_next = "prefill"
+        with pytest.raises(corun.CorunError) as ei:
+            sch.step()
+        assert ei.value.status == corun.ECUDA and sch.counts() == (1, 0)      # nothing moved
+        assert sch.step()[:2] == (corun.SCHED_PREFILL, a)
+        eng.fail_next = "decode"
+        with pytest.raises(corun.CorunError) as ei:
+            sch.step()
+        assert ei.value.status == corun.ETIMEOUT and sch.counts() == (0, 1) and len(sch.poll(a)[0]) == 1
+        assert sch.step()[0] == corun.SCHED_DECODE and len(sch.poll(a)[0]) == 2
+    finally:
+        sch.close()
