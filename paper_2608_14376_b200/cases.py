@@ -3,6 +3,7 @@
     python -m paper_2608_14376_b200.cases gemm      [--N 24576 --K 4096 --R 64 --reps 3]
     python -m paper_2608_14376_b200.cases kernels   [--layers 4 --B 64 --active-frac 0.625 --vocab 32768]
     python -m paper_2608_14376_b200.cases attention [--layers 2 --B 64 --active 40 --ctx-lo 512 --ctx-hi 4096 --reps 2]
+    python -m paper_2608_14376_b200.cases sampler   [--B 64 --active 40 --vocab 151936]
     python -m paper_2608_14376_b200.cases sweep     [--Bs 1,8,32,128,256 --fractions 0.125,0.5,1 --steps 10]
     python -m paper_2608_14376_b200.cases trace     [--requests 200 --rate 4 --B 128 --replay 4]
 
@@ -120,6 +121,26 @@ def case_kernels(a):
               "(p90 %.2f); of which waiting for the data median %.2f us; issue->group start median %.2f; span %.1f us"
               % (ok.sum(), np.median(load), np.percentile(load, 90), np.median(hold), np.percentile(hold, 90),
                  np.median(np.maximum(stall, 0)), np.median(wait), (t[:, :, 3][ok].max() - t0) / 1e3))
+    eng.close()
+
+
+def case_sampler(a):
+    """LM head and sampler at the full vocabulary on a one-layer engine (a profiling target of a few GB)."""
+    from . import corun, synth
+
+    sh = synth.ModelShape(1, 4096, 32, 8, 128, 12288, a.vocab, 1e-6, 1e6)
+    w = synth.make_weights_torch(sh, seed=0, device="cuda")
+    eng = corun.Engine(sh, w, a.B, 512)
+    slots = synth.pick_slots(a.B, a.active, seed=7)
+    for i, s in enumerate(slots):
+        eng.adopt(int(s), 0, 100, pending=1 + i, temperature=0.7, top_p=0.95)
+        eng.kv_fill(int(s), 36, 1.28, seed=100 + i)
+    active = np.zeros(a.B, np.uint8); active[slots] = 1
+    seeds = np.arange(a.B, dtype=np.uint64) + 1000
+    for _ in range(3):
+        eng.decode_step(active, seeds)
+    for name in ("gemm_lm_head", "sampler"):
+        print("%-14s %8.1f us per launch" % (name, eng.time_kernel(eng.KERNEL_KINDS.index(name), 6) * 1e3))
     eng.close()
 
 
@@ -266,12 +287,15 @@ def main():
     w = sub.add_parser("sweep")
     w.add_argument("--Bs", default="1,8,32,128,256"); w.add_argument("--fractions", default="0.125,0.5,1")
     w.add_argument("--steps", type=int, default=10)
+    sm = sub.add_parser("sampler")
+    sm.add_argument("--B", type=int, default=64); sm.add_argument("--active", type=int, default=40)
+    sm.add_argument("--vocab", type=int, default=151936)
     tr = sub.add_parser("trace")
     tr.add_argument("--requests", type=int, default=200); tr.add_argument("--rate", type=float, default=4.0)
     tr.add_argument("--B", type=int, default=128); tr.add_argument("--replay", type=int, default=4)
     a = ap.parse_args()
-    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "sweep": case_sweep,
-     "trace": case_trace}[a.case](a)
+    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "sampler": case_sampler,
+     "sweep": case_sweep, "trace": case_trace}[a.case](a)
 
 
 if __name__ == "__main__":
