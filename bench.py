@@ -281,6 +281,39 @@ def run_corun(args, rank, world):
     kernels["attention"]["GBs"] = att_bytes / (kt["attention"] * 1e-3) / 1e9
     launches = eng.decode_launches()
 
+    # ---- isolated prefill of one request into a free slot (the other half of the hot path): wall time of
+    # corun_prefill with the prompt in host memory; roofline per 256-token chunk = max(executed MMA work at the
+    # measured dense bf16 rate, the layers' weights streamed once), plus the LM head for the last position
+    prefill = None
+    free = [s for s in range(B) if not active[s]]
+    n_pf = min(1024, max_ctx - 8)
+    if free and n_pf >= 16:
+        prompt = synth.make_prompts(sh.vocab, [n_pf], seed=9)[0]
+        dt = 0.0
+        for _ in range(2):                                   # the second call is timed
+            sync_all()
+            t0 = time.perf_counter()
+            eng.prefill(free[0], prompt, n_pf + 4, T, P, seed=7)
+            torch.cuda.synchronize()
+            dt = time.perf_counter() - t0
+            eng.release(free[0])
+        w_lm = 2 * sh.vocab * sh.hidden
+        w_layers = w_bytes - w_lm
+        tf_s = tf
+        pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+        if os.path.exists(pk):
+            tf_s = float(json.load(open(pk)).get("bf16_tflops_sustained", tf))
+        t_roof = w_lm / (hbm * 1e9)
+        left = n_pf
+        while left > 0:
+            rows = min(256, left)
+            t_roof += max(2 * 2 * (w_layers // 2) * rows / (tf_s * 1e12), w_layers / (hbm * 1e9))
+            left -= rows
+        prefill = {"tokens": n_pf, "ms": dt * 1e3, "tok_per_s": n_pf / dt, "roofline_ms": t_roof * 1e3,
+                   "frac": t_roof / dt, "bound": "tensor",
+                   "note": "executed MMA work counted (activations are a bf16 hi/lo pair: two MMAs per weight tile) at "
+                           "%.0f TFLOP/s sustained; attention not counted" % tf_s}
+
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:
         w_np = synth.weights_torch_to_numpy(w_t)
@@ -313,7 +346,7 @@ def run_corun(args, rank, world):
         "clocks": clk, "gpu_launches": launches * K,
         "e2e": {"value": e2e_val, "unit": "tok/s", "ms_per_step": 1e3 * e2e_s / K,
                 "h2d_bytes_per_step": B * 9, "d2h_bytes_per_step": B * 4 + 4},
-        "roofline": roofline, "step_roofline": step_roof, "kernels": kernels, "cpu_baseline": cpu,
+        "roofline": roofline, "step_roofline": step_roof, "kernels": kernels, "prefill": prefill, "cpu_baseline": cpu,
     }))
 
 
