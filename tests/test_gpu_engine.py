@@ -280,3 +280,45 @@ def test_multi_split_attention_matches_oracle(orc, tiny, n_ctx):
     np.testing.assert_array_equal(k_back, cache[0][1, :n_ctx])
     e.close()
     assert err <= TOL, err
+
+
+@pytest.mark.parametrize("nq,nkv,hd", [(4, 4, 64), (8, 1, 64), (4, 2, 128), (8, 8, 128)])
+def test_other_head_groupings_match_oracle(orc, nq, nkv, hd):
+    """Query heads per KV head 1, 2 and 8 (the tiny and the Qwen shapes have 2 and 4), both head sizes:
+    prefill of a prompt that spans several attention splits, then teacher-forced decode steps among
+    co-tenants, against the oracle."""
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2608_14376_b200 import corun
+    from tests.helpers import oracle_model
+
+    sh = synth.ModelShape(2, 256, nq, nkv, hd, 512, 1024, 1e-6, 1e4)
+    w_np = synth.make_weights_numpy(sh, seed=nq * 10 + nkv)
+    w_t = synth.weights_numpy_to_torch(w_np, "cuda")
+    model = oracle_model(orc, sh, w_np)
+    eng = corun.Engine(sh, w_t, 4, 512)
+    try:
+        prompts = synth.make_prompts(sh.vocab, [300, 37, 130], seed=nq + nkv)
+        reqs, worst = [], 0.0
+        for slot, p in zip((2, 0, 3), prompts):
+            r = orc.Request(model, p, 77 + slot, max_T=512)
+            want = r.prefill()
+            eng.prefill(slot, p, len(p) + 8, seed=77 + slot)
+            worst = max(worst, float(np.abs(eng.logits(slot) - r.logits).max()))
+            eng.force_token(slot, want)
+            reqs.append((slot, r))
+        active = np.zeros(4, np.uint8); active[[2, 0, 3]] = 1
+        seeds = np.zeros(4, np.uint64)
+        for step in range(4):
+            toks = eng.decode_step(active, seeds)
+            assert toks[1] == -1
+            for slot, r in reqs:
+                want = r.decode()
+                worst = max(worst, float(np.abs(eng.logits(slot) - r.logits).max()))
+                if top2_gap(r.logits) > GAP:
+                    assert toks[slot] == want
+                eng.force_token(slot, want)
+        assert worst <= TOL, worst
+    finally:
+        eng.close()
