@@ -749,11 +749,12 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
       const int l = i % s.n_layers;   // rotate over the layers so that L2 cannot hold the weights
       GemmOut prev = P.p_down.out();
       switch (kind) {
-        case 0: ce = gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st); break;
-        case 1: ce = gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st); break;
-        case 2: ce = gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st); break;
-        case 3: ce = gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st); break;
-        case 4: ce = gemm_launch(P.p_lm, nullptr, e->d_status, e->st);
+        // launched as in the step's graph: with programmatic stream serialization
+        case 0: ce = gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, nullptr, true); break;
+        case 1: ce = gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st, nullptr, true); break;
+        case 2: ce = gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st, nullptr, true); break;
+        case 3: ce = gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st, nullptr, true); break;
+        case 4: ce = gemm_launch(P.p_lm, nullptr, e->d_status, e->st, nullptr, true);
                 if (ce == cudaSuccess) ce = gemm_fixup_launch(P.p_lm, e->st);
                 break;
         case 5: ce = cudaMemsetAsync(P.att_pool + l, 0, sizeof(int), e->st);   // the launch does not reset its pool counter
