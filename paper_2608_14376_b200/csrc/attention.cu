@@ -694,6 +694,8 @@ cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, con
   (void)layer;   // the tensor maps are the layer's
   const int group = nq / kv.n_kv;
   if (group * kv.n_kv != nq || max_splits > 256) return cudaErrorInvalidValue;
+  if (reuse)   // a prefill chunk: consecutive tokens of one request
+    return launch_attention_prefill(tmK, tmV, q, rows, nq, kv, out_hi, out_lo, d_status, st);
   const long long most = (long long)rows.R * max_splits * kv.n_kv;
   const int grid = (int)(most < grid_ctas ? most : grid_ctas);
   if (kv.hd == 128)

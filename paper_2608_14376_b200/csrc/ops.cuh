@@ -63,8 +63,8 @@ cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *
 // Split-KV paged attention partials and their fixed-order combine -> bf16 hi/lo [R, nq*hd] (rows that are
 // not active keep what they held).  done_count: [R * n_kv] ints, zero before the first launch (the kernel
 // leaves them zero).  pool_count: one int, zero before the launch (not reset by it): the items beyond the
-// CTAs' fixed stretches are drawn through it.  reuse: nonzero when the rows read the same cache rows one after
-// the other (the rows of a prefill chunk): the tiles are then kept in L2 instead of being marked evict-first.
+// CTAs' fixed stretches are drawn through it.  reuse: nonzero when the rows are the
+// consecutive tokens of one request in one slot (a prefill chunk): launch_attention_prefill runs instead.
 // tmK / tmV: tensor maps over this layer's pages: keys as rows of hd halfs with a [16, 64] box (128-byte
 // swizzle), values as rows of 16 halfs with an [hd, 16] box (32-byte swizzle); see attention.cu.
 // work / n_work: the step's (row, kv head, split) items from launch_attn_worklist (the same for every layer);
@@ -76,6 +76,11 @@ cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, con
                              unsigned long long *trace = nullptr);   // optional [grid][64][8] stamps (debug)
 cudaError_t launch_attn_worklist(const Rows &rows, int n_kv, int *work, int *n_work, int *pool_counts,
                                  int n_pool_counts, cudaStream_t st);   // also zeroes the launches' pool counters
+// Causal attention of a prefill chunk (rows = consecutive tokens of one request, all of one slot): query
+// tiles share the key / value tiles they read; writes the bf16 hi/lo output directly (attention_prefill.cu).
+cudaError_t launch_attention_prefill(const CUtensorMap &tmK, const CUtensorMap &tmV, const float *q, const Rows &rows,
+                                     int nq, const KvLayout &kv, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
+                                     int *d_status, cudaStream_t st);
 cudaError_t attention_prepare();   // opts the kernels into their shared-memory size (idempotent)
 // y = silu(gate) * up from the gate-up GEMM result -> bf16 hi/lo [R, F].
 cudaError_t launch_swiglu(const GemmOut &gu, int R, int F, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, cudaStream_t st);
