@@ -344,6 +344,12 @@ int gemm_plan_fill(GemmPlan *p, const void *W, int N, int K, const void *Xhi, co
   p->KB = K / GEMM_BLOCK_K;
   const long long total = (long long)p->n_tiles * p->KB;
   p->grid = (int)(total < num_sms ? total : num_sms);
+  // With several CTAs per tile the ranges are cut tile by tile (the same number of CTAs for every tile, a few
+  // SMs left out): no CTA then crosses a tile boundary, so none has two epilogues in a row, and above 128
+  // rows -- where the two row blocks of a tile fill TMEM and the epilogue of a segment cannot overlap the MMAs
+  // of the next -- none stops in the middle of its range.
+  const int per_tile = p->grid >= 2 * p->n_tiles ? p->grid / p->n_tiles : 0;
+  if (per_tile) p->grid = per_tile * p->n_tiles;
   if (total * (long long)p->grid >= (1ll << 31)) return CORUN_EINVAL;
   const size_t stage = (size_t)W_TILE_BYTES + (BN <= 64 ? (size_t)A_BLOCK_BYTES : 2 * (size_t)BN * GEMM_BLOCK_K * 2);
   // the MMA always reads 128 activation rows: leave that much readable behind the last stage
@@ -371,7 +377,9 @@ int gemm_plan_fill(GemmPlan *p, const void *W, int N, int K, const void *Xhi, co
   const int n_ints = p->grid + 1 + 3 * p->n_tiles;
   if (n_ints > tab_cap) return CORUN_ELIMIT;
   int *cs = tab, *cb = cs + p->grid + 1, *ce = cb + p->n_tiles, *sp = ce + p->n_tiles;
-  for (int c = 0; c <= p->grid; ++c) cs[c] = (int)((long long)c * total / p->grid);
+  for (int c = 0; c <= p->grid; ++c)
+    cs[c] = per_tile ? (c / per_tile) * p->KB + (int)((long long)(c % per_tile) * p->KB / per_tile)
+                     : (int)((long long)c * total / p->grid);
   p->n_split_tiles = 0;
   for (int t = 0, c = 0; t < p->n_tiles; ++t) {
     const int first = t * p->KB, last = first + p->KB - 1;
