@@ -4,12 +4,14 @@
     python -m paper_2608_14376_b200.cases kernels   [--layers 4 --B 64 --active-frac 0.625 --vocab 32768]
     python -m paper_2608_14376_b200.cases attention [--layers 2 --B 64 --active 40 --ctx-lo 512 --ctx-hi 4096 --reps 2]
     python -m paper_2608_14376_b200.cases sampler   [--B 64 --active 40 --vocab 151936]
+    python -m paper_2608_14376_b200.cases prefill   [--layers 2 --tokens 4096 --reps 2]
     python -m paper_2608_14376_b200.cases sweep     [--Bs 1,8,32,128,256 --fractions 0.125,0.5,1 --steps 10]
     python -m paper_2608_14376_b200.cases trace     [--requests 200 --rate 4 --B 128 --replay 4]
 
 ``gemm`` runs the stand-alone decode GEMM on seeded inputs; ``attention`` builds a Qwen3-8B-shaped
 engine with few layers, fills the cache of the active slots on the device and runs decode steps.
 Each prints the CUDA-event time per launch, for comparison with what a profiler reports.
+``prefill`` runs the isolated prefill of one seeded prompt on a Qwen3-8B-shaped engine with few layers.
 ``sweep`` is the occupancy sweep on the full Qwen3-8B shape: one engine per padded batch B, contexts
 uniform in 256..8192 (seed 3) filled on the device, requests admitted in seeded order until the KV
 pool is full; prints decode tok/s, time per output token and the fraction of the step roofline.
@@ -62,6 +64,31 @@ def case_attention(a):
     ms = eng.time_kernel(5, 2 * a.layers)
     print("attention: %d active, mean ctx %.0f, %.1f MB of KV per layer, %.1f us per launch pair (%.0f GB/s)"
           % (a.active, float(np.mean(ctx)), kv_bytes / 1e6, ms * 1e3, kv_bytes / ms / 1e6))
+    eng.close()
+
+
+def case_prefill(a):
+    import time
+
+    import torch
+
+    from . import corun, synth
+
+    sh = synth.ModelShape(a.layers, 4096, 32, 8, 128, 12288, 4096, 1e-6, 1e6)
+    w = synth.make_weights_torch(sh, seed=0, device="cuda")
+    eng = corun.Engine(sh, w, 2, a.tokens + 64)
+    prompt = synth.make_prompts(sh.vocab, [a.tokens], seed=11)[0]
+    first = None
+    for _ in range(a.reps):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        tok = eng.prefill(0, prompt, a.tokens + 16, 0.7, 0.95, seed=5)
+        torch.cuda.synchronize()
+        ms = (time.perf_counter() - t0) * 1e3
+        eng.release(0)
+        assert first is None or tok == first, "prefill of the same prompt gave another token"
+        first = tok
+    print("prefill: %d tokens, %d layers: %.2f ms (%.0f tok/s), first token %d" % (a.tokens, a.layers, ms, a.tokens / ms * 1e3, first))
     eng.close()
 
 
@@ -284,6 +311,9 @@ def main():
     k.add_argument("--active-frac", type=float, default=0.625); k.add_argument("--ctx-lo", type=int, default=512)
     k.add_argument("--ctx-hi", type=int, default=4096); k.add_argument("--vocab", type=int, default=32768)
     k.add_argument("--trace", action="store_true")
+    pf = sub.add_parser("prefill")
+    pf.add_argument("--layers", type=int, default=2); pf.add_argument("--tokens", type=int, default=4096)
+    pf.add_argument("--reps", type=int, default=2)
     w = sub.add_parser("sweep")
     w.add_argument("--Bs", default="1,8,32,128,256"); w.add_argument("--fractions", default="0.125,0.5,1")
     w.add_argument("--steps", type=int, default=10)
@@ -294,7 +324,7 @@ def main():
     tr.add_argument("--requests", type=int, default=200); tr.add_argument("--rate", type=float, default=4.0)
     tr.add_argument("--B", type=int, default=128); tr.add_argument("--replay", type=int, default=4)
     a = ap.parse_args()
-    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "sampler": case_sampler,
+    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "prefill": case_prefill, "sampler": case_sampler,
      "sweep": case_sweep, "trace": case_trace}[a.case](a)
 
 
