@@ -184,8 +184,10 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
   const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
   const KvLayout kv = kv_layout(e);
   int n = 0;
-  CK(launch_attn_worklist(rows, e->sh.n_kv_heads, P.att_work, P.att_n_work, P.att_pool, s.n_layers, e->st));   // the same items serve every layer
-  n += 1;
+  if (&P == &e->dec) {                              // the prefill attention kernel needs no item list
+    CK(launch_attn_worklist(rows, e->sh.n_kv_heads, P.att_work, P.att_n_work, P.att_pool, s.n_layers, e->st));   // the same items serve every layer
+    n += 1;
+  }
   // (debug) slice of the step trace for the idx-th GEMM of the decode program: [num_sms][8] stamps
   auto tr = [&](int idx) -> unsigned long long * {
     return (e->step_trace && &P == &e->dec) ? e->step_trace + (size_t)idx * e->num_sms * 8 : nullptr;
