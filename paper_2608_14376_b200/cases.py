@@ -5,6 +5,7 @@
     python -m paper_2608_14376_b200.cases attention [--layers 2 --B 64 --active 40 --ctx-lo 512 --ctx-hi 4096 --reps 2]
     python -m paper_2608_14376_b200.cases sampler   [--B 64 --active 40 --vocab 151936]
     python -m paper_2608_14376_b200.cases prefill   [--layers 2 --tokens 4096 --reps 2]
+    python -m paper_2608_14376_b200.cases ablation  [--layers 2 --B 64 --actives 1,4,16,40,64]
     python -m paper_2608_14376_b200.cases sweep     [--Bs 1,8,32,128,256 --fractions 0.125,0.5,1 --steps 10]
     python -m paper_2608_14376_b200.cases trace     [--requests 200 --rate 4 --B 128 --replay 4]
 
@@ -12,6 +13,9 @@
 engine with few layers, fills the cache of the active slots on the device and runs decode steps.
 Each prints the CUDA-event time per launch, for comparison with what a profiler reports.
 ``prefill`` runs the isolated prefill of one seeded prompt on a Qwen3-8B-shaped engine with few layers.
+``ablation`` compares the request-local split of the decode attention (every 128-token split of a request is
+an item any SM may take) with the same kernel handing out whole (row, kv head) pairs, i.e. no parallelism
+inside a request's attention, on ragged and on equal context lengths; the logits are the same bytes either way.
 ``sweep`` is the occupancy sweep on the full Qwen3-8B shape: one engine per padded batch B, contexts
 uniform in 256..8192 (seed 3) filled on the device, requests admitted in seeded order until the KV
 pool is full; prints decode tok/s, time per output token and the fraction of the step roofline.
@@ -90,6 +94,48 @@ def case_prefill(a):
         first = tok
     print("prefill: %d tokens, %d layers: %.2f ms (%.0f tok/s), first token %d" % (a.tokens, a.layers, ms, a.tokens / ms * 1e3, first))
     eng.close()
+
+
+def case_ablation(a):
+    import os
+
+    import torch
+
+    from . import corun, synth
+
+    sh = synth.ModelShape(a.layers, 4096, 32, 8, 128, 12288, 4096, 1e-6, 1e6)
+    w = synth.make_weights_torch(sh, seed=0, device="cuda")
+    actives = [int(x) for x in a.actives.split(",")]
+    print("| contexts | active | request-local split us | whole pairs us | ratio | same bytes |")
+    print("|---|---|---|---|---|---|")
+    for mix in ("ragged", "equal"):
+        for n_act in actives:
+            ctx = (synth.uniform_lengths(a.ctx_lo, a.ctx_hi, n_act, seed=2) if mix == "ragged"
+                   else np.full(n_act, (a.ctx_lo + a.ctx_hi) // 2))
+            slots = synth.pick_slots(a.B, n_act, seed=7)
+            res = []
+            for whole in (0, 1):
+                if whole:
+                    os.environ["CORUN_ATTN_WHOLE_PAIRS"] = "1"
+                try:
+                    eng = corun.Engine(sh, w, a.B, -(-(int(ctx.max()) + 64) // 256) * 256)
+                finally:
+                    os.environ.pop("CORUN_ATTN_WHOLE_PAIRS", None)
+                for i, (s_, c) in enumerate(zip(slots, ctx)):
+                    eng.adopt(int(s_), 0, int(c) + 16, pending=1 + i, temperature=0.7, top_p=0.95)
+                    eng.kv_fill(int(s_), int(c), 1.28, seed=100 + i)
+                active = np.zeros(a.B, np.uint8); active[slots] = 1
+                seeds = np.arange(a.B, dtype=np.uint64) + 1000
+                toks = eng.decode_step(active, seeds)
+                bytes_ = b"".join(eng.logits(int(s_)).tobytes() for s_ in slots)
+                us = eng.time_kernel(5, 4 * a.layers) * 1e3
+                res.append((us, bytes_, toks.tobytes()))
+                eng.close()
+            same = res[0][1] == res[1][1] and res[0][2] == res[1][2]
+            print("| %s %d..%d | %d | %.1f | %.1f | %.2f | %s |" % (mix, int(ctx.min()), int(ctx.max()), n_act, res[0][0], res[1][0],
+                                                           res[1][0] / res[0][0], "yes" if same else "NO"))
+            if not same:
+                raise SystemExit(1)
 
 
 def case_kernels(a):
@@ -314,6 +360,10 @@ def main():
     pf = sub.add_parser("prefill")
     pf.add_argument("--layers", type=int, default=2); pf.add_argument("--tokens", type=int, default=4096)
     pf.add_argument("--reps", type=int, default=2)
+    ab = sub.add_parser("ablation")
+    ab.add_argument("--layers", type=int, default=2); ab.add_argument("--B", type=int, default=64)
+    ab.add_argument("--actives", default="1,4,16,40,64"); ab.add_argument("--ctx-lo", type=int, default=512)
+    ab.add_argument("--ctx-hi", type=int, default=4096)
     w = sub.add_parser("sweep")
     w.add_argument("--Bs", default="1,8,32,128,256"); w.add_argument("--fractions", default="0.125,0.5,1")
     w.add_argument("--steps", type=int, default=10)
@@ -324,7 +374,7 @@ def main():
     tr.add_argument("--requests", type=int, default=200); tr.add_argument("--rate", type=float, default=4.0)
     tr.add_argument("--B", type=int, default=128); tr.add_argument("--replay", type=int, default=4)
     a = ap.parse_args()
-    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "prefill": case_prefill, "sampler": case_sampler,
+    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "prefill": case_prefill, "ablation": case_ablation, "sampler": case_sampler,
      "sweep": case_sweep, "trace": case_trace}[a.case](a)
 
 

@@ -189,7 +189,8 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   const int n_total = *n_work;
   if (n_total <= 0) return;
   // this CTA's stretch of the item list, and where the shared pool begins
-  const int n_fixed = (int)(((long long)n_total * 15 / 16) / gridDim.x);
+  const int n_pairs = n_work[1];                 // > 0: the ablation that hands out whole (row, kv head) pairs (see item_of)
+  const int n_fixed = n_pairs > 0 ? 0 : (int)(((long long)n_total * 15 / 16) / gridDim.x);
   const int item_lo = (int)blockIdx.x * n_fixed, pool_lo = (int)gridDim.x * n_fixed;
 
   extern __shared__ uint8_t smem_raw[];
@@ -239,8 +240,35 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   // Item of this CTA's k-th slot (every role walks the slots 0, 1, 2, ... with the same ring indices):
   // first the fixed stretch, then pairs drawn from the pool.  The key producer draws (draw = true, whole
   // warp) and publishes the pair; the other roles wait for it.  -1: no more work; -2: nothing in this slot.
+  // Ablation mode (n_pairs > 0): no parallelism inside a (row, kv head) pair.  A CTA draws whole pairs from
+  // the counter, one at a time, and walks each pair's splits in order (its two groups in turn); the table
+  // behind the item count gives every pair's first item and split count.  The values are the same either way.
+  const int *pair_tab = n_work + 2;
   int pair_j = -1, pair_c = 0;
+  int wp_base = 0, wp_ns = 0, wp_start = 0;
   auto item_of = [&](int k, bool draw) -> int {
+    if (n_pairs > 0) {
+      while (wp_start >= 0 && k >= wp_base + wp_ns) {
+        wp_base += wp_ns;
+        ++pair_j;
+        int c = 0;
+        if (draw) {
+          if (lane == 0) {
+            c = atomicAdd(pool_count, 1);
+            pool_pair[pair_j & 3] = c;
+            mbar_arrive(smem_u32(&pool_bar[pair_j & 3]));
+          }
+          c = __shfl_sync(0xffffffffu, c, 0);
+        } else {
+          if (!mbar_wait(smem_u32(&pool_bar[pair_j & 3]), (uint32_t)(pair_j >> 2) & 1u, &abort_flag)) return -1;
+          c = pool_pair[pair_j & 3];
+        }
+        if (c >= n_pairs) { wp_start = -1; break; }
+        wp_start = __ldg(pair_tab + 2 * c);
+        wp_ns = __ldg(pair_tab + 2 * c + 1);
+      }
+      return wp_start < 0 ? -1 : wp_start + (k - wp_base);
+    }
     if (k < n_fixed)   // even slots walk the first half of the stretch (group 0), odd slots the second half (group 1)
       return item_lo + ((k & 1) ? ((n_fixed + 1) >> 1) + (k >> 1) : (k >> 1));
     const int j = (k - n_fixed) >> 1;
@@ -609,9 +637,11 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 
 // Lists the items of the step: active rows ascending, kv heads ascending, splits ascending.
 // One CTA; rows <= 256.  Entry = row << 16 | kv head << 8 | split.
+// n_work[0] = number of items; n_work[1] = number of (row, kv head) pairs listed behind it as (first item,
+// split count) when whole_pairs is set (the ablation without parallelism inside a pair), else 0.
 __global__ void __launch_bounds__(256) attn_worklist_kernel(Rows rows, int n_kv, int *__restrict__ work,
                                                             int *__restrict__ n_work, int *__restrict__ pool_counts,
-                                                            int n_pool_counts) {
+                                                            int n_pool_counts, int whole_pairs) {
   griddep_launch_dependents();
   griddep_wait();
   for (int i = threadIdx.x; i < n_pool_counts; i += 256) pool_counts[i] = 0;   // one pool counter per attention launch of the step
@@ -629,11 +659,22 @@ __global__ void __launch_bounds__(256) attn_worklist_kernel(Rows rows, int n_kv,
     for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
     const int ns = cnt[row];
     for (int i = lane; i < ns * n_kv; i += 32) work[before * n_kv + i] = (row << 16) | ((i / ns) << 8) | (i % ns);
+    if (whole_pairs && ns > 0) {
+      int rows_before = 0;                          // active rows before this one
+      for (int i = lane; i < row; i += 32) rows_before += cnt[i] > 0;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) rows_before += __shfl_xor_sync(0xffffffffu, rows_before, o);
+      for (int g = lane; g < n_kv; g += 32) {
+        n_work[2 + 2 * (rows_before * n_kv + g)] = before * n_kv + g * ns;
+        n_work[3 + 2 * (rows_before * n_kv + g)] = ns;
+      }
+    }
   }
   if (r == 255) {
-    int tot = 0;
-    for (int i = 0; i < 256; ++i) tot += cnt[i];
-    *n_work = tot * n_kv;
+    int tot = 0, act = 0;
+    for (int i = 0; i < 256; ++i) { tot += cnt[i]; act += cnt[i] > 0; }
+    n_work[0] = tot * n_kv;
+    n_work[1] = whole_pairs ? act * n_kv : 0;
   }
 }
 
@@ -680,10 +721,10 @@ cudaError_t attention_prepare() {
 }
 
 cudaError_t launch_attn_worklist(const Rows &rows, int n_kv, int *work, int *n_work, int *pool_counts,
-                                 int n_pool_counts, cudaStream_t st) {
+                                 int n_pool_counts, int whole_pairs, cudaStream_t st) {
   if (rows.R > 256 || n_kv > 255) return cudaErrorInvalidValue;
   return launch_k(attn_worklist_kernel, dim3(1), dim3(256), 0, st, true, rows, n_kv, work, n_work, pool_counts,
-                  n_pool_counts);
+                  n_pool_counts, whole_pairs);
 }
 
 cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, const float *q, const Rows &rows, int nq,

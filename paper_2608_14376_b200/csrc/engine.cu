@@ -53,6 +53,7 @@ struct Program {
 struct corun_engine {
   corun_shape sh{};
   int B = 0, max_ctx = 0, max_blocks = 0, max_splits = 0, chunk = 0, num_sms = 0;
+  int whole_pairs = 0;               // ablation: attention without parallelism inside a (row, kv head) pair
   int64_t pool_blocks = 0;
   cudaStream_t st = nullptr;
   bool own_stream = false;
@@ -139,7 +140,7 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm) {
     RC(dmalloc(A, &P.part_acc, (size_t)R * s.n_q_heads * e->max_splits * s.head_dim));
     RC(dmalloc(A, &P.part_ml, (size_t)R * s.n_q_heads * e->max_splits * 2));
     RC(dmalloc(A, &P.att_work, (size_t)R * e->max_splits * e->sh.n_kv_heads));
-    RC(dmalloc(A, &P.att_n_work, 1));
+    RC(dmalloc(A, &P.att_n_work, 2 + 2 * (size_t)R * e->sh.n_kv_heads));
     RC(dmalloc(A, &P.att_done, (size_t)R * e->sh.n_kv_heads));
     RC(dmalloc(A, &P.att_pool, (size_t)s.n_layers));
     RC(dmalloc(A, &P.qkv_out, (size_t)R * (QD + 2 * KD)));
@@ -185,7 +186,7 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
   const KvLayout kv = kv_layout(e);
   int n = 0;
   if (&P == &e->dec) {                              // the prefill attention kernel needs no item list
-    CK(launch_attn_worklist(rows, e->sh.n_kv_heads, P.att_work, P.att_n_work, P.att_pool, s.n_layers, e->st));   // the same items serve every layer
+    CK(launch_attn_worklist(rows, e->sh.n_kv_heads, P.att_work, P.att_n_work, P.att_pool, s.n_layers, e->whole_pairs, e->st));   // the same items serve every layer
     n += 1;
   }
   // (debug) slice of the step trace for the idx-th GEMM of the decode program: [num_sms][8] stamps
@@ -373,6 +374,7 @@ int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int3
     if (e->pool_blocks < 1) return fail(CORUN_ENOMEM);
   }
   e->chunk = 256;
+  if (const char *c = getenv("CORUN_ATTN_WHOLE_PAIRS")) e->whole_pairs = atoi(c) != 0;   // ablation only
   if (const char *c = getenv("CORUN_PREFILL_CHUNK")) {
     const int v = atoi(c);
     if (v >= 16 && v <= 256 && v % 16 == 0) e->chunk = v;

@@ -399,7 +399,7 @@ __device__ __noinline__ void smp_tail_full_row(SmpShared &sh, const SampleArgs &
 // the drawn token.
 constexpr int SMP_CLUSTER = 4;
 
-__global__ void __cluster_dims__(SMP_CLUSTER, 1, 1) __launch_bounds__(SMP_THREADS) sampler_kernel(SampleArgs a) {
+__global__ void __cluster_dims__(SMP_CLUSTER, 1, 1) __launch_bounds__(SMP_THREADS, 2) sampler_kernel(SampleArgs a) {
   namespace cg = cooperative_groups;
   griddep_launch_dependents();
   griddep_wait();

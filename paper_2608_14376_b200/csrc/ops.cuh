@@ -74,8 +74,11 @@ cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, con
                              int grid_ctas, float *part_acc, float *part_ml, int *done_count, int *pool_count,
                              __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int reuse, int *d_status, cudaStream_t st,
                              unsigned long long *trace = nullptr);   // optional [grid][64][8] stamps (debug)
+// n_work: 2 + 2 * rows * n_kv ints (item count, pair count, then the pairs' (first item, split count) when
+// whole_pairs is set: the ablation in which a CTA takes whole (row, kv head) pairs).  Also zeroes the
+// launches' pool counters.
 cudaError_t launch_attn_worklist(const Rows &rows, int n_kv, int *work, int *n_work, int *pool_counts,
-                                 int n_pool_counts, cudaStream_t st);   // also zeroes the launches' pool counters
+                                 int n_pool_counts, int whole_pairs, cudaStream_t st);
 // Causal attention of a prefill chunk (rows = consecutive tokens of one request, all of one slot): query
 // tiles share the key / value tiles they read; writes the bf16 hi/lo output directly (attention_prefill.cu).
 cudaError_t launch_attention_prefill(const CUtensorMap &tmK, const CUtensorMap &tmV, const float *q, const Rows &rows,

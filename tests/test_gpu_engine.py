@@ -322,3 +322,34 @@ def test_other_head_groupings_match_oracle(orc, nq, nkv, hd):
         assert worst <= TOL, worst
     finally:
         eng.close()
+
+
+def test_attention_item_assignment_changes_no_bit(tiny):
+    """Which SM computes which split of a request's attention has no influence on any value: the
+    ablation mode, in which a CTA takes whole (row, kv head) pairs instead of single splits, yields
+    the same logit bytes and tokens as the request-local split."""
+    from paper_2608_14376_b200 import corun
+
+    sh = tiny.sh
+    ctxs = [700, 130, 1023, 257, 64]
+    slots = [6, 1, 3, 0, 5]
+    out = []
+    for whole in (0, 1):
+        if whole:
+            os.environ["CORUN_ATTN_WHOLE_PAIRS"] = "1"
+        try:
+            e = corun.Engine(sh, tiny.w_t, B, 1040)
+        finally:
+            os.environ.pop("CORUN_ATTN_WHOLE_PAIRS", None)
+        for i, (s, n) in enumerate(zip(slots, ctxs)):
+            e.adopt(s, 0, n + 8, pending=11 + i, temperature=0.7, top_p=0.95)
+            e.kv_fill(s, n, 0.5, seed=40 + i)
+        active = np.zeros(B, np.uint8); active[slots] = 1
+        seeds = np.arange(B, dtype=np.uint64) + 9
+        got = []
+        for _ in range(3):
+            toks = e.decode_step(active, seeds)
+            got.append((toks.tobytes(), b"".join(e.logits(s).tobytes() for s in slots)))
+        e.close()
+        out.append(got)
+    assert out[0] == out[1]
