@@ -112,6 +112,27 @@ int corun_prefill(corun_engine *e, int32_t slot, const int32_t *tokens, int32_t 
                   const corun_sampling *sampling, uint64_t seed, int32_t *out_first_token);
 
 /*
+ * Prefill of several requests in shared chunks (paper, Future Work, "Batch-
+ * Invariant Kernels for Prefill": prefill requests batched with other prefill
+ * requests, never with decode).  The prompts go through the same fixed-shape
+ * prefill program as corun_prefill; the rows of a chunk are dealt in request
+ * order, every piece of a request starting on a boundary of the attention
+ * kernel's query tiles, so that short prompts share a chunk instead of padding
+ * one each.  All kernels of the program are position-invariant in the chunk
+ * and attention reads every key from the cache, so each request's cache,
+ * logits and first token are bitwise those of corun_prefill on it alone.
+ *   slots, n_tokens, reserve_lens, samplings, seeds   host, n_req entries
+ *                (slots distinct and free).
+ *   tokens       host, the prompts one after the other (sum of n_tokens ids).
+ *   out_first_tokens  host, n_req entries, may be NULL.
+ * Errors as corun_prefill; ENOSPACE if the reservations do not all fit (the
+ * engine is unchanged).
+ */
+int corun_prefill_batch(corun_engine *e, int32_t n_req, const int32_t *slots, const int32_t *tokens,
+                        const int32_t *n_tokens, const int32_t *reserve_lens, const corun_sampling *samplings,
+                        const uint64_t *seeds, int32_t *out_first_tokens);
+
+/*
  * One fixed-shape decode iteration (paper, Design, "Fixed-Shape Batched
  * Decode", "Shape-Aligned Sampling", "Determinism Argument"): every slot with
  * active[s] != 0 feeds its pending token at position = its context length,

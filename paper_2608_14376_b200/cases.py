@@ -5,6 +5,7 @@
     python -m paper_2608_14376_b200.cases attention [--layers 2 --B 64 --active 40 --ctx-lo 512 --ctx-hi 4096 --reps 2]
     python -m paper_2608_14376_b200.cases sampler   [--B 64 --active 40 --vocab 151936]
     python -m paper_2608_14376_b200.cases prefill   [--layers 2 --tokens 4096 --reps 2]
+    python -m paper_2608_14376_b200.cases prefill_batch [--layers 36 --lengths 40,100,200,500,1000 --n 8]
     python -m paper_2608_14376_b200.cases ablation  [--layers 2 --B 64 --actives 1,4,16,40,64]
     python -m paper_2608_14376_b200.cases sweep     [--Bs 1,8,32,128,256 --fractions 0.125,0.5,1 --steps 10]
     python -m paper_2608_14376_b200.cases trace     [--requests 200 --rate 4 --B 128 --replay 4]
@@ -13,6 +14,8 @@
 engine with few layers, fills the cache of the active slots on the device and runs decode steps.
 Each prints the CUDA-event time per launch, for comparison with what a profiler reports.
 ``prefill`` runs the isolated prefill of one seeded prompt on a Qwen3-8B-shaped engine with few layers.
+``prefill_batch`` times n prompts of one length prefilled one by one (isolated) and in shared chunks
+(``corun_prefill_batch``) and checks that the first tokens and logits are the same bytes.
 ``ablation`` compares the request-local split of the decode attention (every 128-token split of a request is
 an item any SM may take) with the same kernel handing out whole (row, kv head) pairs, i.e. no parallelism
 inside a request's attention, on ragged and on equal context lengths; the logits are the same bytes either way.
@@ -93,6 +96,43 @@ def case_prefill(a):
         assert first is None or tok == first, "prefill of the same prompt gave another token"
         first = tok
     print("prefill: %d tokens, %d layers: %.2f ms (%.0f tok/s), first token %d" % (a.tokens, a.layers, ms, a.tokens / ms * 1e3, first))
+    eng.close()
+
+
+def case_prefill_batch(a):
+    import time
+
+    import torch
+
+    from . import corun, synth
+
+    sh = synth.ModelShape(a.layers, 4096, 32, 8, 128, 12288, 151936 if a.layers == 36 else 4096, 1e-6, 1e6)
+    w = synth.make_weights_torch(sh, seed=0, device="cuda")
+    lengths = [int(x) for x in a.lengths.split(",")]
+    eng = corun.Engine(sh, w, max(a.n, 2), max(lengths) + 64)
+    slots = list(range(a.n))
+    print("| prompt tokens | requests | isolated ms | batched ms | ratio | same bytes |")
+    print("|---|---|---|---|---|---|")
+    for L in lengths:
+        prompts = synth.make_prompts(sh.vocab, [L] * a.n, seed=50 + L)
+        seeds = np.arange(a.n, dtype=np.uint64) + 7
+        res = []
+        for batched in (0, 1, 0, 1):                # the first pair warms up
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            if batched:
+                first = list(eng.prefill_batch(slots, prompts, [L + 8] * a.n, 0.7, 0.95, seeds))
+            else:
+                first = [eng.prefill(s_, p, L + 8, 0.7, 0.95, seed=int(sd)) for s_, p, sd in zip(slots, prompts, seeds)]
+            torch.cuda.synchronize()
+            ms = (time.perf_counter() - t0) * 1e3
+            res.append((ms, first, b"".join(eng.logits(s_).tobytes() for s_ in slots)))
+            for s_ in slots:
+                eng.release(s_)
+        same = res[2][1:] == res[3][1:]
+        print("| %d | %d | %.1f | %.1f | %.2f | %s |" % (L, a.n, res[2][0], res[3][0], res[2][0] / res[3][0], "yes" if same else "NO"))
+        if not same:
+            raise SystemExit(1)
     eng.close()
 
 
@@ -360,6 +400,9 @@ def main():
     pf = sub.add_parser("prefill")
     pf.add_argument("--layers", type=int, default=2); pf.add_argument("--tokens", type=int, default=4096)
     pf.add_argument("--reps", type=int, default=2)
+    pb = sub.add_parser("prefill_batch")
+    pb.add_argument("--layers", type=int, default=36); pb.add_argument("--lengths", default="40,100,200,500,1000")
+    pb.add_argument("--n", type=int, default=8)
     ab = sub.add_parser("ablation")
     ab.add_argument("--layers", type=int, default=2); ab.add_argument("--B", type=int, default=64)
     ab.add_argument("--actives", default="1,4,16,40,64"); ab.add_argument("--ctx-lo", type=int, default=512)
@@ -374,7 +417,7 @@ def main():
     tr.add_argument("--requests", type=int, default=200); tr.add_argument("--rate", type=float, default=4.0)
     tr.add_argument("--B", type=int, default=128); tr.add_argument("--replay", type=int, default=4)
     a = ap.parse_args()
-    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "prefill": case_prefill, "ablation": case_ablation, "sampler": case_sampler,
+    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "prefill": case_prefill, "ablation": case_ablation, "prefill_batch": case_prefill_batch, "sampler": case_sampler,
      "sweep": case_sweep, "trace": case_trace}[a.case](a)
 
 

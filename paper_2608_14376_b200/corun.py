@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libcorun.so")
 OK, EINVAL, ESLOT, ENOSPACE, ECTX, ECUDA, ETIMEOUT, ENOMEM, ELIMIT = 0, -1, -2, -3, -4, -5, -6, -7, -8
 
 EXPORTS = [
-    "corun_init", "corun_prefill", "corun_decode_step", "corun_decode_enqueue", "corun_decode_wait",
+    "corun_init", "corun_prefill", "corun_prefill_batch", "corun_decode_step", "corun_decode_enqueue", "corun_decode_wait",
     "corun_release", "corun_destroy", "corun_get_logits", "corun_force_token", "corun_context_len",
     "corun_free_blocks", "corun_debug_kv_read", "corun_debug_kv_write", "corun_debug_adopt",
     "corun_debug_set_eager", "corun_debug_read", "corun_debug_gemm_trace", "corun_debug_attn_trace", "corun_debug_step_trace", "corun_debug_kv_fill", "corun_debug_time_kernel", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
@@ -82,6 +82,7 @@ def lib():
         vp, i32, i64, u64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64
         L.corun_init.argtypes = [C.POINTER(Shape), C.POINTER(Weights), i32, i32, i32, i64, vp, C.POINTER(vp)]
         L.corun_prefill.argtypes = [vp, i32, vp, i32, i32, C.POINTER(Sampling), u64, C.POINTER(i32)]
+        L.corun_prefill_batch.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp]
         L.corun_decode_step.argtypes = [vp, vp, vp, vp]
         L.corun_decode_enqueue.argtypes = [vp, vp, vp]
         L.corun_decode_wait.argtypes = [vp, vp]
@@ -190,6 +191,21 @@ class Engine:
         _check(lib().corun_prefill(self._h, slot, t.ctypes.data, t.shape[0], reserve_len, C.byref(s),
                                    seed & (2**64 - 1), C.byref(first)), "corun_prefill")
         return int(first.value)
+
+    def prefill_batch(self, slots, prompts, reserve_lens, temperature: float = 0.0, top_p: float = 1.0, seeds=None) -> np.ndarray:
+        """Prefill of several requests in shared chunks; returns their first tokens."""
+        n = len(slots)
+        sl = np.ascontiguousarray(slots, dtype=np.int32)
+        lens = np.ascontiguousarray([len(p) for p in prompts], dtype=np.int32)
+        toks = np.ascontiguousarray(np.concatenate([np.asarray(p, dtype=np.int32) for p in prompts]), dtype=np.int32)
+        res = np.ascontiguousarray(reserve_lens, dtype=np.int32)
+        smp = (Sampling * n)(*[Sampling(temperature, top_p) for _ in range(n)])
+        sd = np.ascontiguousarray(seeds if seeds is not None else np.zeros(n), dtype=np.uint64)
+        out = np.full(n, -1, np.int32)
+        assert sl.shape == lens.shape == res.shape == sd.shape == (n,)
+        _check(lib().corun_prefill_batch(self._h, n, sl.ctypes.data, toks.ctypes.data, lens.ctypes.data, res.ctypes.data,
+                                         C.cast(smp, C.c_void_p), sd.ctypes.data, out.ctypes.data), "corun_prefill_batch")
+        return out
 
     def decode_step(self, active, seeds) -> np.ndarray:
         a = np.ascontiguousarray(active, dtype=np.uint8)

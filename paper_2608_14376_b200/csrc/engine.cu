@@ -497,70 +497,150 @@ void corun_destroy(corun_engine *e) {
   delete e;
 }
 
+}  // extern "C"
+
+namespace {
+
+struct PfReq {
+  int slot;
+  const int32_t *tokens;
+  int n, reserve;
+  corun_sampling smp;
+  uint64_t seed;
+  int first;
+};
+
+// Final norm -> LM head (one row) -> sample with R(seed, 0) for the request whose last prompt token is row
+// `row` of the chunk that has just run; the logits go to the slot's row of the decode logits.
+int prefill_finish_row(corun_engine *e, int row, PfReq &r) {
+  const corun_shape &s = e->sh;
+  Program &P = e->pre, &L = e->lm1;
+  GemmOut prev = P.p_down.out();
+  prev.direct += (size_t)row * prev.N;
+  prev.ws += (size_t)row * GEMM_TILE_N;
+  const Rows one{P.row_token + row, P.row_pos + row, P.row_active + row, P.row_slot + row, 1};
+  CK(launch_resid_norm(P.h + (size_t)row * s.hidden, s.hidden, nullptr, one, &prev, e->final_norm, s.rms_eps, L.xn_hi,
+                       L.xn_lo, e->st));
+  CK(gemm_launch(L.p_lm, nullptr, e->d_status, e->st));
+  CK(gemm_fixup_launch(L.p_lm, e->st));
+  const int zero = 0;
+  CK(cudaMemcpyAsync(e->d_pf_temp, &r.smp.temperature, sizeof(float), cudaMemcpyHostToDevice, e->st));
+  CK(cudaMemcpyAsync(e->d_pf_top_p, &r.smp.top_p, sizeof(float), cudaMemcpyHostToDevice, e->st));
+  CK(cudaMemcpyAsync(e->d_pf_seed, &r.seed, sizeof(uint64_t), cudaMemcpyHostToDevice, e->st));
+  CK(cudaMemcpyAsync(e->d_pf_step, &zero, sizeof(int), cudaMemcpyHostToDevice, e->st));
+  SampleArgs sa{L.logits, s.vocab, e->d_pf_one, e->d_pf_temp, e->d_pf_top_p, e->d_pf_seed, e->d_pf_step, nullptr,
+                e->d_pf_tok};
+  CK(launch_sampler(sa, 1, e->st));
+  CK(cudaMemcpyAsync(e->dec.logits + (size_t)r.slot * s.vocab, L.logits, (size_t)s.vocab * sizeof(float),
+                     cudaMemcpyDeviceToDevice, e->st));
+  CK(cudaMemcpyAsync(&r.first, e->d_pf_tok, sizeof(int), cudaMemcpyDeviceToHost, e->st));
+  CK(cudaStreamSynchronize(e->st));   // the one-row buffers and the sampling staging serve the next request
+  return CORUN_OK;
+}
+
+// Prefill of one or several requests through the fixed-shape prefill program (chunks of `chunk` rows).  The
+// rows of a chunk are dealt in request order; every piece of a request starts on a tile boundary of the
+// prefill attention kernel (a tile's rows share one slot), so a chunk may hold pieces of several requests.
+// Every kernel of the program treats its rows independently of each other and of where they sit in the
+// chunk, and attention reads all keys -- the chunk's own too -- from the cache, so a request's values do not
+// depend on how its prompt is cut into pieces nor on what else shares its chunks.
+int prefill_many(corun_engine *e, PfReq *reqs, int n_req) {
+  const corun_shape &s = e->sh;
+  RC(sync_stream(e));
+  size_t need = 0;
+  for (int i = 0; i < n_req; ++i) need += (size_t)(reqs[i].reserve + KV_BLOCK - 1) / KV_BLOCK;
+  if (need > e->free_blocks.size()) return CORUN_ENOSPACE;
+  for (int i = 0; i < n_req; ++i) RC(reserve_blocks(e, reqs[i].slot, reqs[i].reserve));
+  Program &P = e->pre;
+  const int CH = e->chunk;
+  int unit = 128 / (s.n_q_heads / s.n_kv_heads);    // tokens per attention tile
+  if (unit > CH || CH % unit) unit = CH;
+  int *tok = e->h_rows, *pos = tok + CH, *act = pos + CH, *slt = act + CH;
+  std::vector<std::pair<int, int>> fins;           // (request, chunk row of its last prompt token)
+  int fill = 0, pad_slot = reqs[0].slot;
+  auto run_chunk = [&]() -> int {
+    for (int i = fill; i < CH; ++i) { tok[i] = 0; pos[i] = 0; act[i] = 0; slt[i] = pad_slot; }
+    CK(cudaMemcpyAsync(P.row_token, tok, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
+    CK(cudaMemcpyAsync(P.row_pos, pos, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
+    CK(cudaMemcpyAsync(P.row_active, act, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
+    CK(cudaMemcpyAsync(P.row_slot, slt, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
+    RC(run_layers(e, P, nullptr));
+    for (auto &f : fins) RC(prefill_finish_row(e, f.second, reqs[f.first]));
+    CK(cudaStreamSynchronize(e->st));   // the staging arrays are reused by the next chunk
+    fins.clear();
+    fill = 0;
+    return CORUN_OK;
+  };
+  for (int r = 0; r < n_req; ++r) {
+    const PfReq &q = reqs[r];
+    for (int done = 0; done < q.n;) {
+      while (fill % unit) { tok[fill] = 0; pos[fill] = 0; act[fill] = 0; slt[fill] = pad_slot; ++fill; }   // rest of the tile before
+      if (fill == CH) RC(run_chunk());
+      const int take = q.n - done < CH - fill ? q.n - done : CH - fill;
+      for (int i = 0; i < take; ++i) {
+        tok[fill + i] = q.tokens[done + i];
+        pos[fill + i] = done + i;
+        act[fill + i] = 1;
+        slt[fill + i] = q.slot;
+      }
+      fill += take;
+      done += take;
+      pad_slot = q.slot;                            // padding up to the tile's end belongs to this request's tile
+      if (done == q.n) fins.emplace_back(r, fill - 1);
+      if (fill == CH) RC(run_chunk());
+    }
+  }
+  if (fill > 0 || !fins.empty()) RC(run_chunk());
+  CK(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, e->st));
+  CK(cudaStreamSynchronize(e->st));
+  RC(check_status(e));
+  for (int i = 0; i < n_req; ++i) {
+    PfReq &q = reqs[i];
+    RC(set_slot_state(e, q.slot, 1, q.n, 1, q.first, q.smp.temperature, q.smp.top_p));
+    e->in_use[q.slot] = 1;
+    e->ctx[q.slot] = q.n;
+    e->reserve[q.slot] = q.reserve;
+    e->step[q.slot] = 1;
+  }
+  return CORUN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
 int corun_prefill(corun_engine *e, int32_t slot, const int32_t *tokens, int32_t n, int32_t reserve_len,
                   const corun_sampling *sampling, uint64_t seed, int32_t *out_first_token) {
   if (!e || !tokens || !sampling || n < 1 || reserve_len < n || reserve_len > e->max_ctx) return CORUN_EINVAL;
   if (!slot_ok(e, slot) || e->in_use[slot]) return CORUN_ESLOT;
   for (int i = 0; i < n; ++i)
     if (tokens[i] < 0 || tokens[i] >= e->sh.vocab) return CORUN_EINVAL;
-  RC(sync_stream(e));
-  RC(reserve_blocks(e, slot, reserve_len));
-  Program &P = e->pre;
-  const corun_shape &s = e->sh;
-  const int CH = e->chunk;
-  int last_row = 0;
-  for (int pos0 = 0; pos0 < n; pos0 += CH) {
-    const int rows_here = (n - pos0 < CH) ? n - pos0 : CH;
-    int *tok = e->h_rows, *pos = tok + CH, *act = pos + CH, *slt = act + CH;
-    for (int i = 0; i < CH; ++i) {
-      const bool on = i < rows_here;
-      tok[i] = on ? tokens[pos0 + i] : 0;
-      pos[i] = on ? pos0 + i : 0;
-      act[i] = on ? 1 : 0;
-      slt[i] = slot;
-    }
-    CK(cudaMemcpyAsync(P.row_token, tok, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
-    CK(cudaMemcpyAsync(P.row_pos, pos, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
-    CK(cudaMemcpyAsync(P.row_active, act, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
-    CK(cudaMemcpyAsync(P.row_slot, slt, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
-    RC(run_layers(e, P, nullptr));
-    CK(cudaStreamSynchronize(e->st));   // the staging arrays are reused by the next chunk
-    last_row = rows_here - 1;
+  PfReq r{slot, tokens, n, reserve_len, *sampling, seed, -1};
+  RC(prefill_many(e, &r, 1));
+  if (out_first_token) *out_first_token = r.first;
+  return CORUN_OK;
+}
+
+int corun_prefill_batch(corun_engine *e, int32_t n_req, const int32_t *slots, const int32_t *tokens,
+                        const int32_t *n_tokens, const int32_t *reserve_lens, const corun_sampling *samplings,
+                        const uint64_t *seeds, int32_t *out_first_tokens) {
+  if (!e || n_req < 1 || !slots || !tokens || !n_tokens || !reserve_lens || !samplings || !seeds) return CORUN_EINVAL;
+  std::vector<PfReq> reqs((size_t)n_req);
+  size_t off = 0;
+  for (int i = 0; i < n_req; ++i) {
+    const int n = n_tokens[i];
+    if (n < 1 || reserve_lens[i] < n || reserve_lens[i] > e->max_ctx) return CORUN_EINVAL;
+    if (!slot_ok(e, slots[i]) || e->in_use[slots[i]]) return CORUN_ESLOT;
+    for (int j = 0; j < i; ++j)
+      if (slots[j] == slots[i]) return CORUN_ESLOT;
+    for (int t = 0; t < n; ++t)
+      if (tokens[off + t] < 0 || tokens[off + t] >= e->sh.vocab) return CORUN_EINVAL;
+    reqs[i] = PfReq{slots[i], tokens + off, n, reserve_lens[i], samplings[i], seeds[i], -1};
+    off += (size_t)n;
   }
-  // last position only: final norm -> LM head (one row) -> sample with R(seed, 0)
-  {
-    Program &L = e->lm1;
-    GemmOut prev = P.p_down.out();
-    prev.direct += (size_t)last_row * prev.N;
-    prev.ws += (size_t)last_row * GEMM_TILE_N;
-    const Rows one{P.row_token + last_row, P.row_pos + last_row, P.row_active + last_row, P.row_slot + last_row, 1};
-    CK(launch_resid_norm(P.h + (size_t)last_row * s.hidden, s.hidden, nullptr, one, &prev, e->final_norm, s.rms_eps,
-                         L.xn_hi, L.xn_lo, e->st));
-    CK(gemm_launch(L.p_lm, nullptr, e->d_status, e->st));
-    CK(gemm_fixup_launch(L.p_lm, e->st));
-    const int zero = 0;
-    CK(cudaMemcpyAsync(e->d_pf_temp, &sampling->temperature, sizeof(float), cudaMemcpyHostToDevice, e->st));
-    CK(cudaMemcpyAsync(e->d_pf_top_p, &sampling->top_p, sizeof(float), cudaMemcpyHostToDevice, e->st));
-    CK(cudaMemcpyAsync(e->d_pf_seed, &seed, sizeof(uint64_t), cudaMemcpyHostToDevice, e->st));
-    CK(cudaMemcpyAsync(e->d_pf_step, &zero, sizeof(int), cudaMemcpyHostToDevice, e->st));
-    SampleArgs sa{L.logits, s.vocab, e->d_pf_one, e->d_pf_temp, e->d_pf_top_p, e->d_pf_seed, e->d_pf_step, nullptr,
-                  e->d_pf_tok};
-    CK(launch_sampler(sa, 1, e->st));
-    CK(cudaMemcpyAsync(e->dec.logits + (size_t)slot * s.vocab, L.logits, (size_t)s.vocab * sizeof(float),
-                       cudaMemcpyDeviceToDevice, e->st));
-    CK(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, e->st));
-    CK(cudaStreamSynchronize(e->st));
-  }
-  int first = -1;
-  CK(cudaMemcpyAsync(&first, e->d_pf_tok, sizeof(int), cudaMemcpyDeviceToHost, e->st));
-  CK(cudaStreamSynchronize(e->st));
-  RC(check_status(e));
-  RC(set_slot_state(e, slot, 1, n, 1, first, sampling->temperature, sampling->top_p));
-  e->in_use[slot] = 1;
-  e->ctx[slot] = n;
-  e->reserve[slot] = reserve_len;
-  e->step[slot] = 1;
-  if (out_first_token) *out_first_token = first;
+  RC(prefill_many(e, reqs.data(), n_req));
+  if (out_first_tokens)
+    for (int i = 0; i < n_req; ++i) out_first_tokens[i] = reqs[i].first;
   return CORUN_OK;
 }
 

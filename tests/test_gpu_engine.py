@@ -353,3 +353,61 @@ def test_attention_item_assignment_changes_no_bit(tiny):
         e.close()
         out.append(got)
     assert out[0] == out[1]
+
+
+def test_batched_prefill_equals_isolated_prefill(tiny):
+    """Prefill requests batched with other prefill requests (the paper's future work on prefill): prompts
+    that share chunks -- pieces starting on attention-tile boundaries, a prompt cut differently than when
+    it runs alone -- leave the same cache, logits, first tokens and following decode steps, byte for byte,
+    as isolated prefill of each."""
+    from paper_2608_14376_b200 import corun
+
+    sh = tiny.sh
+    lens = [5, 70, 64, 1, 300, 33, 129]
+    slots = [3, 0, 6, 1, 7, 2, 5]
+    prompts = synth.make_prompts(sh.vocab, lens, seed=91)
+    seeds = np.array([synth.request_seed(i) for i in range(len(lens))], np.uint64)
+    res = [n + 8 for n in lens]
+    T, P_ = 0.7, 0.95
+
+    def after(e):
+        active = np.zeros(B, np.uint8); active[slots] = 1
+        sd = np.zeros(B, np.uint64); sd[slots] = seeds
+        out = []
+        out.append(b"".join(e.logits(s).tobytes() for s in slots))
+        for layer in range(sh.n_layers):
+            for s, n in zip(slots, lens):
+                k, v = e.kv_read(s, layer, 0, n)
+                out.append(k.tobytes() + v.tobytes())
+        for _ in range(3):
+            out.append(e.decode_step(active, sd).tobytes())
+            out.append(b"".join(e.logits(s).tobytes() for s in slots))
+        return out
+
+    e = corun.Engine(sh, tiny.w_t, B, 512)
+    first_iso = [e.prefill(s, p, r, T, P_, seed=int(sd)) for s, p, r, sd in zip(slots, prompts, res, seeds)]
+    iso = after(e)
+    for s in slots:
+        e.release(s)
+    first_bat = e.prefill_batch(slots, prompts, res, T, P_, seeds)
+    bat = after(e)
+    assert list(first_bat) == first_iso
+    assert bat == iso
+    # error paths: a busy slot, a slot named twice, a reservation beyond max_context -- the engine stays as it was
+    with pytest.raises(corun.CorunError):
+        e.prefill_batch([slots[0]], [prompts[0]], [res[0]])
+    e.release(slots[0]); e.release(slots[1])
+    free = e.free_blocks()
+    with pytest.raises(corun.CorunError):
+        e.prefill_batch([slots[0], slots[0]], prompts[:2], res[:2])
+    with pytest.raises(corun.CorunError):
+        e.prefill_batch([slots[0], slots[1]], prompts[:2], [res[0], 10 ** 6])
+    assert e.free_blocks() == free
+    e.close()
+    # reservations that do not all fit: nothing is taken
+    small = corun.Engine(sh, tiny.w_t, B, 512, kv_pool_blocks=12)
+    with pytest.raises(corun.CorunError) as ei:
+        small.prefill_batch([0, 1], prompts[1:3], [100, 100])     # 7 + 7 pages of 16 tokens
+    assert ei.value.status == corun.ENOSPACE and small.free_blocks() == 12
+    assert list(small.prefill_batch([0], prompts[1:2], [100], T, P_, seeds[1:2])) == [first_iso[1]]
+    small.close()
