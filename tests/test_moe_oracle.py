@@ -1,0 +1,104 @@
+"""Pins of the Mixture-of-Experts block oracle against things other than itself (CPU)."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import moe_oracle as mo
+
+
+def _rand(shape, seed, scale=1.0):
+    return np.random.default_rng(seed).standard_normal(shape) * scale
+
+
+def test_hand_computed_routing_and_output():
+    """H = 2, E = 4 experts that only scale: the router weights are chosen so that the logits are
+    log 4, log 3, log 2, log 1 -> p = .4 .3 .2 .1; top-2 keeps experts 0 and 1 with .4 and .3 (no
+    renormalisation).  Expert e: Wg = Wu = rows that read x0, Wd = c_e, so FFN_e(x) = c_e * silu(x0) * x0."""
+    x = np.array([1.0, 0.0])
+    Wr = np.array([[math.log(4), 0], [math.log(3), 0], [math.log(2), 0], [0.0, 0]])
+    c = [1.0, 10.0, 100.0, 1000.0]
+    Wg = np.array([[[1.0, 0.0]]] * 4)            # [E, F=1, H=2]
+    Wu = np.array([[[1.0, 0.0]]] * 4)
+    Wd = np.array([[[ce], [0.0]] for ce in c])   # [E, H=2, F=1]
+    ids, ps, p_all = mo.router(x, Wr, 2)
+    assert list(ids) == [0, 1]
+    np.testing.assert_allclose(p_all, [0.4, 0.3, 0.2, 0.1], rtol=1e-12)
+    Y, ids2, p2 = mo.moe_ffn(x[None], Wr, Wg, Wu, Wd, [], 2)
+    s = 1.0 / (1.0 + math.exp(-1.0))             # silu(1) * 1
+    np.testing.assert_allclose(Y[0], [(0.4 * 1.0 + 0.3 * 10.0) * s, 0.0], rtol=1e-12)
+    # with a shared expert of weight 1 on top
+    Ys, _, _ = mo.moe_ffn(x[None], Wr, Wg, Wu, Wd, [(Wg[0], Wu[0], np.array([[7.0], [0.0]]))], 2)
+    np.testing.assert_allclose(Ys[0], [(0.4 + 3.0 + 7.0) * s, 0.0], rtol=1e-12)
+
+
+def test_ties_go_to_the_lower_expert_id():
+    x = np.array([1.0, 2.0])
+    Wr = np.zeros((6, 2))                        # all logits equal
+    ids, ps, _ = mo.router(x, Wr, 3)
+    assert list(ids) == [0, 1, 2]
+    np.testing.assert_allclose(ps, 1 / 6)
+    Wr[4] = [1.0, 0.0]                           # one clear winner, the rest tied
+    ids, _, _ = mo.router(x, Wr, 3)
+    assert list(ids) == [4, 0, 1]
+
+
+def test_all_experts_selected_and_identical_is_the_dense_ffn():
+    """top_k = E with identical experts: the probabilities sum to 1, so y = FFN(x) whatever the router says."""
+    H, F, E, B = 12, 20, 5, 4
+    X = _rand((B, H), 1)
+    wg, wu, wd = _rand((F, H), 2, 0.3), _rand((F, H), 3, 0.3), _rand((H, F), 4, 0.3)
+    Wg, Wu, Wd = np.stack([wg] * E), np.stack([wu] * E), np.stack([wd] * E)
+    Y, _, P = mo.moe_ffn(X, _rand((E, H), 5), Wg, Wu, Wd, [], E)
+    np.testing.assert_allclose(P.sum(1), 1.0, rtol=1e-12)
+    torch = pytest.importorskip("torch")
+    xt = torch.tensor(X, dtype=torch.float64)
+    ref = (torch.nn.functional.silu(xt @ torch.tensor(wg).T) * (xt @ torch.tensor(wu).T)) @ torch.tensor(wd).T
+    np.testing.assert_allclose(Y, ref.numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_brute_force_scalar_loops_on_a_tiny_case():
+    H, F, E, B, K = 5, 3, 6, 3, 2
+    X, Wr = _rand((B, H), 11), _rand((E, H), 12)
+    Wg, Wu, Wd = _rand((E, F, H), 13), _rand((E, F, H), 14), _rand((E, H, F), 15)
+    sh = [(_rand((F, H), 16), _rand((F, H), 17), _rand((H, F), 18))]
+    Y, ids, ps = mo.moe_ffn(X, Wr, Wg, Wu, Wd, sh, K)
+    for b in range(B):
+        logit = [sum(Wr[e][h] * X[b][h] for h in range(H)) for e in range(E)]
+        den = sum(math.exp(l) for l in logit)
+        p = [math.exp(l) / den for l in logit]
+        chosen = sorted(range(E), key=lambda e: (-p[e], e))[:K]
+        assert list(ids[b]) == chosen
+        def one(wg, wu, wd, scale):
+            hid = []
+            for f in range(F):
+                g = sum(wg[f][h] * X[b][h] for h in range(H))
+                u = sum(wu[f][h] * X[b][h] for h in range(H))
+                hid.append(g / (1.0 + math.exp(-g)) * u)
+            return [scale * sum(wd[h][f] * hid[f] for f in range(F)) for h in range(H)]
+        want = [0.0] * H
+        for e in chosen:
+            want = [a + c for a, c in zip(want, one(Wg[e], Wu[e], Wd[e], p[e]))]
+        want = [a + c for a, c in zip(want, one(*sh[0], 1.0))]
+        np.testing.assert_allclose(Y[b], want, rtol=1e-10, atol=1e-12)
+
+
+def test_rows_are_independent_and_the_override_keeps_the_routers_probabilities():
+    H, F, E, B, K = 8, 6, 7, 5, 3
+    X, Wr = _rand((B, H), 21), _rand((E, H), 22)
+    Wg, Wu, Wd = _rand((E, F, H), 23), _rand((E, F, H), 24), _rand((E, H, F), 25)
+    Y, ids, ps = mo.moe_ffn(X, Wr, Wg, Wu, Wd, [], K)
+    perm = np.array([3, 0, 4, 2, 1])
+    Yp, idp, _ = mo.moe_ffn(X[perm], Wr, Wg, Wu, Wd, [], K)
+    np.testing.assert_array_equal(Yp, Y[perm])
+    np.testing.assert_array_equal(idp, ids[perm])
+    # forcing the router's own choice changes nothing; forcing another choice uses that choice's probabilities
+    Y2, _, _ = mo.moe_ffn(X, Wr, Wg, Wu, Wd, [], K, experts=ids)
+    np.testing.assert_array_equal(Y2, Y)
+    other = np.array([[0, 1, 2]] * B)
+    Y3, _, p3 = mo.moe_ffn(X, Wr, Wg, Wu, Wd, [], K, experts=other)
+    for b in range(B):
+        _, _, p_all = mo.router(X[b], Wr, K)
+        np.testing.assert_allclose(p3[b], p_all[:3])
+        want = sum(p_all[e] * mo.ffn(X[b], Wg[e], Wu[e], Wd[e]) for e in range(3))
+        np.testing.assert_allclose(Y3[b], want, rtol=1e-12)
