@@ -8,9 +8,9 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcorun.so")
-SOURCES = ["engine.cu", "gemm.cu", "ops.cu", "attention.cu", "attention_prefill.cu", "no_alloc.cu", "sched.cu"]
+SOURCES = ["engine.cu", "gemm.cu", "ops.cu", "attention.cu", "attention_prefill.cu", "no_alloc.cu", "sched.cu", "moe.cu"]
 HEADERS = ["gemm.cuh", "ops.cuh", "ptx.cuh", os.path.join("..", "..", "include", "corun.h"),
-           os.path.join("..", "..", "include", "corun_sched.h")]
+           os.path.join("..", "..", "include", "corun_sched.h"), os.path.join("..", "..", "include", "corun_moe.h")]
 
 
 def _nvcc() -> str:

@@ -6,6 +6,7 @@
     python -m paper_2608_14376_b200.cases sampler   [--B 64 --active 40 --vocab 151936]
     python -m paper_2608_14376_b200.cases prefill   [--layers 2 --tokens 4096 --reps 2]
     python -m paper_2608_14376_b200.cases prefill_batch [--layers 36 --lengths 40,100,200,500,1000 --n 8]
+    python -m paper_2608_14376_b200.cases moe       [--B 128 --reps 20]      # DeepSeek-V2-Lite MoE block shape
     python -m paper_2608_14376_b200.cases ablation  [--layers 2 --B 64 --actives 1,4,16,40,64]
     python -m paper_2608_14376_b200.cases sweep     [--Bs 1,8,32,128,256 --fractions 0.125,0.5,1 --steps 10]
     python -m paper_2608_14376_b200.cases trace     [--requests 200 --rate 4 --B 128 --replay 4]
@@ -16,6 +17,8 @@ Each prints the CUDA-event time per launch, for comparison with what a profiler 
 ``prefill`` runs the isolated prefill of one seeded prompt on a Qwen3-8B-shaped engine with few layers.
 ``prefill_batch`` times n prompts of one length prefilled one by one (isolated) and in shared chunks
 (``corun_prefill_batch``) and checks that the first tokens and logits are the same bytes.
+``moe`` times the Mixture-of-Experts feed-forward block (64 routed experts of 1408, top-6, 2 shared, hidden
+2048) on B padded rows against the bytes of expert weights a call streams.
 ``ablation`` compares the request-local split of the decode attention (every 128-token split of a request is
 an item any SM may take) with the same kernel handing out whole (row, kv head) pairs, i.e. no parallelism
 inside a request's attention, on ragged and on equal context lengths; the logits are the same bytes either way.
@@ -134,6 +137,34 @@ def case_prefill_batch(a):
         if not same:
             raise SystemExit(1)
     eng.close()
+
+
+def case_moe(a):
+    import torch
+
+    from . import corun
+
+    H, E, K, F, S = a.hidden, a.experts, a.top_k, a.ffn, a.shared
+    g = torch.Generator(device="cuda").manual_seed(0)
+    mk = lambda *shape: (torch.randn(shape, generator=g, device="cuda") * 0.02).to(torch.bfloat16).contiguous()
+    router, gate_up, down = mk(E, H), mk((E + S) * 2 * F, H), mk(H, (E + S) * F)
+    op = corun.MoeFfn(H, E, K, F, S, router, gate_up, down, a.B)
+    x = torch.randn((a.B, H), generator=g, device="cuda")
+    for _ in range(3):
+        y, ex, pr = op.forward(x)
+    op.sync()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(a.reps):
+        op.forward(x, want_routing=False)
+    t1.record()
+    op.sync()
+    ms = t0.elapsed_time(t1) / a.reps
+    wb = op.weight_bytes()
+    hit = len(torch.unique(ex))
+    print("moe: B=%d H=%d E=%d top-%d F=%d shared=%d: %.1f us per call, %.1f MB of weights -> %.0f GB/s; %d of %d experts selected; %d launches"
+          % (a.B, H, E, K, F, S, ms * 1e3, wb / 1e6, wb / ms / 1e6, hit, E, op.launches()))
+    op.close()
 
 
 def case_ablation(a):
@@ -403,6 +434,11 @@ def main():
     pb = sub.add_parser("prefill_batch")
     pb.add_argument("--layers", type=int, default=36); pb.add_argument("--lengths", default="40,100,200,500,1000")
     pb.add_argument("--n", type=int, default=8)
+    mo = sub.add_parser("moe")
+    mo.add_argument("--B", type=int, default=128); mo.add_argument("--reps", type=int, default=20)
+    mo.add_argument("--hidden", type=int, default=2048); mo.add_argument("--experts", type=int, default=64)
+    mo.add_argument("--top-k", type=int, default=6); mo.add_argument("--ffn", type=int, default=1408)
+    mo.add_argument("--shared", type=int, default=2)
     ab = sub.add_parser("ablation")
     ab.add_argument("--layers", type=int, default=2); ab.add_argument("--B", type=int, default=64)
     ab.add_argument("--actives", default="1,4,16,40,64"); ab.add_argument("--ctx-lo", type=int, default=512)
@@ -417,7 +453,7 @@ def main():
     tr.add_argument("--requests", type=int, default=200); tr.add_argument("--rate", type=float, default=4.0)
     tr.add_argument("--B", type=int, default=128); tr.add_argument("--replay", type=int, default=4)
     a = ap.parse_args()
-    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "prefill": case_prefill, "ablation": case_ablation, "prefill_batch": case_prefill_batch, "sampler": case_sampler,
+    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "prefill": case_prefill, "ablation": case_ablation, "moe": case_moe, "prefill_batch": case_prefill_batch, "sampler": case_sampler,
      "sweep": case_sweep, "trace": case_trace}[a.case](a)
 
 

@@ -24,7 +24,14 @@ EXPORTS = [
     "corun_debug_sample", "corun_gemm_static", "corun_strerror", "corun_last_cuda_error", "corun_engine_info",
     "corun_sched_create", "corun_sched_create_for_engine", "corun_sched_destroy", "corun_sched_submit",
     "corun_sched_step", "corun_sched_poll", "corun_sched_slot_of", "corun_sched_counts",
+    "corun_moe_create", "corun_moe_destroy", "corun_moe_forward", "corun_moe_sync", "corun_moe_weight_bytes",
+    "corun_moe_launches",
 ]
+
+
+class MoeShape(C.Structure):
+    _fields_ = [("hidden", C.c_int32), ("n_experts", C.c_int32), ("top_k", C.c_int32), ("expert_ffn", C.c_int32),
+                ("n_shared", C.c_int32)]
 
 
 class CorunError(RuntimeError):
@@ -122,6 +129,14 @@ def lib():
         L.corun_sched_poll.argtypes = [vp, i64, vp, i32, C.POINTER(i32), C.POINTER(i32)]
         L.corun_sched_slot_of.argtypes = [vp, i64, C.POINTER(i32)]
         L.corun_sched_counts.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
+        L.corun_moe_create.argtypes = [C.POINTER(MoeShape), vp, vp, vp, i32, vp, C.POINTER(vp)]
+        L.corun_moe_destroy.argtypes = [vp]
+        L.corun_moe_destroy.restype = None
+        L.corun_moe_forward.argtypes = [vp, vp, vp, vp, vp]
+        L.corun_moe_sync.argtypes = [vp]
+        L.corun_moe_weight_bytes.argtypes = [vp]
+        L.corun_moe_weight_bytes.restype = i64
+        L.corun_moe_launches.argtypes = [vp]
         for n in EXPORTS:
             getattr(L, n)
         _lib = L
@@ -403,3 +418,58 @@ def debug_sample(logits, temperature: float, top_p: float, u24) -> np.ndarray:
     _check(lib().corun_debug_sample(lg.ctypes.data, lg.shape[0], lg.shape[1], C.byref(s), u.ctypes.data,
                                     out.ctypes.data), "corun_debug_sample")
     return out
+
+
+class MoeFfn:
+    """Mixture-of-Experts feed-forward block (``include/corun_moe.h``).  Weights are CUDA bf16 tensors:
+    router [E, H], gate_up [(E + S) * 2F, H], down [H, (E + S) * F]; B padded rows per call."""
+
+    def __init__(self, hidden: int, n_experts: int, top_k: int, expert_ffn: int, n_shared: int, router, gate_up, down,
+                 B: int):
+        import torch
+
+        self._torch = torch
+        self.B, self.H, self.top_k = B, hidden, top_k
+        self._w = (router, gate_up, down)                     # keep the borrowed tensors alive
+        for t in self._w:
+            assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+        assert tuple(router.shape) == (n_experts, hidden)
+        assert tuple(gate_up.shape) == ((n_experts + n_shared) * 2 * expert_ffn, hidden)
+        assert tuple(down.shape) == (hidden, (n_experts + n_shared) * expert_ffn)
+        sh = MoeShape(hidden, n_experts, top_k, expert_ffn, n_shared)
+        h = C.c_void_p()
+        self._stream = torch.cuda.current_stream()
+        _check(lib().corun_moe_create(C.byref(sh), router.data_ptr(), gate_up.data_ptr(), down.data_ptr(), B,
+                                      self._stream.cuda_stream, C.byref(h)), "corun_moe_create")
+        self._h = h
+
+    def forward(self, x, want_routing: bool = True):
+        """x: CUDA fp32 [B, H] -> (y fp32 [B, H], experts int32 [B, top_k], probs fp32 [B, top_k]); asynchronous."""
+        torch = self._torch
+        assert x.is_cuda and x.dtype == torch.float32 and tuple(x.shape) == (self.B, self.H) and x.is_contiguous()
+        y = torch.empty_like(x)
+        ex = torch.empty((self.B, self.top_k), dtype=torch.int32, device=x.device) if want_routing else None
+        pr = torch.empty((self.B, self.top_k), dtype=torch.float32, device=x.device) if want_routing else None
+        _check(lib().corun_moe_forward(self._h, x.data_ptr(), y.data_ptr(), ex.data_ptr() if want_routing else None,
+                                       pr.data_ptr() if want_routing else None), "corun_moe_forward")
+        return y, ex, pr
+
+    def sync(self):
+        _check(lib().corun_moe_sync(self._h), "corun_moe_sync")
+
+    def weight_bytes(self) -> int:
+        return int(lib().corun_moe_weight_bytes(self._h))
+
+    def launches(self) -> int:
+        return int(lib().corun_moe_launches(self._h))
+
+    def close(self):
+        if self._h:
+            lib().corun_moe_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,248 @@
+// Mixture-of-Experts feed-forward block without groups: two plain decode GEMMs over all experts with a
+// masked, probability-weighted SwiGLU between them (see include/corun_moe.h for the formulation and why
+// it is position-invariant).  The kernels here are the router's softmax / top-k, the masked SwiGLU and
+// the read-out of the second GEMM; the GEMMs are gemm.cu's.
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/corun_moe.h"
+#include "gemm.cuh"
+#include "launch.cuh"
+#include "ops.cuh"
+#include "ptx.cuh"
+
+using namespace corun;
+
+namespace {
+
+using bf16 = __nv_bfloat16;
+constexpr int MOE_MAX_TOPK = 16;
+constexpr int MOE_MAX_EXPERTS = 256;
+
+#define MCK(call)                               \
+  do {                                          \
+    cudaError_t ce_ = (call);                   \
+    if (ce_ != cudaSuccess) {                   \
+      g_last_cuda_error = (int)ce_;             \
+      return CORUN_ECUDA;                       \
+    }                                           \
+  } while (0)
+
+__device__ __forceinline__ void moe_split(float x, bf16 &hi, bf16 &lo) {
+  hi = __float2bfloat16_rn(x);
+  lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+// One warp per row: softmax over the E router logits, then top_k by repeated arg-max with ties to the lower
+// id.  Lane l holds experts l, l + 32, ...; the sum of the exponentials is each lane's experts in ascending
+// id, then a fixed butterfly over the lanes.  Writes the routing and the row of SwiGLU weights
+// w[r, 0 .. E + S): p_e for the selected experts, 0 for the others, 1 for the shared ones.
+__global__ void __launch_bounds__(256) moe_route_kernel(GemmOut logits, int B, int E, int S, int top_k, float *__restrict__ w,
+                                                        int *__restrict__ experts, float *__restrict__ probs) {
+  griddep_launch_dependents();
+  griddep_wait();
+  const int lane = threadIdx.x & 31;
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= B) return;
+  constexpr int PER = MOE_MAX_EXPERTS / 32;
+  float z[PER];
+  float mx = -CUDART_INF_F;
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    const int e = lane + 32 * j;
+    z[j] = e < E ? gemm_load(logits, r, e) : -CUDART_INF_F;
+    mx = fmaxf(mx, z[j]);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  float sum = 0.f;
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    const int e = lane + 32 * j;
+    z[j] = e < E ? expf(z[j] - mx) : -1.f;           // -1: not an expert
+    if (e < E) sum += z[j];
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  float *wr = w + (size_t)r * (E + S);
+  for (int e = lane; e < E; e += 32) wr[e] = 0.f;
+  for (int s = lane; s < S; s += 32) wr[E + s] = 1.f;
+  __syncwarp();
+  for (int k = 0; k < top_k; ++k) {
+    float bz = -1.f;                                 // this lane's best: largest value, lowest id on ties
+    int be = 0x7fffffff;
+#pragma unroll
+    for (int j = 0; j < PER; ++j)
+      if (z[j] > bz) { bz = z[j]; be = lane + 32 * j; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float oz = __shfl_xor_sync(0xffffffffu, bz, o);
+      const int oe = __shfl_xor_sync(0xffffffffu, be, o);
+      if (oz > bz || (oz == bz && oe < be)) { bz = oz; be = oe; }
+    }
+    if (be >= E) be = k;                             // a row of NaNs: any valid id
+    const float p = __fdiv_rn(bz, sum);
+#pragma unroll
+    for (int j = 0; j < PER; ++j)
+      if (lane + 32 * j == be) z[j] = -2.f;          // taken
+    if (lane == 0) {
+      wr[be] = p;
+      if (experts) experts[(size_t)r * top_k + k] = be;
+      if (probs) probs[(size_t)r * top_k + k] = p;
+    }
+  }
+}
+
+// h[r, e*F + f] = w[r, e] * silu(gate) * up as a bf16 hi/lo pair; zeros where w[r, e] == 0 (nothing is read
+// there).  gate = GEMM-1 column e*2F + f, up = column e*2F + F + f.  Four f per thread.
+__global__ void __launch_bounds__(256) moe_swiglu_kernel(GemmOut gu, const float *__restrict__ w, int F, int n_blocks,
+                                                         bf16 *__restrict__ out_hi, bf16 *__restrict__ out_lo) {
+  griddep_launch_dependents();
+  griddep_wait();
+  const int r = blockIdx.y;
+  const int per_block = F / 4;
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= per_block * n_blocks) return;
+  const int e = idx / per_block, f = (idx - e * per_block) * 4;
+  const float we = w[(size_t)r * n_blocks + e];
+  float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (we != 0.f) {
+    const float4 g = gemm_load4(gu, r, e * 2 * F + f), u = gemm_load4(gu, r, e * 2 * F + F + f);
+    y = make_float4(we * (g.x / (1.f + expf(-g.x)) * u.x), we * (g.y / (1.f + expf(-g.y)) * u.y),
+                    we * (g.z / (1.f + expf(-g.z)) * u.z), we * (g.w / (1.f + expf(-g.w)) * u.w));
+  }
+  bf16 a[4], b[4];
+  moe_split(y.x, a[0], b[0]);
+  moe_split(y.y, a[1], b[1]);
+  moe_split(y.z, a[2], b[2]);
+  moe_split(y.w, a[3], b[3]);
+  const size_t o = (size_t)r * n_blocks * F + (size_t)e * F + f;
+  *reinterpret_cast<uint2 *>(out_hi + o) = *reinterpret_cast<const uint2 *>(a);
+  *reinterpret_cast<uint2 *>(out_lo + o) = *reinterpret_cast<const uint2 *>(b);
+}
+
+// y[r, :] = the second GEMM's result (partials of a tile added in ascending CTA order).
+__global__ void __launch_bounds__(256) moe_readout_kernel(GemmOut d, int H, float *__restrict__ y) {
+  griddep_launch_dependents();
+  griddep_wait();
+  const int r = blockIdx.y;
+  const int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i >= H) return;
+  *reinterpret_cast<float4 *>(y + (size_t)r * H + i) = gemm_load4(d, r, i);
+}
+
+}  // namespace
+
+struct corun_moe {
+  corun_moe_shape sh{};
+  int B = 0, BN = 0, num_sms = 0;
+  cudaStream_t st = nullptr;
+  std::vector<void *> allocs;
+  bf16 *router_pad = nullptr;                       // [256, H]: the router rows, zero rows behind them
+  bf16 *x_hi = nullptr, *x_lo = nullptr, *h_hi = nullptr, *h_lo = nullptr;
+  float *out_r = nullptr, *out_gu = nullptr, *out_d = nullptr, *ws = nullptr, *w = nullptr;
+  int *d_status = nullptr;
+  GemmPlan p_r, p_gu, p_d;
+  int64_t weight_bytes = 0;
+};
+
+namespace {
+
+template <typename T>
+int moe_alloc(corun_moe *m, T **p, size_t n) {
+  void *q = nullptr;
+  if (cudaMalloc(&q, n * sizeof(T)) != cudaSuccess) return CORUN_ENOMEM;
+  m->allocs.push_back(q);
+  if (cudaMemset(q, 0, n * sizeof(T)) != cudaSuccess) return CORUN_ECUDA;
+  *p = (T *)q;
+  return CORUN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int corun_moe_create(const corun_moe_shape *shape, const void *router, const void *gate_up, const void *down,
+                     int32_t B, void *cuda_stream, corun_moe **out) {
+  if (!shape || !router || !gate_up || !down || !out || B < 1 || B > 256) return CORUN_EINVAL;
+  const corun_moe_shape &s = *shape;
+  if (s.hidden < 64 || s.hidden % 64 || s.n_experts < 1 || s.n_experts > MOE_MAX_EXPERTS || s.top_k < 1 ||
+      s.top_k > MOE_MAX_TOPK || s.top_k > s.n_experts || s.expert_ffn < 64 || s.expert_ffn % 64 || s.n_shared < 0)
+    return CORUN_EINVAL;
+  corun_moe *m = new (std::nothrow) corun_moe();
+  if (!m) return CORUN_ENOMEM;
+  auto fail = [&](int rc) { corun_moe_destroy(m); return rc; };
+  m->sh = s;
+  m->B = B;
+  m->BN = (B + 15) / 16 * 16;
+  m->st = (cudaStream_t)cuda_stream;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&m->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return fail(CORUN_ECUDA);
+  const int H = s.hidden, E = s.n_experts, F = s.expert_ffn, NB = E + s.n_shared;
+  const size_t N1 = (size_t)NB * 2 * F, K2 = (size_t)NB * F;
+  if (N1 > (size_t)1 << 30 || K2 > (size_t)1 << 30) return fail(CORUN_EINVAL);
+  int rc;
+  if ((rc = moe_alloc(m, &m->router_pad, (size_t)GEMM_TILE_N * H)) || (rc = moe_alloc(m, &m->x_hi, (size_t)m->BN * H)) ||
+      (rc = moe_alloc(m, &m->x_lo, (size_t)m->BN * H)) || (rc = moe_alloc(m, &m->h_hi, (size_t)m->BN * K2)) ||
+      (rc = moe_alloc(m, &m->h_lo, (size_t)m->BN * K2)) || (rc = moe_alloc(m, &m->out_r, (size_t)m->BN * GEMM_TILE_N)) ||
+      (rc = moe_alloc(m, &m->out_gu, (size_t)m->BN * N1)) || (rc = moe_alloc(m, &m->out_d, (size_t)m->BN * H)) ||
+      (rc = moe_alloc(m, &m->ws, gemm_ws_floats(m->num_sms, m->BN))) || (rc = moe_alloc(m, &m->w, (size_t)B * NB)) ||
+      (rc = moe_alloc(m, &m->d_status, 1)))
+    return fail(rc);
+  if (cudaMemcpy(m->router_pad, router, (size_t)E * H * sizeof(bf16), cudaMemcpyDeviceToDevice) != cudaSuccess)
+    return fail(CORUN_ECUDA);
+  // the three GEMMs run one after the other and their results are consumed in between: one workspace serves all
+  if ((rc = gemm_plan_create(&m->p_r, m->router_pad, GEMM_TILE_N, H, m->x_hi, m->x_lo, B, m->BN, m->out_r, m->ws, m->num_sms)) ||
+      (rc = gemm_plan_create(&m->p_gu, gate_up, (int)N1, H, m->x_hi, m->x_lo, B, m->BN, m->out_gu, m->ws, m->num_sms)) ||
+      (rc = gemm_plan_create(&m->p_d, down, H, (int)K2, m->h_hi, m->h_lo, B, m->BN, m->out_d, m->ws, m->num_sms)))
+    return fail(rc);
+  m->weight_bytes = ((int64_t)E * H + (int64_t)N1 * H + (int64_t)H * K2) * 2;
+  if (cudaDeviceSynchronize() != cudaSuccess) return fail(CORUN_ECUDA);
+  *out = m;
+  return CORUN_OK;
+}
+
+void corun_moe_destroy(corun_moe *m) {
+  if (!m) return;
+  cudaStreamSynchronize(m->st);
+  gemm_plan_destroy(&m->p_r);
+  gemm_plan_destroy(&m->p_gu);
+  gemm_plan_destroy(&m->p_d);
+  for (void *p : m->allocs) cudaFree(p);
+  delete m;
+}
+
+int corun_moe_forward(corun_moe *m, const float *x, float *y, int32_t *experts, float *probs) {
+  if (!m || !x || !y || x == y) return CORUN_EINVAL;
+  const corun_moe_shape &s = m->sh;
+  const int H = s.hidden, E = s.n_experts, F = s.expert_ffn, NB = E + s.n_shared;
+  MCK(launch_split(x, m->B, H, m->x_hi, m->x_lo, m->st));
+  MCK(gemm_launch(m->p_r, nullptr, m->d_status, m->st, nullptr, true));
+  MCK(launch_k(moe_route_kernel, dim3((m->B + 7) / 8), dim3(256), 0, m->st, true, m->p_r.out(), m->B, E, s.n_shared,
+               s.top_k, m->w, experts, probs));
+  MCK(gemm_launch(m->p_gu, nullptr, m->d_status, m->st, nullptr, true));
+  MCK(launch_k(moe_swiglu_kernel, dim3((NB * (F / 4) + 255) / 256, m->B), dim3(256), 0, m->st, true, m->p_gu.out(),
+               (const float *)m->w, F, NB, m->h_hi, m->h_lo));
+  MCK(gemm_launch(m->p_d, nullptr, m->d_status, m->st, nullptr, true));
+  MCK(launch_k(moe_readout_kernel, dim3((H / 4 + 255) / 256, m->B), dim3(256), 0, m->st, true, m->p_d.out(), H, y));
+  return CORUN_OK;
+}
+
+int corun_moe_sync(corun_moe *m) {
+  if (!m) return CORUN_EINVAL;
+  int hs = 0;
+  MCK(cudaMemcpyAsync(&hs, m->d_status, sizeof(int), cudaMemcpyDeviceToHost, m->st));
+  MCK(cudaStreamSynchronize(m->st));
+  return hs ? CORUN_ETIMEOUT : CORUN_OK;
+}
+
+int64_t corun_moe_weight_bytes(const corun_moe *m) { return m ? m->weight_bytes : 0; }
+
+int corun_moe_launches(const corun_moe *m) { return m ? 7 : CORUN_EINVAL; }
+
+}  // extern "C"
