@@ -35,7 +35,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmHi,
                     const __grid_constant__ CUtensorMap tmLo, float *__restrict__ direct, float *__restrict__ ws,
                     const int *__restrict__ cta_start, int N, int KB, int BN, int R, int stages, int tmem_cols,
-                    uint32_t idesc, int *status, unsigned long long *trace) {
+                    uint32_t idesc, const float *row_keep, int keep_pitch, int keep_div, int *status,
+                    unsigned long long *trace) {
   extern __shared__ uint8_t smem_raw[];
   // optional per-CTA timeline (debug): 8 globaltimer stamps
 #define TRACE(i) do { if (trace) trace[(size_t)blockIdx.x * 8 + (i)] = globaltimer_ns(); } while (0)
@@ -199,6 +200,8 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       tc_fence_after();
       if (g + (kb_end - kb_begin) >= k1 && threadIdx.x == 64) TRACE(6);   // last accumulator is ready
       const int n0 = tile * GEMM_TILE_N;
+      // optional: rows whose entry for this tile's column group is zero are not stored (nobody reads them)
+      const float *keep = row_keep ? row_keep + tile / keep_div : nullptr;
       if (stacked) {
         // lanes 0-63 (warps with lane_base 0, 32) hold W*hi of rows 0-63, lanes 64-127 hold W*lo of the
         // same rows: every warp parks 32 columns of its rows in shared memory, then the 128 threads add
@@ -227,7 +230,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int r = i * 16 + srow;
-            if (r < rows_valid) {
+            if (r < rows_valid && (!keep || r >= R || keep[(size_t)r * keep_pitch] != 0.f)) {
               const float *h = xch[0] + r * 33 + scol, *l = xch[1] + r * 33 + scol;
               const float4 f = make_float4(h[0] + l[0], h[1] + l[1], h[2] + l[2], h[3] + l[3]);
               float *d = dst0 + (size_t)r * pitch + c0 + scol;
@@ -250,7 +253,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const int rows_valid = whole ? R : BN;      // partials keep the padded row count
         if (row_base >= rows_valid) continue;        // warp-uniform: nothing of this warp's lanes is needed
         const int row = row_base + lane;
-        const bool row_ok = row < rows_valid;
+        const bool row_ok = row < rows_valid && (!keep || row >= R || keep[(size_t)row * keep_pitch] != 0.f);
         float *dst = whole ? direct + (size_t)row * N + n0
                            : ws + ((size_t)(cta * 2 + (seg == 0 ? 0 : 1)) * BN + row) * GEMM_TILE_N;
         const bool vec_ok = whole ? ((N & 3) == 0) : true;
@@ -432,7 +435,7 @@ cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int 
                         unsigned long long *trace, bool pdl) {
   return launch_k(gemm_streamk_kernel, dim3(p.grid), dim3(GEMM_THREADS), p.smem_bytes, st, pdl,
                   tmW_override ? *tmW_override : p.tmW, p.tmHi, p.tmLo, p.direct, p.ws, p.d_cta_start, p.N, p.KB, p.BN,
-                  p.R, p.stages, p.tmem_cols, p.idesc, d_status, trace);
+                  p.R, p.stages, p.tmem_cols, p.idesc, p.row_keep, p.keep_pitch, p.keep_div, d_status, trace);
 }
 
 cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st, bool pdl) {

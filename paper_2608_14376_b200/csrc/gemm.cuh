@@ -82,6 +82,10 @@ struct GemmPlan {
   int *d_cta_start = nullptr, *d_tile_first = nullptr, *d_tile_cend = nullptr;  // owned (one allocation)
   int *d_split_tiles = nullptr;      // tiles with partials (same allocation)
   int n_split_tiles = 0;
+  // Optional store mask (device, not owned): row r of weight tile t is stored only if
+  // row_keep[r * keep_pitch + t / keep_div] != 0 (rows that no consumer will read are skipped).
+  const float *row_keep = nullptr;
+  int keep_pitch = 0, keep_div = 1;
   GemmOut out() const { return GemmOut{direct, ws, d_tile_first, d_tile_cend, N, KB, BN}; }
 };
 

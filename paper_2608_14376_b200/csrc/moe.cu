@@ -201,6 +201,11 @@ int corun_moe_create(const corun_moe_shape *shape, const void *router, const voi
       (rc = gemm_plan_create(&m->p_gu, gate_up, (int)N1, H, m->x_hi, m->x_lo, B, m->BN, m->out_gu, m->ws, m->num_sms)) ||
       (rc = gemm_plan_create(&m->p_d, down, H, (int)K2, m->h_hi, m->h_lo, B, m->BN, m->out_d, m->ws, m->num_sms)))
     return fail(rc);
+  if ((2 * F) % GEMM_TILE_N == 0) {                 // a weight tile then belongs to one expert: skip the rows that
+    m->p_gu.row_keep = m->w;                        // did not select it (the SwiGLU kernel does not read them)
+    m->p_gu.keep_pitch = NB;
+    m->p_gu.keep_div = 2 * F / GEMM_TILE_N;
+  }
   m->weight_bytes = ((int64_t)E * H + (int64_t)N1 * H + (int64_t)H * K2) * 2;
   if (cudaDeviceSynchronize() != cudaSuccess) return fail(CORUN_ECUDA);
   *out = m;

@@ -33,7 +33,8 @@ def _device_op(corun, torch, w, H, E, K, F, S, B):
     return corun.MoeFfn(H, E, K, F, S, t(w["router"]), t(gate_up), t(down), B)
 
 
-@pytest.mark.parametrize("H,E,K,F,S,B", [(256, 8, 2, 128, 1, 16), (512, 64, 6, 192, 2, 40), (128, 5, 5, 64, 0, 3)])
+@pytest.mark.parametrize("H,E,K,F,S,B", [(256, 8, 2, 128, 1, 16), (512, 64, 6, 192, 2, 40), (128, 5, 5, 64, 0, 3),
+                                           (256, 16, 4, 128, 1, 100)])
 def test_moe_matches_oracle_and_is_position_invariant(H, E, K, F, S, B):
     torch = pytest.importorskip("torch")
     if not torch.cuda.is_available():
