@@ -31,6 +31,9 @@ constexpr uint32_t A_BLOCK_BYTES = GEMM_ROW_BLOCK * GEMM_BLOCK_K * 2;      // 16
 // per block of 128 activation rows.  When fewer than 128 rows are loaded the
 // MMA still reads 128 rows of shared memory; the extra accumulator lanes hold
 // meaningless values that are never read back.
+// MASKED: the optional store mask of the epilogue (a separate instantiation, so that the plain kernel is
+// exactly the code it was without it).
+template <bool MASKED>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmHi,
                     const __grid_constant__ CUtensorMap tmLo, float *__restrict__ direct, float *__restrict__ ws,
@@ -201,7 +204,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       if (g + (kb_end - kb_begin) >= k1 && threadIdx.x == 64) TRACE(6);   // last accumulator is ready
       const int n0 = tile * GEMM_TILE_N;
       // optional: rows whose entry for this tile's column group is zero are not stored (nobody reads them)
-      const float *keep = row_keep ? row_keep + tile / keep_div : nullptr;
+      const float *keep = MASKED ? row_keep + tile / keep_div : nullptr;
       if (stacked) {
         // lanes 0-63 (warps with lane_base 0, 32) hold W*hi of rows 0-63, lanes 64-127 hold W*lo of the
         // same rows: every warp parks 32 columns of its rows in shared memory, then the 128 threads add
@@ -230,7 +233,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int r = i * 16 + srow;
-            if (r < rows_valid && (!keep || r >= R || keep[(size_t)r * keep_pitch] != 0.f)) {
+            if (r < rows_valid && (!MASKED || r >= R || keep[(size_t)r * keep_pitch] != 0.f)) {
               const float *h = xch[0] + r * 33 + scol, *l = xch[1] + r * 33 + scol;
               const float4 f = make_float4(h[0] + l[0], h[1] + l[1], h[2] + l[2], h[3] + l[3]);
               float *d = dst0 + (size_t)r * pitch + c0 + scol;
@@ -253,7 +256,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const int rows_valid = whole ? R : BN;      // partials keep the padded row count
         if (row_base >= rows_valid) continue;        // warp-uniform: nothing of this warp's lanes is needed
         const int row = row_base + lane;
-        const bool row_ok = row < rows_valid && (!keep || row >= R || keep[(size_t)row * keep_pitch] != 0.f);
+        const bool row_ok = row < rows_valid && (!MASKED || row >= R || keep[(size_t)row * keep_pitch] != 0.f);
         float *dst = whole ? direct + (size_t)row * N + n0
                            : ws + ((size_t)(cta * 2 + (seg == 0 ? 0 : 1)) * BN + row) * GEMM_TILE_N;
         const bool vec_ok = whole ? ((N & 3) == 0) : true;
@@ -423,7 +426,9 @@ int gemm_plan_create(GemmPlan *p, const void *W, int N, int K, const void *Xhi, 
 }
 
 cudaError_t gemm_prepare_kernel() {
-  return cudaFuncSetAttribute(gemm_streamk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  cudaError_t e = cudaFuncSetAttribute(gemm_streamk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(gemm_streamk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
 }
 
 void gemm_plan_destroy(GemmPlan *p) {
@@ -433,9 +438,13 @@ void gemm_plan_destroy(GemmPlan *p) {
 
 cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int *d_status, cudaStream_t st,
                         unsigned long long *trace, bool pdl) {
-  return launch_k(gemm_streamk_kernel, dim3(p.grid), dim3(GEMM_THREADS), p.smem_bytes, st, pdl,
+  if (p.row_keep)
+    return launch_k(gemm_streamk_kernel<true>, dim3(p.grid), dim3(GEMM_THREADS), p.smem_bytes, st, pdl,
+                    tmW_override ? *tmW_override : p.tmW, p.tmHi, p.tmLo, p.direct, p.ws, p.d_cta_start, p.N, p.KB, p.BN,
+                    p.R, p.stages, p.tmem_cols, p.idesc, p.row_keep, p.keep_pitch, p.keep_div, d_status, trace);
+  return launch_k(gemm_streamk_kernel<false>, dim3(p.grid), dim3(GEMM_THREADS), p.smem_bytes, st, pdl,
                   tmW_override ? *tmW_override : p.tmW, p.tmHi, p.tmLo, p.direct, p.ws, p.d_cta_start, p.N, p.KB, p.BN,
-                  p.R, p.stages, p.tmem_cols, p.idesc, p.row_keep, p.keep_pitch, p.keep_div, d_status, trace);
+                  p.R, p.stages, p.tmem_cols, p.idesc, (const float *)nullptr, 0, 1, d_status, trace);
 }
 
 cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st, bool pdl) {
