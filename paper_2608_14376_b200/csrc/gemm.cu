@@ -33,7 +33,7 @@ constexpr uint32_t A_BLOCK_BYTES = GEMM_ROW_BLOCK * GEMM_BLOCK_K * 2;      // 16
 // meaningless values that are never read back.
 // MASKED: the optional store mask of the epilogue (a separate instantiation, so that the plain kernel is
 // exactly the code it was without it).
-template <bool MASKED>
+template <bool MASKED, bool STACKED>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmHi,
                     const __grid_constant__ CUtensorMap tmLo, float *__restrict__ direct, float *__restrict__ ws,
@@ -59,7 +59,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   const uint32_t x_bytes = (uint32_t)BN * GEMM_BLOCK_K * 2;         // BN * 128 B
   // Up to 64 rows: hi and lo share one 128-row A tile (hi in rows 0.., lo in rows 64..), so one MMA
   // per k-slice yields W*hi in accumulator lanes 0-63 and W*lo in lanes 64-127; the epilogue adds them.
-  const bool stacked = BN <= 64;
+  constexpr bool stacked = STACKED;                 // = (BN <= 64), fixed at compile time
   const uint32_t lo_off = stacked ? (uint32_t)(64 * GEMM_BLOCK_K * 2) : x_bytes;
   const uint32_t stage_bytes = W_TILE_BYTES + (stacked ? A_BLOCK_BYTES : 2 * x_bytes);
   const uint32_t tx_bytes = W_TILE_BYTES + 2 * x_bytes;
@@ -426,9 +426,11 @@ int gemm_plan_create(GemmPlan *p, const void *W, int N, int K, const void *Xhi, 
 }
 
 cudaError_t gemm_prepare_kernel() {
-  cudaError_t e = cudaFuncSetAttribute(gemm_streamk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(gemm_streamk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  cudaError_t e = cudaFuncSetAttribute(gemm_streamk_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  return e;
 }
 
 void gemm_plan_destroy(GemmPlan *p) {
@@ -438,13 +440,14 @@ void gemm_plan_destroy(GemmPlan *p) {
 
 cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int *d_status, cudaStream_t st,
                         unsigned long long *trace, bool pdl) {
-  if (p.row_keep)
-    return launch_k(gemm_streamk_kernel<true>, dim3(p.grid), dim3(GEMM_THREADS), p.smem_bytes, st, pdl,
-                    tmW_override ? *tmW_override : p.tmW, p.tmHi, p.tmLo, p.direct, p.ws, p.d_cta_start, p.N, p.KB, p.BN,
-                    p.R, p.stages, p.tmem_cols, p.idesc, p.row_keep, p.keep_pitch, p.keep_div, d_status, trace);
-  return launch_k(gemm_streamk_kernel<false>, dim3(p.grid), dim3(GEMM_THREADS), p.smem_bytes, st, pdl,
-                  tmW_override ? *tmW_override : p.tmW, p.tmHi, p.tmLo, p.direct, p.ws, p.d_cta_start, p.N, p.KB, p.BN,
-                  p.R, p.stages, p.tmem_cols, p.idesc, (const float *)nullptr, 0, 1, d_status, trace);
+  const bool masked = p.row_keep != nullptr, stacked = p.BN <= 64;
+  auto go = [&](auto kernel) {
+    return launch_k(kernel, dim3(p.grid), dim3(GEMM_THREADS), p.smem_bytes, st, pdl, tmW_override ? *tmW_override : p.tmW,
+                    p.tmHi, p.tmLo, p.direct, p.ws, p.d_cta_start, p.N, p.KB, p.BN, p.R, p.stages, p.tmem_cols, p.idesc,
+                    p.row_keep, p.keep_pitch, p.keep_div, d_status, trace);
+  };
+  if (masked) return stacked ? go(gemm_streamk_kernel<true, true>) : go(gemm_streamk_kernel<true, false>);
+  return stacked ? go(gemm_streamk_kernel<false, true>) : go(gemm_streamk_kernel<false, false>);
 }
 
 cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st, bool pdl) {
