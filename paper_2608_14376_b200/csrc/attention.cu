@@ -171,7 +171,9 @@ struct AttLayout {
   static constexpr size_t SMEM = (size_t)ATT_NBUF * ITEM_BYTES + ATT_GROUPS * GROUP_BYTES + PAD_BYTES + 1024;
 };
 
-template <int HD, int GROUP>
+// WHOLE_PAIRS: the ablation that hands out whole (row, kv head) pairs (a separate instantiation, so that the
+// kernel of the product is exactly the code it is without it).
+template <int HD, int GROUP, bool WHOLE_PAIRS>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                   const float *__restrict__ q, Rows rows, int nq, KvLayout kv, int max_splits,
@@ -189,7 +191,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   const int n_total = *n_work;
   if (n_total <= 0) return;
   // this CTA's stretch of the item list, and where the shared pool begins
-  const int n_pairs = n_work[1];                 // > 0: the ablation that hands out whole (row, kv head) pairs (see item_of)
+  const int n_pairs = WHOLE_PAIRS ? n_work[1] : 0;   // > 0: the ablation that hands out whole (row, kv head) pairs (see item_of)
   const int n_fixed = n_pairs > 0 ? 0 : (int)(((long long)n_total * 15 / 16) / gridDim.x);
   const int item_lo = (int)blockIdx.x * n_fixed, pool_lo = (int)gridDim.x * n_fixed;
 
@@ -247,7 +249,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   int pair_j = -1, pair_c = 0;
   int wp_base = 0, wp_ns = 0, wp_start = 0;
   auto item_of = [&](int k, bool draw) -> int {
-    if (n_pairs > 0) {
+    if (WHOLE_PAIRS && n_pairs > 0) {
       while (wp_start >= 0 && k >= wp_base + wp_ns) {
         wp_base += wp_ns;
         ++pair_j;
@@ -683,18 +685,24 @@ __global__ void __launch_bounds__(256) attn_worklist_kernel(Rows rows, int n_kv,
 namespace {
 template <int HD, int GROUP>
 cudaError_t prepare_one() {
-  return cudaFuncSetAttribute(attn_split_kernel<HD, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<HD, GROUP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)AttLayout<HD>::SMEM);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attn_split_kernel<HD, GROUP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)AttLayout<HD>::SMEM);
 }
 template <int HD>
 cudaError_t launch_attn_split(int group, int grid, cudaStream_t st, const CUtensorMap &tmK, const CUtensorMap &tmV,
                          const float *q, const Rows &rows, int nq, const KvLayout &kv, int max_splits, const int *work,
                          const int *n_work, float *part_acc, float *part_ml, int *done_count, int *pool_count,
-                         __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int reuse, int *d_status,
+                         __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int reuse, int whole_pairs, int *d_status,
                          unsigned long long *trace) {
 #define CORUN_ATT_CASE(G)                                                                                          \
   case G:                                                                                                          \
-    return launch_k(attn_split_kernel<HD, G>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
+    if (whole_pairs)                                                                                               \
+      return launch_k(attn_split_kernel<HD, G, true>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
+                      rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, reuse, d_status, trace); \
+    return launch_k(attn_split_kernel<HD, G, false>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
                     rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, reuse, d_status, trace);
   switch (group) {
     CORUN_ATT_CASE(1)
@@ -735,16 +743,17 @@ cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, con
   (void)layer;   // the tensor maps are the layer's
   const int group = nq / kv.n_kv;
   if (group * kv.n_kv != nq || max_splits > 256) return cudaErrorInvalidValue;
-  if (reuse)   // a prefill chunk: consecutive tokens of one request
+  if (reuse == 1)   // a prefill chunk: consecutive tokens of one request
     return launch_attention_prefill(tmK, tmV, q, rows, nq, kv, out_hi, out_lo, d_status, st);
+  const int whole_pairs = reuse == 2;   // the ablation: the item list carries the pair table
   const long long most = (long long)rows.R * max_splits * kv.n_kv;
   const int grid = (int)(most < grid_ctas ? most : grid_ctas);
   if (kv.hd == 128)
     return launch_attn_split<128>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml,
-                                  done_count, pool_count, out_hi, out_lo, reuse, d_status, trace);
+                                  done_count, pool_count, out_hi, out_lo, 0, whole_pairs, d_status, trace);
   if (kv.hd == 64)
     return launch_attn_split<64>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml,
-                                 done_count, pool_count, out_hi, out_lo, reuse, d_status, trace);
+                                 done_count, pool_count, out_hi, out_lo, 0, whole_pairs, d_status, trace);
   return cudaErrorInvalidValue;
 }
 

@@ -208,7 +208,7 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
     STAGE(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, tr(4 * l + 0), true));
     STAGE(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st));
     STAGE(launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work, P.att_n_work,
-                           e->num_sms, P.part_acc, P.part_ml, P.att_done, P.att_pool + l, P.ao_hi, P.ao_lo, &P == &e->dec ? 0 : 1,
+                           e->num_sms, P.part_acc, P.part_ml, P.att_done, P.att_pool + l, P.ao_hi, P.ao_lo, &P == &e->dec ? (e->whole_pairs ? 2 : 0) : 1,
                            e->d_status, e->st));
     STAGE(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st, tr(4 * l + 1), true));
     GemmOut o = P.p_o.out();
@@ -845,7 +845,7 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
                 if (ce == cudaSuccess)
                   ce = launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work,
                                         P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_done, P.att_pool + l,
-                                        P.ao_hi, P.ao_lo, 0, e->d_status, e->st);
+                                        P.ao_hi, P.ao_lo, e->whole_pairs ? 2 : 0, e->d_status, e->st);
                 break;
         case 6: ce = launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->attn_norm[l], s.rms_eps, P.xn_hi,
                                        P.xn_lo, e->st); break;
@@ -905,7 +905,7 @@ int corun_debug_attn_trace(corun_engine *e, int32_t layer, uint64_t *stamps, int
     if (ce == cudaSuccess)
       ce = launch_attention(e->tm_k[layer], e->tm_v[layer], P.q, rows, s.n_q_heads, kv_layout(e), layer, e->max_splits,
                             P.att_work, P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_done, P.att_pool + layer,
-                            P.ao_hi, P.ao_lo, 0, e->d_status, e->st, i == 1 ? d : nullptr);   // only the second launch is recorded
+                            P.ao_hi, P.ao_lo, e->whole_pairs ? 2 : 0, e->d_status, e->st, i == 1 ? d : nullptr);   // only the second launch is recorded
   }
   if (ce == cudaSuccess) ce = cudaMemcpyAsync(stamps, d, n * sizeof(unsigned long long), cudaMemcpyDeviceToHost, e->st);
   if (ce == cudaSuccess) ce = cudaStreamSynchronize(e->st);

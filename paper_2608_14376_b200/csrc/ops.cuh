@@ -63,8 +63,9 @@ cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *
 // Split-KV paged attention partials and their fixed-order combine -> bf16 hi/lo [R, nq*hd] (rows that are
 // not active keep what they held).  done_count: [R * n_kv] ints, zero before the first launch (the kernel
 // leaves them zero).  pool_count: one int, zero before the launch (not reset by it): the items beyond the
-// CTAs' fixed stretches are drawn through it.  reuse: nonzero when the rows are the
-// consecutive tokens of one request in one slot (a prefill chunk): launch_attention_prefill runs instead.
+// CTAs' fixed stretches are drawn through it.  reuse: 1 when the rows are the consecutive tokens of one
+// request in one slot (a prefill chunk): launch_attention_prefill runs instead; 2 for the ablation in which a
+// CTA takes whole (row, kv head) pairs (the work list then carries the pair table); else 0.
 // tmK / tmV: tensor maps over this layer's pages: keys as rows of hd halfs with a [16, 64] box (128-byte
 // swizzle), values as rows of 16 halfs with an [hd, 16] box (32-byte swizzle); see attention.cu.
 // work / n_work: the step's (row, kv head, split) items from launch_attn_worklist (the same for every layer);
