@@ -173,7 +173,8 @@ struct AttLayout {
 
 // WHOLE_PAIRS: the ablation that hands out whole (row, kv head) pairs (a separate instantiation, so that the
 // kernel of the product is exactly the code it is without it).
-template <int HD, int GROUP, bool WHOLE_PAIRS>
+// TRACED: the per-item globaltimer stamps (debug), likewise.
+template <int HD, int GROUP, bool WHOLE_PAIRS, bool TRACED>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                   const float *__restrict__ q, Rows rows, int nq, KvLayout kv, int max_splits,
@@ -183,7 +184,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                   unsigned long long *trace) {
   using L = AttLayout<HD>;
   // optional timeline (debug): per CTA and item (first 64): [key load issued, keys landed, group starts, released, scores done, weights written, values landed, output done]
-#define ATRACE(k, i) do { if (trace && (k) < 64) trace[((size_t)blockIdx.x * 64 + (k)) * 8 + (i)] = globaltimer_ns(); } while (0)
+#define ATRACE(k, i) do { if (TRACED && trace && (k) < 64) trace[((size_t)blockIdx.x * 64 + (k)) * 8 + (i)] = globaltimer_ns(); } while (0)
   constexpr int KSTEPS = HD / 16;
   griddep_launch_dependents();
   griddep_wait();                                // the item list and q come from earlier kernels
@@ -300,7 +301,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     const bool is_v = warp == 1;
     // decode streams the cache once per step; the rows of a prefill chunk belong to one request and read the
     // same keys and values one after the other, so there they are kept in L2
-    const uint64_t pol = reuse ? l2_policy_evict_last() : l2_policy_evict_first();
+    const uint64_t pol = l2_policy_evict_first();
     uint64_t *full = is_v ? vfull_bar : kfull_bar, *empty = is_v ? vempty_bar : kempty_bar;
     for (int k = 0;; ++k) {
       const int item = item_of(k, !is_v);
@@ -685,11 +686,15 @@ __global__ void __launch_bounds__(256) attn_worklist_kernel(Rows rows, int n_kv,
 namespace {
 template <int HD, int GROUP>
 cudaError_t prepare_one() {
-  cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<HD, GROUP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<HD, GROUP, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)AttLayout<HD>::SMEM);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(attn_split_kernel<HD, GROUP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)AttLayout<HD>::SMEM);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(attn_split_kernel<HD, GROUP, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)AttLayout<HD>::SMEM);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(attn_split_kernel<HD, GROUP, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)AttLayout<HD>::SMEM);
+  return e;
 }
 template <int HD>
 cudaError_t launch_attn_split(int group, int grid, cudaStream_t st, const CUtensorMap &tmK, const CUtensorMap &tmV,
@@ -700,9 +705,12 @@ cudaError_t launch_attn_split(int group, int grid, cudaStream_t st, const CUtens
 #define CORUN_ATT_CASE(G)                                                                                          \
   case G:                                                                                                          \
     if (whole_pairs)                                                                                               \
-      return launch_k(attn_split_kernel<HD, G, true>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
+      return launch_k(attn_split_kernel<HD, G, true, false>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
                       rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, reuse, d_status, trace); \
-    return launch_k(attn_split_kernel<HD, G, false>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
+    if (trace)                                                                                                     \
+      return launch_k(attn_split_kernel<HD, G, false, true>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
+                      rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, reuse, d_status, trace); \
+    return launch_k(attn_split_kernel<HD, G, false, false>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
                     rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, reuse, d_status, trace);
   switch (group) {
     CORUN_ATT_CASE(1)
