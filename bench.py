@@ -314,6 +314,32 @@ def run_corun(args, rank, world):
                    "note": "executed MMA work counted (activations are a bf16 hi/lo pair: two MMAs per weight tile) at "
                            "%.0f TFLOP/s sustained; attention not counted" % tf_s}
 
+    # ---- the Mixture-of-Experts feed-forward block (DeepSeek-V2-Lite block shape, B = 128 padded rows): time per
+    # call with CUDA events against the bytes of expert weights a call streams (rank 0, full-size workload only)
+    moe = None
+    if rank == 0 and sh.n_layers > 8:
+        from paper_2608_14376_b200.corun import MoeFfn
+        gm = torch.Generator(device="cuda").manual_seed(3)
+        mk = lambda *shape: (torch.randn(shape, generator=gm, device="cuda") * 0.02).to(torch.bfloat16).contiguous()
+        mH, mE, mK, mF, mS, mB = 2048, 64, 6, 1408, 2, 128
+        op = MoeFfn(mH, mE, mK, mF, mS, mk(mE, mH), mk((mE + mS) * 2 * mF, mH), mk(mH, (mE + mS) * mF), mB)
+        xm = torch.randn((mB, mH), generator=gm, device="cuda")
+        for _ in range(3):
+            op.forward(xm, want_routing=False)
+        op.sync()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(20):
+            op.forward(xm, want_routing=False)
+        e1.record()
+        op.sync()
+        mms = e0.elapsed_time(e1) / 20
+        moe = {"workload": "deepseek_v2_lite_moe_block_b128", "us_per_call": mms * 1e3, "weight_bytes": op.weight_bytes(),
+               "GBs": op.weight_bytes() / mms / 1e6, "frac_of_measured_hbm": op.weight_bytes() / mms / 1e6 / hbm,
+               "launches_per_call": op.launches()}
+        op.close()
+        del op, xm
+
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:
         w_np = synth.weights_torch_to_numpy(w_t)
@@ -346,7 +372,8 @@ def run_corun(args, rank, world):
         "clocks": clk, "gpu_launches": launches * K,
         "e2e": {"value": e2e_val, "unit": "tok/s", "ms_per_step": 1e3 * e2e_s / K,
                 "h2d_bytes_per_step": B * 9, "d2h_bytes_per_step": B * 4 + 4},
-        "roofline": roofline, "step_roofline": step_roof, "kernels": kernels, "prefill": prefill, "cpu_baseline": cpu,
+        "roofline": roofline, "step_roofline": step_roof, "kernels": kernels, "prefill": prefill, "moe_ffn": moe,
+        "cpu_baseline": cpu,
     }))
 
 
