@@ -124,3 +124,34 @@ def test_long_context_decode_parity_and_invariance(orc, qwen):
     assert eng.logits(slot2).tobytes() == rows[20]
     assert toks2[slot2] == toks[20]
     eng.release(slot2)
+
+
+def test_batched_prefill_equals_isolated_prefill_at_full_size(qwen):
+    """Prompts sharing prefill chunks (pieces on 32-token query-tile boundaries, one prompt cut across two
+    chunks) against isolated prefill of each: first tokens, logits and two sampled decode steps, byte for byte."""
+    sh, model, eng = qwen
+    lens = [40, 100, 7, 300, 129]
+    slots = [9, 33, 2, 60, 17]
+    prompts = synth.make_prompts(sh.vocab, lens, seed=123)
+    seeds = np.array([synth.request_seed(100 + i) for i in range(len(lens))], np.uint64)
+    res = [n + 8 for n in lens]
+
+    def after():
+        active = np.zeros(B, np.uint8); active[slots] = 1
+        sd = np.zeros(B, np.uint64); sd[slots] = seeds
+        out = [b"".join(eng.logits(s).tobytes() for s in slots)]
+        for _ in range(2):
+            out.append(eng.decode_step(active, sd).tobytes())
+            out.append(b"".join(eng.logits(s).tobytes() for s in slots))
+        return out
+
+    first_iso = [eng.prefill(s, p, r, T, P, seed=int(sd)) for s, p, r, sd in zip(slots, prompts, res, seeds)]
+    iso = after()
+    for s in slots:
+        eng.release(s)
+    first_bat = list(eng.prefill_batch(slots, prompts, res, T, P, seeds))
+    bat = after()
+    for s in slots:
+        eng.release(s)
+    assert first_bat == first_iso
+    assert bat == iso
