@@ -180,7 +180,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                   const float *__restrict__ q, Rows rows, int nq, KvLayout kv, int max_splits,
                   const int *__restrict__ work, const int *__restrict__ n_work, float *__restrict__ part_acc,
                   float *__restrict__ part_ml, int *__restrict__ done_count, int *__restrict__ pool_count,
-                  __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo, int reuse, int *status,
+                  __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo, int *status,
                   unsigned long long *trace) {
   using L = AttLayout<HD>;
   // optional timeline (debug): per CTA and item (first 64): [key load issued, keys landed, group starts, released, scores done, weights written, values landed, output done]
@@ -299,8 +299,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   if (warp < 2) {
     // ---------------- producers: warp 0 keys, warp 1 values; one lane per page ----------------
     const bool is_v = warp == 1;
-    // decode streams the cache once per step; the rows of a prefill chunk belong to one request and read the
-    // same keys and values one after the other, so there they are kept in L2
+    // decode streams the cache once per step: nothing of it is worth keeping in L2
     const uint64_t pol = l2_policy_evict_first();
     uint64_t *full = is_v ? vfull_bar : kfull_bar, *empty = is_v ? vempty_bar : kempty_bar;
     for (int k = 0;; ++k) {
@@ -700,18 +699,18 @@ template <int HD>
 cudaError_t launch_attn_split(int group, int grid, cudaStream_t st, const CUtensorMap &tmK, const CUtensorMap &tmV,
                          const float *q, const Rows &rows, int nq, const KvLayout &kv, int max_splits, const int *work,
                          const int *n_work, float *part_acc, float *part_ml, int *done_count, int *pool_count,
-                         __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int reuse, int whole_pairs, int *d_status,
+                         __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int whole_pairs, int *d_status,
                          unsigned long long *trace) {
 #define CORUN_ATT_CASE(G)                                                                                          \
   case G:                                                                                                          \
     if (whole_pairs)                                                                                               \
       return launch_k(attn_split_kernel<HD, G, true, false>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
-                      rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, reuse, d_status, trace); \
+                      rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, d_status, trace); \
     if (trace)                                                                                                     \
       return launch_k(attn_split_kernel<HD, G, false, true>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
-                      rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, reuse, d_status, trace); \
+                      rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, d_status, trace); \
     return launch_k(attn_split_kernel<HD, G, false, false>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
-                    rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, reuse, d_status, trace);
+                    rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, d_status, trace);
   switch (group) {
     CORUN_ATT_CASE(1)
     CORUN_ATT_CASE(2)
@@ -758,10 +757,10 @@ cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, con
   const int grid = (int)(most < grid_ctas ? most : grid_ctas);
   if (kv.hd == 128)
     return launch_attn_split<128>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml,
-                                  done_count, pool_count, out_hi, out_lo, 0, whole_pairs, d_status, trace);
+                                  done_count, pool_count, out_hi, out_lo, whole_pairs, d_status, trace);
   if (kv.hd == 64)
     return launch_attn_split<64>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml,
-                                 done_count, pool_count, out_hi, out_lo, 0, whole_pairs, d_status, trace);
+                                 done_count, pool_count, out_hi, out_lo, whole_pairs, d_status, trace);
   return cudaErrorInvalidValue;
 }
 
