@@ -160,6 +160,30 @@ def case_moe(a):
     t1.record()
     op.sync()
     ms = t0.elapsed_time(t1) / a.reps
+    # the same call captured once and replayed as a CUDA graph (the call allocates nothing and never touches the host)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        op_g = corun.MoeFfn(H, E, K, F, S, router, gate_up, down, a.B)     # bound to the side stream
+        yg = torch.empty_like(x)
+        corun.lib().corun_moe_forward(op_g._h, x.data_ptr(), yg.data_ptr(), None, None)
+        op_g.sync()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            corun.lib().corun_moe_forward(op_g._h, x.data_ptr(), yg.data_ptr(), None, None)
+        for _ in range(3):
+            graph.replay()
+        t0.record()
+        for _ in range(a.reps):
+            graph.replay()
+        t1.record()
+    torch.cuda.synchronize()
+    ms_g = t0.elapsed_time(t1) / a.reps
+    same = bool((yg == y).all().item())
+    op_g.close()
+    print("moe: graph replay %.1f us per call (%.0f GB/s); output identical to the direct call: %s"
+          % (ms_g * 1e3, op.weight_bytes() / ms_g / 1e6, same))
+    if not same:
+        raise SystemExit(1)
     wb = op.weight_bytes()
     hit = len(torch.unique(ex))
     print("moe: B=%d H=%d E=%d top-%d F=%d shared=%d: %.1f us per call, %.1f MB of weights -> %.0f GB/s; %d of %d experts selected; %d launches"
