@@ -258,13 +258,14 @@ def test_adopted_slot_with_written_cache_matches_oracle(orc, tiny, engine):
     assert np.abs(engine.logits(6) - want).max() <= TOL
 
 
-@pytest.mark.parametrize("n_ctx", [255, 256, 257, 700, 1023])
+@pytest.mark.parametrize("n_ctx", [255, 256, 257, 700, 1023, 8191, 8193, 9000])
 def test_multi_split_attention_matches_oracle(orc, tiny, n_ctx):
-    """Contexts spanning several 256-token splits and ragged tails (synthetic cache rows)."""
+    """Contexts spanning several 128-token splits and ragged tails (synthetic cache rows), up to more than
+    64 splits (the combine's general path)."""
     from paper_2608_14376_b200 import corun
 
     sh = tiny.sh
-    e = corun.Engine(sh, tiny.w_t, B, 1040)
+    e = corun.Engine(sh, tiny.w_t, B, 1040 if n_ctx < 1024 else 9216)
     cache = tiny.oracle.new_cache(n_ctx + 2)
     e.adopt(2, 0, n_ctx + 2, pending=33)
     for layer in range(sh.n_layers):
