@@ -412,3 +412,28 @@ def test_batched_prefill_equals_isolated_prefill(tiny):
     assert ei.value.status == corun.ENOSPACE and small.free_blocks() == 12
     assert list(small.prefill_batch([0], prompts[1:2], [100], T, P_, seeds[1:2])) == [first_iso[1]]
     small.close()
+
+
+@pytest.mark.parametrize("n", [129, 1100, 1793])
+def test_long_prompt_prefill_matches_oracle(orc, tiny, n):
+    """Prompts of 2, 9 and 15 key blocks of 128 tokens (odd and even counts for the two CTAs of a tile's
+    cluster, several chunks): last-position logits and the cache against the oracle, then one decode step."""
+    from paper_2608_14376_b200 import corun
+
+    prompt = synth.make_prompts(tiny.sh.vocab, [n], seed=500 + n)[0]
+    r = orc.Request(tiny.oracle, prompt, 1, max_T=n + 8)
+    r.prefill()
+    e = corun.Engine(tiny.sh, tiny.w_t, B, n + 8)
+    e.prefill(4, prompt, n + 4)
+    assert np.abs(e.logits(4) - r.logits).max() <= TOL
+    for layer in range(tiny.sh.n_layers):
+        k, v = e.kv_read(4, layer, 0, n)
+        np.testing.assert_allclose(k, r.cache[0][layer, :n], atol=2e-3, rtol=2e-3)
+        np.testing.assert_allclose(v, r.cache[1][layer, :n], atol=2e-3, rtol=2e-3)
+    tok = int(np.argmax(r.logits))
+    e.force_token(4, tok)
+    active = np.zeros(B, np.uint8); active[4] = 1
+    e.decode_step(active, np.zeros(B, np.uint64))
+    r.decode(force_token=tok)
+    assert np.abs(e.logits(4) - r.logits).max() <= TOL
+    e.close()
