@@ -185,6 +185,9 @@ int64_t corun_free_blocks(corun_engine *e);
 /* The engine's fixed dimensions: slots, largest context, tokens per page, pages in the pool
  * (any of the out pointers may be NULL). */
 int corun_engine_info(corun_engine *e, int32_t *B, int32_t *max_context, int32_t *kv_block, int64_t *pool_blocks);
+/* How corun_prefill_batch packs prompts: rows per prefill chunk, and the row granularity on which every
+ * piece of a request starts (the query tile of the prefill attention kernel).  Either pointer may be NULL. */
+int corun_prefill_geometry(corun_engine *e, int32_t *chunk_rows, int32_t *tile_rows);
 /* Reads / writes n cached positions [pos0, pos0+n) of one layer as fp32 rows of
  * n_kv_heads*head_dim (host).  Writing beyond the current context length
  * extends it (up to reserve_len); values are rounded to the cache's fp16. */

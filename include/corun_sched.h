@@ -54,6 +54,12 @@ typedef struct {
   int64_t (*free_blocks)(void *ctx);
 } corun_sched_ops;
 
+/* Optional: several prompts in shared prefill chunks (the signature of corun_prefill_batch). */
+typedef int (*corun_sched_prefill_batch_fn)(void *ctx, int32_t n_req, const int32_t *slots, const int32_t *tokens,
+                                            const int32_t *n_tokens, const int32_t *reserve_lens,
+                                            const corun_sampling *samplings, const uint64_t *seeds,
+                                            int32_t *out_first_tokens);
+
 /* What one corun_sched_step did. */
 enum { CORUN_SCHED_IDLE = 0, CORUN_SCHED_PREFILL = 1, CORUN_SCHED_DECODE = 2 };
 
@@ -65,14 +71,31 @@ int corun_sched_create(const corun_sched_ops *ops, void *ctx, int32_t B, int32_t
 int corun_sched_create_for_engine(corun_engine *e, corun_sched **out);
 void corun_sched_destroy(corun_sched *s);
 
+/*
+ * Batched prefill, off by default (paper, Future Work, "Batch-Invariant Kernels for Prefill": prefill
+ * requests batched with each other, never with decode; an extension of Algorithms 1 and 2, not part of
+ * them).  When on, a prefill decision takes the head of `waiting` exactly as before and then, in queue
+ * order, every following request that (a) still finds a free slot, (b) fits the pool together with the
+ * ones taken before it, and (c) fits into the padding of the chunks the requests taken so far occupy
+ * anyway: a request's rows start on a multiple of tile_rows, and the number of chunks of chunk_rows rows
+ * must not grow.  It stops at the first request that fails one of the three (no request overtakes
+ * another), so the head is never delayed by more than the others' LM heads, and short prompts ride in
+ * chunks that would have been padding.  The tokens of every request are those of isolated prefill.
+ * fn NULL: the engine's corun_prefill_batch and geometry (scheduler made by _create_for_engine; chunk_rows
+ * and tile_rows are then ignored); else chunk_rows >= tile_rows >= 1, chunk_rows % tile_rows == 0.
+ * corun_sched_step reports the number of requests prefilled in *n_active and the first one's id.
+ */
+int corun_sched_enable_batched_prefill(corun_sched *s, corun_sched_prefill_batch_fn fn, int32_t chunk_rows,
+                                       int32_t tile_rows);
+
 /* Appends a request to `waiting`; the prompt is copied.  n >= 1, max_new_tokens >= 1 and
  * n + max_new_tokens <= max_context, else EINVAL.  *request_id counts up from 0 in submission order. */
 int corun_sched_submit(corun_sched *s, const int32_t *prompt, int32_t n, int32_t max_new_tokens,
                        const corun_sampling *sampling, uint64_t seed, int64_t *request_id);
 
 /* One scheduling decision (see above).  *action: CORUN_SCHED_*; *request_id: the prefilled request
- * (PREFILL) else -1; *n_active: requests that took part (1 for a prefill, the running count for a
- * decode iteration, 0 when idle).  An engine error is returned as is and leaves the queues as they
+ * (PREFILL; the first one of a batched prefill) else -1; *n_active: requests that took part (those
+ * prefilled, the running count for a decode iteration, 0 when idle).  An engine error is returned as is and leaves the queues as they
  * were before the call. */
 int corun_sched_step(corun_sched *s, int32_t *action, int64_t *request_id, int32_t *n_active);
 

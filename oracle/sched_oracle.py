@@ -155,3 +155,51 @@ class Scheduler:
             nxt = self.schedule()
             assert nxt.kind == "prefill" and nxt.requests == [rid]
             it.tokens += nxt.tokens
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Extension (not in the paper's algorithms): prefill requests batched with each other, the first direction
+# of the paper's Future Work ("Batch-Invariant Kernels for Prefill").  The rule, stated once here and
+# pinned by hand-derived traces (tests/golden/sched_batched_prefill_traces.txt):
+#   a prefill decision takes the head of `waiting` exactly as Algorithm 1 does, then, in queue order, every
+#   following request that still finds a slot, fits the pool together with those taken before it, and does
+#   not add a chunk: each request's rows start on a multiple of `tile`, and ceil(rows / chunk) must stay what
+#   it is without the request.  The first request that fails any of the three ends the batch.
+def fill_batch(waiting, n_running: int, max_num_reqs: int, free_pages: int, kv_block: int, chunk: int, tile: int):
+    """``waiting``: list of (num_prompt_tokens, max_new) in queue order, its head already admissible.
+    Returns how many requests from the front are prefilled together (>= 1)."""
+    pages = lambda r: -(-(r[0] + r[1]) // kv_block)
+    chunks = lambda rows: -(-rows // chunk)
+    taken, rows, used = 1, waiting[0][0], pages(waiting[0])
+    for r in waiting[1:]:
+        if n_running + taken >= max_num_reqs:
+            break
+        if used + pages(r) > free_pages:
+            break
+        start = -(-rows // tile) * tile
+        if chunks(start + r[0]) != chunks(rows):
+            break
+        taken, rows, used = taken + 1, start + r[0], used + pages(r)
+    return taken
+
+
+class BatchedScheduler(Scheduler):
+    """The collapsed scheduler (``decision``) with the extension: one record per batched prefill."""
+
+    def __init__(self, max_num_reqs: int, pool_pages: int, kv_block: int = 16, chunk: int = 256, tile: int = 32):
+        super().__init__(max_num_reqs, pool_pages, kv_block, chunk)
+        self.tile = tile
+
+    def decision(self) -> Iteration:
+        det = self.find_prefill_request()
+        if det is None or det in self.running:
+            return super().decision()
+        n = fill_batch([(r.num_prompt_tokens, r.max_new) for r in self.waiting], len(self.running), self.max_num_reqs,
+                       self.free_pages, self.kv_block, self.chunk, self.tile)
+        out = Iteration("prefill")
+        for _ in range(n):                                    # each taken request is admitted as Algorithm 1 admits one
+            it = super().decision()
+            assert it.kind == "prefill" and len(it.requests) == 1
+            out.requests += it.requests
+            out.tokens += it.tokens
+        return out

@@ -9,7 +9,7 @@
     python -m paper_2608_14376_b200.cases moe       [--B 128 --reps 20]      # DeepSeek-V2-Lite MoE block shape
     python -m paper_2608_14376_b200.cases ablation  [--layers 2 --B 64 --actives 1,4,16,40,64]
     python -m paper_2608_14376_b200.cases sweep     [--Bs 1,8,32,128,256 --fractions 0.125,0.5,1 --steps 10]
-    python -m paper_2608_14376_b200.cases trace     [--requests 200 --rate 4 --B 128 --replay 4]
+    python -m paper_2608_14376_b200.cases trace     [--requests 200 --rate 4 --B 128 --replay 4 --batched]
 
 ``gemm`` runs the stand-alone decode GEMM on seeded inputs; ``attention`` builds a Qwen3-8B-shaped
 engine with few layers, fills the cache of the active slots on the device and runs decode steps.
@@ -380,13 +380,15 @@ def case_trace(a):
     rng = np.random.default_rng(5)
     n = a.requests
     arrival = np.cumsum(rng.exponential(1.0 / a.rate, n))
-    plen = np.minimum(8192, np.maximum(1, np.round(np.exp(np.log(1024) + rng.standard_normal(n))))).astype(int)
-    olen = np.minimum(2048, np.maximum(2, np.round(np.exp(np.log(256) + rng.standard_normal(n))))).astype(int)
+    plen = np.minimum(8192, np.maximum(1, np.round(np.exp(np.log(a.prompt_median) + rng.standard_normal(n))))).astype(int)
+    olen = np.minimum(2048, np.maximum(2, np.round(np.exp(np.log(a.output_median) + rng.standard_normal(n))))).astype(int)
     prompts = synth.make_prompts(sh.vocab, plen, seed=6)
     eng = corun.Engine(sh, w, a.B, 10240)
     sch = corun.Scheduler(engine=eng)
+    if a.batched:
+        sch.enable_batched_prefill()
     now, nxt = 0.0, 0
-    t_first, t_done, busy_s, n_dec, n_pre, act_sum = {}, {}, 0.0, 0, 0, 0
+    t_first, t_done, busy_s, n_dec, n_pre, act_sum, n_shared = {}, {}, 0.0, 0, 0, 0, 0
     ids = []
     while len(t_done) < n:
         while nxt < n and arrival[nxt] <= now:
@@ -402,7 +404,9 @@ def case_trace(a):
         busy_s += dt
         if action == corun.SCHED_PREFILL:
             n_pre += 1
-            t_first[rid] = now
+            n_shared += n_act - 1
+            for j in range(n_act):                          # a batched prefill takes consecutive request ids
+                t_first[rid + j] = now
         else:
             n_dec += 1
             act_sum += n_act
@@ -414,8 +418,8 @@ def case_trace(a):
     total_out = int(olen.sum())
     print("trace: %d requests, %.1f req/s, prompt median %d (mean %.0f), output median %d (mean %.0f); B = %d"
           % (n, a.rate, int(np.median(plen)), plen.mean(), int(np.median(olen)), olen.mean(), a.B))
-    print("virtual makespan %.1f s (engine busy %.1f s); %d prefills, %d decode iterations, mean %.1f running per iteration"
-          % (now, busy_s, n_pre, n_dec, act_sum / max(1, n_dec)))
+    print("virtual makespan %.1f s (engine busy %.1f s); %d prefill decisions (%d requests rode along in another's chunks), "
+          "%d decode iterations, mean %.1f running per iteration" % (now, busy_s, n_pre, n_shared, n_dec, act_sum / max(1, n_dec)))
     print("output tokens/s over the makespan %.0f; over busy time %.0f" % (total_out / now, total_out / busy_s))
     print("TTFT  p50 %.3f s  p99 %.3f s;  TPOT  p50 %.2f ms  p99 %.2f ms"
           % (np.percentile(ttft, 50), np.percentile(ttft, 99), np.percentile(tpot, 50) * 1e3, np.percentile(tpot, 99) * 1e3))
@@ -476,6 +480,8 @@ def main():
     tr = sub.add_parser("trace")
     tr.add_argument("--requests", type=int, default=200); tr.add_argument("--rate", type=float, default=4.0)
     tr.add_argument("--B", type=int, default=128); tr.add_argument("--replay", type=int, default=4)
+    tr.add_argument("--batched", action="store_true", help="scheduler with batched prefill on")
+    tr.add_argument("--prompt-median", type=float, default=1024.0); tr.add_argument("--output-median", type=float, default=256.0)
     a = ap.parse_args()
     {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "prefill": case_prefill, "ablation": case_ablation, "moe": case_moe, "prefill_batch": case_prefill_batch, "sampler": case_sampler,
      "sweep": case_sweep, "trace": case_trace}[a.case](a)

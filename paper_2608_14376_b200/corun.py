@@ -24,6 +24,7 @@ EXPORTS = [
     "corun_debug_sample", "corun_gemm_static", "corun_strerror", "corun_last_cuda_error", "corun_engine_info",
     "corun_sched_create", "corun_sched_create_for_engine", "corun_sched_destroy", "corun_sched_submit",
     "corun_sched_step", "corun_sched_poll", "corun_sched_slot_of", "corun_sched_counts",
+    "corun_sched_enable_batched_prefill", "corun_prefill_geometry",
     "corun_moe_create", "corun_moe_destroy", "corun_moe_forward", "corun_moe_sync", "corun_moe_weight_bytes",
     "corun_moe_launches",
 ]
@@ -65,6 +66,9 @@ PREFILL_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C
 DECODE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.POINTER(C.c_uint8), C.POINTER(C.c_uint64), C.POINTER(C.c_int32))
 RELEASE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32)
 FREE_BLOCKS_FN = C.CFUNCTYPE(C.c_int64, C.c_void_p)
+PREFILL_BATCH_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32),
+                               C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(Sampling), C.POINTER(C.c_uint64),
+                               C.POINTER(C.c_int32))
 
 
 class SchedOps(C.Structure):
@@ -341,6 +345,15 @@ class Scheduler:
         if self._h:
             lib().corun_sched_destroy(self._h)
             self._h = None
+
+    def enable_batched_prefill(self, fn=None, chunk_rows: int = 0, tile_rows: int = 0):
+        """Prefill decisions take the requests behind the head that fit into the padding of the head's chunks
+        (``fn``: a PREFILL_BATCH_FN for a stand-in engine; None = the engine's corun_prefill_batch)."""
+        self._batch_fn = fn                                   # keep the callback alive
+        L = lib()
+        L.corun_sched_enable_batched_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32]
+        _check(L.corun_sched_enable_batched_prefill(self._h, C.cast(fn, C.c_void_p) if fn is not None else None,
+                                                    chunk_rows, tile_rows), "corun_sched_enable_batched_prefill")
 
     def submit(self, prompt, max_new_tokens: int, temperature: float = 0.0, top_p: float = 1.0, seed: int = 0) -> int:
         t = np.ascontiguousarray(prompt, dtype=np.int32)

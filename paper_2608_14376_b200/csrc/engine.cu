@@ -741,6 +741,15 @@ int corun_engine_info(corun_engine *e, int32_t *B, int32_t *max_context, int32_t
   return CORUN_OK;
 }
 
+int corun_prefill_geometry(corun_engine *e, int32_t *chunk_rows, int32_t *tile_rows) {
+  if (!e) return CORUN_EINVAL;
+  int unit = 128 / (e->sh.n_q_heads / e->sh.n_kv_heads);
+  if (unit > e->chunk || e->chunk % unit) unit = e->chunk;
+  if (chunk_rows) *chunk_rows = e->chunk;
+  if (tile_rows) *tile_rows = unit;
+  return CORUN_OK;
+}
+
 static int kv_io(corun_engine *e, int slot, int layer, int pos0, int n, float *k, float *v, int write) {
   if (!e || !k || !v || n < 0 || pos0 < 0 || layer < 0 || layer >= e->sh.n_layers) return CORUN_EINVAL;
   if (!slot_ok(e, slot) || !e->in_use[slot]) return CORUN_ESLOT;

@@ -34,6 +34,10 @@ struct corun_sched {
   std::vector<uint8_t> active;
   std::vector<uint64_t> seeds;
   std::vector<int32_t> toks;
+  // batched prefill (off unless enabled)
+  corun_sched_prefill_batch_fn prefill_batch = nullptr;
+  int32_t chunk_rows = 0, tile_rows = 0;
+  bool for_engine = false;
 };
 
 namespace {
@@ -63,6 +67,25 @@ int eng_prefill(void *c, int32_t slot, const int32_t *t, int32_t n, int32_t rese
 int eng_decode(void *c, const uint8_t *a, const uint64_t *sd, int32_t *out) { return corun_decode_step((corun_engine *)c, a, sd, out); }
 int eng_release(void *c, int32_t slot) { return corun_release((corun_engine *)c, slot); }
 int64_t eng_free(void *c) { return corun_free_blocks((corun_engine *)c); }
+int eng_prefill_batch(void *c, int32_t n, const int32_t *slots, const int32_t *t, const int32_t *nt, const int32_t *res,
+                      const corun_sampling *sp, const uint64_t *seeds, int32_t *first) {
+  return corun_prefill_batch((corun_engine *)c, n, slots, t, nt, res, sp, seeds, first);
+}
+
+// After its prefill a request runs in `slot` with its first token; it may be finished already.
+int admitted(corun_sched *s, int64_t id, int32_t slot, int32_t first) {
+  Request &r = s->reqs[(size_t)id];
+  r.slot = slot;
+  s->slot_owner[(size_t)slot] = id;
+  s->running.insert(s->running.begin(), id);   // Algorithm 2 puts the prefilled request in front of `running`
+  r.out.push_back(first);
+  if ((int32_t)r.out.size() >= r.max_new) {
+    const int rr = s->ops.release(s->ctx, slot);
+    finish(s, id);
+    return rr;
+  }
+  return CORUN_OK;
+}
 
 }  // namespace
 
@@ -91,7 +114,25 @@ extern "C" int corun_sched_create_for_engine(corun_engine *e, corun_sched **out)
   const int rc = corun_engine_info(e, &B, &max_context, &kv_block, nullptr);
   if (rc != CORUN_OK) return rc;
   const corun_sched_ops ops{eng_prefill, eng_decode, eng_release, eng_free};
-  return corun_sched_create(&ops, e, B, kv_block, max_context, out);
+  const int rc2 = corun_sched_create(&ops, e, B, kv_block, max_context, out);
+  if (rc2 == CORUN_OK) (*out)->for_engine = true;
+  return rc2;
+}
+
+extern "C" int corun_sched_enable_batched_prefill(corun_sched *s, corun_sched_prefill_batch_fn fn, int32_t chunk_rows,
+                                                  int32_t tile_rows) {
+  if (!s) return CORUN_EINVAL;
+  if (!fn) {
+    if (!s->for_engine) return CORUN_EINVAL;
+    const int rc = corun_prefill_geometry((corun_engine *)s->ctx, &chunk_rows, &tile_rows);
+    if (rc != CORUN_OK) return rc;
+    fn = eng_prefill_batch;
+  }
+  if (tile_rows < 1 || chunk_rows < tile_rows || chunk_rows % tile_rows) return CORUN_EINVAL;
+  s->prefill_batch = fn;
+  s->chunk_rows = chunk_rows;
+  s->tile_rows = tile_rows;
+  return CORUN_OK;
 }
 
 extern "C" void corun_sched_destroy(corun_sched *s) { delete s; }
@@ -124,6 +165,56 @@ extern "C" int corun_sched_step(corun_sched *s, int32_t *action, int64_t *reques
     Request &r = s->reqs[(size_t)id];
     int status = CORUN_OK;
     if (can_fit_full_sequence(s, r, &status)) {
+      if (s->prefill_batch) {
+        // ---- extension: the requests behind the head that fit into the padding of the head's chunks
+        const int64_t free_pages = s->ops.free_blocks(s->ctx);
+        if (free_pages < 0) return (int)free_pages;
+        auto pages_of = [&](const Request &q) { return ((int64_t)q.prompt.size() + q.max_new + s->kv_block - 1) / s->kv_block; };
+        auto chunks_of = [&](int64_t rows) { return (rows + s->chunk_rows - 1) / s->chunk_rows; };
+        std::vector<int64_t> ids{id};
+        int64_t rows = (int64_t)r.prompt.size(), pages = pages_of(r);
+        for (size_t w = 1; w < s->waiting.size(); ++w) {
+          const Request &q = s->reqs[(size_t)s->waiting[w]];
+          if ((int32_t)(s->running.size() + ids.size()) >= s->B) break;
+          if (pages + pages_of(q) > free_pages) break;
+          const int64_t start = (rows + s->tile_rows - 1) / s->tile_rows * s->tile_rows;
+          if (chunks_of(start + (int64_t)q.prompt.size()) != chunks_of(rows)) break;
+          ids.push_back(s->waiting[w]);
+          rows = start + (int64_t)q.prompt.size();
+          pages += pages_of(q);
+        }
+        if (ids.size() > 1) {
+          const int n = (int)ids.size();
+          std::vector<int32_t> slots, toks, lens, res, first((size_t)n, -1);
+          std::vector<corun_sampling> smp;
+          std::vector<uint64_t> seeds;
+          int32_t next = 0;
+          for (int64_t q : ids) {
+            const Request &rq = s->reqs[(size_t)q];
+            while (next < s->B && s->slot_owner[(size_t)next] >= 0) ++next;
+            if (next >= s->B) return CORUN_ESLOT;   // cannot happen: running + taken < B
+            slots.push_back(next++);
+            toks.insert(toks.end(), rq.prompt.begin(), rq.prompt.end());
+            lens.push_back((int32_t)rq.prompt.size());
+            res.push_back((int32_t)rq.prompt.size() + rq.max_new);
+            smp.push_back(rq.sampling);
+            seeds.push_back(rq.seed);
+          }
+          const int rc = s->prefill_batch(s->ctx, n, slots.data(), toks.data(), lens.data(), res.data(), smp.data(),
+                                          seeds.data(), first.data());
+          if (rc != CORUN_OK) return rc;
+          int worst = CORUN_OK;
+          for (int i = 0; i < n; ++i) {
+            s->waiting.pop_front();
+            const int rr = admitted(s, ids[(size_t)i], slots[(size_t)i], first[(size_t)i]);
+            if (rr != CORUN_OK) worst = rr;
+          }
+          *action = CORUN_SCHED_PREFILL;
+          *request_id = id;
+          *n_active = n;
+          return worst;
+        }
+      }
       // ---- Algorithm 2: the selected request is the only one the engine sees in this iteration
       int32_t slot = -1;
       for (int32_t i = 0; i < s->B; ++i)
@@ -134,19 +225,10 @@ extern "C" int corun_sched_step(corun_sched *s, int32_t *action, int64_t *reques
                                     (int32_t)r.prompt.size() + r.max_new, &r.sampling, r.seed, &first);
       if (rc != CORUN_OK) return rc;
       s->waiting.pop_front();
-      r.slot = slot;
-      s->slot_owner[(size_t)slot] = id;
-      s->running.insert(s->running.begin(), id);   // Algorithm 2 puts the prefilled request in front of `running`
-      r.out.push_back(first);
       *action = CORUN_SCHED_PREFILL;
       *request_id = id;
       *n_active = 1;
-      if ((int32_t)r.out.size() >= r.max_new) {
-        const int rr = s->ops.release(s->ctx, slot);
-        finish(s, id);
-        if (rr != CORUN_OK) return rr;
-      }
-      return CORUN_OK;
+      return admitted(s, id, slot, first);
     }
     if (status != CORUN_OK) return status;
   }

@@ -108,3 +108,44 @@ def test_served_together_equals_served_alone_and_follows_the_oracle(orc, tiny):
         assert checked >= 1
     finally:
         eng.close()
+
+
+def test_batched_prefill_policy_serves_the_same_tokens_and_follows_its_oracle(tiny):
+    """The scheduler with batched prefill on (requests behind the head ride in the padding of its chunks):
+    every request's tokens equal those under the isolated policy, bit for bit, the decisions are those of
+    the batched oracle, and some prefill decision did take several requests."""
+    from paper_2608_14376_b200 import corun
+
+    reqs = _requests()
+    eng = corun.Engine(tiny.sh, tiny.w_t, B, MAX_CTX, kv_pool_blocks=POOL)
+    try:
+        bursts = [(6, 2), (5, 3), (7, 1), (6, 4)]
+        sch = corun.Scheduler(engine=eng)
+        isolated, _ = _serve(sch, reqs, bursts)
+        sch.close()
+        sch = corun.Scheduler(engine=eng)
+        sch.enable_batched_prefill()
+        batched, log = _serve(sch, reqs, bursts)
+        sch.close()
+        assert eng.free_blocks() == POOL
+        for (a, fa), (b, fb) in zip(isolated, batched):
+            assert fa and fb
+            np.testing.assert_array_equal(a, b)
+        assert any(a == corun.SCHED_PREFILL and n > 1 for a, _, n in log)
+        chunk, tile = 256, 128 // (tiny.sh.n_q_heads // tiny.sh.n_kv_heads)
+        ref = sched_oracle.BatchedScheduler(B, POOL, 16, chunk, tile)
+        nxt, i = 0, 0
+        for k, steps in bursts + [(0, 10 ** 6)]:
+            for r in reqs[nxt:nxt + k]:
+                ref.add_request(len(r["prompt"]), r["max_new"])
+            nxt += k
+            for _ in range(steps):
+                want = ref.decision()
+                action, rid, n = log[i]; i += 1
+                assert action == {"idle": 0, "prefill": 1, "decode": 2}[want.kind]
+                assert n == len(want.requests) and (want.kind != "prefill" or rid == want.requests[0])
+                if want.kind == "idle" and nxt == len(reqs):
+                    break
+        assert i == len(log)
+    finally:
+        eng.close()

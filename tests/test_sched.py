@@ -239,3 +239,150 @@ def test_library_scheduler_argument_and_engine_errors():
         assert sch.step()[0] == corun.SCHED_DECODE and len(sch.poll(a)[0]) == 2
     finally:
         sch.close()
+
+
+# ------------------------------------------------------------------------------------------------ batched prefill
+def _batched_cases():
+    cases, cur = [], None
+    for line in open(os.path.join(ROOT, "tests", "golden", "sched_batched_prefill_traces.txt")):
+        t = line.split()
+        if not t or t[0].startswith("#"):
+            continue
+        if t[0] == "case":
+            cur = dict(name=t[1], reqs=[], its=[], **{k: int(v) for k, v in (x.split("=") for x in t[2:])})
+            cases.append(cur)
+        elif t[0] == "req":
+            cur["reqs"].append((int(t[1]), int(t[2])))
+        elif t[0] == "P":
+            cut = t.index(":")
+            cur["its"].append(("prefill", [int(x) for x in t[1:cut]], int(t[cut + 1])))
+        elif t[0] == "D":
+            cur["its"].append(("decode", [int(x) for x in t[1:]], 0))
+        elif t[0] == "I":
+            cur["its"].append(("idle", [], 0))
+    return cases
+
+
+@pytest.mark.parametrize("case", _batched_cases(), ids=lambda c: c["name"])
+def test_batched_oracle_reproduces_hand_derived_decisions(case):
+    s = sched_oracle.BatchedScheduler(case["max_num_reqs"], case["pool_pages"], case["kv_block"], case["chunk"], case["tile"])
+    for p, m in case["reqs"]:
+        s.add_request(p, m)
+    got = []
+    for _ in case["its"]:
+        it = s.decision()
+        got.append((it.kind, it.requests, it.tokens))
+    assert got == case["its"]
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_batched_rule_properties(seed):
+    """A batch is a prefix of the queue, never needs more chunks than its head alone, never more slots or
+    pages than there are; and every request is served exactly as under the isolated policy (same number of
+    tokens, nothing preempted, submission order)."""
+    B, kv_block, pool, reqs, script = _random_trace(300 + seed)
+    B, pool = B + 2, 3 * pool                                  # room for batches: at least three slots
+    chunk, tile = 256, 32
+    s = sched_oracle.BatchedScheduler(B, pool, kv_block, chunk, tile)
+    for p, m in reqs:
+        s.add_request(p, m)
+    order, decodes = [], {r: 0 for r in range(len(reqs))}
+    batches = 0
+    for _ in range(100000):
+        waiting_before = [r.rid for r in s.waiting]
+        running_before, free_before = [r.rid for r in s.running], s.free_pages
+        it = s.decision()
+        if it.kind == "idle":
+            break
+        if it.kind == "prefill":
+            n = len(it.requests)
+            batches += n > 1
+            assert it.requests == waiting_before[:n]                               # a prefix of the queue: nobody overtakes
+            assert len(running_before) + n <= B
+            assert sum(-(-sum(reqs[r]) // kv_block) for r in it.requests) <= free_before
+            rows = 0
+            for r in it.requests:
+                rows = -(-rows // tile) * tile + reqs[r][0]
+            assert -(-rows // chunk) == -(-reqs[it.requests[0]][0] // chunk)       # no chunk more than the head alone takes
+            assert it.tokens == sum(reqs[r][0] for r in it.requests)
+            order += it.requests
+        else:
+            assert it.requests == running_before
+            for r in it.requests:
+                decodes[r] += 1
+    assert order == list(range(len(reqs))) and batches > 0
+    assert all(1 + decodes[r] == reqs[r][1] for r in range(len(reqs)))
+    assert s.free_pages == pool and not s.running and not s.waiting
+
+
+class _BatchingStandIn(_StandInEngine):
+    """The stand-in engine with a batched prefill call (records one call for the whole batch)."""
+
+    def __init__(self, B, pool, kv_block):
+        super().__init__(B, pool, kv_block)
+        self.batch_fn = self.corun.PREFILL_BATCH_FN(self._prefill_batch)
+
+    def _prefill_batch(self, ctx, n, slots, tokens, lens, reserves, samplings, seeds, firsts):
+        need = sum(-(-reserves[i] // self.kv_block) for i in range(n))
+        if need > self.free or any(slots[i] in self.pages for i in range(n)):
+            return self.corun.ENOSPACE
+        off = 0
+        for i in range(n):
+            self.pages[slots[i]] = -(-reserves[i] // self.kv_block)
+            self.step_of[slots[i]] = 1
+            firsts[i] = int(seeds[i]) % 1000
+            assert [tokens[off + j] for j in range(lens[i])] == [j % 97 for j in range(lens[i])]
+            off += lens[i]
+        self.free -= need
+        self.calls.append(("prefill_batch", tuple(slots[i] for i in range(n)), tuple(lens[i] for i in range(n)),
+                           tuple(int(seeds[i]) for i in range(n))))
+        return 0
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_library_scheduler_takes_the_batched_oracles_decisions(seed):
+    from paper_2608_14376_b200 import build, corun
+
+    build.build()
+    B, kv_block, pool, reqs, script = _random_trace(200 + seed)
+    B, pool = B + 2, 3 * pool                                  # room for batches: at least three slots
+    chunk, tile = 256, 32
+    eng = _BatchingStandIn(B, pool, kv_block)
+    sch = corun.Scheduler(ops=eng.ops, B=B, kv_block=kv_block, max_context=256)
+    sch.enable_batched_prefill(eng.batch_fn, chunk, tile)
+    ref = sched_oracle.BatchedScheduler(B, pool, kv_block, chunk, tile)
+    nxt, n_batched = 0, 0
+    try:
+        with pytest.raises(corun.CorunError):
+            sch.enable_batched_prefill(eng.batch_fn, 64, 48)                     # tile must divide the chunk
+        for op, k in script + [("step", 10 ** 6)]:
+            if op == "submit":
+                for i, (p, m) in enumerate(reqs[nxt:nxt + k]):
+                    sch.submit(np.arange(p) % 97, m, 0.7, 0.9, seed=5000 + nxt + i)
+                    ref.add_request(p, m)
+                nxt += k
+                continue
+            for _ in range(k):
+                want = ref.decision()
+                action, rid, n = sch.step()
+                assert action == {"idle": corun.SCHED_IDLE, "prefill": corun.SCHED_PREFILL, "decode": corun.SCHED_DECODE}[want.kind]
+                if want.kind == "prefill":
+                    assert rid == want.requests[0] and n == len(want.requests)
+                    if n > 1:
+                        n_batched += 1
+                        call = [c for c in eng.calls if c[0] == "prefill_batch"][-1]
+                        assert call[2] == tuple(reqs[r][0] for r in want.requests)
+                        assert call[3] == tuple(5000 + r for r in want.requests)
+                elif want.kind == "decode":
+                    assert n == len(want.requests)
+                assert sch.counts() == (len(ref.waiting), len(ref.running))
+                assert eng.free == ref.free_pages
+                if want.kind == "idle" and nxt == len(reqs):
+                    break
+        assert n_batched > 0
+        for rid, (p, m) in enumerate(reqs):
+            toks, fin = sch.poll(rid)
+            assert fin and list(toks) == [(5000 + rid) % 1000 + t for t in range(m)]
+        assert eng.free == pool and not eng.pages
+    finally:
+        sch.close()
