@@ -544,13 +544,28 @@ int prefill_finish_row(corun_engine *e, int row, PfReq &r) {
 // Every kernel of the program treats its rows independently of each other and of where they sit in the
 // chunk, and attention reads all keys -- the chunk's own too -- from the cache, so a request's values do not
 // depend on how its prompt is cut into pieces nor on what else shares its chunks.
+int prefill_run(corun_engine *e, PfReq *reqs, int n_req);
+
 int prefill_many(corun_engine *e, PfReq *reqs, int n_req) {
-  const corun_shape &s = e->sh;
   RC(sync_stream(e));
   size_t need = 0;
   for (int i = 0; i < n_req; ++i) need += (size_t)(reqs[i].reserve + KV_BLOCK - 1) / KV_BLOCK;
   if (need > e->free_blocks.size()) return CORUN_ENOSPACE;
-  for (int i = 0; i < n_req; ++i) RC(reserve_blocks(e, reqs[i].slot, reqs[i].reserve));
+  int rc = CORUN_OK;
+  for (int i = 0; i < n_req && rc == CORUN_OK; ++i) rc = reserve_blocks(e, reqs[i].slot, reqs[i].reserve);
+  if (rc == CORUN_OK) rc = prefill_run(e, reqs, n_req);
+  if (rc != CORUN_OK)                               // nothing was admitted: the pages go back to the pool
+    for (int i = 0; i < n_req; ++i) {
+      std::vector<int> &mine = e->slot_blocks[reqs[i].slot];
+      if (e->in_use[reqs[i].slot]) continue;
+      for (int b : mine) e->free_blocks.push_back(b);
+      mine.clear();
+    }
+  return rc;
+}
+
+int prefill_run(corun_engine *e, PfReq *reqs, int n_req) {
+  const corun_shape &s = e->sh;
   Program &P = e->pre;
   const int CH = e->chunk;
   int unit = 128 / (s.n_q_heads / s.n_kv_heads);    // tokens per attention tile
