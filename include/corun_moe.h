@@ -11,8 +11,9 @@
  * no groups at all.  For B padded rows x [B, H]:
  *
  *   router   logits = x Wr^T, p = softmax over all E experts, S = top_k by p
- *            (ties to the lower expert id), weights p_e as they are (no
- *            renormalisation); shared experts always on with weight 1;
+ *            (ties to the lower expert id), weights p_e as they are or, on
+ *            request, renormalised over the selected ones; shared experts always
+ *            on with weight 1;
  *   GEMM 1   [B, H] x all experts' gate and up rows: [B, (E + S) * 2F];
  *   SwiGLU   h[r, e*F + f] = w[r, e] * silu(gate) * up, exactly 0 for the
  *            experts row r did not select;
@@ -48,6 +49,8 @@ typedef struct {
   int32_t top_k;       /* 1..min(E, 16) */
   int32_t expert_ffn;  /* F, multiple of 64; 2F a multiple of 4 */
   int32_t n_shared;    /* always-on experts of the same size, >= 0 */
+  int32_t renormalize; /* 0: the selected probabilities as they are; 1: divided by their sum (added in
+                          descending-probability order) */
 } corun_moe_shape;
 
 /*

@@ -13,8 +13,10 @@ no formulas, so the block is the standard one of the DeepSeek-V2-Lite shape the 
     y        = sum_{e in S} p_e * FFN_e(x)  +  sum_s FFN_shared_s(x)              (no renormalisation of p)
     FFN(x)   = Wd @ (silu(Wg @ x) * (Wu @ x)),   silu(a) = a / (1 + exp(-a))
 
-Readings (the paper is silent): gating is softmax-then-top-k, the selected probabilities are used as
-they are (they sum to less than 1); shared experts are always on with weight 1; the sum over the
+Readings (the paper is silent): gating is softmax-then-top-k; the selected probabilities are used as
+they are (they sum to less than 1; the DeepSeek-V2-Lite convention) or, with ``renormalize``, divided by
+their sum in descending-probability order (the Qwen3-MoE convention; the paper evaluates both families);
+shared experts are always on with weight 1; the sum over the
 selected experts runs in ascending expert id, the shared experts last.  Everything is fp64 on the
 given (already bf16-valued) weights and fp32-valued inputs; loops are plain, one row and one expert
 at a time.
@@ -52,7 +54,7 @@ def router(x: np.ndarray, Wr: np.ndarray, top_k: int):
     return ids, p[ids], p
 
 
-def moe_ffn(X, Wr, Wg, Wu, Wd, shared, top_k: int, experts=None):
+def moe_ffn(X, Wr, Wg, Wu, Wd, shared, top_k: int, experts=None, renormalize: bool = False):
     """X [B, H]; Wr [E, H]; Wg, Wu [E, F, H]; Wd [E, H, F]; shared = list of (Wg, Wu, Wd) always-on
     experts.  ``experts`` ([B, top_k] ids) overrides the router's choice (their probabilities are still
     the router's), for comparing outputs when a near-tie was decided the other way in another precision.
@@ -67,10 +69,16 @@ def moe_ffn(X, Wr, Wg, Wu, Wd, shared, top_k: int, experts=None):
         if experts is not None:
             ids = np.asarray(experts[b], dtype=np.int64)
             ps = p_all[ids]
+        if renormalize:
+            tot = 0.0
+            for v in ps:                                      # in the order of ids: descending probability
+                tot += v
+            ps = ps / tot
         ids_out[b], p_out[b] = ids, ps
+        weight = {int(e): float(w) for e, w in zip(ids, ps)}
         y = np.zeros(X.shape[1], dtype=np.float64)
-        for e in sorted(int(i) for i in ids):                 # ascending expert id
-            y += p_all[e] * ffn(X[b], Wg[e], Wu[e], Wd[e])
+        for e in sorted(weight):                              # ascending expert id
+            y += weight[e] * ffn(X[b], Wg[e], Wu[e], Wd[e])
         for (sg, su, sd) in shared:                           # shared experts last
             y += ffn(X[b], sg, su, sd)
         Y[b] = y

@@ -7,6 +7,7 @@
     python -m paper_2608_14376_b200.cases prefill   [--layers 2 --tokens 4096 --reps 2]
     python -m paper_2608_14376_b200.cases prefill_batch [--layers 36 --lengths 40,100,200,500,1000 --n 8]
     python -m paper_2608_14376_b200.cases moe       [--B 128 --reps 20]      # DeepSeek-V2-Lite MoE block shape
+    python -m paper_2608_14376_b200.cases moe --experts 128 --top-k 8 --ffn 768 --shared 0 --renormalize   # Qwen3-30B-A3B block
     python -m paper_2608_14376_b200.cases ablation  [--layers 2 --B 64 --actives 1,4,16,40,64]
     python -m paper_2608_14376_b200.cases sweep     [--Bs 1,8,32,128,256 --fractions 0.125,0.5,1 --steps 10]
     python -m paper_2608_14376_b200.cases trace     [--requests 200 --rate 4 --B 128 --replay 4 --batched]
@@ -148,7 +149,7 @@ def case_moe(a):
     g = torch.Generator(device="cuda").manual_seed(0)
     mk = lambda *shape: (torch.randn(shape, generator=g, device="cuda") * 0.02).to(torch.bfloat16).contiguous()
     router, gate_up, down = mk(E, H), mk((E + S) * 2 * F, H), mk(H, (E + S) * F)
-    op = corun.MoeFfn(H, E, K, F, S, router, gate_up, down, a.B)
+    op = corun.MoeFfn(H, E, K, F, S, router, gate_up, down, a.B, renormalize=a.renormalize)
     x = torch.randn((a.B, H), generator=g, device="cuda")
     for _ in range(3):
         y, ex, pr = op.forward(x)
@@ -163,7 +164,7 @@ def case_moe(a):
     # the same call captured once and replayed as a CUDA graph (the call allocates nothing and never touches the host)
     side = torch.cuda.Stream()
     with torch.cuda.stream(side):
-        op_g = corun.MoeFfn(H, E, K, F, S, router, gate_up, down, a.B)     # bound to the side stream
+        op_g = corun.MoeFfn(H, E, K, F, S, router, gate_up, down, a.B, renormalize=a.renormalize)     # bound to the side stream
         yg = torch.empty_like(x)
         corun.lib().corun_moe_forward(op_g._h, x.data_ptr(), yg.data_ptr(), None, None)
         op_g.sync()
@@ -467,6 +468,7 @@ def main():
     mo.add_argument("--hidden", type=int, default=2048); mo.add_argument("--experts", type=int, default=64)
     mo.add_argument("--top-k", type=int, default=6); mo.add_argument("--ffn", type=int, default=1408)
     mo.add_argument("--shared", type=int, default=2)
+    mo.add_argument("--renormalize", action="store_true", help="selected probabilities divided by their sum (Qwen3-MoE)")
     ab = sub.add_parser("ablation")
     ab.add_argument("--layers", type=int, default=2); ab.add_argument("--B", type=int, default=64)
     ab.add_argument("--actives", default="1,4,16,40,64"); ab.add_argument("--ctx-lo", type=int, default=512)

@@ -32,7 +32,7 @@ EXPORTS = [
 
 class MoeShape(C.Structure):
     _fields_ = [("hidden", C.c_int32), ("n_experts", C.c_int32), ("top_k", C.c_int32), ("expert_ffn", C.c_int32),
-                ("n_shared", C.c_int32)]
+                ("n_shared", C.c_int32), ("renormalize", C.c_int32)]
 
 
 class CorunError(RuntimeError):
@@ -438,7 +438,7 @@ class MoeFfn:
     router [E, H], gate_up [(E + S) * 2F, H], down [H, (E + S) * F]; B padded rows per call."""
 
     def __init__(self, hidden: int, n_experts: int, top_k: int, expert_ffn: int, n_shared: int, router, gate_up, down,
-                 B: int):
+                 B: int, renormalize: bool = False):
         import torch
 
         self._torch = torch
@@ -449,7 +449,7 @@ class MoeFfn:
         assert tuple(router.shape) == (n_experts, hidden)
         assert tuple(gate_up.shape) == ((n_experts + n_shared) * 2 * expert_ffn, hidden)
         assert tuple(down.shape) == (hidden, (n_experts + n_shared) * expert_ffn)
-        sh = MoeShape(hidden, n_experts, top_k, expert_ffn, n_shared)
+        sh = MoeShape(hidden, n_experts, top_k, expert_ffn, n_shared, 1 if renormalize else 0)
         h = C.c_void_p()
         self._stream = torch.cuda.current_stream()
         _check(lib().corun_moe_create(C.byref(sh), router.data_ptr(), gate_up.data_ptr(), down.data_ptr(), B,

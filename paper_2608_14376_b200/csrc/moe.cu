@@ -40,8 +40,9 @@ __device__ __forceinline__ void moe_split(float x, bf16 &hi, bf16 &lo) {
 // id.  Lane l holds experts l, l + 32, ...; the sum of the exponentials is each lane's experts in ascending
 // id, then a fixed butterfly over the lanes.  Writes the routing and the row of SwiGLU weights
 // w[r, 0 .. E + S): p_e for the selected experts, 0 for the others, 1 for the shared ones.
-__global__ void __launch_bounds__(256) moe_route_kernel(GemmOut logits, int B, int E, int S, int top_k, float *__restrict__ w,
-                                                        int *__restrict__ experts, float *__restrict__ probs) {
+__global__ void __launch_bounds__(256) moe_route_kernel(GemmOut logits, int B, int E, int S, int top_k, int renormalize,
+                                                        float *__restrict__ w, int *__restrict__ experts,
+                                                        float *__restrict__ probs) {
   griddep_launch_dependents();
   griddep_wait();
   const int lane = threadIdx.x & 31;
@@ -71,6 +72,9 @@ __global__ void __launch_bounds__(256) moe_route_kernel(GemmOut logits, int B, i
   for (int e = lane; e < E; e += 32) wr[e] = 0.f;
   for (int s = lane; s < S; s += 32) wr[E + s] = 1.f;
   __syncwarp();
+  int ids[MOE_MAX_TOPK];
+  float ps[MOE_MAX_TOPK];
+  float picked = 0.f;                                // sum of the selected probabilities, in selection order
   for (int k = 0; k < top_k; ++k) {
     float bz = -1.f;                                 // this lane's best: largest value, lowest id on ties
     int be = 0x7fffffff;
@@ -88,12 +92,17 @@ __global__ void __launch_bounds__(256) moe_route_kernel(GemmOut logits, int B, i
 #pragma unroll
     for (int j = 0; j < PER; ++j)
       if (lane + 32 * j == be) z[j] = -2.f;          // taken
-    if (lane == 0) {
-      wr[be] = p;
-      if (experts) experts[(size_t)r * top_k + k] = be;
+    ids[k] = be;
+    ps[k] = p;
+    picked += p;
+  }
+  if (lane == 0)
+    for (int k = 0; k < top_k; ++k) {
+      const float p = renormalize ? __fdiv_rn(ps[k], picked) : ps[k];
+      wr[ids[k]] = p;
+      if (experts) experts[(size_t)r * top_k + k] = ids[k];
       if (probs) probs[(size_t)r * top_k + k] = p;
     }
-  }
 }
 
 // h[r, e*F + f] = w[r, e] * silu(gate) * up as a bf16 hi/lo pair; zeros where w[r, e] == 0 (nothing is read
@@ -229,7 +238,7 @@ int corun_moe_forward(corun_moe *m, const float *x, float *y, int32_t *experts, 
   MCK(launch_split(x, m->B, H, m->x_hi, m->x_lo, m->st));
   MCK(gemm_launch(m->p_r, nullptr, m->d_status, m->st, nullptr, true));
   MCK(launch_k(moe_route_kernel, dim3((m->B + 7) / 8), dim3(256), 0, m->st, true, m->p_r.out(), m->B, E, s.n_shared,
-               s.top_k, m->w, experts, probs));
+               s.top_k, s.renormalize, m->w, experts, probs));
   MCK(gemm_launch(m->p_gu, nullptr, m->d_status, m->st, nullptr, true));
   MCK(launch_k(moe_swiglu_kernel, dim3((NB * (F / 4) + 255) / 256, m->B), dim3(256), 0, m->st, true, m->p_gu.out(),
                (const float *)m->w, F, NB, m->h_hi, m->h_lo));

@@ -102,3 +102,19 @@ def test_rows_are_independent_and_the_override_keeps_the_routers_probabilities()
         np.testing.assert_allclose(p3[b], p_all[:3])
         want = sum(p_all[e] * mo.ffn(X[b], Wg[e], Wu[e], Wd[e]) for e in range(3))
         np.testing.assert_allclose(Y3[b], want, rtol=1e-12)
+
+
+def test_renormalised_gating_hand_computed():
+    """The example above with renormalisation: weights .4 / .7 and .3 / .7."""
+    x = np.array([1.0, 0.0])
+    Wr = np.array([[math.log(4), 0], [math.log(3), 0], [math.log(2), 0], [0.0, 0]])
+    Wg = np.array([[[1.0, 0.0]]] * 4)
+    Wu = np.array([[[1.0, 0.0]]] * 4)
+    Wd = np.array([[[ce], [0.0]] for ce in (1.0, 10.0, 100.0, 1000.0)])
+    Y, ids, ps = mo.moe_ffn(x[None], Wr, Wg, Wu, Wd, [], 2, renormalize=True)
+    s = 1.0 / (1.0 + math.exp(-1.0))
+    np.testing.assert_allclose(ps[0], [4 / 7, 3 / 7], rtol=1e-12)
+    np.testing.assert_allclose(Y[0], [(4 / 7 * 1.0 + 3 / 7 * 10.0) * s, 0.0], rtol=1e-12)
+    # top_k = E renormalised is the plain softmax mixture
+    Y4, _, p4 = mo.moe_ffn(x[None], Wr, Wg, Wu, Wd, [], 4, renormalize=True)
+    np.testing.assert_allclose(p4[0], [0.4, 0.3, 0.2, 0.1], rtol=1e-12)
