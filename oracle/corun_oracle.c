@@ -148,6 +148,81 @@ void orc_attention(const float *q, const float *K, const float *V, int64_t strid
 /* ---- the forward pass ---- */
 
 /*
+ * Optional Mixture-of-Experts feed-forward layers (the paper evaluates MoE
+ * models -- Evaluation, "Setup" -- without giving formulas; this is the
+ * standard block, restated from oracle/moe_oracle.py's definition):
+ *   p = softmax(Wr x) over all E experts; S = top_k by p, ties to the lower
+ *   id; weights p_e as they are or, with renormalize, divided by their sum
+ *   taken in descending-probability order; shared experts always on, weight 1;
+ *   y = sum over S in ascending expert id of w_e FFN_e(x), shared experts last;
+ *   FFN_e(x) = Wd_e (silu(Wg_e x) * (Wu_e x)).
+ * Weight layout per layer: router [E, H]; gate_up [(E + S) * 2F, H], block e =
+ * expert e (gate rows, then up rows; shared experts behind the routed ones);
+ * down [H, (E + S) * F], columns e*F.. of expert e.
+ */
+typedef struct {
+  int32_t n_experts, top_k, expert_ffn, n_shared, renormalize;
+  const uint16_t *const *router;   /* L x [E, H]             */
+  const uint16_t *const *gate_up;  /* L x [(E+S)*2F, H]      */
+  const uint16_t *const *down;     /* L x [H, (E+S)*F]       */
+} orc_moe;
+
+/* One row through one MoE layer: x [H] -> y [H]; ids / probs [top_k] (may be NULL) receive the routing.
+ * Everything accumulates in fp64; the hidden activations of an expert are kept in fp64 too. */
+void orc_moe_ffn(const orc_moe *m, int64_t layer, int64_t H, const float *x, float *y, int32_t *ids, double *probs) {
+  const int64_t E = m->n_experts, F = m->expert_ffn, S = m->n_shared, Kt = m->top_k, NB = E + S;
+  const uint16_t *Wr = m->router[layer], *Wgu = m->gate_up[layer], *Wd = m->down[layer];
+  double *p = (double *)malloc(sizeof(double) * E);
+  double *wt = (double *)calloc((size_t)NB, sizeof(double));
+  double *hid = (double *)malloc(sizeof(double) * F);
+  double *acc = (double *)calloc((size_t)H, sizeof(double));
+  char *taken = (char *)calloc((size_t)E, 1);
+  double mx = -INFINITY, sum = 0.0;
+  for (int64_t e = 0; e < E; ++e) {
+    double d = 0.0;
+    for (int64_t i = 0; i < H; ++i) d += bf16_to_f64(Wr[e * H + i]) * (double)x[i];
+    p[e] = d;
+    if (d > mx) mx = d;
+  }
+  for (int64_t e = 0; e < E; ++e) { p[e] = exp(p[e] - mx); sum += p[e]; }
+  for (int64_t e = 0; e < E; ++e) p[e] /= sum;
+  double picked = 0.0;
+  int32_t chosen[64];
+  for (int64_t k = 0; k < Kt && k < 64; ++k) {
+    int64_t best = -1;
+    for (int64_t e = 0; e < E; ++e)
+      if (!taken[e] && (best < 0 || p[e] > p[best])) best = e;   /* strict: the lower id keeps a tie */
+    taken[best] = 1;
+    chosen[k] = (int32_t)best;
+    picked += p[best];
+  }
+  for (int64_t k = 0; k < Kt && k < 64; ++k) {
+    const double w = m->renormalize ? p[chosen[k]] / picked : p[chosen[k]];
+    wt[chosen[k]] = w;
+    if (ids) ids[k] = chosen[k];
+    if (probs) probs[k] = w;
+  }
+  for (int64_t s = 0; s < S; ++s) wt[E + s] = 1.0;
+  for (int64_t e = 0; e < NB; ++e) {              /* ascending expert id, shared experts last */
+    if (e < E && !taken[e]) continue;
+    for (int64_t f = 0; f < F; ++f) {
+      double g = 0.0, u = 0.0;
+      const uint16_t *wg = Wgu + (e * 2 * F + f) * H, *wu = Wgu + (e * 2 * F + F + f) * H;
+      for (int64_t i = 0; i < H; ++i) { g += bf16_to_f64(wg[i]) * (double)x[i]; u += bf16_to_f64(wu[i]) * (double)x[i]; }
+      hid[f] = orc_silu(g) * u;
+    }
+    for (int64_t i = 0; i < H; ++i) {
+      double d = 0.0;
+      const uint16_t *wd = Wd + i * NB * F + e * F;
+      for (int64_t f = 0; f < F; ++f) d += bf16_to_f64(wd[f]) * hid[f];
+      acc[i] += wt[e] * d;
+    }
+  }
+  for (int64_t i = 0; i < H; ++i) y[i] = (float)acc[i];
+  free(p); free(wt); free(hid); free(acc); free(taken);
+}
+
+/*
  * Runs tokens[0..T) of ONE request at positions pos0..pos0+T-1 through the
  * decoder.  Kc/Vc: the request's cache, [L][max_T][nkv*hd] fp32; positions
  * below pos0 must already be filled, positions pos0.. are written.
@@ -155,8 +230,8 @@ void orc_attention(const float *q, const float *K, const float *V, int64_t strid
  * NULL to skip the LM head.  Returns 0, or -1 on a bad argument.
  * Prefill is T = prompt length at pos0 = 0; a decode step is T = 1.
  */
-int orc_forward(const orc_shape *sh, const orc_weights *w, const int32_t *tokens, int64_t T, int64_t pos0,
-                float *Kc, float *Vc, int64_t max_T, float *logits, int all_logits) {
+int orc_forward_ex(const orc_shape *sh, const orc_weights *w, const orc_moe *moe, const int32_t *tokens, int64_t T,
+                   int64_t pos0, float *Kc, float *Vc, int64_t max_T, float *logits, int all_logits) {
   const int64_t H = sh->hidden, nq = sh->n_q_heads, nkv = sh->n_kv_heads, hd = sh->head_dim;
   const int64_t F = sh->ffn, Vn = sh->vocab, L = sh->n_layers;
   const int64_t QD = nq * hd, KD = nkv * hd, QKV = QD + 2 * KD;
@@ -191,6 +266,12 @@ int orc_forward(const orc_shape *sh, const orc_weights *w, const int32_t *tokens
     orc_matmul_bf16(w->wo[l], H, QD, o, T, y);
     for (int64_t i = 0; i < T * H; ++i) h[i] = h[i] + y[i];
     for (int64_t t = 0; t < T; ++t) orc_rmsnorm(h + t * H, w->mlp_norm[l], H, sh->rms_eps, a + t * H);
+    if (moe) {                                      /* Mixture-of-Experts feed-forward layer */
+#pragma omp parallel for schedule(dynamic)
+      for (int64_t t = 0; t < T; ++t) orc_moe_ffn(moe, l, H, a + t * H, y + t * H, NULL, NULL);
+      for (int64_t i = 0; i < T * H; ++i) h[i] = h[i] + y[i];
+      continue;
+    }
     orc_matmul_bf16(w->wgate_up[l], 2 * F, H, a, T, gu);
     for (int64_t t = 0; t < T; ++t)
       for (int64_t i = 0; i < F; ++i) {
@@ -212,6 +293,11 @@ int orc_forward(const orc_shape *sh, const orc_weights *w, const int32_t *tokens
   }
   free(h); free(a); free(qkv); free(o); free(y); free(gu);
   return 0;
+}
+
+int orc_forward(const orc_shape *sh, const orc_weights *w, const int32_t *tokens, int64_t T, int64_t pos0,
+                float *Kc, float *Vc, int64_t max_T, float *logits, int all_logits) {
+  return orc_forward_ex(sh, w, NULL, tokens, T, pos0, Kc, Vc, max_T, logits, all_logits);
 }
 
 /* ---- request-bound random variate R(seed, t) ---- */

@@ -48,6 +48,11 @@ class _Weights(C.Structure):
                 ("mlp_norm", _PP), ("wgate_up", _PP), ("wdown", _PP)]
 
 
+class _Moe(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_experts", "top_k", "expert_ffn", "n_shared", "renormalize")] + [
+        ("router", _PP), ("gate_up", _PP), ("down", _PP)]
+
+
 def lib():
     global _lib
     if _lib is None:
@@ -55,6 +60,11 @@ def lib():
         L.orc_forward.restype = C.c_int
         L.orc_forward.argtypes = [C.POINTER(_Shape), C.POINTER(_Weights), C.c_void_p, C.c_int64, C.c_int64,
                                   C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int]
+        L.orc_forward_ex.restype = C.c_int
+        L.orc_forward_ex.argtypes = [C.POINTER(_Shape), C.POINTER(_Weights), C.POINTER(_Moe), C.c_void_p, C.c_int64,
+                                     C.c_int64, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int]
+        L.orc_moe_ffn.restype = None
+        L.orc_moe_ffn.argtypes = [C.POINTER(_Moe), C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.orc_matmul_bf16.restype = None
         L.orc_matmul_bf16.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p]
         L.orc_rmsnorm.restype = None
@@ -112,9 +122,14 @@ class Model:
     ``weights`` keys: embed [V,H], lm_head [V,H], final_norm [H], and lists of
     L arrays: attn_norm [H], wqkv [(nq+2nkv)*hd, H] (q rows, then k, then v),
     wo [H, nq*hd], mlp_norm [H], wgate_up [2F, H] (gate rows, then up), wdown [H, F].
+
+    ``moe`` (optional) turns every feed-forward layer into a Mixture-of-Experts block: a dict with
+    n_experts, top_k, expert_ffn, n_shared, renormalize and lists of L arrays router [E, H],
+    gate_up [(E+S)*2F, H] (block e = expert e: gate rows then up rows), down [H, (E+S)*F]; the dense
+    wgate_up / wdown entries are then unused (any placeholders).
     """
 
-    def __init__(self, shape: Shape, weights: dict):
+    def __init__(self, shape: Shape, weights: dict, moe: dict = None):
         self.shape = shape
         self._keep = {k: ([_u16(x) for x in v] if isinstance(v, (list, tuple)) else _u16(v))
                       for k, v in weights.items()}
@@ -130,6 +145,26 @@ class Model:
             self._arrs[k] = arr
             setattr(cw, k, C.cast(arr, _PP))
         self._cw = cw
+        self._cm = None
+        if moe is not None:
+            self._moe_keep = {k: [_u16(x) for x in moe[k]] for k in ("router", "gate_up", "down")}
+            cm = _Moe(moe["n_experts"], moe["top_k"], moe["expert_ffn"], moe["n_shared"], 1 if moe.get("renormalize") else 0)
+            for k in ("router", "gate_up", "down"):
+                arr = (C.c_void_p * sh.n_layers)(*[_ptr(x) for x in self._moe_keep[k]])
+                self._arrs["moe_" + k] = arr
+                setattr(cm, k, C.cast(arr, _PP))
+            self._cm = cm
+            self.moe = dict(moe)
+
+    def moe_ffn_row(self, layer: int, x):
+        """One row through the Mixture-of-Experts block of ``layer``: (y [H], ids [top_k], weights [top_k])."""
+        x = _f32(x)
+        y = np.empty_like(x)
+        k = self.moe["top_k"]
+        ids = np.zeros(k, np.int32)
+        pr = np.zeros(k, np.float64)
+        lib().orc_moe_ffn(C.byref(self._cm), layer, x.shape[0], _ptr(x), _ptr(y), _ptr(ids), _ptr(pr))
+        return y, ids, pr
 
     def new_cache(self, max_T: int):
         sh = self.shape
@@ -149,8 +184,9 @@ class Model:
             out = np.empty((T, self.shape.vocab), np.float32)
         elif want == "last":
             out = np.empty((self.shape.vocab,), np.float32)
-        rc = lib().orc_forward(C.byref(self._cs), C.byref(self._cw), _ptr(toks), T, pos0, _ptr(K), _ptr(V),
-                               K.shape[1], _ptr(out) if out is not None else None, 1 if want == "all" else 0)
+        rc = lib().orc_forward_ex(C.byref(self._cs), C.byref(self._cw), C.byref(self._cm) if self._cm is not None else None,
+                                  _ptr(toks), T, pos0, _ptr(K), _ptr(V), K.shape[1],
+                                  _ptr(out) if out is not None else None, 1 if want == "all" else 0)
         if rc != 0:
             raise ValueError("orc_forward: bad argument")
         return out

@@ -118,3 +118,59 @@ def test_renormalised_gating_hand_computed():
     # top_k = E renormalised is the plain softmax mixture
     Y4, _, p4 = mo.moe_ffn(x[None], Wr, Wg, Wu, Wd, [], 4, renormalize=True)
     np.testing.assert_allclose(p4[0], [0.4, 0.3, 0.2, 0.1], rtol=1e-12)
+
+
+# ---- the C oracle's Mixture-of-Experts layer (used inside the full decoder) against the definition above
+def _bits(a):
+    from paper_2608_14376_b200 import synth
+    return synth.f32_to_bf16_bits(np.asarray(a, np.float32))
+
+
+def _vals(bits):
+    from paper_2608_14376_b200 import synth
+    return synth.bf16_bits_to_f32(bits).astype(np.float64)
+
+
+@pytest.mark.parametrize("renorm", [False, True])
+def test_c_oracle_moe_layer_equals_the_definition(renorm):
+    from oracle import oracle
+    from paper_2608_14376_b200 import synth
+
+    sh = synth.TINY
+    H, E, K, F, S = sh.hidden, 6, 2, 64, 1
+    rng = np.random.default_rng(5)
+    NB = E + S
+    Wg, Wu = _bits(rng.standard_normal((NB, F, H)) * 0.1), _bits(rng.standard_normal((NB, F, H)) * 0.1)
+    Wd, Wr = _bits(rng.standard_normal((NB, H, F)) * 0.1), _bits(rng.standard_normal((E, H)) * 0.3)
+    gate_up = np.concatenate([np.concatenate([Wg[e], Wu[e]], 0) for e in range(NB)], 0)
+    down = np.concatenate([Wd[e] for e in range(NB)], 1)
+    w = synth.make_weights_numpy(sh, seed=1)
+    moe = dict(n_experts=E, top_k=K, expert_ffn=F, n_shared=S, renormalize=renorm,
+               router=[Wr] * sh.n_layers, gate_up=[np.ascontiguousarray(gate_up)] * sh.n_layers,
+               down=[np.ascontiguousarray(down)] * sh.n_layers)
+    model = oracle.Model(oracle.Shape(**sh.dict()), w, moe=moe)
+    X = rng.standard_normal((5, H)).astype(np.float32)
+    shared = [(_vals(Wg[E + s]), _vals(Wu[E + s]), _vals(Wd[E + s])) for s in range(S)]
+    Y, ids, ps = mo.moe_ffn(X, _vals(Wr), _vals(Wg), _vals(Wu), _vals(Wd), shared, K, renormalize=renorm)
+    for b in range(5):
+        y, i, p = model.moe_ffn_row(1, X[b])
+        assert list(i) == list(ids[b])
+        np.testing.assert_allclose(p, ps[b], rtol=1e-12)
+        np.testing.assert_allclose(y, Y[b], rtol=2e-6, atol=1e-7)   # the C function returns fp32
+
+
+def test_c_oracle_decoder_with_one_always_selected_expert_is_the_dense_decoder():
+    """E = 1, top-1, renormalised (weight exactly 1), the expert = the dense FFN: same logits as the dense model."""
+    from oracle import oracle
+    from paper_2608_14376_b200 import synth
+
+    sh = synth.TINY
+    w = synth.make_weights_numpy(sh, seed=2)
+    moe = dict(n_experts=1, top_k=1, expert_ffn=sh.ffn, n_shared=0, renormalize=True,
+               router=[np.zeros((1, sh.hidden), np.uint16)] * sh.n_layers, gate_up=w["wgate_up"], down=w["wdown"])
+    dense = oracle.Model(oracle.Shape(**sh.dict()), w)
+    sparse = oracle.Model(oracle.Shape(**sh.dict()), w, moe=moe)
+    toks = synth.make_prompts(sh.vocab, [9], seed=4)[0]
+    a = dense.forward(toks, 0, dense.new_cache(16))
+    b = sparse.forward(toks, 0, sparse.new_cache(16))
+    np.testing.assert_allclose(b, a, rtol=0, atol=2e-5)
