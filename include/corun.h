@@ -94,6 +94,27 @@ int corun_init(const corun_shape *shape, const corun_weights *weights, int32_t B
                int32_t kv_block, int64_t kv_pool_blocks, void *cuda_stream, corun_engine **out);
 
 /*
+ * The same engine with Mixture-of-Experts feed-forward layers (the paper's evaluated models are MoE
+ * decoders -- Evaluation, "Setup"): grouped-query attention as above, every feed-forward layer a
+ * router + routed experts (+ always-on shared experts) computed without expert groups, so that a row's
+ * result does not depend on which rows share the step (include/corun_moe.h describes the block).
+ * shape->ffn and weights->wgate_up / wdown are ignored (the arrays may be NULL).
+ *   router   L device pointers, bf16 [E, H]
+ *   gate_up  L device pointers, bf16 [(E + n_shared) * 2F, H]: block e = expert e, gate rows then up rows;
+ *            shared experts behind the routed ones
+ *   down     L device pointers, bf16 [H, (E + n_shared) * F]: columns e*F.. of expert e
+ * n_experts 1..256, top_k 1..min(E, 16), expert_ffn a multiple of 64; renormalize: the selected
+ * probabilities divided by their sum.  Errors as corun_init.
+ */
+typedef struct {
+  int32_t n_experts, top_k, expert_ffn, n_shared, renormalize;
+  const void *const *router, *const *gate_up, *const *down;
+} corun_moe_layers;
+int corun_init_moe(const corun_shape *shape, const corun_weights *weights, const corun_moe_layers *moe, int32_t B,
+                   int32_t max_context, int32_t kv_block, int64_t kv_pool_blocks, void *cuda_stream,
+                   corun_engine **out);
+
+/*
  * Isolated prefill (paper, Design, "Isolated Prefill"; Algorithm 1's admission
  * rule): runs the n prompt tokens of one request alone, in fixed-size chunks
  * whose sequence depends on n only, writes its KV cache, samples the first

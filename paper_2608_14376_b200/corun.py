@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libcorun.so")
 OK, EINVAL, ESLOT, ENOSPACE, ECTX, ECUDA, ETIMEOUT, ENOMEM, ELIMIT = 0, -1, -2, -3, -4, -5, -6, -7, -8
 
 EXPORTS = [
-    "corun_init", "corun_prefill", "corun_prefill_batch", "corun_decode_step", "corun_decode_enqueue", "corun_decode_wait",
+    "corun_init", "corun_init_moe", "corun_prefill", "corun_prefill_batch", "corun_decode_step", "corun_decode_enqueue", "corun_decode_wait",
     "corun_release", "corun_destroy", "corun_get_logits", "corun_force_token", "corun_context_len",
     "corun_free_blocks", "corun_debug_kv_read", "corun_debug_kv_write", "corun_debug_adopt",
     "corun_debug_set_eager", "corun_debug_read", "corun_debug_gemm_trace", "corun_debug_attn_trace", "corun_debug_step_trace", "corun_debug_kv_fill", "corun_debug_time_kernel", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
@@ -33,6 +33,13 @@ EXPORTS = [
 class MoeShape(C.Structure):
     _fields_ = [("hidden", C.c_int32), ("n_experts", C.c_int32), ("top_k", C.c_int32), ("expert_ffn", C.c_int32),
                 ("n_shared", C.c_int32), ("renormalize", C.c_int32)]
+
+
+class MoeLayers(C.Structure):
+    """``corun_moe_layers``."""
+    _fields_ = [("n_experts", C.c_int32), ("top_k", C.c_int32), ("expert_ffn", C.c_int32), ("n_shared", C.c_int32),
+                ("renormalize", C.c_int32), ("router", C.POINTER(C.c_void_p)), ("gate_up", C.POINTER(C.c_void_p)),
+                ("down", C.POINTER(C.c_void_p))]
 
 
 class CorunError(RuntimeError):
@@ -159,7 +166,10 @@ class Engine:
     describes (see ``synth.make_weights_*``); they are borrowed, keep them alive.
     """
 
-    def __init__(self, shape, weights: dict, B: int, max_context: int, kv_pool_blocks: int = 0, stream=None):
+    def __init__(self, shape, weights: dict, B: int, max_context: int, kv_pool_blocks: int = 0, stream=None, moe: dict = None):
+        """``moe``: Mixture-of-Experts feed-forward layers instead of the dense ones: a dict with n_experts, top_k,
+        expert_ffn, n_shared, renormalize and lists of L CUDA bf16 tensors router [E, H], gate_up [(E+S)*2F, H],
+        down [H, (E+S)*F] (``weights`` then needs no wgate_up / wdown)."""
         import torch
 
         self._torch = torch
@@ -174,7 +184,7 @@ class Engine:
             t = weights[k]
             assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
             setattr(cw, k, t.data_ptr())
-        for k in ("attn_norm", "wqkv", "wo", "mlp_norm", "wgate_up", "wdown"):
+        for k in ("attn_norm", "wqkv", "wo", "mlp_norm") + (() if moe else ("wgate_up", "wdown")):
             ts = weights[k]
             assert len(ts) == d["n_layers"]
             for t in ts:
@@ -185,8 +195,25 @@ class Engine:
         self._cw = cw
         torch.cuda.synchronize()
         h = C.c_void_p()
-        _check(lib().corun_init(C.byref(self._cs), C.byref(cw), B, max_context, 16, kv_pool_blocks,
-                                C.c_void_p(stream) if stream else None, C.byref(h)), "corun_init")
+        if moe:
+            cm = MoeLayers(moe["n_experts"], moe["top_k"], moe["expert_ffn"], moe["n_shared"], 1 if moe.get("renormalize") else 0)
+            self._moe = moe
+            for k in ("router", "gate_up", "down"):
+                ts = moe[k]
+                assert len(ts) == d["n_layers"]
+                for t in ts:
+                    assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+                arr = (C.c_void_p * len(ts))(*[t.data_ptr() for t in ts])
+                self._arrs["moe_" + k] = arr
+                setattr(cm, k, C.cast(arr, _PP))
+            L = lib()
+            L.corun_init_moe.argtypes = [C.POINTER(Shape), C.POINTER(Weights), C.POINTER(MoeLayers), C.c_int32, C.c_int32,
+                                         C.c_int32, C.c_int64, C.c_void_p, C.POINTER(C.c_void_p)]
+            _check(L.corun_init_moe(C.byref(self._cs), C.byref(cw), C.byref(cm), B, max_context, 16, kv_pool_blocks,
+                                    C.c_void_p(stream) if stream else None, C.byref(h)), "corun_init_moe")
+        else:
+            _check(lib().corun_init(C.byref(self._cs), C.byref(cw), B, max_context, 16, kv_pool_blocks,
+                                    C.c_void_p(stream) if stream else None, C.byref(h)), "corun_init")
         self._h = h
         self.vocab = d["vocab"]
 

@@ -12,6 +12,7 @@
 
 #include "../../include/corun.h"
 #include "gemm.cuh"
+#include "moe.cuh"
 #include "ops.cuh"
 
 using namespace corun;
@@ -44,6 +45,10 @@ struct Program {
   int *row_token = nullptr, *row_pos = nullptr, *row_active = nullptr, *row_slot = nullptr, *do_sample = nullptr;
   int *sampled = nullptr, *att_work = nullptr, *att_n_work = nullptr, *att_done = nullptr, *att_pool = nullptr;
   GemmPlan p_qkv, p_o, p_gu, p_down, p_lm;
+  // Mixture-of-Experts feed-forward layers: p_gu / p_down are then the GEMMs over all experts' gate / up rows
+  // and over the concatenated hidden activations; p_r is the router GEMM (its rows padded to one tile)
+  GemmPlan p_r;
+  float *r_out = nullptr, *moe_w = nullptr;
   bool has_layers = false, has_lm = false;
   std::vector<void *> allocs;
 };
@@ -63,6 +68,10 @@ struct corun_engine {
   std::vector<const bf16 *> attn_norm, mlp_norm;
   std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_down;
   std::vector<CUtensorMap> tm_k, tm_v;   // per layer: key view and transposed-value view of the pages
+  // Mixture-of-Experts feed-forward layers (E = 0: dense).  sh.ffn is then (E + S) * F.
+  int moe_E = 0, moe_K = 0, moe_F = 0, moe_S = 0, moe_renorm = 0;
+  bf16 *router_pad = nullptr;            // [L][256][H]: each layer's router rows, zero rows behind them
+  std::vector<CUtensorMap> tm_router;
   // KV
   __half *kv_pool = nullptr;
   size_t layer_stride = 0;
@@ -156,6 +165,17 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm) {
     RC(gemm_plan_create(&P.p_o, e->w0_o, H, QD, P.ao_hi, P.ao_lo, R, P.BN, P.o_out, P.ws, e->num_sms));
     RC(gemm_plan_create(&P.p_gu, e->w0_gu, 2 * F, H, P.xn_hi, P.xn_lo, R, P.BN, P.gu_out, P.ws, e->num_sms));
     RC(gemm_plan_create(&P.p_down, e->w0_down, H, F, P.ff_hi, P.ff_lo, R, P.BN, P.down_out, P.ws, e->num_sms));
+    if (e->moe_E) {
+      const int NB = e->moe_E + e->moe_S;
+      RC(dmalloc(A, &P.r_out, (size_t)R * GEMM_TILE_N));
+      RC(dmalloc(A, &P.moe_w, (size_t)R * NB));
+      RC(gemm_plan_create(&P.p_r, e->router_pad, GEMM_TILE_N, H, P.xn_hi, P.xn_lo, R, P.BN, P.r_out, P.ws, e->num_sms));
+      if ((2 * e->moe_F) % GEMM_TILE_N == 0) {      // a weight tile belongs to one expert: rows that did not
+        P.p_gu.row_keep = P.moe_w;                  // select it are not stored (the SwiGLU does not read them)
+        P.p_gu.keep_pitch = NB;
+        P.p_gu.keep_div = 2 * e->moe_F / GEMM_TILE_N;
+      }
+    }
   }
   if (lm) {
     RC(dmalloc(A, &P.logits, (size_t)R * V));
@@ -170,6 +190,7 @@ void program_destroy(Program &P) {
   gemm_plan_destroy(&P.p_gu);
   gemm_plan_destroy(&P.p_down);
   gemm_plan_destroy(&P.p_lm);
+  gemm_plan_destroy(&P.p_r);
   for (void *p : P.allocs) cudaFree(p);
   P.allocs.clear();
 }
@@ -213,8 +234,18 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
     STAGE(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st, tr(4 * l + 1), true));
     GemmOut o = P.p_o.out();
     STAGE(launch_resid_norm(P.h, s.hidden, nullptr, rows, &o, e->mlp_norm[l], s.rms_eps, P.xn_hi, P.xn_lo, e->st));
-    STAGE(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st, tr(4 * l + 2), true));
-    STAGE(launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st));
+    if (e->moe_E) {
+      // router -> top-k weights -> all experts' gate / up (rows that did not select a tile's expert are not
+      // stored) -> masked, weighted SwiGLU; the down GEMM then sums over the row's experts in its accumulator
+      STAGE(gemm_launch(P.p_r, &e->tm_router[l], e->d_status, e->st, nullptr, true));
+      STAGE(launch_moe_route(P.p_r.out(), P.R, e->moe_E, e->moe_S, e->moe_K, e->moe_renorm, P.moe_w, nullptr, nullptr, e->st));
+      STAGE(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st, tr(4 * l + 2), true));
+      STAGE(launch_moe_swiglu(P.p_gu.out(), P.moe_w, P.R, e->moe_F, e->moe_E + e->moe_S, P.ff_hi, P.ff_lo, e->st));
+      n += 2;
+    } else {
+      STAGE(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st, tr(4 * l + 2), true));
+      STAGE(launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st));
+    }
     STAGE(gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st, tr(4 * l + 3), true));
     n += 9;
   }
@@ -313,11 +344,20 @@ const char *corun_strerror(int st) {
   }
 }
 
-int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int32_t max_context, int32_t kv_block,
-               int64_t kv_pool_blocks, void *cuda_stream, corun_engine **out) {
+static int engine_create(const corun_shape *shape, const corun_weights *w, const corun_moe_layers *moe, int32_t B,
+                         int32_t max_context, int32_t kv_block, int64_t kv_pool_blocks, void *cuda_stream,
+                         corun_engine **out) {
   if (!shape || !w || !out) return CORUN_EINVAL;
   *out = nullptr;
-  const corun_shape &s = *shape;
+  corun_shape s = *shape;
+  if (moe) {
+    if (moe->n_experts < 1 || moe->n_experts > 256 || moe->top_k < 1 || moe->top_k > 16 || moe->top_k > moe->n_experts ||
+        moe->expert_ffn < 64 || moe->expert_ffn % 64 || moe->n_shared < 0 || !moe->router || !moe->gate_up || !moe->down)
+      return CORUN_EINVAL;
+    for (int l = 0; l < s.n_layers; ++l)
+      if (!moe->router[l] || !moe->gate_up[l] || !moe->down[l]) return CORUN_EINVAL;
+    s.ffn = (moe->n_experts + moe->n_shared) * moe->expert_ffn;   // the feed-forward width the row program sees
+  }
   if (s.arch != 0 || s.n_layers < 1 || s.hidden < 64 || s.hidden % 64 || s.ffn < 64 || s.ffn % 64 || s.vocab < 1)
     return CORUN_EINVAL;
   if (s.head_dim != 64 && s.head_dim != 128) return CORUN_EINVAL;
@@ -328,10 +368,10 @@ int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int3
   if (!(s.rms_eps >= 0.f) || !(s.rope_theta > 0.f)) return CORUN_EINVAL;
   if (B < 1 || B > 256 || max_context < 1 || max_context > 256 * ATT_SPLIT || kv_block != KV_BLOCK || kv_pool_blocks < 0) return CORUN_EINVAL;
   if (!w->embed || !w->lm_head || !w->final_norm || !w->attn_norm || !w->wqkv || !w->wo || !w->mlp_norm ||
-      !w->wgate_up || !w->wdown)
+      (!moe && (!w->wgate_up || !w->wdown)))
     return CORUN_EINVAL;
   for (int l = 0; l < s.n_layers; ++l)
-    if (!w->attn_norm[l] || !w->wqkv[l] || !w->wo[l] || !w->mlp_norm[l] || !w->wgate_up[l] || !w->wdown[l])
+    if (!w->attn_norm[l] || !w->wqkv[l] || !w->wo[l] || !w->mlp_norm[l] || (!moe && (!w->wgate_up[l] || !w->wdown[l])))
       return CORUN_EINVAL;
 
   int dev = 0;
@@ -359,8 +399,15 @@ int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int3
   }
   e->w0_qkv = w->wqkv[0];
   e->w0_o = w->wo[0];
-  e->w0_gu = w->wgate_up[0];
-  e->w0_down = w->wdown[0];
+  e->w0_gu = moe ? moe->gate_up[0] : w->wgate_up[0];
+  e->w0_down = moe ? moe->down[0] : w->wdown[0];
+  if (moe) {
+    e->moe_E = moe->n_experts;
+    e->moe_K = moe->top_k;
+    e->moe_F = moe->expert_ffn;
+    e->moe_S = moe->n_shared;
+    e->moe_renorm = moe->renormalize ? 1 : 0;
+  }
   e->pool_blocks = kv_pool_blocks ? kv_pool_blocks : (int64_t)B * e->max_blocks;
   if (!kv_pool_blocks) {
     // default size: a full reservation for every slot, or as many pages as fit beside 6 GiB that are
@@ -393,8 +440,19 @@ int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int3
     int rc;
     if ((rc = gemm_encode_map(&e->tm_qkv[l], w->wqkv[l], QD + 2 * KD, H, GEMM_TILE_N))) return fail(rc);
     if ((rc = gemm_encode_map(&e->tm_o[l], w->wo[l], H, QD, GEMM_TILE_N))) return fail(rc);
-    if ((rc = gemm_encode_map(&e->tm_gu[l], w->wgate_up[l], 2 * F, H, GEMM_TILE_N))) return fail(rc);
-    if ((rc = gemm_encode_map(&e->tm_down[l], w->wdown[l], H, F, GEMM_TILE_N))) return fail(rc);
+    if ((rc = gemm_encode_map(&e->tm_gu[l], moe ? moe->gate_up[l] : w->wgate_up[l], 2 * F, H, GEMM_TILE_N))) return fail(rc);
+    if ((rc = gemm_encode_map(&e->tm_down[l], moe ? moe->down[l] : w->wdown[l], H, F, GEMM_TILE_N))) return fail(rc);
+  }
+  if (moe) {
+    int rc;
+    if ((rc = dmalloc(e->allocs, &e->router_pad, (size_t)s.n_layers * GEMM_TILE_N * H))) return fail(rc);
+    e->tm_router.resize(s.n_layers);
+    for (int l = 0; l < s.n_layers; ++l) {
+      bf16 *dst = e->router_pad + (size_t)l * GEMM_TILE_N * H;
+      if (cudaMemcpy(dst, moe->router[l], (size_t)moe->n_experts * H * sizeof(bf16), cudaMemcpyDeviceToDevice) != cudaSuccess)
+        return fail(CORUN_ECUDA);
+      if ((rc = gemm_encode_map(&e->tm_router[l], dst, GEMM_TILE_N, H, GEMM_TILE_N))) return fail(rc);
+    }
   }
 
   auto &A = e->allocs;
@@ -477,6 +535,17 @@ int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int3
   if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return fail(CORUN_ECUDA); }
   *out = e;
   return CORUN_OK;
+}
+
+int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int32_t max_context, int32_t kv_block,
+               int64_t kv_pool_blocks, void *cuda_stream, corun_engine **out) {
+  return engine_create(shape, w, nullptr, B, max_context, kv_block, kv_pool_blocks, cuda_stream, out);
+}
+
+int corun_init_moe(const corun_shape *shape, const corun_weights *w, const corun_moe_layers *moe, int32_t B,
+                   int32_t max_context, int32_t kv_block, int64_t kv_pool_blocks, void *cuda_stream, corun_engine **out) {
+  if (!moe) return CORUN_EINVAL;
+  return engine_create(shape, w, moe, B, max_context, kv_block, kv_pool_blocks, cuda_stream, out);
 }
 
 void corun_destroy(corun_engine *e) {
@@ -874,7 +943,9 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
         case 6: ce = launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->attn_norm[l], s.rms_eps, P.xn_hi,
                                        P.xn_lo, e->st); break;
         case 7: ce = launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st); break;
-        case 8: ce = launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st); break;
+        case 8: ce = e->moe_E ? launch_moe_swiglu(P.p_gu.out(), P.moe_w, P.R, e->moe_F, e->moe_E + e->moe_S, P.ff_hi, P.ff_lo, e->st)
+                              : launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st);
+                break;
         case 9: {
           SampleArgs sa{P.logits, s.vocab, P.do_sample, e->d_temp, e->d_top_p, e->d_seeds, e->d_step, nullptr, P.sampled};
           ce = launch_sampler(sa, P.R, e->st);

@@ -11,6 +11,7 @@
 #include "../../include/corun_moe.h"
 #include "gemm.cuh"
 #include "launch.cuh"
+#include "moe.cuh"
 #include "ops.cuh"
 #include "ptx.cuh"
 
@@ -145,6 +146,23 @@ __global__ void __launch_bounds__(256) moe_readout_kernel(GemmOut d, int H, floa
 
 }  // namespace
 
+namespace corun {
+
+cudaError_t launch_moe_route(const GemmOut &logits, int R, int E, int S, int top_k, int renormalize, float *w,
+                             int *experts, float *probs, cudaStream_t st) {
+  if (E < 1 || E > MOE_MAX_EXPERTS || top_k < 1 || top_k > MOE_MAX_TOPK || top_k > E) return cudaErrorInvalidValue;
+  return launch_k(moe_route_kernel, dim3((R + 7) / 8), dim3(256), 0, st, true, logits, R, E, S, top_k, renormalize, w,
+                  experts, probs);
+}
+
+cudaError_t launch_moe_swiglu(const GemmOut &gu, const float *w, int R, int F, int n_blocks, __nv_bfloat16 *out_hi,
+                              __nv_bfloat16 *out_lo, cudaStream_t st) {
+  return launch_k(moe_swiglu_kernel, dim3((n_blocks * (F / 4) + 255) / 256, R), dim3(256), 0, st, true, gu, w, F, n_blocks,
+                  out_hi, out_lo);
+}
+
+}  // namespace corun
+
 struct corun_moe {
   corun_moe_shape sh{};
   int B = 0, BN = 0, num_sms = 0;
@@ -237,11 +255,9 @@ int corun_moe_forward(corun_moe *m, const float *x, float *y, int32_t *experts, 
   const int H = s.hidden, E = s.n_experts, F = s.expert_ffn, NB = E + s.n_shared;
   MCK(launch_split(x, m->B, H, m->x_hi, m->x_lo, m->st));
   MCK(gemm_launch(m->p_r, nullptr, m->d_status, m->st, nullptr, true));
-  MCK(launch_k(moe_route_kernel, dim3((m->B + 7) / 8), dim3(256), 0, m->st, true, m->p_r.out(), m->B, E, s.n_shared,
-               s.top_k, s.renormalize, m->w, experts, probs));
+  MCK(launch_moe_route(m->p_r.out(), m->B, E, s.n_shared, s.top_k, s.renormalize, m->w, experts, probs, m->st));
   MCK(gemm_launch(m->p_gu, nullptr, m->d_status, m->st, nullptr, true));
-  MCK(launch_k(moe_swiglu_kernel, dim3((NB * (F / 4) + 255) / 256, m->B), dim3(256), 0, m->st, true, m->p_gu.out(),
-               (const float *)m->w, F, NB, m->h_hi, m->h_lo));
+  MCK(launch_moe_swiglu(m->p_gu.out(), m->w, m->B, F, NB, m->h_hi, m->h_lo, m->st));
   MCK(gemm_launch(m->p_d, nullptr, m->d_status, m->st, nullptr, true));
   MCK(launch_k(moe_readout_kernel, dim3((H / 4 + 255) / 256, m->B), dim3(256), 0, m->st, true, m->p_d.out(), H, y));
   return CORUN_OK;

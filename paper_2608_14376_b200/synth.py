@@ -142,6 +142,56 @@ def weights_torch_to_numpy(w: dict) -> dict:
     return {k: ([cv(x) for x in v] if isinstance(v, list) else cv(v)) for k, v in w.items()}
 
 
+def make_moe_numpy(sh: ModelShape, n_experts: int, top_k: int, expert_ffn: int, n_shared: int, renormalize: bool = False,
+                   seed: int = 0, std: float = 0.02, router_std: float = 0.2) -> dict:
+    """Mixture-of-Experts feed-forward layers as numpy uint16 (bf16 bits): per layer router [E, H],
+    gate_up [(E+S)*2F, H] (block e = expert e: gate rows then up rows) and down [H, (E+S)*F]."""
+    rng = np.random.Generator(np.random.PCG64(seed + 77))
+    nb = n_experts + n_shared
+    m = dict(n_experts=n_experts, top_k=top_k, expert_ffn=expert_ffn, n_shared=n_shared, renormalize=renormalize,
+             router=[], gate_up=[], down=[])
+    for _ in range(sh.n_layers):
+        m["router"].append(f32_to_bf16_bits(rng.standard_normal((n_experts, sh.hidden), dtype=np.float32) * np.float32(router_std)))
+        m["gate_up"].append(f32_to_bf16_bits(rng.standard_normal((nb * 2 * expert_ffn, sh.hidden), dtype=np.float32) * np.float32(std)))
+        m["down"].append(f32_to_bf16_bits(rng.standard_normal((sh.hidden, nb * expert_ffn), dtype=np.float32) * np.float32(std)))
+    return m
+
+
+def moe_numpy_to_torch(m: dict, device="cuda") -> dict:
+    import torch
+
+    def cv(a):
+        return torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16).to(device)
+
+    return {k: ([cv(x) for x in v] if isinstance(v, list) else v) for k, v in m.items()}
+
+
+def make_moe_torch(sh: ModelShape, n_experts: int, top_k: int, expert_ffn: int, n_shared: int, renormalize: bool = False,
+                   seed: int = 0, std: float = 0.02, router_std: float = 0.2, device="cuda") -> dict:
+    """The same layers drawn on the device (for shapes too large for the host)."""
+    import torch
+
+    g = torch.Generator(device=device)
+    g.manual_seed(seed + 77)
+    nb = n_experts + n_shared
+    m = dict(n_experts=n_experts, top_k=top_k, expert_ffn=expert_ffn, n_shared=n_shared, renormalize=renormalize,
+             router=[], gate_up=[], down=[])
+
+    def draw(shape, sd):
+        t = torch.empty(shape, dtype=torch.bfloat16, device=device)
+        rows = max(1, (1 << 27) // shape[1])
+        for r0 in range(0, shape[0], rows):
+            r1 = min(shape[0], r0 + rows)
+            t[r0:r1] = (torch.randn((r1 - r0, shape[1]), generator=g, device=device, dtype=torch.float32) * sd).to(torch.bfloat16)
+        return t
+
+    for _ in range(sh.n_layers):
+        m["router"].append(draw((n_experts, sh.hidden), router_std))
+        m["gate_up"].append(draw((nb * 2 * expert_ffn, sh.hidden), std))
+        m["down"].append(draw((sh.hidden, nb * expert_ffn), std))
+    return m
+
+
 def make_prompts(vocab: int, lengths, seed: int) -> list:
     rng = np.random.Generator(np.random.PCG64(seed))
     return [rng.integers(0, vocab, size=int(n), dtype=np.int64).astype(np.int32) for n in lengths]
