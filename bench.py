@@ -35,7 +35,10 @@ WORKLOADS = {
     # name: (shape, B, n_active, ctx_lo, ctx_hi, temperature, top_p, kv std)
     "qwen3_8b_b64": (synth.QWEN3_8B, 64, 40, 512, 4096, 0.7, 0.95, 1.28),
     "tiny_b8": (synth.TINY, 8, 5, 16, 64, 0.7, 0.95, 0.3),
+    # Mixture-of-Experts decoder (Qwen3-30B-A3B shape); no CPU baseline (the weights do not fit the host leg)
+    "qwen3_30b_a3b_b64": (synth.QWEN3_30B_A3B, 64, 40, 512, 4096, 0.7, 0.95, 1.28),
 }
+MOE = {"qwen3_30b_a3b_b64": (synth.QWEN3_30B_A3B_MOE, synth.QWEN3_30B_A3B_EFF)}
 
 
 def measured_peaks():
@@ -156,6 +159,10 @@ def run_reference(args, rank, world):
         return
     import torch
 
+    if args.workload in MOE:
+        print(json.dumps({"impl": "reference", "unavailable": "the oracle of this Mixture-of-Experts workload needs its "
+                          "60 GB of weights in host memory; its parity is tested on small shapes"}))
+        return
     sh, B, slots, ctx, T, P, kv_std = workload_inputs(args.workload)
     w_t = make_weights(sh, "cuda" if torch.cuda.is_available() else "cpu")
     w_np = synth.weights_torch_to_numpy(w_t)
@@ -196,9 +203,16 @@ def run_corun(args, rank, world):
     K, W = args.steps, args.warmup
     total_steps = 2 * (K + W) + 8
     max_ctx = -(-(int(ctx.max()) + total_steps + 16) // 256) * 256
-    w_t = make_weights(sh, "cuda")
+    moe_cfg = MOE.get(args.workload)
     stream = torch.cuda.Stream()
-    eng = corun.Engine(sh, w_t, B, max_ctx, stream=stream.cuda_stream)
+    if moe_cfg:
+        w_t = synth.make_weights_torch(sh, seed=0, device="cuda", dense_ffn=False)
+        m_t = synth.make_moe_torch(sh, seed=0, device="cuda", **moe_cfg[0])
+        eng = corun.Engine(sh, w_t, B, max_ctx, stream=stream.cuda_stream, moe=m_t)
+        sh = moe_cfg[1]                               # byte counts below: the feed-forward width the row program sees
+    else:
+        w_t = make_weights(sh, "cuda")
+        eng = corun.Engine(sh, w_t, B, max_ctx, stream=stream.cuda_stream)
     for i, (s, c) in enumerate(zip(slots, ctx)):
         eng.adopt(int(s), 0, int(c) + total_steps, pending=1 + i, temperature=T, top_p=P, step=1)
         eng.kv_fill(int(s), int(c), kv_std, seed=100 + i)
@@ -250,7 +264,7 @@ def run_corun(args, rank, world):
     reps = max(10, min(72, 2 * L))
     kt = {name: eng.time_kernel(i, reps if i != 4 and i != 9 else 10) for i, name in enumerate(eng.KERNEL_KINDS)}
     gemm_ms = L * (kt["gemm_qkv"] + kt["gemm_o"] + kt["gemm_gate_up"] + kt["gemm_down"]) + kt["gemm_lm_head"]
-    n_gemm = 4 * L + 1
+    n_gemm = 4 * L + 1                                 # (the small router GEMMs of an MoE model are left out)
     w_bytes = sh.weight_bytes_per_step()
     cur_ctx = [eng.context_len(int(s)) for s in slots]
     kv_bytes = sum(c * sh.kv_bytes_per_token(2) for c in cur_ctx)
@@ -317,7 +331,7 @@ def run_corun(args, rank, world):
     # ---- the Mixture-of-Experts feed-forward block (DeepSeek-V2-Lite block shape, B = 128 padded rows): time per
     # call with CUDA events against the bytes of expert weights a call streams (rank 0, full-size workload only)
     moe = None
-    if rank == 0 and sh.n_layers > 8:
+    if rank == 0 and sh.n_layers > 8 and not moe_cfg:
         from paper_2608_14376_b200.corun import MoeFfn
         gm = torch.Generator(device="cuda").manual_seed(3)
         mk = lambda *shape: (torch.randn(shape, generator=gm, device="cuda") * 0.02).to(torch.bfloat16).contiguous()
@@ -341,7 +355,7 @@ def run_corun(args, rank, world):
         del op, xm
 
     cpu = None
-    if rank == 0 and not args.no_cpu_baseline:
+    if rank == 0 and not args.no_cpu_baseline and not moe_cfg:
         w_np = synth.weights_torch_to_numpy(w_t)
         n_s = 2 if sh.n_layers > 8 else len(slots)
         sample = [int(c) for c in ctx[:n_s]]

@@ -57,6 +57,13 @@ class ModelShape:
 
 TINY = ModelShape(2, 256, 4, 2, 64, 768, 2048, 1e-6, 10000.0)
 QWEN3_8B = ModelShape(36, 4096, 32, 8, 128, 12288, 151936, 1e-6, 1000000.0)
+# Qwen3-30B-A3B-shaped Mixture-of-Experts decoder: 48 layers, hidden 2048, 32 q / 4 kv heads of 128, 128 experts
+# of 768 (top-8, renormalised, no shared expert).  `ffn` of the attention shape is a placeholder (the dense
+# feed-forward weights are not made); QWEN3_30B_A3B_EFF carries the feed-forward width the row program sees,
+# (E + S) * F, for byte counts.
+QWEN3_30B_A3B = ModelShape(48, 2048, 32, 4, 128, 64, 151936, 1e-6, 1000000.0)
+QWEN3_30B_A3B_MOE = dict(n_experts=128, top_k=8, expert_ffn=768, n_shared=0, renormalize=True)
+QWEN3_30B_A3B_EFF = ModelShape(48, 2048, 32, 4, 128, 128 * 768, 151936, 1e-6, 1000000.0)
 
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
@@ -98,15 +105,18 @@ def make_weights_numpy(sh: ModelShape, seed: int = 0, std: float = 0.02) -> dict
     return w
 
 
-def make_weights_torch(sh: ModelShape, seed: int = 0, std: float = 0.02, device="cuda") -> dict:
+def make_weights_torch(sh: ModelShape, seed: int = 0, std: float = 0.02, device="cuda", dense_ffn: bool = True) -> dict:
     """Weights as torch bf16 tensors drawn on ``device`` (same recipe; the
-    stream differs from the numpy one, so use one generator per experiment)."""
+    stream differs from the numpy one, so use one generator per experiment).
+    ``dense_ffn`` False leaves out wgate_up / wdown (Mixture-of-Experts models bring their own)."""
     import torch
 
     g = torch.Generator(device=device)
     g.manual_seed(seed)
     w = {"attn_norm": [], "mlp_norm": [], "wqkv": [], "wo": [], "wgate_up": [], "wdown": []}
     for name, l, shape in _tensor_list(sh):
+        if not dense_ffn and name in ("wgate_up", "wdown"):
+            continue
         t = torch.empty(shape, dtype=torch.bfloat16, device=device)
         rows = max(1, (1 << 27) // shape[1])  # draw in slabs so the fp32 staging stays small
         for r0 in range(0, shape[0], rows):
