@@ -169,7 +169,8 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm) {
       const int NB = e->moe_E + e->moe_S;
       RC(dmalloc(A, &P.r_out, (size_t)R * GEMM_TILE_N));
       RC(dmalloc(A, &P.moe_w, (size_t)R * NB));
-      RC(gemm_plan_create(&P.p_r, e->router_pad, GEMM_TILE_N, H, P.xn_hi, P.xn_lo, R, P.BN, P.r_out, P.ws, e->num_sms));
+      // few CTAs: the router's weights are small, and the routing kernel adds one partial per CTA for every logit
+      RC(gemm_plan_create(&P.p_r, e->router_pad, GEMM_TILE_N, H, P.xn_hi, P.xn_lo, R, P.BN, P.r_out, P.ws, 8));
       if ((2 * e->moe_F) % GEMM_TILE_N == 0) {      // a weight tile belongs to one expert: rows that did not
         P.p_gu.row_keep = P.moe_w;                  // select it are not stored (the SwiGLU does not read them)
         P.p_gu.keep_pitch = NB;

@@ -224,7 +224,7 @@ int corun_moe_create(const corun_moe_shape *shape, const void *router, const voi
   if (cudaMemcpy(m->router_pad, router, (size_t)E * H * sizeof(bf16), cudaMemcpyDeviceToDevice) != cudaSuccess)
     return fail(CORUN_ECUDA);
   // the three GEMMs run one after the other and their results are consumed in between: one workspace serves all
-  if ((rc = gemm_plan_create(&m->p_r, m->router_pad, GEMM_TILE_N, H, m->x_hi, m->x_lo, B, m->BN, m->out_r, m->ws, m->num_sms)) ||
+  if ((rc = gemm_plan_create(&m->p_r, m->router_pad, GEMM_TILE_N, H, m->x_hi, m->x_lo, B, m->BN, m->out_r, m->ws, 8)) ||
       (rc = gemm_plan_create(&m->p_gu, gate_up, (int)N1, H, m->x_hi, m->x_lo, B, m->BN, m->out_gu, m->ws, m->num_sms)) ||
       (rc = gemm_plan_create(&m->p_d, down, H, (int)K2, m->h_hi, m->h_lo, B, m->BN, m->out_d, m->ws, m->num_sms)))
     return fail(rc);
