@@ -90,3 +90,47 @@ def test_moe_engine_parity_and_invariance(orc, E, K, F, S, renorm):
             assert eng.logits(2).tobytes() == trace[step][0]
     finally:
         eng.close()
+
+
+def test_moe_engine_served_together_equals_served_alone(orc):
+    """The paper's validation protocol on the MoE decoder: requests served together (sampled, through the host
+    scheduler with a pool too small for all of them) produce, bit for bit, the tokens of each served alone."""
+    from paper_2608_14376_b200 import corun
+
+    sh, model, eng0 = _setup(orc, 8, 2, 128, 1, False, seed=5)
+    eng0.close()
+    w_np = synth.make_weights_numpy(sh, seed=5)
+    m_np = synth.make_moe_numpy(sh, 8, 2, 128, 1, False, seed=5)
+    eng = corun.Engine(sh, synth.weights_numpy_to_torch(w_np, "cuda"), B, 128, kv_pool_blocks=24,
+                       moe=synth.moe_numpy_to_torch(m_np, "cuda"))
+    try:
+        rng = np.random.default_rng(2)
+        lens = synth.uniform_lengths(8, 70, 14, seed=8)
+        prompts = synth.make_prompts(sh.vocab, lens, seed=9)
+        reqs = [dict(prompt=p, max_new=int(rng.integers(2, 12)), seed=synth.request_seed(50 + i)) for i, p in enumerate(prompts)]
+
+        def serve(subset, batched=False):
+            sch = corun.Scheduler(engine=eng)
+            if batched:
+                sch.enable_batched_prefill()
+            ids = [sch.submit(r["prompt"], r["max_new"], 0.8, 0.9, r["seed"]) for r in subset]
+            shared = 0
+            while True:
+                action, _, n = sch.step()
+                shared += action == corun.SCHED_DECODE and n >= 3
+                if action == corun.SCHED_IDLE:
+                    break
+            out = [sch.poll(i)[0] for i in ids]
+            sch.close()
+            return out, shared
+
+        together, shared = serve(reqs)
+        assert shared > 0 and eng.free_blocks() == 24
+        batched, _ = serve(reqs, batched=True)
+        for r, a, b in zip(reqs, together, batched):
+            alone, _ = serve([r])
+            assert len(a) == r["max_new"]
+            np.testing.assert_array_equal(alone[0], a)
+            np.testing.assert_array_equal(b, a)
+    finally:
+        eng.close()
