@@ -152,7 +152,7 @@ def case_moe(a):
     op = corun.MoeFfn(H, E, K, F, S, router, gate_up, down, a.B, renormalize=a.renormalize)
     x = torch.randn((a.B, H), generator=g, device="cuda")
     for _ in range(3):
-        y, ex, pr = op.forward(x)
+        y, ex, _ = op.forward(x)
     op.sync()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
