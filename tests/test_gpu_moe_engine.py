@@ -136,3 +136,77 @@ def test_moe_engine_served_together_equals_served_alone(orc):
             np.testing.assert_array_equal(b, a)
     finally:
         eng.close()
+
+
+def test_moe_engine_at_the_qwen3_30b_a3b_layer_shape(orc):
+    """Full layer width of the workload bench.py times for the MoE decoder (hidden 2048, 32 q / 4 kv heads of
+    128, 128 experts of 768, top-8 renormalised, B = 64), two layers deep with a 4096-token vocabulary so that
+    the oracle can follow: one decode step over synthetic cache rows against the oracle, then the same
+    requests in other slots among other co-tenants, byte for byte."""
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    if torch.cuda.get_device_properties(0).total_memory < 40e9:
+        pytest.skip("needs a large-memory GPU")
+    from paper_2608_14376_b200 import corun
+
+    sh = synth.ModelShape(2, 2048, 32, 4, 128, 64, 4096, 1e-6, 1e6)
+    cfg = dict(synth.QWEN3_30B_A3B_MOE)
+    w_t = synth.make_weights_torch(sh, seed=0, device="cuda", dense_ffn=False)
+    m_t = synth.make_moe_torch(sh, seed=0, device="cuda", **cfg)
+    w_np = synth.weights_torch_to_numpy({k: v for k, v in w_t.items() if k not in ("wgate_up", "wdown")})
+    w_np["wgate_up"] = [np.zeros((128, sh.hidden), np.uint16)] * sh.n_layers     # unused placeholders
+    w_np["wdown"] = [np.zeros((sh.hidden, 64), np.uint16)] * sh.n_layers
+    m_np = dict(cfg, **{k: [t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16) for t in m_t[k]]
+                        for k in ("router", "gate_up", "down")})
+    model = orc.Model(orc.Shape(**sh.dict()), w_np, moe=m_np)
+    Bq, max_ctx = 64, 2304
+    eng = corun.Engine(sh, w_t, Bq, max_ctx, moe=m_t)
+    try:
+        rng = np.random.default_rng(12)
+        ctxs = [2000, 700, 129]
+        reqs = []
+        for i, n_ctx in enumerate(ctxs):
+            cache = model.new_cache(n_ctx + 2)
+            kv = []
+            for layer in range(sh.n_layers):
+                k, v = synth.synthetic_kv(n_ctx, sh.kv_dim, 1.28, seed=900 + 10 * i + layer)
+                cache[0][layer, :n_ctx], cache[1][layer, :n_ctx] = k, v
+                kv.append((k, v))
+            reqs.append(dict(ctx=n_ctx, kv=kv, cache=cache, pending=41 + 17 * i))
+
+        def place(slot, r):
+            eng.adopt(slot, 0, r["ctx"] + 2, pending=r["pending"], temperature=0.7, top_p=0.95, step=1)
+            for layer, (k, v) in enumerate(r["kv"]):
+                eng.kv_write(slot, layer, 0, k, v)
+
+        slots = [3, 40, 63]
+        for s, r in zip(slots, reqs):
+            place(s, r)
+        active = np.zeros(Bq, np.uint8); active[slots] = 1
+        seeds = np.zeros(Bq, np.uint64)
+        eng.decode_step(active, seeds)
+        worst = 0.0
+        for s, r in zip(slots, reqs):
+            ref = model.forward([r["pending"]], r["ctx"], r["cache"])
+            lg = eng.logits(s)
+            worst = max(worst, float(np.abs(lg - ref).max()))
+            r["bytes"] = lg.tobytes()
+        assert worst <= TOL, worst
+        for s in slots:
+            eng.release(s)
+        # other slots, 20 co-tenants with device-generated cache rows
+        slots2 = [17, 0, 31]
+        for s, r in zip(slots2, reqs):
+            place(s, r)
+        others = [s for s in rng.permutation(Bq) if s not in slots2][:20]
+        for j, s in enumerate(others):
+            n_ctx = int(rng.integers(64, 2000))
+            eng.adopt(int(s), 0, n_ctx + 2, pending=int(rng.integers(0, sh.vocab)), temperature=0.7, top_p=0.95)
+            eng.kv_fill(int(s), n_ctx, 1.28, seed=7000 + j)
+        active = np.zeros(Bq, np.uint8); active[slots2] = 1; active[others] = 1
+        eng.decode_step(active, seeds)
+        for s, r in zip(slots2, reqs):
+            assert eng.logits(s).tobytes() == r["bytes"]
+    finally:
+        eng.close()
