@@ -319,14 +319,26 @@ def run_corun(args, rank, world):
             tf_s = float(json.load(open(pk)).get("bf16_tflops_sustained", tf))
         t_roof = w_lm / (hbm * 1e9)
         left = n_pf
+        # Mixture-of-Experts layers (grouped form in prefill): a row meets top_k of the experts only, so the MMA
+        # work per row is that of the attention projections plus top_k experts; every expert's weights are still
+        # streamed once per chunk
+        w_mma = w_layers
+        if moe_cfg:
+            mc = moe_cfg[0]
+            w_exp = 2 * 3 * sh.hidden * mc["expert_ffn"] * sh.n_layers      # bytes of one expert over all layers
+            w_mma = w_layers - (mc["n_experts"] - mc["top_k"]) * w_exp
+        t_mma = t_hbm = 0.0
         while left > 0:
             rows = min(256, left)
-            t_roof += max(2 * 2 * (w_layers // 2) * rows / (tf_s * 1e12), w_layers / (hbm * 1e9))
+            t_mma += 2 * 2 * (w_mma // 2) * rows / (tf_s * 1e12)
+            t_hbm += w_layers / (hbm * 1e9)
+            t_roof += max(2 * 2 * (w_mma // 2) * rows / (tf_s * 1e12), w_layers / (hbm * 1e9))
             left -= rows
         prefill = {"tokens": n_pf, "ms": dt * 1e3, "tok_per_s": n_pf / dt, "roofline_ms": t_roof * 1e3,
-                   "frac": t_roof / dt, "bound": "tensor",
-                   "note": "executed MMA work counted (activations are a bf16 hi/lo pair: two MMAs per weight tile) at "
-                           "%.0f TFLOP/s sustained; attention not counted" % tf_s}
+                   "frac": t_roof / dt, "bound": "tensor" if t_mma >= t_hbm else "hbm",
+                   "note": "per 256-token chunk the larger of the executed MMA work (activations are a bf16 hi/lo pair: "
+                           "two MMAs per weight tile; %.0f TFLOP/s sustained) and the layers' weights streamed once; "
+                           "attention not counted" % tf_s}
 
     # ---- the Mixture-of-Experts feed-forward block (DeepSeek-V2-Lite block shape, B = 128 padded rows): time per
     # call with CUDA events against the bytes of expert weights a call streams (rank 0, full-size workload only)

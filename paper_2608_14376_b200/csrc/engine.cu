@@ -49,6 +49,13 @@ struct Program {
   // and over the concatenated hidden activations; p_r is the router GEMM (its rows padded to one tile)
   GemmPlan p_r;
   float *r_out = nullptr, *moe_w = nullptr;
+  // grouped form of the experts' GEMMs (prefill chunks: the rows of an expert gathered into blocks of 64)
+  bool grouped = false;
+  MoeGroups grp{};
+  GemmPlan p_gug, p_dng;
+  bf16 *xg_hi = nullptr, *xg_lo = nullptr, *hg_hi = nullptr, *hg_lo = nullptr;
+  float *gug_out = nullptr, *yg_out = nullptr;
+  int *plain_tiles = nullptr;            // zeros: the table that makes a plain matrix readable as a GEMM result
   bool has_layers = false, has_lm = false;
   std::vector<void *> allocs;
 };
@@ -126,7 +133,7 @@ int dmalloc(std::vector<void *> &keep, T **p, size_t n, bool zero = true) {
 
 int pad16(int x) { return (x + 15) / 16 * 16; }
 
-int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm) {
+int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, bool grouped = false) {
   const corun_shape &s = e->sh;
   const int H = s.hidden, QD = s.n_q_heads * s.head_dim, KD = s.n_kv_heads * s.head_dim, F = s.ffn, V = s.vocab;
   P.R = R;
@@ -176,6 +183,31 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm) {
         P.p_gu.keep_pitch = NB;
         P.p_gu.keep_div = 2 * e->moe_F / GEMM_TILE_N;
       }
+      if (grouped && (2 * e->moe_F) % GEMM_TILE_N == 0 && H % GEMM_TILE_N == 0) {
+        // prefill chunks: every row through every expert would be (E + S) / top_k times the MMA work, which a
+        // chunk of 256 rows does pay for; the rows of an expert are gathered into blocks of 64 instead
+        const int Fm = e->moe_F;
+        MoeGroups &g = P.grp;
+        g.n_groups_max = moe_max_groups(R, e->moe_E, e->moe_S, e->moe_K);
+        const size_t slots = (size_t)g.n_groups_max * MOE_GROUP_ROWS;
+        RC(dmalloc(A, &g.tab_up, (size_t)g.n_groups_max * 3));
+        RC(dmalloc(A, &g.tab_down, (size_t)g.n_groups_max * 3));
+        RC(dmalloc(A, &g.group_expert, (size_t)g.n_groups_max));
+        RC(dmalloc(A, &g.slot_row, slots));
+        RC(dmalloc(A, &g.slot_of, (size_t)R * NB));
+        RC(dmalloc(A, &P.xg_hi, slots * H));
+        RC(dmalloc(A, &P.xg_lo, slots * H));
+        RC(dmalloc(A, &P.hg_hi, slots * Fm));
+        RC(dmalloc(A, &P.hg_lo, slots * Fm));
+        RC(dmalloc(A, &P.gug_out, slots * 2 * Fm));
+        RC(dmalloc(A, &P.yg_out, slots * H));
+        RC(dmalloc(A, &P.plain_tiles, (size_t)(H / GEMM_TILE_N + 1)));
+        RC(gemm_plan_create_grouped(&P.p_gug, e->w0_gu, (long long)NB * 2 * Fm, H, 2 * Fm, H, P.xg_hi, P.xg_lo, g.n_groups_max,
+                                    MOE_GROUP_ROWS, P.gug_out, g.tab_up));
+        RC(gemm_plan_create_grouped(&P.p_dng, e->w0_down, H, NB * Fm, H, Fm, P.hg_hi, P.hg_lo, g.n_groups_max, MOE_GROUP_ROWS,
+                                    P.yg_out, g.tab_down));
+        P.grouped = true;
+      }
     }
   }
   if (lm) {
@@ -192,6 +224,8 @@ void program_destroy(Program &P) {
   gemm_plan_destroy(&P.p_down);
   gemm_plan_destroy(&P.p_lm);
   gemm_plan_destroy(&P.p_r);
+  gemm_plan_destroy(&P.p_gug);
+  gemm_plan_destroy(&P.p_dng);
   for (void *p : P.allocs) cudaFree(p);
   P.allocs.clear();
 }
@@ -199,6 +233,13 @@ void program_destroy(Program &P) {
 KvLayout kv_layout(const corun_engine *e) {
   return KvLayout{e->kv_pool, e->d_block_table, e->max_blocks, e->sh.n_kv_heads, e->sh.head_dim, e->layer_stride,
                   (long long)e->pool_blocks};
+}
+
+// The result of a layer's feed-forward part as the next kernel reads it: the down GEMM's partials, or (grouped
+// Mixture-of-Experts form) the combined plain matrix.
+GemmOut ffn_out(const Program &P) {
+  if (P.grouped) return GemmOut{P.down_out, nullptr, P.plain_tiles, P.plain_tiles, P.p_down.N, P.p_down.KB, P.BN};
+  return P.p_down.out();
 }
 
 // Enqueues embed -> all layers (ends with the last down GEMM).  Counts launches.
@@ -224,7 +265,7 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
     ++stage;                                          \
   } while (0)
   for (int l = 0; l < s.n_layers; ++l) {
-    GemmOut prev = P.p_down.out();
+    GemmOut prev = ffn_out(P);
     STAGE(launch_resid_norm(P.h, s.hidden, e->embed, rows, l == 0 ? nullptr : &prev, e->attn_norm[l], s.rms_eps,
                             P.xn_hi, P.xn_lo, e->st));
     STAGE(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, tr(4 * l + 0), true));
@@ -235,7 +276,21 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
     STAGE(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st, tr(4 * l + 1), true));
     GemmOut o = P.p_o.out();
     STAGE(launch_resid_norm(P.h, s.hidden, nullptr, rows, &o, e->mlp_norm[l], s.rms_eps, P.xn_hi, P.xn_lo, e->st));
-    if (e->moe_E) {
+    if (e->moe_E && P.grouped) {
+      // router -> top-k weights -> rows grouped by expert -> gate / up, SwiGLU and down per group -> the row's
+      // experts summed in ascending expert id
+      const int NB = e->moe_E + e->moe_S;
+      STAGE(gemm_launch(P.p_r, &e->tm_router[l], e->d_status, e->st, nullptr, true));
+      STAGE(launch_moe_route(P.p_r.out(), P.R, e->moe_E, e->moe_S, e->moe_K, e->moe_renorm, P.moe_w, nullptr, nullptr, e->st));
+      STAGE(launch_moe_group(P.moe_w, P.row_active, P.R, e->moe_E, e->moe_S, e->moe_F, P.grp, e->st));
+      STAGE(launch_moe_gather(P.xn_hi, P.xn_lo, s.hidden, P.grp, P.xg_hi, P.xg_lo, e->st));
+      STAGE(gemm_launch(P.p_gug, &e->tm_gu[l], e->d_status, e->st, nullptr, true));
+      STAGE(launch_moe_swiglu_grouped(P.gug_out, P.moe_w, NB, e->moe_F, P.grp, P.hg_hi, P.hg_lo, e->st));
+      STAGE(gemm_launch(P.p_dng, &e->tm_down[l], e->d_status, e->st, nullptr, true));
+      STAGE(launch_moe_combine(P.yg_out, P.row_active, P.R, NB, s.hidden, P.grp, P.down_out, e->st));
+      n += 14;
+      continue;
+    } else if (e->moe_E) {
       // router -> top-k weights -> all experts' gate / up (rows that did not select a tile's expert are not
       // stored) -> masked, weighted SwiGLU; the down GEMM then sums over the row's experts in its accumulator
       STAGE(gemm_launch(P.p_r, &e->tm_router[l], e->d_status, e->st, nullptr, true));
@@ -268,7 +323,7 @@ int enqueue_decode_body(corun_engine *e, int *launches) {
   RC(run_layers(e, P, &n));
   if (!(e->eager && e->stop_after >= 0)) {   // (debug) a truncated layer stack skips the tail too
     const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
-    GemmOut prev = P.p_down.out();
+    GemmOut prev = ffn_out(P);
     CK(launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->final_norm, s.rms_eps, P.xn_hi, P.xn_lo, e->st));
     CK(gemm_launch(P.p_lm, nullptr, e->d_status, e->st, nullptr, true));
     CK(gemm_fixup_launch(P.p_lm, e->st, true));
@@ -517,7 +572,7 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
     if (atoi(ts) != 0 && (rc = dmalloc(A, &e->step_trace, (size_t)4 * s.n_layers * e->num_sms * 8))) return fail(rc);
   }
   if ((rc = program_create(e, e->dec, B, true, true))) return fail(rc);
-  if ((rc = program_create(e, e->pre, e->chunk, true, false))) return fail(rc);
+  if ((rc = program_create(e, e->pre, e->chunk, true, false, e->moe_E > 0 && !getenv("CORUN_MOE_PREFILL_DENSE")))) return fail(rc);
   if ((rc = program_create(e, e->lm1, 1, false, true))) return fail(rc);
 
   // the allocations above were cleared and filled through the legacy stream, which the engine's
@@ -585,9 +640,9 @@ struct PfReq {
 int prefill_finish_row(corun_engine *e, int row, PfReq &r) {
   const corun_shape &s = e->sh;
   Program &P = e->pre, &L = e->lm1;
-  GemmOut prev = P.p_down.out();
+  GemmOut prev = ffn_out(P);
   prev.direct += (size_t)row * prev.N;
-  prev.ws += (size_t)row * GEMM_TILE_N;
+  if (prev.ws) prev.ws += (size_t)row * GEMM_TILE_N;
   const Rows one{P.row_token + row, P.row_pos + row, P.row_active + row, P.row_slot + row, 1};
   CK(launch_resid_norm(P.h + (size_t)row * s.hidden, s.hidden, nullptr, one, &prev, e->final_norm, s.rms_eps, L.xn_hi,
                        L.xn_lo, e->st));
@@ -925,7 +980,7 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
     cudaError_t ce = cudaEventRecord(a, e->st);
     for (int i = 0; i < n && ce == cudaSuccess; ++i) {
       const int l = i % s.n_layers;   // rotate over the layers so that L2 cannot hold the weights
-      GemmOut prev = P.p_down.out();
+      GemmOut prev = ffn_out(P);
       switch (kind) {
         // launched as in the step's graph: with programmatic stream serialization
         case 0: ce = gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, nullptr, true); break;

@@ -33,13 +33,27 @@ constexpr uint32_t A_BLOCK_BYTES = GEMM_ROW_BLOCK * GEMM_BLOCK_K * 2;      // 16
 // meaningless values that are never read back.
 // MASKED: the optional store mask of the epilogue (a separate instantiation, so that the plain kernel is
 // exactly the code it was without it).
-template <bool MASKED, bool STACKED>
+// GROUPED (with STACKED): every CTA owns one whole output tile of one group (an expert's rows, gathered into
+// blocks of BN rows).  group_tab holds, per group, the first weight row, the first weight k-block and the number
+// of rows (0 = the group is empty: its CTAs leave at once); the group's activations are rows group * BN .. of
+// the activation matrices, its output rows group * BN .. of `direct` (N columns wide, tiles_per_group tiles).
+template <bool MASKED, bool STACKED, bool GROUPED>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmHi,
                     const __grid_constant__ CUtensorMap tmLo, float *__restrict__ direct, float *__restrict__ ws,
                     const int *__restrict__ cta_start, int N, int KB, int BN, int R, int stages, int tmem_cols,
-                    uint32_t idesc, const float *row_keep, int keep_pitch, int keep_div, int *status,
-                    unsigned long long *trace) {
+                    uint32_t idesc, const float *row_keep, int keep_pitch, int keep_div, const int *group_tab,
+                    int tiles_per_group, int *status, unsigned long long *trace) {
+  int g_id = 0, g_j = 0, g_wrow = 0, g_wk = 0, g_rows = 0;
+  if (GROUPED) {
+    griddep_wait();                                 // the group table comes from an earlier kernel
+    g_id = (int)blockIdx.x / tiles_per_group;
+    g_j = (int)blockIdx.x - g_id * tiles_per_group;
+    g_wrow = group_tab[3 * g_id];
+    g_wk = group_tab[3 * g_id + 1];
+    g_rows = group_tab[3 * g_id + 2];
+    if (g_rows <= 0) return;                        // the same decision in every thread of the CTA
+  }
   extern __shared__ uint8_t smem_raw[];
   // optional per-CTA timeline (debug): 8 globaltimer stamps
 #define TRACE(i) do { if (trace) trace[(size_t)blockIdx.x * 8 + (i)] = globaltimer_ns(); } while (0)
@@ -112,7 +126,8 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const int g = k0 + it, tile = g / KB, kb = g - tile * KB;
         const uint32_t fb = smem_u32(&full_bar[it]);
         mbar_arrive_expect_tx(fb, tx_bytes);
-        tma_load_2d(tiles_base + (uint32_t)it * stage_bytes, &tmW, kb * GEMM_BLOCK_K, tile * GEMM_TILE_N, fb, pol_w);
+        tma_load_2d(tiles_base + (uint32_t)it * stage_bytes, &tmW, (GROUPED ? g_wk + kb : kb) * GEMM_BLOCK_K,
+                    GROUPED ? g_wrow + g_j * GEMM_TILE_N : tile * GEMM_TILE_N, fb, pol_w);
         if (it == 0) TRACE(2);
       }
       griddep_wait();
@@ -120,8 +135,8 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const int g = k0 + it, tile = g / KB, kb = g - tile * KB;
         const uint32_t fb = smem_u32(&full_bar[it]);
         const uint32_t dst = tiles_base + (uint32_t)it * stage_bytes;
-        tma_load_2d(dst + W_TILE_BYTES, &tmHi, kb * GEMM_BLOCK_K, 0, fb, pol_x);
-        tma_load_2d(dst + W_TILE_BYTES + lo_off, &tmLo, kb * GEMM_BLOCK_K, 0, fb, pol_x);
+        tma_load_2d(dst + W_TILE_BYTES, &tmHi, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
+        tma_load_2d(dst + W_TILE_BYTES + lo_off, &tmLo, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
       }
       int it = n_pre;
       for (int g = k0 + n_pre; g < k1; ++g, ++it) {
@@ -132,9 +147,10 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const uint32_t fb = smem_u32(&full_bar[s]);
         const uint32_t dst = tiles_base + (uint32_t)s * stage_bytes;
         mbar_arrive_expect_tx(fb, tx_bytes);
-        tma_load_2d(dst, &tmW, kb * GEMM_BLOCK_K, tile * GEMM_TILE_N, fb, pol_w);
-        tma_load_2d(dst + W_TILE_BYTES, &tmHi, kb * GEMM_BLOCK_K, 0, fb, pol_x);
-        tma_load_2d(dst + W_TILE_BYTES + lo_off, &tmLo, kb * GEMM_BLOCK_K, 0, fb, pol_x);
+        tma_load_2d(dst, &tmW, (GROUPED ? g_wk + kb : kb) * GEMM_BLOCK_K, GROUPED ? g_wrow + g_j * GEMM_TILE_N : tile * GEMM_TILE_N,
+                    fb, pol_w);
+        tma_load_2d(dst + W_TILE_BYTES, &tmHi, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
+        tma_load_2d(dst + W_TILE_BYTES + lo_off, &tmLo, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
       }
       TRACE(3);
     }
@@ -202,7 +218,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       if (!ok) { fail = DEV_TIMEOUT_EPILOGUE; break; }
       tc_fence_after();
       if (g + (kb_end - kb_begin) >= k1 && threadIdx.x == 64) TRACE(6);   // last accumulator is ready
-      const int n0 = tile * GEMM_TILE_N;
+      const int n0 = GROUPED ? g_j * GEMM_TILE_N : tile * GEMM_TILE_N;
       // optional: rows whose entry for this tile's column group is zero are not stored (nobody reads them)
       const float *keep = MASKED ? row_keep + tile / keep_div : nullptr;
       if (stacked) {
@@ -211,11 +227,12 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         // the two halves and store whole 128-byte row segments (four rows per warp instruction)
         const bool lo_warp = lane_base >= 64;
         const int row = (lane_base & 63) + lane;
-        const int rows_valid = whole ? R : BN;
+        const int rows_valid = GROUPED ? g_rows : (whole ? R : BN);
         const bool warp_needed = (lane_base & 63) < rows_valid;   // warp-uniform
         float *xs = xch[lo_warp ? 1 : 0] + row * 33;
         const int te = (int)threadIdx.x - 64, srow = te >> 3, scol = (te & 7) * 4;
-        float *dst0 = whole ? direct + n0 : ws + (size_t)(cta * 2 + (seg == 0 ? 0 : 1)) * BN * GEMM_TILE_N;
+        float *dst0 = GROUPED ? direct + (size_t)g_id * BN * N + n0
+                              : (whole ? direct + n0 : ws + (size_t)(cta * 2 + (seg == 0 ? 0 : 1)) * BN * GEMM_TILE_N);
         const size_t pitch = whole ? (size_t)N : (size_t)GEMM_TILE_N;
         const bool vec_ok = whole ? ((N & 3) == 0) : true;
         for (int c0 = 0; c0 < GEMM_TILE_N; c0 += 32) {
@@ -425,11 +442,52 @@ int gemm_plan_create(GemmPlan *p, const void *W, int N, int K, const void *Xhi, 
   return CORUN_OK;
 }
 
+int gemm_plan_create_grouped(GemmPlan *p, const void *W, long long w_rows, int w_cols, int N, int K, const void *Xhi,
+                             const void *Xlo, int n_groups, int BN, float *direct, const int *group_tab) {
+  if (N <= 0 || N % GEMM_TILE_N || K <= 0 || K % GEMM_BLOCK_K || w_cols % GEMM_BLOCK_K || BN % 16 || BN < 16 || BN > 64 ||
+      n_groups < 1 || !group_tab || w_rows < N)
+    return CORUN_EINVAL;
+  p->N = N; p->K = K; p->R = BN; p->BN = BN;
+  p->n_tiles = n_groups * (N / GEMM_TILE_N);
+  p->KB = K / GEMM_BLOCK_K;
+  p->grid = p->n_tiles;
+  const size_t stage = (size_t)GEMM_TILE_N * GEMM_BLOCK_K * 2 + (size_t)GEMM_ROW_BLOCK * GEMM_BLOCK_K * 2;
+  int stages = (int)((GEMM_MAX_DYN_SMEM - 1024 - A_BLOCK_BYTES) / stage);
+  if (stages > MAX_STAGES) stages = MAX_STAGES;
+  p->stages = stages;
+  p->smem_bytes = stage * stages + A_BLOCK_BYTES + 1024;
+  p->tmem_cols = 512;
+  p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GEMM_TILE_N >> 3) << 17) |
+             ((uint32_t)(GEMM_ROW_BLOCK >> 4) << 24);
+  p->direct = direct;
+  p->ws = nullptr;
+  p->group_tab = group_tab;
+  p->tiles_per_group = N / GEMM_TILE_N;
+  int rc;
+  if ((rc = tma_encode_2d(&p->tmW, W, 0, (unsigned long long)w_rows, w_cols, GEMM_TILE_N, GEMM_BLOCK_K)) != 0) return rc;
+  if ((rc = tma_encode_2d(&p->tmHi, Xhi, 0, (unsigned long long)n_groups * BN, K, BN, GEMM_BLOCK_K)) != 0) return rc;
+  if ((rc = tma_encode_2d(&p->tmLo, Xlo, 0, (unsigned long long)n_groups * BN, K, BN, GEMM_BLOCK_K)) != 0) return rc;
+  // every CTA's range is exactly one tile
+  std::vector<int> tab((size_t)p->grid + 1);
+  for (int c = 0; c <= p->grid; ++c) tab[(size_t)c] = c * p->KB;
+  int *d_tab = nullptr;
+  if (cudaMalloc(&d_tab, tab.size() * sizeof(int)) != cudaSuccess) return CORUN_ENOMEM;
+  cudaError_t me = cudaMemcpy(d_tab, tab.data(), tab.size() * sizeof(int), cudaMemcpyHostToDevice);
+  if (me != cudaSuccess) { g_last_cuda_error = (int)me; cudaFree(d_tab); return CORUN_ECUDA; }
+  p->d_cta_start = d_tab;
+  p->d_tile_first = p->d_tile_cend = p->d_split_tiles = nullptr;
+  p->n_split_tiles = 0;
+  cudaError_t ae = gemm_prepare_kernel();
+  if (ae != cudaSuccess) { g_last_cuda_error = (int)ae; return CORUN_ECUDA; }
+  return CORUN_OK;
+}
+
 cudaError_t gemm_prepare_kernel() {
-  cudaError_t e = cudaFuncSetAttribute(gemm_streamk_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  cudaError_t e = cudaFuncSetAttribute(gemm_streamk_kernel<false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   return e;
 }
 
@@ -444,10 +502,11 @@ cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int 
   auto go = [&](auto kernel) {
     return launch_k(kernel, dim3(p.grid), dim3(GEMM_THREADS), p.smem_bytes, st, pdl, tmW_override ? *tmW_override : p.tmW,
                     p.tmHi, p.tmLo, p.direct, p.ws, p.d_cta_start, p.N, p.KB, p.BN, p.R, p.stages, p.tmem_cols, p.idesc,
-                    p.row_keep, p.keep_pitch, p.keep_div, d_status, trace);
+                    p.row_keep, p.keep_pitch, p.keep_div, p.group_tab, p.tiles_per_group, d_status, trace);
   };
-  if (masked) return stacked ? go(gemm_streamk_kernel<true, true>) : go(gemm_streamk_kernel<true, false>);
-  return stacked ? go(gemm_streamk_kernel<false, true>) : go(gemm_streamk_kernel<false, false>);
+  if (p.group_tab) return go(gemm_streamk_kernel<false, true, true>);
+  if (masked) return stacked ? go(gemm_streamk_kernel<true, true, false>) : go(gemm_streamk_kernel<true, false, false>);
+  return stacked ? go(gemm_streamk_kernel<false, true, false>) : go(gemm_streamk_kernel<false, false, false>);
 }
 
 cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st, bool pdl) {

@@ -86,6 +86,9 @@ struct GemmPlan {
   // row_keep[r * keep_pitch + t / keep_div] != 0 (rows that no consumer will read are skipped).
   const float *row_keep = nullptr;
   int keep_pitch = 0, keep_div = 1;
+  // Grouped mode (gemm_plan_create_grouped): one CTA per (group, weight tile); see gemm.cu.
+  const int *group_tab = nullptr;    // device, not owned: per group (first weight row, first weight k-block, rows)
+  int tiles_per_group = 0;
   GemmOut out() const { return GemmOut{direct, ws, d_tile_first, d_tile_cend, N, KB, BN}; }
 };
 
@@ -98,6 +101,12 @@ inline size_t gemm_ws_floats(int grid, int BN) { return (size_t)grid * 2 * BN * 
 int gemm_plan_create(GemmPlan *p, const void *W, int N, int K, const void *Xhi, const void *Xlo, int R, int BN,
                      float *direct, float *ws, int num_sms);
 void gemm_plan_destroy(GemmPlan *p);
+// Grouped GEMM over at most n_groups groups of up to BN <= 64 rows each: group g multiplies rows g * BN .. of
+// Xhi / Xlo ([n_groups * BN, K]) with N weight rows starting at the row, and K elements starting at the k-block,
+// that group_tab names for it, into rows g * BN .. of `direct` ([n_groups * BN, N]).  W is [w_rows, w_cols]
+// bf16.  One CTA per (group, tile of 256 weight rows), all k-blocks of it: no partials.  N % 256 == 0.
+int gemm_plan_create_grouped(GemmPlan *p, const void *W, long long w_rows, int w_cols, int N, int K, const void *Xhi,
+                             const void *Xlo, int n_groups, int BN, float *direct, const int *group_tab);
 // The allocation-free half of gemm_plan_create: fills every host-side field and tensor map of the
 // plan and writes the partition tables (cta_start, tile_first, tile_cend, split_tiles) to `tab`
 // (capacity tab_cap ints; *tab_ints = ints used).  gemm_plan_bind_tables points the plan at a device

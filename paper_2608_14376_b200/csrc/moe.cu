@@ -144,9 +144,145 @@ __global__ void __launch_bounds__(256) moe_readout_kernel(GemmOut d, int H, floa
   *reinterpret_cast<float4 *>(y + (size_t)r * H + i) = gemm_load4(d, r, i);
 }
 
+// ---------------------------------------------------------------- grouped form (prefill chunks)
+// One CTA of 256 threads (8 warps).  Phase 1: warp per expert counts its rows; phase 2: one thread turns the
+// counts into first-group indices (experts ascending) and clears the tables; phase 3: warp per expert hands
+// its rows, in ascending row order, consecutive slots of its groups.
+__global__ void __launch_bounds__(256) moe_group_kernel(const float *__restrict__ w, const int *__restrict__ active, int R,
+                                                        int NB, int E, int F, MoeGroups g) {
+  griddep_launch_dependents();
+  griddep_wait();
+  __shared__ int cnt[MOE_MAX_EXPERTS + 8], first[MOE_MAX_EXPERTS + 8];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int e = warp; e < NB; e += 8) {
+    int c = 0;
+    for (int r0 = 0; r0 < R; r0 += 32) {
+      const int r = r0 + lane;
+      const bool on = r < R && active[r] != 0 && w[(size_t)r * NB + e] != 0.f;
+      c += __popc(__ballot_sync(0xffffffffu, on));
+    }
+    if (lane == 0) cnt[e] = c;
+  }
+  for (int i = threadIdx.x; i < g.n_groups_max * MOE_GROUP_ROWS; i += 256) g.slot_row[i] = -1;
+  for (int i = threadIdx.x; i < R * NB; i += 256) g.slot_of[i] = -1;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int u = 0;
+    for (int e = 0; e < NB; ++e) {
+      first[e] = u;
+      int left = cnt[e];
+      while (left > 0 && u < g.n_groups_max) {
+        const int rows = left < MOE_GROUP_ROWS ? left : MOE_GROUP_ROWS;
+        g.tab_up[3 * u] = e * 2 * F; g.tab_up[3 * u + 1] = 0; g.tab_up[3 * u + 2] = rows;
+        g.tab_down[3 * u] = 0; g.tab_down[3 * u + 1] = e * F / GEMM_BLOCK_K; g.tab_down[3 * u + 2] = rows;
+        g.group_expert[u] = e;
+        left -= rows;
+        ++u;
+      }
+    }
+    for (; u < g.n_groups_max; ++u) {
+      g.tab_up[3 * u] = 0; g.tab_up[3 * u + 1] = 0; g.tab_up[3 * u + 2] = 0;
+      g.tab_down[3 * u] = 0; g.tab_down[3 * u + 1] = 0; g.tab_down[3 * u + 2] = 0;
+      g.group_expert[u] = -1;
+    }
+  }
+  __syncthreads();
+  for (int e = warp; e < NB; e += 8) {
+    int base = first[e] * MOE_GROUP_ROWS;            // slot of the expert's next row
+    for (int r0 = 0; r0 < R; r0 += 32) {
+      const int r = r0 + lane;
+      const bool on = r < R && active[r] != 0 && w[(size_t)r * NB + e] != 0.f;
+      const unsigned m = __ballot_sync(0xffffffffu, on);
+      if (on) {
+        const int slot = base + __popc(m & ((1u << lane) - 1u));
+        g.slot_row[slot] = r;
+        g.slot_of[(size_t)r * NB + e] = slot;
+      }
+      base += __popc(m);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) moe_gather_kernel(const bf16 *__restrict__ x_hi, const bf16 *__restrict__ x_lo, int H,
+                                                         MoeGroups g, bf16 *__restrict__ xg_hi, bf16 *__restrict__ xg_lo) {
+  griddep_launch_dependents();
+  griddep_wait();
+  const int slot = blockIdx.x;
+  const int r = g.slot_row[slot];
+  if (r < 0) return;
+  const uint4 *sh = reinterpret_cast<const uint4 *>(x_hi + (size_t)r * H), *sl = reinterpret_cast<const uint4 *>(x_lo + (size_t)r * H);
+  uint4 *dh = reinterpret_cast<uint4 *>(xg_hi + (size_t)slot * H), *dl = reinterpret_cast<uint4 *>(xg_lo + (size_t)slot * H);
+  for (int i = threadIdx.x; i < H / 8; i += blockDim.x) { dh[i] = sh[i]; dl[i] = sl[i]; }
+}
+
+__global__ void __launch_bounds__(256) moe_swiglu_grouped_kernel(const float *__restrict__ gu, const float *__restrict__ w,
+                                                                 int NB, int F, MoeGroups g, bf16 *__restrict__ hg_hi,
+                                                                 bf16 *__restrict__ hg_lo) {
+  griddep_launch_dependents();
+  griddep_wait();
+  const int slot = blockIdx.x;
+  const int r = g.slot_row[slot];
+  if (r < 0) return;
+  const int e = g.group_expert[slot / MOE_GROUP_ROWS];
+  const float we = w[(size_t)r * NB + e];
+  const float *row = gu + (size_t)slot * 2 * F;
+  for (int f = threadIdx.x * 4; f < F; f += blockDim.x * 4) {
+    const float4 a = *reinterpret_cast<const float4 *>(row + f), u = *reinterpret_cast<const float4 *>(row + F + f);
+    const float4 y = make_float4(we * (a.x / (1.f + expf(-a.x)) * u.x), we * (a.y / (1.f + expf(-a.y)) * u.y),
+                                 we * (a.z / (1.f + expf(-a.z)) * u.z), we * (a.w / (1.f + expf(-a.w)) * u.w));
+    bf16 p[4], q[4];
+    moe_split(y.x, p[0], q[0]);
+    moe_split(y.y, p[1], q[1]);
+    moe_split(y.z, p[2], q[2]);
+    moe_split(y.w, p[3], q[3]);
+    *reinterpret_cast<uint2 *>(hg_hi + (size_t)slot * F + f) = *reinterpret_cast<const uint2 *>(p);
+    *reinterpret_cast<uint2 *>(hg_lo + (size_t)slot * F + f) = *reinterpret_cast<const uint2 *>(q);
+  }
+}
+
+__global__ void __launch_bounds__(256) moe_combine_kernel(const float *__restrict__ yg, const int *__restrict__ active, int NB,
+                                                          int H, MoeGroups g, float *__restrict__ y) {
+  griddep_launch_dependents();
+  griddep_wait();
+  const int r = blockIdx.y;
+  if (!active[r]) return;
+  const int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i >= H) return;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int e = 0; e < NB; ++e) {                     // ascending expert id, shared experts last
+    const int slot = g.slot_of[(size_t)r * NB + e];
+    if (slot < 0) continue;
+    const float4 v = *reinterpret_cast<const float4 *>(yg + (size_t)slot * H + i);
+    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+  }
+  *reinterpret_cast<float4 *>(y + (size_t)r * H + i) = acc;
+}
+
 }  // namespace
 
 namespace corun {
+
+cudaError_t launch_moe_group(const float *w, const int *active, int R, int E, int S, int F, const MoeGroups &g,
+                             cudaStream_t st) {
+  if (E + S > MOE_MAX_EXPERTS + 8 || F % GEMM_BLOCK_K) return cudaErrorInvalidValue;
+  return launch_k(moe_group_kernel, dim3(1), dim3(256), 0, st, true, w, active, R, E + S, E, F, g);
+}
+
+cudaError_t launch_moe_gather(const __nv_bfloat16 *x_hi, const __nv_bfloat16 *x_lo, int H, const MoeGroups &g,
+                              __nv_bfloat16 *xg_hi, __nv_bfloat16 *xg_lo, cudaStream_t st) {
+  return launch_k(moe_gather_kernel, dim3(g.n_groups_max * MOE_GROUP_ROWS), dim3(256), 0, st, true, x_hi, x_lo, H, g, xg_hi, xg_lo);
+}
+
+cudaError_t launch_moe_swiglu_grouped(const float *gu, const float *w, int n_blocks, int F, const MoeGroups &g,
+                                      __nv_bfloat16 *hg_hi, __nv_bfloat16 *hg_lo, cudaStream_t st) {
+  return launch_k(moe_swiglu_grouped_kernel, dim3(g.n_groups_max * MOE_GROUP_ROWS), dim3(192), 0, st, true, gu, w, n_blocks, F, g,
+                  hg_hi, hg_lo);
+}
+
+cudaError_t launch_moe_combine(const float *yg, const int *active, int R, int n_blocks, int H, const MoeGroups &g, float *y,
+                               cudaStream_t st) {
+  return launch_k(moe_combine_kernel, dim3((H / 4 + 255) / 256, R), dim3(256), 0, st, true, yg, active, n_blocks, H, g, y);
+}
 
 cudaError_t launch_moe_route(const GemmOut &logits, int R, int E, int S, int top_k, int renormalize, float *w,
                              int *experts, float *probs, cudaStream_t st) {

@@ -17,4 +17,34 @@ cudaError_t launch_moe_route(const GemmOut &logits, int R, int E, int S, int top
 cudaError_t launch_moe_swiglu(const GemmOut &gu, const float *w, int R, int F, int n_blocks, __nv_bfloat16 *out_hi,
                               __nv_bfloat16 *out_lo, cudaStream_t st);
 
+// ---- grouped form (prefill chunks): every expert's rows gathered into blocks of MOE_GROUP_ROWS rows ----
+constexpr int MOE_GROUP_ROWS = 64;
+// Most groups a chunk of R rows can need: one per expert plus one per full block of selected (row, expert) pairs.
+inline int moe_max_groups(int R, int E, int S, int top_k) { return E + S + R * (top_k + S) / MOE_GROUP_ROWS; }
+
+// Buffers of the grouped form (device, owned by the caller).
+struct MoeGroups {
+  int n_groups_max;      // moe_max_groups(...)
+  int *tab_up;           // [n_groups_max][3]: first gate/up weight row (e * 2F), 0, rows   (gemm group table)
+  int *tab_down;         // [n_groups_max][3]: 0, first down k-block (e * F / 64), rows
+  int *group_expert;     // [n_groups_max]
+  int *slot_row;         // [n_groups_max * 64]: the chunk row gathered into the slot, -1 = none
+  int *slot_of;          // [R][E + S]: where the row sits in the expert's groups, -1 = not selected
+};
+
+// Groups the chunk's (row, expert) pairs: experts ascending, an expert's rows ascending, 64 per group; rows with
+// active[r] == 0 are left out.  w: the routing weights [R][E + S] of launch_moe_route.  One CTA.
+cudaError_t launch_moe_group(const float *w, const int *active, int R, int E, int S, int F, const MoeGroups &g,
+                             cudaStream_t st);
+// xg[slot, :] = x[slot_row[slot], :] for both halves of the activations (bf16, H values per row).
+cudaError_t launch_moe_gather(const __nv_bfloat16 *x_hi, const __nv_bfloat16 *x_lo, int H, const MoeGroups &g,
+                              __nv_bfloat16 *xg_hi, __nv_bfloat16 *xg_lo, cudaStream_t st);
+// hg[slot, f] = w[row, expert] * silu(gate) * up from the grouped gate/up result gu [slots][2F] (plain matrix).
+cudaError_t launch_moe_swiglu_grouped(const float *gu, const float *w, int n_blocks, int F, const MoeGroups &g,
+                                      __nv_bfloat16 *hg_hi, __nv_bfloat16 *hg_lo, cudaStream_t st);
+// y[r, :] = sum over the row's experts in ascending expert id (shared experts last) of yg[slot_of[r, e], :];
+// rows that are not active are left alone.
+cudaError_t launch_moe_combine(const float *yg, const int *active, int R, int n_blocks, int H, const MoeGroups &g, float *y,
+                               cudaStream_t st);
+
 }  // namespace corun
