@@ -145,59 +145,80 @@ __global__ void __launch_bounds__(256) moe_readout_kernel(GemmOut d, int H, floa
 }
 
 // ---------------------------------------------------------------- grouped form (prefill chunks)
-// One CTA of 256 threads (8 warps).  Phase 1: warp per expert counts its rows; phase 2: one thread turns the
-// counts into first-group indices (experts ascending) and clears the tables; phase 3: warp per expert hands
-// its rows, in ascending row order, consecutive slots of its groups.
-__global__ void __launch_bounds__(256) moe_group_kernel(const float *__restrict__ w, const int *__restrict__ active, int R,
+// One CTA of 1024 threads (32 warps: everything here waits on memory, so the more warps the better).  Phase 0: the selection w[r, e] != 0 (rows read with coalesced loads) as
+// bytes sel[e][r] in shared memory; phase 1: warp per expert counts its rows; phase 2: one thread turns the
+// counts into first-group indices (experts ascending); phase 3: warp per expert writes its groups' table
+// entries and hands its rows, in ascending row order, consecutive slots (slot_of is expert-major: [E + S][R]).
+__global__ void __launch_bounds__(1024) moe_group_kernel(const float *__restrict__ w, const int *__restrict__ active, int R,
                                                         int NB, int E, int F, MoeGroups g) {
   griddep_launch_dependents();
   griddep_wait();
-  __shared__ int cnt[MOE_MAX_EXPERTS + 8], first[MOE_MAX_EXPERTS + 8];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int e = warp; e < NB; e += 8) {
-    int c = 0;
-    for (int r0 = 0; r0 < R; r0 += 32) {
-      const int r = r0 + lane;
-      const bool on = r < R && active[r] != 0 && w[(size_t)r * NB + e] != 0.f;
-      c += __popc(__ballot_sync(0xffffffffu, on));
+  extern __shared__ unsigned char sel[];            // [NB][R + 4]: the pitch keeps a warp's 32 experts in 32 banks
+  const int SP = R + 4;
+  __shared__ int cnt[MOE_MAX_EXPERTS + 8], first[MOE_MAX_EXPERTS + 9];
+  __shared__ unsigned char act[256];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = (int)blockDim.x >> 5, n_thr = (int)blockDim.x;
+  for (int r = (int)threadIdx.x; r < R; r += n_thr) act[r] = active[r] != 0;
+  __syncthreads();
+  {
+    // eight independent loads per thread in flight (the table is read once, from L2)
+    const int total = R * NB;
+    for (int i0 = (int)threadIdx.x; i0 < total; i0 += n_thr * 8) {
+      float v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = i0 + n_thr * k < total ? w[i0 + n_thr * k] : 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int i = i0 + n_thr * k;
+        if (i < total) {
+          const int r = i / NB, e = i - r * NB;
+          sel[e * SP + r] = (v[k] != 0.f && act[r]) ? 1 : 0;
+        }
+      }
     }
+  }
+  __syncthreads();
+  for (int e = warp; e < NB; e += n_warps) {
+    int c = 0;
+    for (int r0 = 0; r0 < R; r0 += 32) c += __popc(__ballot_sync(0xffffffffu, r0 + lane < R && sel[e * SP + r0 + lane]));
     if (lane == 0) cnt[e] = c;
   }
-  for (int i = threadIdx.x; i < g.n_groups_max * MOE_GROUP_ROWS; i += 256) g.slot_row[i] = -1;
-  for (int i = threadIdx.x; i < R * NB; i += 256) g.slot_of[i] = -1;
   __syncthreads();
   if (threadIdx.x == 0) {
     int u = 0;
     for (int e = 0; e < NB; ++e) {
       first[e] = u;
-      int left = cnt[e];
-      while (left > 0 && u < g.n_groups_max) {
-        const int rows = left < MOE_GROUP_ROWS ? left : MOE_GROUP_ROWS;
-        g.tab_up[3 * u] = e * 2 * F; g.tab_up[3 * u + 1] = 0; g.tab_up[3 * u + 2] = rows;
-        g.tab_down[3 * u] = 0; g.tab_down[3 * u + 1] = e * F / GEMM_BLOCK_K; g.tab_down[3 * u + 2] = rows;
-        g.group_expert[u] = e;
-        left -= rows;
-        ++u;
-      }
+      u += (cnt[e] + MOE_GROUP_ROWS - 1) / MOE_GROUP_ROWS;
     }
-    for (; u < g.n_groups_max; ++u) {
-      g.tab_up[3 * u] = 0; g.tab_up[3 * u + 1] = 0; g.tab_up[3 * u + 2] = 0;
-      g.tab_down[3 * u] = 0; g.tab_down[3 * u + 1] = 0; g.tab_down[3 * u + 2] = 0;
-      g.group_expert[u] = -1;
-    }
+    first[NB] = u < g.n_groups_max ? u : g.n_groups_max;
   }
   __syncthreads();
-  for (int e = warp; e < NB; e += 8) {
+  for (int u = first[NB] + (int)threadIdx.x; u < g.n_groups_max; u += n_thr) {   // groups nobody needs
+    g.tab_up[3 * u] = 0; g.tab_up[3 * u + 1] = 0; g.tab_up[3 * u + 2] = 0;
+    g.tab_down[3 * u] = 0; g.tab_down[3 * u + 1] = 0; g.tab_down[3 * u + 2] = 0;
+    g.group_expert[u] = -1;
+  }
+  for (int e = warp; e < NB; e += n_warps) {
+    const int n_groups = (cnt[e] + MOE_GROUP_ROWS - 1) / MOE_GROUP_ROWS;
+    for (int k = lane; k < n_groups; k += 32) {
+      const int u = first[e] + k;
+      if (u >= g.n_groups_max) break;               // cannot happen: n_groups_max bounds the sum
+      const int rows = min(MOE_GROUP_ROWS, cnt[e] - k * MOE_GROUP_ROWS);
+      g.tab_up[3 * u] = e * 2 * F; g.tab_up[3 * u + 1] = 0; g.tab_up[3 * u + 2] = rows;
+      g.tab_down[3 * u] = 0; g.tab_down[3 * u + 1] = e * F / GEMM_BLOCK_K; g.tab_down[3 * u + 2] = rows;
+      g.group_expert[u] = e;
+    }
     int base = first[e] * MOE_GROUP_ROWS;            // slot of the expert's next row
     for (int r0 = 0; r0 < R; r0 += 32) {
       const int r = r0 + lane;
-      const bool on = r < R && active[r] != 0 && w[(size_t)r * NB + e] != 0.f;
+      const bool on = r < R && sel[e * SP + r];
       const unsigned m = __ballot_sync(0xffffffffu, on);
+      int slot = -1;
       if (on) {
-        const int slot = base + __popc(m & ((1u << lane) - 1u));
+        slot = base + __popc(m & ((1u << lane) - 1u));
         g.slot_row[slot] = r;
-        g.slot_of[(size_t)r * NB + e] = slot;
       }
+      if (r < R) g.slot_of[(size_t)e * R + r] = slot;
       base += __popc(m);
     }
   }
@@ -208,8 +229,8 @@ __global__ void __launch_bounds__(256) moe_gather_kernel(const bf16 *__restrict_
   griddep_launch_dependents();
   griddep_wait();
   const int slot = blockIdx.x;
+  if (slot % MOE_GROUP_ROWS >= g.tab_up[3 * (slot / MOE_GROUP_ROWS) + 2]) return;   // no row in this slot
   const int r = g.slot_row[slot];
-  if (r < 0) return;
   const uint4 *sh = reinterpret_cast<const uint4 *>(x_hi + (size_t)r * H), *sl = reinterpret_cast<const uint4 *>(x_lo + (size_t)r * H);
   uint4 *dh = reinterpret_cast<uint4 *>(xg_hi + (size_t)slot * H), *dl = reinterpret_cast<uint4 *>(xg_lo + (size_t)slot * H);
   for (int i = threadIdx.x; i < H / 8; i += blockDim.x) { dh[i] = sh[i]; dl[i] = sl[i]; }
@@ -221,8 +242,8 @@ __global__ void __launch_bounds__(256) moe_swiglu_grouped_kernel(const float *__
   griddep_launch_dependents();
   griddep_wait();
   const int slot = blockIdx.x;
+  if (slot % MOE_GROUP_ROWS >= g.tab_up[3 * (slot / MOE_GROUP_ROWS) + 2]) return;   // no row in this slot
   const int r = g.slot_row[slot];
-  if (r < 0) return;
   const int e = g.group_expert[slot / MOE_GROUP_ROWS];
   const float we = w[(size_t)r * NB + e];
   const float *row = gu + (size_t)slot * 2 * F;
@@ -246,11 +267,14 @@ __global__ void __launch_bounds__(256) moe_combine_kernel(const float *__restric
   griddep_wait();
   const int r = blockIdx.y;
   if (!active[r]) return;
+  __shared__ int slots[MOE_MAX_EXPERTS + 8];
+  for (int e = threadIdx.x; e < NB; e += blockDim.x) slots[e] = g.slot_of[(size_t)e * gridDim.y + r];
+  __syncthreads();
   const int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i >= H) return;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int e = 0; e < NB; ++e) {                     // ascending expert id, shared experts last
-    const int slot = g.slot_of[(size_t)r * NB + e];
+    const int slot = slots[e];
     if (slot < 0) continue;
     const float4 v = *reinterpret_cast<const float4 *>(yg + (size_t)slot * H + i);
     acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
@@ -265,7 +289,15 @@ namespace corun {
 cudaError_t launch_moe_group(const float *w, const int *active, int R, int E, int S, int F, const MoeGroups &g,
                              cudaStream_t st) {
   if (E + S > MOE_MAX_EXPERTS + 8 || F % GEMM_BLOCK_K) return cudaErrorInvalidValue;
-  return launch_k(moe_group_kernel, dim3(1), dim3(256), 0, st, true, w, active, R, E + S, E, F, g);
+  const size_t smem = (size_t)(E + S) * (R + 4);    // <= 264 * 260 bytes
+  static bool prepared = false;
+  if (!prepared) {
+    cudaError_t e = cudaFuncSetAttribute(moe_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (MOE_MAX_EXPERTS + 8) * 260);
+    if (e != cudaSuccess) return e;
+    prepared = true;
+  }
+  if (R > 256) return cudaErrorInvalidValue;
+  return launch_k(moe_group_kernel, dim3(1), dim3(1024), smem, st, true, w, active, R, E + S, E, F, g);
 }
 
 cudaError_t launch_moe_gather(const __nv_bfloat16 *x_hi, const __nv_bfloat16 *x_lo, int H, const MoeGroups &g,

@@ -28,8 +28,8 @@ struct MoeGroups {
   int *tab_up;           // [n_groups_max][3]: first gate/up weight row (e * 2F), 0, rows   (gemm group table)
   int *tab_down;         // [n_groups_max][3]: 0, first down k-block (e * F / 64), rows
   int *group_expert;     // [n_groups_max]
-  int *slot_row;         // [n_groups_max * 64]: the chunk row gathered into the slot, -1 = none
-  int *slot_of;          // [R][E + S]: where the row sits in the expert's groups, -1 = not selected
+  int *slot_row;         // [n_groups_max * 64]: the chunk row gathered into the slot (valid below the group's row count)
+  int *slot_of;          // [E + S][R]: where the row sits in the expert's groups, -1 = not selected
 };
 
 // Groups the chunk's (row, expert) pairs: experts ascending, an expert's rows ascending, 64 per group; rows with
