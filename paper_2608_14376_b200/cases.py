@@ -10,7 +10,7 @@
     python -m paper_2608_14376_b200.cases moe --experts 128 --top-k 8 --ffn 768 --shared 0 --renormalize   # Qwen3-30B-A3B block
     python -m paper_2608_14376_b200.cases ablation  [--layers 2 --B 64 --actives 1,4,16,40,64]
     python -m paper_2608_14376_b200.cases sweep     [--Bs 1,8,32,128,256 --fractions 0.125,0.5,1 --steps 10]
-    python -m paper_2608_14376_b200.cases trace     [--requests 200 --rate 4 --B 128 --replay 4 --batched]
+    python -m paper_2608_14376_b200.cases trace     [--requests 200 --rate 4 --B 128 --replay 4 --batched --moe]
 
 ``gemm`` runs the stand-alone decode GEMM on seeded inputs; ``attention`` builds a Qwen3-8B-shaped
 engine with few layers, fills the cache of the active slots on the device and runs decode steps.
@@ -376,15 +376,21 @@ def case_trace(a):
 
     from . import corun, synth
 
-    sh = synth.QWEN3_8B
-    w = synth.make_weights_torch(sh, seed=0, device="cuda")
+    moe = None
+    if a.moe:                                             # the Mixture-of-Experts decoder (Qwen3-30B-A3B shape)
+        sh = synth.QWEN3_30B_A3B
+        w = synth.make_weights_torch(sh, seed=0, device="cuda", dense_ffn=False)
+        moe = synth.make_moe_torch(sh, seed=0, device="cuda", **synth.QWEN3_30B_A3B_MOE)
+    else:
+        sh = synth.QWEN3_8B
+        w = synth.make_weights_torch(sh, seed=0, device="cuda")
     rng = np.random.default_rng(5)
     n = a.requests
     arrival = np.cumsum(rng.exponential(1.0 / a.rate, n))
     plen = np.minimum(8192, np.maximum(1, np.round(np.exp(np.log(a.prompt_median) + rng.standard_normal(n))))).astype(int)
     olen = np.minimum(2048, np.maximum(2, np.round(np.exp(np.log(a.output_median) + rng.standard_normal(n))))).astype(int)
     prompts = synth.make_prompts(sh.vocab, plen, seed=6)
-    eng = corun.Engine(sh, w, a.B, 10240)
+    eng = corun.Engine(sh, w, a.B, 10240, moe=moe)
     sch = corun.Scheduler(engine=eng)
     if a.batched:
         sch.enable_batched_prefill()
@@ -483,6 +489,7 @@ def main():
     tr.add_argument("--requests", type=int, default=200); tr.add_argument("--rate", type=float, default=4.0)
     tr.add_argument("--B", type=int, default=128); tr.add_argument("--replay", type=int, default=4)
     tr.add_argument("--batched", action="store_true", help="scheduler with batched prefill on")
+    tr.add_argument("--moe", action="store_true", help="the Mixture-of-Experts decoder instead of the dense one")
     tr.add_argument("--prompt-median", type=float, default=1024.0); tr.add_argument("--output-median", type=float, default=256.0)
     a = ap.parse_args()
     {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "prefill": case_prefill, "ablation": case_ablation, "moe": case_moe, "prefill_batch": case_prefill_batch, "sampler": case_sampler,
