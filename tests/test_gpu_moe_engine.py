@@ -210,3 +210,21 @@ def test_moe_engine_at_the_qwen3_30b_a3b_layer_shape(orc):
             assert eng.logits(s).tobytes() == r["bytes"]
     finally:
         eng.close()
+
+
+def test_moe_engine_argument_errors(orc):
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2608_14376_b200 import corun
+
+    sh = synth.TINY
+    w_t = synth.weights_numpy_to_torch(synth.make_weights_numpy(sh, seed=1), "cuda")
+    good = synth.moe_numpy_to_torch(synth.make_moe_numpy(sh, 8, 2, 128, 1), "cuda")
+    for bad in (dict(top_k=0), dict(top_k=9), dict(n_experts=0), dict(expert_ffn=100), dict(n_shared=-1)):
+        with pytest.raises(corun.CorunError) as ei:
+            corun.Engine(sh, w_t, B, MAX_CTX, moe=dict(good, **bad))
+        assert ei.value.status == corun.EINVAL
+    eng = corun.Engine(sh, w_t, B, MAX_CTX, moe=good)      # and the good one still initialises
+    assert eng.decode_launches() == 7 + 11 * sh.n_layers
+    eng.close()
