@@ -4,7 +4,7 @@
     python -m paper_2608_14376_b200.cases kernels   [--layers 4 --B 64 --active-frac 0.625 --vocab 32768]
     python -m paper_2608_14376_b200.cases attention [--layers 2 --B 64 --active 40 --ctx-lo 512 --ctx-hi 4096 --reps 2]
     python -m paper_2608_14376_b200.cases sampler   [--B 64 --active 40 --vocab 151936]
-    python -m paper_2608_14376_b200.cases prefill   [--layers 2 --tokens 4096 --reps 2]
+    python -m paper_2608_14376_b200.cases prefill   [--layers 2 --tokens 4096 --reps 2 --moe]
     python -m paper_2608_14376_b200.cases prefill_batch [--layers 36 --lengths 40,100,200,500,1000 --n 8]
     python -m paper_2608_14376_b200.cases moe       [--B 128 --reps 20]      # DeepSeek-V2-Lite MoE block shape
     python -m paper_2608_14376_b200.cases moe --experts 128 --top-k 8 --ffn 768 --shared 0 --renormalize   # Qwen3-30B-A3B block
@@ -85,9 +85,14 @@ def case_prefill(a):
 
     from . import corun, synth
 
-    sh = synth.ModelShape(a.layers, 4096, 32, 8, 128, 12288, 4096, 1e-6, 1e6)
-    w = synth.make_weights_torch(sh, seed=0, device="cuda")
-    eng = corun.Engine(sh, w, 2, a.tokens + 64)
+    if a.moe:                                             # the Mixture-of-Experts decoder's layer shape (Qwen3-30B-A3B)
+        sh = synth.ModelShape(a.layers, 2048, 32, 4, 128, 64, 4096, 1e-6, 1e6)
+        w = synth.make_weights_torch(sh, seed=0, device="cuda", dense_ffn=False)
+        eng = corun.Engine(sh, w, 2, a.tokens + 64, moe=synth.make_moe_torch(sh, seed=0, device="cuda", **synth.QWEN3_30B_A3B_MOE))
+    else:
+        sh = synth.ModelShape(a.layers, 4096, 32, 8, 128, 12288, 4096, 1e-6, 1e6)
+        w = synth.make_weights_torch(sh, seed=0, device="cuda")
+        eng = corun.Engine(sh, w, 2, a.tokens + 64)
     prompt = synth.make_prompts(sh.vocab, [a.tokens], seed=11)[0]
     first = None
     for _ in range(a.reps):
@@ -466,6 +471,7 @@ def main():
     pf = sub.add_parser("prefill")
     pf.add_argument("--layers", type=int, default=2); pf.add_argument("--tokens", type=int, default=4096)
     pf.add_argument("--reps", type=int, default=2)
+    pf.add_argument("--moe", action="store_true", help="the Mixture-of-Experts decoder's layer shape")
     pb = sub.add_parser("prefill_batch")
     pb.add_argument("--layers", type=int, default=36); pb.add_argument("--lengths", default="40,100,200,500,1000")
     pb.add_argument("--n", type=int, default=8)
