@@ -8,6 +8,7 @@
     python -m paper_2608_14376_b200.cases prefill_batch [--layers 36 --lengths 40,100,200,500,1000 --n 8]
     python -m paper_2608_14376_b200.cases moe       [--B 128 --reps 20]      # DeepSeek-V2-Lite MoE block shape
     python -m paper_2608_14376_b200.cases moe --experts 128 --top-k 8 --ffn 768 --shared 0 --renormalize   # Qwen3-30B-A3B block
+    python -m paper_2608_14376_b200.cases mla       [--B 128 --ctx-lo 512 --ctx-hi 4096 --reps 10]   # DeepSeek-V2-Lite attention shape
     python -m paper_2608_14376_b200.cases ablation  [--layers 2 --B 64 --actives 1,4,16,40,64]
     python -m paper_2608_14376_b200.cases sweep     [--Bs 1,8,32,128,256 --fractions 0.125,0.5,1 --steps 10]
     python -m paper_2608_14376_b200.cases trace     [--requests 200 --rate 4 --B 128 --replay 4 --batched --moe]
@@ -20,6 +21,8 @@ Each prints the CUDA-event time per launch, for comparison with what a profiler 
 (``corun_prefill_batch``) and checks that the first tokens and logits are the same bytes.
 ``moe`` times the Mixture-of-Experts feed-forward block (64 routed experts of 1408, top-6, 2 shared, hidden
 2048) on B padded rows against the bytes of expert weights a call streams.
+``mla`` times the absorbed multi-head latent attention op (16 heads, latent 512 + rope 64 per cached token) on
+B rows with seeded context lengths against the cache bytes a call reads.
 ``ablation`` compares the request-local split of the decode attention (every 128-token split of a request is
 an item any SM may take) with the same kernel handing out whole (row, kv head) pairs, i.e. no parallelism
 inside a request's attention, on ragged and on equal context lengths; the logits are the same bytes either way.
@@ -195,6 +198,39 @@ def case_moe(a):
     print("moe: B=%d H=%d E=%d top-%d F=%d shared=%d: %.1f us per call, %.1f MB of weights -> %.0f GB/s; %d of %d experts selected; %d launches"
           % (a.B, H, E, K, F, S, ms * 1e3, wb / 1e6, wb / ms / 1e6, hit, E, op.launches()))
     op.close()
+
+
+def case_mla(a):
+    import math
+
+    import torch
+
+    from . import corun, synth
+
+    nh, dc, dr = 16, 512, 64
+    ctx = synth.uniform_lengths(a.ctx_lo, a.ctx_hi, a.B, seed=2).astype(np.int32)
+    T = int(-(-int(ctx.max()) // 128) * 128)
+    g = torch.Generator(device="cuda").manual_seed(0)
+    cache = (torch.randn((a.B, T, dc + dr), generator=g, device="cuda") * 0.5).to(torch.float16)
+    q_lat = torch.randn((a.B, nh, dc), generator=g, device="cuda")
+    q_rope = torch.randn((a.B, nh, dr), generator=g, device="cuda")
+    dctx = torch.tensor(ctx).cuda()
+    scale = 1.0 / math.sqrt(128 + dr)
+    for _ in range(3):
+        out = corun.mla_attend(q_lat, q_rope, cache, dctx, scale)
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(a.reps):
+        out = corun.mla_attend(q_lat, q_rope, cache, dctx, scale)
+    t1.record()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / a.reps
+    nbytes = int(ctx.astype(np.int64).sum()) * (dc + dr) * 2
+    flops = int(ctx.astype(np.int64).sum()) * nh * (dc + dr + dc) * 2
+    print("mla: B=%d, contexts %d..%d (mean %.0f): %.1f us per call, %.1f MB of latent cache -> %.0f GB/s, %.1f TFLOP/s (fp32 FMA)"
+          % (a.B, ctx.min(), ctx.max(), ctx.mean(), ms * 1e3, nbytes / 1e6, nbytes / ms / 1e6, flops / ms / 1e9))
+    assert bool(torch.isfinite(out).all().item())
 
 
 def case_ablation(a):
@@ -481,6 +517,9 @@ def main():
     mo.add_argument("--top-k", type=int, default=6); mo.add_argument("--ffn", type=int, default=1408)
     mo.add_argument("--shared", type=int, default=2)
     mo.add_argument("--renormalize", action="store_true", help="selected probabilities divided by their sum (Qwen3-MoE)")
+    ma = sub.add_parser("mla")
+    ma.add_argument("--B", type=int, default=128); ma.add_argument("--ctx-lo", type=int, default=512)
+    ma.add_argument("--ctx-hi", type=int, default=4096); ma.add_argument("--reps", type=int, default=10)
     ab = sub.add_parser("ablation")
     ab.add_argument("--layers", type=int, default=2); ab.add_argument("--B", type=int, default=64)
     ab.add_argument("--actives", default="1,4,16,40,64"); ab.add_argument("--ctx-lo", type=int, default=512)
@@ -498,7 +537,7 @@ def main():
     tr.add_argument("--moe", action="store_true", help="the Mixture-of-Experts decoder instead of the dense one")
     tr.add_argument("--prompt-median", type=float, default=1024.0); tr.add_argument("--output-median", type=float, default=256.0)
     a = ap.parse_args()
-    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "prefill": case_prefill, "ablation": case_ablation, "moe": case_moe, "prefill_batch": case_prefill_batch, "sampler": case_sampler,
+    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "prefill": case_prefill, "ablation": case_ablation, "mla": case_mla, "moe": case_moe, "prefill_batch": case_prefill_batch, "sampler": case_sampler,
      "sweep": case_sweep, "trace": case_trace}[a.case](a)
 
 

@@ -26,7 +26,7 @@ EXPORTS = [
     "corun_sched_step", "corun_sched_poll", "corun_sched_slot_of", "corun_sched_counts",
     "corun_sched_enable_batched_prefill", "corun_prefill_geometry",
     "corun_moe_create", "corun_moe_destroy", "corun_moe_forward", "corun_moe_sync", "corun_moe_weight_bytes",
-    "corun_moe_launches",
+    "corun_moe_launches", "corun_mla_attend", "corun_mla_workspace_floats",
 ]
 
 
@@ -513,3 +513,28 @@ class MoeFfn:
             self.close()
         except Exception:
             pass
+
+
+def mla_attend(q_lat, q_rope, cache, ctx, scale: float):
+    """Absorbed multi-head latent attention for one query token per row (``include/corun_mla.h``).
+    q_lat fp32 [B, n_heads, d_c], q_rope fp32 [B, n_heads, d_r], cache fp16 [B, T, d_c + d_r], ctx int32 [B]
+    (all CUDA tensors) -> o_lat fp32 [B, n_heads, d_c] (rows with ctx 0 are left as zeros)."""
+    import torch
+
+    B, nh, dc = q_lat.shape
+    dr = q_rope.shape[2]
+    T = cache.shape[1]
+    assert q_lat.is_cuda and q_lat.dtype == torch.float32 and q_lat.is_contiguous()
+    assert q_rope.dtype == torch.float32 and q_rope.is_contiguous() and tuple(q_rope.shape[:2]) == (B, nh)
+    assert cache.dtype == torch.float16 and cache.is_contiguous() and tuple(cache.shape) == (B, T, dc + dr)
+    assert ctx.dtype == torch.int32 and ctx.is_contiguous() and tuple(ctx.shape) == (B,)
+    L = lib()
+    L.corun_mla_workspace_floats.restype = C.c_int64
+    L.corun_mla_workspace_floats.argtypes = [C.c_int32] * 4
+    L.corun_mla_attend.argtypes = [C.c_void_p] * 4 + [C.c_int32] * 5 + [C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
+    ws = torch.empty(int(L.corun_mla_workspace_floats(B, nh, dc, T)), dtype=torch.float32, device=q_lat.device)
+    out = torch.zeros_like(q_lat)
+    _check(L.corun_mla_attend(q_lat.data_ptr(), q_rope.data_ptr(), cache.data_ptr(), ctx.data_ptr(), B, nh, dc, dr, T,
+                              float(scale), out.data_ptr(), ws.data_ptr(), torch.cuda.current_stream().cuda_stream),
+           "corun_mla_attend")
+    return out

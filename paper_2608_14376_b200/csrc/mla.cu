@@ -1,0 +1,204 @@
+// Multi-head latent attention at decode time in the absorbed form, first correct path: fp32 FMA arithmetic on
+// the CUDA cores (see include/corun_mla.h).  One CTA per (row, split of 128 cached tokens): the split's latent
+// rows and the row's absorbed queries are staged in shared memory, scores / softmax / weighted latent sum are
+// computed there, the split's (max, sum, output) goes to the workspace; a second kernel combines a row's
+// splits in ascending order.  Split size fixed, split count = f(own context): nothing depends on other rows.
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <math_constants.h>
+
+#include "../../include/corun_mla.h"
+#include "gemm.cuh"
+
+namespace {
+
+constexpr int MLA_SPLIT = 128;      // cached tokens per split
+constexpr int MLA_THREADS = 256;
+constexpr int MLA_NH = 16;          // head slots of the shared-memory tiles (n_heads <= 16)
+
+__global__ void __launch_bounds__(MLA_THREADS, 1)
+mla_split_kernel(const float *__restrict__ q_lat, const float *__restrict__ q_rope, const __half *__restrict__ cache,
+                 const int *__restrict__ ctx, int n_heads, int d_c, int d_r, int max_context, int max_splits, float scale,
+                 float *__restrict__ part_o, float2 *__restrict__ part_ml) {
+  const int s = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  const int n_ctx = ctx[b];
+  const int t0 = s * MLA_SPLIT;
+  if (t0 >= n_ctx) return;                           // the same decision in every thread
+  const int n = min(MLA_SPLIT, n_ctx - t0);
+  const int DK = d_c + d_r;
+  const int pitch = DK + 2;                          // halfs; an odd number of 32-bit words: rows fall into different banks
+  extern __shared__ __align__(16) unsigned char smem[];
+  float *qs = reinterpret_cast<float *>(smem);                                   // [DK][16]: q[d][h]
+  float *ps = qs + (size_t)DK * MLA_NH;                                          // [128][16]: scores, then weights
+  float *red = ps + MLA_SPLIT * MLA_NH;                                          // [16] maxima, [16] sums
+  __half *cs = reinterpret_cast<__half *>(red + 2 * MLA_NH);                     // [128][pitch]
+
+  // ---- the row's absorbed queries (heads beyond n_heads: zeros)
+  for (int i = tid; i < DK * MLA_NH; i += MLA_THREADS) {
+    const int d = i / MLA_NH, h = i % MLA_NH;
+    float v = 0.f;
+    if (h < n_heads) v = d < d_c ? q_lat[((size_t)b * n_heads + h) * d_c + d] : q_rope[((size_t)b * n_heads + h) * d_r + (d - d_c)];
+    qs[i] = v;
+  }
+  // ---- the split's cache rows (rows beyond the context: zeros): 16-byte loads, several in flight per thread
+  {
+    const int vecs = DK / 8;                         // uint4 per row (DK is a multiple of 8: rows are 16-byte aligned)
+    const uint4 *src = reinterpret_cast<const uint4 *>(cache + ((size_t)b * max_context + t0) * DK);
+    uint32_t *dst = reinterpret_cast<uint32_t *>(cs);
+    const int total = MLA_SPLIT * vecs;
+    for (int i0 = tid; i0 < total; i0 += MLA_THREADS * 6) {
+      uint4 v[6];
+#pragma unroll
+      for (int k = 0; k < 6; ++k) {
+        const int i = i0 + MLA_THREADS * k;
+        const int t = i / vecs;
+        v[k] = (i < total && t < n) ? src[i] : make_uint4(0u, 0u, 0u, 0u);   // rows are contiguous: src[t * vecs + j] = src[i]
+      }
+#pragma unroll
+      for (int k = 0; k < 6; ++k) {
+        const int i = i0 + MLA_THREADS * k;
+        if (i < total) {
+          const int t = i / vecs, j = i - t * vecs;
+          uint32_t *d = dst + t * (pitch / 2) + 4 * j;
+          d[0] = v[k].x; d[1] = v[k].y; d[2] = v[k].z; d[3] = v[k].w;
+        }
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- scores: thread = (tokens tp and tp + 64, heads 4 hq .. 4 hq + 3)
+  {
+    const int tp = tid & 63, hq = tid >> 6;
+    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    const __half2 *c0 = reinterpret_cast<const __half2 *>(cs + (size_t)tp * pitch);
+    const __half2 *c1 = reinterpret_cast<const __half2 *>(cs + (size_t)(tp + 64) * pitch);
+#pragma unroll 4
+    for (int d = 0; d < DK; d += 2) {
+      const float2 a = __half22float2(c0[d >> 1]), e = __half22float2(c1[d >> 1]);
+      const float4 qa = *reinterpret_cast<const float4 *>(qs + (size_t)d * MLA_NH + 4 * hq);
+      const float4 qb = *reinterpret_cast<const float4 *>(qs + (size_t)(d + 1) * MLA_NH + 4 * hq);
+      acc[0][0] = fmaf(a.x, qa.x, acc[0][0]); acc[0][1] = fmaf(a.x, qa.y, acc[0][1]);
+      acc[0][2] = fmaf(a.x, qa.z, acc[0][2]); acc[0][3] = fmaf(a.x, qa.w, acc[0][3]);
+      acc[0][0] = fmaf(a.y, qb.x, acc[0][0]); acc[0][1] = fmaf(a.y, qb.y, acc[0][1]);
+      acc[0][2] = fmaf(a.y, qb.z, acc[0][2]); acc[0][3] = fmaf(a.y, qb.w, acc[0][3]);
+      acc[1][0] = fmaf(e.x, qa.x, acc[1][0]); acc[1][1] = fmaf(e.x, qa.y, acc[1][1]);
+      acc[1][2] = fmaf(e.x, qa.z, acc[1][2]); acc[1][3] = fmaf(e.x, qa.w, acc[1][3]);
+      acc[1][0] = fmaf(e.y, qb.x, acc[1][0]); acc[1][1] = fmaf(e.y, qb.y, acc[1][1]);
+      acc[1][2] = fmaf(e.y, qb.z, acc[1][2]); acc[1][3] = fmaf(e.y, qb.w, acc[1][3]);
+    }
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int t = tp + 64 * k;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) ps[t * MLA_NH + 4 * hq + j] = t < n ? acc[k][j] * scale : -CUDART_INF_F;
+    }
+  }
+  __syncthreads();
+
+  // ---- softmax of the split per head: warp w takes heads 2 w and 2 w + 1; fixed orders throughout
+  {
+    const int warp = tid >> 5, lane = tid & 31;
+    for (int h = 2 * warp; h < 2 * warp + 2; ++h) {
+      float v[4], m = -CUDART_INF_F;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) { v[k] = ps[(lane + 32 * k) * MLA_NH + h]; m = fmaxf(m, v[k]); }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      float l = 0.f;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float p = expf(v[k] - m);             // exp(-inf) = 0 beyond the context
+        ps[(lane + 32 * k) * MLA_NH + h] = p;
+        l += p;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+      if (lane == 0) { red[h] = m; red[MLA_NH + h] = l; }
+    }
+  }
+  __syncthreads();
+
+  // ---- weighted latent sum: thread = dims (2 tid, 2 tid + 1) (+ 512 ...) of all heads, tokens ascending
+  for (int d0 = 2 * tid; d0 < d_c; d0 += 2 * MLA_THREADS) {
+    float acc[MLA_NH][2];
+#pragma unroll
+    for (int h = 0; h < MLA_NH; ++h) { acc[h][0] = 0.f; acc[h][1] = 0.f; }
+#pragma unroll 2
+    for (int t = 0; t < n; ++t) {
+      const float2 c = __half22float2(*reinterpret_cast<const __half2 *>(cs + (size_t)t * pitch + d0));
+      const float4 *p4 = reinterpret_cast<const float4 *>(ps + t * MLA_NH);
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const float4 p = p4[g];
+        acc[4 * g + 0][0] = fmaf(p.x, c.x, acc[4 * g + 0][0]); acc[4 * g + 0][1] = fmaf(p.x, c.y, acc[4 * g + 0][1]);
+        acc[4 * g + 1][0] = fmaf(p.y, c.x, acc[4 * g + 1][0]); acc[4 * g + 1][1] = fmaf(p.y, c.y, acc[4 * g + 1][1]);
+        acc[4 * g + 2][0] = fmaf(p.z, c.x, acc[4 * g + 2][0]); acc[4 * g + 2][1] = fmaf(p.z, c.y, acc[4 * g + 2][1]);
+        acc[4 * g + 3][0] = fmaf(p.w, c.x, acc[4 * g + 3][0]); acc[4 * g + 3][1] = fmaf(p.w, c.y, acc[4 * g + 3][1]);
+      }
+    }
+    for (int h = 0; h < n_heads; ++h)
+      *reinterpret_cast<float2 *>(part_o + (((size_t)b * max_splits + s) * n_heads + h) * d_c + d0) = make_float2(acc[h][0], acc[h][1]);
+  }
+  if (tid < n_heads) part_ml[((size_t)b * max_splits + s) * n_heads + tid] = make_float2(red[tid], red[MLA_NH + tid]);
+}
+
+// One CTA per (head, row): the row's splits in ascending order.
+__global__ void __launch_bounds__(MLA_THREADS)
+mla_combine_kernel(const float *__restrict__ part_o, const float2 *__restrict__ part_ml, const int *__restrict__ ctx,
+                   int n_heads, int d_c, int max_splits, float *__restrict__ o_lat) {
+  const int h = blockIdx.x, b = blockIdx.y;
+  const int n_ctx = ctx[b];
+  if (n_ctx <= 0) return;
+  const int ns = (n_ctx + MLA_SPLIT - 1) / MLA_SPLIT;
+  const float2 *ml = part_ml + (size_t)b * max_splits * n_heads + h;
+  float M = -CUDART_INF_F;
+  for (int s = 0; s < ns; ++s) M = fmaxf(M, ml[(size_t)s * n_heads].x);
+  float den = 0.f;
+  for (int s = 0; s < ns; ++s) den += expf(ml[(size_t)s * n_heads].x - M) * ml[(size_t)s * n_heads].y;
+  for (int d = threadIdx.x; d < d_c; d += blockDim.x) {
+    float o = 0.f;
+    for (int s = 0; s < ns; ++s)
+      o = fmaf(expf(ml[(size_t)s * n_heads].x - M), part_o[(((size_t)b * max_splits + s) * n_heads + h) * d_c + d], o);
+    o_lat[((size_t)b * n_heads + h) * d_c + d] = o / den;
+  }
+}
+
+size_t mla_smem_bytes(int d_c, int d_r) {
+  const int DK = d_c + d_r;
+  return (size_t)DK * MLA_NH * 4 + (size_t)MLA_SPLIT * MLA_NH * 4 + 2 * MLA_NH * 4 + (size_t)MLA_SPLIT * (DK + 2) * 2;
+}
+
+}  // namespace
+
+extern "C" {
+
+int64_t corun_mla_workspace_floats(int32_t B, int32_t n_heads, int32_t d_latent, int32_t max_context) {
+  if (B < 1 || n_heads < 1 || d_latent < 1 || max_context < 1) return 0;
+  const int64_t splits = (max_context + MLA_SPLIT - 1) / MLA_SPLIT;
+  return (int64_t)B * splits * n_heads * (d_latent + 2);
+}
+
+int corun_mla_attend(const float *q_lat, const float *q_rope, const void *cache, const int32_t *ctx, int32_t B,
+                     int32_t n_heads, int32_t d_latent, int32_t d_rope, int32_t max_context, float scale, float *o_lat,
+                     float *ws, void *cuda_stream) {
+  if (!q_lat || !q_rope || !cache || !ctx || !o_lat || !ws || B < 1 || B > 65535 || n_heads < 4 || n_heads > MLA_NH ||
+      n_heads % 4 || d_latent < 64 || d_latent > 512 || d_latent % 64 || d_rope < 2 || d_rope > 64 || d_rope % 2 ||
+      max_context < 1)
+    return CORUN_EINVAL;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const int max_splits = (max_context + MLA_SPLIT - 1) / MLA_SPLIT;
+  const size_t smem = mla_smem_bytes(d_latent, d_rope);
+  cudaError_t ce = cudaFuncSetAttribute(mla_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (ce != cudaSuccess) { corun::g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
+  float *part_o = ws;
+  float2 *part_ml = reinterpret_cast<float2 *>(ws + (size_t)B * max_splits * n_heads * d_latent);
+  mla_split_kernel<<<dim3(max_splits, B), MLA_THREADS, smem, st>>>(q_lat, q_rope, (const __half *)cache, ctx, n_heads, d_latent,
+                                                                  d_rope, max_context, max_splits, scale, part_o, part_ml);
+  mla_combine_kernel<<<dim3(n_heads, B), MLA_THREADS, 0, st>>>(part_o, part_ml, ctx, n_heads, d_latent, max_splits, o_lat);
+  ce = cudaGetLastError();
+  if (ce != cudaSuccess) { corun::g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
+  return CORUN_OK;
+}
+
+}  // extern "C"
