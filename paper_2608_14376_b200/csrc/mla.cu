@@ -34,11 +34,11 @@ mla_split_kernel(const float *__restrict__ q_lat, const float *__restrict__ q_ro
   __half *cs = reinterpret_cast<__half *>(red + 2 * MLA_NH);                     // [128][pitch]
 
   // ---- the row's absorbed queries (heads beyond n_heads: zeros)
-  for (int i = tid; i < DK * MLA_NH; i += MLA_THREADS) {
-    const int d = i / MLA_NH, h = i % MLA_NH;
+  for (int i = tid; i < DK * MLA_NH; i += MLA_THREADS) {   // consecutive threads read consecutive d of one head
+    const int h = i / DK, d = i - h * DK;
     float v = 0.f;
     if (h < n_heads) v = d < d_c ? q_lat[((size_t)b * n_heads + h) * d_c + d] : q_rope[((size_t)b * n_heads + h) * d_r + (d - d_c)];
-    qs[i] = v;
+    qs[d * MLA_NH + h] = v;
   }
   // ---- the split's cache rows (rows beyond the context: zeros): 16-byte loads, several in flight per thread
   {
