@@ -36,7 +36,8 @@ int64_t corun_mla_workspace_floats(int32_t B, int32_t n_heads, int32_t d_latent,
  *   ctx     int32 [B]: cached tokens per row, 0 = padding row (its output is left alone)
  *   o_lat   fp32 [B, n_heads, d_latent]
  *   ws      corun_mla_workspace_floats(...) floats
- * n_heads 1..16 (a multiple of 4), d_latent a multiple of 64 up to 512, d_rope a multiple of 2 up to 64.
+ * n_heads 1..16 (a multiple of 4), d_latent a multiple of 64 up to 512, d_rope a multiple of 8 up to 64
+ * (cache rows are then 16-byte aligned).
  * Errors: EINVAL, ECUDA.
  */
 int corun_mla_attend(const float *q_lat, const float *q_rope, const void *cache, const int32_t *ctx, int32_t B,

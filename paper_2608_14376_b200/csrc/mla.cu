@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <math_constants.h>
 
+#include <cstdlib>
+
 #include "../../include/corun_mla.h"
 #include "gemm.cuh"
 
@@ -143,6 +145,187 @@ mla_split_kernel(const float *__restrict__ q_lat, const float *__restrict__ q_ro
   if (tid < n_heads) part_ml[((size_t)b * max_splits + s) * n_heads + tid] = make_float2(red[tid], red[MLA_NH + tid]);
 }
 
+// ---------------------------------------------------------------- the same split on the warp-level tensor path
+// mma.sync m16n8k16 (fp16 x fp16 -> fp32): the 16 heads are the M dimension of every instruction.  Queries and
+// softmax weights enter as fp16 hi + lo pairs (two instructions per tile), the cache rows are fp16 as stored.
+// Scores: warp w takes tokens 16 w .. 16 w + 15 (B operand = cache rows [token][dim], read with ldmatrix);
+// weighted latent sum: warp w takes dims 64 w .. 64 w + 63 (B operand = the same rows read with ldmatrix.trans).
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const void *p) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], const void *p) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+constexpr int MLA_CP = 8;           // halfs of padding per cache / query row (rows stay 16-byte aligned, ldmatrix conflict-free)
+constexpr int MLA_PP = 8;           // the same for the weight rows
+
+__global__ void __launch_bounds__(MLA_THREADS, 1)
+mla_split_mma_kernel(const float *__restrict__ q_lat, const float *__restrict__ q_rope, const __half *__restrict__ cache,
+                     const int *__restrict__ ctx, int n_heads, int d_c, int d_r, int max_context, int max_splits, float scale,
+                     float *__restrict__ part_o, float2 *__restrict__ part_ml) {
+  const int s = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_ctx = ctx[b];
+  const int t0 = s * MLA_SPLIT;
+  if (t0 >= n_ctx) return;
+  const int n = min(MLA_SPLIT, n_ctx - t0);
+  const int DK = d_c + d_r;                          // a multiple of 16 (d_c % 64 == 0, d_r % 16 == 0 on this path)
+  const int cp = DK + MLA_CP, pp = MLA_SPLIT + MLA_PP;
+  extern __shared__ __align__(16) unsigned char smem[];
+  __half *cs = reinterpret_cast<__half *>(smem);                     // [128][cp]   cache rows
+  __half *qh = cs + (size_t)MLA_SPLIT * cp;                          // [16][cp]    query hi
+  __half *ql = qh + (size_t)MLA_NH * cp;                             // [16][cp]    query lo
+  __half *ph = ql + (size_t)MLA_NH * cp;                             // [16][pp]    weights hi
+  __half *pl = ph + (size_t)MLA_NH * pp;                             // [16][pp]    weights lo
+  float *sc = reinterpret_cast<float *>(pl + (size_t)MLA_NH * pp);   // [16][128]   scores
+  float *red = sc + MLA_NH * MLA_SPLIT;                              // [16] maxima, [16] sums
+
+  // ---- the split's cache rows straight into shared memory (cp.async: the whole tile in flight at once)
+  {
+    const int vecs = DK / 8;
+    const __half *src = cache + ((size_t)b * max_context + t0) * DK;
+    const int total = MLA_SPLIT * vecs;
+    for (int i = tid; i < total; i += MLA_THREADS) {
+      const int t = i / vecs, j = i - t * vecs;
+      __half *d = cs + (size_t)t * cp + 8 * j;
+      if (t < n) {
+        const uint32_t da = (uint32_t)__cvta_generic_to_shared(d);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(da), "l"(src + (size_t)i * 8) : "memory");
+      } else {
+        *reinterpret_cast<uint4 *>(d) = make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+  // ---- the row's absorbed queries as fp16 hi + lo (eight independent loads per thread in flight)
+  for (int i0 = tid; i0 < DK * MLA_NH; i0 += MLA_THREADS * 8) {
+    float v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int i = i0 + MLA_THREADS * k;
+      const int h = i / DK, d = i - h * DK;
+      v[k] = 0.f;
+      if (i < DK * MLA_NH && h < n_heads)
+        v[k] = d < d_c ? q_lat[((size_t)b * n_heads + h) * d_c + d] : q_rope[((size_t)b * n_heads + h) * d_r + (d - d_c)];
+    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int i = i0 + MLA_THREADS * k;
+      if (i < DK * MLA_NH) {
+        const int h = i / DK, d = i - h * DK;
+        const __half hi = __float2half_rn(v[k]);
+        qh[h * cp + d] = hi;
+        ql[h * cp + d] = __float2half_rn(v[k] - __half2float(hi));
+      }
+    }
+  }
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  __syncthreads();
+
+  // ---- scores S[16 heads][tokens 16 warp ..]: two n8 tiles per warp
+  {
+    float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+    const int tok0 = 16 * warp;
+    // A (16 heads x 16 dims): lane -> row lane % 16, column block (lane / 16) * 8
+    const __half *a_hi = qh + (size_t)(lane & 15) * cp + (lane >> 4) * 8;
+    const __half *a_lo = ql + (size_t)(lane & 15) * cp + (lane >> 4) * 8;
+    // B (16 tokens x 16 dims as [token][dim]): matrices (tokens 0-7, dims 0-7), (0-7, 8-15), (8-15, 0-7), (8-15, 8-15)
+    const __half *bp = cs + (size_t)(tok0 + (lane & 7) + ((lane >> 4) << 3)) * cp + ((lane >> 3) & 1) * 8;
+    for (int k0 = 0; k0 < DK; k0 += 16) {
+      uint32_t ah[4], al[4], bb[4];
+      ldsm_x4(ah, a_hi + k0);
+      ldsm_x4(al, a_lo + k0);
+      ldsm_x4(bb, bp + k0);
+      mma16816(c0, ah, bb[0], bb[1]);
+      mma16816(c0, al, bb[0], bb[1]);
+      mma16816(c1, ah, bb[2], bb[3]);
+      mma16816(c1, al, bb[2], bb[3]);
+    }
+    // accumulator layout: rows lane / 4 and lane / 4 + 8, columns 2 (lane % 4), + 1 of each n8 tile
+    const int r0 = lane >> 2, cc = 2 * (lane & 3);
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int ta = tok0 + cc + j, tb = tok0 + 8 + cc + j;
+      sc[r0 * MLA_SPLIT + ta] = ta < n ? c0[j] * scale : -CUDART_INF_F;
+      sc[(r0 + 8) * MLA_SPLIT + ta] = ta < n ? c0[2 + j] * scale : -CUDART_INF_F;
+      sc[r0 * MLA_SPLIT + tb] = tb < n ? c1[j] * scale : -CUDART_INF_F;
+      sc[(r0 + 8) * MLA_SPLIT + tb] = tb < n ? c1[2 + j] * scale : -CUDART_INF_F;
+    }
+  }
+  __syncthreads();
+
+  // ---- softmax of the split per head (warp w: heads 2 w, 2 w + 1); weights as fp16 hi + lo rows
+  for (int h = 2 * warp; h < 2 * warp + 2; ++h) {
+    float v[4], m = -CUDART_INF_F;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { v[k] = sc[h * MLA_SPLIT + lane + 32 * k]; m = fmaxf(m, v[k]); }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    float l = 0.f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float p = expf(v[k] - m);
+      const __half hi = __float2half_rn(p);
+      ph[h * pp + lane + 32 * k] = hi;
+      pl[h * pp + lane + 32 * k] = __float2half_rn(p - __half2float(hi));
+      l += p;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+    if (lane == 0) { red[h] = m; red[MLA_NH + h] = l; }
+  }
+  __syncthreads();
+
+  // ---- O[16 heads][dims 64 warp ..] = P[16 x 128 tokens] * C[128 tokens x dims]: eight n8 tiles per warp and pass
+  for (int dbase = 64 * warp; dbase < d_c; dbase += 64 * (MLA_THREADS / 32)) {
+    float acc[8][4];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { acc[j][0] = 0.f; acc[j][1] = 0.f; acc[j][2] = 0.f; acc[j][3] = 0.f; }
+    const __half *a_hi = ph + (size_t)(lane & 15) * pp + (lane >> 4) * 8;
+    const __half *a_lo = pl + (size_t)(lane & 15) * pp + (lane >> 4) * 8;
+    // B (16 tokens x 16 dims stored [token][dim], read transposed): matrices (tokens 0-7, dims 0-7), (8-15, 0-7),
+    // (0-7, 8-15), (8-15, 8-15)
+    const __half *bp = cs + (size_t)((lane & 7) + ((lane >> 3) & 1) * 8) * cp + dbase + (lane >> 4) * 8;
+    for (int k0 = 0; k0 < MLA_SPLIT; k0 += 16) {
+      uint32_t ah[4], al[4];
+      ldsm_x4(ah, a_hi + k0);
+      ldsm_x4(al, a_lo + k0);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {                  // 16 dims per ldmatrix: two n8 tiles
+        uint32_t bb[4];
+        ldsm_x4_t(bb, bp + (size_t)k0 * cp + 16 * j);
+        mma16816(acc[2 * j], ah, bb[0], bb[1]);
+        mma16816(acc[2 * j], al, bb[0], bb[1]);
+        mma16816(acc[2 * j + 1], ah, bb[2], bb[3]);
+        mma16816(acc[2 * j + 1], al, bb[2], bb[3]);
+      }
+    }
+    const int r0 = lane >> 2, cc = 2 * (lane & 3);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int d = dbase + 8 * j + cc;
+      if (r0 < n_heads)
+        *reinterpret_cast<float2 *>(part_o + (((size_t)b * max_splits + s) * n_heads + r0) * d_c + d) = make_float2(acc[j][0], acc[j][1]);
+      if (r0 + 8 < n_heads)
+        *reinterpret_cast<float2 *>(part_o + (((size_t)b * max_splits + s) * n_heads + r0 + 8) * d_c + d) = make_float2(acc[j][2], acc[j][3]);
+    }
+  }
+  if (tid < n_heads) part_ml[((size_t)b * max_splits + s) * n_heads + tid] = make_float2(red[tid], red[MLA_NH + tid]);
+}
+
+size_t mla_mma_smem_bytes(int d_c, int d_r) {
+  const int DK = d_c + d_r;
+  return (size_t)(MLA_SPLIT + 2 * MLA_NH) * (DK + MLA_CP) * 2 + (size_t)2 * MLA_NH * (MLA_SPLIT + MLA_PP) * 2 +
+         (size_t)MLA_NH * MLA_SPLIT * 4 + 2 * MLA_NH * 4;
+}
+
 // One CTA per (head, row): the row's splits in ascending order.
 __global__ void __launch_bounds__(MLA_THREADS)
 mla_combine_kernel(const float *__restrict__ part_o, const float2 *__restrict__ part_ml, const int *__restrict__ ctx,
@@ -183,18 +366,26 @@ int corun_mla_attend(const float *q_lat, const float *q_rope, const void *cache,
                      int32_t n_heads, int32_t d_latent, int32_t d_rope, int32_t max_context, float scale, float *o_lat,
                      float *ws, void *cuda_stream) {
   if (!q_lat || !q_rope || !cache || !ctx || !o_lat || !ws || B < 1 || B > 65535 || n_heads < 4 || n_heads > MLA_NH ||
-      n_heads % 4 || d_latent < 64 || d_latent > 512 || d_latent % 64 || d_rope < 2 || d_rope > 64 || d_rope % 2 ||
+      n_heads % 4 || d_latent < 64 || d_latent > 512 || d_latent % 64 || d_rope < 8 || d_rope > 64 || d_rope % 8 ||
       max_context < 1)
     return CORUN_EINVAL;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const int max_splits = (max_context + MLA_SPLIT - 1) / MLA_SPLIT;
-  const size_t smem = mla_smem_bytes(d_latent, d_rope);
-  cudaError_t ce = cudaFuncSetAttribute(mla_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  // the warp-level tensor path needs whole k16 steps and 64-dim passes; otherwise (or on request) plain FMAs
+  const bool use_mma = d_rope % 16 == 0 && !(getenv("CORUN_MLA_FMA") && atoi(getenv("CORUN_MLA_FMA")) != 0);
+  const size_t smem = use_mma ? mla_mma_smem_bytes(d_latent, d_rope) : mla_smem_bytes(d_latent, d_rope);
+  cudaError_t ce = use_mma ? cudaFuncSetAttribute(mla_split_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                           : cudaFuncSetAttribute(mla_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (ce != cudaSuccess) { corun::g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
   float *part_o = ws;
   float2 *part_ml = reinterpret_cast<float2 *>(ws + (size_t)B * max_splits * n_heads * d_latent);
-  mla_split_kernel<<<dim3(max_splits, B), MLA_THREADS, smem, st>>>(q_lat, q_rope, (const __half *)cache, ctx, n_heads, d_latent,
-                                                                  d_rope, max_context, max_splits, scale, part_o, part_ml);
+  if (use_mma)
+    mla_split_mma_kernel<<<dim3(max_splits, B), MLA_THREADS, smem, st>>>(q_lat, q_rope, (const __half *)cache, ctx, n_heads,
+                                                                        d_latent, d_rope, max_context, max_splits, scale, part_o,
+                                                                        part_ml);
+  else
+    mla_split_kernel<<<dim3(max_splits, B), MLA_THREADS, smem, st>>>(q_lat, q_rope, (const __half *)cache, ctx, n_heads, d_latent,
+                                                                    d_rope, max_context, max_splits, scale, part_o, part_ml);
   mla_combine_kernel<<<dim3(n_heads, B), MLA_THREADS, 0, st>>>(part_o, part_ml, ctx, n_heads, d_latent, max_splits, o_lat);
   ce = cudaGetLastError();
   if (ce != cudaSuccess) { corun::g_last_cuda_error = (int)ce; return CORUN_ECUDA; }

@@ -9,7 +9,7 @@ from oracle import mla_oracle as ml
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("nh,dc,dr", [(16, 512, 64), (4, 64, 2), (8, 128, 32)])
+@pytest.mark.parametrize("nh,dc,dr", [(16, 512, 64), (4, 64, 8), (8, 128, 32), (16, 512, 24)])
 def test_mla_attend_matches_oracle_and_rows_are_independent(nh, dc, dr):
     torch = pytest.importorskip("torch")
     if not torch.cuda.is_available():
