@@ -1,8 +1,9 @@
 /*
  * Multi-head latent attention (MLA) for one query token per row at decode time, in the absorbed form, for
- * NVIDIA B200 (sm_100a).  FIRST CORRECT PATH: plain fp32 FMA arithmetic on the CUDA cores (the contraction is
- * tensor-core work at ~30 FLOP per cached byte; a tcgen05 kernel is the next step), request-local split of
- * 128 cached tokens, splits combined in ascending order.
+ * NVIDIA B200 (sm_100a).  The contraction runs on the warp-level tensor path (mma.sync m16n8k16, fp16 operands,
+ * fp32 accumulation): one CTA per row and chunk of 512 cached tokens streams the chunk in tiles of 64 tokens
+ * through shared memory with an online softmax; the chunks of a row are combined in ascending order.  (A plain
+ * fp32 FMA kernel over splits of 128 tokens serves the shapes the tensor path does not take.)
  *
  * The paper evaluates an MLA model (Evaluation, "Setup") and turns decode-time Split-KV off because its split
  * count depends on the batch (Design, "Fixed-Shape Batched Decode"); here, as in the dense attention kernel,
@@ -38,11 +39,16 @@ int64_t corun_mla_workspace_floats(int32_t B, int32_t n_heads, int32_t d_latent,
  *   ws      corun_mla_workspace_floats(...) floats
  * n_heads 1..16 (a multiple of 4), d_latent a multiple of 64 up to 512, d_rope a multiple of 8 up to 64
  * (cache rows are then 16-byte aligned).
+ * operand_pairs  1: the fp32 queries and softmax weights enter the tensor cores as fp16 hi + lo pairs (two
+ *                   instructions per tile; results agree with fp64 to ~1e-5);
+ *                0: as single fp16 values, the precision of a conventional fp16 attention kernel, at half the
+ *                   tensor work (needs d_rope a multiple of 16; the weight sum runs over the rounded weights).
+ *                Either way a row's result depends on the row alone.
  * Errors: EINVAL, ECUDA.
  */
 int corun_mla_attend(const float *q_lat, const float *q_rope, const void *cache, const int32_t *ctx, int32_t B,
                      int32_t n_heads, int32_t d_latent, int32_t d_rope, int32_t max_context, float scale, float *o_lat,
-                     float *ws, void *cuda_stream);
+                     float *ws, int32_t operand_pairs, void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -216,20 +216,22 @@ def case_mla(a):
     q_rope = torch.randn((a.B, nh, dr), generator=g, device="cuda")
     dctx = torch.tensor(ctx).cuda()
     scale = 1.0 / math.sqrt(128 + dr)
+    pairs = not a.single
     for _ in range(3):
-        out = corun.mla_attend(q_lat, q_rope, cache, dctx, scale)
+        out = corun.mla_attend(q_lat, q_rope, cache, dctx, scale, pairs)
     torch.cuda.synchronize()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
     for _ in range(a.reps):
-        out = corun.mla_attend(q_lat, q_rope, cache, dctx, scale)
+        out = corun.mla_attend(q_lat, q_rope, cache, dctx, scale, pairs)
     t1.record()
     torch.cuda.synchronize()
     ms = t0.elapsed_time(t1) / a.reps
     nbytes = int(ctx.astype(np.int64).sum()) * (dc + dr) * 2
     flops = int(ctx.astype(np.int64).sum()) * nh * (dc + dr + dc) * 2
-    print("mla: B=%d, contexts %d..%d (mean %.0f): %.1f us per call, %.1f MB of latent cache -> %.0f GB/s, %.1f TFLOP/s (fp32 FMA)"
-          % (a.B, ctx.min(), ctx.max(), ctx.mean(), ms * 1e3, nbytes / 1e6, nbytes / ms / 1e6, flops / ms / 1e9))
+    print("mla: B=%d, contexts %d..%d (mean %.0f): %.1f us per call, %.1f MB of latent cache -> %.0f GB/s, %.1f TFLOP/s (%s)"
+          % (a.B, ctx.min(), ctx.max(), ctx.mean(), ms * 1e3, nbytes / 1e6, nbytes / ms / 1e6, flops / ms / 1e9,
+             "fp16 hi+lo operand pairs" if pairs else "single fp16 operands"))
     assert bool(torch.isfinite(out).all().item())
 
 
@@ -520,6 +522,7 @@ def main():
     ma = sub.add_parser("mla")
     ma.add_argument("--B", type=int, default=128); ma.add_argument("--ctx-lo", type=int, default=512)
     ma.add_argument("--ctx-hi", type=int, default=4096); ma.add_argument("--reps", type=int, default=10)
+    ma.add_argument("--single", action="store_true", help="single fp16 operands instead of hi + lo pairs")
     ab = sub.add_parser("ablation")
     ab.add_argument("--layers", type=int, default=2); ab.add_argument("--B", type=int, default=64)
     ab.add_argument("--actives", default="1,4,16,40,64"); ab.add_argument("--ctx-lo", type=int, default=512)

@@ -515,10 +515,11 @@ class MoeFfn:
             pass
 
 
-def mla_attend(q_lat, q_rope, cache, ctx, scale: float):
+def mla_attend(q_lat, q_rope, cache, ctx, scale: float, operand_pairs: bool = True):
     """Absorbed multi-head latent attention for one query token per row (``include/corun_mla.h``).
     q_lat fp32 [B, n_heads, d_c], q_rope fp32 [B, n_heads, d_r], cache fp16 [B, T, d_c + d_r], ctx int32 [B]
-    (all CUDA tensors) -> o_lat fp32 [B, n_heads, d_c] (rows with ctx 0 are left as zeros)."""
+    (all CUDA tensors) -> o_lat fp32 [B, n_heads, d_c] (rows with ctx 0 are left as zeros).  operand_pairs:
+    queries and softmax weights as fp16 hi + lo pairs (fp32-grade) or as single fp16 values (half the tensor work)."""
     import torch
 
     B, nh, dc = q_lat.shape
@@ -531,10 +532,11 @@ def mla_attend(q_lat, q_rope, cache, ctx, scale: float):
     L = lib()
     L.corun_mla_workspace_floats.restype = C.c_int64
     L.corun_mla_workspace_floats.argtypes = [C.c_int32] * 4
-    L.corun_mla_attend.argtypes = [C.c_void_p] * 4 + [C.c_int32] * 5 + [C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.corun_mla_attend.argtypes = [C.c_void_p] * 4 + [C.c_int32] * 5 + [C.c_float, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
     ws = torch.empty(int(L.corun_mla_workspace_floats(B, nh, dc, T)), dtype=torch.float32, device=q_lat.device)
     out = torch.zeros_like(q_lat)
     _check(L.corun_mla_attend(q_lat.data_ptr(), q_rope.data_ptr(), cache.data_ptr(), ctx.data_ptr(), B, nh, dc, dr, T,
-                              float(scale), out.data_ptr(), ws.data_ptr(), torch.cuda.current_stream().cuda_stream),
+                              float(scale), out.data_ptr(), ws.data_ptr(), 1 if operand_pairs else 0,
+                              torch.cuda.current_stream().cuda_stream),
            "corun_mla_attend")
     return out

@@ -1,8 +1,9 @@
-// Multi-head latent attention at decode time in the absorbed form, first correct path: fp32 FMA arithmetic on
-// the CUDA cores (see include/corun_mla.h).  One CTA per (row, split of 128 cached tokens): the split's latent
-// rows and the row's absorbed queries are staged in shared memory, scores / softmax / weighted latent sum are
-// computed there, the split's (max, sum, output) goes to the workspace; a second kernel combines a row's
-// splits in ascending order.  Split size fixed, split count = f(own context): nothing depends on other rows.
+// Multi-head latent attention at decode time in the absorbed form (see include/corun_mla.h).  Three kernels
+// compute a row's partial (max, sum, output) per fixed-size piece of its cached tokens and a fourth combines
+// the pieces in ascending order: mla_split_kernel (fp32 FMAs, 128-token splits), mla_split_mma_kernel
+// (mma.sync, 128-token splits, staged then computed) and mla_chunk_mma_kernel (mma.sync, 512-token chunks
+// streamed in 64-token tiles with an online softmax: the default).  Piece sizes are fixed and the piece count
+// is a function of the row's own context: nothing depends on other rows.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <math_constants.h>
@@ -320,6 +321,235 @@ mla_split_mma_kernel(const float *__restrict__ q_lat, const float *__restrict__ 
   if (tid < n_heads) part_ml[((size_t)b * max_splits + s) * n_heads + tid] = make_float2(red[tid], red[MLA_NH + tid]);
 }
 
+// ---------------------------------------------------------------- pipelined version of the same path
+// One CTA of 16 warps per (row, chunk of MLA_CHUNK cached tokens).  The chunk's tiles of 64 tokens stream through
+// two shared-memory buffers with cp.async (tile i + 1 loads while tile i is computed); the softmax runs online
+// over the tiles in ascending order (running maximum M, sum l and output O per head, O in the mma accumulators).
+// Instruction issue and shared-memory traffic are the scarce resources (every operand of mma.sync passes through
+// ldmatrix), so the queries never touch shared memory: warp w keeps the fp16 hi / lo A fragments of K group w & 3 (a quarter of the k16 steps
+// of d_c + d_r) in registers for the whole chunk and multiplies them with tokens 16 (w >> 2) .. + 15 of each tile;
+// the four K groups' partial scores are added in a fixed order by the softmax.  The cache tile is read once for
+// the scores and once (transposed) for the output: warp w owns dims 32 w .. 32 w + 31 of O.  The chunk's
+// (M, l, O) goes to the workspace; chunks are combined in ascending order.  Chunk and tile sizes are fixed, so a
+// row's arithmetic depends on its own context length only.
+constexpr int MLA_CHUNK = 512;
+constexpr int MLA_TILE = 64;
+constexpr int MLA_TP = MLA_TILE + 8;   // halfs per weight row
+constexpr int MLA_SP = MLA_TILE + 8;   // floats per partial-score row (conflict-free float2 stores)
+constexpr int MLA_KG = 4;              // K groups
+constexpr int MLA_CTHREADS = 512;     // 16 warps
+constexpr int MLA_KS = 9;              // k16 steps per K group at most: d_c + d_r <= 576
+
+__device__ __forceinline__ void split_half2(float2 v, uint32_t &hi, uint32_t &lo) {
+  const __half2 h = __floats2half2_rn(v.x, v.y);
+  const float2 back = __half22float2(h);
+  const __half2 l = __floats2half2_rn(v.x - back.x, v.y - back.y);
+  hi = *reinterpret_cast<const uint32_t *>(&h);
+  lo = *reinterpret_cast<const uint32_t *>(&l);
+}
+
+template <bool PAIRS>
+__global__ void __launch_bounds__(MLA_CTHREADS, 1)
+mla_chunk_mma_kernel(const float *__restrict__ q_lat, const float *__restrict__ q_rope, const __half *__restrict__ cache,
+                     const int *__restrict__ ctx, int n_heads, int d_c, int d_r, int max_context, int max_chunks, float scale,
+                     float *__restrict__ part_o, float2 *__restrict__ part_ml) {
+  const int ch = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_ctx = ctx[b];
+  const int t_begin = ch * MLA_CHUNK;
+  if (t_begin >= n_ctx) return;
+  const int n_chunk = min(MLA_CHUNK, n_ctx - t_begin);
+  const int n_tiles = (n_chunk + MLA_TILE - 1) / MLA_TILE;
+  const int DK = d_c + d_r, cp = DK + MLA_CP;
+  extern __shared__ __align__(16) unsigned char smem[];
+  __half *cs = reinterpret_cast<__half *>(smem);                     // [2][64][cp]
+  __half *ph = cs + (size_t)2 * MLA_TILE * cp;                       // [16][MLA_TP] weights hi, then the same for lo
+  float *sc = reinterpret_cast<float *>(ph + (size_t)2 * MLA_NH * MLA_TP);   // [4 K groups][16][MLA_SP] partial scores
+  float *run_m = sc + MLA_KG * MLA_NH * MLA_SP;                      // [16] running maxima
+  float *run_l = run_m + MLA_NH;                                     // [16] running sums
+  float *fac = run_l + MLA_NH;                                       // [16] rescale factors of the current tile
+  const int r0 = lane >> 2, cc = 2 * (lane & 3);
+
+  auto load_tile = [&](int ti) {
+    const int t0 = t_begin + ti * MLA_TILE;
+    const int n = min(MLA_TILE, n_ctx - t0);
+    __half *dst = cs + (size_t)(ti & 1) * MLA_TILE * cp;
+    const int vecs = DK / 8;
+    const __half *src = cache + ((size_t)b * max_context + t0) * DK;
+    // warp w: tokens w, w + 16, ...; its lanes the 16-byte pieces of the row
+#pragma unroll
+    for (int t = warp; t < MLA_TILE; t += MLA_CTHREADS / 32) {
+      __half *d = dst + (size_t)t * cp;
+      if (t < n) {
+        const __half *g = src + (size_t)t * DK;
+        for (int j = lane; j < vecs; j += 32) {
+          const uint32_t da = (uint32_t)__cvta_generic_to_shared(d + 8 * j);
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(da), "l"(g + 8 * j) : "memory");
+        }
+      } else {
+        for (int j = lane; j < vecs; j += 32) *reinterpret_cast<uint4 *>(d + 8 * j) = make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  load_tile(0);
+
+  // ---- this warp's query fragments (A operand of m16n8k16: rows = heads, k = 16 dims per step), hi and lo
+  const int kg = warp & (MLA_KG - 1), tg = warp >> 2;   // tg 0..3: tokens 16 tg .. 16 tg + 15 of a tile
+  const int ksteps = DK / 16, per_group = (ksteps + MLA_KG - 1) / MLA_KG;
+  const int my_first = kg * per_group, my_steps = max(0, min(per_group, ksteps - my_first));
+  uint32_t qa_hi[MLA_KS][4], qa_lo[MLA_KS][4];
+#pragma unroll
+  for (int i = 0; i < MLA_KS; ++i) {
+    float2 v[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+    if (i < my_steps) {
+      const int k0 = (my_first + i) * 16;            // a step lies wholly in the latent or in the rotary part
+      const bool lat = k0 < d_c;
+      const float *base = lat ? q_lat + (size_t)b * n_heads * d_c + k0 : q_rope + (size_t)b * n_heads * d_r + (k0 - d_c);
+      const int pitch = lat ? d_c : d_r;
+      if (r0 < n_heads) {
+        v[0] = *reinterpret_cast<const float2 *>(base + (size_t)r0 * pitch + cc);
+        v[2] = *reinterpret_cast<const float2 *>(base + (size_t)r0 * pitch + cc + 8);
+      }
+      if (r0 + 8 < n_heads) {
+        v[1] = *reinterpret_cast<const float2 *>(base + (size_t)(r0 + 8) * pitch + cc);
+        v[3] = *reinterpret_cast<const float2 *>(base + (size_t)(r0 + 8) * pitch + cc + 8);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) split_half2(v[j], qa_hi[i][j], qa_lo[i][j]);
+  }
+  if (tid < MLA_NH) { run_m[tid] = -CUDART_INF_F; run_l[tid] = 0.f; }
+
+  // this warp's output accumulators: dims dbase .. dbase + 31 of all heads (only warps with dbase < d_c have any)
+  const int dbase = 32 * warp;
+  float acc[4][4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) { acc[j][0] = 0.f; acc[j][1] = 0.f; acc[j][2] = 0.f; acc[j][3] = 0.f; }
+
+  for (int ti = 0; ti < n_tiles; ++ti) {
+    if (ti + 1 < n_tiles) {
+      load_tile(ti + 1);                             // into the other buffer: its readers passed the loop's last barrier
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();                                 // tile ti is in shared memory
+    const __half *ct = cs + (size_t)(ti & 1) * MLA_TILE * cp;
+    const int n = min(MLA_TILE, n_chunk - ti * MLA_TILE);
+    // ---- partial scores of K group kg for heads x tokens 16 tg .. 16 tg + 15 (two n8 tiles, hi and lo chains)
+    {
+      float c_hi[2][4], c_lo[2][4];
+#pragma unroll
+      for (int j = 0; j < 2; ++j)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { c_hi[j][e] = 0.f; c_lo[j][e] = 0.f; }
+      // B (16 tokens x 16 dims as [token][dim]): matrices (tokens 0-7, dims 0-7), (0-7, 8-15), (8-15, 0-7), (8-15, 8-15)
+      const __half *bp = ct + (size_t)(16 * tg + (lane & 7) + ((lane >> 4) << 3)) * cp + ((lane >> 3) & 1) * 8 + my_first * 16;
+#pragma unroll
+      for (int i = 0; i < MLA_KS; ++i) {
+        if (i < my_steps) {
+          uint32_t b0[4];
+          ldsm_x4(b0, bp + i * 16);
+          mma16816(c_hi[0], qa_hi[i], b0[0], b0[1]);
+          mma16816(c_hi[1], qa_hi[i], b0[2], b0[3]);
+          if (PAIRS) {
+            mma16816(c_lo[0], qa_lo[i], b0[0], b0[1]);
+            mma16816(c_lo[1], qa_lo[i], b0[2], b0[3]);
+          }
+        }
+      }
+      float *so = sc + (size_t)kg * MLA_NH * MLA_SP;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int t = 16 * tg + 8 * j + cc;
+        *reinterpret_cast<float2 *>(so + r0 * MLA_SP + t) = make_float2(c_hi[j][0] + c_lo[j][0], c_hi[j][1] + c_lo[j][1]);
+        *reinterpret_cast<float2 *>(so + (r0 + 8) * MLA_SP + t) = make_float2(c_hi[j][2] + c_lo[j][2], c_hi[j][3] + c_lo[j][3]);
+      }
+    }
+    __syncthreads();
+    // ---- online softmax: warp w = head w; the K groups' parts are added in a fixed order
+    {
+      const int h = warp;
+      const float *s0 = sc + h * MLA_SP, *s1 = s0 + MLA_NH * MLA_SP, *s2 = s1 + MLA_NH * MLA_SP, *s3 = s2 + MLA_NH * MLA_SP;
+      const float v0 = lane < n ? ((s0[lane] + s1[lane]) + (s2[lane] + s3[lane])) * scale : -CUDART_INF_F;
+      const float v1 = lane + 32 < n ? ((s0[lane + 32] + s1[lane + 32]) + (s2[lane + 32] + s3[lane + 32])) * scale : -CUDART_INF_F;
+      float m = fmaxf(v0, v1);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      const float M_old = run_m[h], M_new = fmaxf(M_old, m);
+      const float p0 = __expf(v0 - M_new), p1 = __expf(v1 - M_new);
+      const __half h0 = __float2half_rn(p0), h1 = __float2half_rn(p1);
+      __half *wh = ph + (size_t)h * MLA_TP, *wl = ph + (size_t)(MLA_NH + h) * MLA_TP;
+      wh[lane] = h0;
+      wh[lane + 32] = h1;
+      if (PAIRS) {
+        wl[lane] = __float2half_rn(p0 - __half2float(h0));
+        wl[lane + 32] = __float2half_rn(p1 - __half2float(h1));
+      }
+      // without the lo parts the sum runs over the rounded weights, so that numerator and denominator agree
+      float l = PAIRS ? p0 + p1 : __half2float(h0) + __half2float(h1);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+      __syncwarp();
+      if (lane == 0) {
+        const float f = __expf(M_old - M_new);       // 0 the first time (M_old = -inf)
+        fac[h] = f;
+        run_l[h] = run_l[h] * f + l;
+        run_m[h] = M_new;
+      }
+    }
+    __syncthreads();
+    // ---- O = O * f + P[16 x 64 tokens] * C[64 tokens x dims]
+    if (dbase < d_c) {
+      const float f0 = fac[r0], f1 = fac[r0 + 8];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { acc[j][0] *= f0; acc[j][1] *= f0; acc[j][2] *= f1; acc[j][3] *= f1; }
+      const __half *a_hi = ph + (size_t)(lane & 15) * MLA_TP + (lane >> 4) * 8;
+      const __half *a_lo = a_hi + (size_t)MLA_NH * MLA_TP;
+      // B (16 tokens x 16 dims stored [token][dim], read transposed): matrices (tokens 0-7, dims 0-7), (8-15, 0-7),
+      // (0-7, 8-15), (8-15, 8-15)
+      const __half *bp = ct + (size_t)((lane & 7) + ((lane >> 3) & 1) * 8) * cp + dbase + (lane >> 4) * 8;
+#pragma unroll
+      for (int k0 = 0; k0 < MLA_TILE; k0 += 16) {
+        uint32_t ah[4], al[4];
+        ldsm_x4(ah, a_hi + k0);
+        if (PAIRS) ldsm_x4(al, a_lo + k0);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          uint32_t bb[4];
+          ldsm_x4_t(bb, bp + (size_t)k0 * cp + 16 * j);
+          mma16816(acc[2 * j], ah, bb[0], bb[1]);
+          mma16816(acc[2 * j + 1], ah, bb[2], bb[3]);
+          if (PAIRS) {
+            mma16816(acc[2 * j], al, bb[0], bb[1]);
+            mma16816(acc[2 * j + 1], al, bb[2], bb[3]);
+          }
+        }
+      }
+    }
+    // the next iteration starts a load into the other buffer and rewrites the score and weight tiles: everyone
+    // must have finished this iteration's reads of the weights (and the previous one's of that buffer) first
+    __syncthreads();
+  }
+  if (dbase < d_c) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int d = dbase + 8 * j + cc;
+      if (r0 < n_heads)
+        *reinterpret_cast<float2 *>(part_o + (((size_t)b * max_chunks + ch) * n_heads + r0) * d_c + d) = make_float2(acc[j][0], acc[j][1]);
+      if (r0 + 8 < n_heads)
+        *reinterpret_cast<float2 *>(part_o + (((size_t)b * max_chunks + ch) * n_heads + r0 + 8) * d_c + d) = make_float2(acc[j][2], acc[j][3]);
+    }
+  }
+  if (tid < n_heads) part_ml[((size_t)b * max_chunks + ch) * n_heads + tid] = make_float2(run_m[tid], run_l[tid]);
+}
+
+size_t mla_chunk_smem_bytes(int d_c, int d_r) {
+  const int DK = d_c + d_r;
+  return (size_t)2 * MLA_TILE * (DK + MLA_CP) * 2 + (size_t)2 * MLA_NH * MLA_TP * 2 +
+         (size_t)MLA_KG * MLA_NH * MLA_SP * 4 + 3 * MLA_NH * 4 + 64;   // + slack: the last row's ldmatrix may read past its padding
+}
+
 size_t mla_mma_smem_bytes(int d_c, int d_r) {
   const int DK = d_c + d_r;
   return (size_t)(MLA_SPLIT + 2 * MLA_NH) * (DK + MLA_CP) * 2 + (size_t)2 * MLA_NH * (MLA_SPLIT + MLA_PP) * 2 +
@@ -329,11 +559,11 @@ size_t mla_mma_smem_bytes(int d_c, int d_r) {
 // One CTA per (head, row): the row's splits in ascending order.
 __global__ void __launch_bounds__(MLA_THREADS)
 mla_combine_kernel(const float *__restrict__ part_o, const float2 *__restrict__ part_ml, const int *__restrict__ ctx,
-                   int n_heads, int d_c, int max_splits, float *__restrict__ o_lat) {
+                   int n_heads, int d_c, int max_splits, int split_len, float *__restrict__ o_lat) {
   const int h = blockIdx.x, b = blockIdx.y;
   const int n_ctx = ctx[b];
   if (n_ctx <= 0) return;
-  const int ns = (n_ctx + MLA_SPLIT - 1) / MLA_SPLIT;
+  const int ns = (n_ctx + split_len - 1) / split_len;
   const float2 *ml = part_ml + (size_t)b * max_splits * n_heads + h;
   float M = -CUDART_INF_F;
   for (int s = 0; s < ns; ++s) M = fmaxf(M, ml[(size_t)s * n_heads].x);
@@ -364,20 +594,41 @@ int64_t corun_mla_workspace_floats(int32_t B, int32_t n_heads, int32_t d_latent,
 
 int corun_mla_attend(const float *q_lat, const float *q_rope, const void *cache, const int32_t *ctx, int32_t B,
                      int32_t n_heads, int32_t d_latent, int32_t d_rope, int32_t max_context, float scale, float *o_lat,
-                     float *ws, void *cuda_stream) {
+                     float *ws, int32_t operand_pairs, void *cuda_stream) {
   if (!q_lat || !q_rope || !cache || !ctx || !o_lat || !ws || B < 1 || B > 65535 || n_heads < 4 || n_heads > MLA_NH ||
       n_heads % 4 || d_latent < 64 || d_latent > 512 || d_latent % 64 || d_rope < 8 || d_rope > 64 || d_rope % 8 ||
-      max_context < 1)
+      max_context < 1 || (operand_pairs != 0 && operand_pairs != 1))
     return CORUN_EINVAL;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const int max_splits = (max_context + MLA_SPLIT - 1) / MLA_SPLIT;
   // the warp-level tensor path needs whole k16 steps and 64-dim passes; otherwise (or on request) plain FMAs
-  const bool use_mma = d_rope % 16 == 0 && !(getenv("CORUN_MLA_FMA") && atoi(getenv("CORUN_MLA_FMA")) != 0);
+  if (reinterpret_cast<uintptr_t>(cache) % 16) return CORUN_EINVAL;
+  auto env_on = [](const char *name) { const char *v = getenv(name); return v && atoi(v) != 0; };
+  // single fp16 operands exist on the pipelined tensor path only
+  if (!operand_pairs && (d_rope % 16 != 0 || env_on("CORUN_MLA_FMA") || env_on("CORUN_MLA_UNPIPELINED"))) return CORUN_EINVAL;
+  const bool use_mma = d_rope % 16 == 0 && !env_on("CORUN_MLA_FMA");
+  const bool use_chunk = use_mma && !env_on("CORUN_MLA_UNPIPELINED");
+  float *part_o = ws;
+  if (use_chunk) {
+    // pipelined path: chunks of MLA_CHUNK tokens (the workspace, sized for 128-token splits, is large enough)
+    const int max_chunks = (max_context + MLA_CHUNK - 1) / MLA_CHUNK;
+    const size_t smem = mla_chunk_smem_bytes(d_latent, d_rope);
+    auto kern = operand_pairs ? mla_chunk_mma_kernel<true> : mla_chunk_mma_kernel<false>;
+    cudaError_t ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (ce != cudaSuccess) { corun::g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
+    float2 *part_ml = reinterpret_cast<float2 *>(ws + (size_t)B * max_chunks * n_heads * d_latent);
+    kern<<<dim3(max_chunks, B), MLA_CTHREADS, smem, st>>>(q_lat, q_rope, (const __half *)cache, ctx, n_heads, d_latent, d_rope,
+                                                        max_context, max_chunks, scale, part_o, part_ml);
+    mla_combine_kernel<<<dim3(n_heads, B), MLA_THREADS, 0, st>>>(part_o, part_ml, ctx, n_heads, d_latent, max_chunks, MLA_CHUNK,
+                                                                o_lat);
+    ce = cudaGetLastError();
+    if (ce != cudaSuccess) { corun::g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
+    return CORUN_OK;
+  }
   const size_t smem = use_mma ? mla_mma_smem_bytes(d_latent, d_rope) : mla_smem_bytes(d_latent, d_rope);
   cudaError_t ce = use_mma ? cudaFuncSetAttribute(mla_split_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
                            : cudaFuncSetAttribute(mla_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (ce != cudaSuccess) { corun::g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
-  float *part_o = ws;
   float2 *part_ml = reinterpret_cast<float2 *>(ws + (size_t)B * max_splits * n_heads * d_latent);
   if (use_mma)
     mla_split_mma_kernel<<<dim3(max_splits, B), MLA_THREADS, smem, st>>>(q_lat, q_rope, (const __half *)cache, ctx, n_heads,
@@ -386,7 +637,8 @@ int corun_mla_attend(const float *q_lat, const float *q_rope, const void *cache,
   else
     mla_split_kernel<<<dim3(max_splits, B), MLA_THREADS, smem, st>>>(q_lat, q_rope, (const __half *)cache, ctx, n_heads, d_latent,
                                                                     d_rope, max_context, max_splits, scale, part_o, part_ml);
-  mla_combine_kernel<<<dim3(n_heads, B), MLA_THREADS, 0, st>>>(part_o, part_ml, ctx, n_heads, d_latent, max_splits, o_lat);
+  mla_combine_kernel<<<dim3(n_heads, B), MLA_THREADS, 0, st>>>(part_o, part_ml, ctx, n_heads, d_latent, max_splits, MLA_SPLIT,
+                                                              o_lat);
   ce = cudaGetLastError();
   if (ce != cudaSuccess) { corun::g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
   return CORUN_OK;
