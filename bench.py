@@ -366,6 +366,35 @@ def run_corun(args, rank, world):
         op.close()
         del op, xm
 
+    # ---- MLA decode attention (DeepSeek-V2-Lite attention shape, 128 rows, the decode workload's context range):
+    # time per call with CUDA events against the bytes of latent cache a call streams (rank 0, full size only)
+    mla = None
+    if rank == 0 and sh.n_layers > 8 and not moe_cfg:
+        import math
+        from paper_2608_14376_b200.corun import mla_attend
+        gl = torch.Generator(device="cuda").manual_seed(4)
+        lB, lh, ldc, ldr = 128, 16, 512, 64
+        lctx = synth.uniform_lengths(512, 4096, lB, seed=2).astype(np.int32)
+        lT = int(-(-int(lctx.max()) // 128) * 128)
+        lcache = (torch.randn((lB, lT, ldc + ldr), generator=gl, device="cuda") * 0.5).to(torch.float16)
+        lq, lr = torch.randn((lB, lh, ldc), generator=gl, device="cuda"), torch.randn((lB, lh, ldr), generator=gl, device="cuda")
+        ldctx = torch.tensor(lctx).cuda()
+        lbytes = int(lctx.astype(np.int64).sum()) * (ldc + ldr) * 2
+        mla = {"workload": "deepseek_v2_lite_mla_b128", "contexts": f"uniform {lctx.min()}..{lctx.max()}", "cache_bytes": lbytes}
+        for name, pairs in (("fp16_pairs", True), ("single_fp16", False)):
+            for _ in range(3):
+                mla_attend(lq, lr, lcache, ldctx, 1.0 / math.sqrt(128 + ldr), pairs)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(20):
+                mla_attend(lq, lr, lcache, ldctx, 1.0 / math.sqrt(128 + ldr), pairs)
+            e1.record()
+            torch.cuda.synchronize()
+            lms = e0.elapsed_time(e1) / 20
+            mla[name] = {"us_per_call": lms * 1e3, "GBs": lbytes / lms / 1e6, "frac_of_measured_hbm": lbytes / lms / 1e6 / hbm}
+        del lcache, lq, lr
+
     cpu = None
     if rank == 0 and not args.no_cpu_baseline and not moe_cfg:
         w_np = synth.weights_torch_to_numpy(w_t)
@@ -398,7 +427,7 @@ def run_corun(args, rank, world):
         "clocks": clk, "gpu_launches": launches * K,
         "e2e": {"value": e2e_val, "unit": "tok/s", "ms_per_step": 1e3 * e2e_s / K,
                 "h2d_bytes_per_step": B * 9, "d2h_bytes_per_step": B * 4 + 4},
-        "roofline": roofline, "step_roofline": step_roof, "kernels": kernels, "prefill": prefill, "moe_ffn": moe,
+        "roofline": roofline, "step_roofline": step_roof, "kernels": kernels, "prefill": prefill, "moe_ffn": moe, "mla_attention": mla,
         "cpu_baseline": cpu,
     }))
 

@@ -326,7 +326,7 @@ mla_split_mma_kernel(const float *__restrict__ q_lat, const float *__restrict__ 
 // two shared-memory buffers with cp.async (tile i + 1 loads while tile i is computed); the softmax runs online
 // over the tiles in ascending order (running maximum M, sum l and output O per head, O in the mma accumulators).
 // Instruction issue and shared-memory traffic are the scarce resources (every operand of mma.sync passes through
-// ldmatrix), so the queries never touch shared memory: warp w keeps the fp16 hi / lo A fragments of K group w & 3 (a quarter of the k16 steps
+// ldmatrix), so the queries pass through shared memory once per chunk only: warp w keeps the fp16 hi / lo A fragments of K group w & 3 (a quarter of the k16 steps
 // of d_c + d_r) in registers for the whole chunk and multiplies them with tokens 16 (w >> 2) .. + 15 of each tile;
 // the four K groups' partial scores are added in a fixed order by the softmax.  The cache tile is read once for
 // the scores and once (transposed) for the output: warp w owns dims 32 w .. 32 w + 31 of O.  The chunk's
@@ -393,6 +393,24 @@ mla_chunk_mma_kernel(const float *__restrict__ q_lat, const float *__restrict__ 
   };
   load_tile(0);
 
+  // ---- the row's queries, fp32, through the second tile buffer (free until the loop starts): coalesced 16-byte
+  // loads, all of a thread's loads in flight at once
+  const int qp = DK + 8;                             // floats per staged query row
+  float *qs = reinterpret_cast<float *>(cs + (size_t)MLA_TILE * cp);   // [16][qp] <= one tile buffer
+  {
+    const float *gl = q_lat + (size_t)b * n_heads * d_c, *gr = q_rope + (size_t)b * n_heads * d_r;
+    const int quads = MLA_NH * DK / 4;               // a quad lies in one head and wholly in its latent or rotary part
+#pragma unroll 5
+    for (int i = tid; i < quads; i += MLA_CTHREADS) {
+      const int h = (4 * i) / DK, d = 4 * i - h * DK;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (h < n_heads)
+        v = d < d_c ? *reinterpret_cast<const float4 *>(gl + (size_t)h * d_c + d)
+                    : *reinterpret_cast<const float4 *>(gr + (size_t)h * d_r + (d - d_c));
+      *reinterpret_cast<float4 *>(qs + (size_t)h * qp + d) = v;
+    }
+  }
+  __syncthreads();
   // ---- this warp's query fragments (A operand of m16n8k16: rows = heads, k = 16 dims per step), hi and lo
   const int kg = warp & (MLA_KG - 1), tg = warp >> 2;   // tg 0..3: tokens 16 tg .. 16 tg + 15 of a tile
   const int ksteps = DK / 16, per_group = (ksteps + MLA_KG - 1) / MLA_KG;
@@ -402,22 +420,16 @@ mla_chunk_mma_kernel(const float *__restrict__ q_lat, const float *__restrict__ 
   for (int i = 0; i < MLA_KS; ++i) {
     float2 v[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
     if (i < my_steps) {
-      const int k0 = (my_first + i) * 16;            // a step lies wholly in the latent or in the rotary part
-      const bool lat = k0 < d_c;
-      const float *base = lat ? q_lat + (size_t)b * n_heads * d_c + k0 : q_rope + (size_t)b * n_heads * d_r + (k0 - d_c);
-      const int pitch = lat ? d_c : d_r;
-      if (r0 < n_heads) {
-        v[0] = *reinterpret_cast<const float2 *>(base + (size_t)r0 * pitch + cc);
-        v[2] = *reinterpret_cast<const float2 *>(base + (size_t)r0 * pitch + cc + 8);
-      }
-      if (r0 + 8 < n_heads) {
-        v[1] = *reinterpret_cast<const float2 *>(base + (size_t)(r0 + 8) * pitch + cc);
-        v[3] = *reinterpret_cast<const float2 *>(base + (size_t)(r0 + 8) * pitch + cc + 8);
-      }
+      const float *base = qs + (my_first + i) * 16 + cc;
+      v[0] = *reinterpret_cast<const float2 *>(base + (size_t)r0 * qp);
+      v[1] = *reinterpret_cast<const float2 *>(base + (size_t)(r0 + 8) * qp);
+      v[2] = *reinterpret_cast<const float2 *>(base + (size_t)r0 * qp + 8);
+      v[3] = *reinterpret_cast<const float2 *>(base + (size_t)(r0 + 8) * qp + 8);
     }
 #pragma unroll
     for (int j = 0; j < 4; ++j) split_half2(v[j], qa_hi[i][j], qa_lo[i][j]);
   }
+  __syncthreads();                                   // the buffer is free for the second tile
   if (tid < MLA_NH) { run_m[tid] = -CUDART_INF_F; run_l[tid] = 0.f; }
 
   // this warp's output accumulators: dims dbase .. dbase + 31 of all heads (only warps with dbase < d_c have any)
@@ -565,15 +577,48 @@ mla_combine_kernel(const float *__restrict__ part_o, const float2 *__restrict__ 
   if (n_ctx <= 0) return;
   const int ns = (n_ctx + split_len - 1) / split_len;
   const float2 *ml = part_ml + (size_t)b * max_splits * n_heads + h;
+  const float *po = part_o + ((size_t)b * max_splits * n_heads + h) * d_c;
+  const size_t o_stride = (size_t)n_heads * d_c;     // floats between a head's consecutive pieces
+  constexpr int FAST = 16;                           // pieces whose weights fit in registers
+  if (ns <= FAST) {
+    // all (max, sum) pairs in one round trip, the weights once, then all pieces of a dim in one round trip;
+    // the arithmetic (maximum first, ascending sums) is that of the general loop below
+    float2 v[FAST];
+#pragma unroll
+    for (int s = 0; s < FAST; ++s) v[s] = s < ns ? ml[(size_t)s * n_heads] : make_float2(-CUDART_INF_F, 0.f);
+    float M = -CUDART_INF_F;
+#pragma unroll
+    for (int s = 0; s < FAST; ++s) M = fmaxf(M, v[s].x);
+    float w[FAST], den = 0.f;
+#pragma unroll
+    for (int s = 0; s < FAST; ++s) {
+      w[s] = s < ns ? expf(v[s].x - M) : 0.f;
+      if (s < ns) den += w[s] * v[s].y;
+    }
+    const float inv = 1.f / den;
+    for (int d = 4 * threadIdx.x; d < d_c; d += 4 * blockDim.x) {
+      float4 x[FAST];
+#pragma unroll
+      for (int s = 0; s < FAST; ++s)
+        x[s] = s < ns ? *reinterpret_cast<const float4 *>(po + (size_t)s * o_stride + d) : make_float4(0.f, 0.f, 0.f, 0.f);
+      float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int s = 0; s < FAST; ++s) {
+        if (s < ns) { o.x = fmaf(w[s], x[s].x, o.x); o.y = fmaf(w[s], x[s].y, o.y); o.z = fmaf(w[s], x[s].z, o.z); o.w = fmaf(w[s], x[s].w, o.w); }
+      }
+      *reinterpret_cast<float4 *>(o_lat + ((size_t)b * n_heads + h) * d_c + d) = make_float4(o.x * inv, o.y * inv, o.z * inv, o.w * inv);
+    }
+    return;
+  }
   float M = -CUDART_INF_F;
   for (int s = 0; s < ns; ++s) M = fmaxf(M, ml[(size_t)s * n_heads].x);
   float den = 0.f;
   for (int s = 0; s < ns; ++s) den += expf(ml[(size_t)s * n_heads].x - M) * ml[(size_t)s * n_heads].y;
+  const float inv = 1.f / den;
   for (int d = threadIdx.x; d < d_c; d += blockDim.x) {
     float o = 0.f;
-    for (int s = 0; s < ns; ++s)
-      o = fmaf(expf(ml[(size_t)s * n_heads].x - M), part_o[(((size_t)b * max_splits + s) * n_heads + h) * d_c + d], o);
-    o_lat[((size_t)b * n_heads + h) * d_c + d] = o / den;
+    for (int s = 0; s < ns; ++s) o = fmaf(expf(ml[(size_t)s * n_heads].x - M), po[(size_t)s * o_stride + d], o);
+    o_lat[((size_t)b * n_heads + h) * d_c + d] = o * inv;
   }
 }
 
@@ -602,7 +647,9 @@ int corun_mla_attend(const float *q_lat, const float *q_rope, const void *cache,
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const int max_splits = (max_context + MLA_SPLIT - 1) / MLA_SPLIT;
   // the warp-level tensor path needs whole k16 steps and 64-dim passes; otherwise (or on request) plain FMAs
-  if (reinterpret_cast<uintptr_t>(cache) % 16) return CORUN_EINVAL;
+  if (reinterpret_cast<uintptr_t>(cache) % 16 || reinterpret_cast<uintptr_t>(q_lat) % 16 || reinterpret_cast<uintptr_t>(q_rope) % 16 ||
+      reinterpret_cast<uintptr_t>(o_lat) % 16 || reinterpret_cast<uintptr_t>(ws) % 16)
+    return CORUN_EINVAL;
   auto env_on = [](const char *name) { const char *v = getenv(name); return v && atoi(v) != 0; };
   // single fp16 operands exist on the pipelined tensor path only
   if (!operand_pairs && (d_rope % 16 != 0 || env_on("CORUN_MLA_FMA") || env_on("CORUN_MLA_UNPIPELINED"))) return CORUN_EINVAL;
@@ -619,7 +666,7 @@ int corun_mla_attend(const float *q_lat, const float *q_rope, const void *cache,
     float2 *part_ml = reinterpret_cast<float2 *>(ws + (size_t)B * max_chunks * n_heads * d_latent);
     kern<<<dim3(max_chunks, B), MLA_CTHREADS, smem, st>>>(q_lat, q_rope, (const __half *)cache, ctx, n_heads, d_latent, d_rope,
                                                         max_context, max_chunks, scale, part_o, part_ml);
-    mla_combine_kernel<<<dim3(n_heads, B), MLA_THREADS, 0, st>>>(part_o, part_ml, ctx, n_heads, d_latent, max_chunks, MLA_CHUNK,
+    mla_combine_kernel<<<dim3(n_heads, B), 128, 0, st>>>(part_o, part_ml, ctx, n_heads, d_latent, max_chunks, MLA_CHUNK,
                                                                 o_lat);
     ce = cudaGetLastError();
     if (ce != cudaSuccess) { corun::g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
@@ -637,7 +684,7 @@ int corun_mla_attend(const float *q_lat, const float *q_rope, const void *cache,
   else
     mla_split_kernel<<<dim3(max_splits, B), MLA_THREADS, smem, st>>>(q_lat, q_rope, (const __half *)cache, ctx, n_heads, d_latent,
                                                                     d_rope, max_context, max_splits, scale, part_o, part_ml);
-  mla_combine_kernel<<<dim3(n_heads, B), MLA_THREADS, 0, st>>>(part_o, part_ml, ctx, n_heads, d_latent, max_splits, MLA_SPLIT,
+  mla_combine_kernel<<<dim3(n_heads, B), 128, 0, st>>>(part_o, part_ml, ctx, n_heads, d_latent, max_splits, MLA_SPLIT,
                                                               o_lat);
   ce = cudaGetLastError();
   if (ce != cudaSuccess) { corun::g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
