@@ -159,6 +159,12 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], const void *p) {
   const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
 }
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t a) {   // a: shared-space byte address
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], uint32_t a) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
 __device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
@@ -348,7 +354,9 @@ __device__ __forceinline__ void split_half2(float2 v, uint32_t &hi, uint32_t &lo
   lo = *reinterpret_cast<const uint32_t *>(&l);
 }
 
-template <bool PAIRS>
+// DC, DR: the latent and rotary widths at compile time (strides and shared-memory offsets fold into the
+// instructions' immediates), or 0, 0 for widths taken from the arguments.
+template <bool PAIRS, int DC, int DR>
 __global__ void __launch_bounds__(MLA_CTHREADS, 1)
 mla_chunk_mma_kernel(const float *__restrict__ q_lat, const float *__restrict__ q_rope, const __half *__restrict__ cache,
                      const int *__restrict__ ctx, int n_heads, int d_c, int d_r, int max_context, int max_chunks, float scale,
@@ -359,34 +367,38 @@ mla_chunk_mma_kernel(const float *__restrict__ q_lat, const float *__restrict__ 
   if (t_begin >= n_ctx) return;
   const int n_chunk = min(MLA_CHUNK, n_ctx - t_begin);
   const int n_tiles = (n_chunk + MLA_TILE - 1) / MLA_TILE;
+  if (DC) { d_c = DC; d_r = DR; }
   const int DK = d_c + d_r, cp = DK + MLA_CP;
   extern __shared__ __align__(16) unsigned char smem[];
   __half *cs = reinterpret_cast<__half *>(smem);                     // [2][64][cp]
+  const uint32_t cs_s = (uint32_t)__cvta_generic_to_shared(cs);      // 32-bit shared-space addresses for ldmatrix / cp.async
   __half *ph = cs + (size_t)2 * MLA_TILE * cp;                       // [16][MLA_TP] weights hi, then the same for lo
   float *sc = reinterpret_cast<float *>(ph + (size_t)2 * MLA_NH * MLA_TP);   // [4 K groups][16][MLA_SP] partial scores
   float *run_m = sc + MLA_KG * MLA_NH * MLA_SP;                      // [16] running maxima
   float *run_l = run_m + MLA_NH;                                     // [16] running sums
   float *fac = run_l + MLA_NH;                                       // [16] rescale factors of the current tile
+  const uint32_t ph_s = (uint32_t)__cvta_generic_to_shared(ph);
   const int r0 = lane >> 2, cc = 2 * (lane & 3);
 
   auto load_tile = [&](int ti) {
     const int t0 = t_begin + ti * MLA_TILE;
     const int n = min(MLA_TILE, n_ctx - t0);
-    __half *dst = cs + (size_t)(ti & 1) * MLA_TILE * cp;
+    const uint32_t dst_s = cs_s + (uint32_t)((ti & 1) * MLA_TILE * cp * 2) + lane * 16;
     const int vecs = DK / 8;
-    const __half *src = cache + ((size_t)b * max_context + t0) * DK;
+    const __half *src = cache + ((size_t)b * max_context + t0) * DK + lane * 8;
     // warp w: tokens w, w + 16, ...; its lanes the 16-byte pieces of the row
 #pragma unroll
     for (int t = warp; t < MLA_TILE; t += MLA_CTHREADS / 32) {
-      __half *d = dst + (size_t)t * cp;
+      const uint32_t d = dst_s + (uint32_t)(t * cp * 2);
       if (t < n) {
         const __half *g = src + (size_t)t * DK;
-        for (int j = lane; j < vecs; j += 32) {
-          const uint32_t da = (uint32_t)__cvta_generic_to_shared(d + 8 * j);
-          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(da), "l"(g + 8 * j) : "memory");
-        }
+#pragma unroll 3
+        for (int j = lane; j < vecs; j += 32)
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d + (uint32_t)(j - lane) * 16), "l"(g + (j - lane) * 8) : "memory");
       } else {
-        for (int j = lane; j < vecs; j += 32) *reinterpret_cast<uint4 *>(d + 8 * j) = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll 3
+        for (int j = lane; j < vecs; j += 32)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(d + (uint32_t)(j - lane) * 16), "r"(0u) : "memory");
       }
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
@@ -446,7 +458,7 @@ mla_chunk_mma_kernel(const float *__restrict__ q_lat, const float *__restrict__ 
       asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
     __syncthreads();                                 // tile ti is in shared memory
-    const __half *ct = cs + (size_t)(ti & 1) * MLA_TILE * cp;
+    const uint32_t ct_s = cs_s + (uint32_t)((ti & 1) * MLA_TILE * cp * 2);
     const int n = min(MLA_TILE, n_chunk - ti * MLA_TILE);
     // ---- partial scores of K group kg for heads x tokens 16 tg .. 16 tg + 15 (two n8 tiles, hi and lo chains)
     {
@@ -456,12 +468,12 @@ mla_chunk_mma_kernel(const float *__restrict__ q_lat, const float *__restrict__ 
 #pragma unroll
         for (int e = 0; e < 4; ++e) { c_hi[j][e] = 0.f; c_lo[j][e] = 0.f; }
       // B (16 tokens x 16 dims as [token][dim]): matrices (tokens 0-7, dims 0-7), (0-7, 8-15), (8-15, 0-7), (8-15, 8-15)
-      const __half *bp = ct + (size_t)(16 * tg + (lane & 7) + ((lane >> 4) << 3)) * cp + ((lane >> 3) & 1) * 8 + my_first * 16;
+      const uint32_t bp = ct_s + 2u * (uint32_t)((16 * tg + (lane & 7) + ((lane >> 4) << 3)) * cp + ((lane >> 3) & 1) * 8 + my_first * 16);
 #pragma unroll
       for (int i = 0; i < MLA_KS; ++i) {
         if (i < my_steps) {
           uint32_t b0[4];
-          ldsm_x4(b0, bp + i * 16);
+          ldsm_x4(b0, bp + i * 32);
           mma16816(c_hi[0], qa_hi[i], b0[0], b0[1]);
           mma16816(c_hi[1], qa_hi[i], b0[2], b0[3]);
           if (PAIRS) {
@@ -516,20 +528,20 @@ mla_chunk_mma_kernel(const float *__restrict__ q_lat, const float *__restrict__ 
       const float f0 = fac[r0], f1 = fac[r0 + 8];
 #pragma unroll
       for (int j = 0; j < 4; ++j) { acc[j][0] *= f0; acc[j][1] *= f0; acc[j][2] *= f1; acc[j][3] *= f1; }
-      const __half *a_hi = ph + (size_t)(lane & 15) * MLA_TP + (lane >> 4) * 8;
-      const __half *a_lo = a_hi + (size_t)MLA_NH * MLA_TP;
+      const uint32_t a_hi = ph_s + 2u * (uint32_t)((lane & 15) * MLA_TP + (lane >> 4) * 8);
+      const uint32_t a_lo = a_hi + 2u * MLA_NH * MLA_TP;
       // B (16 tokens x 16 dims stored [token][dim], read transposed): matrices (tokens 0-7, dims 0-7), (8-15, 0-7),
       // (0-7, 8-15), (8-15, 8-15)
-      const __half *bp = ct + (size_t)((lane & 7) + ((lane >> 3) & 1) * 8) * cp + dbase + (lane >> 4) * 8;
+      const uint32_t bp = ct_s + 2u * (uint32_t)(((lane & 7) + ((lane >> 3) & 1) * 8) * cp + dbase + (lane >> 4) * 8);
 #pragma unroll
       for (int k0 = 0; k0 < MLA_TILE; k0 += 16) {
         uint32_t ah[4], al[4];
-        ldsm_x4(ah, a_hi + k0);
-        if (PAIRS) ldsm_x4(al, a_lo + k0);
+        ldsm_x4(ah, a_hi + 2 * k0);
+        if (PAIRS) ldsm_x4(al, a_lo + 2 * k0);
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
           uint32_t bb[4];
-          ldsm_x4_t(bb, bp + (size_t)k0 * cp + 16 * j);
+          ldsm_x4_t(bb, bp + 2u * (uint32_t)(k0 * cp + 16 * j));
           mma16816(acc[2 * j], ah, bb[0], bb[1]);
           mma16816(acc[2 * j + 1], ah, bb[2], bb[3]);
           if (PAIRS) {
@@ -660,7 +672,10 @@ int corun_mla_attend(const float *q_lat, const float *q_rope, const void *cache,
     // pipelined path: chunks of MLA_CHUNK tokens (the workspace, sized for 128-token splits, is large enough)
     const int max_chunks = (max_context + MLA_CHUNK - 1) / MLA_CHUNK;
     const size_t smem = mla_chunk_smem_bytes(d_latent, d_rope);
-    auto kern = operand_pairs ? mla_chunk_mma_kernel<true> : mla_chunk_mma_kernel<false>;
+    // the DeepSeek-V2 / V3 widths are compiled in; any other shape takes the kernel with run-time widths
+    const bool v2 = d_latent == 512 && d_rope == 64;
+    auto kern = v2 ? (operand_pairs ? mla_chunk_mma_kernel<true, 512, 64> : mla_chunk_mma_kernel<false, 512, 64>)
+                   : (operand_pairs ? mla_chunk_mma_kernel<true, 0, 0> : mla_chunk_mma_kernel<false, 0, 0>);
     cudaError_t ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (ce != cudaSuccess) { corun::g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
     float2 *part_ml = reinterpret_cast<float2 *>(ws + (size_t)B * max_chunks * n_heads * d_latent);
