@@ -64,3 +64,72 @@ def test_mla_single_operands_need_the_tensor_path():
     z = lambda *s: torch.zeros(s, device="cuda")
     with pytest.raises(Exception):                   # d_rope = 8: only the FMA kernel takes it, and only with pairs
         corun.mla_attend(z(1, 4, 64), z(1, 4, 8), z(1, 128, 72).half(), torch.ones(1, dtype=torch.int32, device="cuda"), 1.0, False)
+
+
+def _mla_case(nh, dc, dr, ctxs, T, seed):
+    rng = np.random.default_rng(seed)
+    B = len(ctxs)
+    q_lat = rng.standard_normal((B, nh, dc)).astype(np.float32)
+    q_rope = rng.standard_normal((B, nh, dr)).astype(np.float32)
+    cache = (rng.standard_normal((B, T, dc + dr)) * 0.5).astype(np.float16)
+    return q_lat, q_rope, cache
+
+
+def _mla_worst(out, q_lat, q_rope, cache, ctxs, dc):
+    nh = q_lat.shape[1]
+    eye = np.stack([np.eye(dc)] * nh)
+    worst = 0.0
+    for b, n in enumerate(ctxs):
+        C = cache[b, :n, :dc].astype(np.float64)
+        Rk = cache[b, :n, dc:].astype(np.float64)
+        ref = ml.attend_absorbed(q_lat[b], q_rope[b], C, Rk, eye, eye)
+        worst = max(worst, float(np.abs(out[b] - ref).max()))
+    return worst
+
+
+@pytest.mark.parametrize("path", ["", "CORUN_MLA_UNPIPELINED", "CORUN_MLA_FMA"])
+def test_mla_every_kernel_and_more_pieces_than_the_combine_fast_path(path):
+    """The three kernels (selected by environment variable) on contexts around the chunk boundary and on one with
+    more pieces than the combine kernel keeps in registers (18 chunks of 512, 71 splits of 128)."""
+    import os
+
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2608_14376_b200 import corun
+
+    nh, dc, dr = 4, 64, 16
+    ctxs = [9000, 512, 513, 1024, 63]
+    q_lat, q_rope, cache = _mla_case(nh, dc, dr, ctxs, 9216, seed=7)
+    scale = 1.0 / math.sqrt(dc + dr)
+    dev = lambda a: torch.tensor(a).cuda().contiguous()
+    if path:
+        os.environ[path] = "1"
+    try:
+        out = corun.mla_attend(dev(q_lat), dev(q_rope), dev(cache), dev(np.array(ctxs, np.int32)), scale)
+        torch.cuda.synchronize()
+        again = corun.mla_attend(dev(q_lat), dev(q_rope), dev(cache), dev(np.array(ctxs, np.int32)), scale)
+        torch.cuda.synchronize()
+    finally:
+        if path:
+            os.environ.pop(path, None)
+    assert out.cpu().numpy().tobytes() == again.cpu().numpy().tobytes()
+    assert _mla_worst(out.cpu().numpy(), q_lat, q_rope, cache, ctxs, dc) <= 2e-5
+
+
+def test_mla_v2_widths_match_the_runtime_width_kernel_on_the_oracle():
+    """d_c = 512, d_r = 64 takes the kernel with the widths compiled in: long contexts, several chunks."""
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2608_14376_b200 import corun
+
+    nh, dc, dr = 16, 512, 64
+    ctxs = [2049, 1536, 511]
+    q_lat, q_rope, cache = _mla_case(nh, dc, dr, ctxs, 2176, seed=11)
+    scale = 1.0 / math.sqrt(dc + dr)                 # the oracle's scale for identity up-projections (d_nope = d_c)
+    dev = lambda a: torch.tensor(a).cuda().contiguous()
+    for pairs, tol in ((True, 2e-5), (False, 4e-3)):
+        out = corun.mla_attend(dev(q_lat), dev(q_rope), dev(cache), dev(np.array(ctxs, np.int32)), scale, pairs)
+        torch.cuda.synchronize()
+        assert _mla_worst(out.cpu().numpy(), q_lat, q_rope, cache, ctxs, dc) <= tol
