@@ -34,7 +34,8 @@ int64_t corun_mla_workspace_floats(int32_t B, int32_t n_heads, int32_t d_latent,
 /*
  *   q_lat   fp32 [B, n_heads, d_latent]      q_rope  fp32 [B, n_heads, d_rope]
  *   cache   fp16 [B, max_context, d_latent + d_rope] (row b uses its first ctx[b] tokens)
- *   ctx     int32 [B]: cached tokens per row, 0 = padding row (its output is left alone)
+ *   ctx     int32 [B]: cached tokens per row, 0 = padding row (its output is left alone); a value above
+ *           max_context is treated as max_context (nothing past a row's cache is read)
  *   o_lat   fp32 [B, n_heads, d_latent]
  *   ws      corun_mla_workspace_floats(...) floats
  * n_heads 1..16 (a multiple of 4), d_latent a multiple of 64 up to 512, d_rope a multiple of 8 up to 64

@@ -24,7 +24,7 @@ mla_split_kernel(const float *__restrict__ q_lat, const float *__restrict__ q_ro
                  const int *__restrict__ ctx, int n_heads, int d_c, int d_r, int max_context, int max_splits, float scale,
                  float *__restrict__ part_o, float2 *__restrict__ part_ml) {
   const int s = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
-  const int n_ctx = ctx[b];
+  const int n_ctx = min(ctx[b], max_context);   // a context beyond the cache is cut, never read
   const int t0 = s * MLA_SPLIT;
   if (t0 >= n_ctx) return;                           // the same decision in every thread
   const int n = min(MLA_SPLIT, n_ctx - t0);
@@ -179,7 +179,7 @@ mla_split_mma_kernel(const float *__restrict__ q_lat, const float *__restrict__ 
                      const int *__restrict__ ctx, int n_heads, int d_c, int d_r, int max_context, int max_splits, float scale,
                      float *__restrict__ part_o, float2 *__restrict__ part_ml) {
   const int s = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n_ctx = ctx[b];
+  const int n_ctx = min(ctx[b], max_context);   // a context beyond the cache is cut, never read
   const int t0 = s * MLA_SPLIT;
   if (t0 >= n_ctx) return;
   const int n = min(MLA_SPLIT, n_ctx - t0);
@@ -362,7 +362,7 @@ mla_chunk_mma_kernel(const float *__restrict__ q_lat, const float *__restrict__ 
                      const int *__restrict__ ctx, int n_heads, int d_c, int d_r, int max_context, int max_chunks, float scale,
                      float *__restrict__ part_o, float2 *__restrict__ part_ml) {
   const int ch = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n_ctx = ctx[b];
+  const int n_ctx = min(ctx[b], max_context);   // a context beyond the cache is cut, never read
   const int t_begin = ch * MLA_CHUNK;
   if (t_begin >= n_ctx) return;
   const int n_chunk = min(MLA_CHUNK, n_ctx - t_begin);
@@ -587,7 +587,7 @@ mla_combine_kernel(const float *__restrict__ part_o, const float2 *__restrict__ 
   const int h = blockIdx.x, b = blockIdx.y;
   const int n_ctx = ctx[b];
   if (n_ctx <= 0) return;
-  const int ns = (n_ctx + split_len - 1) / split_len;
+  const int ns = min((n_ctx + split_len - 1) / split_len, max_splits);   // as the piece kernels cut it
   const float2 *ml = part_ml + (size_t)b * max_splits * n_heads + h;
   const float *po = part_o + ((size_t)b * max_splits * n_heads + h) * d_c;
   const size_t o_stride = (size_t)n_heads * d_c;     // floats between a head's consecutive pieces

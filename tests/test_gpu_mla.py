@@ -133,3 +133,19 @@ def test_mla_v2_widths_match_the_runtime_width_kernel_on_the_oracle():
         out = corun.mla_attend(dev(q_lat), dev(q_rope), dev(cache), dev(np.array(ctxs, np.int32)), scale, pairs)
         torch.cuda.synchronize()
         assert _mla_worst(out.cpu().numpy(), q_lat, q_rope, cache, ctxs, dc) <= tol
+
+
+def test_mla_context_beyond_the_cache_is_cut():
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2608_14376_b200 import corun
+
+    nh, dc, dr, T = 8, 128, 32, 640
+    q_lat, q_rope, cache = _mla_case(nh, dc, dr, [T, T], T, seed=3)
+    scale = 1.0 / math.sqrt(dc + dr)
+    dev = lambda a: torch.tensor(a).cuda().contiguous()
+    full = corun.mla_attend(dev(q_lat), dev(q_rope), dev(cache), dev(np.array([T, T], np.int32)), scale)
+    over = corun.mla_attend(dev(q_lat), dev(q_rope), dev(cache), dev(np.array([T + 100, 1 << 30], np.int32)), scale)
+    torch.cuda.synchronize()
+    assert over.cpu().numpy().tobytes() == full.cpu().numpy().tobytes()
