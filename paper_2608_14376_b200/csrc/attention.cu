@@ -20,14 +20,14 @@
 //        weights written as fp16 hi/lo rows of a [16 x 128 tokens] operand tile,
 //     4. O^T[hd dims x 16] = V^T[hd x 128 tokens] * P^T  (one MMA per page), TMEM lane = dim,
 //     5. adds the hi and lo columns and writes the split's partial (max, sum, O) to global memory;
-//   4 combiner warps: when a group leaves a (row, kv head) it reports how many of that pair's splits it
-//   wrote; the combiners add this to the pair's device-wide counter and, when the count is complete,
-//   combine the pair's splits (in ascending split order, so it does not matter who does it).
+// A second kernel, one warp per (row, query head), combines the splits' partials in ascending split order
+// (attn_combine_kernel): as a kernel of its own the combines all run at once, where combiner warps inside the
+// first kernel left a serial tail of several microseconds behind each CTA's last item.
 // The cached K / V are fp16 exactly, accumulation is fp32.
 //
 // Invariance: the split size is fixed, the split count is a function of the row's own context
 // length, every reduction inside an item has one fixed order, and the splits are combined in
-// ascending order by one owner.  The work list only decides which CTA computes an item.
+// ascending order by one warp.  The work list only decides which CTA computes an item.
 #include <cuda_fp16.h>
 #include <math_constants.h>
 
@@ -42,8 +42,7 @@ namespace {
 constexpr int ATT_NBUF = 3;                        // item buffers in the ring
 constexpr int ATT_GROUPS = 2;                      // consumer groups of 4 warps
 constexpr int ATT_SLOTS = 6;                       // barrier slots: a multiple of both
-constexpr int ATT_THREADS = 64 + ATT_GROUPS * 128 + 128; // two producer warps + consumers + combiners
-constexpr int ATT_QDEPTH = 8;                      // reports a group may have outstanding
+constexpr int ATT_THREADS = 64 + ATT_GROUPS * 128; // two producer warps + consumers
 constexpr int ATT_PAGES = ATT_SPLIT / KV_BLOCK;    // 8 pages per split
 constexpr int KBOX_BYTES = KV_BLOCK * 128;         // one [16 tokens x 64 dims] fp16 key box
 constexpr int OPND_BYTES = 16 * 128;               // one [16 rows x 64 cols] fp16 half of a q / p operand tile
@@ -179,8 +178,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 1)
 attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                   const float *__restrict__ q, Rows rows, int nq, KvLayout kv, int max_splits,
                   const int *__restrict__ work, const int *__restrict__ n_work, float *__restrict__ part_acc,
-                  float *__restrict__ part_ml, int *__restrict__ done_count, int *__restrict__ pool_count,
-                  __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo, int *status,
+                  float *__restrict__ part_ml, int *__restrict__ pool_count, int *status,
                   unsigned long long *trace) {
   using L = AttLayout<HD>;
   // optional timeline (debug): per CTA and item (first 64): [key load issued, keys landed, group starts, released, scores done, weights written, values landed, output done]
@@ -204,10 +202,6 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   __shared__ int abort_flag;
   __shared__ int stop_s[ATT_GROUPS];             // group-uniform copy of abort_flag, refreshed once per item
   __shared__ float red_s[ATT_GROUPS][4][8];      // cross-warp softmax reductions
-  // reports of the consumer groups to the combiners: (row << 8 | kv head, splits written), -1 = group is done
-  __shared__ int rep_key[ATT_GROUPS][ATT_QDEPTH], rep_cnt[ATT_GROUPS][ATT_QDEPTH];
-  __shared__ unsigned rep_tail[ATT_GROUPS], rep_head[ATT_GROUPS];
-  __shared__ int cmb_s[2], cmb_list[8][3];       // what the combiners do next: how many pairs, leave?; (row, kv head, split count)
   // pairs of pool items drawn by the key producer for the whole CTA: ring of 4, one barrier each
   __shared__ __align__(8) uint64_t pool_bar[4];
   __shared__ int pool_pair[4];
@@ -216,7 +210,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     abort_flag = 0;
-    for (int g = 0; g < ATT_GROUPS; ++g) { stop_s[g] = 0; rep_tail[g] = 0u; rep_head[g] = 0u; mbar_init(smem_u32(&mma_bar[g]), 1); }
+    for (int g = 0; g < ATT_GROUPS; ++g) { stop_s[g] = 0; mbar_init(smem_u32(&mma_bar[g]), 1); }
     for (int s = 0; s < ATT_SLOTS; ++s) { mbar_init(smem_u32(&kfull_bar[s]), 1); mbar_init(smem_u32(&vfull_bar[s]), 1); }
     for (int b = 0; b < ATT_NBUF; ++b) { mbar_init(smem_u32(&kempty_bar[b]), 1); mbar_init(smem_u32(&vempty_bar[b]), 1); }
     for (int b = 0; b < 4; ++b) mbar_init(smem_u32(&pool_bar[b]), 1);
@@ -307,16 +301,18 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       if (item == -1) break;
       if (item == -2) continue;
       const int buf = k % ATT_NBUF, slot = k % ATT_SLOTS;
-      if (k >= ATT_NBUF) {                               // the buffer's previous item must have been released
-        bool ok = mbar_wait(smem_u32(&empty[buf]), (uint32_t)(k / ATT_NBUF - 1) & 1u, &abort_flag);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) { failed = true; break; }
-      }
+      // where the item's pages are: looked up before the wait for the buffer (three dependent loads)
       const int wi = work[item];
       const int r = wi >> 16, g = (wi >> 8) & 255, split = wi & 255;
       const int ctx = rows.pos[r] + 1;
       const int t0 = split * ATT_SPLIT;
       const int n_pages = min(ATT_PAGES, (ctx - t0 + KV_BLOCK - 1) / KV_BLOCK);
+      const int page = lane < n_pages ? kv.block_table[(size_t)rows.slot[r] * kv.max_blocks + t0 / KV_BLOCK + lane] : 0;
+      if (k >= ATT_NBUF) {                               // the buffer's previous item must have been released
+        bool ok = mbar_wait(smem_u32(&empty[buf]), (uint32_t)(k / ATT_NBUF - 1) & 1u, &abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { failed = true; break; }
+      }
       const uint32_t fb = smem_u32(&full[slot]);
       if (lane == 0) {
         if (!is_v) ATRACE(k, 0);
@@ -324,7 +320,6 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       }
       __syncwarp();
       if (lane < n_pages) {
-        const int page = kv.block_table[(size_t)rows.slot[r] * kv.max_blocks + t0 / KV_BLOCK + lane];
         // this layer's pages as rows of hd halfs: the key tile of (page, head) starts at row
         //   page * 2 * n_kv * 16 + head * 16;
         // as rows of 16 halfs: the transposed value tile starts at row page * 2 * n_kv * hd + (n_kv + head) * hd
@@ -340,25 +335,9 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         }
       }
     }
-  } else if (warp < 2 + 4 * ATT_GROUPS) {
+  } else {
     // ---------------- consumers ----------------
     const int gi = (warp - 2) >> 2, gtid = (tid - 64) & 127;
-    // Report to the combiners (one thread, after a group barrier that follows the group's stores).
-    auto report = [&](int key, int cnt) {
-      const unsigned t = rep_tail[gi];               // written by this thread only
-      if (t - *(volatile unsigned *)&rep_head[gi] >= (unsigned)ATT_QDEPTH) {
-        const uint64_t t0 = globaltimer_ns();
-        while (t - *(volatile unsigned *)&rep_head[gi] >= (unsigned)ATT_QDEPTH) {
-          __nanosleep(64);
-          if (abort_flag || globaltimer_ns() - t0 > 2000000000ull) { abort_flag = 1; return; }
-        }
-      }
-      rep_key[gi][t % ATT_QDEPTH] = key;
-      rep_cnt[gi][t % ATT_QDEPTH] = cnt;
-      __threadfence_block();
-      *(volatile unsigned *)&rep_tail[gi] = t + 1u;
-    };
-    int run_cnt = 0;
     const int quad = warp & 3;                     // the TMEM lane quarter this warp may read
     const int tl = quad * 32 + lane;               // TMEM lane of this thread: token (scores) / dim (values)
     const float sscale = (HD == 128 ? 0.08838834764831845f : 0.125f) * 1.4426950408889634f;   // log2(e)/sqrt(hd)
@@ -417,11 +396,9 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         }
         q_built = q_loaded = wi >> 8;
       }
-      bool run_ends = true;                          // is this the group's last item of its (row, kv head)?
       if (k + ATT_GROUPS < n_fixed) {   // fetch the next item's query values now if they differ
         const int nwi = work[item + 1];
         if ((nwi >> 8) != q_built) { load_q(nwi >> 16, (nwi >> 8) & 255); q_loaded = nwi >> 8; }
-        run_ends = (nwi >> 8) != (wi >> 8);
       }
       fence_proxy_async();                           // the MMA reads this tile through the async proxy
       if (gtid == 0) stop_s[gi] = abort_flag;
@@ -543,89 +520,8 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       tc_fence_before();
       asm volatile("bar.sync %0, 128;" ::"r"(1 + gi) : "memory");   // the group's TMEM and operand tiles are free
       if (gtid == 0) ATRACE(k, 3);
-      ++run_cnt;
-      if (run_ends) {
-        // a group that wrote every split of the pair itself says so: nothing has to be counted then
-        if (gtid == 0) report(wi >> 8, run_cnt | ((run_cnt * ATT_SPLIT >= ctx) ? 0x10000 : 0));
-        run_cnt = 0;
-      }
     }
-    if (gtid == 0) { ATRACE(63, gi); report(-1, 0); }   // always: the combiners wait for every group
-  } else {
-    // ---------------- combiners ----------------
-    const int ctid = tid - 64 - ATT_GROUPS * 128, cw = ctid >> 5;
-    unsigned head[ATT_GROUPS];
-    int groups_done = 0;
-#pragma unroll
-    for (int g = 0; g < ATT_GROUPS; ++g) head[g] = 0u;
-    for (;;) {
-      if (ctid == 0) {
-        // take every hand-in that is waiting (up to 8), make the groups' partial results visible
-        // device-wide with one fence, then count them all
-        int key[8], cnt[8], n = 0;
-        const uint64_t t0 = globaltimer_ns();
-        bool gave_up = false;
-        for (uint32_t spin = 0;; ++spin) {
-#pragma unroll
-          for (int g = 0; g < ATT_GROUPS; ++g) {
-            const unsigned tl_ = *(volatile unsigned *)&rep_tail[g];
-            if (tl_ != head[g]) __threadfence_block();
-            while (head[g] != tl_ && n < 8) {
-              const int k_ = rep_key[g][head[g] % ATT_QDEPTH], c_ = rep_cnt[g][head[g] % ATT_QDEPTH];
-              head[g] += 1u;
-              if (k_ < 0) ++groups_done;
-              else {
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                  if (i == n) { key[i] = k_; cnt[i] = c_; }
-                ++n;
-              }
-            }
-            *(volatile unsigned *)&rep_head[g] = head[g];
-          }
-          if (n > 0 || groups_done == ATT_GROUPS) break;
-          __nanosleep(100);
-          if ((spin & 255u) == 255u && (abort_flag || globaltimer_ns() - t0 > 4000000000ull)) { abort_flag = 1; gave_up = true; break; }
-        }
-        int n_out = 0;
-        if (n > 0) {
-          int ns[8], seen[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i)
-            if (i < n) ns[i] = (rows.pos[key[i] >> 8] + 1 + ATT_SPLIT - 1) / ATT_SPLIT;
-          __threadfence();                           // the partial results are visible device-wide ...
-#pragma unroll
-          for (int i = 0; i < 8; ++i)
-            if (i < n)   // ... before they are counted
-              seen[i] = (cnt[i] & 0x10000) ? ns[i]
-                                           : atomicAdd(done_count + (key[i] >> 8) * kv.n_kv + (key[i] & 255), cnt[i]) + cnt[i];
-#pragma unroll
-          for (int i = 0; i < 8; ++i)
-            if (i < n && seen[i] == ns[i]) {
-              if (!(cnt[i] & 0x10000))
-                done_count[(key[i] >> 8) * kv.n_kv + (key[i] & 255)] = 0;   // complete: nobody else touches it until the next launch
-              cmb_list[n_out][0] = key[i] >> 8; cmb_list[n_out][1] = key[i] & 255; cmb_list[n_out][2] = ns[i];
-              ++n_out;
-            }
-        }
-        cmb_s[0] = n_out;
-        cmb_s[1] = (gave_up || (groups_done == ATT_GROUPS && n == 0)) ? 1 : 0;   // leave once nothing is left
-      }
-      asm volatile("bar.sync %0, 128;" ::"r"(1 + ATT_GROUPS) : "memory");
-      const int n_out = cmb_s[0], leave = cmb_s[1];
-      if (n_out > 0 && ctid == 0 && trace) atomicAdd(&trace[((size_t)blockIdx.x * 64 + 63) * 8 + 3], (unsigned long long)n_out);
-      if (n_out > 0) {
-        __threadfence();                             // the other contributors' partial results are visible here
-        for (int i = 0; i < n_out; ++i) {
-          const int r_ = cmb_list[i][0], g_ = cmb_list[i][1], ns = cmb_list[i][2];
-          for (int h = cw; h < GROUP; h += 4)
-            attn_combine_pair<HD>(r_, g_ * GROUP + h, ns, nq, max_splits, part_acc, part_ml, out_hi, out_lo, lane);
-        }
-      }
-      asm volatile("bar.sync %0, 128;" ::"r"(1 + ATT_GROUPS) : "memory");
-      if (leave) break;
-    }
-    if (ctid == 0) ATRACE(63, 2);
+    if (gtid == 0) ATRACE(63, gi);
   }
   if (failed || abort_flag) {
     if (lane == 0) atomicCAS(status, 0, DEV_TIMEOUT_EPILOGUE);
@@ -680,6 +576,23 @@ __global__ void __launch_bounds__(256) attn_worklist_kernel(Rows rows, int n_kv,
   }
 }
 
+// One warp per (row, query head): adds the row's split partials in ascending split order -> bf16 hi/lo.
+template <int HD>
+__global__ void __launch_bounds__(128) attn_combine_kernel(Rows rows, int nq, int max_splits,
+                                                           const float *__restrict__ part_acc,
+                                                           const float *__restrict__ part_ml,
+                                                           __nv_bfloat16 *__restrict__ out_hi,
+                                                           __nv_bfloat16 *__restrict__ out_lo) {
+  griddep_launch_dependents();
+  griddep_wait();
+  const int w = (int)blockIdx.x * 4 + ((int)threadIdx.x >> 5);
+  if (w >= rows.R * nq) return;
+  const int r = w / nq, j = w - r * nq;
+  if (!rows.active[r]) return;                     // padding rows keep what they held
+  const int ns = (rows.pos[r] + 1 + ATT_SPLIT - 1) / ATT_SPLIT;
+  attn_combine_pair<HD>(r, j, ns, nq, max_splits, part_acc, part_ml, out_hi, out_lo, (int)threadIdx.x & 31);
+}
+
 }  // namespace
 
 namespace {
@@ -698,19 +611,18 @@ cudaError_t prepare_one() {
 template <int HD>
 cudaError_t launch_attn_split(int group, int grid, cudaStream_t st, const CUtensorMap &tmK, const CUtensorMap &tmV,
                          const float *q, const Rows &rows, int nq, const KvLayout &kv, int max_splits, const int *work,
-                         const int *n_work, float *part_acc, float *part_ml, int *done_count, int *pool_count,
-                         __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int whole_pairs, int *d_status,
-                         unsigned long long *trace) {
+                         const int *n_work, float *part_acc, float *part_ml, int *pool_count, int whole_pairs,
+                         int *d_status, unsigned long long *trace) {
 #define CORUN_ATT_CASE(G)                                                                                          \
   case G:                                                                                                          \
     if (whole_pairs)                                                                                               \
       return launch_k(attn_split_kernel<HD, G, true, false>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
-                      rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, d_status, trace); \
+                      rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, pool_count, d_status, trace); \
     if (trace)                                                                                                     \
       return launch_k(attn_split_kernel<HD, G, false, true>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
-                      rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, d_status, trace); \
+                      rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, pool_count, d_status, trace); \
     return launch_k(attn_split_kernel<HD, G, false, false>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
-                    rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, done_count, pool_count, out_hi, out_lo, d_status, trace);
+                    rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, pool_count, d_status, trace);
   switch (group) {
     CORUN_ATT_CASE(1)
     CORUN_ATT_CASE(2)
@@ -744,7 +656,7 @@ cudaError_t launch_attn_worklist(const Rows &rows, int n_kv, int *work, int *n_w
 
 cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, const float *q, const Rows &rows, int nq,
                              const KvLayout &kv, int layer, int max_splits, const int *work, const int *n_work,
-                             int grid_ctas, float *part_acc, float *part_ml, int *done_count, int *pool_count,
+                             int grid_ctas, float *part_acc, float *part_ml, int *pool_count,
                              __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int reuse, int *d_status, cudaStream_t st,
                              unsigned long long *trace) {
   (void)layer;   // the tensor maps are the layer's
@@ -755,13 +667,22 @@ cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, con
   const int whole_pairs = reuse == 2;   // the ablation: the item list carries the pair table
   const long long most = (long long)rows.R * max_splits * kv.n_kv;
   const int grid = (int)(most < grid_ctas ? most : grid_ctas);
-  if (kv.hd == 128)
-    return launch_attn_split<128>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml,
-                                  done_count, pool_count, out_hi, out_lo, whole_pairs, d_status, trace);
-  if (kv.hd == 64)
-    return launch_attn_split<64>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml,
-                                 done_count, pool_count, out_hi, out_lo, whole_pairs, d_status, trace);
-  return cudaErrorInvalidValue;
+  const int cgrid = (rows.R * nq + 3) / 4;
+  cudaError_t ce = cudaErrorInvalidValue;
+  if (kv.hd == 128) {
+    ce = launch_attn_split<128>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml,
+                                pool_count, whole_pairs, d_status, trace);
+    if (ce == cudaSuccess)
+      ce = launch_k(attn_combine_kernel<128>, dim3(cgrid), dim3(128), 0, st, true, rows, nq, max_splits, part_acc, part_ml,
+                    out_hi, out_lo);
+  } else if (kv.hd == 64) {
+    ce = launch_attn_split<64>(group, grid, st, tmK, tmV, q, rows, nq, kv, max_splits, work, n_work, part_acc, part_ml,
+                               pool_count, whole_pairs, d_status, trace);
+    if (ce == cudaSuccess)
+      ce = launch_k(attn_combine_kernel<64>, dim3(cgrid), dim3(128), 0, st, true, rows, nq, max_splits, part_acc, part_ml,
+                    out_hi, out_lo);
+  }
+  return ce;
 }
 
 }  // namespace corun

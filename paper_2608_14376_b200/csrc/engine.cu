@@ -43,7 +43,7 @@ struct Program {
   float *qkv_out = nullptr, *o_out = nullptr, *gu_out = nullptr, *down_out = nullptr, *logits = nullptr, *ws = nullptr;
   bf16 *xn_hi = nullptr, *xn_lo = nullptr, *ao_hi = nullptr, *ao_lo = nullptr, *ff_hi = nullptr, *ff_lo = nullptr;
   int *row_token = nullptr, *row_pos = nullptr, *row_active = nullptr, *row_slot = nullptr, *do_sample = nullptr;
-  int *sampled = nullptr, *att_work = nullptr, *att_n_work = nullptr, *att_done = nullptr, *att_pool = nullptr;
+  int *sampled = nullptr, *att_work = nullptr, *att_n_work = nullptr, *att_pool = nullptr;
   GemmPlan p_qkv, p_o, p_gu, p_down, p_lm;
   // Mixture-of-Experts feed-forward layers: p_gu / p_down are then the GEMMs over all experts' gate / up rows
   // and over the concatenated hidden activations; p_r is the router GEMM (its rows padded to one tile)
@@ -74,6 +74,7 @@ struct corun_engine {
   const bf16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
   std::vector<const bf16 *> attn_norm, mlp_norm;
   std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_down;
+  std::vector<CUtensorMap> tm_gu_half;     // dense gate / up matrices with the box of the GEMM with SwiGLU in its epilogue
   std::vector<CUtensorMap> tm_k, tm_v;   // per layer: key view and transposed-value view of the pages
   // Mixture-of-Experts feed-forward layers (E = 0: dense).  sh.ffn is then (E + S) * F.
   int moe_E = 0, moe_K = 0, moe_F = 0, moe_S = 0, moe_renorm = 0;
@@ -133,7 +134,10 @@ int dmalloc(std::vector<void *> &keep, T **p, size_t n, bool zero = true) {
 
 int pad16(int x) { return (x + 15) / 16 * 16; }
 
-int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, bool grouped = false) {
+// fuse_swiglu: the gate / up GEMM writes silu(gate) * up itself (dense feed-forward, up to 128 padded rows: the
+// decode program while it is bound by the weight stream; whole tiles on fewer CTAs would cost a prefill chunk,
+// which is bound by the tensor pipe, a third of its gate / up rate).
+int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, bool grouped = false, bool fuse_swiglu = false) {
   const corun_shape &s = e->sh;
   const int H = s.hidden, QD = s.n_q_heads * s.head_dim, KD = s.n_kv_heads * s.head_dim, F = s.ffn, V = s.vocab;
   P.R = R;
@@ -157,7 +161,6 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
     RC(dmalloc(A, &P.part_ml, (size_t)R * s.n_q_heads * e->max_splits * 2));
     RC(dmalloc(A, &P.att_work, (size_t)R * e->max_splits * e->sh.n_kv_heads));
     RC(dmalloc(A, &P.att_n_work, 2 + 2 * (size_t)R * e->sh.n_kv_heads));
-    RC(dmalloc(A, &P.att_done, (size_t)R * e->sh.n_kv_heads));
     RC(dmalloc(A, &P.att_pool, (size_t)s.n_layers));
     RC(dmalloc(A, &P.qkv_out, (size_t)R * (QD + 2 * KD)));
     RC(dmalloc(A, &P.o_out, (size_t)R * H));
@@ -170,7 +173,10 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
     // the plans carry layer 0's weights; the per-layer tensor maps override them at launch
     RC(gemm_plan_create(&P.p_qkv, e->w0_qkv, QD + 2 * KD, H, P.xn_hi, P.xn_lo, R, P.BN, P.qkv_out, P.ws, e->num_sms));
     RC(gemm_plan_create(&P.p_o, e->w0_o, H, QD, P.ao_hi, P.ao_lo, R, P.BN, P.o_out, P.ws, e->num_sms));
-    RC(gemm_plan_create(&P.p_gu, e->w0_gu, 2 * F, H, P.xn_hi, P.xn_lo, R, P.BN, P.gu_out, P.ws, e->num_sms));
+    if (fuse_swiglu && !e->moe_E && P.BN <= 128)
+      RC(gemm_plan_create_swiglu(&P.p_gu, e->w0_gu, F, H, P.xn_hi, P.xn_lo, R, P.BN, P.ff_hi, P.ff_lo, e->num_sms));
+    else
+      RC(gemm_plan_create(&P.p_gu, e->w0_gu, 2 * F, H, P.xn_hi, P.xn_lo, R, P.BN, P.gu_out, P.ws, e->num_sms));
     RC(gemm_plan_create(&P.p_down, e->w0_down, H, F, P.ff_hi, P.ff_lo, R, P.BN, P.down_out, P.ws, e->num_sms));
     if (e->moe_E) {
       const int NB = e->moe_E + e->moe_S;
@@ -271,7 +277,7 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
     STAGE(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, tr(4 * l + 0), true));
     STAGE(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st));
     STAGE(launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work, P.att_n_work,
-                           e->num_sms, P.part_acc, P.part_ml, P.att_done, P.att_pool + l, P.ao_hi, P.ao_lo, &P == &e->dec ? (e->whole_pairs ? 2 : 0) : 1,
+                           e->num_sms, P.part_acc, P.part_ml, P.att_pool + l, P.ao_hi, P.ao_lo, &P == &e->dec ? (e->whole_pairs ? 2 : 0) : 1,
                            e->d_status, e->st));
     STAGE(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st, tr(4 * l + 1), true));
     GemmOut o = P.p_o.out();
@@ -288,7 +294,7 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
       STAGE(launch_moe_swiglu_grouped(P.gug_out, P.moe_w, NB, e->moe_F, P.grp, P.hg_hi, P.hg_lo, e->st));
       STAGE(gemm_launch(P.p_dng, &e->tm_down[l], e->d_status, e->st, nullptr, true));
       STAGE(launch_moe_combine(P.yg_out, P.row_active, P.R, NB, s.hidden, P.grp, P.down_out, e->st));
-      n += 14;
+      n += 14 + (&P == &e->dec ? 1 : 0);
       continue;
     } else if (e->moe_E) {
       // router -> top-k weights -> all experts' gate / up (rows that did not select a tile's expert are not
@@ -299,11 +305,16 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
       STAGE(launch_moe_swiglu(P.p_gu.out(), P.moe_w, P.R, e->moe_F, e->moe_E + e->moe_S, P.ff_hi, P.ff_lo, e->st));
       n += 2;
     } else {
-      STAGE(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st, tr(4 * l + 2), true));
-      STAGE(launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st));
+      if (P.p_gu.sw_hi) {                             // SwiGLU in the GEMM's epilogue
+        STAGE(gemm_launch(P.p_gu, &e->tm_gu_half[l], e->d_status, e->st, tr(4 * l + 2), true));
+        n -= 1;
+      } else {
+        STAGE(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st, tr(4 * l + 2), true));
+        STAGE(launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st));
+      }
     }
     STAGE(gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st, tr(4 * l + 3), true));
-    n += 9;
+    n += 9 + (&P == &e->dec ? 1 : 0);   // decode attention is two kernels (splits, combine)
   }
 #undef STAGE
   if (launches) *launches += n;
@@ -490,6 +501,7 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
   e->tm_o.resize(s.n_layers);
   e->tm_gu.resize(s.n_layers);
   e->tm_down.resize(s.n_layers);
+  if (!moe) e->tm_gu_half.resize(s.n_layers);
   for (int l = 0; l < s.n_layers; ++l) {
     e->attn_norm.push_back((const bf16 *)w->attn_norm[l]);
     e->mlp_norm.push_back((const bf16 *)w->mlp_norm[l]);
@@ -498,6 +510,7 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
     if ((rc = gemm_encode_map(&e->tm_o[l], w->wo[l], H, QD, GEMM_TILE_N))) return fail(rc);
     if ((rc = gemm_encode_map(&e->tm_gu[l], moe ? moe->gate_up[l] : w->wgate_up[l], 2 * F, H, GEMM_TILE_N))) return fail(rc);
     if ((rc = gemm_encode_map(&e->tm_down[l], moe ? moe->down[l] : w->wdown[l], H, F, GEMM_TILE_N))) return fail(rc);
+    if (!moe && (rc = gemm_encode_map(&e->tm_gu_half[l], w->wgate_up[l], 2 * F, H, gemm_swiglu_half(F, e->num_sms)))) return fail(rc);
   }
   if (moe) {
     int rc;
@@ -571,7 +584,7 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
   if (const char *ts = getenv("CORUN_TRACE_STEP")) {
     if (atoi(ts) != 0 && (rc = dmalloc(A, &e->step_trace, (size_t)4 * s.n_layers * e->num_sms * 8))) return fail(rc);
   }
-  if ((rc = program_create(e, e->dec, B, true, true))) return fail(rc);
+  if ((rc = program_create(e, e->dec, B, true, true, false, true))) return fail(rc);
   if ((rc = program_create(e, e->pre, e->chunk, true, false, e->moe_E > 0 && !getenv("CORUN_MOE_PREFILL_DENSE")))) return fail(rc);
   if ((rc = program_create(e, e->lm1, 1, false, true))) return fail(rc);
 
@@ -985,7 +998,7 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
         // launched as in the step's graph: with programmatic stream serialization
         case 0: ce = gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, nullptr, true); break;
         case 1: ce = gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st, nullptr, true); break;
-        case 2: ce = gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st, nullptr, true); break;
+        case 2: ce = gemm_launch(P.p_gu, P.p_gu.sw_hi ? &e->tm_gu_half[l] : &e->tm_gu[l], e->d_status, e->st, nullptr, true); break;
         case 3: ce = gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st, nullptr, true); break;
         case 4: ce = gemm_launch(P.p_lm, nullptr, e->d_status, e->st, nullptr, true);
                 if (ce == cudaSuccess) ce = gemm_fixup_launch(P.p_lm, e->st);
@@ -993,13 +1006,14 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
         case 5: ce = cudaMemsetAsync(P.att_pool + l, 0, sizeof(int), e->st);   // the launch does not reset its pool counter
                 if (ce == cudaSuccess)
                   ce = launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work,
-                                        P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_done, P.att_pool + l,
+                                        P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_pool + l,
                                         P.ao_hi, P.ao_lo, e->whole_pairs ? 2 : 0, e->d_status, e->st);
                 break;
         case 6: ce = launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->attn_norm[l], s.rms_eps, P.xn_hi,
                                        P.xn_lo, e->st); break;
         case 7: ce = launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st); break;
-        case 8: ce = e->moe_E ? launch_moe_swiglu(P.p_gu.out(), P.moe_w, P.R, e->moe_F, e->moe_E + e->moe_S, P.ff_hi, P.ff_lo, e->st)
+        case 8: if (P.p_gu.sw_hi) break;             // no such kernel: the SwiGLU is in the GEMM's epilogue
+                ce = e->moe_E ? launch_moe_swiglu(P.p_gu.out(), P.moe_w, P.R, e->moe_F, e->moe_E + e->moe_S, P.ff_hi, P.ff_lo, e->st)
                               : launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st);
                 break;
         case 9: {
@@ -1026,7 +1040,8 @@ int corun_debug_gemm_trace(corun_engine *e, int32_t kind, int32_t layer, uint64_
   RC(sync_stream(e));
   Program &P = e->dec;
   const GemmPlan *pl[5] = {&P.p_qkv, &P.p_o, &P.p_gu, &P.p_down, &P.p_lm};
-  const CUtensorMap *tm[5] = {&e->tm_qkv[layer], &e->tm_o[layer], &e->tm_gu[layer], &e->tm_down[layer], nullptr};
+  const CUtensorMap *tm[5] = {&e->tm_qkv[layer], &e->tm_o[layer], P.p_gu.sw_hi ? &e->tm_gu_half[layer] : &e->tm_gu[layer],
+                              &e->tm_down[layer], nullptr};
   const GemmPlan &p = *pl[kind];
   unsigned long long *d = nullptr;
   if (cudaMalloc(&d, (size_t)p.grid * 8 * sizeof(unsigned long long)) != cudaSuccess) return CORUN_ENOMEM;
@@ -1055,7 +1070,7 @@ int corun_debug_attn_trace(corun_engine *e, int32_t layer, uint64_t *stamps, int
     ce = cudaMemsetAsync(P.att_pool + layer, 0, sizeof(int), e->st);   // the launch does not reset its pool counter
     if (ce == cudaSuccess)
       ce = launch_attention(e->tm_k[layer], e->tm_v[layer], P.q, rows, s.n_q_heads, kv_layout(e), layer, e->max_splits,
-                            P.att_work, P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_done, P.att_pool + layer,
+                            P.att_work, P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_pool + layer,
                             P.ao_hi, P.ao_lo, e->whole_pairs ? 2 : 0, e->d_status, e->st, i == 1 ? d : nullptr);   // only the second launch is recorded
   }
   if (ce == cudaSuccess) ce = cudaMemcpyAsync(stamps, d, n * sizeof(unsigned long long), cudaMemcpyDeviceToHost, e->st);

@@ -37,13 +37,18 @@ constexpr uint32_t A_BLOCK_BYTES = GEMM_ROW_BLOCK * GEMM_BLOCK_K * 2;      // 16
 // blocks of BN rows).  group_tab holds, per group, the first weight row, the first weight k-block and the number
 // of rows (0 = the group is empty: its CTAs leave at once); the group's activations are rows group * BN .. of
 // the activation matrices, its output rows group * BN .. of `direct` (N columns wide, tiles_per_group tiles).
-template <bool MASKED, bool STACKED, bool GROUPED>
+// SWIGLU: W is a gate / up matrix ([2F, K]: F gate rows, then F up rows).  A tile is sw_half gate rows and the
+// sw_half up rows of the same outputs (two boxes of sw_half rows land in one stage; the MMA's N is 2 * sw_half),
+// every CTA owns whole tiles, and the epilogue writes silu(gate) * up as a bf16 hi/lo pair ([BN, F]) instead of
+// fp32 sums: no partials, no separate SwiGLU kernel.  tmW then has a box of sw_half rows.
+template <bool MASKED, bool STACKED, bool GROUPED, bool SWIGLU>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmHi,
                     const __grid_constant__ CUtensorMap tmLo, float *__restrict__ direct, float *__restrict__ ws,
                     const int *__restrict__ cta_start, int N, int KB, int BN, int R, int stages, int tmem_cols,
                     uint32_t idesc, const float *row_keep, int keep_pitch, int keep_div, const int *group_tab,
-                    int tiles_per_group, int *status, unsigned long long *trace) {
+                    int tiles_per_group, int *status, unsigned long long *trace, __nv_bfloat16 *__restrict__ sw_hi,
+                    __nv_bfloat16 *__restrict__ sw_lo, int sw_half) {
   int g_id = 0, g_j = 0, g_wrow = 0, g_wk = 0, g_rows = 0;
   if (GROUPED) {
     griddep_wait();                                 // the group table comes from an earlier kernel
@@ -75,8 +80,9 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   // per k-slice yields W*hi in accumulator lanes 0-63 and W*lo in lanes 64-127; the epilogue adds them.
   constexpr bool stacked = STACKED;                 // = (BN <= 64), fixed at compile time
   const uint32_t lo_off = stacked ? (uint32_t)(64 * GEMM_BLOCK_K * 2) : x_bytes;
-  const uint32_t stage_bytes = W_TILE_BYTES + (stacked ? A_BLOCK_BYTES : 2 * x_bytes);
-  const uint32_t tx_bytes = W_TILE_BYTES + 2 * x_bytes;
+  const uint32_t w_tile_bytes = SWIGLU ? (uint32_t)(2 * sw_half * GEMM_BLOCK_K * 2) : W_TILE_BYTES;
+  const uint32_t stage_bytes = w_tile_bytes + (stacked ? A_BLOCK_BYTES : 2 * x_bytes);
+  const uint32_t tx_bytes = w_tile_bytes + 2 * x_bytes;
   const int n_rb = (BN + GEMM_ROW_BLOCK - 1) / GEMM_ROW_BLOCK;      // blocks of 128 activation rows
   // up to 128 rows need 256 TMEM columns: two accumulator buffers fit, so the epilogue of one
   // segment overlaps the MMAs of the next
@@ -126,6 +132,11 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const int g = k0 + it, tile = g / KB, kb = g - tile * KB;
         const uint32_t fb = smem_u32(&full_bar[it]);
         mbar_arrive_expect_tx(fb, tx_bytes);
+        if (SWIGLU) {
+          tma_load_2d(tiles_base + (uint32_t)it * stage_bytes, &tmW, kb * GEMM_BLOCK_K, tile * sw_half, fb, pol_w);
+          tma_load_2d(tiles_base + (uint32_t)it * stage_bytes + w_tile_bytes / 2, &tmW, kb * GEMM_BLOCK_K,
+                      N / 2 + tile * sw_half, fb, pol_w);
+        } else
         tma_load_2d(tiles_base + (uint32_t)it * stage_bytes, &tmW, (GROUPED ? g_wk + kb : kb) * GEMM_BLOCK_K,
                     GROUPED ? g_wrow + g_j * GEMM_TILE_N : tile * GEMM_TILE_N, fb, pol_w);
         if (it == 0) TRACE(2);
@@ -135,8 +146,8 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const int g = k0 + it, tile = g / KB, kb = g - tile * KB;
         const uint32_t fb = smem_u32(&full_bar[it]);
         const uint32_t dst = tiles_base + (uint32_t)it * stage_bytes;
-        tma_load_2d(dst + W_TILE_BYTES, &tmHi, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
-        tma_load_2d(dst + W_TILE_BYTES + lo_off, &tmLo, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
+        tma_load_2d(dst + w_tile_bytes, &tmHi, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
+        tma_load_2d(dst + w_tile_bytes + lo_off, &tmLo, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
       }
       int it = n_pre;
       for (int g = k0 + n_pre; g < k1; ++g, ++it) {
@@ -147,10 +158,14 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const uint32_t fb = smem_u32(&full_bar[s]);
         const uint32_t dst = tiles_base + (uint32_t)s * stage_bytes;
         mbar_arrive_expect_tx(fb, tx_bytes);
+        if (SWIGLU) {
+          tma_load_2d(dst, &tmW, kb * GEMM_BLOCK_K, tile * sw_half, fb, pol_w);
+          tma_load_2d(dst + w_tile_bytes / 2, &tmW, kb * GEMM_BLOCK_K, N / 2 + tile * sw_half, fb, pol_w);
+        } else
         tma_load_2d(dst, &tmW, (GROUPED ? g_wk + kb : kb) * GEMM_BLOCK_K, GROUPED ? g_wrow + g_j * GEMM_TILE_N : tile * GEMM_TILE_N,
                     fb, pol_w);
-        tma_load_2d(dst + W_TILE_BYTES, &tmHi, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
-        tma_load_2d(dst + W_TILE_BYTES + lo_off, &tmLo, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
+        tma_load_2d(dst + w_tile_bytes, &tmHi, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
+        tma_load_2d(dst + w_tile_bytes + lo_off, &tmLo, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
       }
       TRACE(3);
     }
@@ -174,7 +189,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           const uint32_t w_addr = tiles_base + (uint32_t)s * stage_bytes;
           const uint64_t w_desc = umma_desc_sw128(w_addr);
           if (stacked) {
-            const uint64_t a_desc = umma_desc_sw128(w_addr + W_TILE_BYTES);
+            const uint64_t a_desc = umma_desc_sw128(w_addr + w_tile_bytes);
             const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_cols;
 #pragma unroll
             for (int k = 0; k < GEMM_BLOCK_K / 16; ++k) {
@@ -183,8 +198,8 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             }
           } else {
             for (int rb = 0; rb < n_rb; ++rb) {
-              const uint64_t hi_desc = umma_desc_sw128(w_addr + W_TILE_BYTES + (uint32_t)rb * A_BLOCK_BYTES);
-              const uint64_t lo_desc = umma_desc_sw128(w_addr + W_TILE_BYTES + x_bytes + (uint32_t)rb * A_BLOCK_BYTES);
+              const uint64_t hi_desc = umma_desc_sw128(w_addr + w_tile_bytes + (uint32_t)rb * A_BLOCK_BYTES);
+              const uint64_t lo_desc = umma_desc_sw128(w_addr + w_tile_bytes + x_bytes + (uint32_t)rb * A_BLOCK_BYTES);
               const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_cols + (uint32_t)rb * GEMM_TILE_N;
 #pragma unroll
               for (int k = 0; k < GEMM_BLOCK_K / 16; ++k) {
@@ -221,6 +236,88 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       const int n0 = GROUPED ? g_j * GEMM_TILE_N : tile * GEMM_TILE_N;
       // optional: rows whose entry for this tile's column group is zero are not stored (nobody reads them)
       const float *keep = MASKED ? row_keep + tile / keep_div : nullptr;
+      if (SWIGLU) {
+        // accumulator columns 0 .. sw_half-1: gate sums of outputs tile * sw_half .., the next sw_half columns: the
+        // up sums of the same outputs; every tile is whole
+        const int HALF = sw_half;
+        const int F = N / 2, f0 = tile * HALF;
+        auto silu_mul = [](float gt, float up) { return __fdividef(gt, 1.f + __expf(-gt)) * up; };
+        if (stacked) {
+          const bool lo_warp = lane_base >= 64;
+          const int row = (lane_base & 63) + lane;
+          const bool warp_needed = (lane_base & 63) < R;   // warp-uniform
+          float *xs = xch[lo_warp ? 1 : 0] + row * 33;
+          const int te = (int)threadIdx.x - 64, srow = te >> 3, scol = (te & 7) * 4;
+          for (int c0 = 0; c0 < HALF; c0 += 32) {
+            if (f0 + c0 >= F) break;                   // outputs beyond the matrix (last tile); uniform
+            float gt[4][4];
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {     // 0: the gate columns, 1: the up columns
+              if (warp_needed) {
+                uint32_t v[32];
+                const uint32_t ta = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)acc * acc_cols +
+                                    (uint32_t)(part * HALF + c0);
+                tmem_ld16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+                tmem_ld16(ta + 16, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) xs[j] = __uint_as_float(v[j]);
+              }
+              asm volatile("bar.sync 1, 128;" ::: "memory");
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const int r = i * 16 + srow;
+                if (r < R) {
+                  const float *h = xch[0] + r * 33 + scol, *l = xch[1] + r * 33 + scol;
+                  const float s0 = h[0] + l[0], s1 = h[1] + l[1], s2 = h[2] + l[2], s3 = h[3] + l[3];
+                  if (part == 0) {
+                    gt[i][0] = s0; gt[i][1] = s1; gt[i][2] = s2; gt[i][3] = s3;
+                  } else if (c0 + scol < HALF && f0 + c0 + scol < F) {   // HALF % 4 == 0, F % 4 == 0
+                    const float y[4] = {silu_mul(gt[i][0], s0), silu_mul(gt[i][1], s1), silu_mul(gt[i][2], s2),
+                                        silu_mul(gt[i][3], s3)};
+                    __nv_bfloat16 a[4], b[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                      a[q] = __float2bfloat16_rn(y[q]);
+                      b[q] = __float2bfloat16_rn(y[q] - __bfloat162float(a[q]));
+                    }
+                    const size_t o = (size_t)r * F + f0 + c0 + scol;
+                    *reinterpret_cast<uint2 *>(sw_hi + o) = *reinterpret_cast<const uint2 *>(a);
+                    *reinterpret_cast<uint2 *>(sw_lo + o) = *reinterpret_cast<const uint2 *>(b);
+                  }
+                }
+              }
+              asm volatile("bar.sync 1, 128;" ::: "memory");
+            }
+          }
+        } else {
+          for (int rb = 0; rb < n_rb; ++rb) {
+            const int row_base = rb * GEMM_ROW_BLOCK + lane_base;
+            if (row_base >= R) continue;                 // warp-uniform
+            const int row = row_base + lane;
+            for (int c0 = 0; c0 < HALF; c0 += 8) {
+              if (f0 + c0 >= F) break;                   // F % 8 == 0
+              uint32_t vg[8], vu[8];
+              const uint32_t ta = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)acc * acc_cols +
+                                  (uint32_t)(rb * GEMM_TILE_N + c0);
+              tmem_ld8(ta, vg);
+              tmem_ld8(ta + HALF, vu);
+              tmem_ld_wait();
+              if (row >= R) continue;
+              __nv_bfloat16 a[8], b[8];
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {
+                const float y = silu_mul(__uint_as_float(vg[q]), __uint_as_float(vu[q]));
+                a[q] = __float2bfloat16_rn(y);
+                b[q] = __float2bfloat16_rn(y - __bfloat162float(a[q]));
+              }
+              const size_t o = (size_t)row * F + f0 + c0;
+              *reinterpret_cast<uint4 *>(sw_hi + o) = *reinterpret_cast<const uint4 *>(a);
+              *reinterpret_cast<uint4 *>(sw_lo + o) = *reinterpret_cast<const uint4 *>(b);
+            }
+          }
+        }
+      } else
       if (stacked) {
         // lanes 0-63 (warps with lane_base 0, 32) hold W*hi of rows 0-63, lanes 64-127 hold W*lo of the
         // same rows: every warp parks 32 columns of its rows in shared memory, then the 128 threads add
@@ -442,6 +539,59 @@ int gemm_plan_create(GemmPlan *p, const void *W, int N, int K, const void *Xhi, 
   return CORUN_OK;
 }
 
+int gemm_swiglu_half(int F, int num_sms) {
+  int half = ((F + num_sms - 1) / num_sms + 7) / 8 * 8;
+  if (half < 64) half = 64;
+  if (half > GEMM_TILE_N / 2) half = GEMM_TILE_N / 2;
+  return half;
+}
+
+int gemm_plan_create_swiglu(GemmPlan *p, const void *W, int F, int K, const void *Xhi, const void *Xlo, int R, int BN,
+                            __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int num_sms) {
+  if (F <= 0 || F % 8 || K <= 0 || K % GEMM_BLOCK_K || BN % 16 || BN < 16 || BN > 256 || R < 1 || R > BN || !out_hi || !out_lo ||
+      num_sms < 1)
+    return CORUN_EINVAL;
+  // as many whole tiles as there are SMs, if the matrix is large enough: the narrowest tile (a multiple of 8 gate
+  // rows, at least 64) that still gives every CTA at most one
+  const int HALF = gemm_swiglu_half(F, num_sms);
+  p->sw_half = HALF;
+  p->N = 2 * F; p->K = K; p->R = R; p->BN = BN;
+  p->n_tiles = (F + HALF - 1) / HALF;
+  p->KB = K / GEMM_BLOCK_K;
+  p->grid = p->n_tiles < num_sms ? p->n_tiles : num_sms;
+  if ((long long)p->n_tiles * p->KB >= (1ll << 31)) return CORUN_EINVAL;
+  const size_t stage = (size_t)2 * HALF * GEMM_BLOCK_K * 2 + (BN <= 64 ? (size_t)A_BLOCK_BYTES : 2 * (size_t)BN * GEMM_BLOCK_K * 2);
+  int stages = (int)((GEMM_MAX_DYN_SMEM - 1024 - A_BLOCK_BYTES) / stage);
+  if (stages > MAX_STAGES) stages = MAX_STAGES;
+  if (stages < 2) return CORUN_EINVAL;
+  p->stages = stages;
+  p->smem_bytes = stage * stages + A_BLOCK_BYTES + 1024;
+  p->tmem_cols = 512;
+  p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * HALF) >> 3) << 17) |
+             ((uint32_t)(GEMM_ROW_BLOCK >> 4) << 24);
+  p->direct = nullptr;
+  p->ws = nullptr;
+  p->sw_hi = out_hi;
+  p->sw_lo = out_lo;
+  int rc;
+  if ((rc = gemm_encode_map(&p->tmW, W, 2 * F, K, HALF)) != 0) return rc;
+  if ((rc = gemm_encode_map(&p->tmHi, Xhi, BN, K, BN)) != 0) return rc;
+  if ((rc = gemm_encode_map(&p->tmLo, Xlo, BN, K, BN)) != 0) return rc;
+  // whole tiles only: CTA c takes tiles [c * n_tiles / grid, (c + 1) * n_tiles / grid)
+  std::vector<int> tab((size_t)p->grid + 1);
+  for (int c = 0; c <= p->grid; ++c) tab[(size_t)c] = (int)((long long)c * p->n_tiles / p->grid) * p->KB;
+  int *d_tab = nullptr;
+  if (cudaMalloc(&d_tab, tab.size() * sizeof(int)) != cudaSuccess) return CORUN_ENOMEM;
+  cudaError_t me = cudaMemcpy(d_tab, tab.data(), tab.size() * sizeof(int), cudaMemcpyHostToDevice);
+  if (me != cudaSuccess) { g_last_cuda_error = (int)me; cudaFree(d_tab); return CORUN_ECUDA; }
+  p->d_cta_start = d_tab;
+  p->d_tile_first = p->d_tile_cend = p->d_split_tiles = nullptr;
+  p->n_split_tiles = 0;
+  cudaError_t ae = gemm_prepare_kernel();
+  if (ae != cudaSuccess) { g_last_cuda_error = (int)ae; return CORUN_ECUDA; }
+  return CORUN_OK;
+}
+
 int gemm_plan_create_grouped(GemmPlan *p, const void *W, long long w_rows, int w_cols, int N, int K, const void *Xhi,
                              const void *Xlo, int n_groups, int BN, float *direct, const int *group_tab) {
   if (N <= 0 || N % GEMM_TILE_N || K <= 0 || K % GEMM_BLOCK_K || w_cols % GEMM_BLOCK_K || BN % 16 || BN < 16 || BN > 64 ||
@@ -483,11 +633,13 @@ int gemm_plan_create_grouped(GemmPlan *p, const void *W, long long w_rows, int w
 }
 
 cudaError_t gemm_prepare_kernel() {
-  cudaError_t e = cudaFuncSetAttribute(gemm_streamk_kernel<false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  cudaError_t e = cudaFuncSetAttribute(gemm_streamk_kernel<false, false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   return e;
 }
 
@@ -502,11 +654,13 @@ cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int 
   auto go = [&](auto kernel) {
     return launch_k(kernel, dim3(p.grid), dim3(GEMM_THREADS), p.smem_bytes, st, pdl, tmW_override ? *tmW_override : p.tmW,
                     p.tmHi, p.tmLo, p.direct, p.ws, p.d_cta_start, p.N, p.KB, p.BN, p.R, p.stages, p.tmem_cols, p.idesc,
-                    p.row_keep, p.keep_pitch, p.keep_div, p.group_tab, p.tiles_per_group, d_status, trace);
+                    p.row_keep, p.keep_pitch, p.keep_div, p.group_tab, p.tiles_per_group, d_status, trace, p.sw_hi, p.sw_lo,
+                    p.sw_half);
   };
-  if (p.group_tab) return go(gemm_streamk_kernel<false, true, true>);
-  if (masked) return stacked ? go(gemm_streamk_kernel<true, true, false>) : go(gemm_streamk_kernel<true, false, false>);
-  return stacked ? go(gemm_streamk_kernel<false, true, false>) : go(gemm_streamk_kernel<false, false, false>);
+  if (p.sw_hi) return stacked ? go(gemm_streamk_kernel<false, true, false, true>) : go(gemm_streamk_kernel<false, false, false, true>);
+  if (p.group_tab) return go(gemm_streamk_kernel<false, true, true, false>);
+  if (masked) return stacked ? go(gemm_streamk_kernel<true, true, false, false>) : go(gemm_streamk_kernel<true, false, false, false>);
+  return stacked ? go(gemm_streamk_kernel<false, true, false, false>) : go(gemm_streamk_kernel<false, false, false, false>);
 }
 
 cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st, bool pdl) {

@@ -11,6 +11,7 @@
 // adds the partials in ascending CTA order (gemm_load).  No atomics anywhere.
 #pragma once
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -89,6 +90,9 @@ struct GemmPlan {
   // Grouped mode (gemm_plan_create_grouped): one CTA per (group, weight tile); see gemm.cu.
   const int *group_tab = nullptr;    // device, not owned: per group (first weight row, first weight k-block, rows)
   int tiles_per_group = 0;
+  // Gate / up GEMM with SwiGLU in the epilogue (gemm_plan_create_swiglu): the bf16 hi/lo output [BN, N / 2].
+  __nv_bfloat16 *sw_hi = nullptr, *sw_lo = nullptr;
+  int sw_half = 0;                   // gate rows (= up rows) per tile
   GemmOut out() const { return GemmOut{direct, ws, d_tile_first, d_tile_cend, N, KB, BN}; }
 };
 
@@ -107,6 +111,14 @@ void gemm_plan_destroy(GemmPlan *p);
 // bf16.  One CTA per (group, tile of 256 weight rows), all k-blocks of it: no partials.  N % 256 == 0.
 int gemm_plan_create_grouped(GemmPlan *p, const void *W, long long w_rows, int w_cols, int N, int K, const void *Xhi,
                              const void *Xlo, int n_groups, int BN, float *direct, const int *group_tab);
+// Gate / up GEMM with the SwiGLU in its epilogue: W is [2F, K] (F gate rows, then F up rows; F % 8 == 0);
+// out_hi / out_lo [BN, F] receive silu(gate) * up of rows 0 .. R-1 as a bf16 hi/lo pair.  A tile is
+// gemm_swiglu_half(F, num_sms) gate rows with the up rows of the same outputs, and every CTA owns whole tiles
+// (one each when the SMs allow), so there are no partials; a tensor map that overrides the plan's at launch
+// must have a box of that many rows (gemm_encode_map(.., box_rows = gemm_swiglu_half(..))).
+int gemm_swiglu_half(int F, int num_sms);
+int gemm_plan_create_swiglu(GemmPlan *p, const void *W, int F, int K, const void *Xhi, const void *Xlo, int R, int BN,
+                            __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int num_sms);
 // The allocation-free half of gemm_plan_create: fills every host-side field and tensor map of the
 // plan and writes the partition tables (cta_start, tile_first, tile_cend, split_tiles) to `tab`
 // (capacity tab_cap ints; *tab_ints = ints used).  gemm_plan_bind_tables points the plan at a device

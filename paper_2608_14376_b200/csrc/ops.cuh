@@ -60,9 +60,8 @@ cudaError_t launch_resid_norm(float *h, int H, const __nv_bfloat16 *embed, const
 // RoPE on q and k, q -> q_out fp32 [R, nq*hd], k/v -> pages (fp16) at the row's position.
 cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *rope_tab, int nq, const KvLayout &kv,
                             int layer, float *q_out, cudaStream_t st);
-// Split-KV paged attention partials and their fixed-order combine -> bf16 hi/lo [R, nq*hd] (rows that are
-// not active keep what they held).  done_count: [R * n_kv] ints, zero before the first launch (the kernel
-// leaves them zero).  pool_count: one int, zero before the launch (not reset by it): the items beyond the
+// Split-KV paged attention partials and, in a second kernel, their fixed-order combine -> bf16 hi/lo
+// [R, nq*hd] (rows that are not active keep what they held).  pool_count: one int, zero before the launch (not reset by it): the items beyond the
 // CTAs' fixed stretches are drawn through it.  reuse: 1 when the rows are the consecutive tokens of one
 // request in one slot (a prefill chunk): launch_attention_prefill runs instead; 2 for the ablation in which a
 // CTA takes whole (row, kv head) pairs (the work list then carries the pair table); else 0.
@@ -72,7 +71,7 @@ cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *
 // grid_ctas: persistent CTAs to launch (one per SM).
 cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, const float *q, const Rows &rows, int nq,
                              const KvLayout &kv, int layer, int max_splits, const int *work, const int *n_work,
-                             int grid_ctas, float *part_acc, float *part_ml, int *done_count, int *pool_count,
+                             int grid_ctas, float *part_acc, float *part_ml, int *pool_count,
                              __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int reuse, int *d_status, cudaStream_t st,
                              unsigned long long *trace = nullptr);   // optional [grid][64][8] stamps (debug)
 // n_work: 2 + 2 * rows * n_kv ints (item count, pair count, then the pairs' (first item, split count) when
