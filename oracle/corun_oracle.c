@@ -457,6 +457,154 @@ int32_t orc_sample(const float *logits, int64_t V, float temperature, float top_
   return tok;
 }
 
+/*
+ * The plain definition of S, kept beside the integer specification above as its pin: everything in fp64 with
+ * the C library's exp, no integers.
+ *   p_i     = exp((logit_i - max) / temperature)
+ *   nucleus = tokens in descending logit order (ties: lower id first) up to and including the first whose
+ *             running sum of p reaches top_p * sum_i p_i
+ *   token   = first nucleus member, in ascending id order, whose running sum of p exceeds u * Z,
+ *             u = u24 / 2^24, Z = nucleus mass.
+ * `margin` receives how close, relative to sum_i p_i, any of these comparisons came to going the other way.
+ * The integer specification must give the same token whenever the margin exceeds the accuracy of its weights
+ * (2e-7 relative per weight, hence per running sum); tests/test_oracle_sampler.py checks exactly that.
+ * orc_sample_plain_many / orc_sample_many evaluate n variates against one row (the row is sorted once).
+ */
+typedef struct {
+  int64_t V, n_in;
+  double total, Z, edge_margin;
+  double *p;       /* per token */
+  char *in;        /* nucleus membership */
+} orc_plain_row;
+
+static void orc_plain_prepare(orc_plain_row *R, const float *logits, int64_t V, float temperature, float top_p) {
+  int64_t best = 0;
+  for (int64_t i = 1; i < V; ++i)
+    if (logits[i] > logits[best]) best = i;
+  R->V = V;
+  R->p = (double *)malloc(sizeof(double) * (size_t)V);
+  R->in = (char *)calloc((size_t)V, 1);
+  orc_item *it = (orc_item *)malloc(sizeof(orc_item) * (size_t)V);
+  double total = 0.0;
+  for (int64_t i = 0; i < V; ++i) {
+    R->p[i] = exp(((double)logits[i] - (double)logits[best]) / (double)temperature);
+    it[i].idx = i;
+    it[i].logit = logits[i];
+  }
+  qsort(it, (size_t)V, sizeof(orc_item), orc_item_desc);
+  for (int64_t r = 0; r < V; ++r) total += R->p[it[r].idx];   /* summed in the order the nucleus is built in */
+  const double cut = (double)top_p * total;
+  double run = 0.0;
+  R->total = total;
+  R->Z = total;
+  R->edge_margin = 1.0;
+  R->n_in = V;
+  for (int64_t r = 0; r < V; ++r) {
+    const double before = run;
+    run += R->p[it[r].idx];
+    R->in[it[r].idx] = 1;
+    if (run >= cut || r == V - 1) {
+      R->Z = run;
+      R->n_in = r + 1;
+      if (r < V - 1) {
+        const double d1 = (run - cut) / total, d0 = (cut - before) / total;
+        R->edge_margin = d1 < d0 ? d1 : d0;
+      }
+      break;
+    }
+  }
+  free(it);
+}
+
+static int32_t orc_plain_draw(const orc_plain_row *R, uint32_t u24, double *margin) {
+  const double target = ((double)u24 / 16777216.0) * R->Z;
+  double run = 0.0, mg = R->edge_margin;
+  int32_t tok = -1;
+  int64_t last = -1;
+  for (int64_t i = 0; i < R->V; ++i) {
+    if (!R->in[i]) continue;
+    last = i;
+    const double before = run;
+    run += R->p[i];
+    if (run > target) {
+      tok = (int32_t)i;
+      const double d0 = (target - before) / R->total, d1 = (run - target) / R->total;
+      if (d0 < mg) mg = d0;
+      if (d1 < mg) mg = d1;
+      break;
+    }
+  }
+  if (tok < 0) { tok = (int32_t)last; mg = 0.0; }   /* rounding left the target at the very end: undecided */
+  if (margin) *margin = mg;
+  return tok;
+}
+
+int32_t orc_sample_plain(const float *logits, int64_t V, float temperature, float top_p, uint32_t u24, double *margin) {
+  if (temperature <= 0.0f) {
+    int64_t best = 0;
+    for (int64_t i = 1; i < V; ++i)
+      if (logits[i] > logits[best]) best = i;
+    if (margin) *margin = 1.0;
+    return (int32_t)best;
+  }
+  orc_plain_row R;
+  orc_plain_prepare(&R, logits, V, temperature, top_p);
+  const int32_t tok = orc_plain_draw(&R, u24, margin);
+  free(R.p); free(R.in);
+  return tok;
+}
+
+void orc_sample_plain_many(const float *logits, int64_t V, float temperature, float top_p, const uint32_t *u24, int64_t n,
+                           int32_t *tokens, double *margins) {
+  orc_plain_row R;
+  orc_plain_prepare(&R, logits, V, temperature, top_p);
+  for (int64_t k = 0; k < n; ++k) tokens[k] = orc_plain_draw(&R, u24[k], margins ? margins + k : NULL);
+  free(R.p); free(R.in);
+}
+
+/* The integer specification (orc_sample) for n variates against one row: the same weights, cut and draw,
+ * with the row sorted once.  temperature > 0. */
+void orc_sample_many(const float *logits, int64_t V, float temperature, float top_p, const uint32_t *u24, int64_t n,
+                     int32_t *tokens) {
+  int64_t best = 0;
+  for (int64_t i = 1; i < V; ++i)
+    if (logits[i] > logits[best]) best = i;
+  const float mx = logits[best];
+  const float inv_t_log2e = 0x1.715476p+0f / temperature;
+  uint64_t *wgt = (uint64_t *)malloc(sizeof(uint64_t) * (size_t)V);
+  orc_item *it = (orc_item *)malloc(sizeof(orc_item) * (size_t)V);
+  uint64_t total = 0;
+  for (int64_t i = 0; i < V; ++i) {
+    wgt[i] = orc_weight(logits[i], mx, inv_t_log2e);
+    total += wgt[i];
+    it[i].idx = i;
+    it[i].logit = logits[i];
+  }
+  qsort(it, (size_t)V, sizeof(orc_item), orc_item_desc);
+  uint64_t cut = (uint64_t)floor((double)top_p * (double)total);
+  if (cut > total) cut = total;
+  char *in = (char *)calloc((size_t)V, 1);
+  uint64_t run = 0, Z = 0;
+  for (int64_t r = 0; r < V; ++r) {
+    run += wgt[it[r].idx];
+    in[it[r].idx] = 1;
+    if (run >= cut) { Z = run; break; }
+  }
+  for (int64_t k = 0; k < n; ++k) {
+    const unsigned __int128 prod = (unsigned __int128)u24[k] * (unsigned __int128)Z;
+    const uint64_t rdraw = (uint64_t)(prod >> 24);
+    int32_t tok = -1;
+    uint64_t acc = 0;
+    for (int64_t i = 0; i < V; ++i) {
+      if (!in[i]) continue;
+      acc += wgt[i];
+      if (acc > rdraw) { tok = (int32_t)i; break; }
+    }
+    tokens[k] = tok;
+  }
+  free(wgt); free(it); free(in);
+}
+
 int orc_num_threads(void) {
   int n = 1;
 #ifdef _OPENMP

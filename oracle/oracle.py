@@ -82,6 +82,12 @@ def lib():
         L.orc_variate_u24.argtypes = [C.c_uint64, C.c_uint64]
         L.orc_sample.restype = C.c_int32
         L.orc_sample.argtypes = [C.c_void_p, C.c_int64, C.c_float, C.c_float, C.c_uint32, C.POINTER(C.c_double)]
+        L.orc_sample_plain.restype = C.c_int32
+        L.orc_sample_plain.argtypes = [C.c_void_p, C.c_int64, C.c_float, C.c_float, C.c_uint32, C.POINTER(C.c_double)]
+        L.orc_sample_plain_many.restype = None
+        L.orc_sample_plain_many.argtypes = [C.c_void_p, C.c_int64, C.c_float, C.c_float, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
+        L.orc_sample_many.restype = None
+        L.orc_sample_many.argtypes = [C.c_void_p, C.c_int64, C.c_float, C.c_float, C.c_void_p, C.c_int64, C.c_void_p]
         L.orc_num_threads.restype = C.c_int
         L.orc_weight.restype = C.c_uint64
         L.orc_weight.argtypes = [C.c_float, C.c_float, C.c_float]
@@ -286,6 +292,33 @@ def sample(logits, temperature: float, top_p: float, u24: int):
     m = C.c_double(0.0)
     tok = lib().orc_sample(_ptr(lg), lg.shape[0], temperature, top_p, u24, C.byref(m))
     return int(tok), float(m.value)
+
+
+def sample_plain(logits, temperature: float, top_p: float, u24: int):
+    """The plain fp64 definition of S (the pin of the integer specification): returns (token, margin)."""
+    lg = _f32(logits)
+    m = C.c_double(0.0)
+    tok = lib().orc_sample_plain(_ptr(lg), lg.shape[0], temperature, top_p, u24, C.byref(m))
+    return int(tok), float(m.value)
+
+
+def sample_plain_many(logits, temperature: float, top_p: float, u24s):
+    """Plain S for many variates against one row: (tokens int32[n], margins float64[n])."""
+    lg = _f32(logits)
+    u = np.ascontiguousarray(u24s, dtype=np.uint32)
+    tok = np.empty(u.shape[0], np.int32)
+    mg = np.empty(u.shape[0], np.float64)
+    lib().orc_sample_plain_many(_ptr(lg), lg.shape[0], temperature, top_p, _ptr(u), u.shape[0], _ptr(tok), _ptr(mg))
+    return tok, mg
+
+
+def sample_many(logits, temperature: float, top_p: float, u24s):
+    """The integer specification S for many variates against one row (temperature > 0): tokens int32[n]."""
+    lg = _f32(logits)
+    u = np.ascontiguousarray(u24s, dtype=np.uint32)
+    tok = np.empty(u.shape[0], np.int32)
+    lib().orc_sample_many(_ptr(lg), lg.shape[0], temperature, top_p, _ptr(u), u.shape[0], _ptr(tok))
+    return tok
 
 
 def weight(logit: float, max_logit: float, inv_t_log2e: float) -> int:

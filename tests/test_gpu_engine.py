@@ -138,6 +138,8 @@ def test_sampled_decoding_is_invariant_and_matches_S_on_gpu_logits(orc, tiny, en
         lg = np.frombuffer(row, np.float32)
         want, _ = orc.sample(lg, T, P, orc.variate_u24(seed, t))
         assert tok == want, t
+        plain, plain_margin = orc.sample_plain(lg, T, P, orc.variate_u24(seed, t))   # the plain fp64 definition
+        assert plain_margin < 1e-6 or tok == plain, t
         checked += 1
     assert checked == 13
     # a different seed draws different variates

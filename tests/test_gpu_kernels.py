@@ -71,10 +71,15 @@ def _check_sampler(orc, logits, T, top_p, us):
     rows = np.repeat(logits[None], len(us), axis=0)
     got = corun.debug_sample(rows, T, top_p, np.array(us, np.uint32))
     n_checked = 0
-    for u, g in zip(us, got):
+    # the plain fp64 definition of S decides the same token wherever its own margin exceeds the accuracy of
+    # the specification's integer weights (2e-7 relative): checked on the GPU's tokens too
+    plain, plain_margin = orc.sample_plain_many(logits, T, top_p, np.array(us, np.uint32))
+    for k, (u, g) in enumerate(zip(us, got)):
         # the sampling weights are integers in a stated fp32 arithmetic: the decision is exact
         want, margin = orc.sample(logits, T, top_p, int(u))
         assert g == want, (u, g, want, margin)
+        if plain_margin[k] >= 1e-6:
+            assert g == plain[k], (u, g, int(plain[k]), float(plain_margin[k]))
         n_checked += 1
     return n_checked
 

@@ -141,3 +141,79 @@ def test_integer_weight_follows_the_exponential(orc):
     assert orc.weight(0.0, 0.0, c) == 1 << 40
     assert orc.weight(-100.0, 0.0, c) == 0
     assert orc.weight(-19.4, 0.0, c) > 0          # 2^40 * 2^-39.98: the last non-zero weights
+
+
+# ---------------------------------------------------------------------------------------------------------
+# The integer specification of S (orc_sample: the contract both the oracle and the kernel implement) against
+# the plain fp64 definition (orc_sample_plain: exp from the C library, no integers).  The specification's
+# weights are within 2e-7 of the exact exponential, so the two must pick the same token whenever the plain
+# definition's own margin (distance of its comparisons to flipping, relative to the total mass) exceeds that
+# accuracy; 1e-6 is asserted, which contains the 1e-5 band.
+MARGIN = 1e-6
+
+
+def _rows_for_spec_vs_plain():
+    rng = np.random.default_rng(11)
+    rows = []
+    # the benchmark's regime: full vocabulary, logit std 1.28
+    for _ in range(6):
+        rows.append(("full-vocab", (rng.standard_normal(151936) * 1.28).astype(np.float32)))
+    # heavily tied rows: few distinct values
+    rows.append(("tied-8-values", rng.integers(0, 8, 151936).astype(np.float32) * 0.37))
+    rows.append(("tied-small", rng.integers(0, 3, 4096).astype(np.float32)))
+    # a dominant token
+    dom = (rng.standard_normal(151936) * 1.28).astype(np.float32)
+    dom[77777] = 25.0
+    rows.append(("dominant", dom))
+    for v in (2048, 8192, 32768):
+        for _ in range(4):
+            rows.append((f"V{v}", (rng.standard_normal(v) * 1.28).astype(np.float32)))
+    return rows
+
+
+def test_integer_specification_equals_plain_definition_outside_its_margin(orc):
+    rng = np.random.default_rng(5)
+    T, P = 0.7, 0.95
+    n_pairs = n_checked = n_band = 0
+    for name, lg in _rows_for_spec_vs_plain():
+        u = rng.integers(0, 1 << 24, 1000, dtype=np.uint32)
+        u[:3] = (0, (1 << 24) - 1, 1 << 23)
+        spec = orc.sample_many(lg, T, P, u)
+        plain, mg = orc.sample_plain_many(lg, T, P, u)
+        ok = mg >= MARGIN
+        assert (spec[ok] == plain[ok]).all(), name
+        # the many-variate entry points are the single-variate ones
+        for k in (0, 1, 2, 3, 250, 999):
+            assert orc.sample(lg, T, P, int(u[k]))[0] == spec[k]
+            t1, m1 = orc.sample_plain(lg, T, P, int(u[k]))
+            assert t1 == plain[k] and m1 == mg[k]
+        n_pairs += len(u)
+        n_checked += int(ok.sum())
+        n_band += int((mg >= 1e-5).sum())
+    # about half of the pairs are decided outside the margin (per-token mass at V = 151936 is ~7e-6, so the
+    # 1e-5 band alone would leave few of the full-vocabulary draws)
+    print(f"spec-S == plain-S on {n_checked} of {n_pairs} pairs (margin >= {MARGIN:g}); "
+          f"{n_pairs - n_checked} inside the margin; {n_band} have margin >= 1e-5")
+    assert n_checked >= 10_000 and n_checked >= 0.5 * n_pairs
+
+
+def test_other_temperatures_and_nucleus_sizes(orc):
+    rng = np.random.default_rng(6)
+    lg = (rng.standard_normal(20000) * 1.5).astype(np.float32)
+    for T, P in ((0.3, 0.5), (1.0, 1.0), (1.3, 0.9), (0.7, 0.05)):
+        u = rng.integers(0, 1 << 24, 300, dtype=np.uint32)
+        spec = orc.sample_many(lg, T, P, u)
+        plain, mg = orc.sample_plain_many(lg, T, P, u)
+        ok = mg >= MARGIN
+        assert ok.mean() > 0.5
+        assert (spec[ok] == plain[ok]).all(), (T, P)
+
+
+def test_plain_definition_two_logit_closed_form(orc):
+    # P(token 0) = sigmoid((l0 - l1) / T): the plain definition switches tokens at u = that probability
+    l0, l1, T = 0.3, -0.9, 0.8
+    p0 = 1.0 / (1.0 + math.exp(-(l0 - l1) / T))
+    lg = np.array([l0, l1], np.float32)
+    for u24 in range(0, 1 << 24, 1 << 16):
+        tok, _ = orc.sample_plain(lg, T, 1.0, u24)
+        assert tok == (0 if u24 / 2**24 < p0 else 1) or abs(u24 / 2**24 - p0) < 1e-6
