@@ -1,8 +1,9 @@
 """Full-size parity at the Qwen3-8B shape (36 layers, hidden 4096, 32 q / 8 kv heads, head_dim 128,
 FFN 12288, vocab 151936; B = 64), in the launch configuration bench.py times: sampled outputs the
-oracle can compute one by one.  (i) real isolated prefill + teacher-forced decode steps for two
+oracle can compute one by one.  (i) real isolated prefill + eight teacher-forced decode steps for four
 requests; (ii) long contexts via seeded synthetic cache rows (the oracle cannot afford to prefill
-them), one decode step, run among co-tenants; (iii) bitwise slot / co-tenant invariance."""
+them), one decode step, run among co-tenants; (iii) the same for ALL 40 active slots of the timed
+workload (bench.py's slots, contexts and seeds); (iv) bitwise slot / co-tenant invariance."""
 import numpy as np
 import pytest
 
@@ -29,7 +30,7 @@ def qwen(orc):
     w_t = synth.make_weights_torch(sh, seed=0, device="cuda")
     w_np = synth.weights_torch_to_numpy(w_t)
     model = oracle_model(orc, sh, w_np)
-    eng = corun.Engine(sh, w_t, B, MAX_CTX, kv_pool_blocks=6000)
+    eng = corun.Engine(sh, w_t, B, MAX_CTX, kv_pool_blocks=6400)
     yield sh, model, eng
     eng.close()
 
@@ -42,8 +43,8 @@ def _compare(eng, slot, ref_logits, stats):
 
 def test_prefill_and_decode_parity_with_sampling(orc, qwen):
     sh, model, eng = qwen
-    prompts = synth.make_prompts(sh.vocab, [48, 150], seed=5)
-    slots = [9, 41]
+    prompts = synth.make_prompts(sh.vocab, [48, 150, 17, 230], seed=5)
+    slots = [9, 41, 0, 63]
     stats = {"worst": 0.0}
     reqs = []
     for i, (s, p) in enumerate(zip(slots, prompts)):
@@ -62,7 +63,7 @@ def test_prefill_and_decode_parity_with_sampling(orc, qwen):
     seeds = np.zeros(B, np.uint64)
     for i, s in enumerate(slots):
         seeds[s] = synth.request_seed(i)
-    for step in range(3):
+    for step in range(8):
         toks = eng.decode_step(active, seeds)
         for i, s in enumerate(slots):
             r = reqs[i]
@@ -124,6 +125,54 @@ def test_long_context_decode_parity_and_invariance(orc, qwen):
     assert eng.logits(slot2).tobytes() == rows[20]
     assert toks2[slot2] == toks[20]
     eng.release(slot2)
+
+
+def test_all_active_slots_of_the_timed_workload(orc, qwen):
+    """One decode step of the workload bench.py times (its 40 active slots of 64, contexts 654..4071, request
+    seeds, T 0.7 / top-p 0.95), every active row's logits against the oracle.  The caches hold seeded synthetic
+    rows (one draw per slot, shifted by 7 tokens per layer, pre-rounded to the cache's fp16 so that both sides
+    hold the same numbers); the oracle runs the slots one after the other."""
+    import bench
+
+    sh, model, eng = qwen
+    sh_b, B_b, slots, ctx, T_b, P_b, kv_std = bench.workload_inputs("qwen3_8b_b64")
+    assert B_b == B and (T_b, P_b) == (T, P) and len(slots) == 40
+
+    def layer_rows(k0, v0, layer):
+        return np.roll(k0, 7 * layer, axis=0), np.roll(v0, 7 * layer, axis=0)
+
+    active = np.zeros(B, np.uint8)
+    seeds = np.zeros(B, np.uint64)
+    for i, (s, c) in enumerate(zip(slots, ctx)):
+        s, c = int(s), int(c)
+        eng.adopt(s, 0, c + 2, pending=1 + i, temperature=T, top_p=P, step=1)
+        k0, v0 = synth.synthetic_kv(c, sh.kv_dim, kv_std, seed=9000 + i)
+        for layer in range(sh.n_layers):
+            k, v = layer_rows(k0, v0, layer)
+            eng.kv_write(s, layer, 0, np.ascontiguousarray(k), np.ascontiguousarray(v))
+        active[s] = 1
+        seeds[s] = synth.request_seed(i)
+    toks = eng.decode_step(active, seeds)
+    worst, n_gap = 0.0, 0
+    for i, (s, c) in enumerate(zip(slots, ctx)):
+        s, c = int(s), int(c)
+        cache = model.new_cache(c + 2)
+        k0, v0 = synth.synthetic_kv(c, sh.kv_dim, kv_std, seed=9000 + i)
+        for layer in range(sh.n_layers):
+            cache[0][layer, :c], cache[1][layer, :c] = layer_rows(k0, v0, layer)
+        ref = model.forward([1 + i], c, cache)
+        del cache
+        lg = eng.logits(s)
+        worst = max(worst, float(np.abs(lg - ref).max()))
+        assert toks[s] == orc.sample(lg, T, P, orc.variate_u24(int(seeds[s]), 1))[0]
+        if top2_gap(ref) > GAP:
+            n_gap += 1
+            assert int(np.argmax(lg)) == int(np.argmax(ref))
+    assert all(toks[s] == -1 for s in range(B) if not active[s])
+    print("qwen timed workload, 40 active rows: max |delta logit| = %.4g (%d rows with a top-2 gap > %.1f)" % (worst, n_gap, GAP))
+    assert worst <= TOL, worst
+    for s in slots:
+        eng.release(int(s))
 
 
 def test_batched_prefill_equals_isolated_prefill_at_full_size(qwen):
