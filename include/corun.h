@@ -209,64 +209,13 @@ int corun_engine_info(corun_engine *e, int32_t *B, int32_t *max_context, int32_t
 /* How corun_prefill_batch packs prompts: rows per prefill chunk, and the row granularity on which every
  * piece of a request starts (the query tile of the prefill attention kernel).  Either pointer may be NULL. */
 int corun_prefill_geometry(corun_engine *e, int32_t *chunk_rows, int32_t *tile_rows);
-/* Reads / writes n cached positions [pos0, pos0+n) of one layer as fp32 rows of
- * n_kv_heads*head_dim (host).  Writing beyond the current context length
- * extends it (up to reserve_len); values are rounded to the cache's fp16. */
-int corun_debug_kv_read(corun_engine *e, int32_t slot, int32_t layer, int32_t pos0, int32_t n, float *k, float *v);
-int corun_debug_kv_write(corun_engine *e, int32_t slot, int32_t layer, int32_t pos0, int32_t n, const float *k,
-                         const float *v);
-/* Occupies an empty slot without running a prefill: reserves pages, sets the
- * context length to n_ctx (cache contents undefined until written with
- * corun_debug_kv_write), the pending token and the sampling state. */
-int corun_debug_adopt(corun_engine *e, int32_t slot, int32_t n_ctx, int32_t reserve_len, int32_t pending_token,
-                      const corun_sampling *sampling, int32_t step);
-/* Bench set-up: fills cached positions [0, n_ctx) of every layer of an occupied slot
- * with seeded N(0, std^2) values generated on the device and sets its context length. */
-int corun_debug_kv_fill(corun_engine *e, int32_t slot, int32_t n_ctx, float std, uint64_t seed);
-/* Times one kernel kind of the decode program in isolation, on the engine's stream,
- * with CUDA events: `reps` launches rotating over the layers' weights (so that L2
- * cannot hold them), after a short warm-up; *avg_ms = mean duration of one launch.
- * kind: 0 QKV GEMM, 1 O GEMM, 2 gate-up GEMM, 3 down GEMM, 4 LM-head GEMM (+ partial
- * fix-up), 5 attention (split + combine), 6 residual + RMSNorm, 7 RoPE + KV append,
- * 8 SwiGLU, 9 sampler.  Uses the rows of the last decode step; overwrites
- * intermediate buffers (not the cache beyond each active slot's next position). */
-int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *avg_ms);
-/* Runs GEMM `kind` (0 QKV, 1 O, 2 gate-up, 3 down, 4 LM head) of the decode program on one layer's
- * weights three times and returns the last launch's per-CTA timeline: stamps[cta*8 + i] (host, room for
- * 8 * 256 values) are globaltimer nanoseconds at: 0 kernel entry, 1 set-up done, 2 first TMA issued,
- * 3 last TMA issued, 4 first stage landed, 5 last MMA issued, 6 last accumulator complete, 7 epilogue done. */
-int corun_debug_gemm_trace(corun_engine *e, int32_t kind, int32_t layer, uint64_t *stamps, int32_t *n_ctas);
-/* With CORUN_TRACE_STEP=1 in the environment at corun_init, every layer GEMM of the decode program records
- * its per-CTA timeline (the 8 stamps of corun_debug_gemm_trace) on every step; this copies the last step's
- * stamps, [4 * n_layers][n_sms][8] values (n must equal that count), to the host. */
-int corun_debug_step_trace(corun_engine *e, uint64_t *stamps, int64_t n);
-/* Runs the attention of one layer twice on the rows of the last decode step and returns the second launch's
- * timeline: stamps[(cta*64 + k)*4 + i] (host, room for 256*64*4 values), globaltimer ns of the CTA's k-th item
- * (k < 64): 0 load issued, 1 item landed (seen by its consumer group), 2 the group starts on it, 3 released. */
-int corun_debug_attn_trace(corun_engine *e, int32_t layer, uint64_t *stamps, int32_t *n_ctas);
-/* Copies the first n floats of an intermediate buffer of the decode program to the host, as left by
- * the last decode step: which = 0 rotated queries [B, nq*hd]; 1 attention split partials
- * [B][nq][max_splits][hd]; 2 their (max, sum) pairs [B][nq][max_splits][2] (base-2 domain);
- * 3 the residual stream [B, hidden]; 4 / 5 the attention output's bf16 hi / lo halves [BN, nq*hd] as raw
- * memory (two bf16 per float); 6 the O-projection's direct output [B, hidden]; 7 the GEMM partial workspace. */
-int corun_debug_read(corun_engine *e, int32_t which, float *out, int64_t n);
-/* eager != 0: launch the decode kernels one by one instead of replaying the graph. */
-int corun_debug_set_eager(corun_engine *e, int32_t eager);
 /* Number of kernel launches in one decode iteration. */
 int corun_decode_launches(corun_engine *e);
-/* Stand-alone run of the decode GEMM: out[r, n] = sum_k W[n, k] * X[r, k] with X
- * fp32 [R, K] (device), W bf16 [N, K] (device), out fp32 [R, N] (device); R <= 256,
- * K % 64 == 0.  Uses the engine-independent kernel path (split activations,
- * tcgen05 MMA, fixed K order). */
-int corun_debug_gemm(const void *W, int32_t N, int32_t K, const float *X, int32_t R, float *out, void *cuda_stream);
-/* R(seed, t) as the engine computes it (top 24 bits of the first Philox word), on the device. */
-int corun_debug_variate(uint64_t seed, uint64_t t, uint32_t *out_u24 /* host */);
-/* Runs the engine's sampler on host logits rows [n_rows, vocab] (copied to the device). */
-int corun_debug_sample(const float *logits, int32_t n_rows, int32_t vocab, const corun_sampling *sampling,
-                       const uint32_t *u24, int32_t *out_tokens);
+/* Test and measurement accessors (cache read / write, adopting a slot without a prefill, eager launches,
+ * per-kernel timing, the stand-alone GEMM and sampler, kernel timelines) are declared in corun_debug.h. */
 
 /*
- * corun_gemm_static -- corun_debug_gemm for callers that cannot allocate.
+ * corun_gemm_static -- the stand-alone GEMM (corun_debug_gemm of corun_debug.h) for callers that cannot allocate.
  * (The paper has no counterpart; this is a service entry point of the library.)
  *
  * Same operation and argument meaning as corun_debug_gemm:
@@ -285,12 +234,19 @@ int corun_debug_sample(const float *logits, int32_t n_rows, int32_t vocab, const
  * call returns CORUN_ELIMIT and does nothing.  The call makes no cudaMalloc,
  * cudaFree or any other allocating call.
  *
+ * `out` and `W` must start on a 16-byte boundary (the kernels store and load
+ * 16 bytes at a time), `X` on a 4-byte one; otherwise CORUN_EINVAL, before
+ * anything is launched.
+ *
  * The first call on each device resolves the array's device address and sets a
- * kernel attribute; make that first call outside any stream capture.  All calls
- * share the one array, which keeps the previous call's contents (the call clears
- * the parts that must start at zero): two calls that overlap on the GPU -- from
- * two threads, or on two streams -- race on it.  The call is synchronous on
- * `cuda_stream`.  Errors: EINVAL, ELIMIT, ECUDA, ETIMEOUT.
+ * kernel attribute (safe from several host threads); that first call should come
+ * before any stream capture.  Every call is synchronous on `cuda_stream`: it ends
+ * with a stream synchronisation and a copy of the kernel's status word to the
+ * host, so a call made while `cuda_stream` is capturing is refused with
+ * CORUN_EINVAL.  All calls share the one array, which keeps the previous call's
+ * contents (the call clears the parts that must start at zero): two calls that
+ * overlap on the GPU -- from two threads, or on two streams -- race on it.
+ * Errors: EINVAL, ELIMIT, ECUDA, ETIMEOUT.
  */
 #define CORUN_STATIC_MAX_ROWS 16
 #define CORUN_STATIC_MAX_K 4096

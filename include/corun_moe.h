@@ -66,7 +66,8 @@ int corun_moe_create(const corun_moe_shape *shape, const void *router, const voi
 void corun_moe_destroy(corun_moe *m);
 
 /*
- * y = MoE(x) for all B rows.  x, y: fp32 [B, H] (y may not alias x).  experts (int32 [B, top_k], by
+ * y = MoE(x) for all B rows.  x, y: fp32 [B, H] (y may not alias x; y must start on a 16-byte boundary, x on a
+ * 4-byte one: EINVAL otherwise, before anything is launched).  experts (int32 [B, top_k], by
  * descending probability) and probs (fp32 [B, top_k]) receive the routing when not NULL.
  * Asynchronous; corun_moe_sync waits and reports a device-side timeout (ETIMEOUT).
  */

@@ -95,8 +95,11 @@ int corun_sched_submit(corun_sched *s, const int32_t *prompt, int32_t n, int32_t
 
 /* One scheduling decision (see above).  *action: CORUN_SCHED_*; *request_id: the prefilled request
  * (PREFILL; the first one of a batched prefill) else -1; *n_active: requests that took part (those
- * prefilled, the running count for a decode iteration, 0 when idle).  An engine error is returned as is and leaves the queues as they
- * were before the call. */
+ * prefilled, the running count for a decode iteration, 0 when idle).  An engine error is returned as is and
+ * leaves the queues as they were before the call.  One case ends a request without serving it: when nothing
+ * runs (so the whole pool is free) and the head of `waiting` still does not fit, it can never fit; the step
+ * then removes it, marks it finished with no tokens, sets *request_id to it and returns CORUN_ENOSPACE (action
+ * IDLE), so that the requests behind it are not blocked for good. */
 int corun_sched_step(corun_sched *s, int32_t *action, int64_t *request_id, int32_t *n_active);
 
 /* Tokens produced so far by a request (at most cap are copied; *n_tokens is the full count) and

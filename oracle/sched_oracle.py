@@ -55,6 +55,7 @@ class Scheduler:
         self.running: list[Request] = []
         self.waiting: list[Request] = []
         self.finished: list[int] = []
+        self.failed: list[int] = []      # requests dropped because they can never fit the pool
         self._next = 0
 
     # ------------------------------------------------------------------ requests
@@ -68,16 +69,19 @@ class Scheduler:
         need = -(-(r.num_prompt_tokens + r.max_new) // self.kv_block)
         return need <= self.free_pages
 
-    # ------------------------------------------------------------------ Algorithm 1
-    def find_prefill_request(self):
-        if self.running:
-            head = self.running[0]
-            if head.num_computed_tokens < head.num_prompt_tokens:
-                return head                                   # continue chunked prefill
-        if self.waiting and len(self.running) < self.max_num_reqs:
-            head = self.waiting[0]                            # peek_request
-            if self.can_fit_full_sequence(head):
-                return head
+    # ------------------------------------------------------------------ which request gets an isolated prefill
+    def isolated_prefill_candidate(self):
+        """The paper's selection rule (Algorithm 1), from its prose: a request whose prompt is only partly
+        computed is finished first (it can only be the one at the front of `running`, where the previous
+        isolated prefill put it); otherwise the oldest waiting request is taken, provided the number of running
+        requests is below the limit and the pool can hold its whole configured sequence.  None: no isolated
+        prefill in this iteration."""
+        partly = [r for r in self.running[:1] if r.num_computed_tokens < r.num_prompt_tokens]
+        if partly:
+            return partly[0]
+        has_slot = len(self.running) < self.max_num_reqs
+        if self.waiting and has_slot and self.can_fit_full_sequence(self.waiting[0]):
+            return self.waiting[0]
         return None
 
     # ------------------------------------------------------------------ the wrapped scheduler
@@ -118,26 +122,32 @@ class Scheduler:
                 self.free_pages += r.pages
                 self.finished.append(r.rid)
 
-    # ------------------------------------------------------------------ Algorithm 2
+    # ------------------------------------------------------------------ one iteration with the isolation wrapper
     def schedule(self) -> Iteration:
-        det = self.find_prefill_request()
-        if det is None:
+        """The paper's wrapper (Algorithm 2), from its prose: when a request was selected, the wrapped scheduler
+        runs on a view of the queues that holds nothing but that request -- so it cannot batch anything with it
+        -- and afterwards everything that was hidden is put back behind it in the order it had: the rest of
+        `running` behind the request (which now runs), the rest of `waiting` untouched.  Without a selected
+        request the wrapped scheduler sees the real queues (an ordinary decode iteration)."""
+        chosen = self.isolated_prefill_candidate()
+        if chosen is None:
+            if not self.running and self.waiting:
+                # nothing runs, the pool is all free, and the oldest request still does not fit: it never will;
+                # it is dropped (reported as finished without tokens) so that the queue behind it can move
+                dead = self.waiting.pop(0)
+                self.finished.append(dead.rid)
+                self.failed.append(dead.rid)
+                return Iteration("idle", [dead.rid])
             return self.schedule_origin()
-        stashed_running = list(self.running)
-        stashed_waiting = list(self.waiting)
-        self.waiting.clear()
-        if det in self.running:
-            self.running = [det]
-            stashed_running.remove(det)
-        else:
-            self.running = []
-            self.waiting.append(det)
-            stashed_waiting.remove(det)
-        output = self.schedule_origin()
-        self.running = self.running + stashed_running
-        for request in stashed_waiting:
-            self.waiting.append(request)
-        return output
+        was_running = any(r is chosen for r in self.running)
+        hidden_running = [r for r in self.running if r is not chosen]
+        hidden_waiting = [r for r in self.waiting if r is not chosen]
+        self.running = [chosen] if was_running else []
+        self.waiting = [] if was_running else [chosen]
+        result = self.schedule_origin()
+        self.running = self.running + hidden_running
+        self.waiting = self.waiting + hidden_waiting
+        return result
 
     # ------------------------------------------------------------------ one decision of the collapsed form
     def decision(self) -> Iteration:
@@ -191,7 +201,7 @@ class BatchedScheduler(Scheduler):
         self.tile = tile
 
     def decision(self) -> Iteration:
-        det = self.find_prefill_request()
+        det = self.isolated_prefill_candidate()
         if det is None or det in self.running:
             return super().decision()
         n = fill_batch([(r.num_prompt_tokens, r.max_new) for r in self.waiting], len(self.running), self.max_num_reqs,

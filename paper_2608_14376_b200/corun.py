@@ -20,14 +20,24 @@ EXPORTS = [
     "corun_init", "corun_init_moe", "corun_prefill", "corun_prefill_batch", "corun_decode_step", "corun_decode_enqueue", "corun_decode_wait",
     "corun_release", "corun_destroy", "corun_get_logits", "corun_force_token", "corun_context_len",
     "corun_free_blocks", "corun_debug_kv_read", "corun_debug_kv_write", "corun_debug_adopt",
-    "corun_debug_set_eager", "corun_debug_read", "corun_debug_gemm_trace", "corun_debug_attn_trace", "corun_debug_step_trace", "corun_debug_kv_fill", "corun_debug_time_kernel", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
-    "corun_debug_sample", "corun_gemm_static", "corun_strerror", "corun_last_cuda_error", "corun_engine_info",
+    "corun_debug_set_eager", "corun_debug_read", "corun_debug_kv_fill", "corun_debug_time_kernel", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
+    "corun_debug_sample", "corun_debug_wait_probe", "corun_debug_check_index", "corun_gemm_static", "corun_strerror", "corun_last_cuda_error", "corun_engine_info",
     "corun_sched_create", "corun_sched_create_for_engine", "corun_sched_destroy", "corun_sched_submit",
     "corun_sched_step", "corun_sched_poll", "corun_sched_slot_of", "corun_sched_counts",
     "corun_sched_enable_batched_prefill", "corun_prefill_geometry",
     "corun_moe_create", "corun_moe_destroy", "corun_moe_forward", "corun_moe_sync", "corun_moe_weight_bytes",
     "corun_moe_launches", "corun_mla_attend", "corun_mla_workspace_floats",
 ]
+
+
+# kernel timelines: present only in a library built with CORUN_BUILD_DEBUG=1 (include/corun_debug.h)
+DEBUG_EXPORTS = ["corun_debug_gemm_trace", "corun_debug_attn_trace", "corun_debug_step_trace"]
+
+
+def _need_debug_build():
+    if not hasattr(lib(), "corun_debug_step_trace"):
+        raise RuntimeError("kernel timelines need a library built with CORUN_BUILD_DEBUG=1 "
+                           "(CORUN_BUILD_DEBUG=1 python -m paper_2608_14376_b200.build --force)")
 
 
 class MoeShape(C.Structure):
@@ -117,9 +127,10 @@ def lib():
         L.corun_debug_adopt.argtypes = [vp, i32, i32, i32, i32, C.POINTER(Sampling), i32]
         L.corun_debug_set_eager.argtypes = [vp, i32]
         L.corun_debug_read.argtypes = [vp, i32, vp, i64]
-        L.corun_debug_gemm_trace.argtypes = [vp, i32, i32, vp, C.POINTER(i32)]
-        L.corun_debug_attn_trace.argtypes = [vp, i32, vp, C.POINTER(i32)]
-        L.corun_debug_step_trace.argtypes = [vp, vp, i64]
+        if hasattr(L, "corun_debug_step_trace"):              # a library built with CORUN_BUILD_DEBUG=1
+            L.corun_debug_gemm_trace.argtypes = [vp, i32, i32, vp, C.POINTER(i32)]
+            L.corun_debug_attn_trace.argtypes = [vp, i32, vp, C.POINTER(i32)]
+            L.corun_debug_step_trace.argtypes = [vp, vp, i64]
         L.corun_debug_kv_fill.argtypes = [vp, i32, i32, C.c_float, u64]
         L.corun_debug_time_kernel.argtypes = [vp, i32, i32, C.POINTER(C.c_float)]
         L.corun_decode_launches.argtypes = [vp]
@@ -324,6 +335,7 @@ class Engine:
         """Per-CTA timeline [n_ctas, 8] (ns, relative to the earliest kernel entry) of one GEMM launch."""
         st = np.zeros(8 * 256, np.uint64)
         n = C.c_int32(0)
+        _need_debug_build()
         _check(lib().corun_debug_gemm_trace(self._h, kind, layer, st.ctypes.data, C.byref(n)), "gemm_trace")
         t = st[:8 * n.value].reshape(n.value, 8).astype(np.int64)
         return t - t[:, 0].min()
@@ -332,6 +344,7 @@ class Engine:
         """GEMM timelines of the last decode step, [4 * n_layers, n_sms, 8] ns (engine made with CORUN_TRACE_STEP=1)."""
         n = 4 * self._cs.n_layers * n_sms * 8
         st = np.zeros(n, np.uint64)
+        _need_debug_build()
         _check(lib().corun_debug_step_trace(self._h, st.ctypes.data, n), "step_trace")
         return st.reshape(4 * self._cs.n_layers, n_sms, 8).astype(np.int64)
 
@@ -339,6 +352,7 @@ class Engine:
         """Per-CTA, per-item attention timeline [n_ctas, 64, 8] in ns (0 where an item does not exist)."""
         st = np.zeros(256 * 64 * 8, np.uint64)
         n = C.c_int32(0)
+        _need_debug_build()
         _check(lib().corun_debug_attn_trace(self._h, layer, st.ctypes.data, C.byref(n)), "attn_trace")
         return st[:n.value * 512].reshape(n.value, 64, 8).astype(np.int64)
 

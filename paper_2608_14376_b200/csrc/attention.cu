@@ -31,6 +31,7 @@
 #include <cuda_fp16.h>
 #include <math_constants.h>
 
+#include "checks.cuh"
 #include "launch.cuh"
 #include "ops.cuh"
 #include "ptx.cuh"
@@ -307,7 +308,13 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       const int ctx = rows.pos[r] + 1;
       const int t0 = split * ATT_SPLIT;
       const int n_pages = min(ATT_PAGES, (ctx - t0 + KV_BLOCK - 1) / KV_BLOCK);
-      const int page = lane < n_pages ? kv.block_table[(size_t)rows.slot[r] * kv.max_blocks + t0 / KV_BLOCK + lane] : 0;
+      int page = lane < n_pages ? kv.block_table[(size_t)rows.slot[r] * kv.max_blocks + t0 / KV_BLOCK + lane] : 0;
+#ifdef CORUN_CHECKED
+      if (!check_item(r, rows.R, g, kv.n_kv, split, ctx, ATT_SPLIT) || !check_page(page, kv.pool_blocks)) {
+        atomicCAS(status, 0, DEV_BAD_INDEX);       // the load goes to the reserved page 0 instead: nothing faults
+        page = 0;
+      }
+#endif
       if (k >= ATT_NBUF) {                               // the buffer's previous item must have been released
         bool ok = mbar_wait(smem_u32(&empty[buf]), (uint32_t)(k / ATT_NBUF - 1) & 1u, &abort_flag);
         ok = __all_sync(0xffffffffu, ok);
@@ -600,9 +607,11 @@ template <int HD, int GROUP>
 cudaError_t prepare_one() {
   cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<HD, GROUP, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)AttLayout<HD>::SMEM);
+#ifdef CORUN_BUILD_DEBUG
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(attn_split_kernel<HD, GROUP, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)AttLayout<HD>::SMEM);
+#endif
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(attn_split_kernel<HD, GROUP, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)AttLayout<HD>::SMEM);
@@ -613,14 +622,20 @@ cudaError_t launch_attn_split(int group, int grid, cudaStream_t st, const CUtens
                          const float *q, const Rows &rows, int nq, const KvLayout &kv, int max_splits, const int *work,
                          const int *n_work, float *part_acc, float *part_ml, int *pool_count, int whole_pairs,
                          int *d_status, unsigned long long *trace) {
+#ifdef CORUN_BUILD_DEBUG   // the stamped instantiation exists in debug builds only
+#define CORUN_ATT_TRACED(G)                                                                                        \
+    if (trace)                                                                                                     \
+      return launch_k(attn_split_kernel<HD, G, false, true>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
+                      rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, pool_count, d_status, trace);
+#else
+#define CORUN_ATT_TRACED(G)
+#endif
 #define CORUN_ATT_CASE(G)                                                                                          \
   case G:                                                                                                          \
     if (whole_pairs)                                                                                               \
       return launch_k(attn_split_kernel<HD, G, true, false>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
                       rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, pool_count, d_status, trace); \
-    if (trace)                                                                                                     \
-      return launch_k(attn_split_kernel<HD, G, false, true>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
-                      rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, pool_count, d_status, trace); \
+    CORUN_ATT_TRACED(G)                                                                                            \
     return launch_k(attn_split_kernel<HD, G, false, false>, dim3(grid), dim3(ATT_THREADS), AttLayout<HD>::SMEM, st, true, tmK, tmV, q, \
                     rows, nq, kv, max_splits, work, n_work, part_acc, part_ml, pool_count, d_status, trace);
   switch (group) {
@@ -631,6 +646,7 @@ cudaError_t launch_attn_split(int group, int grid, cudaStream_t st, const CUtens
     default: return cudaErrorInvalidValue;
   }
 #undef CORUN_ATT_CASE
+#undef CORUN_ATT_TRACED
 }
 }  // namespace
 

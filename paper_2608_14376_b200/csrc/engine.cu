@@ -11,6 +11,7 @@
 #include <vector>
 
 #include "../../include/corun.h"
+#include "../../include/corun_debug.h"
 #include "gemm.cuh"
 #include "moe.cuh"
 #include "ops.cuh"
@@ -238,7 +239,7 @@ void program_destroy(Program &P) {
 
 KvLayout kv_layout(const corun_engine *e) {
   return KvLayout{e->kv_pool, e->d_block_table, e->max_blocks, e->sh.n_kv_heads, e->sh.head_dim, e->layer_stride,
-                  (long long)e->pool_blocks};
+                  (long long)e->pool_blocks, e->B};
 }
 
 // The result of a layer's feed-forward part as the next kernel reads it: the down GEMM's partials, or (grouped
@@ -275,7 +276,7 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
     STAGE(launch_resid_norm(P.h, s.hidden, e->embed, rows, l == 0 ? nullptr : &prev, e->attn_norm[l], s.rms_eps,
                             P.xn_hi, P.xn_lo, e->st));
     STAGE(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, tr(4 * l + 0), true));
-    STAGE(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st));
+    STAGE(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->d_status, e->st));
     STAGE(launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work, P.att_n_work,
                            e->num_sms, P.part_acc, P.part_ml, P.att_pool + l, P.ao_hi, P.ao_lo, &P == &e->dec ? (e->whole_pairs ? 2 : 0) : 1,
                            e->d_status, e->st));
@@ -350,6 +351,7 @@ int enqueue_decode_body(corun_engine *e, int *launches) {
 }
 
 int check_status(corun_engine *e) {
+  if (*e->h_status == 4) return CORUN_EINVAL;   // DEV_BAD_INDEX: an index check of a -DCORUN_CHECKED build failed
   if (*e->h_status != 0) return CORUN_ETIMEOUT;
   return CORUN_OK;
 }
@@ -581,9 +583,11 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
   memset(e->h_seeds, 0, B * sizeof(uint64_t));
   *e->h_status = 0;
 
+#ifdef CORUN_BUILD_DEBUG
   if (const char *ts = getenv("CORUN_TRACE_STEP")) {
     if (atoi(ts) != 0 && (rc = dmalloc(A, &e->step_trace, (size_t)4 * s.n_layers * e->num_sms * 8))) return fail(rc);
   }
+#endif
   if ((rc = program_create(e, e->dec, B, true, true, false, true))) return fail(rc);
   if ((rc = program_create(e, e->pre, e->chunk, true, false, e->moe_E > 0 && !getenv("CORUN_MOE_PREFILL_DENSE")))) return fail(rc);
   if ((rc = program_create(e, e->lm1, 1, false, true))) return fail(rc);
@@ -1011,7 +1015,7 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
                 break;
         case 6: ce = launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->attn_norm[l], s.rms_eps, P.xn_hi,
                                        P.xn_lo, e->st); break;
-        case 7: ce = launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->st); break;
+        case 7: ce = launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->d_status, e->st); break;
         case 8: if (P.p_gu.sw_hi) break;             // no such kernel: the SwiGLU is in the GEMM's epilogue
                 ce = e->moe_E ? launch_moe_swiglu(P.p_gu.out(), P.moe_w, P.R, e->moe_F, e->moe_E + e->moe_S, P.ff_hi, P.ff_lo, e->st)
                               : launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st);
@@ -1035,6 +1039,7 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
   return rc;
 }
 
+#ifdef CORUN_BUILD_DEBUG   // kernel timelines: not part of the serving build
 int corun_debug_gemm_trace(corun_engine *e, int32_t kind, int32_t layer, uint64_t *stamps, int32_t *n_ctas) {
   if (!e || !stamps || !n_ctas || kind < 0 || kind > 4 || layer < 0 || layer >= e->sh.n_layers) return CORUN_EINVAL;
   RC(sync_stream(e));
@@ -1092,6 +1097,8 @@ int corun_debug_step_trace(corun_engine *e, uint64_t *stamps, int64_t n) {
   return CORUN_OK;
 }
 
+#endif  // CORUN_BUILD_DEBUG
+
 int corun_debug_read(corun_engine *e, int32_t which, float *out, int64_t n) {
   if (!e || !out || n < 0) return CORUN_EINVAL;
   RC(sync_stream(e));
@@ -1129,6 +1136,8 @@ int corun_decode_launches(corun_engine *e) { return e ? e->decode_launches : COR
 
 int corun_debug_gemm(const void *W, int32_t N, int32_t K, const float *X, int32_t R, float *out, void *cuda_stream) {
   if (!W || !X || !out || N < 1 || K < 64 || K % 64 || R < 1 || R > 256) return CORUN_EINVAL;
+  // 16-byte stores of the output, tensor-map loads of W: misaligned buffers are refused before any launch
+  if (((uintptr_t)out & 15u) || ((uintptr_t)W & 15u) || ((uintptr_t)X & 3u)) return CORUN_EINVAL;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   int dev = 0, sms = 0;
   CK(cudaGetDevice(&dev));

@@ -475,10 +475,6 @@ int gemm_plan_fill(GemmPlan *p, const void *W, int N, int K, const void *Xhi, co
   // the MMA always reads 128 activation rows: leave that much readable behind the last stage
   int stages = (int)((GEMM_MAX_DYN_SMEM - 1024 - A_BLOCK_BYTES) / stage);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
-  if (const char *ev = getenv("CORUN_GEMM_STAGES")) {   // experiments only: shallower ring
-    const int v = atoi(ev);
-    if (v >= 2 && v < stages) stages = v;
-  }
   if (stages < 2) return CORUN_EINVAL;
   p->stages = stages;
   p->smem_bytes = stage * stages + A_BLOCK_BYTES + 1024;

@@ -419,6 +419,7 @@ void corun_moe_destroy(corun_moe *m) {
 
 int corun_moe_forward(corun_moe *m, const float *x, float *y, int32_t *experts, float *probs) {
   if (!m || !x || !y || x == y) return CORUN_EINVAL;
+  if (((uintptr_t)y & 15u) || ((uintptr_t)x & 3u)) return CORUN_EINVAL;   // y is stored 16 bytes at a time
   const corun_moe_shape &s = m->sh;
   const int H = s.hidden, E = s.n_experts, F = s.expert_ffn, NB = E + s.n_shared;
   MCK(launch_split(x, m->B, H, m->x_hi, m->x_lo, m->st));

@@ -11,6 +11,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "../../include/corun.h"
 #include "gemm.cuh"
 #include "ops.cuh"
@@ -42,7 +44,10 @@ constexpr size_t NA_BYTES = NA_OFF_STATUS + 256;
 static __device__ __align__(256) unsigned char g_static_scratch[NA_BYTES];
 
 constexpr int NA_MAX_DEVICES = 64;
-unsigned char *g_scratch_addr[NA_MAX_DEVICES] = {nullptr};
+// Per-device cache of the set-up.  The address is published last (release) and read first (acquire), so a
+// thread that sees it also sees the SM count written before it; two threads that both find it empty do the
+// same idempotent set-up and store the same values.
+std::atomic<unsigned char *> g_scratch_addr[NA_MAX_DEVICES];
 int g_num_sms[NA_MAX_DEVICES] = {0};
 
 // One-time set-up per device (the device must be current): resolves the
@@ -50,7 +55,8 @@ int g_num_sms[NA_MAX_DEVICES] = {0};
 // shared-memory size.  Allocates nothing.
 int static_setup(int dev, unsigned char **base, int *sms) {
   if (dev < 0 || dev >= NA_MAX_DEVICES) return CORUN_EINVAL;
-  if (!g_scratch_addr[dev]) {
+  unsigned char *cached = g_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!cached) {
     void *p = nullptr;
     cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
     if (e != cudaSuccess || !p) { g_last_cuda_error = (int)e; return CORUN_ECUDA; }
@@ -58,12 +64,14 @@ int static_setup(int dev, unsigned char **base, int *sms) {
     e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
     if (e == cudaSuccess) e = gemm_prepare_kernel();
     if (e != cudaSuccess) { g_last_cuda_error = (int)e; return CORUN_ECUDA; }
+    if (n < 1) return CORUN_ECUDA;
     g_num_sms[dev] = n;
-    g_scratch_addr[dev] = (unsigned char *)p;
+    cached = (unsigned char *)p;
+    g_scratch_addr[dev].store(cached, std::memory_order_release);
   }
-  *base = g_scratch_addr[dev];
+  *base = cached;
   *sms = g_num_sms[dev];
-  return CORUN_OK;
+  return *sms >= 1 ? CORUN_OK : CORUN_ECUDA;
 }
 
 }  // namespace
@@ -71,8 +79,17 @@ int static_setup(int dev, unsigned char **base, int *sms) {
 extern "C" int corun_gemm_static(const void *W, int32_t N, int32_t K, const float *X, int32_t R, float *out,
                                  void *cuda_stream) {
   if (!W || !X || !out || N < 1 || K < 64 || K % 64 || R < 1) return CORUN_EINVAL;
+  // the kernels store the output 16 bytes at a time and read W through a tensor map: a buffer that starts
+  // elsewhere (a view into an arena, say) would fault on the device, so it is refused here, before any launch
+  if (((uintptr_t)out & 15u) || ((uintptr_t)W & 15u) || ((uintptr_t)X & 3u)) return CORUN_EINVAL;
   if (R > NA_MAX_R || K > NA_MAX_K || N > NA_MAX_N) return CORUN_ELIMIT;
   cudaStream_t st = (cudaStream_t)cuda_stream;
+  {
+    // every call ends with a stream synchronisation and a copy of the status word to the host, neither of which
+    // a capturing stream permits: refuse instead of breaking the caller's capture
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) == cudaSuccess && cs != cudaStreamCaptureStatusNone) return CORUN_EINVAL;
+  }
   int dev = 0;
   cudaError_t ce = cudaGetDevice(&dev);
   if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return CORUN_ECUDA; }

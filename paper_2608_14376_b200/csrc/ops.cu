@@ -4,6 +4,7 @@
 // that depends on the row's own data and the model shape only; no float atomics.
 #include "ops.cuh"
 
+#include "checks.cuh"
 #include "launch.cuh"
 #include "ptx.cuh"
 
@@ -85,7 +86,7 @@ resid_norm_kernel(float *__restrict__ h, int H, const __nv_bfloat16 *__restrict_
 // One CTA per (head, row): heads 0..nq-1 are q, nq..nq+nkv-1 are k, the rest are v; hd/2 threads.
 __global__ void __launch_bounds__(64)
 qkv_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, int nq, KvLayout kv, int layer,
-                float *__restrict__ q_out) {
+                float *__restrict__ q_out, int *status) {
   griddep_launch_dependents();
   griddep_wait();
   const int head = blockIdx.x, r = blockIdx.y, i = threadIdx.x;
@@ -102,7 +103,19 @@ qkv_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, int
     q[half] = a * t.y + b * t.x;
     return;
   }
+#ifdef CORUN_CHECKED
+  if (!check_slot_pos(rows.slot[r], kv.n_slots, pos, kv.max_blocks, KV_BLOCK)) {   // the write is skipped
+    atomicCAS(status, 0, DEV_BAD_INDEX);
+    return;
+  }
+#endif
   const int blk = kv.block_table[(size_t)rows.slot[r] * kv.max_blocks + pos / KV_BLOCK];
+#ifdef CORUN_CHECKED
+  if (!check_page(blk, kv.pool_blocks)) {
+    atomicCAS(status, 0, DEV_BAD_INDEX);
+    return;
+  }
+#endif
   __half *page = kv.pool + (size_t)layer * kv.layer_stride + (size_t)blk * 2 * nkv * KV_BLOCK * hd;
   const int tok = pos % KV_BLOCK;
   if (head < nq + nkv) {
@@ -805,9 +818,9 @@ cudaError_t launch_resid_norm(float *h, int H, const __nv_bfloat16 *embed, const
 }
 
 cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *rope_tab, int nq, const KvLayout &kv,
-                            int layer, float *q_out, cudaStream_t st) {
+                            int layer, float *q_out, int *d_status, cudaStream_t st) {
   return launch_k(qkv_post_kernel, dim3(nq + 2 * kv.n_kv, rows.R), dim3(kv.hd / 2), 0, st, true, qkv, rows, rope_tab, nq,
-                  kv, layer, q_out);
+                  kv, layer, q_out, d_status);
 }
 
 cudaError_t launch_swiglu(const GemmOut &gu, int R, int F, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, cudaStream_t st) {

@@ -39,6 +39,7 @@ struct KvLayout {
   int max_blocks, n_kv, hd;
   size_t layer_stride;     // halfs per layer
   long long pool_blocks;   // pages per layer
+  int n_slots;             // rows of the block table
 };
 
 struct SampleArgs {
@@ -59,7 +60,7 @@ cudaError_t launch_resid_norm(float *h, int H, const __nv_bfloat16 *embed, const
                               cudaStream_t st);
 // RoPE on q and k, q -> q_out fp32 [R, nq*hd], k/v -> pages (fp16) at the row's position.
 cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *rope_tab, int nq, const KvLayout &kv,
-                            int layer, float *q_out, cudaStream_t st);
+                            int layer, float *q_out, int *d_status, cudaStream_t st);
 // Split-KV paged attention partials and, in a second kernel, their fixed-order combine -> bf16 hi/lo
 // [R, nq*hd] (rows that are not active keep what they held).  pool_count: one int, zero before the launch (not reset by it): the items beyond the
 // CTAs' fixed stretches are drawn through it.  reuse: 1 when the rows are the consecutive tokens of one

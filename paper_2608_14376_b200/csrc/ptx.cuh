@@ -48,22 +48,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: gives up after ~2 s of wall time (or as soon as another role
+// Bounded wait: gives up after limit_ns of wall time (or as soon as another role
 // of the CTA has given up), sets *abort_flag and returns false.  The caller
 // then leaves its loop; the kernel records the failure and exits normally.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 0u) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > 2000000000ull) {
+      if (globaltimer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         return false;
       }
     }
   }
+}
+// The kernels' waits: ~2 s, far beyond anything a healthy launch needs.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+  return mbar_wait_limit(bar, parity, abort_flag, 2000000000ull);
 }
 
 // 2D tiled TMA load, global -> shared, completion on an mbarrier, with an L2 policy.

@@ -231,6 +231,14 @@ extern "C" int corun_sched_step(corun_sched *s, int32_t *action, int64_t *reques
       return admitted(s, id, slot, first);
     }
     if (status != CORUN_OK) return status;
+    if (s->running.empty()) {
+      // Nothing runs, so every page the pool has is free, and the head still does not fit: it never will.
+      // Left in place it would block the queue for good (nothing overtakes the head): the request fails.
+      s->waiting.pop_front();
+      r.finished = true;
+      *request_id = id;
+      return CORUN_ENOSPACE;
+    }
   }
   // ---- no prefill: a normal decode iteration over everything that runs
   if (s->running.empty()) return CORUN_OK;

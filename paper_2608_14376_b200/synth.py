@@ -3,7 +3,7 @@
 Holds none of the method's arithmetic.  Both the CUDA path's callers and the
 CPU oracle's callers take their inputs from here, as bytes.
 
-Recipe (BASELINE configs): every matrix (embedding, projections, LM head) is
+Recipe (the benchmark configurations): every matrix (embedding, projections, LM head) is
 N(0, 0.02) drawn in fp32 and rounded to bf16 (round to nearest even); RMSNorm
 gains are 1; prompts are i.i.d. uniform token ids; request seed = 1000 + index.
 Tensor draw order: embed, then per layer wqkv, wo, wgate_up, wdown, then lm_head.

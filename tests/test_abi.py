@@ -24,6 +24,8 @@ def _declared():
             continue
         src = open(os.path.join(inc, f)).read()
         src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+        # declarations that exist only in a library built with -DCORUN_BUILD_DEBUG (kernel timelines)
+        src = re.sub(r"#ifdef CORUN_BUILD_DEBUG.*?#endif", "", src, flags=re.S)
         names |= set(re.findall(r"\b(corun_[a-z_0-9]+)\s*\(", src))
     return sorted(names)
 
@@ -55,6 +57,22 @@ def test_argument_validation_needs_no_gpu(lib):
     assert lib.corun_prefill(None, 0, None, 0, 0, None, 0, None) == corun.EINVAL
     assert lib.corun_debug_gemm(None, 1, 64, None, 1, None, None) == corun.EINVAL
     lib.corun_destroy(None)
+
+
+def test_misaligned_buffers_are_refused_before_any_launch(lib):
+    """The raw-pointer entry points store their output 16 bytes at a time: a buffer that starts elsewhere must
+    come back as EINVAL from the argument checks (no CUDA call, so this runs without a GPU)."""
+    from paper_2608_14376_b200 import corun
+
+    base = 0x7F0000001000                     # never dereferenced: the checks come first
+    for fn in (lib.corun_debug_gemm, lib.corun_gemm_static):
+        fn.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+        for off in (4, 8, 12):
+            assert fn(base, 256, 64, base + 0x10000, 1, base + 0x20000 + off, None) == corun.EINVAL
+        assert fn(base + 8, 256, 64, base + 0x10000, 1, base + 0x20000, None) == corun.EINVAL
+        assert fn(base, 256, 64, base + 0x10002, 1, base + 0x20000, None) == corun.EINVAL
+    lib.corun_moe_forward.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    assert lib.corun_moe_forward(base, base + 0x10000, base + 0x20004, None, None) == corun.EINVAL
 
 
 def test_strerror_covers_every_status(lib):

@@ -123,3 +123,29 @@ def test_sampler_ties_and_degenerate_rows(orc, torch_cuda):
     # argmax picks the lowest id among equal maxima
     two = np.zeros(777, np.float32); two[[5, 300]] = 3.0
     assert corun.debug_sample(two, 0.0, 1.0, [0])[0] == 5
+
+
+def test_a_bounded_wait_runs_out_and_the_context_stays_usable(orc, torch_cuda):
+    """A one-CTA kernel waits, with the library's own wait routine and a limit of 1 ms, on a barrier nothing
+    arrives at: the wait gives up, the kernel returns normally with its status word set and the call reports
+    ETIMEOUT.  Nothing traps or faults, so an ordinary kernel launched afterwards works."""
+    import ctypes as C
+    import time
+
+    import torch
+    from paper_2608_14376_b200 import corun
+
+    L = corun.lib()
+    L.corun_debug_wait_probe.argtypes = [C.c_uint64, C.c_void_p]
+    t0 = time.perf_counter()
+    assert L.corun_debug_wait_probe(1_000_000, None) == corun.ETIMEOUT
+    assert time.perf_counter() - t0 < 2.0
+    assert L.corun_debug_wait_probe(10, None) == corun.EINVAL          # limits outside 1 us .. 100 ms are refused
+    assert L.corun_debug_wait_probe(10**10, None) == corun.EINVAL
+    # the device is fine: a GEMM against the oracle
+    rng = np.random.default_rng(1)
+    Wb = synth.f32_to_bf16_bits(rng.standard_normal((512, 256)).astype(np.float32) * 0.02)
+    X = rng.standard_normal((3, 256)).astype(np.float32)
+    Wt = torch.from_numpy(Wb.view(np.int16).copy()).view(torch.bfloat16).cuda()
+    got = corun.debug_gemm(Wt, torch.from_numpy(X).cuda()).cpu().numpy()
+    assert np.abs(got - orc.matmul_bf16(Wb, X)).max() < 1e-4

@@ -241,6 +241,48 @@ def test_library_scheduler_argument_and_engine_errors():
         sch.close()
 
 
+def test_a_request_that_can_never_fit_is_failed_and_the_queue_moves_on():
+    """The pool holds 8 pages.  A request of 9 pages at the head of `waiting` can never be admitted: with
+    nothing running the whole pool is free already.  Oracle and library drop it (finished, no tokens,
+    ENOSPACE from the step) and serve the request behind it; while something runs the head only waits."""
+    from paper_2608_14376_b200 import build, corun
+
+    build.build()
+    B, kv_block, pool = 2, 16, 8
+    eng = _StandInEngine(B, pool, kv_block)
+    sch = corun.Scheduler(ops=eng.ops, B=B, kv_block=kv_block, max_context=256)
+    ref = sched_oracle.Scheduler(B, pool, kv_block, chunk=64)
+    try:
+        reqs = [(40, 3), (100, 40), (20, 2)]          # 3 pages, 9 pages (never fits), 2 pages
+        ids = [sch.submit(np.arange(p) % 97, m, 0.7, 0.9, seed=7000 + i) for i, (p, m) in enumerate(reqs)]
+        for p, m in reqs:
+            ref.add_request(p, m)
+        kinds, failed_at = [], None
+        for i in range(12):
+            want = ref.decision()
+            try:
+                action, rid, n = sch.step()
+                assert want.kind != "idle" or not want.requests
+                assert action == {"idle": corun.SCHED_IDLE, "prefill": corun.SCHED_PREFILL, "decode": corun.SCHED_DECODE}[want.kind]
+            except corun.CorunError as e:
+                assert e.status == corun.ENOSPACE and want.kind == "idle" and want.requests == [ids[1]]
+                failed_at = i
+            kinds.append(want.kind)
+            assert sch.counts() == (len(ref.waiting), len(ref.running))
+        # request 0 is served first (the big one waits behind it while it runs), then the big one is dropped,
+        # then request 2 is served
+        assert kinds[:3] == ["prefill", "decode", "decode"] and failed_at == 3 and kinds[4:6] == ["prefill", "decode"]
+        assert ref.failed == [ids[1]]
+        toks, fin = sch.poll(ids[1])
+        assert fin and len(toks) == 0
+        for i in (0, 2):
+            toks, fin = sch.poll(ids[i])
+            assert fin and len(toks) == reqs[i][1]
+        assert eng.free == pool
+    finally:
+        sch.close()
+
+
 # ------------------------------------------------------------------------------------------------ batched prefill
 def _batched_cases():
     cases, cur = [], None
