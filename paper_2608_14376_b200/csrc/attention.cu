@@ -6,9 +6,10 @@
 // time through a counter, so that CTAs that got through their stretch sooner take more of it (which CTA
 // computes an item has no influence on any value).  One persistent CTA per SM:
 //   warp 0        streams the items' keys with TMA into a ring of 3 key buffers ([16 tokens x 64 dims]
-//                 boxes, 128-byte swizzle), warp 1 their values into a ring of 3 value buffers (cached
-//                 transposed: [hd dims x 16 tokens] boxes, 32-byte swizzle), straight from the page pool
-//                 through two tensor maps per layer.  A key buffer is free again as soon as the scores
+//                 boxes, 128-byte swizzle), warp 1 their values into a ring of 3 value buffers (cached like
+//                 the keys and fetched through the same kind of box: rows of 128 bytes, which the TMA unit
+//                 moves four times as fast as the 32-byte rows of a transposed value tile), straight from
+//                 the page pool.  A key buffer is free again as soon as the scores
 //                 exist, a value buffer at the end of the item, so the key loads run ahead of the value
 //                 loads and more bytes are in flight than with whole-item buffers;
 //   2 groups of 4 warps take the items alternately.  Per item a group
@@ -18,7 +19,8 @@
 //        -> TMEM lane = token, so each of the 128 threads owns one cached token,
 //     3. softmax over the item: exact max and a fixed-order sum over the 128 tokens,
 //        weights written as fp16 hi/lo rows of a [16 x 128 tokens] operand tile,
-//     4. O^T[hd dims x 16] = V^T[hd x 128 tokens] * P^T  (one MMA per page), TMEM lane = dim,
+//     4. O^T[hd dims x 16] = V^T[hd x 128 tokens] * P^T  (one MMA per page; the token-major value tile is
+//        its MN-major A operand), TMEM lane = dim,
 //     5. adds the hi and lo columns and writes the split's partial (max, sum, O) to global memory;
 // A second kernel, one warp per (row, query head), combines the splits' partials in ascending split order
 // (attn_combine_kernel): as a kernel of its own the combines all run at once, where combiner warps inside the
@@ -160,14 +162,14 @@ template <int HD>
 struct AttLayout {
   static constexpr int NHALF = HD / 64;                          // 64-dim halves of a key row
   static constexpr int K_BYTES = NHALF * ATT_PAGES * KBOX_BYTES; // keys of an item: [half][page][16 x 128 B]
-  static constexpr int VT_BYTES = HD * KV_BLOCK * 2;             // one page's V^T tile: [hd x 32 B]
-  static constexpr int V_BYTES = ATT_PAGES * VT_BYTES;           // values of an item
+  static constexpr int V_BYTES = K_BYTES;                        // values of an item: the same arrangement
   static constexpr int ITEM_BYTES = K_BYTES + V_BYTES;
   static constexpr int Q_BYTES = NHALF * OPND_BYTES;             // [half][16 x 128 B]
   static constexpr int P_BYTES = 2 * OPND_BYTES;                 // 128 tokens = 2 halves of 64
   static constexpr int GROUP_BYTES = Q_BYTES + P_BYTES;
-  // the value MMA always reads 128 rows of V^T (M = 128): with hd = 64 that runs into what follows
-  static constexpr int PAD_BYTES = (HD < 128) ? 128 * KV_BLOCK * 2 : 0;
+  // the value MMA always covers 128 dims (M = 128), i.e. two blocks of 64 dims one key-tile half apart: with
+  // hd = 64 the second one lies in whatever follows the value tile (never used; it must only be readable)
+  static constexpr int PAD_BYTES = (HD < 128) ? ATT_PAGES * KBOX_BYTES + KBOX_BYTES : 0;
   static constexpr size_t SMEM = (size_t)ATT_NBUF * ITEM_BYTES + ATT_GROUPS * GROUP_BYTES + PAD_BYTES + 1024;
 };
 
@@ -323,16 +325,18 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       const uint32_t fb = smem_u32(&full[slot]);
       if (lane == 0) {
         if (!is_v) ATRACE(k, 0);
-        mbar_arrive_expect_tx(fb, (uint32_t)(n_pages * (is_v ? L::VT_BYTES : L::NHALF * KBOX_BYTES)));
+        mbar_arrive_expect_tx(fb, (uint32_t)(n_pages * L::NHALF * KBOX_BYTES));
       }
       __syncwarp();
       if (lane < n_pages) {
         // this layer's pages as rows of hd halfs: the key tile of (page, head) starts at row
-        //   page * 2 * n_kv * 16 + head * 16;
-        // as rows of 16 halfs: the transposed value tile starts at row page * 2 * n_kv * hd + (n_kv + head) * hd
+        //   page * 2 * n_kv * 16 + head * 16, its value tile n_kv * 16 rows further on
         if (is_v) {
-          const int row_v = (page * 2 * kv.n_kv + kv.n_kv + g) * HD;
-          tma_load_2d(vring + (uint32_t)buf * L::V_BYTES + (uint32_t)lane * L::VT_BYTES, &tmV, 0, row_v, fb, pol);
+          const int row_v = (page * 2 * kv.n_kv + kv.n_kv + g) * KV_BLOCK;
+          const uint32_t vb = vring + (uint32_t)buf * L::V_BYTES;
+#pragma unroll
+          for (int x = 0; x < L::NHALF; ++x)
+            tma_load_2d(vb + (uint32_t)(x * ATT_PAGES + lane) * KBOX_BYTES, &tmV, x * 64, row_v, fb, pol);
         } else {
           const int row_k = (page * 2 * kv.n_kv + g) * KV_BLOCK;
           const uint32_t kb = ring + (uint32_t)buf * L::K_BYTES;
@@ -489,9 +493,11 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         ATRACE(k, 6);
         tc_fence_after();
         for (int p = 0; ok && p < n_pages; ++p) {
-          const uint64_t a = umma_desc_sw32(v_tiles + (uint32_t)p * L::VT_BYTES);
+          // A = V^T of the page: [128 dims x 16 tokens] read MN-major from the token-major tile (two blocks of
+          // 64 dims a key-tile half apart, two groups of 8 tokens 1 KiB apart)
+          const uint64_t a = umma_desc_sw128_mn(v_tiles + (uint32_t)p * KBOX_BYTES, ATT_PAGES * KBOX_BYTES, 1024u);
           const uint64_t b = umma_desc_sw128(p_tile + (uint32_t)(p >> 2) * OPND_BYTES) + (uint64_t)((p & 3) * 2);
-          umma_bf16(o_tmem, a, b, idesc, p > 0 ? 1u : 0u);
+          umma_bf16(o_tmem, a, b, idesc | (1u << 15), p > 0 ? 1u : 0u);
         }
         umma_commit(mbar);                           // also arrives if the wait gave up
       }

@@ -15,8 +15,8 @@
 // output; the keys come from L2 the second time.
 // S[128 rows x 128 keys] = Q[128 x hd] * K^T on tcgen05.mma (M = 128, N = 128, fp16, Q as a hi/lo pair: two
 // MMAs per k-slice), TMEM lane = row, so the softmax of a row is local to one thread; P goes to shared memory
-// as fp16 (its values lie in [0, 1]); O[128 x hd] += P[128 x 128] * V[128 x hd], one MMA per page from the
-// transposed value tiles.  Roles: warp 0 streams the key tiles and warp 10 the value tiles with TMA (a ring of
+// as fp16 (its values lie in [0, 1]); O[128 x hd] += P[128 x 128] * V[128 x hd], one MMA per page with the
+// token-major value tile as its MN-major B operand.  Roles: warp 0 streams the key tiles and warp 10 the value tiles with TMA (a ring of
 // two each), warp 1 issues the MMAs, warps 2-9 own the rows: two threads per row, one for
 // keys 0..63 and one for keys 64..127 of every block (two warps per scheduler hide each other's latencies);
 // the two exchange their maxima after pass 1 and their sums at the end.  The scores and the weights
@@ -60,9 +60,9 @@ struct PfLayout {
   static constexpr int Q_BYTES = NHALF * 128 * 128;           // one of hi / lo: [half][128 rows x 128 B]
   static constexpr int P_BYTES = 2 * 128 * 128;               // one weight tile: [key half][128 rows x 128 B]
   static constexpr int K_BYTES = NHALF * PF_PAGES * KV_BLOCK * 128;   // [half][page][16 x 128 B]
-  static constexpr int VT_BYTES = HD * KV_BLOCK * 2;          // one page: [hd x 32 B]
-  static constexpr int V_BYTES = PF_PAGES * VT_BYTES;
-  // the value MMA reads hd rows of V^T as its N operand; nothing runs past the tile
+  static constexpr int VT_BYTES = NHALF * KV_BLOCK * 128;     // one page's values
+  static constexpr int V_BYTES = PF_PAGES * VT_BYTES;         // [half][page][16 x 128 B], like the keys
+  // the value MMA reads hd dims of V as its N operand (MN-major); nothing runs past the tile
   static constexpr size_t SMEM = (size_t)2 * Q_BYTES + P_BYTES + PF_NK * K_BYTES + PF_NV * V_BYTES + 1024;
 };
 
@@ -152,7 +152,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const uint32_t s_tmem = tmem_base, o_tmem = tmem_base + 256;   // score buffer i at s_tmem + 128 i
   // fp16 x fp16 -> fp32, K-major operands; N at bit 17 (>> 3), M = 128 at bit 24 (>> 4)
   const uint32_t idesc_s = (1u << 4) | ((uint32_t)(PF_KEYS >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-  const uint32_t idesc_o = (1u << 4) | ((uint32_t)(HD >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+  const uint32_t idesc_o = (1u << 4) | (1u << 16) | ((uint32_t)(HD >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);   // B (values) MN-major
   bool failed = false;
 
   // pages of key block b that exist for this tile (the last block may be partial)
@@ -216,8 +216,11 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         if (lane == 0) mbar_arrive_expect_tx(fv, (uint32_t)(n_pages * L::VT_BYTES));
         __syncwarp();
         if (lane < n_pages) {
-          const int row_v = (page * 2 * kv.n_kv + kv.n_kv + g) * HD;
-          tma_load_2d(v_buf + (uint32_t)vbuf * L::V_BYTES + (uint32_t)lane * L::VT_BYTES, &tmV, 0, row_v, fv, pol);
+          const int row_v = (page * 2 * kv.n_kv + kv.n_kv + g) * KV_BLOCK;
+#pragma unroll
+          for (int x = 0; x < L::NHALF; ++x)
+            tma_load_2d(v_buf + (uint32_t)vbuf * L::V_BYTES + (uint32_t)(x * PF_PAGES + lane) * (KV_BLOCK * 128), &tmV, x * 64,
+                        row_v, fv, pol);
         }
       }
     }
@@ -232,7 +235,10 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const int n_pages = pages_of(blk(j));
         for (int p = 0; p < n_pages; ++p) {
           const uint64_t a = umma_desc_sw128(p_tile + (uint32_t)(p >> 2) * (128 * 128)) + (uint64_t)((p & 3) * 2);
-          const uint64_t bv = umma_desc_sw32(v_buf + (uint32_t)vbuf * L::V_BYTES + (uint32_t)p * L::VT_BYTES);
+          // B = the page's values [hd dims x 16 tokens], MN-major in the token-major tile: blocks of 64 dims a
+          // tile half apart, groups of 8 tokens 1 KiB apart
+          const uint64_t bv = umma_desc_sw128_mn(v_buf + (uint32_t)vbuf * L::V_BYTES + (uint32_t)p * (KV_BLOCK * 128),
+                                                 PF_PAGES * KV_BLOCK * 128, 1024u);
           umma_bf16(o_tmem, a, bv, idesc_o, (j > 0 || p > 0) ? 1u : 0u);
         }
         umma_commit(smem_u32(&vempty[vbuf]));       // the value buffer is free

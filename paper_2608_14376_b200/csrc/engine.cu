@@ -76,7 +76,7 @@ struct corun_engine {
   std::vector<const bf16 *> attn_norm, mlp_norm;
   std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_down;
   std::vector<CUtensorMap> tm_gu_half;     // dense gate / up matrices with the box of the GEMM with SwiGLU in its epilogue
-  std::vector<CUtensorMap> tm_k, tm_v;   // per layer: key view and transposed-value view of the pages
+  std::vector<CUtensorMap> tm_k, tm_v;   // per layer: the pages as rows of head_dim halfs (keys and values alike)
   // Mixture-of-Experts feed-forward layers (E = 0: dense).  sh.ffn is then (E + S) * F.
   int moe_E = 0, moe_K = 0, moe_F = 0, moe_S = 0, moe_renorm = 0;
   bf16 *router_pad = nullptr;            // [L][256][H]: each layer's router rows, zero rows behind them
@@ -532,7 +532,7 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
   // zero-filled: masked positions of a page are multiplied by zero weights, so they must be finite
   if ((rc = dmalloc(A, &e->kv_pool, e->layer_stride * s.n_layers, true))) return fail(rc);
   {
-    // one layer's pages seen as rows of hd halfs (keys) and as rows of 16 halfs (transposed values)
+    // one layer's pages seen as rows of hd halfs (16 rows per page and head, keys first, then values)
     const unsigned long long halfs = (unsigned long long)e->layer_stride;
     if (halfs / KV_BLOCK >= (1ull << 31)) return fail(CORUN_EINVAL);
     e->tm_k.resize(s.n_layers);
@@ -540,7 +540,7 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
     for (int l = 0; l < s.n_layers; ++l) {
       const __half *base = e->kv_pool + (size_t)l * e->layer_stride;
       if ((rc = tma_encode_2d(&e->tm_k[l], base, 1, halfs / s.head_dim, s.head_dim, KV_BLOCK, 64))) return fail(rc);
-      if ((rc = tma_encode_2d(&e->tm_v[l], base, 1, halfs / KV_BLOCK, KV_BLOCK, s.head_dim, KV_BLOCK))) return fail(rc);
+      e->tm_v[l] = e->tm_k[l];   // keys and values are cached alike: the same view serves both
     }
     if (attention_prepare() != cudaSuccess) return fail(CORUN_ECUDA);
   }

@@ -23,18 +23,18 @@ struct Rows {
   int R;
 };
 
-// Offsets (in halfs) inside one page: keys as [head][token][dim], then values TRANSPOSED as
-// [head][dim][token], so that both are K-major operands of the attention MMAs (scores contract over
-// dims, weighted values contract over tokens).
+// Offsets (in halfs) inside one page: keys as [head][token][dim], then values the same way.  The scores
+// contract over dims (the key tile is a K-major operand); the weighted values contract over tokens, for which
+// the value tile, read through the same kind of TMA box as the keys (rows of 128 bytes), is an MN-major operand.
 __host__ __device__ inline size_t kv_k_off(int hd, int g, int tok, int dim) {
   return ((size_t)g * KV_BLOCK + tok) * hd + dim;
 }
 __host__ __device__ inline size_t kv_v_off(int n_kv, int hd, int g, int tok, int dim) {
-  return (size_t)n_kv * KV_BLOCK * hd + ((size_t)g * hd + dim) * KV_BLOCK + tok;
+  return (size_t)n_kv * KV_BLOCK * hd + ((size_t)g * KV_BLOCK + tok) * hd + dim;
 }
 
 struct KvLayout {
-  __half *pool;            // [layer][page][ K: [n_kv][16][hd] | V^T: [n_kv][hd][16] ]
+  __half *pool;            // [layer][page][ K: [n_kv][16][hd] | V: [n_kv][16][hd] ]
   const int *block_table;  // [n_slots][max_blocks]
   int max_blocks, n_kv, hd;
   size_t layer_stride;     // halfs per layer
@@ -67,7 +67,7 @@ cudaError_t launch_qkv_post(const GemmOut &qkv, const Rows &rows, const float2 *
 // request in one slot (a prefill chunk): launch_attention_prefill runs instead; 2 for the ablation in which a
 // CTA takes whole (row, kv head) pairs (the work list then carries the pair table); else 0.
 // tmK / tmV: tensor maps over this layer's pages: keys as rows of hd halfs with a [16, 64] box (128-byte
-// swizzle), values as rows of 16 halfs with an [hd, 16] box (32-byte swizzle); see attention.cu.
+// swizzle), and the values, cached alike, through the same view; see attention.cu.
 // work / n_work: the step's (row, kv head, split) items from launch_attn_worklist (the same for every layer);
 // grid_ctas: persistent CTAs to launch (one per SM).
 cudaError_t launch_attention(const CUtensorMap &tmK, const CUtensorMap &tmV, const float *q, const Rows &rows, int nq,

@@ -152,15 +152,18 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
   return d;
 }
 
-// Same for rows of 32 bytes (16 halfs) stored with the 32-byte swizzle: 8-row groups 256 bytes apart,
-// layout type 6 = SWIZZLE_32B.
-__device__ __forceinline__ uint64_t umma_desc_sw32(uint32_t smem_addr) {
+// Descriptor of an MN-major operand (the M or N index runs along the 128-byte rows, K across rows) stored with
+// the 128-byte swizzle: every 128-byte row holds 64 consecutive M (N) elements of one K index, eight consecutive
+// K rows form a 1 KiB swizzle atom.  mn_block_bytes: distance between the tiles of consecutive blocks of 64 M (N)
+// elements (leading byte offset); k_group_bytes: distance between consecutive groups of 8 K rows (stride byte
+// offset).  The instruction descriptor must mark the operand MN-major (bit 15 for A, bit 16 for B).
+__device__ __forceinline__ uint64_t umma_desc_sw128_mn(uint32_t smem_addr, uint32_t mn_block_bytes, uint32_t k_group_bytes) {
   uint64_t d = 0;
   d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
-  d |= (uint64_t)1u << 16;
-  d |= (uint64_t)(256u >> 4) << 32;
-  d |= (uint64_t)1u << 46;
-  d |= (uint64_t)6u << 61;
+  d |= (uint64_t)((mn_block_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((k_group_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1u << 46;                 // version
+  d |= (uint64_t)2u << 61;                 // SWIZZLE_128B
   return d;
 }
 
