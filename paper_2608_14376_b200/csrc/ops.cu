@@ -410,7 +410,7 @@ __device__ __noinline__ void smp_tail_full_row(SmpShared &sh, const SampleArgs &
 // the running weight reaches the cut (the nucleus edge is then found among those few tokens in shared
 // memory); per-warp totals of the nucleus weights in id order, after which one warp walks its range to
 // the drawn token.
-constexpr int SMP_CLUSTER = 4;
+constexpr int SMP_CLUSTER = 6;
 
 __global__ void __cluster_dims__(SMP_CLUSTER, 1, 1) __launch_bounds__(SMP_THREADS, 2) sampler_kernel(SampleArgs a) {
   namespace cg = cooperative_groups;
