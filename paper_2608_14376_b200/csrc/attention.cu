@@ -2,7 +2,7 @@
 //
 // An item is (row, kv head, split of 128 cached tokens = 8 pages); the step's items are listed in that
 // order and every CTA takes one contiguous stretch of the list (its two consumer groups one half each),
-// so consecutive items of a group mostly share their query rows.  That covers the first 15/16 of the list; the rest is dealt out two items at a
+// so consecutive items of a group mostly share their query rows.  That covers the first 7/8 of the list; the rest is dealt out two items at a
 // time through a counter, so that CTAs that got through their stretch sooner take more of it (which CTA
 // computes an item has no influence on any value).  One persistent CTA per SM:
 //   warp 0        streams the items' keys with TMA into a ring of 3 key buffers ([16 tokens x 64 dims]
@@ -194,7 +194,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   if (n_total <= 0) return;
   // this CTA's stretch of the item list, and where the shared pool begins
   const int n_pairs = WHOLE_PAIRS ? n_work[1] : 0;   // > 0: the ablation that hands out whole (row, kv head) pairs (see item_of)
-  const int n_fixed = n_pairs > 0 ? 0 : (int)(((long long)n_total * 15 / 16) / gridDim.x);
+  const int n_fixed = n_pairs > 0 ? 0 : (int)(((long long)n_total * 7 / 8) / gridDim.x);
   const int item_lo = (int)blockIdx.x * n_fixed, pool_lo = (int)gridDim.x * n_fixed;
 
   extern __shared__ uint8_t smem_raw[];

@@ -332,6 +332,12 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                               : (whole ? direct + n0 : ws + (size_t)(cta * 2 + (seg == 0 ? 0 : 1)) * BN * GEMM_TILE_N);
         const size_t pitch = whole ? (size_t)N : (size_t)GEMM_TILE_N;
         const bool vec_ok = whole ? ((N & 3) == 0) : true;
+        bool row_on[4];                               // which of this thread's four rows are stored at all
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int r = i * 16 + srow;
+          row_on[i] = r < rows_valid && (!MASKED || r >= R || keep[(size_t)r * keep_pitch] != 0.f);
+        }
         for (int c0 = 0; c0 < GEMM_TILE_N; c0 += 32) {
           if (whole && n0 + c0 >= N) break;          // columns beyond the matrix (last tile); uniform
           if (warp_needed) {
@@ -347,7 +353,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int r = i * 16 + srow;
-            if (r < rows_valid && (!MASKED || r >= R || keep[(size_t)r * keep_pitch] != 0.f)) {
+            if (row_on[i]) {
               const float *h = xch[0] + r * 33 + scol, *l = xch[1] + r * 33 + scol;
               const float4 f = make_float4(h[0] + l[0], h[1] + l[1], h[2] + l[2], h[3] + l[3]);
               float *d = dst0 + (size_t)r * pitch + c0 + scol;
