@@ -327,9 +327,9 @@ int enqueue_decode_body(corun_engine *e, int *launches) {
   Program &P = e->dec;
   const corun_shape &s = e->sh;
   int n = 0;
-  CK(cudaMemcpyAsync(e->d_active, e->h_active, e->B, cudaMemcpyHostToDevice, e->st));
-  CK(cudaMemcpyAsync(e->d_seeds, e->h_seeds, e->B * sizeof(uint64_t), cudaMemcpyHostToDevice, e->st));
-  CK(launch_prepare_rows(e->d_active, e->d_in_use, e->d_ctx, e->d_pending, e->B, P.row_token, P.row_pos, P.row_active,
+  // mask and seeds are read from the pinned staging buffers by the first kernel, tokens and status are written to
+  // them by the last one (zero-copy): a copy node in a graph costs several microseconds, these are 836 bytes
+  CK(launch_prepare_rows(e->h_active, e->h_seeds, e->d_seeds, e->d_in_use, e->d_ctx, e->d_pending, e->B, P.row_token, P.row_pos, P.row_active,
                          P.row_slot, P.do_sample, e->st));
   n += 1;
   RC(run_layers(e, P, &n));
@@ -341,11 +341,11 @@ int enqueue_decode_body(corun_engine *e, int *launches) {
     CK(gemm_fixup_launch(P.p_lm, e->st, true));
     SampleArgs sa{P.logits, s.vocab, P.do_sample, e->d_temp, e->d_top_p, e->d_seeds, e->d_step, nullptr, P.sampled};
     CK(launch_sampler(sa, P.R, e->st, true));
-    CK(launch_advance(P.row_active, P.sampled, e->B, e->d_ctx, e->d_step, e->d_pending, e->d_out_tokens, e->st));
+    CK(launch_advance(P.row_active, P.sampled, e->B, e->d_ctx, e->d_step, e->d_pending, e->h_out_tokens, e->d_status, e->h_status, e->st));
     n += 4 + (P.p_lm.n_split_tiles ? 1 : 0);
   }
-  CK(cudaMemcpyAsync(e->h_out_tokens, e->d_out_tokens, e->B * sizeof(int), cudaMemcpyDeviceToHost, e->st));
-  CK(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, e->st));
+  if (e->eager && e->stop_after >= 0)            // (debug) no last kernel ran: fetch the status word the plain way
+    CK(cudaMemcpyAsync(e->h_status, e->d_status, sizeof(int), cudaMemcpyDeviceToHost, e->st));
   if (launches) *launches = n;
   return CORUN_OK;
 }

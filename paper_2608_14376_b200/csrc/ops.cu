@@ -724,7 +724,11 @@ __global__ void __cluster_dims__(SMP_CLUSTER, 1, 1) __launch_bounds__(SMP_THREAD
 #undef SMP_FOREACH
 
 // ---------------------------------------------------------------- decode bookkeeping
-__global__ void prepare_rows_kernel(const uint8_t *active_mask, const int *in_use, const int *ctx_len,
+// active_mask / seeds_in are the step's inputs in PINNED HOST memory, read here through their device mapping:
+// 9 bytes per slot cross the bus inside this kernel instead of in two copy nodes in front of it; the seeds
+// go to seeds_out (device) for the sampler.
+__global__ void prepare_rows_kernel(const uint8_t *active_mask, const uint64_t *seeds_in, uint64_t *seeds_out,
+                                    const int *in_use, const int *ctx_len,
                                     const int *pending, int B, int *row_token, int *row_pos, int *row_active,
                                     int *row_slot, int *do_sample) {
   griddep_launch_dependents();
@@ -732,6 +736,7 @@ __global__ void prepare_rows_kernel(const uint8_t *active_mask, const int *in_us
   const int s = blockIdx.x * blockDim.x + threadIdx.x;
   if (s >= B) return;
   const int act = (active_mask[s] != 0 && in_use[s] != 0) ? 1 : 0;
+  seeds_out[s] = seeds_in[s];
   row_active[s] = act;
   row_slot[s] = s;
   row_pos[s] = act ? ctx_len[s] : 0;
@@ -739,12 +744,15 @@ __global__ void prepare_rows_kernel(const uint8_t *active_mask, const int *in_us
   do_sample[s] = act;
 }
 
+// out_tokens / status_out are PINNED HOST memory written through their device mapping (the step's results: 4
+// bytes per slot and the status word), fenced system-wide; the host reads them after synchronising the stream.
 __global__ void advance_kernel(const int *row_active, const int *sampled, int B, int *ctx_len, int *step, int *pending,
-                               int *out_tokens) {
+                               int *out_tokens, const int *status_in, int *status_out) {
   griddep_launch_dependents();
   griddep_wait();
   const int s = blockIdx.x * blockDim.x + threadIdx.x;
-  if (s >= B) return;
+  if (s == 0) *status_out = *status_in;
+  if (s >= B) { __threadfence_system(); return; }
   if (row_active[s]) {
     const int tok = sampled[s];
     pending[s] = tok;
@@ -754,6 +762,7 @@ __global__ void advance_kernel(const int *row_active, const int *sampled, int B,
   } else {
     out_tokens[s] = -1;
   }
+  __threadfence_system();
 }
 
 __global__ void kv_copy_kernel(KvLayout kv, int layer, int slot, int pos0, int n, float *k, float *v, int write) {
@@ -837,18 +846,19 @@ cudaError_t launch_sampler(const SampleArgs &a, int R, cudaStream_t st, bool pdl
   return launch_k(sampler_kernel, dim3(R * SMP_CLUSTER), dim3(SMP_THREADS), 0, st, pdl, a);
 }
 
-cudaError_t launch_prepare_rows(const uint8_t *active_mask, const int *in_use, const int *ctx_len, const int *pending,
+cudaError_t launch_prepare_rows(const uint8_t *active_mask, const uint64_t *seeds_in, uint64_t *seeds_out, const int *in_use,
+                                const int *ctx_len, const int *pending,
                                 int B, int *row_token, int *row_pos, int *row_active, int *row_slot, int *do_sample,
                                 cudaStream_t st) {
-  prepare_rows_kernel<<<(B + 127) / 128, 128, 0, st>>>(active_mask, in_use, ctx_len, pending, B, row_token, row_pos,
-                                                       row_active, row_slot, do_sample);
+  prepare_rows_kernel<<<(B + 127) / 128, 128, 0, st>>>(active_mask, seeds_in, seeds_out, in_use, ctx_len, pending, B, row_token,
+                                                       row_pos, row_active, row_slot, do_sample);
   return cudaGetLastError();
 }
 
 cudaError_t launch_advance(const int *row_active, const int *sampled, int B, int *ctx_len, int *step, int *pending,
-                           int *out_tokens, cudaStream_t st) {
+                           int *out_tokens, const int *status_in, int *status_out, cudaStream_t st) {
   return launch_k(advance_kernel, dim3((B + 127) / 128), dim3(128), 0, st, true, row_active, sampled, B, ctx_len, step,
-                  pending, out_tokens);
+                  pending, out_tokens, status_in, status_out);
 }
 
 cudaError_t launch_kv_copy(const KvLayout &kv, int layer, int slot, int pos0, int n, float *k, float *v, int write,

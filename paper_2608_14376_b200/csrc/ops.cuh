@@ -92,11 +92,14 @@ cudaError_t launch_swiglu(const GemmOut &gu, int R, int F, __nv_bfloat16 *out_hi
 cudaError_t launch_split(const float *x, int R, int K, __nv_bfloat16 *hi, __nv_bfloat16 *lo, cudaStream_t st);
 cudaError_t launch_sampler(const SampleArgs &a, int R, cudaStream_t st, bool pdl = false);
 // decode bookkeeping
-cudaError_t launch_prepare_rows(const uint8_t *active_mask, const int *in_use, const int *ctx_len, const int *pending,
+// The step's inputs (active mask, seeds) and results (tokens, status word) live in pinned host memory and are
+// read / written by these two kernels through its device mapping: no copy nodes around the step.
+cudaError_t launch_prepare_rows(const uint8_t *active_mask, const uint64_t *seeds_in, uint64_t *seeds_out, const int *in_use,
+                                const int *ctx_len, const int *pending,
                                 int B, int *row_token, int *row_pos, int *row_active, int *row_slot, int *do_sample,
                                 cudaStream_t st);
 cudaError_t launch_advance(const int *row_active, const int *sampled, int B, int *ctx_len, int *step, int *pending,
-                           int *out_tokens, cudaStream_t st);
+                           int *out_tokens, const int *status_in, int *status_out, cudaStream_t st);
 // debug cache access (fp32 rows of n_kv*hd)
 cudaError_t launch_kv_copy(const KvLayout &kv, int layer, int slot, int pos0, int n, float *k, float *v, int write,
                            cudaStream_t st);
