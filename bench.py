@@ -406,29 +406,28 @@ def run_corun(args, rank, world):
     mla = None
     if rank == 0 and sh.n_layers > 8 and not moe_cfg:
         import math
-        from paper_2608_14376_b200.corun import mla_attend
+        from paper_2608_14376_b200.corun import MlaAttention
         gl = torch.Generator(device="cuda").manual_seed(4)
         lB, lh, ldc, ldr = 128, 16, 512, 64
-        lctx = synth.uniform_lengths(512, 4096, lB, seed=2).astype(np.int32)
-        lT = int(-(-int(lctx.max()) // 128) * 128)
-        lcache = (torch.randn((lB, lT, ldc + ldr), generator=gl, device="cuda") * 0.5).to(torch.float16)
+        lpool, ltable, ldctx = synth.mla_paged_case(lB, ldc + ldr, 512, 4096, seed=2)
+        lctx = ldctx.cpu().numpy()
         lq, lr = torch.randn((lB, lh, ldc), generator=gl, device="cuda"), torch.randn((lB, lh, ldr), generator=gl, device="cuda")
-        ldctx = torch.tensor(lctx).cuda()
         lbytes = int(lctx.astype(np.int64).sum()) * (ldc + ldr) * 2
-        mla = {"workload": "deepseek_v2_lite_mla_b128", "contexts": f"uniform {lctx.min()}..{lctx.max()}", "cache_bytes": lbytes}
-        for name, pairs in (("fp16_pairs", True), ("single_fp16", False)):
-            for _ in range(3):
-                mla_attend(lq, lr, lcache, ldctx, 1.0 / math.sqrt(128 + ldr), pairs)
-            torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            for _ in range(20):
-                mla_attend(lq, lr, lcache, ldctx, 1.0 / math.sqrt(128 + ldr), pairs)
-            e1.record()
-            torch.cuda.synchronize()
-            lms = e0.elapsed_time(e1) / 20
-            mla[name] = {"us_per_call": lms * 1e3, "GBs": lbytes / lms / 1e6, "frac_of_measured_hbm": lbytes / lms / 1e6 / hbm}
-        del lcache, lq, lr
+        lop = MlaAttention(lB, lh, ldc, ldr, ltable.shape[1])
+        for _ in range(3):
+            lop.run(lq, lr, lpool, ltable, ldctx, 1.0 / math.sqrt(128 + ldr))
+        lop.sync()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(20):
+            lop.run(lq, lr, lpool, ltable, ldctx, 1.0 / math.sqrt(128 + ldr))
+        e1.record()
+        lop.sync()
+        lms = e0.elapsed_time(e1) / 20
+        mla = {"workload": "deepseek_v2_lite_mla_b128", "contexts": f"uniform {lctx.min()}..{lctx.max()}", "cache": "paged, 16 tokens per page",
+               "cache_bytes": lbytes, "us_per_call": lms * 1e3, "GBs": lbytes / lms / 1e6, "frac_of_measured_hbm": lbytes / lms / 1e6 / hbm,
+               "operands": "fp16 hi + lo pairs (tcgen05)"}
+        del lpool, lq, lr, lop
 
     cpu = None
     if rank == 0 and not args.no_cpu_baseline and not moe_cfg:

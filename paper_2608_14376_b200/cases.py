@@ -208,30 +208,27 @@ def case_mla(a):
     from . import corun, synth
 
     nh, dc, dr = 16, 512, 64
-    ctx = synth.uniform_lengths(a.ctx_lo, a.ctx_hi, a.B, seed=2).astype(np.int32)
-    T = int(-(-int(ctx.max()) // 128) * 128)
+    pool, table, dctx = synth.mla_paged_case(a.B, dc + dr, a.ctx_lo, a.ctx_hi, seed=2)
+    ctx = dctx.cpu().numpy()
     g = torch.Generator(device="cuda").manual_seed(0)
-    cache = (torch.randn((a.B, T, dc + dr), generator=g, device="cuda") * 0.5).to(torch.float16)
     q_lat = torch.randn((a.B, nh, dc), generator=g, device="cuda")
     q_rope = torch.randn((a.B, nh, dr), generator=g, device="cuda")
-    dctx = torch.tensor(ctx).cuda()
     scale = 1.0 / math.sqrt(128 + dr)
-    pairs = not a.single
+    op = corun.MlaAttention(a.B, nh, dc, dr, table.shape[1])
     for _ in range(3):
-        out = corun.mla_attend(q_lat, q_rope, cache, dctx, scale, pairs)
-    torch.cuda.synchronize()
+        out = op.run(q_lat, q_rope, pool, table, dctx, scale)
+    op.sync()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
     for _ in range(a.reps):
-        out = corun.mla_attend(q_lat, q_rope, cache, dctx, scale, pairs)
+        out = op.run(q_lat, q_rope, pool, table, dctx, scale)
     t1.record()
-    torch.cuda.synchronize()
+    op.sync()
     ms = t0.elapsed_time(t1) / a.reps
     nbytes = int(ctx.astype(np.int64).sum()) * (dc + dr) * 2
     flops = int(ctx.astype(np.int64).sum()) * nh * (dc + dr + dc) * 2
-    print("mla: B=%d, contexts %d..%d (mean %.0f): %.1f us per call, %.1f MB of latent cache -> %.0f GB/s, %.1f TFLOP/s (%s)"
-          % (a.B, ctx.min(), ctx.max(), ctx.mean(), ms * 1e3, nbytes / 1e6, nbytes / ms / 1e6, flops / ms / 1e9,
-             "fp16 hi+lo operand pairs" if pairs else "single fp16 operands"))
+    print("mla: B=%d, contexts %d..%d (mean %.0f), paged latent cache: %.1f us per call, %.1f MB -> %.0f GB/s, %.1f TFLOP/s"
+          % (a.B, ctx.min(), ctx.max(), ctx.mean(), ms * 1e3, nbytes / 1e6, nbytes / ms / 1e6, flops / ms / 1e9))
     assert bool(torch.isfinite(out).all().item())
 
 

@@ -26,7 +26,7 @@ EXPORTS = [
     "corun_sched_step", "corun_sched_poll", "corun_sched_slot_of", "corun_sched_counts",
     "corun_sched_enable_batched_prefill", "corun_prefill_geometry",
     "corun_moe_create", "corun_moe_destroy", "corun_moe_forward", "corun_moe_sync", "corun_moe_weight_bytes",
-    "corun_moe_launches", "corun_mla_attend", "corun_mla_workspace_floats",
+    "corun_moe_launches", "corun_mla_attend", "corun_mla_workspace_floats", "corun_mla_sync",
 ]
 
 
@@ -529,28 +529,51 @@ class MoeFfn:
             pass
 
 
-def mla_attend(q_lat, q_rope, cache, ctx, scale: float, operand_pairs: bool = True):
-    """Absorbed multi-head latent attention for one query token per row (``include/corun_mla.h``).
-    q_lat fp32 [B, n_heads, d_c], q_rope fp32 [B, n_heads, d_r], cache fp16 [B, T, d_c + d_r], ctx int32 [B]
-    (all CUDA tensors) -> o_lat fp32 [B, n_heads, d_c] (rows with ctx 0 are left as zeros).  operand_pairs:
-    queries and softmax weights as fp16 hi + lo pairs (fp32-grade) or as single fp16 values (half the tensor work)."""
-    import torch
+class MlaAttention:
+    """Absorbed multi-head latent attention for one query token per row over a paged latent cache
+    (``include/corun_mla.h``) with its workspace and output allocated once: ``run`` only enqueues."""
 
-    B, nh, dc = q_lat.shape
-    dr = q_rope.shape[2]
-    T = cache.shape[1]
-    assert q_lat.is_cuda and q_lat.dtype == torch.float32 and q_lat.is_contiguous()
-    assert q_rope.dtype == torch.float32 and q_rope.is_contiguous() and tuple(q_rope.shape[:2]) == (B, nh)
-    assert cache.dtype == torch.float16 and cache.is_contiguous() and tuple(cache.shape) == (B, T, dc + dr)
-    assert ctx.dtype == torch.int32 and ctx.is_contiguous() and tuple(ctx.shape) == (B,)
-    L = lib()
-    L.corun_mla_workspace_floats.restype = C.c_int64
-    L.corun_mla_workspace_floats.argtypes = [C.c_int32] * 4
-    L.corun_mla_attend.argtypes = [C.c_void_p] * 4 + [C.c_int32] * 5 + [C.c_float, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
-    ws = torch.empty(int(L.corun_mla_workspace_floats(B, nh, dc, T)), dtype=torch.float32, device=q_lat.device)
-    out = torch.zeros_like(q_lat)
-    _check(L.corun_mla_attend(q_lat.data_ptr(), q_rope.data_ptr(), cache.data_ptr(), ctx.data_ptr(), B, nh, dc, dr, T,
-                              float(scale), out.data_ptr(), ws.data_ptr(), 1 if operand_pairs else 0,
-                              torch.cuda.current_stream().cuda_stream),
-           "corun_mla_attend")
+    def __init__(self, B: int, n_heads: int, d_latent: int, d_rope: int, max_blocks: int, device="cuda"):
+        import torch
+
+        L = lib()
+        L.corun_mla_workspace_floats.restype = C.c_int64
+        L.corun_mla_workspace_floats.argtypes = [C.c_int32] * 4
+        L.corun_mla_attend.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32, C.c_void_p] + \
+            [C.c_int32] * 4 + [C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.corun_mla_sync.argtypes = [C.c_void_p, C.c_void_p]
+        self.shape = (B, n_heads, d_latent, d_rope, max_blocks)
+        self.ws = torch.empty(int(L.corun_mla_workspace_floats(B, n_heads, d_latent, max_blocks * 16)), dtype=torch.float32, device=device)
+        self.out = torch.zeros((B, n_heads, d_latent), dtype=torch.float32, device=device)
+
+    def run(self, q_lat, q_rope, pool, block_table, ctx, scale: float):
+        """q_lat fp32 [B, n_heads, d_c], q_rope fp32 [B, n_heads, d_r], pool fp16 [pool_pages, 16, d_c + d_r],
+        block_table int32 [B, max_blocks], ctx int32 [B] (contiguous CUDA tensors) -> o_lat fp32 [B, n_heads, d_c]
+        (rows with ctx 0 keep what they held).  Asynchronous on torch's current stream."""
+        import torch
+
+        B, nh, dc, dr, mb = self.shape
+        assert tuple(q_lat.shape) == (B, nh, dc) and q_lat.dtype == torch.float32 and q_lat.is_contiguous() and q_lat.is_cuda
+        assert tuple(q_rope.shape) == (B, nh, dr) and q_rope.dtype == torch.float32 and q_rope.is_contiguous()
+        assert pool.dtype == torch.float16 and pool.is_contiguous() and tuple(pool.shape[1:]) == (16, dc + dr)
+        assert block_table.dtype == torch.int32 and block_table.is_contiguous() and tuple(block_table.shape) == (B, mb)
+        assert ctx.dtype == torch.int32 and ctx.is_contiguous() and tuple(ctx.shape) == (B,)
+        st = torch.cuda.current_stream().cuda_stream
+        _check(lib().corun_mla_attend(q_lat.data_ptr(), q_rope.data_ptr(), pool.data_ptr(), pool.shape[0], block_table.data_ptr(),
+                                      mb, ctx.data_ptr(), B, nh, dc, dr, float(scale), self.out.data_ptr(), self.ws.data_ptr(), st),
+               "corun_mla_attend")
+        return self.out
+
+    def sync(self):
+        """Waits for the stream; raises if a bounded device-side wait expired."""
+        import torch
+
+        _check(lib().corun_mla_sync(self.ws.data_ptr(), torch.cuda.current_stream().cuda_stream), "corun_mla_sync")
+
+
+def mla_attend(q_lat, q_rope, pool, block_table, ctx, scale: float):
+    """One call of ``MlaAttention`` with fresh buffers (rows with ctx 0 come back as zeros); waits for the result."""
+    op = MlaAttention(q_lat.shape[0], q_lat.shape[1], q_lat.shape[2], q_rope.shape[2], block_table.shape[1], q_lat.device)
+    out = op.run(q_lat, q_rope, pool, block_table, ctx, scale)
+    op.sync()
     return out

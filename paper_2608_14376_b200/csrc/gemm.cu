@@ -457,6 +457,28 @@ int tma_encode_2d(CUtensorMap *m, const void *base, int is_fp16, unsigned long l
   return r == CUDA_SUCCESS ? CORUN_OK : CORUN_ECUDA;
 }
 
+int tma_encode_fp16_4d(CUtensorMap *m, const void *base, const unsigned long long dims[4], const unsigned long long strides[3],
+                       const unsigned box[4]) {
+  auto enc = get_encode();
+  if (!enc) { g_last_cuda_error = 99999; return CORUN_ECUDA; }
+  if (((uintptr_t)base & 15u) || box[0] * 2 != 128) return CORUN_EINVAL;
+  cuuint64_t d[4], s[3];
+  cuuint32_t b[4], estr[4] = {1, 1, 1, 1};
+  for (int i = 0; i < 4; ++i) {
+    if (dims[i] < 1 || box[i] < 1 || box[i] > 256) return CORUN_EINVAL;
+    d[i] = dims[i];
+    b[i] = box[i];
+  }
+  for (int i = 0; i < 3; ++i) {
+    if (strides[i] % 16) return CORUN_EINVAL;
+    s[i] = strides[i];
+  }
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void *>(base), d, s, b, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) g_last_cuda_error = 100000 + (int)r;
+  return r == CUDA_SUCCESS ? CORUN_OK : CORUN_ECUDA;
+}
+
 int gemm_encode_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows) {
   if (K % GEMM_BLOCK_K) return CORUN_EINVAL;
   return tma_encode_2d(m, base, 0, (unsigned long long)rows, K, box_rows, GEMM_BLOCK_K);

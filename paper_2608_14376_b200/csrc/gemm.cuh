@@ -139,6 +139,12 @@ cudaError_t gemm_prepare_kernel();
 // (128 bytes, 128-byte swizzle) or 16 columns (32 bytes, 32-byte swizzle).
 int tma_encode_2d(CUtensorMap *m, const void *base, int is_fp16, unsigned long long rows, int cols, int box_rows,
                   int box_cols);
+// Tensor map over fp16 data seen as a 4-dimensional array: dims[0] elements are contiguous, strides[i] is the byte
+// distance between consecutive indices of dimension i + 1 (a multiple of 16; they need not ascend); the box's
+// innermost extent is 64 elements (128 bytes, 128-byte swizzle).  The box lands in shared memory densely,
+// dimension 0 fastest.
+int tma_encode_fp16_4d(CUtensorMap *m, const void *base, const unsigned long long dims[4], const unsigned long long strides[3],
+                       const unsigned box[4]);
 // direct[r, n] = gemm_load(r, n) for every tile that has partials (makes `direct` a plain matrix).
 cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st, bool pdl = false);
 

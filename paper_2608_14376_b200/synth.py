@@ -229,3 +229,24 @@ def synthetic_kv(n_tokens: int, kv_dim: int, std: float, seed: int, dtype=np.flo
     k = (rng.standard_normal((n_tokens, kv_dim), dtype=np.float32) * np.float32(std)).astype(dtype).astype(np.float32)
     v = (rng.standard_normal((n_tokens, kv_dim), dtype=np.float32) * np.float32(std)).astype(dtype).astype(np.float32)
     return k, v
+
+
+def mla_paged_case(B: int, d_k: int, ctx_lo: int, ctx_hi: int, seed: int, device="cuda", page: int = 16, std: float = 0.5):
+    """Seeded paged latent cache on the device for timing: contexts uniform in [ctx_lo, ctx_hi], a pool of exactly the
+    pages they need (fp16 N(0, std^2), every position finite) and a block table that scatters every row's pages over
+    the pool (a seeded permutation).  Returns (pool [P, page, d_k], block_table int32 [B, max_blocks], ctx int32 [B])."""
+    import torch
+
+    ctx = uniform_lengths(ctx_lo, ctx_hi, B, seed=seed).astype(np.int32)
+    blocks = -(-ctx // page)
+    max_blocks = int(blocks.max())
+    n_pages = int(blocks.sum())
+    g = torch.Generator(device=device).manual_seed(seed)
+    pool = (torch.randn((n_pages, page, d_k), generator=g, device=device) * std).to(torch.float16)
+    perm = np.random.Generator(np.random.PCG64(seed)).permutation(n_pages).astype(np.int32)
+    table = np.zeros((B, max_blocks), np.int32)
+    k = 0
+    for b in range(B):
+        table[b, :blocks[b]] = perm[k:k + blocks[b]]
+        k += int(blocks[b])
+    return pool, torch.tensor(table, device=device), torch.tensor(ctx, device=device)

@@ -1,4 +1,5 @@
-"""Absorbed multi-head latent attention against its oracle, and row independence."""
+"""Absorbed multi-head latent attention over a paged latent cache against its oracle; independence of a row from
+the other rows of the call and from where its pages lie in the pool."""
 import math
 
 import numpy as np
@@ -8,144 +9,139 @@ from oracle import mla_oracle as ml
 
 pytestmark = pytest.mark.gpu
 
+PAGE = 16
 
-@pytest.mark.parametrize("nh,dc,dr,pairs", [(16, 512, 64, True), (4, 64, 8, True), (8, 128, 32, True), (16, 512, 24, True),
-                                            (4, 64, 16, True), (16, 512, 64, False), (8, 128, 32, False), (4, 64, 16, False)])
-def test_mla_attend_matches_oracle_and_rows_are_independent(nh, dc, dr, pairs):
+
+def _torch():
     torch = pytest.importorskip("torch")
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
-    from paper_2608_14376_b200 import corun
+    return torch
 
-    rng = np.random.default_rng(nh + dc)
-    ctxs = [0, 1, 127, 128, 129, 700, 385]
-    B, T = len(ctxs), 768
+
+def _paged(rng, caches, ctxs, dk, spare=7, fill=0.25):
+    """Scatters every row's tokens over randomly chosen pages of one pool.  Returns (pool fp16 [P, 16, dk],
+    block table int32 [B, max_blocks]).  Pages and positions that no row uses hold finite filler values."""
+    max_blocks = max(1, max(-(-c // PAGE) for c in ctxs))
+    need = sum(-(-c // PAGE) for c in ctxs)
+    n_pages = need + spare
+    pool = (rng.standard_normal((n_pages, PAGE, dk)) * fill).astype(np.float16)
+    order = rng.permutation(n_pages)
+    table = np.zeros((len(ctxs), max_blocks), np.int32)
+    k = 0
+    for b, c in enumerate(ctxs):
+        for i in range(-(-c // PAGE)):
+            pg = int(order[k]); k += 1
+            table[b, i] = pg
+            n = min(PAGE, c - i * PAGE)
+            pool[pg, :n] = caches[b][i * PAGE:i * PAGE + n]
+    return pool, table
+
+
+def _case(nh, dc, dr, ctxs, seed):
+    rng = np.random.default_rng(seed)
+    B = len(ctxs)
     q_lat = rng.standard_normal((B, nh, dc)).astype(np.float32)
     q_rope = rng.standard_normal((B, nh, dr)).astype(np.float32)
-    cache = (rng.standard_normal((B, T, dc + dr)) * 0.5).astype(np.float16)
-    scale = 1.0 / math.sqrt(dc + dr)
+    caches = [(rng.standard_normal((c, dc + dr)) * 0.5).astype(np.float16) for c in ctxs]
+    return rng, q_lat, q_rope, caches
+
+
+def _run(torch, q_lat, q_rope, pool, table, ctxs, scale):
+    from paper_2608_14376_b200 import corun
+
     dev = lambda a: torch.tensor(a).cuda().contiguous()
-    out = corun.mla_attend(dev(q_lat), dev(q_rope), dev(cache), dev(np.array(ctxs, np.int32)), scale, pairs)
+    out = corun.mla_attend(dev(q_lat), dev(q_rope), dev(pool), dev(table), dev(np.array(ctxs, np.int32)), scale)
     torch.cuda.synchronize()
-    out = out.cpu().numpy()
+    return out.cpu().numpy()
+
+
+def _worst(out, q_lat, q_rope, caches, ctxs, dc):
+    nh = q_lat.shape[1]
     eye = np.stack([np.eye(dc)] * nh)               # W_uk = W_uv = identity: the absorbed level itself
     worst = 0.0
     for b, n in enumerate(ctxs):
         if n == 0:
             assert not out[b].any()                  # a padding row is left alone
             continue
-        C = cache[b, :n, :dc].astype(np.float64)
-        Rk = cache[b, :n, dc:].astype(np.float64)
-        ref = ml.attend_absorbed(q_lat[b], q_rope[b], C, Rk, eye, eye)
-        worst = max(worst, float(np.abs(out[b] - ref).max()))
-    # hi + lo pairs: fp32 accumulation chains of <= 576 and <= 512 terms on O(1) values.  Single fp16 operands:
-    # queries rounded to 2^-11 relative move a score by <= 2^-11 * scale * sum |q_d c_d| (~ 1e-3 here: 576 terms of
-    # ~0.4 times 0.04), which moves the weights, and so the outputs of size <= ~2, by that fraction at most;
-    # the rounding of the weights themselves adds 2^-11 relative.
-    assert worst <= (2e-5 if pairs else 4e-3), worst
-    # the same rows in another order among other rows: byte-identical
-    perm = [5, 2, 6]
-    q2 = rng.standard_normal((B, nh, dc)).astype(np.float32); r2 = rng.standard_normal((B, nh, dr)).astype(np.float32)
-    c2 = (rng.standard_normal((B, T, dc + dr)) * 0.5).astype(np.float16)
-    ctx2 = np.array([300, 5, 64, 9, 0, 17, 640], np.int32)
-    for i, src in enumerate(perm):
-        q2[i], r2[i], c2[i], ctx2[i] = q_lat[src], q_rope[src], cache[src], ctxs[src]
-    out2 = corun.mla_attend(dev(q2), dev(r2), dev(c2), dev(ctx2), scale, pairs).cpu().numpy()
-    for i, src in enumerate(perm):
-        assert out2[i].tobytes() == out[src].tobytes()
-
-
-def test_mla_single_operands_need_the_tensor_path():
-    torch = pytest.importorskip("torch")
-    if not torch.cuda.is_available():
-        pytest.skip("no CUDA device")
-    from paper_2608_14376_b200 import corun
-
-    z = lambda *s: torch.zeros(s, device="cuda")
-    with pytest.raises(Exception):                   # d_rope = 8: only the FMA kernel takes it, and only with pairs
-        corun.mla_attend(z(1, 4, 64), z(1, 4, 8), z(1, 128, 72).half(), torch.ones(1, dtype=torch.int32, device="cuda"), 1.0, False)
-
-
-def _mla_case(nh, dc, dr, ctxs, T, seed):
-    rng = np.random.default_rng(seed)
-    B = len(ctxs)
-    q_lat = rng.standard_normal((B, nh, dc)).astype(np.float32)
-    q_rope = rng.standard_normal((B, nh, dr)).astype(np.float32)
-    cache = (rng.standard_normal((B, T, dc + dr)) * 0.5).astype(np.float16)
-    return q_lat, q_rope, cache
-
-
-def _mla_worst(out, q_lat, q_rope, cache, ctxs, dc):
-    nh = q_lat.shape[1]
-    eye = np.stack([np.eye(dc)] * nh)
-    worst = 0.0
-    for b, n in enumerate(ctxs):
-        C = cache[b, :n, :dc].astype(np.float64)
-        Rk = cache[b, :n, dc:].astype(np.float64)
+        C = caches[b][:n, :dc].astype(np.float64)
+        Rk = caches[b][:n, dc:].astype(np.float64)
         ref = ml.attend_absorbed(q_lat[b], q_rope[b], C, Rk, eye, eye)
         worst = max(worst, float(np.abs(out[b] - ref).max()))
     return worst
 
 
-@pytest.mark.parametrize("path", ["", "CORUN_MLA_UNPIPELINED", "CORUN_MLA_FMA"])
-def test_mla_every_kernel_and_more_pieces_than_the_combine_fast_path(path):
-    """The three kernels (selected by environment variable) on contexts around the chunk boundary and on one with
-    more pieces than the combine kernel keeps in registers (18 chunks of 512, 71 splits of 128)."""
-    import os
-
-    torch = pytest.importorskip("torch")
-    if not torch.cuda.is_available():
-        pytest.skip("no CUDA device")
-    from paper_2608_14376_b200 import corun
-
-    nh, dc, dr = 4, 64, 16
-    ctxs = [9000, 512, 513, 1024, 63]
-    q_lat, q_rope, cache = _mla_case(nh, dc, dr, ctxs, 9216, seed=7)
+@pytest.mark.parametrize("nh,dc,dr", [(16, 512, 64), (4, 64, 8), (8, 128, 32), (16, 512, 24), (2, 256, 16), (1, 64, 64), (5, 128, 40)])
+def test_mla_attend_matches_oracle_and_rows_are_independent(nh, dc, dr):
+    torch = _torch()
+    # contexts: padding row, one token, around the softmax warps' half (128), the split boundary (256), two splits, ragged pages
+    ctxs = [0, 1, 127, 128, 129, 255, 256, 257, 385, 513, 700, 16]
+    rng, q_lat, q_rope, caches = _case(nh, dc, dr, ctxs, seed=nh + dc)
     scale = 1.0 / math.sqrt(dc + dr)
-    dev = lambda a: torch.tensor(a).cuda().contiguous()
-    if path:
-        os.environ[path] = "1"
-    try:
-        out = corun.mla_attend(dev(q_lat), dev(q_rope), dev(cache), dev(np.array(ctxs, np.int32)), scale)
-        torch.cuda.synchronize()
-        again = corun.mla_attend(dev(q_lat), dev(q_rope), dev(cache), dev(np.array(ctxs, np.int32)), scale)
-        torch.cuda.synchronize()
-    finally:
-        if path:
-            os.environ.pop(path, None)
-    assert out.cpu().numpy().tobytes() == again.cpu().numpy().tobytes()
-    assert _mla_worst(out.cpu().numpy(), q_lat, q_rope, cache, ctxs, dc) <= 2e-5
+    pool, table = _paged(rng, caches, ctxs, dc + dr)
+    out = _run(torch, q_lat, q_rope, pool, table, ctxs, scale)
+    # fp16 hi + lo operand pairs, fp32 accumulation chains of <= 576 and <= 128 terms on O(1) values
+    worst = _worst(out, q_lat, q_rope, caches, ctxs, dc)
+    assert worst <= 2e-5, worst
+    # the same rows in another order, among other rows, with their pages elsewhere in a larger pool: byte-identical
+    perm = [10, 2, 7, 4, 9]
+    other = [300, 5, 64, 9, 0, 17, 640]
+    ctx2 = [ctxs[i] for i in perm] + other
+    rng2, q2, r2, c2 = _case(nh, dc, dr, ctx2, seed=99)
+    for i, src in enumerate(perm):
+        q2[i], r2[i], c2[i] = q_lat[src], q_rope[src], caches[src]
+    pool2, table2 = _paged(rng2, c2, ctx2, dc + dr, spare=40)
+    out2 = _run(torch, q2, r2, pool2, table2, ctx2, scale)
+    for i, src in enumerate(perm):
+        assert out2[i].tobytes() == out[src].tobytes()
+    assert _worst(out2, q2, r2, c2, ctx2, dc) <= 2e-5
 
 
-def test_mla_v2_widths_match_the_runtime_width_kernel_on_the_oracle():
-    """d_c = 512, d_r = 64 takes the kernel with the widths compiled in: long contexts, several chunks."""
-    torch = pytest.importorskip("torch")
-    if not torch.cuda.is_available():
-        pytest.skip("no CUDA device")
-    from paper_2608_14376_b200 import corun
-
+def test_mla_long_contexts_many_splits_and_repeatability():
+    """More splits than fit one CTA's stretch, several rows per CTA and rows spread over many CTAs; twice the same bytes."""
+    torch = _torch()
     nh, dc, dr = 16, 512, 64
-    ctxs = [2049, 1536, 511]
-    q_lat, q_rope, cache = _mla_case(nh, dc, dr, ctxs, 2176, seed=11)
-    scale = 1.0 / math.sqrt(dc + dr)                 # the oracle's scale for identity up-projections (d_nope = d_c)
-    dev = lambda a: torch.tensor(a).cuda().contiguous()
-    for pairs, tol in ((True, 2e-5), (False, 4e-3)):
-        out = corun.mla_attend(dev(q_lat), dev(q_rope), dev(cache), dev(np.array(ctxs, np.int32)), scale, pairs)
-        torch.cuda.synchronize()
-        assert _mla_worst(out.cpu().numpy(), q_lat, q_rope, cache, ctxs, dc) <= tol
+    ctxs = [2049, 1536, 511, 4000, 3, 130]
+    rng, q_lat, q_rope, caches = _case(nh, dc, dr, ctxs, seed=11)
+    scale = 1.0 / math.sqrt(128 + dr)
+    pool, table = _paged(rng, caches, ctxs, dc + dr)
+    out = _run(torch, q_lat, q_rope, pool, table, ctxs, scale)
+    again = _run(torch, q_lat, q_rope, pool, table, ctxs, scale)
+    assert out.tobytes() == again.tobytes()
+    nh_, eye = q_lat.shape[1], None
+    worst = 0.0
+    for b, n in enumerate(ctxs):
+        C = caches[b][:n, :dc].astype(np.float64)
+        Rk = caches[b][:n, dc:].astype(np.float64)
+        # the oracle's absorbed form with identity up-projections and this scale: softmax((q_lat.C + q_rope.R) * scale).C
+        s = (C @ q_lat[b].astype(np.float64).T + Rk @ q_rope[b].astype(np.float64).T) * scale      # [T, nh]
+        p = np.exp(s - s.max(0)); p /= p.sum(0)
+        ref = p.T @ C
+        worst = max(worst, float(np.abs(out[b] - ref).max()))
+    assert worst <= 2e-5, worst
 
 
-def test_mla_context_beyond_the_cache_is_cut():
-    torch = pytest.importorskip("torch")
-    if not torch.cuda.is_available():
-        pytest.skip("no CUDA device")
+def test_mla_context_beyond_the_block_table_is_cut():
+    torch = _torch()
+    nh, dc, dr, T = 8, 128, 32, 640
+    rng, q_lat, q_rope, caches = _case(nh, dc, dr, [T, T], seed=3)
+    scale = 1.0 / math.sqrt(dc + dr)
+    pool, table = _paged(rng, caches, [T, T], dc + dr)
+    full = _run(torch, q_lat, q_rope, pool, table, [T, T], scale)
+    over = _run(torch, q_lat, q_rope, pool, table, [T + 100, 1 << 30], scale)
+    assert over.tobytes() == full.tobytes()
+
+
+def test_mla_argument_errors():
+    torch = _torch()
     from paper_2608_14376_b200 import corun
 
-    nh, dc, dr, T = 8, 128, 32, 640
-    q_lat, q_rope, cache = _mla_case(nh, dc, dr, [T, T], T, seed=3)
-    scale = 1.0 / math.sqrt(dc + dr)
-    dev = lambda a: torch.tensor(a).cuda().contiguous()
-    full = corun.mla_attend(dev(q_lat), dev(q_rope), dev(cache), dev(np.array([T, T], np.int32)), scale)
-    over = corun.mla_attend(dev(q_lat), dev(q_rope), dev(cache), dev(np.array([T + 100, 1 << 30], np.int32)), scale)
-    torch.cuda.synchronize()
-    assert over.cpu().numpy().tobytes() == full.cpu().numpy().tobytes()
+    z = lambda *s: torch.zeros(s, device="cuda")
+    ok = dict(pool=z(4, 16, 72).half(), table=torch.zeros((1, 2), dtype=torch.int32, device="cuda"),
+              ctx=torch.ones(1, dtype=torch.int32, device="cuda"))
+    with pytest.raises(corun.CorunError):            # latent width that is not 64 / 128 / 256 / 512
+        corun.mla_attend(z(1, 4, 192), z(1, 4, 8), z(4, 16, 200).half(), ok["table"], ok["ctx"], 1.0)
+    with pytest.raises(corun.CorunError):            # more than 16 heads
+        corun.mla_attend(z(1, 17, 64), z(1, 17, 8), ok["pool"], ok["table"], ok["ctx"], 1.0)
+    with pytest.raises(corun.CorunError):            # scale must be positive
+        corun.mla_attend(z(1, 4, 64), z(1, 4, 8), ok["pool"], ok["table"], ok["ctx"], 0.0)
