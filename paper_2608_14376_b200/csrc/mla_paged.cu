@@ -91,6 +91,7 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   __shared__ int abort_flag;
   __shared__ float xs_mx[2][32], xs_sum[2][32];   // the two token halves of an item exchange maximum and sum
   __shared__ int row_start[MP_MAXB + 1];           // first item of every row
+  __shared__ int row_ctx[MP_MAXB];                 // cached tokens of every row (cut to the block table's reach)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -124,7 +125,8 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
         int c = ctx[r];
         c = c < 0 ? 0 : (c > max_blocks * MP_PAGE ? max_blocks * MP_PAGE : c);
         n = (c + MP_T - 1) / MP_T;
-        if (n > max_splits) n = max_splits;
+        if (n > max_splits) { n = max_splits; c = n * MP_T; }
+        row_ctx[r] = c;
       }
       int inc = n;
 #pragma unroll
@@ -158,11 +160,7 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
     r = cur_row;
     split = item - row_start[cur_row];
   };
-  auto tokens_of = [&](int r, int split) {
-    int c = ctx[r];
-    c = c > max_blocks * MP_PAGE ? max_blocks * MP_PAGE : c;
-    return min(MP_T, c - split * MP_T);
-  };
+  auto tokens_of = [&](int r, int split) { return min(MP_T, row_ctx[r] - split * MP_T); };
 
   if (warp == 0) {
     // ---------------- producer ----------------
@@ -174,13 +172,18 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
       bool ok = mbar_wait(smem_u32(&empty_bar[unit % MP_RING]), (uint32_t)(unit / MP_RING - 1) & 1u, &abort_flag);
       return (bool)__all_sync(0xffffffffu, ok);
     };
+    auto pages_of = [&](int it, int &n) {             // lane l: page l of the item (0 beyond its pages)
+      if (it >= item_hi) { n = 0; return 0; }
+      int r, split;
+      locate(it, r, split);
+      n = (tokens_of(r, split) + MP_PAGE - 1) / MP_PAGE;
+      return lane < n ? __ldg(block_table + (size_t)r * max_blocks + split * MP_PAGES + lane) : 0;
+    };
+    int np_ahead = 0, page_ahead = pages_of(item_lo, np_ahead);
     for (int it = item_lo; it <= item_hi && !failed; ++it) {
-      int page = 0, np = 0;
+      const int page = page_ahead, np = np_ahead;      // looked up one item ahead of its use
+      page_ahead = pages_of(it + 1, np_ahead);
       if (it < item_hi) {
-        int r, split;
-        locate(it, r, split);
-        np = (tokens_of(r, split) + MP_PAGE - 1) / MP_PAGE;
-        page = lane < np ? block_table[(size_t)r * max_blocks + split * MP_PAGES + lane] : 0;
         for (int j = 0; j <= NLB; ++j, ++u) {           // latent blocks, then the rope block
           if (!slot_free(u)) { failed = true; break; }
           const uint32_t bar = smem_u32(&full_bar[u % MP_RING]);
@@ -289,19 +292,36 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { failed = true; break; }
       }
-      for (int i = qtid; i < total; i += 128) {
-        const int h = i / chunks, d = (i - h * chunks) << 3;
-        const float *src = d < d_c ? q_lat + ((size_t)r * n_heads + h) * d_c + d : q_rope + ((size_t)r * n_heads + h) * d_r + (d - d_c);
-        const float4 x0 = __ldg(reinterpret_cast<const float4 *>(src)), x1 = __ldg(reinterpret_cast<const float4 *>(src) + 1);
-        uint4 hi, lo;
-        mp_split2(x0.x, x0.y, hi.x, lo.x);
-        mp_split2(x0.z, x0.w, hi.y, lo.y);
-        mp_split2(x1.x, x1.y, hi.z, lo.z);
-        mp_split2(x1.z, x1.w, hi.w, lo.w);
-        const int blk = d < d_c ? (d >> 6) : NLB, cc = d < d_c ? ((d & 63) >> 3) : ((d - d_c) >> 3);
-        uint8_t *t = q_ptr + (size_t)blk * MP_QBLK;
-        *reinterpret_cast<uint4 *>(t + mp_swz(2 * h, cc)) = hi;
-        *reinterpret_cast<uint4 *>(t + mp_swz(2 * h + 1, cc)) = lo;
+      for (int i0 = qtid; i0 < total; i0 += 3 * 128) {   // three chunks per thread at a time: their loads overlap
+        float4 x0[3], x1[3];
+        int hh[3], dd[3];
+#pragma unroll
+        for (int e = 0; e < 3; ++e) {
+          const int i = i0 + e * 128;
+          hh[e] = -1;
+          if (i < total) {
+            const int h = i / chunks, d = (i - h * chunks) << 3;
+            const float *src = d < d_c ? q_lat + ((size_t)r * n_heads + h) * d_c + d : q_rope + ((size_t)r * n_heads + h) * d_r + (d - d_c);
+            x0[e] = __ldg(reinterpret_cast<const float4 *>(src));
+            x1[e] = __ldg(reinterpret_cast<const float4 *>(src) + 1);
+            hh[e] = h;
+            dd[e] = d;
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 3; ++e) {
+          if (hh[e] < 0) continue;
+          const int h = hh[e], d = dd[e];
+          uint4 hi, lo;
+          mp_split2(x0[e].x, x0[e].y, hi.x, lo.x);
+          mp_split2(x0[e].z, x0[e].w, hi.y, lo.y);
+          mp_split2(x1[e].x, x1[e].y, hi.z, lo.z);
+          mp_split2(x1[e].z, x1[e].w, hi.w, lo.w);
+          const int blk = d < d_c ? (d >> 6) : NLB, cc = d < d_c ? ((d & 63) >> 3) : ((d - d_c) >> 3);
+          uint8_t *t = q_ptr + (size_t)blk * MP_QBLK;
+          *reinterpret_cast<uint4 *>(t + mp_swz(2 * h, cc)) = hi;
+          *reinterpret_cast<uint4 *>(t + mp_swz(2 * h + 1, cc)) = lo;
+        }
       }
       fence_proxy_async();
       __syncwarp();
@@ -443,35 +463,46 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   if (warp == 0) tmem_dealloc(tmem_base, MP_TMEM_COLS);
 }
 
-// One warp per (row, head): the row's splits in ascending order -> o_lat.
+// One block per (row, head), one thread per four latent dims: the row's splits in ascending order -> o_lat.
 __global__ void __launch_bounds__(128) mla_paged_combine_kernel(const float2 *__restrict__ part_ml, const float *__restrict__ part_o,
                                                                 const int *__restrict__ ctx, int B, int n_heads, int d_c,
                                                                 int max_blocks, int max_splits, float *__restrict__ o_lat) {
-  const int w = (int)blockIdx.x * 4 + ((int)threadIdx.x >> 5), lane = threadIdx.x & 31;
-  if (w >= B * n_heads) return;
-  const int r = w / n_heads, h = w - r * n_heads;
+  const int r = (int)blockIdx.x / n_heads, h = (int)blockIdx.x - r * n_heads;
+  const int d = 4 * (int)threadIdx.x;
   int c = ctx[r];
-  if (c <= 0) return;                               // a padding row is left alone
+  if (c <= 0 || d >= d_c) return;                   // a padding row is left alone
+  griddep_wait();
   c = c > max_blocks * MP_PAGE ? max_blocks * MP_PAGE : c;
   int ns = (c + MP_T - 1) / MP_T;
   if (ns > max_splits) ns = max_splits;
   const float2 *ml = part_ml + (size_t)r * max_splits * n_heads + h;
   float M = -CUDART_INF_F;
-  for (int s = 0; s < ns; ++s) M = fmaxf(M, ml[(size_t)s * n_heads].x);
+  for (int s = 0; s < ns; ++s) M = fmaxf(M, __ldcg(&ml[(size_t)s * n_heads]).x);
   float den = 0.f;
-  for (int s = 0; s < ns; ++s) den += exp2f(ml[(size_t)s * n_heads].x - M) * ml[(size_t)s * n_heads].y;
-  const float inv = 1.f / den;
-  const float *po = part_o + ((size_t)r * max_splits * n_heads + h) * d_c;
-  const size_t stride = (size_t)n_heads * d_c;
-  for (int d = 4 * lane; d < d_c; d += 128) {
-    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < ns; ++s) {
-      const float ws = exp2f(ml[(size_t)s * n_heads].x - M);
-      const float4 x = __ldcg(reinterpret_cast<const float4 *>(po + (size_t)s * stride + d));
-      o.x = fmaf(ws, x.x, o.x); o.y = fmaf(ws, x.y, o.y); o.z = fmaf(ws, x.z, o.z); o.w = fmaf(ws, x.w, o.w);
-    }
-    *reinterpret_cast<float4 *>(o_lat + ((size_t)r * n_heads + h) * d_c + d) = make_float4(o.x * inv, o.y * inv, o.z * inv, o.w * inv);
+  for (int s = 0; s < ns; ++s) {
+    const float2 v = __ldcg(&ml[(size_t)s * n_heads]);
+    den += exp2f(v.x - M) * v.y;
   }
+  const float inv = 1.f / den;
+  const float *po = part_o + ((size_t)r * max_splits * n_heads + h) * d_c + d;
+  const size_t stride = (size_t)n_heads * d_c;
+  float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s0 = 0; s0 < ns; s0 += 4) {              // four splits' loads in flight; the sums stay in ascending order
+    float4 x[4];
+    float w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (s0 + e < ns) {
+        x[e] = __ldcg(reinterpret_cast<const float4 *>(po + (size_t)(s0 + e) * stride));
+        w[e] = exp2f(__ldcg(&ml[(size_t)(s0 + e) * n_heads]).x - M);
+      }
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (s0 + e < ns) {
+        o.x = fmaf(w[e], x[e].x, o.x); o.y = fmaf(w[e], x[e].y, o.y); o.z = fmaf(w[e], x[e].z, o.z); o.w = fmaf(w[e], x[e].w, o.w);
+      }
+  }
+  *reinterpret_cast<float4 *>(o_lat + ((size_t)r * n_heads + h) * d_c + d) = make_float4(o.x * inv, o.y * inv, o.z * inv, o.w * inv);
 }
 
 }  // namespace
@@ -528,7 +559,7 @@ int corun_mla_attend(const float *q_lat, const float *q_rope, const void *pool, 
     ce = launch_k(mla_paged_kernel, dim3(sms), dim3(MP_THREADS), MP_SMEM, st, false, tm, tv, q_lat, q_rope, block_table, max_blocks, ctx, B,
                   n_heads, d_latent, d_rope, scale * 1.4426950408889634f, max_splits, part_ml, part_o, status);
   if (ce == cudaSuccess)
-    ce = launch_k(mla_paged_combine_kernel, dim3((B * n_heads + 3) / 4), dim3(128), 0, st, false, part_ml, part_o, ctx, B, n_heads,
+    ce = launch_k(mla_paged_combine_kernel, dim3(B * n_heads), dim3(128), 0, st, true, part_ml, part_o, ctx, B, n_heads,
                   d_latent, max_blocks, max_splits, o_lat);
   if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
   return CORUN_OK;
