@@ -295,6 +295,135 @@ int orc_forward_ex(const orc_shape *sh, const orc_weights *w, const orc_moe *moe
   return 0;
 }
 
+/* ---- multi-head latent attention (MLA) decoder ----
+ *
+ * The paper evaluates one model with MLA and Mixture-of-Experts layers (Evaluation, "Setup") without giving
+ * the layer's formulas; this is the published definition of that layer, in the form that caches one latent
+ * vector per token (the same definition oracle/mla_oracle.py states for a single query):
+ *   a = RMSNorm(h);  [q | kv_a] = W_qkv a,  q: nh heads of (nope + rope) dims,  kv_a: rank + rope dims
+ *   c_t = RMSNorm(kv_a[:rank]) * g_kv            the cached latent of the token
+ *   r_t = RoPE(kv_a[rank:], t)                   the cached rotary key, shared by all heads
+ *   per head h, with W_kv_b's block h = [W_uk (nope rows) ; W_uv (v rows)], both [.., rank]:
+ *     k_nope[t] = W_uk c_t,  v[t] = W_uv c_t
+ *     s_t = (q_nope . k_nope[t] + RoPE(q_rope, p) . r_t) / sqrt(nope + rope),  t = 0..p
+ *     o_h = sum_t softmax(s)_t v[t]
+ *   y = W_o [o_0 | o_1 | ...]
+ * RoPE is the half-split rotation of orc_rope on the rope dims.  Layers below first_dense have the dense SwiGLU
+ * feed-forward of orc_forward_ex (width sh->ffn), the others the Mixture-of-Experts block (moe may be NULL: all
+ * layers dense).  sh->n_q_heads = nh; sh->n_kv_heads and sh->head_dim are not used.
+ */
+typedef struct {
+  int32_t kv_lora_rank, qk_nope, qk_rope, v_head, first_dense;
+  const uint16_t *const *kv_norm; /* L x [rank]                      */
+  const uint16_t *const *wkv_b;   /* L x [nh * (nope + v), rank]     */
+} orc_mla;
+
+/* One query token at position p over cached rows 0..p.  q: [nh][nope + rope] (rope part already rotated);
+ * Cc: cache rows of rank + rope floats, `stride` floats apart; out: [nh][v]. */
+void orc_mla_attention(const float *q, const float *Cc, int64_t stride, int64_t p, int32_t nh, int32_t rank,
+                       int32_t nope, int32_t rope, int32_t vh, const uint16_t *wkv_b, float *out) {
+  const double scale = 1.0 / sqrt((double)(nope + rope));
+#pragma omp parallel for schedule(static)
+  for (int32_t h = 0; h < nh; ++h) {
+    const uint16_t *Wuk = wkv_b + (int64_t)h * (nope + vh) * rank, *Wuv = Wuk + (int64_t)nope * rank;
+    const float *qh = q + (int64_t)h * (nope + rope);
+    double *s = (double *)malloc(sizeof(double) * (size_t)(p + 1));
+    double *kn = (double *)malloc(sizeof(double) * (size_t)nope);
+    double m = -INFINITY;
+    for (int64_t t = 0; t <= p; ++t) {
+      const float *c = Cc + t * stride;
+      double d = 0.0;
+      for (int32_t i = 0; i < nope; ++i) {            /* k_nope[t] = W_uk c_t, then its product with q_nope */
+        double k = 0.0;
+        for (int32_t j = 0; j < rank; ++j) k += bf16_to_f64(Wuk[(int64_t)i * rank + j]) * (double)c[j];
+        kn[i] = k;
+      }
+      for (int32_t i = 0; i < nope; ++i) d += (double)qh[i] * kn[i];
+      for (int32_t i = 0; i < rope; ++i) d += (double)qh[nope + i] * (double)c[rank + i];
+      s[t] = d * scale;
+      if (s[t] > m) m = s[t];
+    }
+    double z = 0.0;
+    for (int64_t t = 0; t <= p; ++t) { s[t] = exp(s[t] - m); z += s[t]; }
+    for (int32_t i = 0; i < vh; ++i) {
+      double o = 0.0;
+      for (int64_t t = 0; t <= p; ++t) {              /* v[t] = W_uv c_t, weighted */
+        const float *c = Cc + t * stride;
+        double v = 0.0;
+        for (int32_t j = 0; j < rank; ++j) v += bf16_to_f64(Wuv[(int64_t)i * rank + j]) * (double)c[j];
+        o += s[t] * v;
+      }
+      out[(int64_t)h * vh + i] = (float)(o / z);
+    }
+    free(s); free(kn);
+  }
+}
+
+/* As orc_forward_ex for the MLA decoder.  Cc: the request's cache, [L][max_T][rank + rope] fp32. */
+int orc_forward_mla(const orc_shape *sh, const orc_weights *w, const orc_mla *ml, const orc_moe *moe,
+                    const int32_t *tokens, int64_t T, int64_t pos0, float *Cc, int64_t max_T, float *logits,
+                    int all_logits) {
+  const int64_t H = sh->hidden, nh = sh->n_q_heads, F = sh->ffn, Vn = sh->vocab, L = sh->n_layers;
+  const int64_t rank = ml->kv_lora_rank, nope = ml->qk_nope, rope = ml->qk_rope, vh = ml->v_head;
+  const int64_t QD = nh * (nope + rope), CD = rank + rope, QKV = QD + CD, OD = nh * vh;
+  if (T <= 0 || pos0 < 0 || pos0 + T > max_T || rope % 2 || ml->first_dense < 0 || (!moe && ml->first_dense < L)) return -1;
+  for (int64_t t = 0; t < T; ++t)
+    if (tokens[t] < 0 || tokens[t] >= Vn) return -1;
+  int64_t wide = H > F ? H : F;
+  float *h = (float *)malloc(sizeof(float) * T * H);
+  float *a = (float *)malloc(sizeof(float) * T * wide);
+  float *qkv = (float *)malloc(sizeof(float) * T * QKV);
+  float *o = (float *)malloc(sizeof(float) * T * OD);
+  float *y = (float *)malloc(sizeof(float) * T * H);
+  float *gu = (float *)malloc(sizeof(float) * T * 2 * F);
+  for (int64_t t = 0; t < T; ++t)
+    for (int64_t i = 0; i < H; ++i) h[t * H + i] = (float)bf16_to_f64(w->embed[(int64_t)tokens[t] * H + i]);
+  for (int64_t l = 0; l < L; ++l) {
+    float *Cl = Cc + l * max_T * CD;
+    for (int64_t t = 0; t < T; ++t) orc_rmsnorm(h + t * H, w->attn_norm[l], H, sh->rms_eps, a + t * H);
+    orc_matmul_bf16(w->wqkv[l], QKV, H, a, T, qkv);
+    for (int64_t t = 0; t < T; ++t) {
+      float *row = qkv + t * QKV;
+      const int64_t p = pos0 + t;
+      for (int64_t j = 0; j < nh; ++j) orc_rope(row + j * (nope + rope) + nope, (int32_t)rope, p, sh->rope_theta);
+      orc_rmsnorm(row + QD, ml->kv_norm[l], rank, sh->rms_eps, Cl + p * CD);
+      orc_rope(row + QD + rank, (int32_t)rope, p, sh->rope_theta);
+      memcpy(Cl + p * CD + rank, row + QD + rank, sizeof(float) * rope);
+    }
+    for (int64_t t = 0; t < T; ++t)
+      orc_mla_attention(qkv + t * QKV, Cl, CD, pos0 + t, (int32_t)nh, (int32_t)rank, (int32_t)nope, (int32_t)rope,
+                        (int32_t)vh, ml->wkv_b[l], o + t * OD);
+    orc_matmul_bf16(w->wo[l], H, OD, o, T, y);
+    for (int64_t i = 0; i < T * H; ++i) h[i] = h[i] + y[i];
+    for (int64_t t = 0; t < T; ++t) orc_rmsnorm(h + t * H, w->mlp_norm[l], H, sh->rms_eps, a + t * H);
+    if (l >= ml->first_dense) {                     /* Mixture-of-Experts feed-forward layer */
+#pragma omp parallel for schedule(dynamic)
+      for (int64_t t = 0; t < T; ++t) orc_moe_ffn(moe, l, H, a + t * H, y + t * H, NULL, NULL);
+      for (int64_t i = 0; i < T * H; ++i) h[i] = h[i] + y[i];
+      continue;
+    }
+    orc_matmul_bf16(w->wgate_up[l], 2 * F, H, a, T, gu);
+    for (int64_t t = 0; t < T; ++t)
+      for (int64_t i = 0; i < F; ++i) {
+        double g = gu[t * 2 * F + i], u = gu[t * 2 * F + F + i];
+        a[t * F + i] = (float)(orc_silu(g) * u);
+      }
+    orc_matmul_bf16(w->wdown[l], H, F, a, T, y);
+    for (int64_t i = 0; i < T * H; ++i) h[i] = h[i] + y[i];
+  }
+  if (logits) {
+    if (all_logits) {
+      for (int64_t t = 0; t < T; ++t) orc_rmsnorm(h + t * H, w->final_norm, H, sh->rms_eps, a + t * H);
+      orc_matmul_bf16(w->lm_head, Vn, H, a, T, logits);
+    } else {
+      orc_rmsnorm(h + (T - 1) * H, w->final_norm, H, sh->rms_eps, a);
+      orc_matmul_bf16(w->lm_head, Vn, H, a, 1, logits);
+    }
+  }
+  free(h); free(a); free(qkv); free(o); free(y); free(gu);
+  return 0;
+}
+
 int orc_forward(const orc_shape *sh, const orc_weights *w, const int32_t *tokens, int64_t T, int64_t pos0,
                 float *Kc, float *Vc, int64_t max_T, float *logits, int all_logits) {
   return orc_forward_ex(sh, w, NULL, tokens, T, pos0, Kc, Vc, max_T, logits, all_logits);

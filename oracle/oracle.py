@@ -53,6 +53,11 @@ class _Moe(C.Structure):
         ("router", _PP), ("gate_up", _PP), ("down", _PP)]
 
 
+class _Mla(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("kv_lora_rank", "qk_nope", "qk_rope", "v_head", "first_dense")] + [
+        ("kv_norm", _PP), ("wkv_b", _PP)]
+
+
 def lib():
     global _lib
     if _lib is None:
@@ -63,6 +68,11 @@ def lib():
         L.orc_forward_ex.restype = C.c_int
         L.orc_forward_ex.argtypes = [C.POINTER(_Shape), C.POINTER(_Weights), C.POINTER(_Moe), C.c_void_p, C.c_int64,
                                      C.c_int64, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int]
+        L.orc_forward_mla.restype = C.c_int
+        L.orc_forward_mla.argtypes = [C.POINTER(_Shape), C.POINTER(_Weights), C.POINTER(_Mla), C.POINTER(_Moe), C.c_void_p,
+                                      C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int]
+        L.orc_mla_attention.restype = None
+        L.orc_mla_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64] + [C.c_int32] * 5 + [C.c_void_p, C.c_void_p]
         L.orc_moe_ffn.restype = None
         L.orc_moe_ffn.argtypes = [C.POINTER(_Moe), C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.orc_matmul_bf16.restype = None
@@ -135,8 +145,9 @@ class Model:
     wgate_up / wdown entries are then unused (any placeholders).
     """
 
-    def __init__(self, shape: Shape, weights: dict, moe: dict = None):
+    def __init__(self, shape: Shape, weights: dict, moe: dict = None, mla: dict = None):
         self.shape = shape
+        self.mla = None
         self._keep = {k: ([_u16(x) for x in v] if isinstance(v, (list, tuple)) else _u16(v))
                       for k, v in weights.items()}
         sh = shape
@@ -162,6 +173,18 @@ class Model:
             self._cm = cm
             self.moe = dict(moe)
 
+        if mla is not None:
+            # MLA decoder: wqkv is [nh*(nope+rope) + rank + rope, H], wo [H, nh*v]; kv_norm L x [rank], wkv_b L x
+            # [nh*(nope+v), rank]; layers below first_dense are dense (wgate_up / wdown), the others MoE
+            self._mla_keep = {k: [_u16(x) for x in mla[k]] for k in ("kv_norm", "wkv_b")}
+            cl = _Mla(mla["kv_lora_rank"], mla["qk_nope"], mla["qk_rope"], mla["v_head"], mla["first_dense"])
+            for k in ("kv_norm", "wkv_b"):
+                arr = (C.c_void_p * sh.n_layers)(*[_ptr(x) for x in self._mla_keep[k]])
+                self._arrs["mla_" + k] = arr
+                setattr(cl, k, C.cast(arr, _PP))
+            self._cl = cl
+            self.mla = dict(mla)
+
     def moe_ffn_row(self, layer: int, x):
         """One row through the Mixture-of-Experts block of ``layer``: (y [H], ids [top_k], weights [top_k])."""
         x = _f32(x)
@@ -174,6 +197,8 @@ class Model:
 
     def new_cache(self, max_T: int):
         sh = self.shape
+        if self.mla is not None:                        # one latent + rotary key per token and layer
+            return (np.zeros((sh.n_layers, max_T, self.mla["kv_lora_rank"] + self.mla["qk_rope"]), np.float32), None)
         kd = sh.n_kv_heads * sh.head_dim
         return (np.zeros((sh.n_layers, max_T, kd), np.float32), np.zeros((sh.n_layers, max_T, kd), np.float32))
 
@@ -190,9 +215,14 @@ class Model:
             out = np.empty((T, self.shape.vocab), np.float32)
         elif want == "last":
             out = np.empty((self.shape.vocab,), np.float32)
-        rc = lib().orc_forward_ex(C.byref(self._cs), C.byref(self._cw), C.byref(self._cm) if self._cm is not None else None,
-                                  _ptr(toks), T, pos0, _ptr(K), _ptr(V), K.shape[1],
-                                  _ptr(out) if out is not None else None, 1 if want == "all" else 0)
+        if self.mla is not None:
+            rc = lib().orc_forward_mla(C.byref(self._cs), C.byref(self._cw), C.byref(self._cl),
+                                       C.byref(self._cm) if self._cm is not None else None, _ptr(toks), T, pos0, _ptr(K),
+                                       K.shape[1], _ptr(out) if out is not None else None, 1 if want == "all" else 0)
+        else:
+            rc = lib().orc_forward_ex(C.byref(self._cs), C.byref(self._cw), C.byref(self._cm) if self._cm is not None else None,
+                                      _ptr(toks), T, pos0, _ptr(K), _ptr(V), K.shape[1],
+                                      _ptr(out) if out is not None else None, 1 if want == "all" else 0)
         if rc != 0:
             raise ValueError("orc_forward: bad argument")
         return out

@@ -66,6 +66,28 @@ QWEN3_30B_A3B_MOE = dict(n_experts=128, top_k=8, expert_ffn=768, n_shared=0, ren
 QWEN3_30B_A3B_EFF = ModelShape(48, 2048, 32, 4, 128, 128 * 768, 151936, 1e-6, 1000000.0)
 
 
+# DeepSeek-V2-Lite-shaped decoder with multi-head latent attention: 27 layers, hidden 2048, 16 heads, latent 512,
+# per-head query 128 (no rope) + 64 (rope), value 128; layer 0 a dense feed-forward of 10944, the others 64 routed
+# experts of 1408 (top-6, probabilities as they are) plus 2 shared experts.  n_kv_heads / head_dim are placeholders.
+DEEPSEEK_V2_LITE = ModelShape(27, 2048, 16, 16, 128, 10944, 102400, 1e-6, 10000.0)
+DEEPSEEK_V2_LITE_MLA = dict(kv_lora_rank=512, qk_nope=128, qk_rope=64, v_head=128, first_dense=1)
+DEEPSEEK_V2_LITE_MOE = dict(n_experts=64, top_k=6, expert_ffn=1408, n_shared=2, renormalize=False)
+
+
+def mla_weight_bytes_per_step(sh: ModelShape, mla: dict, moe: dict) -> int:
+    """bf16 bytes of every matrix one decode step of the MLA decoder streams (all experts: none is skipped)."""
+    nh, rank, nope, rope, vh = sh.n_q_heads, mla["kv_lora_rank"], mla["qk_nope"], mla["qk_rope"], mla["v_head"]
+    attn = (nh * (nope + rope) + rank + rope) * sh.hidden + 2 * nh * (nope + vh) * rank - nh * vh * rank + sh.hidden * nh * vh
+    # the key up-projections are read from their transposed copy, W_kv_b once more as a whole for the values
+    dense = 3 * sh.ffn * sh.hidden
+    nd = mla["first_dense"]
+    per_moe = 0
+    if moe is not None and nd < sh.n_layers:
+        nb = moe["n_experts"] + moe["n_shared"]
+        per_moe = moe["n_experts"] * sh.hidden + 3 * nb * moe["expert_ffn"] * sh.hidden
+    return 2 * (sh.n_layers * attn + nd * dense + (sh.n_layers - nd) * per_moe + sh.vocab * sh.hidden)
+
+
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     """fp32 -> bf16 bit patterns, round to nearest even (format conversion only)."""
     u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
@@ -250,3 +272,95 @@ def mla_paged_case(B: int, d_k: int, ctx_lo: int, ctx_hi: int, seed: int, device
         table[b, :blocks[b]] = perm[k:k + blocks[b]]
         k += int(blocks[b])
     return pool, torch.tensor(table, device=device), torch.tensor(ctx, device=device)
+
+
+def _mla_tensor_list(sh: ModelShape, mla: dict):
+    nh, rank, nope, rope, vh = sh.n_q_heads, mla["kv_lora_rank"], mla["qk_nope"], mla["qk_rope"], mla["v_head"]
+    yield "embed", None, (sh.vocab, sh.hidden)
+    for l in range(sh.n_layers):
+        yield "wqkv", l, (nh * (nope + rope) + rank + rope, sh.hidden)
+        yield "wkv_b", l, (nh * (nope + vh), rank)
+        yield "wo", l, (sh.hidden, nh * vh)
+        if l < mla["first_dense"]:
+            yield "wgate_up", l, (2 * sh.ffn, sh.hidden)
+            yield "wdown", l, (sh.hidden, sh.ffn)
+    yield "lm_head", None, (sh.vocab, sh.hidden)
+
+
+def make_mla_weights_numpy(sh: ModelShape, mla: dict, seed: int = 0, std: float = 0.02):
+    """Weights of a decoder with multi-head latent attention as numpy uint16 (bf16 bits): (weights, mla) where
+    ``weights`` has the keys of ``make_weights_numpy`` (wqkv [nh*(nope+rope) + rank + rope, H], wo [H, nh*v];
+    wgate_up / wdown drawn for the layers below first_dense, one shared dummy array for the others) and ``mla`` is the given dict plus kv_norm
+    (ones) and wkv_b [nh*(nope+v), rank] per layer.  Draw order: embed, per layer wqkv, wkv_b, wo (, wgate_up,
+    wdown), then lm_head."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    w = {"attn_norm": [], "mlp_norm": [], "wqkv": [], "wo": [], "wgate_up": [], "wdown": []}
+    m = dict(mla, kv_norm=[], wkv_b=[])
+    dummy = np.zeros((1,), np.uint16)
+    for name, l, shape in _mla_tensor_list(sh, mla):
+        t = f32_to_bf16_bits(rng.standard_normal(shape, dtype=np.float32) * np.float32(std))
+        if l is None:
+            w[name] = t
+        elif name == "wkv_b":
+            m["wkv_b"].append(t)
+        else:
+            w[name].append(t)
+    one = f32_to_bf16_bits(np.ones(sh.hidden, np.float32))
+    w["final_norm"] = one.copy()
+    for l in range(sh.n_layers):
+        w["attn_norm"].append(one.copy())
+        w["mlp_norm"].append(one.copy())
+        m["kv_norm"].append(f32_to_bf16_bits(np.ones(mla["kv_lora_rank"], np.float32)))
+        if l >= mla["first_dense"]:
+            w["wgate_up"].append(dummy)
+            w["wdown"].append(dummy)
+    return w, m
+
+
+def mla_numpy_to_torch(w: dict, m: dict, device="cuda"):
+    """The same as CUDA bf16 tensors; the feed-forward placeholders of expert layers become None."""
+    import torch
+
+    def cv(a):
+        return torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16).to(device)
+
+    nd = m["first_dense"]
+    wt = {}
+    for k, v in w.items():
+        if k in ("wgate_up", "wdown"):
+            wt[k] = [cv(x) if l < nd else None for l, x in enumerate(v)]
+        else:
+            wt[k] = [cv(x) for x in v] if isinstance(v, list) else cv(v)
+    mt = {k: ([cv(x) for x in v] if isinstance(v, list) else v) for k, v in m.items()}
+    return wt, mt
+
+
+def make_mla_weights_torch(sh: ModelShape, mla: dict, seed: int = 0, std: float = 0.02, device="cuda"):
+    """The same recipe drawn on the device (for shapes too large for the host): (weights, mla)."""
+    import torch
+
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    w = {"attn_norm": [], "mlp_norm": [], "wqkv": [], "wo": [], "wgate_up": [], "wdown": []}
+    m = dict(mla, kv_norm=[], wkv_b=[])
+    for name, l, shape in _mla_tensor_list(sh, mla):
+        t = torch.empty(shape, dtype=torch.bfloat16, device=device)
+        rows = max(1, (1 << 27) // shape[1])
+        for r0 in range(0, shape[0], rows):
+            r1 = min(shape[0], r0 + rows)
+            t[r0:r1] = (torch.randn((r1 - r0, shape[1]), generator=g, device=device, dtype=torch.float32) * std).to(torch.bfloat16)
+        if l is None:
+            w[name] = t
+        elif name == "wkv_b":
+            m["wkv_b"].append(t)
+        else:
+            w[name].append(t)
+    w["final_norm"] = torch.ones(sh.hidden, dtype=torch.bfloat16, device=device)
+    for l in range(sh.n_layers):
+        w["attn_norm"].append(torch.ones(sh.hidden, dtype=torch.bfloat16, device=device))
+        w["mlp_norm"].append(torch.ones(sh.hidden, dtype=torch.bfloat16, device=device))
+        m["kv_norm"].append(torch.ones(mla["kv_lora_rank"], dtype=torch.bfloat16, device=device))
+        if l >= mla["first_dense"]:
+            w["wgate_up"].append(None)
+            w["wdown"].append(None)
+    return w, m
