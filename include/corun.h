@@ -51,7 +51,8 @@ typedef struct corun_engine corun_engine; /* opaque, owned by the library */
 /* Decoder shape.  arch 0 = dense GQA decoder: pre-norm RMSNorm, half-split
  * RoPE on q and k, causal softmax attention, SwiGLU FFN, untied LM head, no
  * biases.  Requirements: hidden, ffn and n_q_heads*head_dim multiples of 64;
- * head_dim 64 or 128; n_q_heads / n_kv_heads in {1,2,4,8}. */
+ * head_dim 64 or 128; n_q_heads / n_kv_heads in {1,2,4,8}.  arch is 0 here; the other
+ * architectures have their own creation calls (corun_init_moe, corun_init_mla), which take arch 0 too. */
 typedef struct {
   int32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
   float rms_eps, rope_theta;
@@ -113,6 +114,35 @@ typedef struct {
 int corun_init_moe(const corun_shape *shape, const corun_weights *weights, const corun_moe_layers *moe, int32_t B,
                    int32_t max_context, int32_t kv_block, int64_t kv_pool_blocks, void *cuda_stream,
                    corun_engine **out);
+
+/*
+ * The same engine for a decoder with multi-head latent attention (MLA) -- the paper evaluates one MLA /
+ * Mixture-of-Experts model (Evaluation, "Setup") -- at decode time in the absorbed form over a paged cache of
+ * one latent vector and one shared rotary key per token (include/corun_mla.h describes the attention):
+ *   [q | kv_a] = W_qkv RMSNorm(h):   q  = n_q_heads x [qk_nope | qk_rope],   kv_a = [kv_lora_rank | qk_rope]
+ *   cached per token (fp16):  c = RMSNorm(kv_a[:rank]) * kv_norm,  r = RoPE(kv_a[rank:]) (half-split rotation)
+ *   per head h, W_kv_b's block h = [W_uk (qk_nope rows) ; W_uv (v_head rows)] x rank:
+ *     q_lat = W_uk^T q_nope,  s_t = (q_lat . c_t + RoPE(q_rope) . r_t) / sqrt(qk_nope + qk_rope),
+ *     o_h = W_uv sum_t softmax(s)_t c_t;    y = W_o [o_0 | o_1 | ...]
+ * shape->n_q_heads heads (at most 16); shape->n_kv_heads and shape->head_dim are ignored.  Weights as in
+ * corun_weights except  wqkv [n_q_heads * (qk_nope + qk_rope) + rank + qk_rope, hidden]  and
+ * wo [hidden, n_q_heads * v_head].  Layers 0 .. first_dense-1 have the dense SwiGLU feed-forward of width
+ * shape->ffn (weights->wgate_up / wdown, entries of the other layers unused); the other layers are
+ * Mixture-of-Experts layers as in corun_init_moe (entries of moe's arrays below first_dense unused).  moe may
+ * be NULL when first_dense == n_layers.
+ *   kv_norm  L device pointers, bf16 [rank]          wkv_b  L device pointers, bf16 [n_q_heads * (qk_nope + v_head), rank]
+ * kv_lora_rank 256 or 512; qk_nope a multiple of 64; qk_rope even, a multiple of 8, at most 64;
+ * qk_nope + v_head a multiple of 256; n_q_heads * v_head a multiple of 64.  A decode step of B slots and a
+ * prefill chunk run the same kernels; a prefill row attends to its request's cache up to its own position.
+ * Errors as corun_init.
+ */
+typedef struct {
+  int32_t kv_lora_rank, qk_nope, qk_rope, v_head, first_dense;
+  const void *const *kv_norm, *const *wkv_b;
+} corun_mla_layers;
+int corun_init_mla(const corun_shape *shape, const corun_weights *weights, const corun_mla_layers *mla,
+                   const corun_moe_layers *moe, int32_t B, int32_t max_context, int32_t kv_block, int64_t kv_pool_blocks,
+                   void *cuda_stream, corun_engine **out);
 
 /*
  * Isolated prefill (paper, Design, "Isolated Prefill"; Algorithm 1's admission

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libcorun.so")
 OK, EINVAL, ESLOT, ENOSPACE, ECTX, ECUDA, ETIMEOUT, ENOMEM, ELIMIT = 0, -1, -2, -3, -4, -5, -6, -7, -8
 
 EXPORTS = [
-    "corun_init", "corun_init_moe", "corun_prefill", "corun_prefill_batch", "corun_decode_step", "corun_decode_enqueue", "corun_decode_wait",
+    "corun_init", "corun_init_moe", "corun_init_mla", "corun_prefill", "corun_prefill_batch", "corun_decode_step", "corun_decode_enqueue", "corun_decode_wait",
     "corun_release", "corun_destroy", "corun_get_logits", "corun_force_token", "corun_context_len",
     "corun_free_blocks", "corun_debug_kv_read", "corun_debug_kv_write", "corun_debug_adopt",
     "corun_debug_set_eager", "corun_debug_read", "corun_debug_kv_fill", "corun_debug_time_kernel", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
@@ -50,6 +50,12 @@ class MoeLayers(C.Structure):
     _fields_ = [("n_experts", C.c_int32), ("top_k", C.c_int32), ("expert_ffn", C.c_int32), ("n_shared", C.c_int32),
                 ("renormalize", C.c_int32), ("router", C.POINTER(C.c_void_p)), ("gate_up", C.POINTER(C.c_void_p)),
                 ("down", C.POINTER(C.c_void_p))]
+
+
+class MlaLayers(C.Structure):
+    """``corun_mla_layers``."""
+    _fields_ = [("kv_lora_rank", C.c_int32), ("qk_nope", C.c_int32), ("qk_rope", C.c_int32), ("v_head", C.c_int32),
+                ("first_dense", C.c_int32), ("kv_norm", C.POINTER(C.c_void_p)), ("wkv_b", C.POINTER(C.c_void_p))]
 
 
 class CorunError(RuntimeError):
@@ -177,10 +183,15 @@ class Engine:
     describes (see ``synth.make_weights_*``); they are borrowed, keep them alive.
     """
 
-    def __init__(self, shape, weights: dict, B: int, max_context: int, kv_pool_blocks: int = 0, stream=None, moe: dict = None):
+    def __init__(self, shape, weights: dict, B: int, max_context: int, kv_pool_blocks: int = 0, stream=None, moe: dict = None,
+                 mla: dict = None):
         """``moe``: Mixture-of-Experts feed-forward layers instead of the dense ones: a dict with n_experts, top_k,
         expert_ffn, n_shared, renormalize and lists of L CUDA bf16 tensors router [E, H], gate_up [(E+S)*2F, H],
-        down [H, (E+S)*F] (``weights`` then needs no wgate_up / wdown)."""
+        down [H, (E+S)*F] (``weights`` then needs no wgate_up / wdown).
+        ``mla``: multi-head latent attention layers (``corun_init_mla``): a dict with kv_lora_rank, qk_nope, qk_rope,
+        v_head, first_dense and lists of L CUDA bf16 tensors kv_norm [rank], wkv_b [nh*(nope+v), rank]; wqkv / wo of
+        ``weights`` then have the MLA shapes, layers below first_dense are dense (wgate_up / wdown entries; None for
+        the other layers), the others take ``moe`` (its entries below first_dense may be None)."""
         import torch
 
         self._torch = torch
@@ -195,28 +206,42 @@ class Engine:
             t = weights[k]
             assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
             setattr(cw, k, t.data_ptr())
-        for k in ("attn_norm", "wqkv", "wo", "mlp_norm") + (() if moe else ("wgate_up", "wdown")):
-            ts = weights[k]
+        def ptr_array(ts):
             assert len(ts) == d["n_layers"]
             for t in ts:
-                assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
-            arr = (C.c_void_p * len(ts))(*[t.data_ptr() for t in ts])
+                assert t is None or (t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous())
+            return (C.c_void_p * len(ts))(*[(t.data_ptr() if t is not None else None) for t in ts])
+
+        dense_needed = (not moe) or (mla is not None and mla["first_dense"] > 0)
+        for k in ("attn_norm", "wqkv", "wo", "mlp_norm") + (("wgate_up", "wdown") if dense_needed else ()):
+            arr = ptr_array(weights[k])
             self._arrs[k] = arr
             setattr(cw, k, C.cast(arr, _PP))
         self._cw = cw
         torch.cuda.synchronize()
         h = C.c_void_p()
+        cm = None
         if moe:
             cm = MoeLayers(moe["n_experts"], moe["top_k"], moe["expert_ffn"], moe["n_shared"], 1 if moe.get("renormalize") else 0)
             self._moe = moe
             for k in ("router", "gate_up", "down"):
-                ts = moe[k]
-                assert len(ts) == d["n_layers"]
-                for t in ts:
-                    assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
-                arr = (C.c_void_p * len(ts))(*[t.data_ptr() for t in ts])
+                arr = ptr_array(moe[k])
                 self._arrs["moe_" + k] = arr
                 setattr(cm, k, C.cast(arr, _PP))
+        if mla is not None:
+            cl = MlaLayers(mla["kv_lora_rank"], mla["qk_nope"], mla["qk_rope"], mla["v_head"], mla["first_dense"])
+            self._mla = mla
+            for k in ("kv_norm", "wkv_b"):
+                arr = ptr_array(mla[k])
+                self._arrs["mla_" + k] = arr
+                setattr(cl, k, C.cast(arr, _PP))
+            L = lib()
+            L.corun_init_mla.argtypes = [C.POINTER(Shape), C.POINTER(Weights), C.POINTER(MlaLayers), C.POINTER(MoeLayers), C.c_int32,
+                                         C.c_int32, C.c_int32, C.c_int64, C.c_void_p, C.POINTER(C.c_void_p)]
+            _check(L.corun_init_mla(C.byref(self._cs), C.byref(cw), C.byref(cl), C.byref(cm) if cm is not None else None, B,
+                                    max_context, 16, kv_pool_blocks, C.c_void_p(stream) if stream else None, C.byref(h)),
+                   "corun_init_mla")
+        elif moe:
             L = lib()
             L.corun_init_moe.argtypes = [C.POINTER(Shape), C.POINTER(Weights), C.POINTER(MoeLayers), C.c_int32, C.c_int32,
                                          C.c_int32, C.c_int64, C.c_void_p, C.POINTER(C.c_void_p)]
@@ -304,6 +329,10 @@ class Engine:
         return int(lib().corun_free_blocks(self._h))
 
     def kv_read(self, slot: int, layer: int, pos0: int, n: int):
+        if getattr(self, "_mla", None):                   # latent cache: rows of rank + rope values, no second array
+            k = np.empty((n, self._mla["kv_lora_rank"] + self._mla["qk_rope"]), np.float32)
+            _check(lib().corun_debug_kv_read(self._h, slot, layer, pos0, n, k.ctypes.data, None), "kv_read")
+            return k, None
         kd = self._cs.n_kv_heads * self._cs.head_dim
         k = np.empty((n, kd), np.float32)
         v = np.empty((n, kd), np.float32)
@@ -312,6 +341,9 @@ class Engine:
 
     def kv_write(self, slot: int, layer: int, pos0: int, k, v):
         k = np.ascontiguousarray(k, dtype=np.float32)
+        if v is None:                                     # latent cache
+            _check(lib().corun_debug_kv_write(self._h, slot, layer, pos0, k.shape[0], k.ctypes.data, None), "kv_write")
+            return
         v = np.ascontiguousarray(v, dtype=np.float32)
         _check(lib().corun_debug_kv_write(self._h, slot, layer, pos0, k.shape[0], k.ctypes.data, v.ctypes.data),
                "kv_write")

@@ -13,6 +13,7 @@
 #include "../../include/corun.h"
 #include "../../include/corun_debug.h"
 #include "gemm.cuh"
+#include "mla.cuh"
 #include "moe.cuh"
 #include "ops.cuh"
 
@@ -57,6 +58,15 @@ struct Program {
   bf16 *xg_hi = nullptr, *xg_lo = nullptr, *hg_hi = nullptr, *hg_lo = nullptr;
   float *gug_out = nullptr, *yg_out = nullptr;
   int *plain_tiles = nullptr;            // zeros: the table that makes a plain matrix readable as a GEMM result
+  // multi-head latent attention: head-major matrices of RPH rows per head for the grouped up-projections
+  // (p_uk: q_lat = W_uk^T q_nope; p_uv: [. | o] = W_kv_b o_lat), the attention's partials, and the dense
+  // feed-forward GEMMs of the layers that have no experts
+  int RPH = 0;
+  bf16 *qn_hi = nullptr, *qn_lo = nullptr, *ol_hi = nullptr, *ol_lo = nullptr;
+  float *q_lat = nullptr, *q_rope = nullptr, *uv_out = nullptr, *mla_po = nullptr;
+  float2 *mla_ml = nullptr;
+  int *tab_uk = nullptr, *tab_uv = nullptr;
+  GemmPlan p_uk, p_uv, p_gu_d, p_down_d;
   bool has_layers = false, has_lm = false;
   std::vector<void *> allocs;
 };
@@ -81,6 +91,15 @@ struct corun_engine {
   int moe_E = 0, moe_K = 0, moe_F = 0, moe_S = 0, moe_renorm = 0;
   bf16 *router_pad = nullptr;            // [L][256][H]: each layer's router rows, zero rows behind them
   std::vector<CUtensorMap> tm_router;
+  // multi-head latent attention (corun_init_mla): sh.head_dim is the value width, the cache holds rank + rope
+  // halfs per token; layers below first_dense have a dense feed-forward of width dense_ffn
+  bool mla = false;
+  MlaDims md{};
+  int first_dense = 0, dense_ffn = 0, mla_splits = 0;
+  std::vector<const bf16 *> kv_norm;
+  bf16 *w_ukT = nullptr;                 // [L][nh * rank][nope]: the key up-projections transposed
+  std::vector<CUtensorMap> tm_uk, tm_uv, tm_c, tm_cv, tm_gu_d, tm_down_d;
+  const void *w0_uv = nullptr, *w0_gu_d = nullptr, *w0_down_d = nullptr;
   // KV
   __half *kv_pool = nullptr;
   size_t layer_stride = 0;
@@ -141,6 +160,11 @@ int pad16(int x) { return (x + 15) / 16 * 16; }
 int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, bool grouped = false, bool fuse_swiglu = false) {
   const corun_shape &s = e->sh;
   const int H = s.hidden, QD = s.n_q_heads * s.head_dim, KD = s.n_kv_heads * s.head_dim, F = s.ffn, V = s.vocab;
+  const MlaDims &md = e->md;
+  // columns of the q / k / v (MLA: q / kv_a) projection
+  const int QKVN = e->mla ? md.nh * (md.nope + md.rope) + md.rank + md.rope : QD + 2 * KD;
+  const int Fd = e->dense_ffn;                      // MLA: width of the dense feed-forward layers beside expert layers
+  const int Fmax = F > Fd ? F : Fd;
   P.R = R;
   P.BN = pad16(R);
   P.has_layers = layers;
@@ -157,22 +181,56 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
   RC(dmalloc(A, &P.sampled, R));
   if (layers) {
     RC(dmalloc(A, &P.h, (size_t)R * H));
-    RC(dmalloc(A, &P.q, (size_t)R * QD));
-    RC(dmalloc(A, &P.part_acc, (size_t)R * s.n_q_heads * e->max_splits * s.head_dim));
-    RC(dmalloc(A, &P.part_ml, (size_t)R * s.n_q_heads * e->max_splits * 2));
-    RC(dmalloc(A, &P.att_work, (size_t)R * e->max_splits * e->sh.n_kv_heads));
-    RC(dmalloc(A, &P.att_n_work, 2 + 2 * (size_t)R * e->sh.n_kv_heads));
-    RC(dmalloc(A, &P.att_pool, (size_t)s.n_layers));
-    RC(dmalloc(A, &P.qkv_out, (size_t)R * (QD + 2 * KD)));
+    if (!e->mla) {
+      RC(dmalloc(A, &P.q, (size_t)R * QD));
+      RC(dmalloc(A, &P.part_acc, (size_t)R * s.n_q_heads * e->max_splits * s.head_dim));
+      RC(dmalloc(A, &P.part_ml, (size_t)R * s.n_q_heads * e->max_splits * 2));
+      RC(dmalloc(A, &P.att_work, (size_t)R * e->max_splits * e->sh.n_kv_heads));
+      RC(dmalloc(A, &P.att_n_work, 2 + 2 * (size_t)R * e->sh.n_kv_heads));
+      RC(dmalloc(A, &P.att_pool, (size_t)s.n_layers));
+    } else {
+      const int BG = mla_group_rows(P.BN), n_groups = md.nh * (mla_rows_per_head(P.BN) / BG);
+      P.RPH = mla_rows_per_head(P.BN);
+      const size_t hr = (size_t)md.nh * P.RPH;      // rows of the head-major matrices
+      RC(dmalloc(A, &P.qn_hi, hr * md.nope));
+      RC(dmalloc(A, &P.qn_lo, hr * md.nope));
+      RC(dmalloc(A, &P.q_lat, hr * md.rank));
+      RC(dmalloc(A, &P.q_rope, (size_t)R * md.nh * md.rope));
+      RC(dmalloc(A, &P.ol_hi, hr * md.rank));
+      RC(dmalloc(A, &P.ol_lo, hr * md.rank));
+      RC(dmalloc(A, &P.uv_out, hr * (md.nope + md.vh)));
+      RC(dmalloc(A, &P.mla_ml, (size_t)mla_part_ml_floats(R, md.nh, e->max_ctx) / 2));
+      RC(dmalloc(A, &P.mla_po, (size_t)mla_part_o_floats(R, md.nh, md.rank, e->max_ctx)));
+      RC(dmalloc(A, &P.tab_uk, (size_t)n_groups * 3));
+      RC(dmalloc(A, &P.tab_uv, (size_t)n_groups * 3));
+      std::vector<int> tk((size_t)n_groups * 3), tv((size_t)n_groups * 3);
+      for (int g = 0; g < n_groups; ++g) {          // group = (head, block of BG rows): its weight rows, rows in use
+        const int h = g / (P.RPH / BG), rb = g % (P.RPH / BG);
+        const int valid = R - rb * BG < BG ? (R - rb * BG > 0 ? R - rb * BG : 0) : BG;
+        tk[3 * g] = h * md.rank; tk[3 * g + 1] = 0; tk[3 * g + 2] = valid;
+        tv[3 * g] = h * (md.nope + md.vh); tv[3 * g + 1] = 0; tv[3 * g + 2] = valid;
+      }
+      CK(cudaMemcpy(P.tab_uk, tk.data(), tk.size() * sizeof(int), cudaMemcpyHostToDevice));
+      CK(cudaMemcpy(P.tab_uv, tv.data(), tv.size() * sizeof(int), cudaMemcpyHostToDevice));
+      RC(gemm_plan_create_grouped(&P.p_uk, e->w_ukT, (long long)md.nh * md.rank, md.nope, md.rank, md.nope, P.qn_hi, P.qn_lo, n_groups,
+                                  BG, P.q_lat, P.tab_uk));
+      RC(gemm_plan_create_grouped(&P.p_uv, e->w0_uv, (long long)md.nh * (md.nope + md.vh), md.rank, md.nope + md.vh, md.rank, P.ol_hi,
+                                  P.ol_lo, n_groups, BG, P.uv_out, P.tab_uv));
+    }
+    RC(dmalloc(A, &P.qkv_out, (size_t)R * QKVN));
     RC(dmalloc(A, &P.o_out, (size_t)R * H));
-    RC(dmalloc(A, &P.gu_out, (size_t)R * 2 * F));
+    RC(dmalloc(A, &P.gu_out, (size_t)R * 2 * Fmax));
     RC(dmalloc(A, &P.down_out, (size_t)R * H));
     RC(dmalloc(A, &P.ao_hi, (size_t)P.BN * QD));
     RC(dmalloc(A, &P.ao_lo, (size_t)P.BN * QD));
-    RC(dmalloc(A, &P.ff_hi, (size_t)P.BN * F));
-    RC(dmalloc(A, &P.ff_lo, (size_t)P.BN * F));
+    RC(dmalloc(A, &P.ff_hi, (size_t)P.BN * Fmax));
+    RC(dmalloc(A, &P.ff_lo, (size_t)P.BN * Fmax));
+    if (e->mla && e->moe_E && e->first_dense > 0) {   // the dense feed-forward layers of a decoder with expert layers
+      RC(gemm_plan_create(&P.p_gu_d, e->w0_gu_d, 2 * Fd, H, P.xn_hi, P.xn_lo, R, P.BN, P.gu_out, P.ws, e->num_sms));
+      RC(gemm_plan_create(&P.p_down_d, e->w0_down_d, H, Fd, P.ff_hi, P.ff_lo, R, P.BN, P.down_out, P.ws, e->num_sms));
+    }
     // the plans carry layer 0's weights; the per-layer tensor maps override them at launch
-    RC(gemm_plan_create(&P.p_qkv, e->w0_qkv, QD + 2 * KD, H, P.xn_hi, P.xn_lo, R, P.BN, P.qkv_out, P.ws, e->num_sms));
+    RC(gemm_plan_create(&P.p_qkv, e->w0_qkv, QKVN, H, P.xn_hi, P.xn_lo, R, P.BN, P.qkv_out, P.ws, e->num_sms));
     RC(gemm_plan_create(&P.p_o, e->w0_o, H, QD, P.ao_hi, P.ao_lo, R, P.BN, P.o_out, P.ws, e->num_sms));
     if (fuse_swiglu && !e->moe_E && P.BN <= 128)
       RC(gemm_plan_create_swiglu(&P.p_gu, e->w0_gu, F, H, P.xn_hi, P.xn_lo, R, P.BN, P.ff_hi, P.ff_lo, e->num_sms));
@@ -233,6 +291,10 @@ void program_destroy(Program &P) {
   gemm_plan_destroy(&P.p_r);
   gemm_plan_destroy(&P.p_gug);
   gemm_plan_destroy(&P.p_dng);
+  gemm_plan_destroy(&P.p_uk);
+  gemm_plan_destroy(&P.p_uv);
+  gemm_plan_destroy(&P.p_gu_d);
+  gemm_plan_destroy(&P.p_down_d);
   for (void *p : P.allocs) cudaFree(p);
   P.allocs.clear();
 }
@@ -244,7 +306,10 @@ KvLayout kv_layout(const corun_engine *e) {
 
 // The result of a layer's feed-forward part as the next kernel reads it: the down GEMM's partials, or (grouped
 // Mixture-of-Experts form) the combined plain matrix.
-GemmOut ffn_out(const Program &P) {
+bool dense_layer(const corun_engine *e, int layer) { return e->mla && e->moe_E && layer < e->first_dense; }
+
+GemmOut ffn_out(const corun_engine *e, const Program &P, int layer) {
+  if (dense_layer(e, layer)) return P.p_down_d.out();
   if (P.grouped) return GemmOut{P.down_out, nullptr, P.plain_tiles, P.plain_tiles, P.p_down.N, P.p_down.KB, P.BN};
   return P.p_down.out();
 }
@@ -255,7 +320,7 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
   const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
   const KvLayout kv = kv_layout(e);
   int n = 0;
-  if (&P == &e->dec) {                              // the prefill attention kernel needs no item list
+  if (&P == &e->dec && !e->mla) {                   // the prefill attention kernel needs no item list
     CK(launch_attn_worklist(rows, e->sh.n_kv_heads, P.att_work, P.att_n_work, P.att_pool, s.n_layers, e->whole_pairs, e->st));   // the same items serve every layer
     n += 1;
   }
@@ -272,18 +337,40 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
     ++stage;                                          \
   } while (0)
   for (int l = 0; l < s.n_layers; ++l) {
-    GemmOut prev = ffn_out(P);
+    GemmOut prev = ffn_out(e, P, l > 0 ? l - 1 : 0);
     STAGE(launch_resid_norm(P.h, s.hidden, e->embed, rows, l == 0 ? nullptr : &prev, e->attn_norm[l], s.rms_eps,
                             P.xn_hi, P.xn_lo, e->st));
     STAGE(gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, tr(4 * l + 0), true));
+    if (e->mla) {
+      // cache append and query parts -> q_lat = W_uk^T q_nope per head -> absorbed attention over the row's latent
+      // pages (decode rows and prefill rows alike) -> [. | o] = W_kv_b o_lat per head -> the value part, split
+      const MlaDims &md = e->md;
+      const MlaCache cache{e->kv_pool + (size_t)l * e->layer_stride, e->d_block_table, e->max_blocks, e->B, (long long)e->pool_blocks};
+      STAGE(launch_mla_post(P.p_qkv.out(), rows, e->d_rope, md, e->kv_norm[l], s.rms_eps, cache, P.RPH, P.qn_hi, P.qn_lo, P.q_rope,
+                            e->d_status, e->st));
+      STAGE(gemm_launch(P.p_uk, &e->tm_uk[l], e->d_status, e->st, nullptr, true));
+      STAGE(launch_mla_attention(e->tm_c[l], e->tm_cv[l], P.q_lat, md.rank, (long long)P.RPH * md.rank, P.q_rope, e->d_block_table,
+                                 e->max_blocks, nullptr, &rows, P.R, md, 1.0f / sqrtf((float)(md.nope + md.rope)), e->mla_splits,
+                                 P.mla_ml, P.mla_po, nullptr, P.ol_hi, P.ol_lo, P.RPH, e->num_sms, e->d_status, true, e->st));
+      STAGE(gemm_launch(P.p_uv, &e->tm_uv[l], e->d_status, e->st, nullptr, true));
+      STAGE(launch_mla_ao_split(P.uv_out, P.R, P.RPH, md, P.ao_hi, P.ao_lo, e->st));
+      n += 3 + (&P == &e->dec ? 0 : 1);               // beyond the count below: two grouped GEMMs, the split, and in prefill too a second attention kernel
+    } else {
     STAGE(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->d_status, e->st));
     STAGE(launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work, P.att_n_work,
                            e->num_sms, P.part_acc, P.part_ml, P.att_pool + l, P.ao_hi, P.ao_lo, &P == &e->dec ? (e->whole_pairs ? 2 : 0) : 1,
                            e->d_status, e->st));
+    }
     STAGE(gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st, tr(4 * l + 1), true));
     GemmOut o = P.p_o.out();
     STAGE(launch_resid_norm(P.h, s.hidden, nullptr, rows, &o, e->mlp_norm[l], s.rms_eps, P.xn_hi, P.xn_lo, e->st));
-    if (e->moe_E && P.grouped) {
+    if (dense_layer(e, l)) {
+      STAGE(gemm_launch(P.p_gu_d, &e->tm_gu_d[l], e->d_status, e->st, nullptr, true));
+      STAGE(launch_swiglu(P.p_gu_d.out(), P.R, e->dense_ffn, P.ff_hi, P.ff_lo, e->st));
+      STAGE(gemm_launch(P.p_down_d, &e->tm_down_d[l], e->d_status, e->st, nullptr, true));
+      n += 9 + (&P == &e->dec ? 1 : 0);
+      continue;
+    } else if (e->moe_E && P.grouped) {
       // router -> top-k weights -> rows grouped by expert -> gate / up, SwiGLU and down per group -> the row's
       // experts summed in ascending expert id
       const int NB = e->moe_E + e->moe_S;
@@ -335,7 +422,7 @@ int enqueue_decode_body(corun_engine *e, int *launches) {
   RC(run_layers(e, P, &n));
   if (!(e->eager && e->stop_after >= 0)) {   // (debug) a truncated layer stack skips the tail too
     const Rows rows{P.row_token, P.row_pos, P.row_active, P.row_slot, P.R};
-    GemmOut prev = ffn_out(P);
+    GemmOut prev = ffn_out(e, P, s.n_layers - 1);
     CK(launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->final_norm, s.rms_eps, P.xn_hi, P.xn_lo, e->st));
     CK(gemm_launch(P.p_lm, nullptr, e->d_status, e->st, nullptr, true));
     CK(gemm_fixup_launch(P.p_lm, e->st, true));
@@ -413,23 +500,44 @@ const char *corun_strerror(int st) {
   }
 }
 
-static int engine_create(const corun_shape *shape, const corun_weights *w, const corun_moe_layers *moe, int32_t B,
-                         int32_t max_context, int32_t kv_block, int64_t kv_pool_blocks, void *cuda_stream,
-                         corun_engine **out) {
+static int engine_create(const corun_shape *shape, const corun_weights *w, const corun_moe_layers *moe,
+                         const corun_mla_layers *mla, int32_t B, int32_t max_context, int32_t kv_block,
+                         int64_t kv_pool_blocks, void *cuda_stream, corun_engine **out) {
   if (!shape || !w || !out) return CORUN_EINVAL;
   *out = nullptr;
   corun_shape s = *shape;
+  if (s.n_layers < 1) return CORUN_EINVAL;
+  int first_dense = 0, dense_ffn = 0;                // MLA: layers with a dense feed-forward, and its width
+  if (mla) {
+    if (s.arch != 0 && s.arch != 1) return CORUN_EINVAL;
+    s.arch = 0;
+    if ((mla->kv_lora_rank != 256 && mla->kv_lora_rank != 512) || mla->qk_nope < 64 || mla->qk_nope % 64 || mla->qk_rope < 8 ||
+        mla->qk_rope > 64 || mla->qk_rope % 8 || mla->v_head < 64 || (mla->qk_nope + mla->v_head) % 256 || s.n_q_heads < 1 ||
+        s.n_q_heads > 16 || mla->first_dense < 0 || mla->first_dense > s.n_layers || (!moe && mla->first_dense != s.n_layers) ||
+        !mla->kv_norm || !mla->wkv_b)
+      return CORUN_EINVAL;
+    for (int l = 0; l < s.n_layers; ++l)
+      if (!mla->kv_norm[l] || !mla->wkv_b[l]) return CORUN_EINVAL;
+    first_dense = mla->first_dense;
+    dense_ffn = s.ffn;
+    if (first_dense > 0 && (dense_ffn < 64 || dense_ffn % 64 || !w->wgate_up || !w->wdown)) return CORUN_EINVAL;
+    for (int l = 0; l < first_dense; ++l)
+      if (!w->wgate_up[l] || !w->wdown[l]) return CORUN_EINVAL;
+    if (first_dense == s.n_layers) moe = nullptr;   // no expert layer at all
+    s.head_dim = mla->v_head;                        // the o-projection's K is n_q_heads * v_head
+    s.n_kv_heads = s.n_q_heads;
+  }
   if (moe) {
     if (moe->n_experts < 1 || moe->n_experts > 256 || moe->top_k < 1 || moe->top_k > 16 || moe->top_k > moe->n_experts ||
         moe->expert_ffn < 64 || moe->expert_ffn % 64 || moe->n_shared < 0 || !moe->router || !moe->gate_up || !moe->down)
       return CORUN_EINVAL;
-    for (int l = 0; l < s.n_layers; ++l)
+    for (int l = first_dense; l < s.n_layers; ++l)
       if (!moe->router[l] || !moe->gate_up[l] || !moe->down[l]) return CORUN_EINVAL;
     s.ffn = (moe->n_experts + moe->n_shared) * moe->expert_ffn;   // the feed-forward width the row program sees
   }
   if (s.arch != 0 || s.n_layers < 1 || s.hidden < 64 || s.hidden % 64 || s.ffn < 64 || s.ffn % 64 || s.vocab < 1)
     return CORUN_EINVAL;
-  if (s.head_dim != 64 && s.head_dim != 128) return CORUN_EINVAL;
+  if (!mla && s.head_dim != 64 && s.head_dim != 128) return CORUN_EINVAL;
   if (s.n_q_heads < 1 || s.n_kv_heads < 1 || s.n_q_heads % s.n_kv_heads) return CORUN_EINVAL;
   const int group = s.n_q_heads / s.n_kv_heads;
   if (group != 1 && group != 2 && group != 4 && group != 8) return CORUN_EINVAL;
@@ -442,6 +550,7 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
   for (int l = 0; l < s.n_layers; ++l)
     if (!w->attn_norm[l] || !w->wqkv[l] || !w->wo[l] || !w->mlp_norm[l] || (!moe && (!w->wgate_up[l] || !w->wdown[l])))
       return CORUN_EINVAL;
+  const int Lm = moe ? first_dense : 0;              // the first layer with experts (whose weights the plans are made on)
 
   int dev = 0;
   CK(cudaGetDevice(&dev));
@@ -468,8 +577,17 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
   }
   e->w0_qkv = w->wqkv[0];
   e->w0_o = w->wo[0];
-  e->w0_gu = moe ? moe->gate_up[0] : w->wgate_up[0];
-  e->w0_down = moe ? moe->down[0] : w->wdown[0];
+  e->w0_gu = moe ? moe->gate_up[Lm] : w->wgate_up[0];
+  e->w0_down = moe ? moe->down[Lm] : w->wdown[0];
+  if (mla) {
+    e->mla = true;
+    e->md = MlaDims{s.n_q_heads, mla->kv_lora_rank, mla->qk_nope, mla->qk_rope, mla->v_head};
+    e->first_dense = first_dense;
+    e->dense_ffn = moe ? dense_ffn : 0;
+    e->mla_splits = mla_max_splits(max_context);
+    e->w0_uv = mla->wkv_b[0];
+    if (moe && first_dense > 0) { e->w0_gu_d = w->wgate_up[0]; e->w0_down_d = w->wdown[0]; }
+  }
   if (moe) {
     e->moe_E = moe->n_experts;
     e->moe_K = moe->top_k;
@@ -483,7 +601,8 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
     // left for the programs' buffers, whichever is less (admission then refuses what does not fit)
     size_t free_b = 0, total_b = 0;
     if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess) return fail(CORUN_ECUDA);
-    const size_t page_b = (size_t)s.n_layers * 2 * s.n_kv_heads * KV_BLOCK * s.head_dim * sizeof(__half);
+    const size_t page_b = mla ? (size_t)s.n_layers * KV_BLOCK * (mla->kv_lora_rank + mla->qk_rope) * sizeof(__half)
+                              : (size_t)s.n_layers * 2 * s.n_kv_heads * KV_BLOCK * s.head_dim * sizeof(__half);
     const size_t keep = (size_t)6 << 30;
     const int64_t fit = free_b > keep ? (int64_t)((free_b - keep) / page_b) : 0;
     if (fit < e->pool_blocks) e->pool_blocks = fit;
@@ -508,17 +627,41 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
     e->attn_norm.push_back((const bf16 *)w->attn_norm[l]);
     e->mlp_norm.push_back((const bf16 *)w->mlp_norm[l]);
     int rc;
-    if ((rc = gemm_encode_map(&e->tm_qkv[l], w->wqkv[l], QD + 2 * KD, H, GEMM_TILE_N))) return fail(rc);
+    const int qkv_rows = mla ? s.n_q_heads * (mla->qk_nope + mla->qk_rope) + mla->kv_lora_rank + mla->qk_rope : QD + 2 * KD;
+    if ((rc = gemm_encode_map(&e->tm_qkv[l], w->wqkv[l], qkv_rows, H, GEMM_TILE_N))) return fail(rc);
     if ((rc = gemm_encode_map(&e->tm_o[l], w->wo[l], H, QD, GEMM_TILE_N))) return fail(rc);
+    if (moe && l < first_dense) {                   // a dense feed-forward layer of a decoder with expert layers
+      if (e->tm_gu_d.empty()) { e->tm_gu_d.resize(s.n_layers); e->tm_down_d.resize(s.n_layers); }
+      if ((rc = gemm_encode_map(&e->tm_gu_d[l], w->wgate_up[l], 2 * dense_ffn, H, GEMM_TILE_N))) return fail(rc);
+      if ((rc = gemm_encode_map(&e->tm_down_d[l], w->wdown[l], H, dense_ffn, GEMM_TILE_N))) return fail(rc);
+      continue;
+    }
     if ((rc = gemm_encode_map(&e->tm_gu[l], moe ? moe->gate_up[l] : w->wgate_up[l], 2 * F, H, GEMM_TILE_N))) return fail(rc);
     if ((rc = gemm_encode_map(&e->tm_down[l], moe ? moe->down[l] : w->wdown[l], H, F, GEMM_TILE_N))) return fail(rc);
     if (!moe && (rc = gemm_encode_map(&e->tm_gu_half[l], w->wgate_up[l], 2 * F, H, gemm_swiglu_half(F, e->num_sms)))) return fail(rc);
+  }
+  if (mla) {
+    // the key up-projections transposed (q_lat = W_uk^T q_nope is a GEMM over rows of W_uk^T), and per layer
+    // the maps of the two grouped up-projection GEMMs
+    int rc;
+    const MlaDims &md = e->md;
+    const size_t per_layer = (size_t)md.nh * md.rank * md.nope;
+    if ((rc = dmalloc(e->allocs, &e->w_ukT, per_layer * s.n_layers, false))) return fail(rc);
+    e->tm_uk.resize(s.n_layers);
+    e->tm_uv.resize(s.n_layers);
+    for (int l = 0; l < s.n_layers; ++l) {
+      e->kv_norm.push_back((const bf16 *)mla->kv_norm[l]);
+      bf16 *dst = e->w_ukT + (size_t)l * per_layer;
+      if (launch_mla_transpose_uk((const bf16 *)mla->wkv_b[l], md, dst, 0) != cudaSuccess) return fail(CORUN_ECUDA);
+      if ((rc = gemm_encode_map(&e->tm_uk[l], dst, md.nh * md.rank, md.nope, GEMM_TILE_N))) return fail(rc);
+      if ((rc = gemm_encode_map(&e->tm_uv[l], mla->wkv_b[l], md.nh * (md.nope + md.vh), md.rank, GEMM_TILE_N))) return fail(rc);
+    }
   }
   if (moe) {
     int rc;
     if ((rc = dmalloc(e->allocs, &e->router_pad, (size_t)s.n_layers * GEMM_TILE_N * H))) return fail(rc);
     e->tm_router.resize(s.n_layers);
-    for (int l = 0; l < s.n_layers; ++l) {
+    for (int l = first_dense; l < s.n_layers; ++l) {
       bf16 *dst = e->router_pad + (size_t)l * GEMM_TILE_N * H;
       if (cudaMemcpy(dst, moe->router[l], (size_t)moe->n_experts * H * sizeof(bf16), cudaMemcpyDeviceToDevice) != cudaSuccess)
         return fail(CORUN_ECUDA);
@@ -528,10 +671,18 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
 
   auto &A = e->allocs;
   int rc;
-  e->layer_stride = (size_t)e->pool_blocks * 2 * s.n_kv_heads * KV_BLOCK * s.head_dim;
+  e->layer_stride = mla ? (size_t)e->pool_blocks * KV_BLOCK * (e->md.rank + e->md.rope)
+                        : (size_t)e->pool_blocks * 2 * s.n_kv_heads * KV_BLOCK * s.head_dim;
   // zero-filled: masked positions of a page are multiplied by zero weights, so they must be finite
   if ((rc = dmalloc(A, &e->kv_pool, e->layer_stride * s.n_layers, true))) return fail(rc);
-  {
+  if (mla) {
+    // one layer's pages: rows of rank + rope halfs, 16 per page
+    e->tm_c.resize(s.n_layers);
+    e->tm_cv.resize(s.n_layers);
+    for (int l = 0; l < s.n_layers; ++l)
+      if ((rc = mla_encode_maps(&e->tm_c[l], &e->tm_cv[l], e->kv_pool + (size_t)l * e->layer_stride, e->pool_blocks, e->md.rank, e->md.rope)))
+        return fail(rc);
+  } else {
     // one layer's pages seen as rows of hd halfs (16 rows per page and head, keys first, then values)
     const unsigned long long halfs = (unsigned long long)e->layer_stride;
     if (halfs / KV_BLOCK >= (1ull << 31)) return fail(CORUN_EINVAL);
@@ -553,12 +704,12 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
       (rc = dmalloc(A, &e->d_pf_tok, 1)))
     return fail(rc);
   {
-    // cos/sin of pos * theta^(-2i/hd), evaluated in fp64 on the host
-    const int half = s.head_dim / 2;
+    // cos/sin of pos * theta^(-2i/hd), evaluated in fp64 on the host (hd: the rotated width)
+    const int rot = mla ? mla->qk_rope : s.head_dim, half = rot / 2;
     std::vector<float2> tab((size_t)max_context * half);
     for (int p = 0; p < max_context; ++p)
       for (int i = 0; i < half; ++i) {
-        const double ang = (double)p * std::pow((double)s.rope_theta, -2.0 * (double)i / (double)s.head_dim);
+        const double ang = (double)p * std::pow((double)s.rope_theta, -2.0 * (double)i / (double)rot);
         tab[(size_t)p * half + i] = make_float2((float)std::cos(ang), (float)std::sin(ang));
       }
     if ((rc = dmalloc(A, &e->d_rope, tab.size(), false))) return fail(rc);
@@ -612,13 +763,20 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
 
 int corun_init(const corun_shape *shape, const corun_weights *w, int32_t B, int32_t max_context, int32_t kv_block,
                int64_t kv_pool_blocks, void *cuda_stream, corun_engine **out) {
-  return engine_create(shape, w, nullptr, B, max_context, kv_block, kv_pool_blocks, cuda_stream, out);
+  return engine_create(shape, w, nullptr, nullptr, B, max_context, kv_block, kv_pool_blocks, cuda_stream, out);
 }
 
 int corun_init_moe(const corun_shape *shape, const corun_weights *w, const corun_moe_layers *moe, int32_t B,
                    int32_t max_context, int32_t kv_block, int64_t kv_pool_blocks, void *cuda_stream, corun_engine **out) {
   if (!moe) return CORUN_EINVAL;
-  return engine_create(shape, w, moe, B, max_context, kv_block, kv_pool_blocks, cuda_stream, out);
+  return engine_create(shape, w, moe, nullptr, B, max_context, kv_block, kv_pool_blocks, cuda_stream, out);
+}
+
+int corun_init_mla(const corun_shape *shape, const corun_weights *w, const corun_mla_layers *mla, const corun_moe_layers *moe,
+                   int32_t B, int32_t max_context, int32_t kv_block, int64_t kv_pool_blocks, void *cuda_stream,
+                   corun_engine **out) {
+  if (!mla) return CORUN_EINVAL;
+  return engine_create(shape, w, moe, mla, B, max_context, kv_block, kv_pool_blocks, cuda_stream, out);
 }
 
 void corun_destroy(corun_engine *e) {
@@ -657,7 +815,7 @@ struct PfReq {
 int prefill_finish_row(corun_engine *e, int row, PfReq &r) {
   const corun_shape &s = e->sh;
   Program &P = e->pre, &L = e->lm1;
-  GemmOut prev = ffn_out(P);
+  GemmOut prev = ffn_out(e, P, s.n_layers - 1);
   prev.direct += (size_t)row * prev.N;
   if (prev.ws) prev.ws += (size_t)row * GEMM_TILE_N;
   const Rows one{P.row_token + row, P.row_pos + row, P.row_active + row, P.row_slot + row, 1};
@@ -711,6 +869,7 @@ int prefill_run(corun_engine *e, PfReq *reqs, int n_req) {
   Program &P = e->pre;
   const int CH = e->chunk;
   int unit = 128 / (s.n_q_heads / s.n_kv_heads);    // tokens per attention tile
+  if (e->mla) unit = 16;                            // no query tiles there: every row is on its own
   if (unit > CH || CH % unit) unit = CH;
   int *tok = e->h_rows, *pos = tok + CH, *act = pos + CH, *slt = act + CH;
   std::vector<std::pair<int, int>> fins;           // (request, chunk row of its last prompt token)
@@ -901,19 +1060,48 @@ int corun_engine_info(corun_engine *e, int32_t *B, int32_t *max_context, int32_t
 int corun_prefill_geometry(corun_engine *e, int32_t *chunk_rows, int32_t *tile_rows) {
   if (!e) return CORUN_EINVAL;
   int unit = 128 / (e->sh.n_q_heads / e->sh.n_kv_heads);
+  if (e->mla) unit = 16;
   if (unit > e->chunk || e->chunk % unit) unit = e->chunk;
   if (chunk_rows) *chunk_rows = e->chunk;
   if (tile_rows) *tile_rows = unit;
   return CORUN_OK;
 }
 
+// MLA engines: k holds the cached rows ([n][rank + rope]), v is not used (may be NULL).
+static int latent_io(corun_engine *e, int slot, int layer, int pos0, int n, float *k, int write) {
+  const int row = e->md.rank + e->md.rope;
+  const size_t elems = (size_t)n * row;
+  float *dk = nullptr;
+  if (cudaMalloc(&dk, elems * sizeof(float)) != cudaSuccess) return CORUN_ENOMEM;
+  const MlaCache cache{e->kv_pool + (size_t)layer * e->layer_stride, e->d_block_table, e->max_blocks, e->B, (long long)e->pool_blocks};
+  cudaError_t ce = cudaSuccess;
+  if (write) ce = cudaMemcpyAsync(dk, k, elems * sizeof(float), cudaMemcpyHostToDevice, e->st);
+  if (ce == cudaSuccess) ce = launch_mla_copy(cache, row, slot, pos0, n, dk, write, e->st);
+  if (ce == cudaSuccess && !write) ce = cudaMemcpyAsync(k, dk, elems * sizeof(float), cudaMemcpyDeviceToHost, e->st);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(e->st);
+  cudaFree(dk);
+  if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
+  return CORUN_OK;
+}
+
 static int kv_io(corun_engine *e, int slot, int layer, int pos0, int n, float *k, float *v, int write) {
+  if (e && e->mla && !v) v = k;                     // the latent cache has no second array
   if (!e || !k || !v || n < 0 || pos0 < 0 || layer < 0 || layer >= e->sh.n_layers) return CORUN_EINVAL;
   if (!slot_ok(e, slot) || !e->in_use[slot]) return CORUN_ESLOT;
   const int limit = write ? e->reserve[slot] : e->ctx[slot];
   if (pos0 + n > limit) return CORUN_EINVAL;
   if (n == 0) return CORUN_OK;
   RC(sync_stream(e));
+  if (e->mla) {
+    RC(latent_io(e, slot, layer, pos0, n, k, write));
+    if (write && pos0 + n > e->ctx[slot]) {
+      e->ctx[slot] = pos0 + n;
+      const int c = e->ctx[slot];
+      CK(cudaMemcpyAsync(e->d_ctx + slot, &c, sizeof(int), cudaMemcpyHostToDevice, e->st));
+      CK(cudaStreamSynchronize(e->st));
+    }
+    return CORUN_OK;
+  }
   const size_t elems = (size_t)n * e->sh.n_kv_heads * e->sh.head_dim;
   float *dk = nullptr, *dv = nullptr;
   if (cudaMalloc(&dk, elems * sizeof(float)) != cudaSuccess) return CORUN_ENOMEM;
@@ -974,7 +1162,14 @@ int corun_debug_kv_fill(corun_engine *e, int32_t slot, int32_t n_ctx, float std,
   if (!slot_ok(e, slot) || !e->in_use[slot]) return CORUN_ESLOT;
   if (n_ctx > e->reserve[slot]) return CORUN_EINVAL;
   RC(sync_stream(e));
-  CK(launch_kv_fill(kv_layout(e), e->sh.n_layers, slot, n_ctx, std, seed, e->st));
+  if (e->mla) {
+    for (int l = 0; l < e->sh.n_layers; ++l) {
+      const MlaCache cache{e->kv_pool + (size_t)l * e->layer_stride, e->d_block_table, e->max_blocks, e->B, (long long)e->pool_blocks};
+      CK(launch_mla_fill(cache, e->md.rank + e->md.rope, l, slot, n_ctx, std, seed, e->st));
+    }
+  } else {
+    CK(launch_kv_fill(kv_layout(e), e->sh.n_layers, slot, n_ctx, std, seed, e->st));
+  }
   CK(cudaMemcpyAsync(e->d_ctx + slot, &n_ctx, sizeof(int), cudaMemcpyHostToDevice, e->st));
   CK(cudaStreamSynchronize(e->st));
   e->ctx[slot] = n_ctx;
@@ -982,7 +1177,7 @@ int corun_debug_kv_fill(corun_engine *e, int32_t slot, int32_t n_ctx, float std,
 }
 
 int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *avg_ms) {
-  if (!e || !avg_ms || reps < 1 || kind < 0 || kind > 9) return CORUN_EINVAL;
+  if (!e || !avg_ms || reps < 1 || kind < 0 || kind > 9 || e->mla) return CORUN_EINVAL;
   RC(sync_stream(e));
   Program &P = e->dec;
   const corun_shape &s = e->sh;
@@ -997,7 +1192,7 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
     cudaError_t ce = cudaEventRecord(a, e->st);
     for (int i = 0; i < n && ce == cudaSuccess; ++i) {
       const int l = i % s.n_layers;   // rotate over the layers so that L2 cannot hold the weights
-      GemmOut prev = ffn_out(P);
+      GemmOut prev = ffn_out(e, P, 0);
       switch (kind) {
         // launched as in the step's graph: with programmatic stream serialization
         case 0: ce = gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, nullptr, true); break;
@@ -1062,7 +1257,7 @@ int corun_debug_gemm_trace(corun_engine *e, int32_t kind, int32_t layer, uint64_
 }
 
 int corun_debug_attn_trace(corun_engine *e, int32_t layer, uint64_t *stamps, int32_t *n_ctas) {
-  if (!e || !stamps || !n_ctas || layer < 0 || layer >= e->sh.n_layers) return CORUN_EINVAL;
+  if (!e || !stamps || !n_ctas || layer < 0 || layer >= e->sh.n_layers || e->mla) return CORUN_EINVAL;
   RC(sync_stream(e));
   Program &P = e->dec;
   const corun_shape &s = e->sh;

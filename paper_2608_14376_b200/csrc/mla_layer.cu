@@ -1,0 +1,185 @@
+// Token-wise kernels of a multi-head latent attention (MLA) layer around the attention kernel: cache append with
+// the latent's RMSNorm and the rotary key's rotation, the query's parts, the value part of the up-projection,
+// and the set-up / debug helpers of the latent pool.  Every reduction has one fixed order.
+#include "mla.cuh"
+
+#include "checks.cuh"
+#include "launch.cuh"
+#include "ptx.cuh"
+
+namespace corun {
+
+namespace {
+
+__device__ __forceinline__ void mla_split_bf16(float x, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
+  hi = __float2bfloat16_rn(x);
+  lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+constexpr int MLA_POST_THREADS = 256;
+
+// One CTA per row.
+__global__ void __launch_bounds__(MLA_POST_THREADS)
+mla_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, MlaDims d, const __nv_bfloat16 *__restrict__ gains,
+                float eps, MlaCache cache, int rows_per_head, __nv_bfloat16 *__restrict__ qn_hi, __nv_bfloat16 *__restrict__ qn_lo,
+                float *__restrict__ q_rope, int *status) {
+  griddep_launch_dependents();
+  griddep_wait();
+  __shared__ float scratch[MLA_POST_THREADS / 32];
+  const int r = blockIdx.x, tid = threadIdx.x;
+  if (rows.active[r] == 0) return;                   // a padding row: no cache write, its query is never used
+  const int pos = rows.pos[r];
+  const int qw = d.nope + d.rope, QD = d.nh * qw, half = d.rope >> 1;
+  // ---- the query: no-rope parts as bf16 hi/lo (head-major), rotary parts rotated, fp32
+  for (int i = tid; i < d.nh * d.nope; i += MLA_POST_THREADS) {
+    const int h = i / d.nope, j = i - h * d.nope;
+    __nv_bfloat16 a, b;
+    mla_split_bf16(gemm_load(qkv, r, h * qw + j), a, b);
+    const size_t o = ((size_t)h * rows_per_head + r) * d.nope + j;
+    qn_hi[o] = a;
+    qn_lo[o] = b;
+  }
+  for (int i = tid; i < d.nh * half; i += MLA_POST_THREADS) {
+    const int h = i / half, j = i - h * half;
+    const float a = gemm_load(qkv, r, h * qw + d.nope + j), b = gemm_load(qkv, r, h * qw + d.nope + j + half);
+    const float2 t = rope_tab[(size_t)pos * half + j];   // (cos, sin)
+    float *q = q_rope + ((size_t)r * d.nh + h) * d.rope + j;
+    q[0] = a * t.x - b * t.y;
+    q[half] = a * t.y + b * t.x;
+  }
+  // ---- the cache row: RMSNorm of the latent (sum of squares: thread-serial ascending, xor butterfly in the warp,
+  //      warp totals ascending), rotated rotary key
+#ifdef CORUN_CHECKED
+  if (!check_slot_pos(rows.slot[r], cache.n_slots, pos, cache.max_blocks, KV_BLOCK)) {
+    if (tid == 0) atomicCAS(status, 0, DEV_BAD_INDEX);
+    return;
+  }
+#endif
+  const int blk = cache.block_table[(size_t)rows.slot[r] * cache.max_blocks + pos / KV_BLOCK];
+#ifdef CORUN_CHECKED
+  if (!check_page(blk, cache.pool_blocks)) {
+    if (tid == 0) atomicCAS(status, 0, DEV_BAD_INDEX);
+    return;
+  }
+#endif
+  __half *dst = cache.pool + ((size_t)blk * KV_BLOCK + pos % KV_BLOCK) * (d.rank + d.rope);
+  float x[4];                                        // rank <= 4 * threads
+  float ss = 0.f;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const int i = tid + e * MLA_POST_THREADS;
+    x[e] = i < d.rank ? gemm_load(qkv, r, QD + i) : 0.f;
+    ss = fmaf(x[e], x[e], ss);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((tid & 31) == 0) scratch[tid >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+  for (int w = 0; w < MLA_POST_THREADS / 32; ++w) tot += scratch[w];
+  const float inv = rsqrtf(tot / (float)d.rank + eps);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const int i = tid + e * MLA_POST_THREADS;
+    if (i < d.rank) dst[i] = __float2half_rn(x[e] * inv * __bfloat162float(gains[i]));
+  }
+  if (tid < half) {
+    const float a = gemm_load(qkv, r, QD + d.rank + tid), b = gemm_load(qkv, r, QD + d.rank + tid + half);
+    const float2 t = rope_tab[(size_t)pos * half + tid];
+    dst[d.rank + tid] = __float2half_rn(a * t.x - b * t.y);
+    dst[d.rank + tid + half] = __float2half_rn(a * t.y + b * t.x);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+mla_ao_split_kernel(const float *__restrict__ uv, int R, int rows_per_head, MlaDims d, __nv_bfloat16 *__restrict__ ao_hi,
+                    __nv_bfloat16 *__restrict__ ao_lo) {
+  griddep_launch_dependents();
+  griddep_wait();
+  const int r = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= d.nh * d.vh) return;
+  const int h = i / d.vh, j = i - h * d.vh;
+  __nv_bfloat16 a, b;
+  mla_split_bf16(uv[((size_t)h * rows_per_head + r) * (d.nope + d.vh) + d.nope + j], a, b);
+  ao_hi[(size_t)r * d.nh * d.vh + i] = a;
+  ao_lo[(size_t)r * d.nh * d.vh + i] = b;
+}
+
+__global__ void mla_transpose_uk_kernel(const __nv_bfloat16 *__restrict__ wkv_b, MlaDims d, __nv_bfloat16 *__restrict__ out) {
+  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t n = (size_t)d.nh * d.rank * d.nope;
+  if (idx >= n) return;
+  const int i = (int)(idx % d.nope);
+  const int c = (int)((idx / d.nope) % d.rank);
+  const int h = (int)(idx / ((size_t)d.nope * d.rank));
+  out[idx] = wkv_b[((size_t)h * (d.nope + d.vh) + i) * d.rank + c];
+}
+
+__device__ __forceinline__ uint64_t mla_mix64(uint64_t z) {
+  z += 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+// Synthetic cache contents for timing runs: position-hashed normals, one thread per pair of values.
+__global__ void mla_fill_kernel(MlaCache cache, int row_halfs, int layer, int slot, int n, float std, uint64_t seed) {
+  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int pairs = row_halfs / 2;
+  if (idx >= (size_t)n * pairs) return;
+  const int t = (int)(idx / pairs), e = (int)(idx - (size_t)t * pairs);
+  const uint64_t h = mla_mix64(seed ^ mla_mix64(((uint64_t)slot << 48) ^ ((uint64_t)layer << 40) ^ ((uint64_t)t << 16) ^ (uint64_t)e));
+  const float u1 = ((float)(uint32_t)(h >> 40) + 1.0f) * (1.0f / 16777217.0f);
+  const float u2 = (float)(uint32_t)((h >> 8) & 0xFFFFFFu) * (1.0f / 16777216.0f);
+  const float rad = sqrtf(-2.0f * logf(u1)) * std;
+  const int blk = cache.block_table[(size_t)slot * cache.max_blocks + t / KV_BLOCK];
+  __half *row = cache.pool + ((size_t)blk * KV_BLOCK + t % KV_BLOCK) * row_halfs;
+  row[2 * e] = __float2half_rn(rad * cospif(2.0f * u2));
+  row[2 * e + 1] = __float2half_rn(rad * sinpif(2.0f * u2));
+}
+
+__global__ void mla_copy_kernel(MlaCache cache, int row_halfs, int slot, int pos0, int n, float *buf, int write) {
+  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (size_t)n * row_halfs) return;
+  const int t = pos0 + (int)(idx / row_halfs), e = (int)(idx % row_halfs);
+  const int blk = cache.block_table[(size_t)slot * cache.max_blocks + t / KV_BLOCK];
+  __half *p = cache.pool + ((size_t)blk * KV_BLOCK + t % KV_BLOCK) * row_halfs + e;
+  if (write) *p = __float2half_rn(buf[idx]);
+  else buf[idx] = __half2float(*p);
+}
+
+}  // namespace
+
+cudaError_t launch_mla_post(const GemmOut &qkv, const Rows &rows, const float2 *rope_tab, const MlaDims &d,
+                            const __nv_bfloat16 *kv_gains, float eps, const MlaCache &cache, int rows_per_head,
+                            __nv_bfloat16 *qn_hi, __nv_bfloat16 *qn_lo, float *q_rope, int *d_status, cudaStream_t st) {
+  return launch_k(mla_post_kernel, dim3(rows.R), dim3(MLA_POST_THREADS), 0, st, true, qkv, rows, rope_tab, d, kv_gains, eps, cache,
+                  rows_per_head, qn_hi, qn_lo, q_rope, d_status);
+}
+
+cudaError_t launch_mla_ao_split(const float *uv, int R, int rows_per_head, const MlaDims &d, __nv_bfloat16 *ao_hi,
+                                __nv_bfloat16 *ao_lo, cudaStream_t st) {
+  return launch_k(mla_ao_split_kernel, dim3((d.nh * d.vh + 255) / 256, R), dim3(256), 0, st, true, uv, R, rows_per_head, d, ao_hi, ao_lo);
+}
+
+cudaError_t launch_mla_transpose_uk(const __nv_bfloat16 *wkv_b, const MlaDims &d, __nv_bfloat16 *out, cudaStream_t st) {
+  const size_t n = (size_t)d.nh * d.rank * d.nope;
+  mla_transpose_uk_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(wkv_b, d, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_mla_fill(const MlaCache &cache, int row_halfs, int layer, int slot, int n, float std, uint64_t seed, cudaStream_t st) {
+  const size_t tot = (size_t)n * (row_halfs / 2);
+  if (tot == 0) return cudaSuccess;
+  mla_fill_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(cache, row_halfs, layer, slot, n, std, seed);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_mla_copy(const MlaCache &cache, int row_halfs, int slot, int pos0, int n, float *buf, int write, cudaStream_t st) {
+  const size_t tot = (size_t)n * row_halfs;
+  if (tot == 0) return cudaSuccess;
+  mla_copy_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(cache, row_halfs, slot, pos0, n, buf, write);
+  return cudaGetLastError();
+}
+
+}  // namespace corun

@@ -36,6 +36,7 @@
 #include "../../include/corun_mla.h"
 #include "gemm.cuh"
 #include "launch.cuh"
+#include "mla.cuh"
 #include "ptx.cuh"
 
 namespace corun {
@@ -81,9 +82,10 @@ __device__ __forceinline__ void mp_tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) 
 // part_ml [B][max_splits][n_heads] (max in the base-2 domain, sum), part_o [B][max_splits][n_heads][d_c]
 __global__ void __launch_bounds__(MP_THREADS, 1)
 mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmV, const float *__restrict__ q_lat,
-                 const float *__restrict__ q_rope, const int *__restrict__ block_table, int max_blocks, const int *__restrict__ ctx,
-                 int B, int n_heads, int d_c, int d_r, float scale_log2e, int max_splits, float2 *__restrict__ part_ml,
-                 float *__restrict__ part_o, int *status) {
+                 long long q_rs, long long q_hs, const float *__restrict__ q_rope, const int *__restrict__ block_table, int max_blocks,
+                 const int *__restrict__ ctx, const int *__restrict__ row_slot, const int *__restrict__ row_pos,
+                 const int *__restrict__ row_active, int B, int n_heads, int d_c, int d_r, float scale_log2e, int max_splits,
+                 float2 *__restrict__ part_ml, float *__restrict__ part_o, int *status) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[MP_RING], empty_bar[MP_RING];
   __shared__ __align__(8) uint64_t q_ready_bar, q_free_bar, s_full_bar, s_free_bar, p_ready_bar, o_full_bar, o_free_bar, x_bar;
@@ -96,6 +98,7 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
 
+  griddep_wait();                                    // (programmatic launch) the queries are the previous kernel's results
   if (tid == 0) {
     abort_flag = 0;
     for (int s = 0; s < MP_RING; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
@@ -122,7 +125,7 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
       const int r = r0 + lane;
       int n = 0;
       if (r < B) {
-        int c = ctx[r];
+        int c = row_pos ? (row_active[r] ? row_pos[r] + 1 : 0) : ctx[r];
         c = c < 0 ? 0 : (c > max_blocks * MP_PAGE ? max_blocks * MP_PAGE : c);
         n = (c + MP_T - 1) / MP_T;
         if (n > max_splits) { n = max_splits; c = n * MP_T; }
@@ -177,7 +180,8 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
       int r, split;
       locate(it, r, split);
       n = (tokens_of(r, split) + MP_PAGE - 1) / MP_PAGE;
-      return lane < n ? __ldg(block_table + (size_t)r * max_blocks + split * MP_PAGES + lane) : 0;
+      const int tr = row_slot ? __ldg(row_slot + r) : r;     // whose block table the row reads
+      return lane < n ? __ldg(block_table + (size_t)tr * max_blocks + split * MP_PAGES + lane) : 0;
     };
     int np_ahead = 0, page_ahead = pages_of(item_lo, np_ahead);
     for (int it = item_lo; it <= item_hi && !failed; ++it) {
@@ -301,7 +305,7 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
           hh[e] = -1;
           if (i < total) {
             const int h = i / chunks, d = (i - h * chunks) << 3;
-            const float *src = d < d_c ? q_lat + ((size_t)r * n_heads + h) * d_c + d : q_rope + ((size_t)r * n_heads + h) * d_r + (d - d_c);
+            const float *src = d < d_c ? q_lat + (size_t)r * q_rs + (size_t)h * q_hs + d : q_rope + ((size_t)r * n_heads + h) * d_r + (d - d_c);
             x0[e] = __ldg(reinterpret_cast<const float4 *>(src));
             x1[e] = __ldg(reinterpret_cast<const float4 *>(src) + 1);
             hh[e] = h;
@@ -463,13 +467,18 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   if (warp == 0) tmem_dealloc(tmem_base, MP_TMEM_COLS);
 }
 
-// One block per (row, head), one thread per four latent dims: the row's splits in ascending order -> o_lat.
+// One block per (row, head), one thread per four latent dims: the row's splits in ascending order -> o_lat (fp32
+// [B][n_heads][d_c]) or, when that is null, a bf16 hi/lo pair laid out head-major [n_heads][rows_per_head][d_c].
 __global__ void __launch_bounds__(128) mla_paged_combine_kernel(const float2 *__restrict__ part_ml, const float *__restrict__ part_o,
-                                                                const int *__restrict__ ctx, int B, int n_heads, int d_c,
-                                                                int max_blocks, int max_splits, float *__restrict__ o_lat) {
+                                                                const int *__restrict__ ctx, const int *__restrict__ row_pos,
+                                                                const int *__restrict__ row_active, int B, int n_heads, int d_c,
+                                                                int max_blocks, int max_splits, float *__restrict__ o_lat,
+                                                                __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo,
+                                                                int rows_per_head) {
+  griddep_launch_dependents();
   const int r = (int)blockIdx.x / n_heads, h = (int)blockIdx.x - r * n_heads;
   const int d = 4 * (int)threadIdx.x;
-  int c = ctx[r];
+  int c = row_pos ? (row_active[r] ? row_pos[r] + 1 : 0) : ctx[r];
   if (c <= 0 || d >= d_c) return;                   // a padding row is left alone
   griddep_wait();
   c = c > max_blocks * MP_PAGE ? max_blocks * MP_PAGE : c;
@@ -502,10 +511,68 @@ __global__ void __launch_bounds__(128) mla_paged_combine_kernel(const float2 *__
         o.x = fmaf(w[e], x[e].x, o.x); o.y = fmaf(w[e], x[e].y, o.y); o.z = fmaf(w[e], x[e].z, o.z); o.w = fmaf(w[e], x[e].w, o.w);
       }
   }
-  *reinterpret_cast<float4 *>(o_lat + ((size_t)r * n_heads + h) * d_c + d) = make_float4(o.x * inv, o.y * inv, o.z * inv, o.w * inv);
+  o = make_float4(o.x * inv, o.y * inv, o.z * inv, o.w * inv);
+  if (o_lat) {
+    *reinterpret_cast<float4 *>(o_lat + ((size_t)r * n_heads + h) * d_c + d) = o;
+  } else {
+    const size_t at = ((size_t)h * rows_per_head + r) * d_c + d;
+    const float v[4] = {o.x, o.y, o.z, o.w};
+    __nv_bfloat16 hi[4], lo[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      hi[e] = __float2bfloat16_rn(v[e]);
+      lo[e] = __float2bfloat16_rn(v[e] - __bfloat162float(hi[e]));
+    }
+    *reinterpret_cast<uint2 *>(out_hi + at) = *reinterpret_cast<const uint2 *>(hi);
+    *reinterpret_cast<uint2 *>(out_lo + at) = *reinterpret_cast<const uint2 *>(lo);
+  }
 }
 
 }  // namespace
+}  // namespace corun
+
+namespace corun {
+
+int mla_max_splits(int max_context) { return (max_context + MP_T - 1) / MP_T; }
+long long mla_part_ml_floats(int R, int nh, int max_context) { return ((long long)R * mla_max_splits(max_context) * nh * 2 + 3) / 4 * 4; }
+long long mla_part_o_floats(int R, int nh, int rank, int max_context) { return (long long)R * mla_max_splits(max_context) * nh * rank; }
+
+int mla_encode_maps(CUtensorMap *tmC, CUtensorMap *tmV, const void *pool, long long pool_pages, int rank, int rope) {
+  if (pool_pages < 1 || pool_pages * MP_PAGE >= (1ll << 31)) return CORUN_EINVAL;
+  // the pool as rows of rank + rope halfs, fetched in [16 tokens x 64 dims] boxes (the rope box reads past the
+  // row's end when rope < 64: those columns arrive as zeros)
+  int rc = tma_encode_2d(tmC, pool, 1, (unsigned long long)pool_pages * MP_PAGE, rank + rope, MP_PAGE, 64);
+  if (rc != CORUN_OK) return rc;
+  // the latent part once more as [8-token group][token in group][block of 64 dims][64 dims]: one box fetches a page's
+  // 16 tokens x (up to) 256 dims as [2 groups][blocks][8 tokens][64 dims], the layout of an MN-major MMA operand
+  const int bph = rank > 256 ? 4 : rank / 64;
+  const unsigned long long row_bytes = (unsigned long long)(rank + rope) * 2;
+  const unsigned long long dims[4] = {64, 8, (unsigned long long)(rank / 64), (unsigned long long)pool_pages * 2};
+  const unsigned long long strides[3] = {row_bytes, 128, 8 * row_bytes};
+  const unsigned box[4] = {64, 8, (unsigned)bph, 2};
+  return tma_encode_fp16_4d(tmV, pool, dims, strides, box);
+}
+
+cudaError_t launch_mla_attention(const CUtensorMap &tmC, const CUtensorMap &tmV, const float *q_lat, long long q_row_stride,
+                                 long long q_head_stride, const float *q_rope, const int *block_table, int max_blocks,
+                                 const int *ctx, const Rows *rows, int R, const MlaDims &d, float scale, int max_splits,
+                                 float2 *part_ml, float *part_o, float *o_lat, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
+                                 int rows_per_head, int num_sms, int *d_status, bool pdl, cudaStream_t st) {
+  static bool prepared = false;                     // idempotent; a race only repeats it
+  if (!prepared) {
+    cudaError_t e = cudaFuncSetAttribute(mla_paged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MP_SMEM);
+    if (e != cudaSuccess) return e;
+    prepared = true;
+  }
+  const int *row_slot = rows ? rows->slot : nullptr, *row_pos = rows ? rows->pos : nullptr, *row_active = rows ? rows->active : nullptr;
+  cudaError_t ce = launch_k(mla_paged_kernel, dim3(num_sms), dim3(MP_THREADS), MP_SMEM, st, pdl, tmC, tmV, q_lat, q_row_stride,
+                            q_head_stride, q_rope, block_table, max_blocks, ctx, row_slot, row_pos, row_active, R, d.nh, d.rank, d.rope,
+                            scale * 1.4426950408889634f, max_splits, part_ml, part_o, d_status);
+  if (ce != cudaSuccess) return ce;
+  return launch_k(mla_paged_combine_kernel, dim3(R * d.nh), dim3(128), 0, st, true, part_ml, part_o, ctx, row_pos, row_active, R, d.nh,
+                  d.rank, max_blocks, max_splits, o_lat, out_hi, out_lo, rows_per_head);
+}
+
 }  // namespace corun
 
 using namespace corun;
@@ -514,8 +581,7 @@ extern "C" {
 
 int64_t corun_mla_workspace_floats(int32_t B, int32_t n_heads, int32_t d_latent, int32_t max_context) {
   if (B < 1 || n_heads < 1 || d_latent < 1 || max_context < 1) return 0;
-  const int64_t splits = (max_context + MP_T - 1) / MP_T;
-  return 64 + ((int64_t)B * splits * n_heads * 2 + 3) / 4 * 4 + (int64_t)B * splits * n_heads * d_latent;
+  return 64 + mla_part_ml_floats(B, n_heads, max_context) + mla_part_o_floats(B, n_heads, d_latent, max_context);
 }
 
 int corun_mla_attend(const float *q_lat, const float *q_rope, const void *pool, int64_t pool_pages, const int32_t *block_table,
@@ -533,34 +599,18 @@ int corun_mla_attend(const float *q_lat, const float *q_rope, const void *pool, 
   cudaError_t ce = cudaGetDevice(&dev);
   if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (ce != cudaSuccess || sms < 1) { g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
-  // the pool as rows of d_latent + d_rope halfs, fetched in [16 tokens x 64 dims] boxes (the rope box reads past the
-  // row's end when d_rope < 64: those columns arrive as zeros)
-  CUtensorMap tm;
-  int rc = tma_encode_2d(&tm, pool, 1, (unsigned long long)pool_pages * MP_PAGE, d_latent + d_rope, MP_PAGE, 64);
+  CUtensorMap tm, tv;
+  int rc = mla_encode_maps(&tm, &tv, pool, pool_pages, d_latent, d_rope);
   if (rc != CORUN_OK) return rc;
-  // the latent part once more as [8-token group][token in group][block of 64 dims][64 dims]: one box fetches a page's
-  // 16 tokens x (up to) 256 dims as [2 groups][blocks][8 tokens][64 dims], the layout of an MN-major MMA operand
-  CUtensorMap tv;
-  {
-    const int bph = d_latent > 256 ? 4 : d_latent / 64;
-    const unsigned long long row_bytes = (unsigned long long)(d_latent + d_rope) * 2;
-    const unsigned long long dims[4] = {64, 8, (unsigned long long)(d_latent / 64), (unsigned long long)pool_pages * 2};
-    const unsigned long long strides[3] = {row_bytes, 128, 8 * row_bytes};
-    const unsigned box[4] = {64, 8, (unsigned)bph, 2};
-    if ((rc = tma_encode_fp16_4d(&tv, pool, dims, strides, box)) != CORUN_OK) return rc;
-  }
-  const int max_splits = (max_blocks * MP_PAGE + MP_T - 1) / MP_T;
+  const int max_splits = mla_max_splits(max_blocks * MP_PAGE);
   int *status = reinterpret_cast<int *>(ws);
   float2 *part_ml = reinterpret_cast<float2 *>(ws + 64);
-  float *part_o = ws + 64 + ((size_t)B * max_splits * n_heads * 2 + 3) / 4 * 4;
-  ce = cudaFuncSetAttribute(mla_paged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MP_SMEM);
-  if (ce == cudaSuccess) ce = cudaMemsetAsync(status, 0, sizeof(int), st);
+  float *part_o = ws + 64 + mla_part_ml_floats(B, n_heads, max_blocks * MP_PAGE);
+  const MlaDims dims{n_heads, d_latent, 0, d_rope, 0};
+  ce = cudaMemsetAsync(status, 0, sizeof(int), st);
   if (ce == cudaSuccess)
-    ce = launch_k(mla_paged_kernel, dim3(sms), dim3(MP_THREADS), MP_SMEM, st, false, tm, tv, q_lat, q_rope, block_table, max_blocks, ctx, B,
-                  n_heads, d_latent, d_rope, scale * 1.4426950408889634f, max_splits, part_ml, part_o, status);
-  if (ce == cudaSuccess)
-    ce = launch_k(mla_paged_combine_kernel, dim3(B * n_heads), dim3(128), 0, st, true, part_ml, part_o, ctx, B, n_heads,
-                  d_latent, max_blocks, max_splits, o_lat);
+    ce = launch_mla_attention(tm, tv, q_lat, (long long)n_heads * d_latent, d_latent, q_rope, block_table, max_blocks, ctx, nullptr, B, dims,
+                              scale, max_splits, part_ml, part_o, o_lat, nullptr, nullptr, 0, sms, status, false, st);
   if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
   return CORUN_OK;
 }

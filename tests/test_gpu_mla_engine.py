@@ -1,0 +1,166 @@
+"""The engine with multi-head latent attention layers (a dense first layer, expert layers behind it): prefill and
+teacher-forced decode steps against the C oracle, bitwise invariance to slot, co-tenants and batched prefill, and
+the DeepSeek-V2-Lite layer shape at full width."""
+import numpy as np
+import pytest
+
+from paper_2608_14376_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+B, MAX_CTX = 8, 320
+TOL = 3e-2
+SMALL = synth.ModelShape(3, 256, 4, 4, 128, 384, 2048, 1e-6, 10000.0)
+SMALL_MLA = dict(kv_lora_rank=256, qk_nope=128, qk_rope=32, v_head=128, first_dense=1)
+SMALL_MOE = dict(n_experts=8, top_k=2, expert_ffn=128, n_shared=1, renormalize=False)
+
+
+def _torch():
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    return torch
+
+
+def _setup(orc, sh, mla, moe, seed, B=B, max_ctx=MAX_CTX, **kw):
+    _torch()
+    from paper_2608_14376_b200 import corun
+
+    w_np, m_np = synth.make_mla_weights_numpy(sh, mla, seed=seed)
+    e_np = synth.make_moe_numpy(sh, seed=seed, **moe) if moe else None
+    model = orc.Model(orc.Shape(**sh.dict()), w_np, moe=e_np, mla=m_np)
+    w_t, m_t = synth.mla_numpy_to_torch(w_np, m_np, "cuda")
+    e_t = synth.moe_numpy_to_torch(e_np, "cuda") if moe else None
+    eng = corun.Engine(sh, w_t, B, max_ctx, moe=e_t, mla=m_t, **kw)
+    return model, eng
+
+
+@pytest.mark.parametrize("first_dense,moe", [(1, SMALL_MOE), (3, None)])
+def test_mla_engine_parity_and_invariance(orc, first_dense, moe):
+    sh = SMALL
+    mla = dict(SMALL_MLA, first_dense=first_dense)
+    model, eng = _setup(orc, sh, mla, moe, seed=3)
+    try:
+        lens = [21, 270, 64, 9]                          # one prompt beyond a 256-token attention split and a prefill chunk
+        prompts = synth.make_prompts(sh.vocab, lens, seed=31)
+        slots = [5, 0, 2, 7]
+        reqs = [orc.Request(model, p, 1, max_T=MAX_CTX) for p in prompts]
+        worst = 0.0
+        for s, p, r in zip(slots, prompts, reqs):
+            r.prefill()
+            eng.prefill(s, p, len(p) + 8)
+            worst = max(worst, float(np.abs(eng.logits(s) - r.logits).max()))
+        active = np.zeros(B, np.uint8); active[slots] = 1
+        seeds = np.zeros(B, np.uint64)
+        trace = []
+        for _ in range(4):                              # teacher-forced with the oracle's greedy tokens
+            toks = [int(np.argmax(r.logits)) for r in reqs]
+            for s, t in zip(slots, toks):
+                eng.force_token(s, t)
+            eng.decode_step(active, seeds)
+            for s, r, t in zip(slots, reqs, toks):
+                r.decode(force_token=t)
+                worst = max(worst, float(np.abs(eng.logits(s) - r.logits).max()))
+            trace.append([eng.logits(s).tobytes() for s in slots])
+        assert worst <= TOL, worst
+        # per layer: 10 around the attention (2 norms, 4 GEMMs, cache append, attention splits and combine, value split)
+        # + 3 (dense feed-forward) or 5 (router, routing, 2 GEMMs, masked SwiGLU)
+        n_dense = first_dense if moe else sh.n_layers
+        assert eng.decode_launches() == 6 + 13 * n_dense + 15 * (sh.n_layers - n_dense) - (0 if moe else n_dense)
+
+        # the same requests in other slots, prefilled together in shared chunks: same bytes
+        for s in slots:
+            eng.release(s)
+        slots2 = [1, 6, 3, 4]
+        first = eng.prefill_batch(slots2, prompts, [len(p) + 8 for p in prompts])
+        assert all(0 <= int(t) < sh.vocab for t in first)
+        cur = [orc.Request(model, p, 1, max_T=MAX_CTX) for p in prompts]
+        for r in cur:
+            r.prefill()
+        active = np.zeros(B, np.uint8); active[slots2] = 1
+        for step in range(4):
+            toks = [int(np.argmax(r.logits)) for r in cur]
+            for s, t in zip(slots2, toks):
+                eng.force_token(s, t)
+            eng.decode_step(active, seeds)
+            for r, t in zip(cur, toks):
+                r.decode(force_token=t)
+            assert [eng.logits(s).tobytes() for s in slots2] == trace[step]
+        # one request alone: still the same bytes as among co-tenants
+        for s in slots2:
+            eng.release(s)
+        eng.prefill(2, prompts[1], lens[1] + 8)
+        solo = orc.Request(model, prompts[1], 1, max_T=MAX_CTX)
+        solo.prefill()
+        active = np.zeros(B, np.uint8); active[2] = 1
+        for step in range(4):
+            t = int(np.argmax(solo.logits))
+            eng.force_token(2, t)
+            eng.decode_step(active, seeds)
+            solo.decode(force_token=t)
+            assert eng.logits(2).tobytes() == trace[step][1]
+    finally:
+        eng.close()
+
+
+def test_mla_engine_cache_rows_are_the_oracles(orc):
+    """What prefill and decode append to the latent cache (normalised latent, rotated rotary key) against the oracle's
+    cache, through the debug read."""
+    sh, mla = SMALL, dict(SMALL_MLA, first_dense=3)
+    model, eng = _setup(orc, sh, mla, None, seed=9)
+    try:
+        p = synth.make_prompts(sh.vocab, [37], seed=2)[0]
+        r = orc.Request(model, p, 1, max_T=MAX_CTX)
+        r.prefill()
+        eng.prefill(3, p, 48)
+        for layer in range(sh.n_layers):
+            got, _ = eng.kv_read(3, layer, 0, 37)
+            ref = r.cache[0][layer, :37]
+            assert got.shape == ref.shape
+            assert np.abs(got - ref).max() <= 2e-2, (layer, np.abs(got - ref).max())
+    finally:
+        eng.close()
+
+
+def test_mla_engine_at_the_deepseek_v2_lite_layer_shape(orc):
+    """Full layer width (hidden 2048, 16 heads, latent 512, rope 64, dense feed-forward 10944, 64 routed experts of
+    1408 top-6 + 2 shared), two layers, a small vocabulary; prompts of a few dozen tokens (the oracle's definition
+    form decompresses every cached token for every query)."""
+    full = synth.DEEPSEEK_V2_LITE
+    sh = synth.ModelShape(2, full.hidden, full.n_q_heads, full.n_q_heads, 128, full.ffn, 4096, full.rms_eps, full.rope_theta)
+    model, eng = _setup(orc, sh, dict(synth.DEEPSEEK_V2_LITE_MLA), dict(synth.DEEPSEEK_V2_LITE_MOE), seed=0, B=8, max_ctx=128)
+    try:
+        lens = [33, 5, 48]
+        prompts = synth.make_prompts(sh.vocab, lens, seed=12)
+        slots = [6, 1, 3]
+        reqs = [orc.Request(model, p, 1, max_T=128) for p in prompts]
+        worst = 0.0
+        for s, p, r in zip(slots, prompts, reqs):
+            r.prefill()
+            eng.prefill(s, p, len(p) + 4)
+            worst = max(worst, float(np.abs(eng.logits(s) - r.logits).max()))
+        active = np.zeros(8, np.uint8); active[slots] = 1
+        seeds = np.zeros(8, np.uint64)
+        for _ in range(2):
+            toks = [int(np.argmax(r.logits)) for r in reqs]
+            for s, t in zip(slots, toks):
+                eng.force_token(s, t)
+            eng.decode_step(active, seeds)
+            for s, r, t in zip(slots, reqs, toks):
+                r.decode(force_token=t)
+                worst = max(worst, float(np.abs(eng.logits(s) - r.logits).max()))
+        assert worst <= TOL, worst
+    finally:
+        eng.close()
+
+
+def test_mla_engine_argument_errors(orc):
+    torch = _torch()
+    from paper_2608_14376_b200 import corun
+
+    sh = SMALL
+    w_np, m_np = synth.make_mla_weights_numpy(sh, dict(SMALL_MLA, first_dense=3), seed=1)
+    w_t, m_t = synth.mla_numpy_to_torch(w_np, m_np, "cuda")
+    for bad in (dict(kv_lora_rank=128), dict(qk_nope=96), dict(qk_rope=20), dict(v_head=64), dict(first_dense=1)):
+        with pytest.raises(corun.CorunError):        # first_dense below the layer count needs expert layers
+            corun.Engine(sh, w_t, 4, 64, mla=dict(m_t, **bad))
