@@ -18,7 +18,23 @@ __device__ __forceinline__ void mla_split_bf16(float x, __nv_bfloat16 &hi, __nv_
 
 constexpr int MLA_POST_THREADS = 256;
 
-// One CTA per row.
+__device__ __forceinline__ void mla_store_split4(float4 y, __nv_bfloat16 *hi, __nv_bfloat16 *lo) {
+  __nv_bfloat16 a[4], b[4];
+  mla_split_bf16(y.x, a[0], b[0]);
+  mla_split_bf16(y.y, a[1], b[1]);
+  mla_split_bf16(y.z, a[2], b[2]);
+  mla_split_bf16(y.w, a[3], b[3]);
+  *reinterpret_cast<uint2 *>(hi) = *reinterpret_cast<const uint2 *>(a);
+  *reinterpret_cast<uint2 *>(lo) = *reinterpret_cast<const uint2 *>(b);
+}
+// (a, b) pairs of four consecutive rotation indices -> rotated (a', b'); t: (cos, sin) of those indices
+__device__ __forceinline__ void mla_rotate4(const float4 a, const float4 b, const float2 *t, float4 &ra, float4 &rb) {
+  const float4 t01 = *reinterpret_cast<const float4 *>(t), t23 = *reinterpret_cast<const float4 *>(t + 2);
+  ra = make_float4(a.x * t01.x - b.x * t01.y, a.y * t01.z - b.y * t01.w, a.z * t23.x - b.z * t23.y, a.w * t23.z - b.w * t23.w);
+  rb = make_float4(a.x * t01.y + b.x * t01.x, a.y * t01.w + b.y * t01.z, a.z * t23.y + b.z * t23.x, a.w * t23.w + b.w * t23.z);
+}
+
+// One CTA per row; four consecutive columns per thread and pass (nope, rope / 2 and rank are multiples of 4).
 __global__ void __launch_bounds__(MLA_POST_THREADS)
 mla_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, MlaDims d, const __nv_bfloat16 *__restrict__ gains,
                 float eps, MlaCache cache, int rows_per_head, __nv_bfloat16 *__restrict__ qn_hi, __nv_bfloat16 *__restrict__ qn_lo,
@@ -30,25 +46,9 @@ mla_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, Mla
   if (rows.active[r] == 0) return;                   // a padding row: no cache write, its query is never used
   const int pos = rows.pos[r];
   const int qw = d.nope + d.rope, QD = d.nh * qw, half = d.rope >> 1;
-  // ---- the query: no-rope parts as bf16 hi/lo (head-major), rotary parts rotated, fp32
-  for (int i = tid; i < d.nh * d.nope; i += MLA_POST_THREADS) {
-    const int h = i / d.nope, j = i - h * d.nope;
-    __nv_bfloat16 a, b;
-    mla_split_bf16(gemm_load(qkv, r, h * qw + j), a, b);
-    const size_t o = ((size_t)h * rows_per_head + r) * d.nope + j;
-    qn_hi[o] = a;
-    qn_lo[o] = b;
-  }
-  for (int i = tid; i < d.nh * half; i += MLA_POST_THREADS) {
-    const int h = i / half, j = i - h * half;
-    const float a = gemm_load(qkv, r, h * qw + d.nope + j), b = gemm_load(qkv, r, h * qw + d.nope + j + half);
-    const float2 t = rope_tab[(size_t)pos * half + j];   // (cos, sin)
-    float *q = q_rope + ((size_t)r * d.nh + h) * d.rope + j;
-    q[0] = a * t.x - b * t.y;
-    q[half] = a * t.y + b * t.x;
-  }
-  // ---- the cache row: RMSNorm of the latent (sum of squares: thread-serial ascending, xor butterfly in the warp,
-  //      warp totals ascending), rotated rotary key
+  const float2 *tab = rope_tab + (size_t)pos * half;   // (cos, sin) of the row's position
+  // ---- the cache row first (the longest chain): RMSNorm of the latent (sum of squares: thread-serial ascending,
+  //      xor butterfly in the warp, warp totals ascending), rotated rotary key
 #ifdef CORUN_CHECKED
   if (!check_slot_pos(rows.slot[r], cache.n_slots, pos, cache.max_blocks, KV_BLOCK)) {
     if (tid == 0) atomicCAS(status, 0, DEV_BAD_INDEX);
@@ -63,14 +63,10 @@ mla_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, Mla
   }
 #endif
   __half *dst = cache.pool + ((size_t)blk * KV_BLOCK + pos % KV_BLOCK) * (d.rank + d.rope);
-  float x[4];                                        // rank <= 4 * threads
+  float4 x = make_float4(0.f, 0.f, 0.f, 0.f);        // rank <= 4 * threads
+  if (4 * tid < d.rank) x = gemm_load4(qkv, r, QD + 4 * tid);
   float ss = 0.f;
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const int i = tid + e * MLA_POST_THREADS;
-    x[e] = i < d.rank ? gemm_load(qkv, r, QD + i) : 0.f;
-    ss = fmaf(x[e], x[e], ss);
-  }
+  ss = fmaf(x.x, x.x, ss); ss = fmaf(x.y, x.y, ss); ss = fmaf(x.z, x.z, ss); ss = fmaf(x.w, x.w, ss);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
   if ((tid & 31) == 0) scratch[tid >> 5] = ss;
@@ -78,16 +74,35 @@ mla_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, Mla
   float tot = 0.f;
   for (int w = 0; w < MLA_POST_THREADS / 32; ++w) tot += scratch[w];
   const float inv = rsqrtf(tot / (float)d.rank + eps);
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const int i = tid + e * MLA_POST_THREADS;
-    if (i < d.rank) dst[i] = __float2half_rn(x[e] * inv * __bfloat162float(gains[i]));
+  if (4 * tid < d.rank) {
+    const uint2 raw = *reinterpret_cast<const uint2 *>(gains + 4 * tid);
+    const __nv_bfloat162 *g2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+    const float2 ga = __bfloat1622float2(g2[0]), gb = __bfloat1622float2(g2[1]);
+    __half2 o[2] = {__floats2half2_rn(x.x * inv * ga.x, x.y * inv * ga.y), __floats2half2_rn(x.z * inv * gb.x, x.w * inv * gb.y)};
+    *reinterpret_cast<uint2 *>(dst + 4 * tid) = *reinterpret_cast<const uint2 *>(o);
   }
-  if (tid < half) {
-    const float a = gemm_load(qkv, r, QD + d.rank + tid), b = gemm_load(qkv, r, QD + d.rank + tid + half);
-    const float2 t = rope_tab[(size_t)pos * half + tid];
-    dst[d.rank + tid] = __float2half_rn(a * t.x - b * t.y);
-    dst[d.rank + tid + half] = __float2half_rn(a * t.y + b * t.x);
+  if (4 * tid < half) {
+    const int j = 4 * tid;
+    float4 ra, rb;
+    mla_rotate4(gemm_load4(qkv, r, QD + d.rank + j), gemm_load4(qkv, r, QD + d.rank + j + half), tab + j, ra, rb);
+    __half2 oa[2] = {__floats2half2_rn(ra.x, ra.y), __floats2half2_rn(ra.z, ra.w)};
+    __half2 ob[2] = {__floats2half2_rn(rb.x, rb.y), __floats2half2_rn(rb.z, rb.w)};
+    *reinterpret_cast<uint2 *>(dst + d.rank + j) = *reinterpret_cast<const uint2 *>(oa);
+    *reinterpret_cast<uint2 *>(dst + d.rank + j + half) = *reinterpret_cast<const uint2 *>(ob);
+  }
+  // ---- the query: no-rope parts as bf16 hi/lo (head-major), rotary parts rotated, fp32
+  for (int i = 4 * tid; i < d.nh * d.nope; i += 4 * MLA_POST_THREADS) {
+    const int h = i / d.nope, j = i - h * d.nope;
+    const size_t o = ((size_t)h * rows_per_head + r) * d.nope + j;
+    mla_store_split4(gemm_load4(qkv, r, h * qw + j), qn_hi + o, qn_lo + o);
+  }
+  for (int i = 4 * tid; i < d.nh * half; i += 4 * MLA_POST_THREADS) {
+    const int h = i / half, j = i - h * half;
+    float4 ra, rb;
+    mla_rotate4(gemm_load4(qkv, r, h * qw + d.nope + j), gemm_load4(qkv, r, h * qw + d.nope + j + half), tab + j, ra, rb);
+    float *q = q_rope + ((size_t)r * d.nh + h) * d.rope + j;
+    *reinterpret_cast<float4 *>(q) = ra;
+    *reinterpret_cast<float4 *>(q + half) = rb;
   }
 }
 
