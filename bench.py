@@ -421,11 +421,11 @@ def run_corun(args, rank, world):
         lop.sync()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for _ in range(20):
+        for _ in range(100):
             lop.run(lq, lr, lpool, ltable, ldctx, 1.0 / math.sqrt(128 + ldr))
         e1.record()
         lop.sync()
-        lms = e0.elapsed_time(e1) / 20
+        lms = e0.elapsed_time(e1) / 100
         mla = {"workload": "deepseek_v2_lite_mla_b128", "contexts": f"uniform {lctx.min()}..{lctx.max()}", "cache": "paged, 16 tokens per page",
                "cache_bytes": lbytes, "us_per_call": lms * 1e3, "GBs": lbytes / lms / 1e6, "frac_of_measured_hbm": lbytes / lms / 1e6 / hbm,
                "operands": "fp16 hi + lo pairs (tcgen05)"}

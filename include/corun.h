@@ -51,8 +51,8 @@ typedef struct corun_engine corun_engine; /* opaque, owned by the library */
 /* Decoder shape.  arch 0 = dense GQA decoder: pre-norm RMSNorm, half-split
  * RoPE on q and k, causal softmax attention, SwiGLU FFN, untied LM head, no
  * biases.  Requirements: hidden, ffn and n_q_heads*head_dim multiples of 64;
- * head_dim 64 or 128; n_q_heads / n_kv_heads in {1,2,4,8}.  arch is 0 here; the other
- * architectures have their own creation calls (corun_init_moe, corun_init_mla), which take arch 0 too. */
+ * head_dim 64 or 128; n_q_heads / n_kv_heads in {1,2,4,8}.  arch 1 = decoder with multi-head latent
+ * attention: accepted by corun_init_mla only (which takes 0 as well and ignores n_kv_heads and head_dim). */
 typedef struct {
   int32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
   float rms_eps, rope_theta;

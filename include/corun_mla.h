@@ -5,7 +5,7 @@
  *
  * The paper evaluates an MLA model (Evaluation, "Setup") and turns decode-time Split-KV off because its split
  * count depends on the batch (Design, "Fixed-Shape Batched Decode"); here, as in the dense attention kernel,
- * the split size is fixed (128 tokens) and the split count depends on the row's own context length only, so a
+ * the split size is fixed (256 tokens) and the split count depends on the row's own context length only, so a
  * row's result does not depend on the other rows of the step, nor on where its pages lie in the pool.
  *
  * Per cached token the cache holds the latent c_t [d_c] followed by the shared rotary key r_t [d_r] (fp16,
@@ -31,7 +31,7 @@ extern "C" {
 int64_t corun_mla_workspace_floats(int32_t B, int32_t n_heads, int32_t d_latent, int32_t max_context);
 
 /*
- *   q_lat        fp32 [B, n_heads, d_latent]      q_rope  fp32 [B, n_heads, d_rope]
+ *   q_lat        fp32 [B, n_heads, d_latent]      q_rope  fp32 [B, n_heads, d_rope]   (both 16-byte aligned)
  *   pool         fp16 [pool_pages][16 tokens][d_latent + d_rope]: the page pool (16-byte aligned).  Every value
  *                of a page that is listed for a row must be finite, also at positions beyond the row's context
  *                (they are multiplied by zero weights)

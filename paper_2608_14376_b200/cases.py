@@ -519,7 +519,6 @@ def main():
     ma = sub.add_parser("mla")
     ma.add_argument("--B", type=int, default=128); ma.add_argument("--ctx-lo", type=int, default=512)
     ma.add_argument("--ctx-hi", type=int, default=4096); ma.add_argument("--reps", type=int, default=10)
-    ma.add_argument("--single", action="store_true", help="single fp16 operands instead of hi + lo pairs")
     ab = sub.add_parser("ablation")
     ab.add_argument("--layers", type=int, default=2); ab.add_argument("--B", type=int, default=64)
     ab.add_argument("--actives", default="1,4,16,40,64"); ab.add_argument("--ctx-lo", type=int, default=512)

@@ -47,8 +47,6 @@ mla_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, Mla
   const int pos = rows.pos[r];
   const int qw = d.nope + d.rope, QD = d.nh * qw, half = d.rope >> 1;
   const float2 *tab = rope_tab + (size_t)pos * half;   // (cos, sin) of the row's position
-  // ---- the cache row first (the longest chain): RMSNorm of the latent (sum of squares: thread-serial ascending,
-  //      xor butterfly in the warp, warp totals ascending), rotated rotary key
 #ifdef CORUN_CHECKED
   if (!check_slot_pos(rows.slot[r], cache.n_slots, pos, cache.max_blocks, KV_BLOCK)) {
     if (tid == 0) atomicCAS(status, 0, DEV_BAD_INDEX);
@@ -63,8 +61,35 @@ mla_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, Mla
   }
 #endif
   __half *dst = cache.pool + ((size_t)blk * KV_BLOCK + pos % KV_BLOCK) * (d.rank + d.rope);
+  // the latent's values are requested first and used last: the sums of the GEMM's partials behind every load
+  // below overlap instead of queueing behind the block-wide reduction
   float4 x = make_float4(0.f, 0.f, 0.f, 0.f);        // rank <= 4 * threads
   if (4 * tid < d.rank) x = gemm_load4(qkv, r, QD + 4 * tid);
+  // ---- the query: no-rope parts as bf16 hi/lo (head-major), rotary parts rotated, fp32
+  for (int i = 4 * tid; i < d.nh * d.nope; i += 4 * MLA_POST_THREADS) {
+    const int h = i / d.nope, j = i - h * d.nope;
+    const size_t o = ((size_t)h * rows_per_head + r) * d.nope + j;
+    mla_store_split4(gemm_load4(qkv, r, h * qw + j), qn_hi + o, qn_lo + o);
+  }
+  for (int i = 4 * tid; i < d.nh * half; i += 4 * MLA_POST_THREADS) {
+    const int h = i / half, j = i - h * half;
+    float4 ra, rb;
+    mla_rotate4(gemm_load4(qkv, r, h * qw + d.nope + j), gemm_load4(qkv, r, h * qw + d.nope + j + half), tab + j, ra, rb);
+    float *q = q_rope + ((size_t)r * d.nh + h) * d.rope + j;
+    *reinterpret_cast<float4 *>(q) = ra;
+    *reinterpret_cast<float4 *>(q + half) = rb;
+  }
+  // ---- the cache row: rotated rotary key; RMSNorm of the latent (sum of squares: thread-serial ascending, xor
+  //      butterfly in the warp, warp totals ascending)
+  if (4 * tid < half) {
+    const int j = 4 * tid;
+    float4 ra, rb;
+    mla_rotate4(gemm_load4(qkv, r, QD + d.rank + j), gemm_load4(qkv, r, QD + d.rank + j + half), tab + j, ra, rb);
+    __half2 oa[2] = {__floats2half2_rn(ra.x, ra.y), __floats2half2_rn(ra.z, ra.w)};
+    __half2 ob[2] = {__floats2half2_rn(rb.x, rb.y), __floats2half2_rn(rb.z, rb.w)};
+    *reinterpret_cast<uint2 *>(dst + d.rank + j) = *reinterpret_cast<const uint2 *>(oa);
+    *reinterpret_cast<uint2 *>(dst + d.rank + j + half) = *reinterpret_cast<const uint2 *>(ob);
+  }
   float ss = 0.f;
   ss = fmaf(x.x, x.x, ss); ss = fmaf(x.y, x.y, ss); ss = fmaf(x.z, x.z, ss); ss = fmaf(x.w, x.w, ss);
 #pragma unroll
@@ -80,29 +105,6 @@ mla_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, Mla
     const float2 ga = __bfloat1622float2(g2[0]), gb = __bfloat1622float2(g2[1]);
     __half2 o[2] = {__floats2half2_rn(x.x * inv * ga.x, x.y * inv * ga.y), __floats2half2_rn(x.z * inv * gb.x, x.w * inv * gb.y)};
     *reinterpret_cast<uint2 *>(dst + 4 * tid) = *reinterpret_cast<const uint2 *>(o);
-  }
-  if (4 * tid < half) {
-    const int j = 4 * tid;
-    float4 ra, rb;
-    mla_rotate4(gemm_load4(qkv, r, QD + d.rank + j), gemm_load4(qkv, r, QD + d.rank + j + half), tab + j, ra, rb);
-    __half2 oa[2] = {__floats2half2_rn(ra.x, ra.y), __floats2half2_rn(ra.z, ra.w)};
-    __half2 ob[2] = {__floats2half2_rn(rb.x, rb.y), __floats2half2_rn(rb.z, rb.w)};
-    *reinterpret_cast<uint2 *>(dst + d.rank + j) = *reinterpret_cast<const uint2 *>(oa);
-    *reinterpret_cast<uint2 *>(dst + d.rank + j + half) = *reinterpret_cast<const uint2 *>(ob);
-  }
-  // ---- the query: no-rope parts as bf16 hi/lo (head-major), rotary parts rotated, fp32
-  for (int i = 4 * tid; i < d.nh * d.nope; i += 4 * MLA_POST_THREADS) {
-    const int h = i / d.nope, j = i - h * d.nope;
-    const size_t o = ((size_t)h * rows_per_head + r) * d.nope + j;
-    mla_store_split4(gemm_load4(qkv, r, h * qw + j), qn_hi + o, qn_lo + o);
-  }
-  for (int i = 4 * tid; i < d.nh * half; i += 4 * MLA_POST_THREADS) {
-    const int h = i / half, j = i - h * half;
-    float4 ra, rb;
-    mla_rotate4(gemm_load4(qkv, r, h * qw + d.nope + j), gemm_load4(qkv, r, h * qw + d.nope + j + half), tab + j, ra, rb);
-    float *q = q_rope + ((size_t)r * d.nh + h) * d.rope + j;
-    *reinterpret_cast<float4 *>(q) = ra;
-    *reinterpret_cast<float4 *>(q + half) = rb;
   }
 }
 

@@ -103,6 +103,51 @@ def test_mla_engine_parity_and_invariance(orc, first_dense, moe):
         eng.close()
 
 
+def test_mla_engine_served_together_equals_served_alone(orc):
+    """The paper's validation protocol on the MLA decoder: requests served together (sampled, through the host
+    scheduler with a pool too small for all of them, isolated and batched prefill) produce, bit for bit, the tokens
+    of each served alone."""
+    _torch()
+    from paper_2608_14376_b200 import corun
+
+    sh, mla = SMALL, dict(SMALL_MLA)
+    w_np, m_np = synth.make_mla_weights_numpy(sh, mla, seed=5)
+    e_np = synth.make_moe_numpy(sh, seed=5, **SMALL_MOE)
+    w_t, m_t = synth.mla_numpy_to_torch(w_np, m_np, "cuda")
+    eng = corun.Engine(sh, w_t, B, 128, kv_pool_blocks=24, moe=synth.moe_numpy_to_torch(e_np, "cuda"), mla=m_t)
+    try:
+        rng = np.random.default_rng(2)
+        lens = synth.uniform_lengths(8, 70, 12, seed=8)
+        prompts = synth.make_prompts(sh.vocab, lens, seed=9)
+        reqs = [dict(prompt=p, max_new=int(rng.integers(2, 12)), seed=synth.request_seed(50 + i)) for i, p in enumerate(prompts)]
+
+        def serve(subset, batched=False):
+            sch = corun.Scheduler(engine=eng)
+            if batched:
+                sch.enable_batched_prefill()
+            ids = [sch.submit(r["prompt"], r["max_new"], 0.8, 0.9, r["seed"]) for r in subset]
+            shared = 0
+            while True:
+                action, _, n = sch.step()
+                shared += action == corun.SCHED_DECODE and n >= 3
+                if action == corun.SCHED_IDLE:
+                    break
+            out = [sch.poll(i)[0] for i in ids]
+            sch.close()
+            return out, shared
+
+        together, shared = serve(reqs)
+        assert shared > 0 and eng.free_blocks() == 24
+        batched, _ = serve(reqs, batched=True)
+        for r, a, b in zip(reqs, together, batched):
+            alone, _ = serve([r])
+            assert len(a) == r["max_new"]
+            np.testing.assert_array_equal(alone[0], a)
+            np.testing.assert_array_equal(b, a)
+    finally:
+        eng.close()
+
+
 def test_mla_engine_cache_rows_are_the_oracles(orc):
     """What prefill and decode append to the latent cache (normalised latent, rotated rotary key) against the oracle's
     cache, through the debug read."""
