@@ -74,6 +74,24 @@ int corun_debug_wait_probe(uint64_t limit_ns, void *cuda_stream);
  * (cta, slot, grid).  Unused arguments are ignored.  Needs no GPU. */
 int corun_debug_check_index(int32_t kind, int64_t a, int64_t b, int64_t c, int64_t d, int64_t e, int64_t f, int64_t g);
 
+/*
+ * Micro-benchmark of three reductions with a tiling fixed for every batch size against one that adapts to it
+ * (paper, Introduction and the operator comparison of its motivation: batch-invariant kernels pay for one tiling
+ * everywhere; this library's path only keeps the tiling fixed for its one padded shape).  Not part of the
+ * decode path.
+ *   kind     0 RMSNorm of every row of x [R, N] -> y [R, N]; 1 row softmax, same shapes; 2 sum over the R rows
+ *            -> y [N]
+ *   variant  0 fixed (one CTA per row, or per 256 columns with the rows added in ascending order: a result's
+ *            bits do not depend on R); 1 adaptive (few rows: a row split over a cluster of up to 8 CTAs; kind 2:
+ *            the rows split over CTAs whose partial sums meet in atomics, so the order is not fixed at all)
+ *   x, y     device, fp32, 16-byte aligned; N a multiple of 32
+ *   avg_us   host: mean duration of `reps` launches after one warm-up launch (CUDA events on the stream)
+ *   tiling   host, may be NULL: CTAs per row (kinds 0, 1) or row chunks (kind 2) that were used
+ * Synchronous.  Errors: EINVAL, ECUDA.
+ */
+int corun_debug_microbench(int32_t kind, int32_t variant, const float *x, int32_t R, int32_t N, float *y, int32_t reps,
+                           float *avg_us, int32_t *tiling, void *cuda_stream);
+
 #ifdef CORUN_BUILD_DEBUG
 /* Runs GEMM `kind` (0 QKV, 1 O, 2 gate-up, 3 down, 4 LM head) of the decode program on one layer's
  * weights three times and returns the last launch's per-CTA timeline: stamps[cta*8 + i] (host, room for

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcorun.so")
-SOURCES = ["engine.cu", "gemm.cu", "ops.cu", "attention.cu", "attention_prefill.cu", "no_alloc.cu", "sched.cu", "moe.cu", "mla_paged.cu", "mla_layer.cu", "wait_probe.cu"]
+SOURCES = ["engine.cu", "gemm.cu", "ops.cu", "attention.cu", "attention_prefill.cu", "no_alloc.cu", "sched.cu", "moe.cu", "mla_paged.cu", "mla_layer.cu", "wait_probe.cu", "microbench.cu"]
 HEADERS = ["gemm.cuh", "ops.cuh", "ptx.cuh", "launch.cuh", "checks.cuh", os.path.join("..", "..", "include", "corun.h"),
            os.path.join("..", "..", "include", "corun_sched.h"), os.path.join("..", "..", "include", "corun_moe.h"),
            os.path.join("..", "..", "include", "corun_mla.h"), os.path.join("..", "..", "include", "corun_debug.h"), "moe.cuh", "mla.cuh"]

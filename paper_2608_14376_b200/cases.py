@@ -353,6 +353,26 @@ def case_sampler(a):
     eng.close()
 
 
+def case_microbench(a):
+    """RMSNorm, row softmax and a sum across the batch with a tiling fixed for every batch size against one that
+    adapts to it, per padded batch size R (microseconds per launch, CUDA events)."""
+    import torch
+
+    from . import corun
+
+    g = torch.Generator(device="cuda").manual_seed(0)
+    shapes = {0: a.hidden, 1: a.vocab, 2: a.hidden}
+    print("%-11s %6s %7s | %10s %10s %8s | adaptive tiling" % ("operator", "R", "N", "fixed us", "adaptive", "ratio"))
+    for kind, name in enumerate(corun.MICROBENCH_KINDS):
+        N = shapes[kind]
+        for R in a.Rs:
+            x = torch.randn((R, N), generator=g, device="cuda")
+            _, t_fixed, _ = corun.microbench(kind, 0, x, a.reps)
+            _, t_adapt, til = corun.microbench(kind, 1, x, a.reps)
+            what = ("%d CTAs per row" % til) if kind < 2 else ("%d row chunks, atomics" % til)
+            print("%-11s %6d %7d | %10.1f %10.1f %8.2f | %s" % (name, R, N, t_fixed, t_adapt, t_fixed / t_adapt, what))
+
+
 def case_sweep(a):
     import json
     import os
@@ -516,6 +536,11 @@ def main():
     mo.add_argument("--top-k", type=int, default=6); mo.add_argument("--ffn", type=int, default=1408)
     mo.add_argument("--shared", type=int, default=2)
     mo.add_argument("--renormalize", action="store_true", help="selected probabilities divided by their sum (Qwen3-MoE)")
+    mb = sub.add_parser("microbench")
+    mb.add_argument("--Rs", type=lambda v: [int(t) for t in v.split(",")], default=[1, 8, 32, 64, 128, 256, 1024, 4096])
+    mb.add_argument("--hidden", type=int, default=4096)
+    mb.add_argument("--vocab", type=int, default=151936)
+    mb.add_argument("--reps", type=int, default=50)
     ma = sub.add_parser("mla")
     ma.add_argument("--B", type=int, default=128); ma.add_argument("--ctx-lo", type=int, default=512)
     ma.add_argument("--ctx-hi", type=int, default=4096); ma.add_argument("--reps", type=int, default=10)
@@ -536,7 +561,7 @@ def main():
     tr.add_argument("--moe", action="store_true", help="the Mixture-of-Experts decoder instead of the dense one")
     tr.add_argument("--prompt-median", type=float, default=1024.0); tr.add_argument("--output-median", type=float, default=256.0)
     a = ap.parse_args()
-    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "prefill": case_prefill, "ablation": case_ablation, "mla": case_mla, "moe": case_moe, "prefill_batch": case_prefill_batch, "sampler": case_sampler,
+    {"gemm": case_gemm, "attention": case_attention, "kernels": case_kernels, "prefill": case_prefill, "ablation": case_ablation, "mla": case_mla, "microbench": case_microbench, "moe": case_moe, "prefill_batch": case_prefill_batch, "sampler": case_sampler,
      "sweep": case_sweep, "trace": case_trace}[a.case](a)
 
 

@@ -21,7 +21,7 @@ EXPORTS = [
     "corun_release", "corun_destroy", "corun_get_logits", "corun_force_token", "corun_context_len",
     "corun_free_blocks", "corun_debug_kv_read", "corun_debug_kv_write", "corun_debug_adopt",
     "corun_debug_set_eager", "corun_debug_read", "corun_debug_kv_fill", "corun_debug_time_kernel", "corun_decode_launches", "corun_debug_gemm", "corun_debug_variate",
-    "corun_debug_sample", "corun_debug_wait_probe", "corun_debug_check_index", "corun_gemm_static", "corun_strerror", "corun_last_cuda_error", "corun_engine_info",
+    "corun_debug_sample", "corun_debug_wait_probe", "corun_debug_microbench", "corun_debug_check_index", "corun_gemm_static", "corun_strerror", "corun_last_cuda_error", "corun_engine_info",
     "corun_sched_create", "corun_sched_create_for_engine", "corun_sched_destroy", "corun_sched_submit",
     "corun_sched_step", "corun_sched_poll", "corun_sched_slot_of", "corun_sched_counts",
     "corun_sched_enable_batched_prefill", "corun_prefill_geometry",
@@ -609,3 +609,23 @@ def mla_attend(q_lat, q_rope, pool, block_table, ctx, scale: float):
     out = op.run(q_lat, q_rope, pool, block_table, ctx, scale)
     op.sync()
     return out
+
+
+MICROBENCH_KINDS = ("rmsnorm", "softmax", "column_sum")
+
+
+def microbench(kind: int, variant: int, x, reps: int = 20):
+    """``corun_debug_microbench`` on a CUDA fp32 matrix x [R, N]: (y, microseconds per launch, tiling used).
+    kind: index into MICROBENCH_KINDS; variant 0 = tiling fixed for every R, 1 = adapted to R."""
+    import torch
+
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous() and x.dim() == 2
+    R, N = x.shape
+    y = torch.empty((N,) if kind == 2 else (R, N), dtype=torch.float32, device=x.device)
+    us, til = C.c_float(0.0), C.c_int32(0)
+    L = lib()
+    L.corun_debug_microbench.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32,
+                                         C.POINTER(C.c_float), C.POINTER(C.c_int32), C.c_void_p]
+    _check(L.corun_debug_microbench(kind, variant, x.data_ptr(), R, N, y.data_ptr(), reps, C.byref(us), C.byref(til),
+                                    torch.cuda.current_stream().cuda_stream), "corun_debug_microbench")
+    return y, float(us.value), int(til.value)
