@@ -575,6 +575,26 @@ def run_corun_mla(args, rank, world):
                  "note": "all %d experts of a layer are streamed every step (no expert groups: the padding that keeps a row's "
                          "result independent of its co-tenants); flops count every row through every expert" % nb}
     launches = eng.decode_launches()
+    # ---- isolated prefill of one request (its slot freed first): wall time of corun_prefill with the prompt in host
+    # memory.  A prefill row attends to its request's latent cache up to its own position with the decode kernel,
+    # so the attention part grows with the square of the prompt length.
+    prefill = None
+    n_pf = min(1024, max_ctx - 8)
+    s_pf = int(slots[0])
+    eng.release(s_pf)
+    prompt = synth.make_prompts(sh.vocab, [n_pf], seed=9)[0]
+    dt = 0.0
+    for _ in range(2):                                       # the second call is timed
+        sync_all()
+        t0 = time.perf_counter()
+        eng.prefill(s_pf, prompt, n_pf + 4, T, P, seed=7)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        eng.release(s_pf)
+    chunks = -(-n_pf // 256)
+    prefill = {"tokens": n_pf, "ms": dt * 1e3, "tok_per_s": n_pf / dt,
+               "weights_streamed_once_per_chunk_ms": chunks * (w_bytes - 2 * sh.vocab * sh.hidden) / (hbm * 1e9) * 1e3,
+               "note": "chunks of 256 rows; expert layers in their grouped form; attention by the decode kernel row by row"}
     eng.close()
     del eng, w_t, m_t, e_t
     torch.cuda.empty_cache()
@@ -638,7 +658,7 @@ def run_corun_mla(args, rank, world):
         "clocks": clk, "gpu_launches": launches * K,
         "e2e": {"value": e2e_val, "unit": "tok/s", "ms_per_step": 1e3 * e2e_s / K,
                 "h2d_bytes_per_step": B * 9, "d2h_bytes_per_step": B * 4 + 4},
-        "sustained": sustained, "roofline": roofline, "step_roofline": step_roof,
+        "sustained": sustained, "roofline": roofline, "step_roofline": step_roof, "prefill": prefill,
         "cpu_baseline": {"value": None, "unit": "tok/s", "kind": "oracle", "cores": 0,
                          "sample": "absent: the oracle of this decoder needs its 31 GB of weights as host arrays and, in its definition "
                                    "form, decompresses every cached token for every query (about 0.1 TFLOP of scalar fp64 per decode "
