@@ -232,9 +232,12 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
     // the plans carry layer 0's weights; the per-layer tensor maps override them at launch
     RC(gemm_plan_create(&P.p_qkv, e->w0_qkv, QKVN, H, P.xn_hi, P.xn_lo, R, P.BN, P.qkv_out, P.ws, e->num_sms));
     RC(gemm_plan_create(&P.p_o, e->w0_o, H, QD, P.ao_hi, P.ao_lo, R, P.BN, P.o_out, P.ws, e->num_sms));
+    // expert layers: the routing weight and the SwiGLU in the epilogue of the GEMM over all experts' gate / up rows
+    const bool moe_fused = fuse_swiglu && e->moe_E && P.BN <= 128 &&
+                           gemm_swiglu_blocks_half(e->moe_F, e->moe_E + e->moe_S, e->num_sms) > 0;
     if (fuse_swiglu && !e->moe_E && P.BN <= 128)
       RC(gemm_plan_create_swiglu(&P.p_gu, e->w0_gu, F, H, P.xn_hi, P.xn_lo, R, P.BN, P.ff_hi, P.ff_lo, e->num_sms));
-    else
+    else if (!moe_fused)
       RC(gemm_plan_create(&P.p_gu, e->w0_gu, 2 * F, H, P.xn_hi, P.xn_lo, R, P.BN, P.gu_out, P.ws, e->num_sms));
     RC(gemm_plan_create(&P.p_down, e->w0_down, H, F, P.ff_hi, P.ff_lo, R, P.BN, P.down_out, P.ws, e->num_sms));
     if (e->moe_E) {
@@ -243,7 +246,10 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
       RC(dmalloc(A, &P.moe_w, (size_t)R * NB));
       // few CTAs: the router's weights are small, and the routing kernel adds one partial per CTA for every logit
       RC(gemm_plan_create(&P.p_r, e->router_pad, GEMM_TILE_N, H, P.xn_hi, P.xn_lo, R, P.BN, P.r_out, P.ws, 8));
-      if ((2 * e->moe_F) % GEMM_TILE_N == 0) {      // a weight tile belongs to one expert: rows that did not
+      if (moe_fused)
+        RC(gemm_plan_create_swiglu_blocks(&P.p_gu, e->w0_gu, NB, e->moe_F, H, P.xn_hi, P.xn_lo, R, P.BN, P.ff_hi, P.ff_lo, P.moe_w,
+                                          e->num_sms));
+      else if ((2 * e->moe_F) % GEMM_TILE_N == 0) {   // a weight tile belongs to one expert: rows that did not
         P.p_gu.row_keep = P.moe_w;                  // select it are not stored (the SwiGLU does not read them)
         P.p_gu.keep_pitch = NB;
         P.p_gu.keep_div = 2 * e->moe_F / GEMM_TILE_N;
@@ -389,9 +395,14 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
       // stored) -> masked, weighted SwiGLU; the down GEMM then sums over the row's experts in its accumulator
       STAGE(gemm_launch(P.p_r, &e->tm_router[l], e->d_status, e->st, nullptr, true));
       STAGE(launch_moe_route(P.p_r.out(), P.R, e->moe_E, e->moe_S, e->moe_K, e->moe_renorm, P.moe_w, nullptr, nullptr, e->st));
-      STAGE(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st, tr(4 * l + 2), true));
-      STAGE(launch_moe_swiglu(P.p_gu.out(), P.moe_w, P.R, e->moe_F, e->moe_E + e->moe_S, P.ff_hi, P.ff_lo, e->st));
-      n += 2;
+      if (P.p_gu.sw_hi) {                             // routing weight and SwiGLU in the GEMM's epilogue
+        STAGE(gemm_launch(P.p_gu, &e->tm_gu_half[l], e->d_status, e->st, tr(4 * l + 2), true));
+        n += 1;
+      } else {
+        STAGE(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st, tr(4 * l + 2), true));
+        STAGE(launch_moe_swiglu(P.p_gu.out(), P.moe_w, P.R, e->moe_F, e->moe_E + e->moe_S, P.ff_hi, P.ff_lo, e->st));
+        n += 2;
+      }
     } else {
       if (P.p_gu.sw_hi) {                             // SwiGLU in the GEMM's epilogue
         STAGE(gemm_launch(P.p_gu, &e->tm_gu_half[l], e->d_status, e->st, tr(4 * l + 2), true));
@@ -622,7 +633,8 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
   e->tm_o.resize(s.n_layers);
   e->tm_gu.resize(s.n_layers);
   e->tm_down.resize(s.n_layers);
-  if (!moe) e->tm_gu_half.resize(s.n_layers);
+  const int moe_half = moe ? gemm_swiglu_blocks_half(moe->expert_ffn, moe->n_experts + moe->n_shared, e->num_sms) : 0;
+  if (!moe || moe_half) e->tm_gu_half.resize(s.n_layers);
   for (int l = 0; l < s.n_layers; ++l) {
     e->attn_norm.push_back((const bf16 *)w->attn_norm[l]);
     e->mlp_norm.push_back((const bf16 *)w->mlp_norm[l]);
@@ -639,6 +651,7 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
     if ((rc = gemm_encode_map(&e->tm_gu[l], moe ? moe->gate_up[l] : w->wgate_up[l], 2 * F, H, GEMM_TILE_N))) return fail(rc);
     if ((rc = gemm_encode_map(&e->tm_down[l], moe ? moe->down[l] : w->wdown[l], H, F, GEMM_TILE_N))) return fail(rc);
     if (!moe && (rc = gemm_encode_map(&e->tm_gu_half[l], w->wgate_up[l], 2 * F, H, gemm_swiglu_half(F, e->num_sms)))) return fail(rc);
+    if (moe && moe_half && (rc = gemm_encode_map(&e->tm_gu_half[l], moe->gate_up[l], 2 * F, H, moe_half))) return fail(rc);
   }
   if (mla) {
     // the key up-projections transposed (q_lat = W_uk^T q_nope is a GEMM over rows of W_uk^T), and per layer

@@ -41,6 +41,10 @@ constexpr uint32_t A_BLOCK_BYTES = GEMM_ROW_BLOCK * GEMM_BLOCK_K * 2;      // 16
 // sw_half up rows of the same outputs (two boxes of sw_half rows land in one stage; the MMA's N is 2 * sw_half),
 // every CTA owns whole tiles, and the epilogue writes silu(gate) * up as a bf16 hi/lo pair ([BN, F]) instead of
 // fp32 sums: no partials, no separate SwiGLU kernel.  tmW then has a box of sw_half rows.
+// SWIGLU with MASKED: W is a stack of keep_pitch such matrices (the experts of a Mixture-of-Experts layer: block e =
+// Fb gate rows, then Fb up rows, Fb = N / (2 * keep_pitch)), a tile belongs to one block (keep_div tiles per block),
+// and the epilogue writes row_keep[r, e] * silu(gate) * up, exact zeros where row r did not select block e, to
+// columns e * Fb .. of the bf16 hi/lo output [BN, N / 2].
 template <bool MASKED, bool STACKED, bool GROUPED, bool SWIGLU>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmHi,
@@ -81,6 +85,15 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   constexpr bool stacked = STACKED;                 // = (BN <= 64), fixed at compile time
   const uint32_t lo_off = stacked ? (uint32_t)(64 * GEMM_BLOCK_K * 2) : x_bytes;
   const uint32_t w_tile_bytes = SWIGLU ? (uint32_t)(2 * sw_half * GEMM_BLOCK_K * 2) : W_TILE_BYTES;
+  // SWIGLU: first gate row of a tile, and the distance to the up rows of the same outputs
+  const int sw_fb = (SWIGLU && MASKED) ? N / (2 * keep_pitch) : N / 2;
+  auto sw_gate_row = [&](int tile) {
+    if (SWIGLU && MASKED) {
+      const int e = tile / keep_div;
+      return e * 2 * sw_fb + (tile - e * keep_div) * sw_half;
+    }
+    return tile * sw_half;
+  };
   const uint32_t stage_bytes = w_tile_bytes + (stacked ? A_BLOCK_BYTES : 2 * x_bytes);
   const uint32_t tx_bytes = w_tile_bytes + 2 * x_bytes;
   const int n_rb = (BN + GEMM_ROW_BLOCK - 1) / GEMM_ROW_BLOCK;      // blocks of 128 activation rows
@@ -133,9 +146,9 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const uint32_t fb = smem_u32(&full_bar[it]);
         mbar_arrive_expect_tx(fb, tx_bytes);
         if (SWIGLU) {
-          tma_load_2d(tiles_base + (uint32_t)it * stage_bytes, &tmW, kb * GEMM_BLOCK_K, tile * sw_half, fb, pol_w);
+          tma_load_2d(tiles_base + (uint32_t)it * stage_bytes, &tmW, kb * GEMM_BLOCK_K, sw_gate_row(tile), fb, pol_w);
           tma_load_2d(tiles_base + (uint32_t)it * stage_bytes + w_tile_bytes / 2, &tmW, kb * GEMM_BLOCK_K,
-                      N / 2 + tile * sw_half, fb, pol_w);
+                      sw_gate_row(tile) + sw_fb, fb, pol_w);
         } else
         tma_load_2d(tiles_base + (uint32_t)it * stage_bytes, &tmW, (GROUPED ? g_wk + kb : kb) * GEMM_BLOCK_K,
                     GROUPED ? g_wrow + g_j * GEMM_TILE_N : tile * GEMM_TILE_N, fb, pol_w);
@@ -159,8 +172,8 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const uint32_t dst = tiles_base + (uint32_t)s * stage_bytes;
         mbar_arrive_expect_tx(fb, tx_bytes);
         if (SWIGLU) {
-          tma_load_2d(dst, &tmW, kb * GEMM_BLOCK_K, tile * sw_half, fb, pol_w);
-          tma_load_2d(dst + w_tile_bytes / 2, &tmW, kb * GEMM_BLOCK_K, N / 2 + tile * sw_half, fb, pol_w);
+          tma_load_2d(dst, &tmW, kb * GEMM_BLOCK_K, sw_gate_row(tile), fb, pol_w);
+          tma_load_2d(dst + w_tile_bytes / 2, &tmW, kb * GEMM_BLOCK_K, sw_gate_row(tile) + sw_fb, fb, pol_w);
         } else
         tma_load_2d(dst, &tmW, (GROUPED ? g_wk + kb : kb) * GEMM_BLOCK_K, GROUPED ? g_wrow + g_j * GEMM_TILE_N : tile * GEMM_TILE_N,
                     fb, pol_w);
@@ -240,7 +253,11 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         // accumulator columns 0 .. sw_half-1: gate sums of outputs tile * sw_half .., the next sw_half columns: the
         // up sums of the same outputs; every tile is whole
         const int HALF = sw_half;
-        const int F = N / 2, f0 = tile * HALF;
+        // F: outputs per block (the whole matrix unless MASKED); f0: the tile's first output inside its block;
+        // o_base: its first column in the output row of N / 2 values; blk: the block (expert) of the tile
+        const int blk = MASKED ? tile / keep_div : 0;
+        const int F = sw_fb, f0 = (MASKED ? tile - blk * keep_div : tile) * HALF;
+        const int o_pitch = N / 2, o_base = blk * F + f0;
         auto silu_mul = [](float gt, float up) { return __fdividef(gt, 1.f + __expf(-gt)) * up; };
         if (stacked) {
           const bool lo_warp = lane_base >= 64;
@@ -273,15 +290,20 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                   if (part == 0) {
                     gt[i][0] = s0; gt[i][1] = s1; gt[i][2] = s2; gt[i][3] = s3;
                   } else if (c0 + scol < HALF && f0 + c0 + scol < F) {   // HALF % 4 == 0, F % 4 == 0
-                    const float y[4] = {silu_mul(gt[i][0], s0), silu_mul(gt[i][1], s1), silu_mul(gt[i][2], s2),
-                                        silu_mul(gt[i][3], s3)};
+                    float y[4] = {silu_mul(gt[i][0], s0), silu_mul(gt[i][1], s1), silu_mul(gt[i][2], s2),
+                                  silu_mul(gt[i][3], s3)};
+                    if (MASKED) {                      // the row's routing weight for this expert; 0: not selected
+                      const float wgt = row_keep[(size_t)r * keep_pitch + blk];
+#pragma unroll
+                      for (int q = 0; q < 4; ++q) y[q] = wgt != 0.f ? wgt * y[q] : 0.f;
+                    }
                     __nv_bfloat16 a[4], b[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                       a[q] = __float2bfloat16_rn(y[q]);
                       b[q] = __float2bfloat16_rn(y[q] - __bfloat162float(a[q]));
                     }
-                    const size_t o = (size_t)r * F + f0 + c0 + scol;
+                    const size_t o = (size_t)r * o_pitch + o_base + c0 + scol;
                     *reinterpret_cast<uint2 *>(sw_hi + o) = *reinterpret_cast<const uint2 *>(a);
                     *reinterpret_cast<uint2 *>(sw_lo + o) = *reinterpret_cast<const uint2 *>(b);
                   }
@@ -304,14 +326,16 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
               tmem_ld8(ta + HALF, vu);
               tmem_ld_wait();
               if (row >= R) continue;
+              const float wgt = MASKED ? row_keep[(size_t)row * keep_pitch + blk] : 1.f;
               __nv_bfloat16 a[8], b[8];
 #pragma unroll
               for (int q = 0; q < 8; ++q) {
-                const float y = silu_mul(__uint_as_float(vg[q]), __uint_as_float(vu[q]));
+                float y = silu_mul(__uint_as_float(vg[q]), __uint_as_float(vu[q]));
+                if (MASKED) y = wgt != 0.f ? wgt * y : 0.f;
                 a[q] = __float2bfloat16_rn(y);
                 b[q] = __float2bfloat16_rn(y - __bfloat162float(a[q]));
               }
-              const size_t o = (size_t)row * F + f0 + c0;
+              const size_t o = (size_t)row * o_pitch + o_base + c0;
               *reinterpret_cast<uint4 *>(sw_hi + o) = *reinterpret_cast<const uint4 *>(a);
               *reinterpret_cast<uint4 *>(sw_lo + o) = *reinterpret_cast<const uint4 *>(b);
             }
@@ -616,6 +640,69 @@ int gemm_plan_create_swiglu(GemmPlan *p, const void *W, int F, int K, const void
   return CORUN_OK;
 }
 
+int gemm_swiglu_blocks_half(int Fb, int n_blocks, int num_sms) {
+  // the widest tile (a multiple of 8 gate rows that divides Fb, 64..128) for which the busiest CTA streams the
+  // fewest weight rows; wider tiles mean fewer MMA instructions per byte, so ties go to the wider one
+  int best = 0;
+  long long best_cost = 0;
+  for (int half = GEMM_TILE_N / 2; half >= 64; half -= 8) {
+    if (Fb % half) continue;
+    const long long tiles = (long long)n_blocks * (Fb / half);
+    const long long cost = (tiles + num_sms - 1) / num_sms * half;
+    if (!best || cost < best_cost) { best = half; best_cost = cost; }
+  }
+  return best;
+}
+
+int gemm_plan_create_swiglu_blocks(GemmPlan *p, const void *W, int n_blocks, int Fb, int K, const void *Xhi, const void *Xlo,
+                                   int R, int BN, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, const float *row_scale,
+                                   int num_sms) {
+  if (n_blocks < 1 || Fb <= 0 || Fb % 8 || K <= 0 || K % GEMM_BLOCK_K || BN % 16 || BN < 16 || BN > 256 || R < 1 || R > BN ||
+      !out_hi || !out_lo || !row_scale || num_sms < 1)
+    return CORUN_EINVAL;
+  const int HALF = gemm_swiglu_blocks_half(Fb, n_blocks, num_sms);
+  if (!HALF) return CORUN_EINVAL;
+  p->sw_half = HALF;
+  p->N = n_blocks * 2 * Fb; p->K = K; p->R = R; p->BN = BN;
+  p->n_tiles = n_blocks * (Fb / HALF);
+  p->KB = K / GEMM_BLOCK_K;
+  p->grid = p->n_tiles < num_sms ? p->n_tiles : num_sms;
+  if ((long long)p->n_tiles * p->KB >= (1ll << 31)) return CORUN_EINVAL;
+  const size_t stage = (size_t)2 * HALF * GEMM_BLOCK_K * 2 + (BN <= 64 ? (size_t)A_BLOCK_BYTES : 2 * (size_t)BN * GEMM_BLOCK_K * 2);
+  int stages = (int)((GEMM_MAX_DYN_SMEM - 1024 - A_BLOCK_BYTES) / stage);
+  if (stages > MAX_STAGES) stages = MAX_STAGES;
+  if (stages < 2) return CORUN_EINVAL;
+  p->stages = stages;
+  p->smem_bytes = stage * stages + A_BLOCK_BYTES + 1024;
+  p->tmem_cols = 512;
+  p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * HALF) >> 3) << 17) |
+             ((uint32_t)(GEMM_ROW_BLOCK >> 4) << 24);
+  p->direct = nullptr;
+  p->ws = nullptr;
+  p->sw_hi = out_hi;
+  p->sw_lo = out_lo;
+  p->row_keep = row_scale;
+  p->keep_pitch = n_blocks;
+  p->keep_div = Fb / HALF;
+  int rc;
+  if ((rc = gemm_encode_map(&p->tmW, W, n_blocks * 2 * Fb, K, HALF)) != 0) return rc;
+  if ((rc = gemm_encode_map(&p->tmHi, Xhi, BN, K, BN)) != 0) return rc;
+  if ((rc = gemm_encode_map(&p->tmLo, Xlo, BN, K, BN)) != 0) return rc;
+  // whole tiles only: CTA c takes tiles [c * n_tiles / grid, (c + 1) * n_tiles / grid)
+  std::vector<int> tab((size_t)p->grid + 1);
+  for (int c = 0; c <= p->grid; ++c) tab[(size_t)c] = (int)((long long)c * p->n_tiles / p->grid) * p->KB;
+  int *d_tab = nullptr;
+  if (cudaMalloc(&d_tab, tab.size() * sizeof(int)) != cudaSuccess) return CORUN_ENOMEM;
+  cudaError_t me = cudaMemcpy(d_tab, tab.data(), tab.size() * sizeof(int), cudaMemcpyHostToDevice);
+  if (me != cudaSuccess) { g_last_cuda_error = (int)me; cudaFree(d_tab); return CORUN_ECUDA; }
+  p->d_cta_start = d_tab;
+  p->d_tile_first = p->d_tile_cend = p->d_split_tiles = nullptr;
+  p->n_split_tiles = 0;
+  cudaError_t ae = gemm_prepare_kernel();
+  if (ae != cudaSuccess) { g_last_cuda_error = (int)ae; return CORUN_ECUDA; }
+  return CORUN_OK;
+}
+
 int gemm_plan_create_grouped(GemmPlan *p, const void *W, long long w_rows, int w_cols, int N, int K, const void *Xhi,
                              const void *Xlo, int n_groups, int BN, float *direct, const int *group_tab) {
   if (N <= 0 || N % GEMM_TILE_N || K <= 0 || K % GEMM_BLOCK_K || w_cols % GEMM_BLOCK_K || BN % 16 || BN < 16 || BN > 64 ||
@@ -664,6 +751,8 @@ cudaError_t gemm_prepare_kernel() {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   return e;
 }
 
@@ -681,6 +770,7 @@ cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int 
                     p.row_keep, p.keep_pitch, p.keep_div, p.group_tab, p.tiles_per_group, d_status, trace, p.sw_hi, p.sw_lo,
                     p.sw_half);
   };
+  if (p.sw_hi && masked) return stacked ? go(gemm_streamk_kernel<true, true, false, true>) : go(gemm_streamk_kernel<true, false, false, true>);
   if (p.sw_hi) return stacked ? go(gemm_streamk_kernel<false, true, false, true>) : go(gemm_streamk_kernel<false, false, false, true>);
   if (p.group_tab) return go(gemm_streamk_kernel<false, true, true, false>);
   if (masked) return stacked ? go(gemm_streamk_kernel<true, true, false, false>) : go(gemm_streamk_kernel<true, false, false, false>);

@@ -119,6 +119,15 @@ int gemm_plan_create_grouped(GemmPlan *p, const void *W, long long w_rows, int w
 int gemm_swiglu_half(int F, int num_sms);
 int gemm_plan_create_swiglu(GemmPlan *p, const void *W, int F, int K, const void *Xhi, const void *Xlo, int R, int BN,
                             __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int num_sms);
+// The same for a stack of n_blocks gate / up matrices (the experts of a Mixture-of-Experts layer): W is
+// [n_blocks * 2 * Fb, K], block e = Fb gate rows then Fb up rows; out_hi / out_lo [BN, n_blocks * Fb] receive
+// row_scale[r * n_blocks + e] * silu(gate) * up in columns e * Fb .., exact zeros where the scale is zero (the
+// row did not select the expert).  A tile is gemm_swiglu_blocks_half(Fb, n_blocks, num_sms) gate rows of one
+// block with their up rows (0: no multiple of 8 in 64..128 divides Fb); whole tiles, no partials.
+int gemm_swiglu_blocks_half(int Fb, int n_blocks, int num_sms);
+int gemm_plan_create_swiglu_blocks(GemmPlan *p, const void *W, int n_blocks, int Fb, int K, const void *Xhi, const void *Xlo,
+                                   int R, int BN, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, const float *row_scale,
+                                   int num_sms);
 // The allocation-free half of gemm_plan_create: fills every host-side field and tensor map of the
 // plan and writes the partition tables (cta_start, tile_first, tile_cend, split_tiles) to `tab`
 // (capacity tab_cap ints; *tab_ints = ints used).  gemm_plan_bind_tables points the plan at a device

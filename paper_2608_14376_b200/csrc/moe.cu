@@ -392,11 +392,15 @@ int corun_moe_create(const corun_moe_shape *shape, const void *router, const voi
   if (cudaMemcpy(m->router_pad, router, (size_t)E * H * sizeof(bf16), cudaMemcpyDeviceToDevice) != cudaSuccess)
     return fail(CORUN_ECUDA);
   // the three GEMMs run one after the other and their results are consumed in between: one workspace serves all
+  // up to 128 rows the first GEMM applies the routing weight and the SwiGLU in its epilogue (where a tile width
+  // divides the experts' width); else it stores gate / up sums and a kernel of its own follows
+  const bool fused = m->BN <= 128 && gemm_swiglu_blocks_half(F, NB, m->num_sms) > 0;
   if ((rc = gemm_plan_create(&m->p_r, m->router_pad, GEMM_TILE_N, H, m->x_hi, m->x_lo, B, m->BN, m->out_r, m->ws, 8)) ||
-      (rc = gemm_plan_create(&m->p_gu, gate_up, (int)N1, H, m->x_hi, m->x_lo, B, m->BN, m->out_gu, m->ws, m->num_sms)) ||
+      (rc = fused ? gemm_plan_create_swiglu_blocks(&m->p_gu, gate_up, NB, F, H, m->x_hi, m->x_lo, B, m->BN, m->h_hi, m->h_lo, m->w, m->num_sms)
+                  : gemm_plan_create(&m->p_gu, gate_up, (int)N1, H, m->x_hi, m->x_lo, B, m->BN, m->out_gu, m->ws, m->num_sms)) ||
       (rc = gemm_plan_create(&m->p_d, down, H, (int)K2, m->h_hi, m->h_lo, B, m->BN, m->out_d, m->ws, m->num_sms)))
     return fail(rc);
-  if ((2 * F) % GEMM_TILE_N == 0) {                 // a weight tile then belongs to one expert: skip the rows that
+  if (!fused && (2 * F) % GEMM_TILE_N == 0) {       // a weight tile then belongs to one expert: skip the rows that
     m->p_gu.row_keep = m->w;                        // did not select it (the SwiGLU kernel does not read them)
     m->p_gu.keep_pitch = NB;
     m->p_gu.keep_div = 2 * F / GEMM_TILE_N;
@@ -426,7 +430,7 @@ int corun_moe_forward(corun_moe *m, const float *x, float *y, int32_t *experts, 
   MCK(gemm_launch(m->p_r, nullptr, m->d_status, m->st, nullptr, true));
   MCK(launch_moe_route(m->p_r.out(), m->B, E, s.n_shared, s.top_k, s.renormalize, m->w, experts, probs, m->st));
   MCK(gemm_launch(m->p_gu, nullptr, m->d_status, m->st, nullptr, true));
-  MCK(launch_moe_swiglu(m->p_gu.out(), m->w, m->B, F, NB, m->h_hi, m->h_lo, m->st));
+  if (!m->p_gu.sw_hi) MCK(launch_moe_swiglu(m->p_gu.out(), m->w, m->B, F, NB, m->h_hi, m->h_lo, m->st));
   MCK(gemm_launch(m->p_d, nullptr, m->d_status, m->st, nullptr, true));
   MCK(launch_k(moe_readout_kernel, dim3((H / 4 + 255) / 256, m->B), dim3(256), 0, m->st, true, m->p_d.out(), H, y));
   return CORUN_OK;
@@ -442,6 +446,6 @@ int corun_moe_sync(corun_moe *m) {
 
 int64_t corun_moe_weight_bytes(const corun_moe *m) { return m ? m->weight_bytes : 0; }
 
-int corun_moe_launches(const corun_moe *m) { return m ? 7 : CORUN_EINVAL; }
+int corun_moe_launches(const corun_moe *m) { return m ? (m->p_gu.sw_hi ? 6 : 7) : CORUN_EINVAL; }
 
 }  // extern "C"

@@ -88,7 +88,8 @@ def test_moe_matches_oracle_and_is_position_invariant(H, E, K, F, S, B, renorm):
     y3, _, _ = op.forward(torch.tensor(X2).cuda())
     op.sync()
     assert y3.cpu().numpy().tobytes() == y2.tobytes()
-    assert op.launches() == 7
+    # six kernels where the first GEMM applies the SwiGLU itself (up to 128 rows, a tile width of 64..128 dividing F), else seven
+    assert op.launches() in (6, 7)
     op.close()
 
 
