@@ -233,7 +233,9 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
     RC(gemm_plan_create(&P.p_qkv, e->w0_qkv, QKVN, H, P.xn_hi, P.xn_lo, R, P.BN, P.qkv_out, P.ws, e->num_sms));
     RC(gemm_plan_create(&P.p_o, e->w0_o, H, QD, P.ao_hi, P.ao_lo, R, P.BN, P.o_out, P.ws, e->num_sms));
     // expert layers: the routing weight and the SwiGLU in the epilogue of the GEMM over all experts' gate / up rows
-    const bool moe_fused = fuse_swiglu && e->moe_E && P.BN <= 128 &&
+    // (65..128 rows; up to 64 rows the masked store plus a SwiGLU kernel measured faster: the epilogue would write
+    // zeros for every pair that was not selected through the shared-memory exchange of the stacked path)
+    const bool moe_fused = fuse_swiglu && e->moe_E && P.BN > 64 && P.BN <= 128 &&
                            gemm_swiglu_blocks_half(e->moe_F, e->moe_E + e->moe_S, e->num_sms) > 0;
     if (fuse_swiglu && !e->moe_E && P.BN <= 128)
       RC(gemm_plan_create_swiglu(&P.p_gu, e->w0_gu, F, H, P.xn_hi, P.xn_lo, R, P.BN, P.ff_hi, P.ff_lo, e->num_sms));

@@ -392,9 +392,10 @@ int corun_moe_create(const corun_moe_shape *shape, const void *router, const voi
   if (cudaMemcpy(m->router_pad, router, (size_t)E * H * sizeof(bf16), cudaMemcpyDeviceToDevice) != cudaSuccess)
     return fail(CORUN_ECUDA);
   // the three GEMMs run one after the other and their results are consumed in between: one workspace serves all
-  // up to 128 rows the first GEMM applies the routing weight and the SwiGLU in its epilogue (where a tile width
-  // divides the experts' width); else it stores gate / up sums and a kernel of its own follows
-  const bool fused = m->BN <= 128 && gemm_swiglu_blocks_half(F, NB, m->num_sms) > 0;
+  // from 65 to 128 rows the first GEMM applies the routing weight and the SwiGLU in its epilogue (where a tile
+  // width divides the experts' width); else it stores gate / up sums and a kernel of its own follows (faster up to
+  // 64 rows, where the masked store skips most of the output)
+  const bool fused = m->BN > 64 && m->BN <= 128 && gemm_swiglu_blocks_half(F, NB, m->num_sms) > 0;
   if ((rc = gemm_plan_create(&m->p_r, m->router_pad, GEMM_TILE_N, H, m->x_hi, m->x_lo, B, m->BN, m->out_r, m->ws, 8)) ||
       (rc = fused ? gemm_plan_create_swiglu_blocks(&m->p_gu, gate_up, NB, F, H, m->x_hi, m->x_lo, B, m->BN, m->h_hi, m->h_lo, m->w, m->num_sms)
                   : gemm_plan_create(&m->p_gu, gate_up, (int)N1, H, m->x_hi, m->x_lo, B, m->BN, m->out_gu, m->ws, m->num_sms)) ||

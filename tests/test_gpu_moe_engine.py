@@ -54,7 +54,7 @@ def test_moe_engine_parity_and_invariance(orc, E, K, F, S, renorm):
                 worst = max(worst, float(np.abs(eng.logits(s) - r.logits).max()))
             trace.append([eng.logits(s).tobytes() for s in slots])
         assert worst <= TOL, worst
-        assert eng.decode_launches() == 7 + 11 * sh.n_layers   # per layer: 4 + 2 GEMMs (the masked SwiGLU in the gate / up GEMM's epilogue), 2 norms, RoPE, attention (splits, combine), routing
+        assert eng.decode_launches() == 7 + 12 * sh.n_layers   # per layer: 4 + 2 GEMMs, 2 norms, RoPE, attention (splits, combine), masked SwiGLU, routing
 
         # the same requests in other slots, two of them alone, then all in one batched prefill: same bytes
         for s in slots:
@@ -88,6 +88,50 @@ def test_moe_engine_parity_and_invariance(orc, E, K, F, S, renorm):
             eng.decode_step(active, seeds)
             solo.decode(force_token=t)
             assert eng.logits(2).tobytes() == trace[step][0]
+    finally:
+        eng.close()
+
+
+def test_moe_engine_with_more_than_64_slots(orc):
+    """From 65 to 128 padded rows the expert layers' first GEMM applies the routing weight and the SwiGLU in its
+    epilogue (one kernel fewer per layer): parity with the oracle and the same bytes in other slots."""
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2608_14376_b200 import corun
+
+    sh, Bw = synth.TINY, 96
+    w_np = synth.make_weights_numpy(sh, seed=4)
+    m_np = synth.make_moe_numpy(sh, 8, 2, 128, 1, False, seed=4)
+    model = orc.Model(orc.Shape(**sh.dict()), w_np, moe=m_np)
+    eng = corun.Engine(sh, synth.weights_numpy_to_torch(w_np, "cuda"), Bw, MAX_CTX, moe=synth.moe_numpy_to_torch(m_np, "cuda"))
+    try:
+        assert eng.decode_launches() == 7 + 11 * sh.n_layers
+        prompts = synth.make_prompts(sh.vocab, [30, 77, 12], seed=6)
+        seeds = np.zeros(Bw, np.uint64)
+        traces = []
+        for slots in ([3, 70, 95], [64, 0, 41]):
+            reqs = [orc.Request(model, p, 1, max_T=MAX_CTX) for p in prompts]
+            worst = 0.0
+            for s, p, r in zip(slots, prompts, reqs):
+                r.prefill()
+                eng.prefill(s, p, len(p) + 8)
+            active = np.zeros(Bw, np.uint8); active[slots] = 1
+            trace = []
+            for _ in range(3):
+                toks = [int(np.argmax(r.logits)) for r in reqs]
+                for s, t in zip(slots, toks):
+                    eng.force_token(s, t)
+                eng.decode_step(active, seeds)
+                for s, r, t in zip(slots, reqs, toks):
+                    r.decode(force_token=t)
+                    worst = max(worst, float(np.abs(eng.logits(s) - r.logits).max()))
+                trace.append([eng.logits(s).tobytes() for s in slots])
+            assert worst <= TOL, worst
+            traces.append(trace)
+            for s in slots:
+                eng.release(s)
+        assert traces[0] == traces[1]
     finally:
         eng.close()
 
@@ -226,5 +270,5 @@ def test_moe_engine_argument_errors(orc):
             corun.Engine(sh, w_t, B, MAX_CTX, moe=dict(good, **bad))
         assert ei.value.status == corun.EINVAL
     eng = corun.Engine(sh, w_t, B, MAX_CTX, moe=good)      # and the good one still initialises
-    assert eng.decode_launches() == 7 + 11 * sh.n_layers   # per layer: 4 + 2 GEMMs (the masked SwiGLU in the gate / up GEMM's epilogue), 2 norms, RoPE, attention (splits, combine), routing
+    assert eng.decode_launches() == 7 + 12 * sh.n_layers   # per layer: 4 + 2 GEMMs, 2 norms, RoPE, attention (splits, combine), masked SwiGLU, routing
     eng.close()
