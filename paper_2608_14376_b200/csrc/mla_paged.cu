@@ -476,20 +476,28 @@ __global__ void __launch_bounds__(128) mla_paged_combine_kernel(const float2 *__
                                                                 __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo,
                                                                 int rows_per_head) {
   griddep_launch_dependents();
+  __shared__ float2 sml[128];                       // the splits' (max, sum) pairs, fetched in one round trip
   const int r = (int)blockIdx.x / n_heads, h = (int)blockIdx.x - r * n_heads;
   const int d = 4 * (int)threadIdx.x;
   int c = row_pos ? (row_active[r] ? row_pos[r] + 1 : 0) : ctx[r];
-  if (c <= 0 || d >= d_c) return;                   // a padding row is left alone
+  if (c <= 0) return;                               // a padding row is left alone (the whole block returns)
   griddep_wait();
   c = c > max_blocks * MP_PAGE ? max_blocks * MP_PAGE : c;
   int ns = (c + MP_T - 1) / MP_T;
   if (ns > max_splits) ns = max_splits;
   const float2 *ml = part_ml + (size_t)r * max_splits * n_heads + h;
+  const bool staged = ns <= 128;
+  if (staged) {
+    for (int s = threadIdx.x; s < ns; s += blockDim.x) sml[s] = __ldcg(&ml[(size_t)s * n_heads]);
+    __syncthreads();
+  }
+  if (d >= d_c) return;
+  auto pair_of = [&](int s) { return staged ? sml[s] : __ldcg(&ml[(size_t)s * n_heads]); };
   float M = -CUDART_INF_F;
-  for (int s = 0; s < ns; ++s) M = fmaxf(M, __ldcg(&ml[(size_t)s * n_heads]).x);
+  for (int s = 0; s < ns; ++s) M = fmaxf(M, pair_of(s).x);
   float den = 0.f;
   for (int s = 0; s < ns; ++s) {
-    const float2 v = __ldcg(&ml[(size_t)s * n_heads]);
+    const float2 v = pair_of(s);
     den += exp2f(v.x - M) * v.y;
   }
   const float inv = 1.f / den;
@@ -503,7 +511,7 @@ __global__ void __launch_bounds__(128) mla_paged_combine_kernel(const float2 *__
     for (int e = 0; e < 4; ++e)
       if (s0 + e < ns) {
         x[e] = __ldcg(reinterpret_cast<const float4 *>(po + (size_t)(s0 + e) * stride));
-        w[e] = exp2f(__ldcg(&ml[(size_t)(s0 + e) * n_heads]).x - M);
+        w[e] = exp2f(pair_of(s0 + e).x - M);
       }
 #pragma unroll
     for (int e = 0; e < 4; ++e)
