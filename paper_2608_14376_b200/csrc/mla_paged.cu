@@ -52,6 +52,7 @@ constexpr int MP_QBLK = 32 * 128;            // bytes of one [32 rows x 64 dims]
 constexpr int MP_PBUF = (MP_T / 64 + 1) * MP_QBLK;   // one weight tile: 4 blocks of 64 tokens + overrun
 constexpr int MP_MAXH = 16;                  // heads (hi + lo rows: 32 of the operand's 64)
 constexpr int MP_MAXB = 1024;                // rows per call
+constexpr int MP_ITEM_COST = 512;            // what an item costs beyond its tokens, in tokens (score MMAs, waits and hand-offs do not shrink with it)
 constexpr int MP_THREADS = 576;
 constexpr uint32_t MP_TMEM_COLS = 512;       // S: 256 columns, O: 256 columns
 // shared memory: [ring][query tile: 9 blocks + overrun][two weight tiles]
@@ -94,6 +95,8 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   __shared__ float xs_mx[2][32], xs_sum[2][32];   // the two token halves of an item exchange maximum and sum
   __shared__ int row_start[MP_MAXB + 1];           // first item of every row
   __shared__ int row_ctx[MP_MAXB];                 // cached tokens of every row (cut to the block table's reach)
+  __shared__ int cost_start[MP_MAXB + 1];          // cost of all items before the row (tokens + MP_ITEM_COST per item)
+  __shared__ int my_items[2];                      // this CTA's stretch of the item list
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -120,27 +123,50 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
     tmem_relinquish();
   } else if (warp == 2) {
     // items per row -> first item of every row (one warp, rows in chunks of 32, ascending)
-    int run = 0;
+    int run = 0, crun = 0;
     for (int r0 = 0; r0 < B; r0 += 32) {
       const int r = r0 + lane;
-      int n = 0;
+      int n = 0, cst = 0;
       if (r < B) {
         int c = row_pos ? (row_active[r] ? row_pos[r] + 1 : 0) : ctx[r];
         c = c < 0 ? 0 : (c > max_blocks * MP_PAGE ? max_blocks * MP_PAGE : c);
         n = (c + MP_T - 1) / MP_T;
         if (n > max_splits) { n = max_splits; c = n * MP_T; }
         row_ctx[r] = c;
+        cst = c + n * MP_ITEM_COST;
       }
-      int inc = n;
+      int inc = n, cinc = cst;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
-        const int v = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += v;
+        const int v = __shfl_up_sync(0xffffffffu, inc, o), cv = __shfl_up_sync(0xffffffffu, cinc, o);
+        if (lane >= o) { inc += v; cinc += cv; }
       }
-      if (r < B) row_start[r] = run + inc - n;
+      if (r < B) { row_start[r] = run + inc - n; cost_start[r] = crun + cinc - cst; }
       run += __shfl_sync(0xffffffffu, inc, 31);
+      crun += __shfl_sync(0xffffffffu, cinc, 31);
     }
-    if (lane == 0) row_start[B] = run;
+    __syncwarp();
+    if (lane == 0) {
+      row_start[B] = run;
+      cost_start[B] = crun;
+      // The CTAs' stretches are cut where the items' accumulated cost passes k / grid of the total (an item goes to
+      // the CTA in whose share it starts), so that CTAs with cheaper (shorter) items take more of them.  Which CTA
+      // computes an item has no influence on any value.
+      auto bound = [&](int k) {
+        if (k >= (int)gridDim.x) return run;
+        const long long t = ((long long)crun * k + gridDim.x - 1) / gridDim.x;
+        int lo = 0, hi = B;                          // last row whose cost_start is <= t
+        while (hi - lo > 1) {
+          const int mid = (lo + hi) >> 1;
+          if (cost_start[mid] <= t) lo = mid; else hi = mid;
+        }
+        const int n_r = row_start[lo + 1] - row_start[lo];
+        const int sidx = (int)((t - cost_start[lo] + (MP_T + MP_ITEM_COST) - 1) / (MP_T + MP_ITEM_COST));
+        return sidx >= n_r ? row_start[lo + 1] : row_start[lo] + sidx;
+      };
+      my_items[0] = bound((int)blockIdx.x);
+      my_items[1] = bound((int)blockIdx.x + 1);
+    }
   } else if (warp >= 4) {
     // the operand tiles start out as zeros: rows of absent heads and rope columns beyond d_r stay zero
     uint4 *z = reinterpret_cast<uint4 *>(base_ptr + MP_OFF_Q);
@@ -153,7 +179,7 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   const uint32_t tmem_base = tmem_base_s;
   const uint32_t s_tmem = tmem_base, o_tmem = tmem_base + 256;
   const int n_items = row_start[B];
-  const int item_lo = (int)(((long long)n_items * blockIdx.x) / gridDim.x), item_hi = (int)(((long long)n_items * (blockIdx.x + 1)) / gridDim.x);
+  const int item_lo = my_items[0], item_hi = n_items > 0 ? my_items[1] : 0;
   const int NLB = d_c / 64;                    // latent blocks (1, 2, 4 or 8)
   const int n_half = d_c > 256 ? 2 : 1, BPH = NLB / n_half, NH = d_c / n_half;   // output halves, blocks and dims per half
   bool failed = false;
