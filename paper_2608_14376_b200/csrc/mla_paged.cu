@@ -101,7 +101,6 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
 
-  griddep_wait();                                    // (programmatic launch) the queries are the previous kernel's results
   if (tid == 0) {
     abort_flag = 0;
     for (int s = 0; s < MP_RING; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
@@ -176,6 +175,9 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  // (programmatic launch) everything above reads nothing the kernels just before this one write: the row lengths
+  // and slots are set at the start of the step; the queries and the newest cache rows are read from here on
+  griddep_wait();
   const uint32_t tmem_base = tmem_base_s;
   const uint32_t s_tmem = tmem_base, o_tmem = tmem_base + 256;
   const int n_items = row_start[B];
