@@ -216,6 +216,7 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
                                   BG, P.q_lat, P.tab_uk));
       RC(gemm_plan_create_grouped(&P.p_uv, e->w0_uv, (long long)md.nh * (md.nope + md.vh), md.rank, md.nope + md.vh, md.rank, P.ol_hi,
                                   P.ol_lo, n_groups, BG, P.uv_out, P.tab_uv));
+      P.p_uk.keep_div = P.p_uv.keep_div = -1;       // the tables are written once, here: the kernels need not wait for them
     }
     RC(dmalloc(A, &P.qkv_out, (size_t)R * QKVN));
     RC(dmalloc(A, &P.o_out, (size_t)R * H));

@@ -55,7 +55,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                     __nv_bfloat16 *__restrict__ sw_lo, int sw_half) {
   int g_id = 0, g_j = 0, g_wrow = 0, g_wk = 0, g_rows = 0;
   if (GROUPED) {
-    griddep_wait();                                 // the group table comes from an earlier kernel
+    if (keep_div >= 0) griddep_wait();              // the group table comes from an earlier kernel (keep_div < 0: it is fixed)
     g_id = (int)blockIdx.x / tiles_per_group;
     g_j = (int)blockIdx.x - g_id * tiles_per_group;
     g_wrow = group_tab[3 * g_id];

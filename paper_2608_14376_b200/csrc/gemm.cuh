@@ -88,7 +88,8 @@ struct GemmPlan {
   const float *row_keep = nullptr;
   int keep_pitch = 0, keep_div = 1;
   // Grouped mode (gemm_plan_create_grouped): one CTA per (group, weight tile); see gemm.cu.
-  const int *group_tab = nullptr;    // device, not owned: per group (first weight row, first weight k-block, rows)
+  const int *group_tab = nullptr;    // device, not owned: per group (first weight row, first weight k-block, rows);
+                                     // keep_div = -1 tells the kernel that no kernel of the same stream writes it
   int tiles_per_group = 0;
   // Gate / up GEMM with SwiGLU in the epilogue (gemm_plan_create_swiglu): the bf16 hi/lo output [BN, N / 2].
   __nv_bfloat16 *sw_hi = nullptr, *sw_lo = nullptr;
