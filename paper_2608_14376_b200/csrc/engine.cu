@@ -48,9 +48,8 @@ struct Program {
   int *sampled = nullptr, *att_work = nullptr, *att_n_work = nullptr, *att_pool = nullptr;
   GemmPlan p_qkv, p_o, p_gu, p_down, p_lm;
   // Mixture-of-Experts feed-forward layers: p_gu / p_down are then the GEMMs over all experts' gate / up rows
-  // and over the concatenated hidden activations; p_r is the router GEMM (its rows padded to one tile)
-  GemmPlan p_r;
-  float *r_out = nullptr, *moe_w = nullptr;
+  // and over the concatenated hidden activations; moe_w the rows' routing weights
+  float *moe_w = nullptr;
   // grouped form of the experts' GEMMs (prefill chunks: the rows of an expert gathered into blocks of 64)
   bool grouped = false;
   MoeGroups grp{};
@@ -89,8 +88,7 @@ struct corun_engine {
   std::vector<CUtensorMap> tm_k, tm_v;   // per layer: the pages as rows of head_dim halfs (keys and values alike)
   // Mixture-of-Experts feed-forward layers (E = 0: dense).  sh.ffn is then (E + S) * F.
   int moe_E = 0, moe_K = 0, moe_F = 0, moe_S = 0, moe_renorm = 0;
-  bf16 *router_pad = nullptr;            // [L][256][H]: each layer's router rows, zero rows behind them
-  std::vector<CUtensorMap> tm_router;
+  std::vector<const bf16 *> router;      // per layer: [E, H], borrowed
   // multi-head latent attention (corun_init_mla): sh.head_dim is the value width, the cache holds rank + rope
   // halfs per token; layers below first_dense have a dense feed-forward of width dense_ffn
   bool mla = false;
@@ -245,10 +243,7 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
     RC(gemm_plan_create(&P.p_down, e->w0_down, H, F, P.ff_hi, P.ff_lo, R, P.BN, P.down_out, P.ws, e->num_sms));
     if (e->moe_E) {
       const int NB = e->moe_E + e->moe_S;
-      RC(dmalloc(A, &P.r_out, (size_t)R * GEMM_TILE_N));
       RC(dmalloc(A, &P.moe_w, (size_t)R * NB));
-      // few CTAs: the router's weights are small, and the routing kernel adds one partial per CTA for every logit
-      RC(gemm_plan_create(&P.p_r, e->router_pad, GEMM_TILE_N, H, P.xn_hi, P.xn_lo, R, P.BN, P.r_out, P.ws, 8));
       if (moe_fused)
         RC(gemm_plan_create_swiglu_blocks(&P.p_gu, e->w0_gu, NB, e->moe_F, H, P.xn_hi, P.xn_lo, R, P.BN, P.ff_hi, P.ff_lo, P.moe_w,
                                           e->num_sms));
@@ -297,7 +292,6 @@ void program_destroy(Program &P) {
   gemm_plan_destroy(&P.p_gu);
   gemm_plan_destroy(&P.p_down);
   gemm_plan_destroy(&P.p_lm);
-  gemm_plan_destroy(&P.p_r);
   gemm_plan_destroy(&P.p_gug);
   gemm_plan_destroy(&P.p_dng);
   gemm_plan_destroy(&P.p_uk);
@@ -383,28 +377,27 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
       // router -> top-k weights -> rows grouped by expert -> gate / up, SwiGLU and down per group -> the row's
       // experts summed in ascending expert id
       const int NB = e->moe_E + e->moe_S;
-      STAGE(gemm_launch(P.p_r, &e->tm_router[l], e->d_status, e->st, nullptr, true));
-      STAGE(launch_moe_route(P.p_r.out(), P.R, e->moe_E, e->moe_S, e->moe_K, e->moe_renorm, P.moe_w, nullptr, nullptr, e->st));
+      STAGE(launch_moe_router(P.xn_hi, P.xn_lo, s.hidden, e->router[l], P.R, e->moe_E, e->moe_S, e->moe_K, e->moe_renorm, P.moe_w, nullptr,
+                              nullptr, e->st));
       STAGE(launch_moe_group(P.moe_w, P.row_active, P.R, e->moe_E, e->moe_S, e->moe_F, P.grp, e->st));
       STAGE(launch_moe_gather(P.xn_hi, P.xn_lo, s.hidden, P.grp, P.xg_hi, P.xg_lo, e->st));
       STAGE(gemm_launch(P.p_gug, &e->tm_gu[l], e->d_status, e->st, nullptr, true));
       STAGE(launch_moe_swiglu_grouped(P.gug_out, P.moe_w, NB, e->moe_F, P.grp, P.hg_hi, P.hg_lo, e->st));
       STAGE(gemm_launch(P.p_dng, &e->tm_down[l], e->d_status, e->st, nullptr, true));
       STAGE(launch_moe_combine(P.yg_out, P.row_active, P.R, NB, s.hidden, P.grp, P.down_out, e->st));
-      n += 14 + (&P == &e->dec ? 1 : 0);
+      n += 13 + (&P == &e->dec ? 1 : 0);
       continue;
     } else if (e->moe_E) {
       // router -> top-k weights -> all experts' gate / up (rows that did not select a tile's expert are not
       // stored) -> masked, weighted SwiGLU; the down GEMM then sums over the row's experts in its accumulator
-      STAGE(gemm_launch(P.p_r, &e->tm_router[l], e->d_status, e->st, nullptr, true));
-      STAGE(launch_moe_route(P.p_r.out(), P.R, e->moe_E, e->moe_S, e->moe_K, e->moe_renorm, P.moe_w, nullptr, nullptr, e->st));
+      STAGE(launch_moe_router(P.xn_hi, P.xn_lo, s.hidden, e->router[l], P.R, e->moe_E, e->moe_S, e->moe_K, e->moe_renorm, P.moe_w, nullptr,
+                              nullptr, e->st));
       if (P.p_gu.sw_hi) {                             // routing weight and SwiGLU in the GEMM's epilogue
         STAGE(gemm_launch(P.p_gu, &e->tm_gu_half[l], e->d_status, e->st, tr(4 * l + 2), true));
-        n += 1;
-      } else {
+      } else {                                        // (the router is the one kernel beyond the count below)
         STAGE(gemm_launch(P.p_gu, &e->tm_gu[l], e->d_status, e->st, tr(4 * l + 2), true));
         STAGE(launch_moe_swiglu(P.p_gu.out(), P.moe_w, P.R, e->moe_F, e->moe_E + e->moe_S, P.ff_hi, P.ff_lo, e->st));
-        n += 2;
+        n += 1;
       }
     } else {
       if (P.p_gu.sw_hi) {                             // SwiGLU in the GEMM's epilogue
@@ -674,14 +667,10 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
     }
   }
   if (moe) {
-    int rc;
-    if ((rc = dmalloc(e->allocs, &e->router_pad, (size_t)s.n_layers * GEMM_TILE_N * H))) return fail(rc);
-    e->tm_router.resize(s.n_layers);
-    for (int l = first_dense; l < s.n_layers; ++l) {
-      bf16 *dst = e->router_pad + (size_t)l * GEMM_TILE_N * H;
-      if (cudaMemcpy(dst, moe->router[l], (size_t)moe->n_experts * H * sizeof(bf16), cudaMemcpyDeviceToDevice) != cudaSuccess)
-        return fail(CORUN_ECUDA);
-      if ((rc = gemm_encode_map(&e->tm_router[l], dst, GEMM_TILE_N, H, GEMM_TILE_N))) return fail(rc);
+    if (H > 12288) return fail(CORUN_EINVAL);       // the router kernel keeps a row in shared memory
+    for (int l = 0; l < s.n_layers; ++l) {
+      if (l >= first_dense && ((uintptr_t)moe->router[l] & 15u)) return fail(CORUN_EINVAL);
+      e->router.push_back(l >= first_dense ? (const bf16 *)moe->router[l] : nullptr);
     }
   }
 

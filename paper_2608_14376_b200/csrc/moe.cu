@@ -37,25 +37,20 @@ __device__ __forceinline__ void moe_split(float x, bf16 &hi, bf16 &lo) {
   lo = __float2bfloat16_rn(x - __bfloat162float(hi));
 }
 
-// One warp per row: softmax over the E router logits, then top_k by repeated arg-max with ties to the lower
-// id.  Lane l holds experts l, l + 32, ...; the sum of the exponentials is each lane's experts in ascending
-// id, then a fixed butterfly over the lanes.  Writes the routing and the row of SwiGLU weights
+// One warp routes one row: softmax over the E router logits (load(e) gives logit e), then top_k by repeated arg-max
+// with ties to the lower id.  Lane l holds experts l, l + 32, ...; the sum of the exponentials is each lane's
+// experts in ascending id, then a fixed butterfly over the lanes.  Writes the routing and the row of SwiGLU weights
 // w[r, 0 .. E + S): p_e for the selected experts, 0 for the others, 1 for the shared ones.
-__global__ void __launch_bounds__(256) moe_route_kernel(GemmOut logits, int B, int E, int S, int top_k, int renormalize,
-                                                        float *__restrict__ w, int *__restrict__ experts,
-                                                        float *__restrict__ probs) {
-  griddep_launch_dependents();
-  griddep_wait();
-  const int lane = threadIdx.x & 31;
-  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (r >= B) return;
+template <typename LoadLogit>
+__device__ __forceinline__ void moe_route_row(LoadLogit load, int r, int lane, int E, int S, int top_k, int renormalize,
+                                              float *__restrict__ w, int *__restrict__ experts, float *__restrict__ probs) {
   constexpr int PER = MOE_MAX_EXPERTS / 32;
   float z[PER];
   float mx = -CUDART_INF_F;
 #pragma unroll
   for (int j = 0; j < PER; ++j) {
     const int e = lane + 32 * j;
-    z[j] = e < E ? gemm_load(logits, r, e) : -CUDART_INF_F;
+    z[j] = e < E ? load(e) : -CUDART_INF_F;
     mx = fmaxf(mx, z[j]);
   }
 #pragma unroll
@@ -104,6 +99,57 @@ __global__ void __launch_bounds__(256) moe_route_kernel(GemmOut logits, int B, i
       if (experts) experts[(size_t)r * top_k + k] = ids[k];
       if (probs) probs[(size_t)r * top_k + k] = p;
     }
+}
+
+// Router of one row per CTA: logits = Wr x on the CUDA cores (E dot products of H terms: far too little for a
+// tensor-core launch of its own), then the routing above.  x is the row's bf16 hi + lo pair (exactly what the
+// GEMMs of the block see); every warp takes experts warp, warp + 32, ...: a lane adds its terms in ascending
+// order (8 consecutive terms per step, the weights of four steps requested together), then a fixed butterfly
+// over the lanes.  A row's routing depends on the row alone.
+constexpr int ROUTER_THREADS = 1024;
+__global__ void __launch_bounds__(ROUTER_THREADS) moe_router_kernel(const bf16 *__restrict__ x_hi, const bf16 *__restrict__ x_lo, int H,
+                                                                    const bf16 *__restrict__ Wr, int E, int S, int top_k,
+                                                                    int renormalize, float *__restrict__ w,
+                                                                    int *__restrict__ experts, float *__restrict__ probs) {
+  griddep_launch_dependents();
+  extern __shared__ float xs[];                      // the row as fp32 [H]
+  __shared__ float logit[MOE_MAX_EXPERTS];
+  const int r = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  griddep_wait();
+  for (int i = 4 * tid; i < H; i += 4 * ROUTER_THREADS) {
+    const uint2 rh = *reinterpret_cast<const uint2 *>(x_hi + (size_t)r * H + i), rl = *reinterpret_cast<const uint2 *>(x_lo + (size_t)r * H + i);
+    const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&rh), *l2 = reinterpret_cast<const __nv_bfloat162 *>(&rl);
+    const float2 h0 = __bfloat1622float2(h2[0]), h1 = __bfloat1622float2(h2[1]), l0 = __bfloat1622float2(l2[0]), l1 = __bfloat1622float2(l2[1]);
+    *reinterpret_cast<float4 *>(xs + i) = make_float4(h0.x + l0.x, h0.y + l0.y, h1.x + l1.x, h1.y + l1.y);
+  }
+  __syncthreads();
+  for (int e = warp; e < E; e += ROUTER_THREADS / 32) {
+    const bf16 *wrow = Wr + (size_t)e * H;
+    float acc = 0.f;
+    for (int i0 = 8 * lane; i0 < H; i0 += 4 * 8 * 32) {
+      uint4 raw[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * 8 * 32;
+        raw[u] = i < H ? __ldg(reinterpret_cast<const uint4 *>(wrow + i)) : make_uint4(0u, 0u, 0u, 0u);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * 8 * 32;
+        if (i >= H) break;
+        const __nv_bfloat162 *w2 = reinterpret_cast<const __nv_bfloat162 *>(&raw[u]);
+        const float4 xa = *reinterpret_cast<const float4 *>(xs + i), xb = *reinterpret_cast<const float4 *>(xs + i + 4);
+        const float2 w0 = __bfloat1622float2(w2[0]), w1 = __bfloat1622float2(w2[1]), w2f = __bfloat1622float2(w2[2]), w3 = __bfloat1622float2(w2[3]);
+        acc = fmaf(w0.x, xa.x, acc); acc = fmaf(w0.y, xa.y, acc); acc = fmaf(w1.x, xa.z, acc); acc = fmaf(w1.y, xa.w, acc);
+        acc = fmaf(w2f.x, xb.x, acc); acc = fmaf(w2f.y, xb.y, acc); acc = fmaf(w3.x, xb.z, acc); acc = fmaf(w3.y, xb.w, acc);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) logit[e] = acc;
+  }
+  __syncthreads();
+  if (warp == 0) moe_route_row([&](int e) { return logit[e]; }, r, lane, E, S, top_k, renormalize, w, experts, probs);
 }
 
 // h[r, e*F + f] = w[r, e] * silu(gate) * up as a bf16 hi/lo pair; zeros where w[r, e] == 0 (nothing is read
@@ -316,11 +362,10 @@ cudaError_t launch_moe_combine(const float *yg, const int *active, int R, int n_
   return launch_k(moe_combine_kernel, dim3((H / 4 + 255) / 256, R), dim3(256), 0, st, true, yg, active, n_blocks, H, g, y);
 }
 
-cudaError_t launch_moe_route(const GemmOut &logits, int R, int E, int S, int top_k, int renormalize, float *w,
-                             int *experts, float *probs, cudaStream_t st) {
-  if (E < 1 || E > MOE_MAX_EXPERTS || top_k < 1 || top_k > MOE_MAX_TOPK || top_k > E) return cudaErrorInvalidValue;
-  return launch_k(moe_route_kernel, dim3((R + 7) / 8), dim3(256), 0, st, true, logits, R, E, S, top_k, renormalize, w,
-                  experts, probs);
+cudaError_t launch_moe_router(const bf16 *x_hi, const bf16 *x_lo, int H, const bf16 *Wr, int R, int E, int S, int top_k,
+                              int renormalize, float *w, int *experts, float *probs, cudaStream_t st) {
+  return launch_k(moe_router_kernel, dim3(R), dim3(ROUTER_THREADS), (size_t)H * sizeof(float), st, true, x_hi, x_lo, H, Wr, E, S, top_k,
+                  renormalize, w, experts, probs);
 }
 
 cudaError_t launch_moe_swiglu(const GemmOut &gu, const float *w, int R, int F, int n_blocks, __nv_bfloat16 *out_hi,
@@ -336,11 +381,11 @@ struct corun_moe {
   int B = 0, BN = 0, num_sms = 0;
   cudaStream_t st = nullptr;
   std::vector<void *> allocs;
-  bf16 *router_pad = nullptr;                       // [256, H]: the router rows, zero rows behind them
+  const bf16 *router = nullptr;                     // [E, H], borrowed
   bf16 *x_hi = nullptr, *x_lo = nullptr, *h_hi = nullptr, *h_lo = nullptr;
-  float *out_r = nullptr, *out_gu = nullptr, *out_d = nullptr, *ws = nullptr, *w = nullptr;
+  float *out_gu = nullptr, *out_d = nullptr, *ws = nullptr, *w = nullptr;
   int *d_status = nullptr;
-  GemmPlan p_r, p_gu, p_d;
+  GemmPlan p_gu, p_d;
   int64_t weight_bytes = 0;
 };
 
@@ -382,22 +427,20 @@ int corun_moe_create(const corun_moe_shape *shape, const void *router, const voi
   const size_t N1 = (size_t)NB * 2 * F, K2 = (size_t)NB * F;
   if (N1 > (size_t)1 << 30 || K2 > (size_t)1 << 30) return fail(CORUN_EINVAL);
   int rc;
-  if ((rc = moe_alloc(m, &m->router_pad, (size_t)GEMM_TILE_N * H)) || (rc = moe_alloc(m, &m->x_hi, (size_t)m->BN * H)) ||
+  if ((rc = moe_alloc(m, &m->x_hi, (size_t)m->BN * H)) ||
       (rc = moe_alloc(m, &m->x_lo, (size_t)m->BN * H)) || (rc = moe_alloc(m, &m->h_hi, (size_t)m->BN * K2)) ||
-      (rc = moe_alloc(m, &m->h_lo, (size_t)m->BN * K2)) || (rc = moe_alloc(m, &m->out_r, (size_t)m->BN * GEMM_TILE_N)) ||
+      (rc = moe_alloc(m, &m->h_lo, (size_t)m->BN * K2)) ||
       (rc = moe_alloc(m, &m->out_gu, (size_t)m->BN * N1)) || (rc = moe_alloc(m, &m->out_d, (size_t)m->BN * H)) ||
       (rc = moe_alloc(m, &m->ws, gemm_ws_floats(m->num_sms, m->BN))) || (rc = moe_alloc(m, &m->w, (size_t)B * NB)) ||
       (rc = moe_alloc(m, &m->d_status, 1)))
     return fail(rc);
-  if (cudaMemcpy(m->router_pad, router, (size_t)E * H * sizeof(bf16), cudaMemcpyDeviceToDevice) != cudaSuccess)
-    return fail(CORUN_ECUDA);
+  m->router = (const bf16 *)router;
   // the three GEMMs run one after the other and their results are consumed in between: one workspace serves all
   // from 65 to 128 rows the first GEMM applies the routing weight and the SwiGLU in its epilogue (where a tile
   // width divides the experts' width); else it stores gate / up sums and a kernel of its own follows (faster up to
   // 64 rows, where the masked store skips most of the output)
   const bool fused = m->BN > 64 && m->BN <= 128 && gemm_swiglu_blocks_half(F, NB, m->num_sms) > 0;
-  if ((rc = gemm_plan_create(&m->p_r, m->router_pad, GEMM_TILE_N, H, m->x_hi, m->x_lo, B, m->BN, m->out_r, m->ws, 8)) ||
-      (rc = fused ? gemm_plan_create_swiglu_blocks(&m->p_gu, gate_up, NB, F, H, m->x_hi, m->x_lo, B, m->BN, m->h_hi, m->h_lo, m->w, m->num_sms)
+  if ((rc = fused ? gemm_plan_create_swiglu_blocks(&m->p_gu, gate_up, NB, F, H, m->x_hi, m->x_lo, B, m->BN, m->h_hi, m->h_lo, m->w, m->num_sms)
                   : gemm_plan_create(&m->p_gu, gate_up, (int)N1, H, m->x_hi, m->x_lo, B, m->BN, m->out_gu, m->ws, m->num_sms)) ||
       (rc = gemm_plan_create(&m->p_d, down, H, (int)K2, m->h_hi, m->h_lo, B, m->BN, m->out_d, m->ws, m->num_sms)))
     return fail(rc);
@@ -415,7 +458,6 @@ int corun_moe_create(const corun_moe_shape *shape, const void *router, const voi
 void corun_moe_destroy(corun_moe *m) {
   if (!m) return;
   cudaStreamSynchronize(m->st);
-  gemm_plan_destroy(&m->p_r);
   gemm_plan_destroy(&m->p_gu);
   gemm_plan_destroy(&m->p_d);
   for (void *p : m->allocs) cudaFree(p);
@@ -428,8 +470,7 @@ int corun_moe_forward(corun_moe *m, const float *x, float *y, int32_t *experts, 
   const corun_moe_shape &s = m->sh;
   const int H = s.hidden, E = s.n_experts, F = s.expert_ffn, NB = E + s.n_shared;
   MCK(launch_split(x, m->B, H, m->x_hi, m->x_lo, m->st));
-  MCK(gemm_launch(m->p_r, nullptr, m->d_status, m->st, nullptr, true));
-  MCK(launch_moe_route(m->p_r.out(), m->B, E, s.n_shared, s.top_k, s.renormalize, m->w, experts, probs, m->st));
+  MCK(launch_moe_router(m->x_hi, m->x_lo, H, m->router, m->B, E, s.n_shared, s.top_k, s.renormalize, m->w, experts, probs, m->st));
   MCK(gemm_launch(m->p_gu, nullptr, m->d_status, m->st, nullptr, true));
   if (!m->p_gu.sw_hi) MCK(launch_moe_swiglu(m->p_gu.out(), m->w, m->B, F, NB, m->h_hi, m->h_lo, m->st));
   MCK(gemm_launch(m->p_d, nullptr, m->d_status, m->st, nullptr, true));
@@ -447,6 +488,6 @@ int corun_moe_sync(corun_moe *m) {
 
 int64_t corun_moe_weight_bytes(const corun_moe *m) { return m ? m->weight_bytes : 0; }
 
-int corun_moe_launches(const corun_moe *m) { return m ? (m->p_gu.sw_hi ? 6 : 7) : CORUN_EINVAL; }
+int corun_moe_launches(const corun_moe *m) { return m ? (m->p_gu.sw_hi ? 5 : 6) : CORUN_EINVAL; }
 
 }  // extern "C"

@@ -64,9 +64,9 @@ def test_mla_engine_parity_and_invariance(orc, first_dense, moe):
             trace.append([eng.logits(s).tobytes() for s in slots])
         assert worst <= TOL, worst
         # per layer: 10 around the attention (2 norms, 4 GEMMs, cache append, attention splits and combine, value split)
-        # + 3 (dense feed-forward) or 5 (router, routing, 2 GEMMs, masked SwiGLU: a kernel of its own up to 64 rows)
+        # + 3 (dense feed-forward) or 4 (router, 2 GEMMs, masked SwiGLU: a kernel of its own up to 64 rows)
         n_dense = first_dense if moe else sh.n_layers
-        assert eng.decode_launches() == 6 + 13 * n_dense + 15 * (sh.n_layers - n_dense) - (0 if moe else n_dense)
+        assert eng.decode_launches() == 6 + 13 * n_dense + 14 * (sh.n_layers - n_dense) - (0 if moe else n_dense)
 
         # the same requests in other slots, prefilled together in shared chunks: same bytes
         for s in slots:
