@@ -121,6 +121,33 @@ def test_mla_long_contexts_many_splits_and_repeatability():
     assert worst <= 2e-5, worst
 
 
+def test_mla_many_rows_and_few_items():
+    """More rows than one warp scans at once and more than there are CTAs (the stretches are cut inside and between
+    rows by accumulated cost), padding rows in between; and a call with fewer items than CTAs."""
+    torch = _torch()
+    nh, dc, dr = 4, 64, 8
+    rng0 = np.random.default_rng(5)
+    for B, hi in ((257, 600), (3, 40)):
+        ctxs = [int(c) for c in rng0.integers(0, hi, size=B)]
+        ctxs[0] = 0
+        ctxs[-1] = hi
+        rng, q_lat, q_rope, caches = _case(nh, dc, dr, ctxs, seed=B)
+        scale = 1.0 / math.sqrt(dc + dr)
+        pool, table = _paged(rng, caches, ctxs, dc + dr)
+        out = _run(torch, q_lat, q_rope, pool, table, ctxs, scale)
+        worst = 0.0
+        for b, n in enumerate(ctxs):
+            if n == 0:
+                assert not out[b].any()
+                continue
+            C = caches[b][:n, :dc].astype(np.float64)
+            Rk = caches[b][:n, dc:].astype(np.float64)
+            s = (C @ q_lat[b].astype(np.float64).T + Rk @ q_rope[b].astype(np.float64).T) * scale
+            p = np.exp(s - s.max(0)); p /= p.sum(0)
+            worst = max(worst, float(np.abs(out[b] - p.T @ C).max()))
+        assert worst <= 2e-5, (B, worst)
+
+
 def test_mla_context_beyond_the_block_table_is_cut():
     torch = _torch()
     nh, dc, dr, T = 8, 128, 32, 640
