@@ -188,14 +188,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 #define ATRACE(k, i) do { if (TRACED && trace && (k) < 64) trace[((size_t)blockIdx.x * 64 + (k)) * 8 + (i)] = globaltimer_ns(); } while (0)
   constexpr int KSTEPS = HD / 16;
   griddep_launch_dependents();
-  griddep_wait();                                // the item list and q come from earlier kernels
   constexpr int group = GROUP;                   // query heads per kv head
-  const int n_total = *n_work;
-  if (n_total <= 0) return;
-  // this CTA's stretch of the item list, and where the shared pool begins
-  const int n_pairs = WHOLE_PAIRS ? n_work[1] : 0;   // > 0: the ablation that hands out whole (row, kv head) pairs (see item_of)
-  const int n_fixed = n_pairs > 0 ? 0 : (int)(((long long)n_total * 7 / 8) / gridDim.x);
-  const int item_lo = (int)blockIdx.x * n_fixed, pool_lo = (int)gridDim.x * n_fixed;
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t kfull_bar[ATT_SLOTS], vfull_bar[ATT_SLOTS];
@@ -232,6 +225,21 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
+  // everything above touches nothing that another kernel writes: it runs while the kernels before this one drain
+  griddep_wait();                                // the item list, q and the newest cache rows come from earlier kernels
+  // (the inputs through after_wait: no load through them may be moved up across the wait)
+  q = after_wait(q); work = after_wait(work); n_work = after_wait(n_work);
+  rows.pos = after_wait(rows.pos); rows.active = after_wait(rows.active); rows.slot = after_wait(rows.slot);
+  kv.block_table = after_wait(kv.block_table);
+  const int n_total = *n_work;
+  if (n_total <= 0) {                            // the same in every thread of the CTA
+    if (warp == 0) tmem_dealloc(tmem_base, ATT_TMEM_COLS);
+    return;
+  }
+  // this CTA's stretch of the item list, and where the shared pool begins
+  const int n_pairs = WHOLE_PAIRS ? n_work[1] : 0;   // > 0: the ablation that hands out whole (row, kv head) pairs (see item_of)
+  const int n_fixed = n_pairs > 0 ? 0 : (int)(((long long)n_total * 7 / 8) / gridDim.x);
+  const int item_lo = (int)blockIdx.x * n_fixed, pool_lo = (int)gridDim.x * n_fixed;
   bool failed = false;
   // instruction descriptor: D fp32 (bits 4-5 = 1), A and B fp16 (0), K-major, N = 16 (N >> 3 at bit 17),
   // M = 128 (M >> 4 at bit 24)

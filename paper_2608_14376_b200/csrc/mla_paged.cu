@@ -120,7 +120,21 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   if (warp == 0) {
     tmem_alloc(smem_u32(&tmem_base_s), MP_TMEM_COLS);
     tmem_relinquish();
-  } else if (warp == 2) {
+  } else if (warp >= 4) {
+    // the operand tiles start out as zeros: rows of absent heads and rope columns beyond d_r stay zero
+    uint4 *z = reinterpret_cast<uint4 *>(base_ptr + MP_OFF_Q);
+    for (int i = tid - 128; i < (10 * MP_QBLK + 2 * MP_PBUF) / 16; i += MP_THREADS - 128) z[i] = make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  // (programmatic launch) everything above reads nothing that another kernel writes: it runs while the kernels before
+  // this one drain.  The inputs are taken through after_wait so that no load is moved up across the wait.
+  griddep_wait();
+  q_lat = after_wait(q_lat); q_rope = after_wait(q_rope); block_table = after_wait(block_table); ctx = after_wait(ctx);
+  row_slot = after_wait(row_slot); row_pos = after_wait(row_pos); row_active = after_wait(row_active);
+  if (warp == 2) {
     // items per row -> first item of every row (one warp, rows in chunks of 32, ascending)
     int run = 0, crun = 0;
     for (int r0 = 0; r0 < B; r0 += 32) {
@@ -166,18 +180,8 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
       my_items[0] = bound((int)blockIdx.x);
       my_items[1] = bound((int)blockIdx.x + 1);
     }
-  } else if (warp >= 4) {
-    // the operand tiles start out as zeros: rows of absent heads and rope columns beyond d_r stay zero
-    uint4 *z = reinterpret_cast<uint4 *>(base_ptr + MP_OFF_Q);
-    for (int i = tid - 128; i < (10 * MP_QBLK + 2 * MP_PBUF) / 16; i += MP_THREADS - 128) z[i] = make_uint4(0u, 0u, 0u, 0u);
-    fence_proxy_async();
   }
-  tc_fence_before();
   __syncthreads();
-  tc_fence_after();
-  // (programmatic launch) everything above reads nothing the kernels just before this one write: the row lengths
-  // and slots are set at the start of the step; the queries and the newest cache rows are read from here on
-  griddep_wait();
   const uint32_t tmem_base = tmem_base_s;
   const uint32_t s_tmem = tmem_base, o_tmem = tmem_base + 256;
   const int n_items = row_start[B];
@@ -507,9 +511,9 @@ __global__ void __launch_bounds__(128) mla_paged_combine_kernel(const float2 *__
   __shared__ float2 sml[128];                       // the splits' (max, sum) pairs, fetched in one round trip
   const int r = (int)blockIdx.x / n_heads, h = (int)blockIdx.x - r * n_heads;
   const int d = 4 * (int)threadIdx.x;
+  griddep_wait();                                   // before the first read of anything another kernel of the step wrote
   int c = row_pos ? (row_active[r] ? row_pos[r] + 1 : 0) : ctx[r];
   if (c <= 0) return;                               // a padding row is left alone (the whole block returns)
-  griddep_wait();
   c = c > max_blocks * MP_PAGE ? max_blocks * MP_PAGE : c;
   int ns = (c + MP_T - 1) / MP_T;
   if (ns > max_splits) ns = max_splits;

@@ -23,6 +23,15 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
 // kernel that was launched without the programmatic attribute.
 __device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// A pointer the compiler knows nothing about any more.  Loads through `const __restrict__` pointers count as
+// invariant and may be moved up across griddepcontrol.wait (even to the kernel's first instruction), where the
+// producing kernel may not have finished: a kernel that does work ahead of its wait takes its input pointers
+// through this after the wait.
+template <typename T>
+__device__ __forceinline__ T *after_wait(T *p) {
+  asm volatile("" : "+l"(p));
+  return p;
+}
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
