@@ -627,12 +627,16 @@ def run_corun_mla(args, rank, world):
         torch.cuda.synchronize()
         mms = e0.elapsed_time(e1) / n_rep
         wb = ops[0][0].weight_bytes()
-        roofline = {"kernel": "expert block of one layer (router GEMM, routing, gate / up GEMM over all experts, masked SwiGLU, down GEMM): "
+        mtraffic = None                                   # ncu DRAM bytes of one call of the block (profiles/)
+        mtp = os.path.join(ROOT, "profiles", "moe_block_dram_traffic.json")
+        if os.path.exists(mtp):
+            mtraffic = json.load(open(mtp)).get("dram_bytes_per_call")
+        roofline = {"kernel": "expert block of one layer (router, gate / up GEMM over all experts with routing weight and SwiGLU in its epilogue, down GEMM): "
                               "%d of a step's %d layers" % (sh.n_layers - mla_cfg["first_dense"], sh.n_layers),
                     "bound": "hbm", "achieved": wb / (mms * 1e-3) / 1e9, "peak": hbm, "unit": "GB/s",
                     "peak_source": which + " (MEASURED_PEAKS.json hbm_gbs)" if which == "measured" else "fallback 6650",
-                    "traffic": None, "bytes_per_launch_avg": wb, "ms_per_launch_avg": mms,
-                    "scope": "one call of the block = 5 kernels; the whole step against its roofline is in step_roofline",
+                    "traffic": mtraffic, "bytes_per_launch_avg": wb, "ms_per_launch_avg": mms,
+                    "scope": "one call of the block (split, router, two GEMMs, read-out); the whole step against its roofline is in step_roofline",
                     "timing": "CUDA events over %d back-to-back calls rotating over %d weight sets (%.0f MB each)" % (n_rep, copies, wb / 1e6)}
         roofline["frac"] = roofline["achieved"] / hbm
         for op, *_ in ops:
