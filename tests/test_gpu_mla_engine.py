@@ -103,6 +103,43 @@ def test_mla_engine_parity_and_invariance(orc, first_dense, moe):
         eng.close()
 
 
+def test_mla_engine_with_more_than_64_slots(orc):
+    """The decode program above 64 padded rows: the grouped up-projections then run on two blocks of rows per head and
+    the expert layers' first GEMM applies the routing weight and the SwiGLU itself.  Parity with the oracle and the
+    same bytes in other slots (rows of both blocks)."""
+    sh, Bw = SMALL, 80
+    model, eng = _setup(orc, sh, dict(SMALL_MLA), SMALL_MOE, seed=6, B=Bw, max_ctx=128)
+    try:
+        assert eng.decode_launches() == 6 + 13 + 13 * (sh.n_layers - 1)
+        prompts = synth.make_prompts(sh.vocab, [30, 77, 12, 50], seed=6)
+        seeds = np.zeros(Bw, np.uint64)
+        traces = []
+        for slots in ([3, 70, 79, 64], [65, 0, 41, 63]):
+            reqs = [orc.Request(model, p, 1, max_T=128) for p in prompts]
+            worst = 0.0
+            for s, p, r in zip(slots, prompts, reqs):
+                r.prefill()
+                eng.prefill(s, p, len(p) + 8)
+            active = np.zeros(Bw, np.uint8); active[slots] = 1
+            trace = []
+            for _ in range(3):
+                toks = [int(np.argmax(r.logits)) for r in reqs]
+                for s, t in zip(slots, toks):
+                    eng.force_token(s, t)
+                eng.decode_step(active, seeds)
+                for s, r, t in zip(slots, reqs, toks):
+                    r.decode(force_token=t)
+                    worst = max(worst, float(np.abs(eng.logits(s) - r.logits).max()))
+                trace.append([eng.logits(s).tobytes() for s in slots])
+            assert worst <= TOL, worst
+            traces.append(trace)
+            for s in slots:
+                eng.release(s)
+        assert traces[0] == traces[1]
+    finally:
+        eng.close()
+
+
 def test_mla_engine_served_together_equals_served_alone(orc):
     """The paper's validation protocol on the MLA decoder: requests served together (sampled, through the host
     scheduler with a pool too small for all of them, isolated and batched prefill) produce, bit for bit, the tokens
