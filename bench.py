@@ -412,24 +412,27 @@ def run_corun(args, rank, world):
         from paper_2608_14376_b200.corun import MlaAttention
         gl = torch.Generator(device="cuda").manual_seed(4)
         lB, lh, ldc, ldr = 128, 16, 512, 64
-        lpool, ltable, ldctx = synth.mla_paged_case(lB, ldc + ldr, 512, 4096, seed=2)
+        # three caches of the same shape, taken in turn: none of a call's 349 MB is left in L2 from the call before
+        lcases = [synth.mla_paged_case(lB, ldc + ldr, 512, 4096, seed=2) for _ in range(3)]
+        lpool, ltable, ldctx = lcases[0]
         lctx = ldctx.cpu().numpy()
         lq, lr = torch.randn((lB, lh, ldc), generator=gl, device="cuda"), torch.randn((lB, lh, ldr), generator=gl, device="cuda")
         lbytes = int(lctx.astype(np.int64).sum()) * (ldc + ldr) * 2
         lop = MlaAttention(lB, lh, ldc, ldr, ltable.shape[1])
-        for _ in range(3):
-            lop.run(lq, lr, lpool, ltable, ldctx, 1.0 / math.sqrt(128 + ldr))
+        for i in range(3):
+            lop.run(lq, lr, lcases[i][0], lcases[i][1], ldctx, 1.0 / math.sqrt(128 + ldr))
         lop.sync()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for _ in range(100):
-            lop.run(lq, lr, lpool, ltable, ldctx, 1.0 / math.sqrt(128 + ldr))
+        for i in range(99):
+            lop.run(lq, lr, lcases[i % 3][0], lcases[i % 3][1], ldctx, 1.0 / math.sqrt(128 + ldr))
         e1.record()
         lop.sync()
-        lms = e0.elapsed_time(e1) / 100
+        lms = e0.elapsed_time(e1) / 99
         mla = {"workload": "deepseek_v2_lite_mla_b128", "contexts": f"uniform {lctx.min()}..{lctx.max()}", "cache": "paged, 16 tokens per page",
                "cache_bytes": lbytes, "us_per_call": lms * 1e3, "GBs": lbytes / lms / 1e6, "frac_of_measured_hbm": lbytes / lms / 1e6 / hbm,
-               "operands": "fp16 hi + lo pairs (tcgen05)"}
+               "operands": "fp16 hi + lo pairs (tcgen05)", "timing": "99 calls rotating over three caches of 349 MB"}
+        del lcases
         del lpool, lq, lr, lop
 
     cpu = None
@@ -576,6 +579,21 @@ def run_corun_mla(args, rank, world):
                  "note": "all %d experts of a layer are streamed every step (no expert groups: the padding that keeps a row's "
                          "result independent of its co-tenants); flops count every row through every expert" % nb}
     launches = eng.decode_launches()
+    # ---- per-kernel durations (isolated launches rotating over the layers' weights, CUDA events)
+    kinds = dict({n: i for i, n in enumerate(eng.KERNEL_KINDS)}, **eng.MLA_KERNEL_KINDS, **eng.MOE_KERNEL_KINDS)
+    kernels = {}
+    for name, kind in kinds.items():
+        v = eng.time_kernel(kind, 10 if name in ("gemm_lm_head", "sampler") else 52)
+        kernels[name] = {"ms_per_launch": v} if v > 5e-4 else {"ms_per_launch": 0.0, "note": "no such launch: fused into a neighbour"}
+    L, nd = sh.n_layers, mla_cfg["first_dense"]
+    kernels["per_step_ms"] = {
+        "gemms": L * (kernels["gemm_qkv"]["ms_per_launch"] + kernels["gemm_o"]["ms_per_launch"] + kernels["mla_up_k"]["ms_per_launch"]
+                      + kernels["mla_up_v"]["ms_per_launch"]) + (L - nd) * (kernels["gemm_gate_up"]["ms_per_launch"]
+                      + kernels["gemm_down"]["ms_per_launch"]) + kernels["gemm_lm_head"]["ms_per_launch"],
+        "attention": L * kernels["attention"]["ms_per_launch"],
+        "token_wise": L * (2 * kernels["resid_norm"]["ms_per_launch"] + kernels["rope_kv_append"]["ms_per_launch"])
+                      + (L - nd) * kernels["moe_router"]["ms_per_launch"] + kernels["sampler"]["ms_per_launch"],
+        "note": "expert layers only for gate / up, down and router (the one dense layer is left out); launched alone, back to back"}
     # ---- isolated prefill of one request (its slot freed first): wall time of corun_prefill with the prompt in host
     # memory.  A prefill row attends to its request's latent cache up to its own position with the decode kernel,
     # so the attention part grows with the square of the prompt length.
@@ -663,7 +681,7 @@ def run_corun_mla(args, rank, world):
         "clocks": clk, "gpu_launches": launches * K,
         "e2e": {"value": e2e_val, "unit": "tok/s", "ms_per_step": 1e3 * e2e_s / K,
                 "h2d_bytes_per_step": B * 9, "d2h_bytes_per_step": B * 4 + 4},
-        "sustained": sustained, "roofline": roofline, "step_roofline": step_roof, "prefill": prefill,
+        "sustained": sustained, "roofline": roofline, "step_roofline": step_roof, "kernels": kernels, "prefill": prefill,
         "cpu_baseline": {"value": None, "unit": "tok/s", "kind": "oracle", "cores": 0,
                          "sample": "absent: the oracle of this decoder needs its 31 GB of weights as host arrays and, in its definition "
                                    "form, decompresses every cached token for every query (about 0.1 TFLOP of scalar fp64 per decode "

@@ -40,7 +40,11 @@ int corun_debug_kv_fill(corun_engine *e, int32_t slot, int32_t n_ctx, float std,
  * cannot hold them), after a short warm-up; *avg_ms = mean duration of one launch.
  * kind: 0 QKV GEMM, 1 O GEMM, 2 gate-up GEMM, 3 down GEMM, 4 LM-head GEMM (+ partial
  * fix-up), 5 attention (split + combine), 6 residual + RMSNorm, 7 RoPE + KV append,
- * 8 SwiGLU, 9 sampler.  Uses the rows of the last decode step; overwrites
+ * 8 SwiGLU (none where the gate / up GEMM applies it), 9 sampler; engines with multi-head latent attention:
+ * 5 = the latent attention (splits + combine), 7 = latent RMSNorm + rotary key + cache append + query parts,
+ * 10 = grouped key up-projection, 11 = grouped value up-projection + split; engines with expert layers:
+ * 2, 3, 6, 8 on the expert layers, 12 = router.  EINVAL for a kind the engine does not have.
+ * Uses the rows of the last decode step; overwrites
  * intermediate buffers (not the cache beyond each active slot's next position). */
 int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *avg_ms);
 /* Copies the first n floats of an intermediate buffer of the decode program to the host, as left by

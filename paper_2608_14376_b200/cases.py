@@ -208,20 +208,22 @@ def case_mla(a):
     from . import corun, synth
 
     nh, dc, dr = 16, 512, 64
-    pool, table, dctx = synth.mla_paged_case(a.B, dc + dr, a.ctx_lo, a.ctx_hi, seed=2)
+    # caches of the same shape taken in turn (--caches 1: the same cache every call, partly served from L2)
+    cs = [synth.mla_paged_case(a.B, dc + dr, a.ctx_lo, a.ctx_hi, seed=2) for _ in range(a.caches)]
+    pool, table, dctx = cs[0]
     ctx = dctx.cpu().numpy()
     g = torch.Generator(device="cuda").manual_seed(0)
     q_lat = torch.randn((a.B, nh, dc), generator=g, device="cuda")
     q_rope = torch.randn((a.B, nh, dr), generator=g, device="cuda")
     scale = 1.0 / math.sqrt(128 + dr)
     op = corun.MlaAttention(a.B, nh, dc, dr, table.shape[1])
-    for _ in range(3):
-        out = op.run(q_lat, q_rope, pool, table, dctx, scale)
+    for i in range(3):
+        out = op.run(q_lat, q_rope, cs[i % a.caches][0], cs[i % a.caches][1], dctx, scale)
     op.sync()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
-    for _ in range(a.reps):
-        out = op.run(q_lat, q_rope, pool, table, dctx, scale)
+    for i in range(a.reps):
+        out = op.run(q_lat, q_rope, cs[i % a.caches][0], cs[i % a.caches][1], dctx, scale)
     t1.record()
     op.sync()
     ms = t0.elapsed_time(t1) / a.reps
@@ -542,6 +544,7 @@ def main():
     mb.add_argument("--vocab", type=int, default=151936)
     mb.add_argument("--reps", type=int, default=50)
     ma = sub.add_parser("mla")
+    ma.add_argument("--caches", type=int, default=3, help="distinct caches taken in turn")
     ma.add_argument("--B", type=int, default=128); ma.add_argument("--ctx-lo", type=int, default=512)
     ma.add_argument("--ctx-hi", type=int, default=4096); ma.add_argument("--reps", type=int, default=10)
     ab = sub.add_parser("ablation")

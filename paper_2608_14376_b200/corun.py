@@ -357,6 +357,9 @@ class Engine:
 
     KERNEL_KINDS = ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head", "attention",
                     "resid_norm", "rope_kv_append", "swiglu", "sampler")
+    # further kinds of corun_debug_time_kernel: engines with multi-head latent attention / with expert layers
+    MLA_KERNEL_KINDS = {"mla_up_k": 10, "mla_up_v": 11}
+    MOE_KERNEL_KINDS = {"moe_router": 12}
 
     def time_kernel(self, kind: int, reps: int) -> float:
         ms = C.c_float(0.0)

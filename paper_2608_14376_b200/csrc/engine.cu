@@ -1182,7 +1182,9 @@ int corun_debug_kv_fill(corun_engine *e, int32_t slot, int32_t n_ctx, float std,
 }
 
 int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *avg_ms) {
-  if (!e || !avg_ms || reps < 1 || kind < 0 || kind > 9 || e->mla) return CORUN_EINVAL;
+  if (!e || !avg_ms || reps < 1 || kind < 0 || kind > 12) return CORUN_EINVAL;
+  if ((kind == 10 || kind == 11) && !e->mla) return CORUN_EINVAL;   // the up-projections of an MLA layer
+  if (kind == 12 && !e->moe_E) return CORUN_EINVAL;                  // the router of an expert layer
   RC(sync_stream(e));
   Program &P = e->dec;
   const corun_shape &s = e->sh;
@@ -1196,8 +1198,13 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
     const int n = pass == 0 ? (reps < 3 ? reps : 3) : reps;
     cudaError_t ce = cudaEventRecord(a, e->st);
     for (int i = 0; i < n && ce == cudaSuccess; ++i) {
-      const int l = i % s.n_layers;   // rotate over the layers so that L2 cannot hold the weights
-      GemmOut prev = ffn_out(e, P, 0);
+      int l = i % s.n_layers;         // rotate over the layers so that L2 cannot hold the weights
+      // feed-forward kinds of a decoder with dense and expert layers: the expert layers
+      if (e->mla && e->moe_E && (kind == 2 || kind == 3 || kind == 6 || kind == 8 || kind == 12))
+        l = e->first_dense + i % (s.n_layers - e->first_dense);
+      GemmOut prev = ffn_out(e, P, l);
+      const MlaCache mcache{e->mla ? e->kv_pool + (size_t)l * e->layer_stride : nullptr, e->d_block_table, e->max_blocks, e->B,
+                            (long long)e->pool_blocks};
       switch (kind) {
         // launched as in the step's graph: with programmatic stream serialization
         case 0: ce = gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, nullptr, true); break;
@@ -1207,7 +1214,14 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
         case 4: ce = gemm_launch(P.p_lm, nullptr, e->d_status, e->st, nullptr, true);
                 if (ce == cudaSuccess) ce = gemm_fixup_launch(P.p_lm, e->st);
                 break;
-        case 5: ce = cudaMemsetAsync(P.att_pool + l, 0, sizeof(int), e->st);   // the launch does not reset its pool counter
+        case 5: if (e->mla) {
+                  ce = launch_mla_attention(e->tm_c[l], e->tm_cv[l], P.q_lat, e->md.rank, (long long)P.RPH * e->md.rank, P.q_rope,
+                                            e->d_block_table, e->max_blocks, nullptr, &rows, P.R, e->md,
+                                            1.0f / sqrtf((float)(e->md.nope + e->md.rope)), e->mla_splits, P.mla_ml, P.mla_po, nullptr,
+                                            P.ol_hi, P.ol_lo, P.RPH, e->num_sms, e->d_status, true, e->st);
+                  break;
+                }
+                ce = cudaMemsetAsync(P.att_pool + l, 0, sizeof(int), e->st);   // the launch does not reset its pool counter
                 if (ce == cudaSuccess)
                   ce = launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work,
                                         P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_pool + l,
@@ -1215,7 +1229,12 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
                 break;
         case 6: ce = launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->attn_norm[l], s.rms_eps, P.xn_hi,
                                        P.xn_lo, e->st); break;
-        case 7: ce = launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->d_status, e->st); break;
+        case 7: if (e->mla) {   // (re-appends the rows' current positions: the same values)
+                  ce = launch_mla_post(P.p_qkv.out(), rows, e->d_rope, e->md, e->kv_norm[l], s.rms_eps, mcache, P.RPH, P.qn_hi, P.qn_lo,
+                                       P.q_rope, e->d_status, e->st);
+                  break;
+                }
+                ce = launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->d_status, e->st); break;
         case 8: if (P.p_gu.sw_hi) break;             // no such kernel: the SwiGLU is in the GEMM's epilogue
                 ce = e->moe_E ? launch_moe_swiglu(P.p_gu.out(), P.moe_w, P.R, e->moe_F, e->moe_E + e->moe_S, P.ff_hi, P.ff_lo, e->st)
                               : launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st);
@@ -1225,6 +1244,13 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
           ce = launch_sampler(sa, P.R, e->st);
           break;
         }
+        case 10: ce = gemm_launch(P.p_uk, &e->tm_uk[l], e->d_status, e->st, nullptr, true); break;
+        case 11: ce = gemm_launch(P.p_uv, &e->tm_uv[l], e->d_status, e->st, nullptr, true);
+                 if (ce == cudaSuccess) ce = launch_mla_ao_split(P.uv_out, P.R, P.RPH, e->md, P.ao_hi, P.ao_lo, e->st);
+                 break;
+        case 12: ce = launch_moe_router(P.xn_hi, P.xn_lo, s.hidden, e->router[l], P.R, e->moe_E, e->moe_S, e->moe_K, e->moe_renorm,
+                                        P.moe_w, nullptr, nullptr, e->st);
+                 break;
       }
     }
     if (ce == cudaSuccess) ce = cudaEventRecord(b, e->st);
