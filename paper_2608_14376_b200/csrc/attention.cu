@@ -161,14 +161,15 @@ __device__ __forceinline__ void attn_combine_pair(int r, int j, int nsplit, int 
 template <int HD>
 struct AttLayout {
   static constexpr int NHALF = HD / 64;                          // 64-dim halves of a key row
-  static constexpr int K_BYTES = NHALF * ATT_PAGES * KBOX_BYTES; // keys of an item: [half][page][16 x 128 B]
+  static constexpr int PAGE_BYTES = NHALF * KBOX_BYTES;          // a page's keys: [8-token group][half][8 x 128 B]
+  static constexpr int K_BYTES = ATT_PAGES * PAGE_BYTES;         // keys of an item: [page][group][half][8 x 128 B]
   static constexpr int V_BYTES = K_BYTES;                        // values of an item: the same arrangement
   static constexpr int ITEM_BYTES = K_BYTES + V_BYTES;
   static constexpr int Q_BYTES = NHALF * OPND_BYTES;             // [half][16 x 128 B]
   static constexpr int P_BYTES = 2 * OPND_BYTES;                 // 128 tokens = 2 halves of 64
   static constexpr int GROUP_BYTES = Q_BYTES + P_BYTES;
-  // the value MMA always covers 128 dims (M = 128), i.e. two blocks of 64 dims one key-tile half apart: with
-  // hd = 64 the second one lies in whatever follows the value tile (never used; it must only be readable)
+  // the value MMA always covers 128 dims (M = 128), i.e. two blocks of 64 dims 1 KiB apart: with hd = 64 the
+  // second one is the page's second token group (results never used); the pad keeps every read inside the buffer
   static constexpr int PAD_BYTES = (HD < 128) ? ATT_PAGES * KBOX_BYTES + KBOX_BYTES : 0;
   static constexpr size_t SMEM = (size_t)ATT_NBUF * ITEM_BYTES + ATT_GROUPS * GROUP_BYTES + PAD_BYTES + 1024;
 };
@@ -337,20 +338,15 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       }
       __syncwarp();
       if (lane < n_pages) {
-        // this layer's pages as rows of hd halfs: the key tile of (page, head) starts at row
-        //   page * 2 * n_kv * 16 + head * 16, its value tile n_kv * 16 rows further on
+        // this layer's pages as groups of eight rows of hd halfs: the key tile of (page, head) is the two groups from
+        //   2 * (page * 2 * n_kv + head), its value tile 2 * n_kv groups further on.  ONE box per tile (the TMA unit
+        //   is bound by the number of boxes: 99 cycles for a 2 KB box): [2 groups][halves of 64 dims][8 tokens][64 dims]
         if (is_v) {
-          const int row_v = (page * 2 * kv.n_kv + kv.n_kv + g) * KV_BLOCK;
-          const uint32_t vb = vring + (uint32_t)buf * L::V_BYTES;
-#pragma unroll
-          for (int x = 0; x < L::NHALF; ++x)
-            tma_load_2d(vb + (uint32_t)(x * ATT_PAGES + lane) * KBOX_BYTES, &tmV, x * 64, row_v, fb, pol);
+          const int grp_v = 2 * (page * 2 * kv.n_kv + kv.n_kv + g);
+          tma_load_4d(vring + (uint32_t)buf * L::V_BYTES + (uint32_t)lane * L::PAGE_BYTES, &tmV, 0, 0, 0, grp_v, fb, pol);
         } else {
-          const int row_k = (page * 2 * kv.n_kv + g) * KV_BLOCK;
-          const uint32_t kb = ring + (uint32_t)buf * L::K_BYTES;
-#pragma unroll
-          for (int x = 0; x < L::NHALF; ++x)
-            tma_load_2d(kb + (uint32_t)(x * ATT_PAGES + lane) * KBOX_BYTES, &tmK, x * 64, row_k, fb, pol);
+          const int grp_k = 2 * (page * 2 * kv.n_kv + g);
+          tma_load_4d(ring + (uint32_t)buf * L::K_BYTES + (uint32_t)lane * L::PAGE_BYTES, &tmK, 0, 0, 0, grp_k, fb, pol);
         }
       }
     }
@@ -433,7 +429,8 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 #pragma unroll
           for (int ks = 0; ks < KSTEPS; ++ks) {
             const uint64_t adv = (uint64_t)((ks & 3) * 2);      // 16 dims = 32 bytes inside the swizzled row
-            const uint64_t a = umma_desc_sw128(k_tiles + (uint32_t)(ks >> 2) * (ATT_PAGES * KBOX_BYTES)) + adv;
+            // the half's 8-token groups lie NHALF KiB apart (the halves of a group are neighbours)
+            const uint64_t a = umma_desc_sw128_sbo(k_tiles + (uint32_t)(ks >> 2) * 1024u, (uint32_t)L::NHALF * 1024u) + adv;
             const uint64_t b = umma_desc_sw128(q_tile + (uint32_t)(ks >> 2) * OPND_BYTES) + adv;
             umma_bf16(s_tmem, a, b, idesc, ks > 0 ? 1u : 0u);   // operand format (fp16) is in idesc
           }
@@ -502,8 +499,8 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         tc_fence_after();
         for (int p = 0; ok && p < n_pages; ++p) {
           // A = V^T of the page: [128 dims x 16 tokens] read MN-major from the token-major tile (two blocks of
-          // 64 dims a key-tile half apart, two groups of 8 tokens 1 KiB apart)
-          const uint64_t a = umma_desc_sw128_mn(v_tiles + (uint32_t)p * KBOX_BYTES, ATT_PAGES * KBOX_BYTES, 1024u);
+          // 64 dims 1 KiB apart, two groups of 8 tokens NHALF KiB apart)
+          const uint64_t a = umma_desc_sw128_mn(v_tiles + (uint32_t)p * L::PAGE_BYTES, 1024u, (uint32_t)L::NHALF * 1024u);
           const uint64_t b = umma_desc_sw128(p_tile + (uint32_t)(p >> 2) * OPND_BYTES) + (uint64_t)((p & 3) * 2);
           umma_bf16(o_tmem, a, b, idesc | (1u << 15), p > 0 ? 1u : 0u);
         }

@@ -86,6 +86,7 @@ struct corun_engine {
   std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_down;
   std::vector<CUtensorMap> tm_gu_half;     // dense gate / up matrices with the box of the GEMM with SwiGLU in its epilogue
   std::vector<CUtensorMap> tm_k, tm_v;   // per layer: the pages as rows of head_dim halfs (keys and values alike)
+  std::vector<CUtensorMap> tm_k4;        // the same memory as [8-token group][64-dim half][8 tokens][64 dims]: one box per (page, head) tile
   // Mixture-of-Experts feed-forward layers (E = 0: dense).  sh.ffn is then (E + S) * F.
   int moe_E = 0, moe_K = 0, moe_F = 0, moe_S = 0, moe_renorm = 0;
   std::vector<const bf16 *> router;      // per layer: [E, H], borrowed
@@ -360,7 +361,8 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
       n += 3 + (&P == &e->dec ? 0 : 1);               // beyond the count below: two grouped GEMMs, the split, and in prefill too a second attention kernel
     } else {
     STAGE(launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->d_status, e->st));
-    STAGE(launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work, P.att_n_work,
+    // (the decode kernel takes the one-box-per-tile view of the pages, the prefill kernel the row view)
+    STAGE(launch_attention(&P == &e->dec ? e->tm_k4[l] : e->tm_k[l], &P == &e->dec ? e->tm_k4[l] : e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work, P.att_n_work,
                            e->num_sms, P.part_acc, P.part_ml, P.att_pool + l, P.ao_hi, P.ao_lo, &P == &e->dec ? (e->whole_pairs ? 2 : 0) : 1,
                            e->d_status, e->st));
     }
@@ -697,6 +699,13 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
       const __half *base = e->kv_pool + (size_t)l * e->layer_stride;
       if ((rc = tma_encode_2d(&e->tm_k[l], base, 1, halfs / s.head_dim, s.head_dim, KV_BLOCK, 64))) return fail(rc);
       e->tm_v[l] = e->tm_k[l];   // keys and values are cached alike: the same view serves both
+      // decode attention: a tile's 16 tokens x head_dim in ONE box, [2 groups of 8 tokens][halves of 64 dims][8][64]
+      const unsigned long long row_b = (unsigned long long)s.head_dim * 2;
+      const unsigned long long d4[4] = {64, 8, (unsigned long long)(s.head_dim / 64), halfs / s.head_dim / 8};
+      const unsigned long long s4[3] = {row_b, 128, 8 * row_b};
+      const unsigned b4[4] = {64, 8, (unsigned)(s.head_dim / 64), 2};
+      e->tm_k4.emplace_back();
+      if ((rc = tma_encode_fp16_4d(&e->tm_k4[l], base, d4, s4, b4))) return fail(rc);
     }
     if (attention_prepare() != cudaSuccess) return fail(CORUN_ECUDA);
   }
@@ -1223,7 +1232,7 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
                 }
                 ce = cudaMemsetAsync(P.att_pool + l, 0, sizeof(int), e->st);   // the launch does not reset its pool counter
                 if (ce == cudaSuccess)
-                  ce = launch_attention(e->tm_k[l], e->tm_v[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work,
+                  ce = launch_attention(e->tm_k4[l], e->tm_k4[l], P.q, rows, s.n_q_heads, kv, l, e->max_splits, P.att_work,
                                         P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_pool + l,
                                         P.ao_hi, P.ao_lo, e->whole_pairs ? 2 : 0, e->d_status, e->st);
                 break;
@@ -1300,7 +1309,7 @@ int corun_debug_attn_trace(corun_engine *e, int32_t layer, uint64_t *stamps, int
   for (int i = 0; i < 2 && ce == cudaSuccess; ++i) {
     ce = cudaMemsetAsync(P.att_pool + layer, 0, sizeof(int), e->st);   // the launch does not reset its pool counter
     if (ce == cudaSuccess)
-      ce = launch_attention(e->tm_k[layer], e->tm_v[layer], P.q, rows, s.n_q_heads, kv_layout(e), layer, e->max_splits,
+      ce = launch_attention(e->tm_k4[layer], e->tm_k4[layer], P.q, rows, s.n_q_heads, kv_layout(e), layer, e->max_splits,
                             P.att_work, P.att_n_work, e->num_sms, P.part_acc, P.part_ml, P.att_pool + layer,
                             P.ao_hi, P.ao_lo, e->whole_pairs ? 2 : 0, e->d_status, e->st, i == 1 ? d : nullptr);   // only the second launch is recorded
   }

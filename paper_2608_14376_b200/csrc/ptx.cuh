@@ -170,6 +170,18 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
   return d;
 }
 
+// The same with the groups of eight rows `group_bytes` apart (tiles whose 1 KiB atoms are interleaved with those
+// of other column blocks).
+__device__ __forceinline__ uint64_t umma_desc_sw128_sbo(uint32_t smem_addr, uint32_t group_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
+  d |= (uint64_t)1u << 16;                 // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)((group_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1u << 46;                 // version
+  d |= (uint64_t)2u << 61;                 // SWIZZLE_128B
+  return d;
+}
+
 // Descriptor of an MN-major operand (the M or N index runs along the 128-byte rows, K across rows) stored with
 // the 128-byte swizzle: every 128-byte row holds 64 consecutive M (N) elements of one K index, eight consecutive
 // K rows form a 1 KiB swizzle atom.  mn_block_bytes: distance between the tiles of consecutive blocks of 64 M (N)
