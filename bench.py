@@ -571,16 +571,22 @@ def run_corun_mla(args, rank, world):
     w_bytes = synth.mla_weight_bytes_per_step(sh, mla_cfg, moe_cfg)
     kv_bytes_mid = sum((int(c) + W + K // 2) * row_bytes * sh.n_layers for c in ctx)
     nb = moe_cfg["n_experts"] + moe_cfg["n_shared"]
-    flops = 2 * B * (w_bytes // 2) + 2 * sh.n_q_heads * (2 * mla_cfg["kv_lora_rank"] + mla_cfg["qk_rope"]) * sh.n_layers * sum(int(c) for c in ctx)
+    # a row's own experts only (top-k + shared): the grouped form of the expert layers multiplies nothing else
+    idle_params = (sh.n_layers - mla_cfg["first_dense"]) * (moe_cfg["n_experts"] - moe_cfg["top_k"]) * 3 * sh.hidden * moe_cfg["expert_ffn"]
+    flops = 2 * B * (w_bytes // 2 - idle_params) + 2 * sh.n_q_heads * (2 * mla_cfg["kv_lora_rank"] + mla_cfg["qk_rope"]) * sh.n_layers * sum(int(c) for c in ctx)
     t_roof_ms = max((w_bytes + kv_bytes_mid) / (hbm * 1e9), flops / (tf * 1e12)) * 1e3
     step_roof = {"bytes": w_bytes + kv_bytes_mid, "weight_bytes": w_bytes, "cache_bytes": kv_bytes_mid, "flops": flops,
                  "t_roofline_ms": t_roof_ms, "frac_of_" + which: t_roof_ms / ms_per_step,
                  "frac_of_nominal_8TBs": max((w_bytes + kv_bytes_mid) / 8e12, flops / 2.25e15) * 1e3 / ms_per_step,
-                 "note": "all %d experts of a layer are streamed every step (no expert groups: the padding that keeps a row's "
-                         "result independent of its co-tenants); flops count every row through every expert" % nb}
+                 "note": "all %d experts of a layer are streamed every step (with 128 rows every expert has rows); an expert's rows "
+                         "are gathered into blocks of 64 (a row's result does not depend on what else is in its block); flops count "
+                         "a row's own experts" % nb}
     launches = eng.decode_launches()
     # ---- per-kernel durations (isolated launches rotating over the layers' weights, CUDA events)
     kinds = dict({n: i for i, n in enumerate(eng.KERNEL_KINDS)}, **eng.MLA_KERNEL_KINDS, **eng.MOE_KERNEL_KINDS)
+    grouped = B > 64 and not os.environ.get("CORUN_MOE_DECODE_DENSE")   # the decode program's form of the expert layers
+    if grouped:
+        kinds.update(eng.MOE_GROUPED_KERNEL_KINDS)
     kernels = {}
     for name, kind in kinds.items():
         v = eng.time_kernel(kind, 10 if name in ("gemm_lm_head", "sampler") else 52)
@@ -592,8 +598,11 @@ def run_corun_mla(args, rank, world):
                       + kernels["gemm_down"]["ms_per_launch"]) + kernels["gemm_lm_head"]["ms_per_launch"],
         "attention": L * kernels["attention"]["ms_per_launch"],
         "token_wise": L * (2 * kernels["resid_norm"]["ms_per_launch"] + kernels["rope_kv_append"]["ms_per_launch"])
-                      + (L - nd) * kernels["moe_router"]["ms_per_launch"] + kernels["sampler"]["ms_per_launch"],
-        "note": "expert layers only for gate / up, down and router (the one dense layer is left out); launched alone, back to back"}
+                      + (L - nd) * (kernels["moe_router"]["ms_per_launch"] + (kernels["moe_group_gather"]["ms_per_launch"] if grouped else 0.0))
+                      + kernels["sampler"]["ms_per_launch"],
+        "note": "expert layers only for gate / up, down and router (the one dense layer is left out); launched alone, back to back"
+                + ("; expert layers in their grouped form: gemm_gate_up = per-group GEMM with the SwiGLU in its epilogue, gemm_down = "
+                   "per-group GEMM + the sum over each row's experts, moe_group_gather = grouping + gather" if grouped else "")}
     # ---- isolated prefill of one request (its slot freed first): wall time of corun_prefill with the prompt in host
     # memory.  A prefill row attends to its request's latent cache up to its own position with the decode kernel,
     # so the attention part grows with the square of the prompt length.

@@ -43,7 +43,10 @@ int corun_debug_kv_fill(corun_engine *e, int32_t slot, int32_t n_ctx, float std,
  * 8 SwiGLU (none where the gate / up GEMM applies it), 9 sampler; engines with multi-head latent attention:
  * 5 = the latent attention (splits + combine), 7 = latent RMSNorm + rotary key + cache append + query parts,
  * 10 = grouped key up-projection, 11 = grouped value up-projection + split; engines with expert layers:
- * 2, 3, 6, 8 on the expert layers, 12 = router.  EINVAL for a kind the engine does not have.
+ * 2, 3, 6, 8 on the expert layers, 12 = router; where the decode program runs the expert layers in their grouped
+ * form (more than 64 padded rows): 2 = per-group gate / up GEMM (+ SwiGLU kernel where it is not in the epilogue),
+ * 3 = per-group down GEMM + the sum over each row's experts, 13 = grouping + gather, all on the groups of the last
+ * step's last layer.  EINVAL for a kind the engine does not have.
  * Uses the rows of the last decode step; overwrites
  * intermediate buffers (not the cache beyond each active slot's next position). */
 int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *avg_ms);

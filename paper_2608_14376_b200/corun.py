@@ -360,6 +360,7 @@ class Engine:
     # further kinds of corun_debug_time_kernel: engines with multi-head latent attention / with expert layers
     MLA_KERNEL_KINDS = {"mla_up_k": 10, "mla_up_v": 11}
     MOE_KERNEL_KINDS = {"moe_router": 12}
+    MOE_GROUPED_KERNEL_KINDS = {"moe_group_gather": 13}   # decode programs with more than 64 padded rows
 
     def time_kernel(self, kind: int, reps: int) -> float:
         ms = C.c_float(0.0)

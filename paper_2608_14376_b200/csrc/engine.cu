@@ -200,9 +200,10 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
       RC(dmalloc(A, &P.uv_out, hr * (md.nope + md.vh)));
       RC(dmalloc(A, &P.mla_ml, (size_t)mla_part_ml_floats(R, md.nh, e->max_ctx) / 2));
       RC(dmalloc(A, &P.mla_po, (size_t)mla_part_o_floats(R, md.nh, md.rank, e->max_ctx)));
-      RC(dmalloc(A, &P.tab_uk, (size_t)n_groups * 3));
-      RC(dmalloc(A, &P.tab_uv, (size_t)n_groups * 3));
-      std::vector<int> tk((size_t)n_groups * 3), tv((size_t)n_groups * 3);
+      RC(dmalloc(A, &P.tab_uk, (size_t)n_groups * 3 + 1));
+      RC(dmalloc(A, &P.tab_uv, (size_t)n_groups * 3 + 1));
+      std::vector<int> tk((size_t)n_groups * 3 + 1), tv((size_t)n_groups * 3 + 1);
+      tk[(size_t)n_groups * 3] = tv[(size_t)n_groups * 3] = n_groups;   // all groups are in use
       for (int g = 0; g < n_groups; ++g) {          // group = (head, block of BG rows): its weight rows, rows in use
         const int h = g / (P.RPH / BG), rb = g % (P.RPH / BG);
         const int valid = R - rb * BG < BG ? (R - rb * BG > 0 ? R - rb * BG : 0) : BG;
@@ -212,9 +213,9 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
       CK(cudaMemcpy(P.tab_uk, tk.data(), tk.size() * sizeof(int), cudaMemcpyHostToDevice));
       CK(cudaMemcpy(P.tab_uv, tv.data(), tv.size() * sizeof(int), cudaMemcpyHostToDevice));
       RC(gemm_plan_create_grouped(&P.p_uk, e->w_ukT, (long long)md.nh * md.rank, md.nope, md.rank, md.nope, P.qn_hi, P.qn_lo, n_groups,
-                                  BG, P.q_lat, P.tab_uk));
+                                  BG, P.q_lat, P.tab_uk, e->num_sms));
       RC(gemm_plan_create_grouped(&P.p_uv, e->w0_uv, (long long)md.nh * (md.nope + md.vh), md.rank, md.nope + md.vh, md.rank, P.ol_hi,
-                                  P.ol_lo, n_groups, BG, P.uv_out, P.tab_uv));
+                                  P.ol_lo, n_groups, BG, P.uv_out, P.tab_uv, e->num_sms));
       P.p_uk.keep_div = P.p_uv.keep_div = -1;       // the tables are written once, here: the kernels need not wait for them
     }
     RC(dmalloc(A, &P.qkv_out, (size_t)R * QKVN));
@@ -260,11 +261,12 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
         MoeGroups &g = P.grp;
         g.n_groups_max = moe_max_groups(R, e->moe_E, e->moe_S, e->moe_K);
         const size_t slots = (size_t)g.n_groups_max * MOE_GROUP_ROWS;
-        RC(dmalloc(A, &g.tab_up, (size_t)g.n_groups_max * 3));
-        RC(dmalloc(A, &g.tab_down, (size_t)g.n_groups_max * 3));
+        RC(dmalloc(A, &g.tab_up, (size_t)g.n_groups_max * 3 + 1));
+        RC(dmalloc(A, &g.tab_down, (size_t)g.n_groups_max * 3 + 1));
         RC(dmalloc(A, &g.group_expert, (size_t)g.n_groups_max));
         RC(dmalloc(A, &g.slot_row, slots));
         RC(dmalloc(A, &g.slot_of, (size_t)R * NB));
+        RC(dmalloc(A, &g.slot_w, slots));
         RC(dmalloc(A, &P.xg_hi, slots * H));
         RC(dmalloc(A, &P.xg_lo, slots * H));
         RC(dmalloc(A, &P.hg_hi, slots * Fm));
@@ -272,10 +274,17 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
         RC(dmalloc(A, &P.gug_out, slots * 2 * Fm));
         RC(dmalloc(A, &P.yg_out, slots * H));
         RC(dmalloc(A, &P.plain_tiles, (size_t)(H / GEMM_TILE_N + 1)));
-        RC(gemm_plan_create_grouped(&P.p_gug, e->w0_gu, (long long)NB * 2 * Fm, H, 2 * Fm, H, P.xg_hi, P.xg_lo, g.n_groups_max,
-                                    MOE_GROUP_ROWS, P.gug_out, g.tab_up));
+        // gate / up per group with the routing weight and the SwiGLU in the epilogue where a tile width divides the
+        // experts' width, else fp32 sums and a kernel of its own
+        const int half = gemm_swiglu_blocks_half(Fm, NB, e->num_sms);
+        if (half)
+          RC(gemm_plan_create_grouped_swiglu(&P.p_gug, e->w0_gu, (long long)NB * 2 * Fm, Fm, H, half, P.xg_hi, P.xg_lo, g.n_groups_max,
+                                             MOE_GROUP_ROWS, P.hg_hi, P.hg_lo, g.slot_w, g.tab_up, e->num_sms));
+        else
+          RC(gemm_plan_create_grouped(&P.p_gug, e->w0_gu, (long long)NB * 2 * Fm, H, 2 * Fm, H, P.xg_hi, P.xg_lo, g.n_groups_max,
+                                      MOE_GROUP_ROWS, P.gug_out, g.tab_up, e->num_sms));
         RC(gemm_plan_create_grouped(&P.p_dng, e->w0_down, H, NB * Fm, H, Fm, P.hg_hi, P.hg_lo, g.n_groups_max, MOE_GROUP_ROWS,
-                                    P.yg_out, g.tab_down));
+                                    P.yg_out, g.tab_down, e->num_sms));
         P.grouped = true;
       }
     }
@@ -383,8 +392,13 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
                               nullptr, e->st));
       STAGE(launch_moe_group(P.moe_w, P.row_active, P.R, e->moe_E, e->moe_S, e->moe_F, P.grp, e->st));
       STAGE(launch_moe_gather(P.xn_hi, P.xn_lo, s.hidden, P.grp, P.xg_hi, P.xg_lo, e->st));
-      STAGE(gemm_launch(P.p_gug, &e->tm_gu[l], e->d_status, e->st, nullptr, true));
-      STAGE(launch_moe_swiglu_grouped(P.gug_out, P.moe_w, NB, e->moe_F, P.grp, P.hg_hi, P.hg_lo, e->st));
+      if (P.p_gug.sw_hi) {                            // routing weight and SwiGLU in the GEMM's epilogue
+        STAGE(gemm_launch(P.p_gug, &e->tm_gu_half[l], e->d_status, e->st, nullptr, true));
+        n -= 1;
+      } else {
+        STAGE(gemm_launch(P.p_gug, &e->tm_gu[l], e->d_status, e->st, nullptr, true));
+        STAGE(launch_moe_swiglu_grouped(P.gug_out, P.moe_w, NB, e->moe_F, P.grp, P.hg_hi, P.hg_lo, e->st));
+      }
       STAGE(gemm_launch(P.p_dng, &e->tm_down[l], e->d_status, e->st, nullptr, true));
       STAGE(launch_moe_combine(P.yg_out, P.row_active, P.R, NB, s.hidden, P.grp, P.down_out, e->st));
       n += 13 + (&P == &e->dec ? 1 : 0);
@@ -753,7 +767,11 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
     if (atoi(ts) != 0 && (rc = dmalloc(A, &e->step_trace, (size_t)4 * s.n_layers * e->num_sms * 8))) return fail(rc);
   }
 #endif
-  if ((rc = program_create(e, e->dec, B, true, true, false, true))) return fail(rc);
+  // expert layers of the decode program: above 64 padded rows the grouped form (an expert's rows gathered into blocks of
+  // 64: one MMA per k-slice covers the hi and lo halves of a block, where every row through every expert costs two on
+  // 128 rows and keeps the tensor pipe as busy as the weight stream); up to 64 rows every row through every expert
+  const bool dec_grouped = e->moe_E > 0 && pad16(B) > 64 && !getenv("CORUN_MOE_DECODE_DENSE");
+  if ((rc = program_create(e, e->dec, B, true, true, dec_grouped, true))) return fail(rc);
   if ((rc = program_create(e, e->pre, e->chunk, true, false, e->moe_E > 0 && !getenv("CORUN_MOE_PREFILL_DENSE")))) return fail(rc);
   if ((rc = program_create(e, e->lm1, 1, false, true))) return fail(rc);
 
@@ -1191,9 +1209,10 @@ int corun_debug_kv_fill(corun_engine *e, int32_t slot, int32_t n_ctx, float std,
 }
 
 int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *avg_ms) {
-  if (!e || !avg_ms || reps < 1 || kind < 0 || kind > 12) return CORUN_EINVAL;
+  if (!e || !avg_ms || reps < 1 || kind < 0 || kind > 13) return CORUN_EINVAL;
   if ((kind == 10 || kind == 11) && !e->mla) return CORUN_EINVAL;   // the up-projections of an MLA layer
   if (kind == 12 && !e->moe_E) return CORUN_EINVAL;                  // the router of an expert layer
+  if (kind == 13 && !(e->moe_E && e->dec.grouped)) return CORUN_EINVAL;   // grouping + gather of the grouped form
   RC(sync_stream(e));
   Program &P = e->dec;
   const corun_shape &s = e->sh;
@@ -1209,7 +1228,7 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
     for (int i = 0; i < n && ce == cudaSuccess; ++i) {
       int l = i % s.n_layers;         // rotate over the layers so that L2 cannot hold the weights
       // feed-forward kinds of a decoder with dense and expert layers: the expert layers
-      if (e->mla && e->moe_E && (kind == 2 || kind == 3 || kind == 6 || kind == 8 || kind == 12))
+      if (e->mla && e->moe_E && (kind == 2 || kind == 3 || kind == 6 || kind == 8 || kind == 12 || kind == 13))
         l = e->first_dense + i % (s.n_layers - e->first_dense);
       GemmOut prev = ffn_out(e, P, l);
       const MlaCache mcache{e->mla ? e->kv_pool + (size_t)l * e->layer_stride : nullptr, e->d_block_table, e->max_blocks, e->B,
@@ -1218,8 +1237,19 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
         // launched as in the step's graph: with programmatic stream serialization
         case 0: ce = gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, nullptr, true); break;
         case 1: ce = gemm_launch(P.p_o, &e->tm_o[l], e->d_status, e->st, nullptr, true); break;
-        case 2: ce = gemm_launch(P.p_gu, P.p_gu.sw_hi ? &e->tm_gu_half[l] : &e->tm_gu[l], e->d_status, e->st, nullptr, true); break;
-        case 3: ce = gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st, nullptr, true); break;
+        case 2: if (P.grouped && !dense_layer(e, l)) {   // the groups of the last step's last layer
+                  ce = gemm_launch(P.p_gug, P.p_gug.sw_hi ? &e->tm_gu_half[l] : &e->tm_gu[l], e->d_status, e->st, nullptr, true);
+                  if (ce == cudaSuccess && !P.p_gug.sw_hi)
+                    ce = launch_moe_swiglu_grouped(P.gug_out, P.moe_w, e->moe_E + e->moe_S, e->moe_F, P.grp, P.hg_hi, P.hg_lo, e->st);
+                  break;
+                }
+                ce = gemm_launch(P.p_gu, P.p_gu.sw_hi ? &e->tm_gu_half[l] : &e->tm_gu[l], e->d_status, e->st, nullptr, true); break;
+        case 3: if (P.grouped && !dense_layer(e, l)) {   // per-group down GEMM + the sum over a row's experts
+                  ce = gemm_launch(P.p_dng, &e->tm_down[l], e->d_status, e->st, nullptr, true);
+                  if (ce == cudaSuccess) ce = launch_moe_combine(P.yg_out, P.row_active, P.R, e->moe_E + e->moe_S, s.hidden, P.grp, P.down_out, e->st);
+                  break;
+                }
+                ce = gemm_launch(P.p_down, &e->tm_down[l], e->d_status, e->st, nullptr, true); break;
         case 4: ce = gemm_launch(P.p_lm, nullptr, e->d_status, e->st, nullptr, true);
                 if (ce == cudaSuccess) ce = gemm_fixup_launch(P.p_lm, e->st);
                 break;
@@ -1244,7 +1274,7 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
                   break;
                 }
                 ce = launch_qkv_post(P.p_qkv.out(), rows, e->d_rope, s.n_q_heads, kv, l, P.q, e->d_status, e->st); break;
-        case 8: if (P.p_gu.sw_hi) break;             // no such kernel: the SwiGLU is in the GEMM's epilogue
+        case 8: if (P.p_gu.sw_hi || P.grouped) break;   // no such kernel: the SwiGLU is in the GEMM's epilogue (grouped form: timed with kind 2)
                 ce = e->moe_E ? launch_moe_swiglu(P.p_gu.out(), P.moe_w, P.R, e->moe_F, e->moe_E + e->moe_S, P.ff_hi, P.ff_lo, e->st)
                               : launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st);
                 break;
@@ -1256,6 +1286,9 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
         case 10: ce = gemm_launch(P.p_uk, &e->tm_uk[l], e->d_status, e->st, nullptr, true); break;
         case 11: ce = gemm_launch(P.p_uv, &e->tm_uv[l], e->d_status, e->st, nullptr, true);
                  if (ce == cudaSuccess) ce = launch_mla_ao_split(P.uv_out, P.R, P.RPH, e->md, P.ao_hi, P.ao_lo, e->st);
+                 break;
+        case 13: ce = launch_moe_group(P.moe_w, P.row_active, P.R, e->moe_E, e->moe_S, e->moe_F, P.grp, e->st);
+                 if (ce == cudaSuccess) ce = launch_moe_gather(P.xn_hi, P.xn_lo, s.hidden, P.grp, P.xg_hi, P.xg_lo, e->st);
                  break;
         case 12: ce = launch_moe_router(P.xn_hi, P.xn_lo, s.hidden, e->router[l], P.R, e->moe_E, e->moe_S, e->moe_K, e->moe_renorm,
                                         P.moe_w, nullptr, nullptr, e->st);

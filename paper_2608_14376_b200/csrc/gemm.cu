@@ -33,14 +33,19 @@ constexpr uint32_t A_BLOCK_BYTES = GEMM_ROW_BLOCK * GEMM_BLOCK_K * 2;      // 16
 // meaningless values that are never read back.
 // MASKED: the optional store mask of the epilogue (a separate instantiation, so that the plain kernel is
 // exactly the code it was without it).
-// GROUPED (with STACKED): every CTA owns one whole output tile of one group (an expert's rows, gathered into
-// blocks of BN rows).  group_tab holds, per group, the first weight row, the first weight k-block and the number
-// of rows (0 = the group is empty: its CTAs leave at once); the group's activations are rows group * BN .. of
-// the activation matrices, its output rows group * BN .. of `direct` (N columns wide, tiles_per_group tiles).
+// GROUPED (with STACKED): a tile is one whole output tile of one group (an expert's rows, gathered into blocks
+// of BN rows).  group_tab holds, per group, the first weight row, the first weight k-block and the number of
+// rows, and behind its keep_pitch entries the number of groups in use (the first ones); the CTAs take the tiles
+// of those groups in turn (tile cta, cta + grid, ...), streaming from one tile into the next like the plain
+// kernel.  The group's activations are rows group * BN .. of the activation matrices, its output rows
+// group * BN .. of `direct` (N columns wide, tiles_per_group tiles).
 // SWIGLU: W is a gate / up matrix ([2F, K]: F gate rows, then F up rows).  A tile is sw_half gate rows and the
 // sw_half up rows of the same outputs (two boxes of sw_half rows land in one stage; the MMA's N is 2 * sw_half),
 // every CTA owns whole tiles, and the epilogue writes silu(gate) * up as a bf16 hi/lo pair ([BN, F]) instead of
 // fp32 sums: no partials, no separate SwiGLU kernel.  tmW then has a box of sw_half rows.
+// SWIGLU with GROUPED: a group's N weight rows are one gate / up matrix (N / 2 gate rows, then N / 2 up rows) starting at
+// the group's first weight row; row_keep holds one factor per output row (the routing weight of the gathered row) and
+// the epilogue writes factor * silu(gate) * up to rows group * BN .. of the bf16 hi/lo output ([groups * BN, N / 2]).
 // SWIGLU with MASKED: W is a stack of keep_pitch such matrices (the experts of a Mixture-of-Experts layer: block e =
 // Fb gate rows, then Fb up rows, Fb = N / (2 * keep_pitch)), a tile belongs to one block (keep_div tiles per block),
 // and the epilogue writes row_keep[r, e] * silu(gate) * up, exact zeros where row r did not select block e, to
@@ -53,16 +58,6 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                     uint32_t idesc, const float *row_keep, int keep_pitch, int keep_div, const int *group_tab,
                     int tiles_per_group, int *status, unsigned long long *trace, __nv_bfloat16 *__restrict__ sw_hi,
                     __nv_bfloat16 *__restrict__ sw_lo, int sw_half) {
-  int g_id = 0, g_j = 0, g_wrow = 0, g_wk = 0, g_rows = 0;
-  if (GROUPED) {
-    if (keep_div >= 0) griddep_wait();              // the group table comes from an earlier kernel (keep_div < 0: it is fixed)
-    g_id = (int)blockIdx.x / tiles_per_group;
-    g_j = (int)blockIdx.x - g_id * tiles_per_group;
-    g_wrow = group_tab[3 * g_id];
-    g_wk = group_tab[3 * g_id + 1];
-    g_rows = group_tab[3 * g_id + 2];
-    if (g_rows <= 0) return;                        // the same decision in every thread of the CTA
-  }
   extern __shared__ uint8_t smem_raw[];
   // optional per-CTA timeline (debug): 8 globaltimer stamps
 #define TRACE(i) do { if (trace) trace[(size_t)blockIdx.x * 8 + (i)] = globaltimer_ns(); } while (0)
@@ -78,6 +73,19 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x;
+  // GROUPED: the group of the CTA's i-th tile (read only after the wait for the table below): group, tile inside it, first weight row, first weight k-block, rows in use
+  int g_tile = -1, g_id = 0, g_j = 0, g_wrow = 0, g_wk = 0, g_rows = 0;
+  auto look = [&](int tile) {
+    if (GROUPED && tile != g_tile) {
+      const int t = cta + tile * (int)gridDim.x;
+      g_tile = tile;
+      g_id = t / tiles_per_group;
+      g_j = t - g_id * tiles_per_group;
+      g_wrow = group_tab[3 * g_id];
+      g_wk = group_tab[3 * g_id + 1];
+      g_rows = group_tab[3 * g_id + 2];
+    }
+  };
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t x_bytes = (uint32_t)BN * GEMM_BLOCK_K * 2;         // BN * 128 B
   // Up to 64 rows: hi and lo share one 128-row A tile (hi in rows 0.., lo in rows 64..), so one MMA
@@ -88,6 +96,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   // SWIGLU: first gate row of a tile, and the distance to the up rows of the same outputs
   const int sw_fb = (SWIGLU && MASKED) ? N / (2 * keep_pitch) : N / 2;
   auto sw_gate_row = [&](int tile) {
+    if (GROUPED) return g_wrow + g_j * sw_half;       // (the caller has looked the tile's group up)
     if (SWIGLU && MASKED) {
       const int e = tile / keep_div;
       return e * 2 * sw_fb + (tile - e * keep_div) * sw_half;
@@ -129,7 +138,18 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   volatile int *abort_p = &abort_flag;
   if (threadIdx.x == 0) TRACE(1);
 
-  const int k0 = cta_start[cta], k1 = cta_start[cta + 1];
+  // GROUPED: the CTA walks the tiles cta, cta + grid, ... of the groups in use (their number follows the table's
+  // keep_pitch entries), every tile whole; the flat range counts the k-blocks of those tiles.
+  int k0, k1;
+  if (GROUPED) {
+    if (keep_div >= 0) griddep_wait();              // the group table comes from an earlier kernel (keep_div < 0: it is fixed)
+    const int used = min(group_tab[3 * keep_pitch], keep_pitch) * tiles_per_group;
+    k0 = 0;
+    k1 = cta < used ? (used - cta + (int)gridDim.x - 1) / (int)gridDim.x * KB : 0;
+  } else {
+    k0 = cta_start[cta];
+    k1 = cta_start[cta + 1];
+  }
   int fail = 0;
 
   if (warp == 0) {
@@ -143,6 +163,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       const int n_pre = min(stages, k1 - k0);
       for (int it = 0; it < n_pre; ++it) {
         const int g = k0 + it, tile = g / KB, kb = g - tile * KB;
+        look(tile);
         const uint32_t fb = smem_u32(&full_bar[it]);
         mbar_arrive_expect_tx(fb, tx_bytes);
         if (SWIGLU) {
@@ -157,6 +178,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       griddep_wait();
       for (int it = 0; it < n_pre; ++it) {
         const int g = k0 + it, tile = g / KB, kb = g - tile * KB;
+        look(tile);
         const uint32_t fb = smem_u32(&full_bar[it]);
         const uint32_t dst = tiles_base + (uint32_t)it * stage_bytes;
         tma_load_2d(dst + w_tile_bytes, &tmHi, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
@@ -165,6 +187,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       int it = n_pre;
       for (int g = k0 + n_pre; g < k1; ++g, ++it) {
         const int tile = g / KB, kb = g - tile * KB;
+        look(tile);
         const int s = it % stages;
         const uint32_t ph = (uint32_t)(it / stages) & 1u;
         if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_p)) { fail = DEV_TIMEOUT_PRODUCER; break; }
@@ -246,6 +269,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       if (!ok) { fail = DEV_TIMEOUT_EPILOGUE; break; }
       tc_fence_after();
       if (g + (kb_end - kb_begin) >= k1 && threadIdx.x == 64) TRACE(6);   // last accumulator is ready
+      look(tile);
       const int n0 = GROUPED ? g_j * GEMM_TILE_N : tile * GEMM_TILE_N;
       // optional: rows whose entry for this tile's column group is zero are not stored (nobody reads them)
       const float *keep = MASKED ? row_keep + tile / keep_div : nullptr;
@@ -256,13 +280,15 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         // F: outputs per block (the whole matrix unless MASKED); f0: the tile's first output inside its block;
         // o_base: its first column in the output row of N / 2 values; blk: the block (expert) of the tile
         const int blk = MASKED ? tile / keep_div : 0;
-        const int F = sw_fb, f0 = (MASKED ? tile - blk * keep_div : tile) * HALF;
+        const int F = sw_fb, f0 = (GROUPED ? g_j : MASKED ? tile - blk * keep_div : tile) * HALF;
         const int o_pitch = N / 2, o_base = blk * F + f0;
+        // GROUPED: the group's rows in use, its first output row, and row_keep = one weight per output row
+        const int sw_rows = GROUPED ? g_rows : R, sw_row0 = GROUPED ? g_id * BN : 0;
         auto silu_mul = [](float gt, float up) { return __fdividef(gt, 1.f + __expf(-gt)) * up; };
         if (stacked) {
           const bool lo_warp = lane_base >= 64;
           const int row = (lane_base & 63) + lane;
-          const bool warp_needed = (lane_base & 63) < R;   // warp-uniform
+          const bool warp_needed = (lane_base & 63) < sw_rows;   // warp-uniform
           float *xs = xch[lo_warp ? 1 : 0] + row * 33;
           const int te = (int)threadIdx.x - 64, srow = te >> 3, scol = (te & 7) * 4;
           for (int c0 = 0; c0 < HALF; c0 += 32) {
@@ -284,7 +310,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
                 const int r = i * 16 + srow;
-                if (r < R) {
+                if (r < sw_rows) {
                   const float *h = xch[0] + r * 33 + scol, *l = xch[1] + r * 33 + scol;
                   const float s0 = h[0] + l[0], s1 = h[1] + l[1], s2 = h[2] + l[2], s3 = h[3] + l[3];
                   if (part == 0) {
@@ -292,8 +318,8 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                   } else if (c0 + scol < HALF && f0 + c0 + scol < F) {   // HALF % 4 == 0, F % 4 == 0
                     float y[4] = {silu_mul(gt[i][0], s0), silu_mul(gt[i][1], s1), silu_mul(gt[i][2], s2),
                                   silu_mul(gt[i][3], s3)};
-                    if (MASKED) {                      // the row's routing weight for this expert; 0: not selected
-                      const float wgt = row_keep[(size_t)r * keep_pitch + blk];
+                    if (MASKED || GROUPED) {           // the row's routing weight for this expert; 0: not selected
+                      const float wgt = GROUPED ? row_keep[sw_row0 + r] : row_keep[(size_t)r * keep_pitch + blk];
 #pragma unroll
                       for (int q = 0; q < 4; ++q) y[q] = wgt != 0.f ? wgt * y[q] : 0.f;
                     }
@@ -303,7 +329,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                       a[q] = __float2bfloat16_rn(y[q]);
                       b[q] = __float2bfloat16_rn(y[q] - __bfloat162float(a[q]));
                     }
-                    const size_t o = (size_t)r * o_pitch + o_base + c0 + scol;
+                    const size_t o = (size_t)(sw_row0 + r) * o_pitch + o_base + c0 + scol;
                     *reinterpret_cast<uint2 *>(sw_hi + o) = *reinterpret_cast<const uint2 *>(a);
                     *reinterpret_cast<uint2 *>(sw_lo + o) = *reinterpret_cast<const uint2 *>(b);
                   }
@@ -704,14 +730,15 @@ int gemm_plan_create_swiglu_blocks(GemmPlan *p, const void *W, int n_blocks, int
 }
 
 int gemm_plan_create_grouped(GemmPlan *p, const void *W, long long w_rows, int w_cols, int N, int K, const void *Xhi,
-                             const void *Xlo, int n_groups, int BN, float *direct, const int *group_tab) {
+                             const void *Xlo, int n_groups, int BN, float *direct, const int *group_tab, int num_sms) {
   if (N <= 0 || N % GEMM_TILE_N || K <= 0 || K % GEMM_BLOCK_K || w_cols % GEMM_BLOCK_K || BN % 16 || BN < 16 || BN > 64 ||
-      n_groups < 1 || !group_tab || w_rows < N)
+      n_groups < 1 || !group_tab || w_rows < N || num_sms < 1)
     return CORUN_EINVAL;
   p->N = N; p->K = K; p->R = BN; p->BN = BN;
   p->n_tiles = n_groups * (N / GEMM_TILE_N);
   p->KB = K / GEMM_BLOCK_K;
-  p->grid = p->n_tiles;
+  p->grid = p->n_tiles < num_sms ? p->n_tiles : num_sms;
+  p->keep_pitch = n_groups;                         // where the table's count of groups in use sits
   const size_t stage = (size_t)GEMM_TILE_N * GEMM_BLOCK_K * 2 + (size_t)GEMM_ROW_BLOCK * GEMM_BLOCK_K * 2;
   int stages = (int)((GEMM_MAX_DYN_SMEM - 1024 - A_BLOCK_BYTES) / stage);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
@@ -743,12 +770,50 @@ int gemm_plan_create_grouped(GemmPlan *p, const void *W, long long w_rows, int w
   return CORUN_OK;
 }
 
+int gemm_plan_create_grouped_swiglu(GemmPlan *p, const void *W, long long w_rows, int F, int K, int half, const void *Xhi,
+                                    const void *Xlo, int n_groups, int BN, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
+                                    const float *row_scale, const int *group_tab, int num_sms) {
+  if (F <= 0 || half < 64 || half > GEMM_TILE_N / 2 || half % 8 || F % half || K <= 0 || K % GEMM_BLOCK_K || BN % 16 || BN < 16 ||
+      BN > 64 || n_groups < 1 || !group_tab || !out_hi || !out_lo || !row_scale || w_rows < 2 * F || num_sms < 1)
+    return CORUN_EINVAL;
+  p->sw_half = half;
+  p->N = 2 * F; p->K = K; p->R = BN; p->BN = BN;
+  p->tiles_per_group = F / half;
+  p->n_tiles = n_groups * p->tiles_per_group;
+  p->KB = K / GEMM_BLOCK_K;
+  p->grid = p->n_tiles < num_sms ? p->n_tiles : num_sms;
+  p->keep_pitch = n_groups;
+  const size_t stage = (size_t)2 * half * GEMM_BLOCK_K * 2 + (size_t)A_BLOCK_BYTES;
+  int stages = (int)((GEMM_MAX_DYN_SMEM - 1024 - A_BLOCK_BYTES) / stage);
+  if (stages > MAX_STAGES) stages = MAX_STAGES;
+  p->stages = stages;
+  p->smem_bytes = stage * stages + A_BLOCK_BYTES + 1024;
+  p->tmem_cols = 512;
+  p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * half) >> 3) << 17) | ((uint32_t)(GEMM_ROW_BLOCK >> 4) << 24);
+  p->direct = nullptr;
+  p->ws = nullptr;
+  p->sw_hi = out_hi;
+  p->sw_lo = out_lo;
+  p->row_keep = row_scale;
+  p->group_tab = group_tab;
+  int rc;
+  if ((rc = tma_encode_2d(&p->tmW, W, 0, (unsigned long long)w_rows, K, half, GEMM_BLOCK_K)) != 0) return rc;
+  if ((rc = tma_encode_2d(&p->tmHi, Xhi, 0, (unsigned long long)n_groups * BN, K, BN, GEMM_BLOCK_K)) != 0) return rc;
+  if ((rc = tma_encode_2d(&p->tmLo, Xlo, 0, (unsigned long long)n_groups * BN, K, BN, GEMM_BLOCK_K)) != 0) return rc;
+  p->d_cta_start = p->d_tile_first = p->d_tile_cend = p->d_split_tiles = nullptr;   // the kernel derives its tiles itself
+  p->n_split_tiles = 0;
+  cudaError_t ae = gemm_prepare_kernel();
+  if (ae != cudaSuccess) { g_last_cuda_error = (int)ae; return CORUN_ECUDA; }
+  return CORUN_OK;
+}
+
 cudaError_t gemm_prepare_kernel() {
   cudaError_t e = cudaFuncSetAttribute(gemm_streamk_kernel<false, false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
@@ -770,6 +835,7 @@ cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int 
                     p.row_keep, p.keep_pitch, p.keep_div, p.group_tab, p.tiles_per_group, d_status, trace, p.sw_hi, p.sw_lo,
                     p.sw_half);
   };
+  if (p.group_tab && p.sw_hi) return go(gemm_streamk_kernel<false, true, true, true>);
   if (p.sw_hi && masked) return stacked ? go(gemm_streamk_kernel<true, true, false, true>) : go(gemm_streamk_kernel<true, false, false, true>);
   if (p.sw_hi) return stacked ? go(gemm_streamk_kernel<false, true, false, true>) : go(gemm_streamk_kernel<false, false, false, true>);
   if (p.group_tab) return go(gemm_streamk_kernel<false, true, true, false>);

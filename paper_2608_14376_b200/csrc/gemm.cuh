@@ -87,8 +87,9 @@ struct GemmPlan {
   // row_keep[r * keep_pitch + t / keep_div] != 0 (rows that no consumer will read are skipped).
   const float *row_keep = nullptr;
   int keep_pitch = 0, keep_div = 1;
-  // Grouped mode (gemm_plan_create_grouped): one CTA per (group, weight tile); see gemm.cu.
-  const int *group_tab = nullptr;    // device, not owned: per group (first weight row, first weight k-block, rows);
+  // Grouped mode (gemm_plan_create_grouped): the CTAs take the (group, weight tile) pairs in turn; see gemm.cu.
+  const int *group_tab = nullptr;    // device, not owned: per group (first weight row, first weight k-block, rows),
+                                     // then ONE more int: the number of groups in use (the first ones);
                                      // keep_div = -1 tells the kernel that no kernel of the same stream writes it
   int tiles_per_group = 0;
   // Gate / up GEMM with SwiGLU in the epilogue (gemm_plan_create_swiglu): the bf16 hi/lo output [BN, N / 2].
@@ -109,9 +110,17 @@ void gemm_plan_destroy(GemmPlan *p);
 // Grouped GEMM over at most n_groups groups of up to BN <= 64 rows each: group g multiplies rows g * BN .. of
 // Xhi / Xlo ([n_groups * BN, K]) with N weight rows starting at the row, and K elements starting at the k-block,
 // that group_tab names for it, into rows g * BN .. of `direct` ([n_groups * BN, N]).  W is [w_rows, w_cols]
-// bf16.  One CTA per (group, tile of 256 weight rows), all k-blocks of it: no partials.  N % 256 == 0.
+// bf16.  group_tab has 3 * n_groups + 1 ints: the last one is the number of groups in use (groups 0 .. that - 1).
+// At most num_sms CTAs take the (group, tile of 256 weight rows) pairs of the groups in use in turn, all k-blocks
+// of a tile: no partials.  N % 256 == 0.
 int gemm_plan_create_grouped(GemmPlan *p, const void *W, long long w_rows, int w_cols, int N, int K, const void *Xhi,
-                             const void *Xlo, int n_groups, int BN, float *direct, const int *group_tab);
+                             const void *Xlo, int n_groups, int BN, float *direct, const int *group_tab, int num_sms);
+// The same for gate / up matrices ([2F, K] per group: F gate rows, then F up rows, from the group's first weight row)
+// with the SwiGLU in the epilogue: row_scale[g * BN + r] * silu(gate) * up as a bf16 hi/lo pair [n_groups * BN, F].
+// Tiles of `half` gate rows and the `half` up rows of the same outputs (F % half == 0, 64 <= half <= 128).
+int gemm_plan_create_grouped_swiglu(GemmPlan *p, const void *W, long long w_rows, int F, int K, int half, const void *Xhi,
+                                    const void *Xlo, int n_groups, int BN, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
+                                    const float *row_scale, const int *group_tab, int num_sms);
 // Gate / up GEMM with the SwiGLU in its epilogue: W is [2F, K] (F gate rows, then F up rows; F % 8 == 0);
 // out_hi / out_lo [BN, F] receive silu(gate) * up of rows 0 .. R-1 as a bf16 hi/lo pair.  A tile is
 // gemm_swiglu_half(F, num_sms) gate rows with the up rows of the same outputs, and every CTA owns whole tiles

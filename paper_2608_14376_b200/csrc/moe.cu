@@ -237,6 +237,7 @@ __global__ void __launch_bounds__(1024) moe_group_kernel(const float *__restrict
       u += (cnt[e] + MOE_GROUP_ROWS - 1) / MOE_GROUP_ROWS;
     }
     first[NB] = u < g.n_groups_max ? u : g.n_groups_max;
+    g.tab_up[3 * g.n_groups_max] = g.tab_down[3 * g.n_groups_max] = first[NB];   // groups in use: what the GEMMs walk
   }
   __syncthreads();
   for (int u = first[NB] + (int)threadIdx.x; u < g.n_groups_max; u += n_thr) {   // groups nobody needs
@@ -263,6 +264,7 @@ __global__ void __launch_bounds__(1024) moe_group_kernel(const float *__restrict
       if (on) {
         slot = base + __popc(m & ((1u << lane) - 1u));
         g.slot_row[slot] = r;
+        g.slot_w[slot] = w[(size_t)r * NB + e];
       }
       if (r < R) g.slot_of[(size_t)e * R + r] = slot;
       base += __popc(m);

@@ -27,11 +27,13 @@ inline int moe_max_groups(int R, int E, int S, int top_k) { return E + S + R * (
 // Buffers of the grouped form (device, owned by the caller).
 struct MoeGroups {
   int n_groups_max;      // moe_max_groups(...)
-  int *tab_up;           // [n_groups_max][3]: first gate/up weight row (e * 2F), 0, rows   (gemm group table)
-  int *tab_down;         // [n_groups_max][3]: 0, first down k-block (e * F / 64), rows
+  int *tab_up;           // [n_groups_max][3] + 1: first gate/up weight row (e * 2F), 0, rows   (gemm group table);
+                         //   the last int: groups in use
+  int *tab_down;         // [n_groups_max][3] + 1: 0, first down k-block (e * F / 64), rows; groups in use
   int *group_expert;     // [n_groups_max]
   int *slot_row;         // [n_groups_max * 64]: the chunk row gathered into the slot (valid below the group's row count)
   int *slot_of;          // [E + S][R]: where the row sits in the expert's groups, -1 = not selected
+  float *slot_w;         // [n_groups_max * 64]: the slot's routing weight w[row, expert] (valid below the group's row count)
 };
 
 // Groups the chunk's (row, expert) pairs: experts ascending, an expert's rows ascending, 64 per group; rows with

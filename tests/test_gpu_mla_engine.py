@@ -105,12 +105,13 @@ def test_mla_engine_parity_and_invariance(orc, first_dense, moe):
 
 def test_mla_engine_with_more_than_64_slots(orc):
     """The decode program above 64 padded rows: the grouped up-projections then run on two blocks of rows per head and
-    the expert layers' first GEMM applies the routing weight and the SwiGLU itself.  Parity with the oracle and the
-    same bytes in other slots (rows of both blocks)."""
+    the expert layers in their grouped form (an expert's rows gathered into blocks of 64, routing weight and SwiGLU in
+    the per-group gate / up GEMM's epilogue).  Parity with the oracle and the same bytes in other slots (rows of both
+    blocks)."""
     sh, Bw = SMALL, 80
     model, eng = _setup(orc, sh, dict(SMALL_MLA), SMALL_MOE, seed=6, B=Bw, max_ctx=128)
     try:
-        assert eng.decode_launches() == 6 + 13 + 13 * (sh.n_layers - 1)
+        assert eng.decode_launches() == 6 + 13 + 16 * (sh.n_layers - 1)
         prompts = synth.make_prompts(sh.vocab, [30, 77, 12, 50], seed=6)
         seeds = np.zeros(Bw, np.uint64)
         traces = []
