@@ -6,26 +6,43 @@
  * observes, in its comparison with LLM-42, that a small router perturbation
  * changes the selected experts.  In the fixed-shape decode iteration (Design,
  * "Fixed-Shape Batched Decode") the number of rows that pick an expert depends
- * on the co-tenants, so a grouped per-expert GEMM would give a row a different
- * tile shape, or a different place in it, from step to step.  This block has
- * no groups at all.  For B padded rows x [B, H]:
+ * on the co-tenants, so a per-expert GEMM whose TILE SHAPE followed that number
+ * would compute a row differently from step to step.  Here every shape is a
+ * function of the padded row count B alone.  For B padded rows x [B, H]:
  *
  *   router   logits = x Wr^T, p = softmax over all E experts, S = top_k by p
  *            (ties to the lower expert id), weights p_e as they are or, on
  *            request, renormalised over the selected ones; shared experts always
  *            on with weight 1;
+ *
+ * up to 64 padded rows, without groups (every row through every expert):
  *   GEMM 1   [B, H] x all experts' gate and up rows: [B, (E + S) * 2F];
  *   SwiGLU   h[r, e*F + f] = w[r, e] * silu(gate) * up, exactly 0 for the
  *            experts row r did not select;
  *   GEMM 2   y = h Wd_cat^T with K = (E + S) * F: the sum over a row's experts
  *            happens inside the accumulator, in ascending expert id (shared
  *            experts last), unselected experts contributing exact zeros.
+ *   All experts' weights are streamed once per call whatever was selected: the
+ *   padding the paper's title refers to, applied to experts.
  *
- * Both GEMMs are the library's decode GEMM (fixed tiles and K order for a
- * given B), so a row's result depends on its own x only: not on its row index,
- * not on what the other rows are or select.  All experts' weights are streamed
- * once per call whatever was selected: the padding the paper's title refers to,
- * applied to experts.
+ * above 64 padded rows (where two MMAs per k-slice for the hi and lo halves of
+ * 128 rows would keep the tensor pipe as busy as the weight stream), grouped:
+ *   grouping the rows that selected expert e, in ascending row order, fill blocks
+ *            of exactly 64 rows (the last one padded); experts ascending;
+ *   gather   the rows' hi / lo activations into their blocks;
+ *   GEMM 1   per block: [64, H] x the expert's gate and up rows, w[r, e] *
+ *            silu(gate) * up in the epilogue;
+ *   GEMM 2   per block: [64, F] x the expert's down projection, fp32;
+ *   combine  y[r] = the row's experts' results added in ascending expert id
+ *            (shared experts last).
+ *   The block shape, the tiles and the K order are the same for every block and
+ *   every step; an accumulator row is computed from its own activation row only,
+ *   so neither the row's place in its block nor what else the block holds
+ *   reaches its result.  Experts nobody selected are not streamed.
+ *
+ * Either way the GEMMs are the library's decode GEMM (fixed tiles and K order
+ * for a given B), so a row's result depends on its own x only: not on its row
+ * index, not on what the other rows are or select.
  *
  * All data pointers are DEVICE pointers; calls are asynchronous on the stream
  * given at creation except where stated.  Status codes are those of corun.h.

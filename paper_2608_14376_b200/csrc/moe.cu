@@ -190,81 +190,93 @@ __global__ void __launch_bounds__(256) moe_readout_kernel(GemmOut d, int H, floa
   *reinterpret_cast<float4 *>(y + (size_t)r * H + i) = gemm_load4(d, r, i);
 }
 
-// ---------------------------------------------------------------- grouped form (prefill chunks)
-// One CTA of 1024 threads (32 warps: everything here waits on memory, so the more warps the better).  Phase 0: the selection w[r, e] != 0 (rows read with coalesced loads) as
-// bytes sel[e][r] in shared memory; phase 1: warp per expert counts its rows; phase 2: one thread turns the
-// counts into first-group indices (experts ascending); phase 3: warp per expert writes its groups' table
-// entries and hands its rows, in ascending row order, consecutive slots (slot_of is expert-major: [E + S][R]).
-__global__ void __launch_bounds__(1024) moe_group_kernel(const float *__restrict__ w, const int *__restrict__ active, int R,
-                                                        int NB, int E, int F, MoeGroups g) {
+// ---------------------------------------------------------------- grouped form
+// One CTA per expert (routed experts, then the shared ones).  Every CTA counts the rows of ALL experts (the table
+// w[r, e] != 0 is small and comes from L2), so that it knows where its own expert's groups begin (experts ascending,
+// 64 rows per group) without a second kernel; it then writes its groups' table entries and hands its rows, in
+// ascending row order, consecutive slots (slot_of is expert-major: [E + S][R]).  CTA 0 also clears the entries of
+// the groups nobody needs and publishes the number of groups in use.
+constexpr int MOE_GROUP_THREADS = 512;
+__global__ void __launch_bounds__(MOE_GROUP_THREADS) moe_group_kernel(const float *__restrict__ w, const int *__restrict__ active, int R,
+                                                       int NB, int E, int F, MoeGroups g) {
   griddep_launch_dependents();
-  griddep_wait();
-  extern __shared__ unsigned char sel[];            // [NB][R + 4]: the pitch keeps a warp's 32 experts in 32 banks
-  const int SP = R + 4;
-  __shared__ int cnt[MOE_MAX_EXPERTS + 8], first[MOE_MAX_EXPERTS + 9];
+  __shared__ int cnt[MOE_MAX_EXPERTS + 8];
+  __shared__ float wsel[256];                        // the own expert's weight per row, 0 = not selected
   __shared__ unsigned char act[256];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = (int)blockDim.x >> 5, n_thr = (int)blockDim.x;
-  for (int r = (int)threadIdx.x; r < R; r += n_thr) act[r] = active[r] != 0;
+  __shared__ int first_s, total_s;
+  const int e = (int)blockIdx.x, tid = (int)threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int i = tid; i < NB; i += MOE_GROUP_THREADS) cnt[i] = 0;
+  griddep_wait();
+  w = after_wait(w); active = after_wait(active);    // no load through them may move up across the wait
+  for (int r = tid; r < R; r += MOE_GROUP_THREADS) { act[r] = active[r] != 0; wsel[r] = 0.f; }
   __syncthreads();
   {
-    // eight independent loads per thread in flight (the table is read once, from L2)
+    // sixteen independent loads per thread in flight
     const int total = R * NB;
-    for (int i0 = (int)threadIdx.x; i0 < total; i0 += n_thr * 8) {
-      float v[8];
+    for (int i0 = tid; i0 < total; i0 += MOE_GROUP_THREADS * 16) {
+      float v[16];
 #pragma unroll
-      for (int k = 0; k < 8; ++k) v[k] = i0 + n_thr * k < total ? w[i0 + n_thr * k] : 0.f;
+      for (int k = 0; k < 16; ++k) v[k] = i0 + MOE_GROUP_THREADS * k < total ? w[i0 + MOE_GROUP_THREADS * k] : 0.f;
 #pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const int i = i0 + n_thr * k;
-        if (i < total) {
-          const int r = i / NB, e = i - r * NB;
-          sel[e * SP + r] = (v[k] != 0.f && act[r]) ? 1 : 0;
+      for (int k = 0; k < 16; ++k) {
+        const int i = i0 + MOE_GROUP_THREADS * k;
+        if (i < total && v[k] != 0.f) {
+          const int r = i / NB, ee = i - r * NB;
+          if (act[r]) {
+            atomicAdd(&cnt[ee], 1);                  // integer counts: the order of the additions does not matter
+            if (ee == e) wsel[r] = v[k];
+          }
         }
       }
     }
   }
   __syncthreads();
-  for (int e = warp; e < NB; e += n_warps) {
-    int c = 0;
-    for (int r0 = 0; r0 < R; r0 += 32) c += __popc(__ballot_sync(0xffffffffu, r0 + lane < R && sel[e * SP + r0 + lane]));
-    if (lane == 0) cnt[e] = c;
+  if (warp == 0) {
+    // groups before this expert, and in all: lanes take experts lane, lane + 32, ...
+    int before = 0, all = 0;
+    for (int ee = lane; ee < NB; ee += 32) {
+      const int n = (cnt[ee] + MOE_GROUP_ROWS - 1) / MOE_GROUP_ROWS;
+      all += n;
+      if (ee < e) before += n;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      before += __shfl_xor_sync(0xffffffffu, before, o);
+      all += __shfl_xor_sync(0xffffffffu, all, o);
+    }
+    if (lane == 0) { first_s = before; total_s = all < g.n_groups_max ? all : g.n_groups_max; }
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
-    int u = 0;
-    for (int e = 0; e < NB; ++e) {
-      first[e] = u;
-      u += (cnt[e] + MOE_GROUP_ROWS - 1) / MOE_GROUP_ROWS;
+  const int first = first_s, used = total_s;
+  if (e == 0) {
+    for (int u = used + tid; u < g.n_groups_max; u += MOE_GROUP_THREADS) {   // groups nobody needs
+      g.tab_up[3 * u] = 0; g.tab_up[3 * u + 1] = 0; g.tab_up[3 * u + 2] = 0;
+      g.tab_down[3 * u] = 0; g.tab_down[3 * u + 1] = 0; g.tab_down[3 * u + 2] = 0;
+      g.group_expert[u] = -1;
     }
-    first[NB] = u < g.n_groups_max ? u : g.n_groups_max;
-    g.tab_up[3 * g.n_groups_max] = g.tab_down[3 * g.n_groups_max] = first[NB];   // groups in use: what the GEMMs walk
+    if (tid == 0) g.tab_up[3 * g.n_groups_max] = g.tab_down[3 * g.n_groups_max] = used;   // what the GEMMs walk
   }
-  __syncthreads();
-  for (int u = first[NB] + (int)threadIdx.x; u < g.n_groups_max; u += n_thr) {   // groups nobody needs
-    g.tab_up[3 * u] = 0; g.tab_up[3 * u + 1] = 0; g.tab_up[3 * u + 2] = 0;
-    g.tab_down[3 * u] = 0; g.tab_down[3 * u + 1] = 0; g.tab_down[3 * u + 2] = 0;
-    g.group_expert[u] = -1;
+  const int n_groups = (cnt[e] + MOE_GROUP_ROWS - 1) / MOE_GROUP_ROWS;
+  for (int k = tid; k < n_groups; k += MOE_GROUP_THREADS) {
+    const int u = first + k;
+    if (u >= g.n_groups_max) break;                 // cannot happen: n_groups_max bounds the sum
+    const int rows = min(MOE_GROUP_ROWS, cnt[e] - k * MOE_GROUP_ROWS);
+    g.tab_up[3 * u] = e * 2 * F; g.tab_up[3 * u + 1] = 0; g.tab_up[3 * u + 2] = rows;
+    g.tab_down[3 * u] = 0; g.tab_down[3 * u + 1] = e * F / GEMM_BLOCK_K; g.tab_down[3 * u + 2] = rows;
+    g.group_expert[u] = e;
   }
-  for (int e = warp; e < NB; e += n_warps) {
-    const int n_groups = (cnt[e] + MOE_GROUP_ROWS - 1) / MOE_GROUP_ROWS;
-    for (int k = lane; k < n_groups; k += 32) {
-      const int u = first[e] + k;
-      if (u >= g.n_groups_max) break;               // cannot happen: n_groups_max bounds the sum
-      const int rows = min(MOE_GROUP_ROWS, cnt[e] - k * MOE_GROUP_ROWS);
-      g.tab_up[3 * u] = e * 2 * F; g.tab_up[3 * u + 1] = 0; g.tab_up[3 * u + 2] = rows;
-      g.tab_down[3 * u] = 0; g.tab_down[3 * u + 1] = e * F / GEMM_BLOCK_K; g.tab_down[3 * u + 2] = rows;
-      g.group_expert[u] = e;
-    }
-    int base = first[e] * MOE_GROUP_ROWS;            // slot of the expert's next row
+  if (warp == 0) {
+    int base = first * MOE_GROUP_ROWS;               // slot of the expert's next row
     for (int r0 = 0; r0 < R; r0 += 32) {
       const int r = r0 + lane;
-      const bool on = r < R && sel[e * SP + r];
+      const float wv = r < R ? wsel[r] : 0.f;
+      const bool on = wv != 0.f;
       const unsigned m = __ballot_sync(0xffffffffu, on);
       int slot = -1;
       if (on) {
         slot = base + __popc(m & ((1u << lane) - 1u));
         g.slot_row[slot] = r;
-        g.slot_w[slot] = w[(size_t)r * NB + e];
+        g.slot_w[slot] = wv;
       }
       if (r < R) g.slot_of[(size_t)e * R + r] = slot;
       base += __popc(m);
@@ -272,16 +284,31 @@ __global__ void __launch_bounds__(1024) moe_group_kernel(const float *__restrict
   }
 }
 
+// The gathered activation rows: one warp per slot of the groups in use (all of a row's loads requested before the
+// first store).  H % 256 == 0 up to 4096, else eight 16-byte pieces per lane at a time.
 __global__ void __launch_bounds__(256) moe_gather_kernel(const bf16 *__restrict__ x_hi, const bf16 *__restrict__ x_lo, int H,
                                                          MoeGroups g, bf16 *__restrict__ xg_hi, bf16 *__restrict__ xg_lo) {
   griddep_launch_dependents();
   griddep_wait();
-  const int slot = blockIdx.x;
-  if (slot % MOE_GROUP_ROWS >= g.tab_up[3 * (slot / MOE_GROUP_ROWS) + 2]) return;   // no row in this slot
-  const int r = g.slot_row[slot];
-  const uint4 *sh = reinterpret_cast<const uint4 *>(x_hi + (size_t)r * H), *sl = reinterpret_cast<const uint4 *>(x_lo + (size_t)r * H);
-  uint4 *dh = reinterpret_cast<uint4 *>(xg_hi + (size_t)slot * H), *dl = reinterpret_cast<uint4 *>(xg_lo + (size_t)slot * H);
-  for (int i = threadIdx.x; i < H / 8; i += blockDim.x) { dh[i] = sh[i]; dl[i] = sl[i]; }
+  x_hi = after_wait(x_hi); x_lo = after_wait(x_lo);
+  const int lane = threadIdx.x & 31;
+  const int n_slots = g.tab_up[3 * g.n_groups_max] * MOE_GROUP_ROWS;
+  const int n_warps = (int)(gridDim.x * (blockDim.x >> 5));
+  for (int slot = (int)(blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)); slot < n_slots; slot += n_warps) {
+    if (slot % MOE_GROUP_ROWS >= g.tab_up[3 * (slot / MOE_GROUP_ROWS) + 2]) continue;   // no row in this slot
+    const int r = g.slot_row[slot];
+    const uint4 *sh = reinterpret_cast<const uint4 *>(x_hi + (size_t)r * H), *sl = reinterpret_cast<const uint4 *>(x_lo + (size_t)r * H);
+    uint4 *dh = reinterpret_cast<uint4 *>(xg_hi + (size_t)slot * H), *dl = reinterpret_cast<uint4 *>(xg_lo + (size_t)slot * H);
+    for (int i0 = lane; i0 < H / 8; i0 += 32 * 8) {
+      uint4 a[8], b[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (i0 + 32 * k < H / 8) { a[k] = sh[i0 + 32 * k]; b[k] = sl[i0 + 32 * k]; }
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (i0 + 32 * k < H / 8) { dh[i0 + 32 * k] = a[k]; dl[i0 + 32 * k] = b[k]; }
+    }
+  }
 }
 
 __global__ void __launch_bounds__(256) moe_swiglu_grouped_kernel(const float *__restrict__ gu, const float *__restrict__ w,
@@ -313,19 +340,35 @@ __global__ void __launch_bounds__(256) moe_combine_kernel(const float *__restric
                                                           int H, MoeGroups g, float *__restrict__ y) {
   griddep_launch_dependents();
   griddep_wait();
+  yg = after_wait(yg); active = after_wait(active);
   const int r = blockIdx.y;
   if (!active[r]) return;
-  __shared__ int slots[MOE_MAX_EXPERTS + 8];
-  for (int e = threadIdx.x; e < NB; e += blockDim.x) slots[e] = g.slot_of[(size_t)e * gridDim.y + r];
+  __shared__ int slots[MOE_MAX_EXPERTS + 8];         // the row's slots, experts ascending (shared experts last), compacted
+  __shared__ int n_sel;
+  if (threadIdx.x < 32) {
+    int n = 0;
+    for (int e0 = 0; e0 < NB; e0 += 32) {
+      const int e = e0 + (int)threadIdx.x;
+      const int slot = e < NB ? g.slot_of[(size_t)e * gridDim.y + r] : -1;
+      const unsigned m = __ballot_sync(0xffffffffu, slot >= 0);
+      if (slot >= 0) slots[n + __popc(m & ((1u << threadIdx.x) - 1u))] = slot;
+      n += __popc(m);
+    }
+    if (threadIdx.x == 0) n_sel = n;
+  }
   __syncthreads();
   const int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i >= H) return;
+  const int n = n_sel;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int e = 0; e < NB; ++e) {                     // ascending expert id, shared experts last
-    const int slot = slots[e];
-    if (slot < 0) continue;
-    const float4 v = *reinterpret_cast<const float4 *>(yg + (size_t)slot * H + i);
-    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+  for (int k0 = 0; k0 < n; k0 += 8) {                // eight loads in flight; the additions stay in ascending order
+    float4 v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      if (k0 + k < n) v[k] = *reinterpret_cast<const float4 *>(yg + (size_t)slots[k0 + k] * H + i);
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      if (k0 + k < n) { acc.x += v[k].x; acc.y += v[k].y; acc.z += v[k].z; acc.w += v[k].w; }
   }
   *reinterpret_cast<float4 *>(y + (size_t)r * H + i) = acc;
 }
@@ -336,21 +379,14 @@ namespace corun {
 
 cudaError_t launch_moe_group(const float *w, const int *active, int R, int E, int S, int F, const MoeGroups &g,
                              cudaStream_t st) {
-  if (E + S > MOE_MAX_EXPERTS + 8 || F % GEMM_BLOCK_K) return cudaErrorInvalidValue;
-  const size_t smem = (size_t)(E + S) * (R + 4);    // <= 264 * 260 bytes
-  static bool prepared = false;
-  if (!prepared) {
-    cudaError_t e = cudaFuncSetAttribute(moe_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (MOE_MAX_EXPERTS + 8) * 260);
-    if (e != cudaSuccess) return e;
-    prepared = true;
-  }
-  if (R > 256) return cudaErrorInvalidValue;
-  return launch_k(moe_group_kernel, dim3(1), dim3(1024), smem, st, true, w, active, R, E + S, E, F, g);
+  if (E + S > MOE_MAX_EXPERTS + 8 || F % GEMM_BLOCK_K || R > 256) return cudaErrorInvalidValue;
+  return launch_k(moe_group_kernel, dim3(E + S), dim3(MOE_GROUP_THREADS), 0, st, true, w, active, R, E + S, E, F, g);
 }
 
 cudaError_t launch_moe_gather(const __nv_bfloat16 *x_hi, const __nv_bfloat16 *x_lo, int H, const MoeGroups &g,
                               __nv_bfloat16 *xg_hi, __nv_bfloat16 *xg_lo, cudaStream_t st) {
-  return launch_k(moe_gather_kernel, dim3(g.n_groups_max * MOE_GROUP_ROWS), dim3(256), 0, st, true, x_hi, x_lo, H, g, xg_hi, xg_lo);
+  const int blocks = (g.n_groups_max * MOE_GROUP_ROWS + 7) / 8;   // a warp per slot, as far as 1184 CTAs go
+  return launch_k(moe_gather_kernel, dim3(blocks < 1184 ? blocks : 1184), dim3(256), 0, st, true, x_hi, x_lo, H, g, xg_hi, xg_lo);
 }
 
 cudaError_t launch_moe_swiglu_grouped(const float *gu, const float *w, int n_blocks, int F, const MoeGroups &g,
@@ -388,6 +424,13 @@ struct corun_moe {
   float *out_gu = nullptr, *out_d = nullptr, *ws = nullptr, *w = nullptr;
   int *d_status = nullptr;
   GemmPlan p_gu, p_d;
+  // grouped form (more than 64 padded rows): an expert's rows gathered into blocks of 64
+  bool grouped = false;
+  MoeGroups grp{};
+  bf16 *xg_hi = nullptr, *xg_lo = nullptr, *hg_hi = nullptr, *hg_lo = nullptr;
+  float *yg = nullptr;
+  int *d_active = nullptr;
+  GemmPlan p_gug, p_dng;
   int64_t weight_bytes = 0;
 };
 
@@ -451,6 +494,30 @@ int corun_moe_create(const corun_moe_shape *shape, const void *router, const voi
     m->p_gu.keep_pitch = NB;
     m->p_gu.keep_div = 2 * F / GEMM_TILE_N;
   }
+  // above 64 padded rows: the grouped form (one MMA per k-slice covers the hi and lo halves of a block of 64 rows,
+  // where every row through every expert costs two on 128 rows), with the routing weight and the SwiGLU in the
+  // per-group gate / up GEMM's epilogue
+  const int g_half = gemm_swiglu_blocks_half(F, NB, m->num_sms);
+  if (m->BN > 64 && g_half > 0 && H % GEMM_TILE_N == 0 && !getenv("CORUN_MOE_DECODE_DENSE")) {
+    MoeGroups &g = m->grp;
+    g.n_groups_max = moe_max_groups(B, E, s.n_shared, s.top_k);
+    const size_t slots = (size_t)g.n_groups_max * MOE_GROUP_ROWS;
+    if ((rc = moe_alloc(m, &g.tab_up, (size_t)g.n_groups_max * 3 + 1)) || (rc = moe_alloc(m, &g.tab_down, (size_t)g.n_groups_max * 3 + 1)) ||
+        (rc = moe_alloc(m, &g.group_expert, (size_t)g.n_groups_max)) || (rc = moe_alloc(m, &g.slot_row, slots)) ||
+        (rc = moe_alloc(m, &g.slot_of, (size_t)B * NB)) || (rc = moe_alloc(m, &g.slot_w, slots)) ||
+        (rc = moe_alloc(m, &m->xg_hi, slots * H)) || (rc = moe_alloc(m, &m->xg_lo, slots * H)) ||
+        (rc = moe_alloc(m, &m->hg_hi, slots * F)) || (rc = moe_alloc(m, &m->hg_lo, slots * F)) ||
+        (rc = moe_alloc(m, &m->yg, slots * H)) || (rc = moe_alloc(m, &m->d_active, (size_t)B)))
+      return fail(rc);
+    std::vector<int> ones((size_t)B, 1);
+    if (cudaMemcpy(m->d_active, ones.data(), (size_t)B * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return fail(CORUN_ECUDA);
+    if ((rc = gemm_plan_create_grouped_swiglu(&m->p_gug, gate_up, (long long)NB * 2 * F, F, H, g_half, m->xg_hi, m->xg_lo, g.n_groups_max,
+                                              MOE_GROUP_ROWS, m->hg_hi, m->hg_lo, g.slot_w, g.tab_up, m->num_sms)) ||
+        (rc = gemm_plan_create_grouped(&m->p_dng, down, H, NB * F, H, F, m->hg_hi, m->hg_lo, g.n_groups_max, MOE_GROUP_ROWS, m->yg,
+                                       g.tab_down, m->num_sms)))
+      return fail(rc);
+    m->grouped = true;
+  }
   m->weight_bytes = ((int64_t)E * H + (int64_t)N1 * H + (int64_t)H * K2) * 2;
   if (cudaDeviceSynchronize() != cudaSuccess) return fail(CORUN_ECUDA);
   *out = m;
@@ -462,6 +529,8 @@ void corun_moe_destroy(corun_moe *m) {
   cudaStreamSynchronize(m->st);
   gemm_plan_destroy(&m->p_gu);
   gemm_plan_destroy(&m->p_d);
+  gemm_plan_destroy(&m->p_gug);
+  gemm_plan_destroy(&m->p_dng);
   for (void *p : m->allocs) cudaFree(p);
   delete m;
 }
@@ -473,6 +542,16 @@ int corun_moe_forward(corun_moe *m, const float *x, float *y, int32_t *experts, 
   const int H = s.hidden, E = s.n_experts, F = s.expert_ffn, NB = E + s.n_shared;
   MCK(launch_split(x, m->B, H, m->x_hi, m->x_lo, m->st));
   MCK(launch_moe_router(m->x_hi, m->x_lo, H, m->router, m->B, E, s.n_shared, s.top_k, s.renormalize, m->w, experts, probs, m->st));
+  if (m->grouped) {
+    // rows grouped by expert -> gate / up with routing weight and SwiGLU, and down, per group -> the row's experts
+    // summed in ascending expert id
+    MCK(launch_moe_group(m->w, m->d_active, m->B, E, s.n_shared, F, m->grp, m->st));
+    MCK(launch_moe_gather(m->x_hi, m->x_lo, H, m->grp, m->xg_hi, m->xg_lo, m->st));
+    MCK(gemm_launch(m->p_gug, nullptr, m->d_status, m->st, nullptr, true));
+    MCK(gemm_launch(m->p_dng, nullptr, m->d_status, m->st, nullptr, true));
+    MCK(launch_moe_combine(m->yg, m->d_active, m->B, NB, H, m->grp, y, m->st));
+    return CORUN_OK;
+  }
   MCK(gemm_launch(m->p_gu, nullptr, m->d_status, m->st, nullptr, true));
   if (!m->p_gu.sw_hi) MCK(launch_moe_swiglu(m->p_gu.out(), m->w, m->B, F, NB, m->h_hi, m->h_lo, m->st));
   MCK(gemm_launch(m->p_d, nullptr, m->d_status, m->st, nullptr, true));
@@ -490,6 +569,6 @@ int corun_moe_sync(corun_moe *m) {
 
 int64_t corun_moe_weight_bytes(const corun_moe *m) { return m ? m->weight_bytes : 0; }
 
-int corun_moe_launches(const corun_moe *m) { return m ? (m->p_gu.sw_hi ? 5 : 6) : CORUN_EINVAL; }
+int corun_moe_launches(const corun_moe *m) { return m ? (m->grouped ? 7 : m->p_gu.sw_hi ? 5 : 6) : CORUN_EINVAL; }
 
 }  // extern "C"
