@@ -627,8 +627,9 @@ def run_corun_mla(args, rank, world):
     del eng, w_t, m_t, e_t
     torch.cuda.empty_cache()
 
-    # ---- the dominant kernels: the expert block of one layer (router, gate / up GEMM over all experts, masked SwiGLU,
-    # down GEMM), timed alone with CUDA events against the expert weights one call streams
+    # ---- the dominant kernels: the expert block of one layer (router, grouping and gather, per-group gate / up GEMM with
+    # the SwiGLU in its epilogue, per-group down GEMM, combine), timed alone with CUDA events against the expert weights
+    # one call streams
     roofline = None
     if rank == 0:
         from paper_2608_14376_b200.corun import MoeFfn
@@ -658,12 +659,12 @@ def run_corun_mla(args, rank, world):
         mtp = os.path.join(ROOT, "profiles", "moe_block_dram_traffic.json")
         if os.path.exists(mtp):
             mtraffic = json.load(open(mtp)).get("dram_bytes_per_call")
-        roofline = {"kernel": "expert block of one layer (router, gate / up GEMM over all experts with routing weight and SwiGLU in its epilogue, down GEMM): "
+        roofline = {"kernel": "expert block of one layer in its grouped form (router, grouping, gather, per-group gate / up GEMM with routing weight and SwiGLU in its epilogue, per-group down GEMM, combine): "
                               "%d of a step's %d layers" % (sh.n_layers - mla_cfg["first_dense"], sh.n_layers),
                     "bound": "hbm", "achieved": wb / (mms * 1e-3) / 1e9, "peak": hbm, "unit": "GB/s",
                     "peak_source": which + " (MEASURED_PEAKS.json hbm_gbs)" if which == "measured" else "fallback 6650",
                     "traffic": mtraffic, "bytes_per_launch_avg": wb, "ms_per_launch_avg": mms,
-                    "scope": "one call of the block (split, router, two GEMMs, read-out); the whole step against its roofline is in step_roofline",
+                    "scope": "one call of the block (split, router, grouping, gather, two grouped GEMMs, combine: %d launches); the whole step against its roofline is in step_roofline" % ops[0][0].launches(),
                     "timing": "CUDA events over %d back-to-back calls rotating over %d weight sets (%.0f MB each)" % (n_rep, copies, wb / 1e6)}
         roofline["frac"] = roofline["achieved"] / hbm
         for op, *_ in ops:
