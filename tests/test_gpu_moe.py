@@ -36,8 +36,10 @@ def _device_op(corun, torch, w, H, E, K, F, S, B, renorm=False):
 @pytest.mark.parametrize("H,E,K,F,S,B,renorm", [(256, 8, 2, 128, 1, 16, False), (512, 64, 6, 192, 2, 40, False),
                                                   (128, 5, 5, 64, 0, 3, False), (256, 16, 4, 128, 1, 100, False),
                                                   (256, 32, 8, 128, 0, 24, True),
-                                                  # 65..128 rows: routing weight and SwiGLU in the first GEMM's epilogue,
-                                                  # with tiles of 96 and of 128 gate rows (the DeepSeek-V2-Lite expert width)
+                                                  # above 64 rows the grouped form (blocks of 64 rows per expert; experts
+                                                  # and shared experts with more than one block), routing weight and SwiGLU
+                                                  # in the per-block GEMM's epilogue, with tiles of 96 and of 128 gate rows
+                                                  # (the DeepSeek-V2-Lite expert width)
                                                   (512, 64, 6, 192, 2, 72, False), (256, 6, 2, 1408, 2, 128, False)])
 def test_moe_matches_oracle_and_is_position_invariant(H, E, K, F, S, B, renorm):
     torch = pytest.importorskip("torch")
