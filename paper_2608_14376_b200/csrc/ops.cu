@@ -240,7 +240,7 @@ struct SmpShared {
 // Horner form, separately rounded multiplies and adds; exact scaling by 2^(n+40).
 __device__ __forceinline__ unsigned long long smp_weight(float l, float mx, float inv_t_log2e) {
   const float x = __fmul_rn(__fsub_rn(l, mx), inv_t_log2e);
-  if (!(x > -64.0f)) return 0ull;
+  if (!(x > -41.5f)) return 0ull;                    // rint(x) <= -42 (ties to even): the weight below is 0 (also NaN)
   const float n = rintf(x);
   const float f = __fsub_rn(x, n);
   float p = 0x1.ffcbfcp-17f;
@@ -255,6 +255,17 @@ __device__ __forceinline__ unsigned long long smp_weight(float l, float mx, floa
   if (ni < -41) return 0ull;
   const float scale = __int_as_float((ni + 40 + 127) << 23);   // 2^(n+40), exact
   return (unsigned long long)__fmul_rn(p, scale);              // truncation = floor
+}
+
+// hist[bin] += w with two 32-bit shared-memory atomics instead of one 64-bit one: the low words wrap modulo 2^32
+// and exactly the additions that wrap carry one into the high word, so the 64-bit total is exact whatever the
+// order (weights below 2^32 that do not wrap take a single atomic).
+__device__ __forceinline__ void smp_hist_add(unsigned long long *h, unsigned long long w) {
+  unsigned int *p = reinterpret_cast<unsigned int *>(h);   // p[0]: low word, p[1]: high word
+  const unsigned int lo = (unsigned int)w, hi = (unsigned int)(w >> 32);
+  const unsigned int old = atomicAdd(p, lo);
+  const unsigned int up = hi + ((old + lo < old) ? 1u : 0u);
+  if (up) atomicAdd(p + 1, up);
 }
 
 // After a histogram pass: finds the first bin (ascending index = descending
@@ -481,7 +492,7 @@ __global__ void __cluster_dims__(SMP_CLUSTER, 1, 1) __launch_bounds__(SMP_THREAD
     (void)i;
     const unsigned long long w = smp_weight(x, mx, inv_t_log2e);
     if (w) {
-      atomicAdd(&sh.hist[min(SMP_BINS - 1, (int)((mx - x) * scale_a))], w);
+      smp_hist_add(&sh.hist[min(SMP_BINS - 1, (int)((mx - x) * scale_a))], w);
       mysum += w;
     }
   })
