@@ -45,6 +45,7 @@ struct Program {
   float *qkv_out = nullptr, *o_out = nullptr, *gu_out = nullptr, *down_out = nullptr, *logits = nullptr, *ws = nullptr;
   bf16 *xn_hi = nullptr, *xn_lo = nullptr, *ao_hi = nullptr, *ao_lo = nullptr, *ff_hi = nullptr, *ff_lo = nullptr;
   int *row_token = nullptr, *row_pos = nullptr, *row_active = nullptr, *row_slot = nullptr, *do_sample = nullptr;
+  int *row_blocks = nullptr;   // decode program: which blocks of 64 rows hold a request this step (GemmPlan::row_blocks)
   int *sampled = nullptr, *att_work = nullptr, *att_n_work = nullptr, *att_pool = nullptr;
   GemmPlan p_qkv, p_o, p_gu, p_down, p_lm;
   // Mixture-of-Experts feed-forward layers: p_gu / p_down are then the GEMMs over all experts' gate / up rows
@@ -178,6 +179,7 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
   RC(dmalloc(A, &P.row_slot, R));
   RC(dmalloc(A, &P.do_sample, R));
   RC(dmalloc(A, &P.sampled, R));
+  RC(dmalloc(A, &P.row_blocks, 1));
   if (layers) {
     RC(dmalloc(A, &P.h, (size_t)R * H));
     if (!e->mla) {
@@ -440,7 +442,7 @@ int enqueue_decode_body(corun_engine *e, int *launches) {
   // mask and seeds are read from the pinned staging buffers by the first kernel, tokens and status are written to
   // them by the last one (zero-copy): a copy node in a graph costs several microseconds, these are 836 bytes
   CK(launch_prepare_rows(e->h_active, e->h_seeds, e->d_seeds, e->d_in_use, e->d_ctx, e->d_pending, e->B, P.row_token, P.row_pos, P.row_active,
-                         P.row_slot, P.do_sample, e->st));
+                         P.row_slot, P.do_sample, P.row_blocks, e->st));
   n += 1;
   RC(run_layers(e, P, &n));
   if (!(e->eager && e->stop_after >= 0)) {   // (debug) a truncated layer stack skips the tail too
@@ -772,6 +774,10 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
   // 128 rows and keeps the tensor pipe as busy as the weight stream); up to 64 rows every row through every expert
   const bool dec_grouped = e->moe_E > 0 && pad16(B) > 64 && !getenv("CORUN_MOE_DECODE_DENSE");
   if ((rc = program_create(e, e->dec, B, true, true, dec_grouped, true))) return fail(rc);
+  // the decode step's first kernel says which blocks of 64 rows hold a request; the GEMMs of 65..128 padded rows leave
+  // the others out (prefill chunks and the one-row program always fill their rows)
+  for (GemmPlan *pl : {&e->dec.p_qkv, &e->dec.p_o, &e->dec.p_gu, &e->dec.p_down, &e->dec.p_lm, &e->dec.p_gu_d, &e->dec.p_down_d})
+    pl->row_blocks = e->dec.row_blocks;
   if ((rc = program_create(e, e->pre, e->chunk, true, false, e->moe_E > 0 && !getenv("CORUN_MOE_PREFILL_DENSE")))) return fail(rc);
   if ((rc = program_create(e, e->lm1, 1, false, true))) return fail(rc);
 

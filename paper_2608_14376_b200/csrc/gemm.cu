@@ -50,14 +50,19 @@ constexpr uint32_t A_BLOCK_BYTES = GEMM_ROW_BLOCK * GEMM_BLOCK_K * 2;      // 16
 // Fb gate rows, then Fb up rows, Fb = N / (2 * keep_pitch)), a tile belongs to one block (keep_div tiles per block),
 // and the epilogue writes row_keep[r, e] * silu(gate) * up, exact zeros where row r did not select block e, to
 // columns e * Fb .. of the bf16 hi/lo output [BN, N / 2].
-template <bool MASKED, bool STACKED, bool GROUPED, bool SWIGLU>
+// NSB = 2 (with STACKED; 65..128 padded rows): TWO stacked blocks of 64 rows, each with its own 128-row A tile (hi rows
+// 0-63, lo rows 64-127) and its own accumulator.  *row_blocks (bit b: rows 64 b .. hold active rows; written by an
+// earlier kernel of the step, or null = both) says which blocks exist this step: an absent block is neither loaded
+// nor multiplied nor stored (its output rows keep what they held: nobody reads rows without a request).  A row's
+// value does not depend on which blocks exist.
+template <bool MASKED, bool STACKED, bool GROUPED, bool SWIGLU, int NSB = 1>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmHi,
                     const __grid_constant__ CUtensorMap tmLo, float *__restrict__ direct, float *__restrict__ ws,
                     const int *__restrict__ cta_start, int N, int KB, int BN, int R, int stages, int tmem_cols,
                     uint32_t idesc, const float *row_keep, int keep_pitch, int keep_div, const int *group_tab,
                     int tiles_per_group, int *status, unsigned long long *trace, __nv_bfloat16 *__restrict__ sw_hi,
-                    __nv_bfloat16 *__restrict__ sw_lo, int sw_half) {
+                    __nv_bfloat16 *__restrict__ sw_lo, int sw_half, const int *row_blocks) {
   extern __shared__ uint8_t smem_raw[];
   // optional per-CTA timeline (debug): 8 globaltimer stamps
 #define TRACE(i) do { if (trace) trace[(size_t)blockIdx.x * 8 + (i)] = globaltimer_ns(); } while (0)
@@ -103,13 +108,24 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
     return tile * sw_half;
   };
-  const uint32_t stage_bytes = w_tile_bytes + (stacked ? A_BLOCK_BYTES : 2 * x_bytes);
-  const uint32_t tx_bytes = w_tile_bytes + 2 * x_bytes;
-  const int n_rb = (BN + GEMM_ROW_BLOCK - 1) / GEMM_ROW_BLOCK;      // blocks of 128 activation rows
+  const uint32_t stage_bytes = w_tile_bytes + (stacked ? (uint32_t)NSB * A_BLOCK_BYTES : 2 * x_bytes);
+  uint32_t tx_bytes = w_tile_bytes + 2 * x_bytes;                   // (NSB = 2: set once the blocks are known)
+  const int n_rb = NSB == 2 ? 1 : (BN + GEMM_ROW_BLOCK - 1) / GEMM_ROW_BLOCK;   // blocks of 128 activation rows
   // up to 128 rows need 256 TMEM columns: two accumulator buffers fit, so the epilogue of one
-  // segment overlaps the MMAs of the next
-  const int n_acc = (n_rb == 1) ? 2 : 1;
+  // segment overlaps the MMAs of the next (NSB = 2: only while one block exists, see below)
+  int n_acc = (n_rb == 1) ? 2 : 1;
   const uint32_t acc_cols = (uint32_t)n_rb * GEMM_TILE_N;
+  // NSB = 2: which blocks exist (read behind the wait for the predecessor), and an accumulator's first column
+  int bmask = (1 << NSB) - 1;
+  auto read_blocks = [&]() {
+    if (NSB == 2) {
+      if (row_blocks) { griddep_wait(); bmask = *reinterpret_cast<const volatile int *>(row_blocks) & 3; }
+      if (bmask == 0) bmask = 1;                    // a step without requests: block 0 is computed and ignored
+      n_acc = bmask == 3 ? 1 : 2;
+      tx_bytes = w_tile_bytes + (uint32_t)__popc(bmask) * A_BLOCK_BYTES;
+    }
+  };
+  auto acc_col = [&](int acc, int b) { return NSB == 2 ? (uint32_t)(n_acc == 2 ? acc : b) * GEMM_TILE_N : (uint32_t)acc * acc_cols; };
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -165,7 +181,8 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const int g = k0 + it, tile = g / KB, kb = g - tile * KB;
         look(tile);
         const uint32_t fb = smem_u32(&full_bar[it]);
-        mbar_arrive_expect_tx(fb, tx_bytes);
+        if (NSB == 2) mbar_expect_tx(fb, w_tile_bytes);   // the activations' bytes and the arrival follow behind the wait
+        else mbar_arrive_expect_tx(fb, tx_bytes);
         if (SWIGLU) {
           tma_load_2d(tiles_base + (uint32_t)it * stage_bytes, &tmW, kb * GEMM_BLOCK_K, sw_gate_row(tile), fb, pol_w);
           tma_load_2d(tiles_base + (uint32_t)it * stage_bytes + w_tile_bytes / 2, &tmW, kb * GEMM_BLOCK_K,
@@ -176,13 +193,28 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         if (it == 0) TRACE(2);
       }
       griddep_wait();
+      read_blocks();
+      // the activation tiles of a stage (NSB = 2: a hi and a lo box of 64 rows per block that exists)
+      auto load_x = [&](uint32_t dst, int kb, uint32_t fb) {
+        if (NSB == 2) {
+#pragma unroll
+          for (int b = 0; b < 2; ++b)
+            if ((bmask >> b) & 1) {
+              tma_load_2d(dst + w_tile_bytes + (uint32_t)b * A_BLOCK_BYTES, &tmHi, kb * GEMM_BLOCK_K, 64 * b, fb, pol_x);
+              tma_load_2d(dst + w_tile_bytes + (uint32_t)b * A_BLOCK_BYTES + lo_off, &tmLo, kb * GEMM_BLOCK_K, 64 * b, fb, pol_x);
+            }
+        } else {
+          tma_load_2d(dst + w_tile_bytes, &tmHi, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
+          tma_load_2d(dst + w_tile_bytes + lo_off, &tmLo, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
+        }
+      };
       for (int it = 0; it < n_pre; ++it) {
         const int g = k0 + it, tile = g / KB, kb = g - tile * KB;
         look(tile);
         const uint32_t fb = smem_u32(&full_bar[it]);
         const uint32_t dst = tiles_base + (uint32_t)it * stage_bytes;
-        tma_load_2d(dst + w_tile_bytes, &tmHi, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
-        tma_load_2d(dst + w_tile_bytes + lo_off, &tmLo, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
+        if (NSB == 2) mbar_arrive_expect_tx(fb, tx_bytes - w_tile_bytes);
+        load_x(dst, kb, fb);
       }
       int it = n_pre;
       for (int g = k0 + n_pre; g < k1; ++g, ++it) {
@@ -200,14 +232,14 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         } else
         tma_load_2d(dst, &tmW, (GROUPED ? g_wk + kb : kb) * GEMM_BLOCK_K, GROUPED ? g_wrow + g_j * GEMM_TILE_N : tile * GEMM_TILE_N,
                     fb, pol_w);
-        tma_load_2d(dst + w_tile_bytes, &tmHi, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
-        tma_load_2d(dst + w_tile_bytes + lo_off, &tmLo, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
+        load_x(dst, kb, fb);
       }
       TRACE(3);
     }
   } else if (warp == 1) {
     if (lane == 0) {
       // ---------------- MMA issuer ----------------
+      read_blocks();
       int it = 0, seg = 0;
       for (int g = k0; g < k1 && !fail; ++seg) {
         const int tile = g / KB, kb_begin = g - tile * KB;
@@ -225,12 +257,16 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           const uint32_t w_addr = tiles_base + (uint32_t)s * stage_bytes;
           const uint64_t w_desc = umma_desc_sw128(w_addr);
           if (stacked) {
-            const uint64_t a_desc = umma_desc_sw128(w_addr + w_tile_bytes);
-            const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_cols;
 #pragma unroll
-            for (int k = 0; k < GEMM_BLOCK_K / 16; ++k) {
-              const uint64_t adv = (uint64_t)(k * 2);
-              umma_bf16(d_tmem, a_desc + adv, w_desc + adv, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
+            for (int b = 0; b < NSB; ++b) {
+              if (NSB == 2 && !((bmask >> b) & 1)) continue;
+              const uint64_t a_desc = umma_desc_sw128(w_addr + w_tile_bytes + (uint32_t)b * A_BLOCK_BYTES);
+              const uint32_t d_tmem = tmem_base + acc_col(acc, b);
+#pragma unroll
+              for (int k = 0; k < GEMM_BLOCK_K / 16; ++k) {
+                const uint64_t adv = (uint64_t)(k * 2);
+                umma_bf16(d_tmem, a_desc + adv, w_desc + adv, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
+              }
             }
           } else {
             for (int rb = 0; rb < n_rb; ++rb) {
@@ -257,6 +293,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   } else {
     // ---------------- epilogue: TMEM -> registers -> global ----------------
     const int lane_base = (warp & 3) * 32;          // the TMEM lanes this warp may read
+    read_blocks();
     int seg = 0;
     for (int g = k0; g < k1; ++seg) {
       const int tile = g / KB, kb_begin = g - tile * KB;
@@ -286,9 +323,12 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const int sw_rows = GROUPED ? g_rows : R, sw_row0 = GROUPED ? g_id * BN : 0;
         auto silu_mul = [](float gt, float up) { return __fdividef(gt, 1.f + __expf(-gt)) * up; };
         if (stacked) {
+         for (int b = 0; b < NSB; ++b) {                // the stacked blocks of 64 rows (one unless NSB = 2)
+          if (NSB == 2 && !((bmask >> b) & 1)) continue;
+          const int rb0 = 64 * b, rows_b = sw_rows - rb0;   // the block's first row, its rows in use
           const bool lo_warp = lane_base >= 64;
           const int row = (lane_base & 63) + lane;
-          const bool warp_needed = (lane_base & 63) < sw_rows;   // warp-uniform
+          const bool warp_needed = (lane_base & 63) < rows_b;   // warp-uniform
           float *xs = xch[lo_warp ? 1 : 0] + row * 33;
           const int te = (int)threadIdx.x - 64, srow = te >> 3, scol = (te & 7) * 4;
           for (int c0 = 0; c0 < HALF; c0 += 32) {
@@ -298,7 +338,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             for (int part = 0; part < 2; ++part) {     // 0: the gate columns, 1: the up columns
               if (warp_needed) {
                 uint32_t v[32];
-                const uint32_t ta = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)acc * acc_cols +
+                const uint32_t ta = tmem_base + ((uint32_t)lane_base << 16) + acc_col(acc, b) +
                                     (uint32_t)(part * HALF + c0);
                 tmem_ld16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
                 tmem_ld16(ta + 16, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
@@ -310,7 +350,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
                 const int r = i * 16 + srow;
-                if (r < sw_rows) {
+                if (r < rows_b) {
                   const float *h = xch[0] + r * 33 + scol, *l = xch[1] + r * 33 + scol;
                   const float s0 = h[0] + l[0], s1 = h[1] + l[1], s2 = h[2] + l[2], s3 = h[3] + l[3];
                   if (part == 0) {
@@ -319,25 +359,26 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                     float y[4] = {silu_mul(gt[i][0], s0), silu_mul(gt[i][1], s1), silu_mul(gt[i][2], s2),
                                   silu_mul(gt[i][3], s3)};
                     if (MASKED || GROUPED) {           // the row's routing weight for this expert; 0: not selected
-                      const float wgt = GROUPED ? row_keep[sw_row0 + r] : row_keep[(size_t)r * keep_pitch + blk];
+                      const float wgt = GROUPED ? row_keep[sw_row0 + r] : row_keep[(size_t)(rb0 + r) * keep_pitch + blk];
 #pragma unroll
                       for (int q = 0; q < 4; ++q) y[q] = wgt != 0.f ? wgt * y[q] : 0.f;
                     }
-                    __nv_bfloat16 a[4], b[4];
+                    __nv_bfloat16 a[4], b2[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                       a[q] = __float2bfloat16_rn(y[q]);
-                      b[q] = __float2bfloat16_rn(y[q] - __bfloat162float(a[q]));
+                      b2[q] = __float2bfloat16_rn(y[q] - __bfloat162float(a[q]));
                     }
-                    const size_t o = (size_t)(sw_row0 + r) * o_pitch + o_base + c0 + scol;
+                    const size_t o = (size_t)(sw_row0 + rb0 + r) * o_pitch + o_base + c0 + scol;
                     *reinterpret_cast<uint2 *>(sw_hi + o) = *reinterpret_cast<const uint2 *>(a);
-                    *reinterpret_cast<uint2 *>(sw_lo + o) = *reinterpret_cast<const uint2 *>(b);
+                    *reinterpret_cast<uint2 *>(sw_lo + o) = *reinterpret_cast<const uint2 *>(b2);
                   }
                 }
               }
               asm volatile("bar.sync 1, 128;" ::: "memory");
             }
           }
+         }
         } else {
           for (int rb = 0; rb < n_rb; ++rb) {
             const int row_base = rb * GEMM_ROW_BLOCK + lane_base;
@@ -369,30 +410,34 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         }
       } else
       if (stacked) {
+       for (int b = 0; b < NSB; ++b) {                  // the stacked blocks of 64 rows (one unless NSB = 2)
+        if (NSB == 2 && !((bmask >> b) & 1)) continue;
+        const int rb0 = 64 * b;                         // the block's first row
         // lanes 0-63 (warps with lane_base 0, 32) hold W*hi of rows 0-63, lanes 64-127 hold W*lo of the
         // same rows: every warp parks 32 columns of its rows in shared memory, then the 128 threads add
         // the two halves and store whole 128-byte row segments (four rows per warp instruction)
         const bool lo_warp = lane_base >= 64;
         const int row = (lane_base & 63) + lane;
-        const int rows_valid = GROUPED ? g_rows : (whole ? R : BN);
+        const int rows_valid = (GROUPED ? g_rows : (whole ? R : BN)) - rb0;
         const bool warp_needed = (lane_base & 63) < rows_valid;   // warp-uniform
         float *xs = xch[lo_warp ? 1 : 0] + row * 33;
         const int te = (int)threadIdx.x - 64, srow = te >> 3, scol = (te & 7) * 4;
-        float *dst0 = GROUPED ? direct + (size_t)g_id * BN * N + n0
-                              : (whole ? direct + n0 : ws + (size_t)(cta * 2 + (seg == 0 ? 0 : 1)) * BN * GEMM_TILE_N);
         const size_t pitch = whole ? (size_t)N : (size_t)GEMM_TILE_N;
+        float *dst0 = (GROUPED ? direct + (size_t)g_id * BN * N + n0
+                               : (whole ? direct + n0 : ws + (size_t)(cta * 2 + (seg == 0 ? 0 : 1)) * BN * GEMM_TILE_N)) +
+                      (size_t)rb0 * pitch;
         const bool vec_ok = whole ? ((N & 3) == 0) : true;
         bool row_on[4];                               // which of this thread's four rows are stored at all
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int r = i * 16 + srow;
-          row_on[i] = r < rows_valid && (!MASKED || r >= R || keep[(size_t)r * keep_pitch] != 0.f);
+          row_on[i] = r < rows_valid && (!MASKED || rb0 + r >= R || keep[(size_t)(rb0 + r) * keep_pitch] != 0.f);
         }
         for (int c0 = 0; c0 < GEMM_TILE_N; c0 += 32) {
           if (whole && n0 + c0 >= N) break;          // columns beyond the matrix (last tile); uniform
           if (warp_needed) {
             uint32_t v[32];
-            const uint32_t ta = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)acc * acc_cols + (uint32_t)c0;
+            const uint32_t ta = tmem_base + ((uint32_t)lane_base << 16) + acc_col(acc, b) + (uint32_t)c0;
             tmem_ld16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
             tmem_ld16(ta + 16, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
             tmem_ld_wait();
@@ -420,6 +465,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           }
           asm volatile("bar.sync 1, 128;" ::: "memory");
         }
+       }
       } else
       for (int rb = 0; rb < n_rb; ++rb) {
         const int row_base = rb * GEMM_ROW_BLOCK + lane_base;
@@ -534,6 +580,14 @@ int gemm_encode_map(CUtensorMap *m, const void *base, int rows, int K, int box_r
   return tma_encode_2d(m, base, 0, (unsigned long long)rows, K, box_rows, GEMM_BLOCK_K);
 }
 
+// Activation rows per TMA box and activation bytes per stage: up to 64 padded rows one stacked tile (hi rows 0..,
+// lo rows 64..), 65..128 rows two stacked tiles of 64 rows each (a box of 64 rows per half; the last box reaches
+// past the matrix when BN < 128: those rows arrive as zeros), above that the hi and the lo matrix whole.
+static int gemm_x_box_rows(int BN) { return BN <= 64 ? BN : BN <= 128 ? 64 : BN; }
+static size_t gemm_x_stage_bytes(int BN) {
+  return BN <= 64 ? (size_t)A_BLOCK_BYTES : BN <= 128 ? 2 * (size_t)A_BLOCK_BYTES : 2 * (size_t)BN * GEMM_BLOCK_K * 2;
+}
+
 int gemm_plan_fill(GemmPlan *p, const void *W, int N, int K, const void *Xhi, const void *Xlo, int R, int BN,
                    float *direct, float *ws, int num_sms, int *tab, int tab_cap, int *tab_ints) {
   if (N <= 0 || K <= 0 || K % GEMM_BLOCK_K || BN % 16 || BN < 16 || BN > 256 || R < 1 || R > BN) return CORUN_EINVAL;
@@ -549,7 +603,7 @@ int gemm_plan_fill(GemmPlan *p, const void *W, int N, int K, const void *Xhi, co
   const int per_tile = p->grid >= 2 * p->n_tiles ? p->grid / p->n_tiles : 0;
   if (per_tile) p->grid = per_tile * p->n_tiles;
   if (total * (long long)p->grid >= (1ll << 31)) return CORUN_EINVAL;
-  const size_t stage = (size_t)W_TILE_BYTES + (BN <= 64 ? (size_t)A_BLOCK_BYTES : 2 * (size_t)BN * GEMM_BLOCK_K * 2);
+  const size_t stage = (size_t)W_TILE_BYTES + gemm_x_stage_bytes(BN);
   // the MMA always reads 128 activation rows: leave that much readable behind the last stage
   int stages = (int)((GEMM_MAX_DYN_SMEM - 1024 - A_BLOCK_BYTES) / stage);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
@@ -565,8 +619,8 @@ int gemm_plan_fill(GemmPlan *p, const void *W, int N, int K, const void *Xhi, co
   p->ws = ws;
   int rc;
   if ((rc = gemm_encode_map(&p->tmW, W, N, K, GEMM_TILE_N)) != 0) return rc;
-  if ((rc = gemm_encode_map(&p->tmHi, Xhi, BN, K, BN)) != 0) return rc;
-  if ((rc = gemm_encode_map(&p->tmLo, Xlo, BN, K, BN)) != 0) return rc;
+  if ((rc = gemm_encode_map(&p->tmHi, Xhi, BN, K, gemm_x_box_rows(BN))) != 0) return rc;
+  if ((rc = gemm_encode_map(&p->tmLo, Xlo, BN, K, gemm_x_box_rows(BN))) != 0) return rc;
 
   const int n_ints = p->grid + 1 + 3 * p->n_tiles;
   if (n_ints > tab_cap) return CORUN_ELIMIT;
@@ -634,7 +688,7 @@ int gemm_plan_create_swiglu(GemmPlan *p, const void *W, int F, int K, const void
   p->KB = K / GEMM_BLOCK_K;
   p->grid = p->n_tiles < num_sms ? p->n_tiles : num_sms;
   if ((long long)p->n_tiles * p->KB >= (1ll << 31)) return CORUN_EINVAL;
-  const size_t stage = (size_t)2 * HALF * GEMM_BLOCK_K * 2 + (BN <= 64 ? (size_t)A_BLOCK_BYTES : 2 * (size_t)BN * GEMM_BLOCK_K * 2);
+  const size_t stage = (size_t)2 * HALF * GEMM_BLOCK_K * 2 + gemm_x_stage_bytes(BN);
   int stages = (int)((GEMM_MAX_DYN_SMEM - 1024 - A_BLOCK_BYTES) / stage);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) return CORUN_EINVAL;
@@ -649,8 +703,8 @@ int gemm_plan_create_swiglu(GemmPlan *p, const void *W, int F, int K, const void
   p->sw_lo = out_lo;
   int rc;
   if ((rc = gemm_encode_map(&p->tmW, W, 2 * F, K, HALF)) != 0) return rc;
-  if ((rc = gemm_encode_map(&p->tmHi, Xhi, BN, K, BN)) != 0) return rc;
-  if ((rc = gemm_encode_map(&p->tmLo, Xlo, BN, K, BN)) != 0) return rc;
+  if ((rc = gemm_encode_map(&p->tmHi, Xhi, BN, K, gemm_x_box_rows(BN))) != 0) return rc;
+  if ((rc = gemm_encode_map(&p->tmLo, Xlo, BN, K, gemm_x_box_rows(BN))) != 0) return rc;
   // whole tiles only: CTA c takes tiles [c * n_tiles / grid, (c + 1) * n_tiles / grid)
   std::vector<int> tab((size_t)p->grid + 1);
   for (int c = 0; c <= p->grid; ++c) tab[(size_t)c] = (int)((long long)c * p->n_tiles / p->grid) * p->KB;
@@ -694,7 +748,7 @@ int gemm_plan_create_swiglu_blocks(GemmPlan *p, const void *W, int n_blocks, int
   p->KB = K / GEMM_BLOCK_K;
   p->grid = p->n_tiles < num_sms ? p->n_tiles : num_sms;
   if ((long long)p->n_tiles * p->KB >= (1ll << 31)) return CORUN_EINVAL;
-  const size_t stage = (size_t)2 * HALF * GEMM_BLOCK_K * 2 + (BN <= 64 ? (size_t)A_BLOCK_BYTES : 2 * (size_t)BN * GEMM_BLOCK_K * 2);
+  const size_t stage = (size_t)2 * HALF * GEMM_BLOCK_K * 2 + gemm_x_stage_bytes(BN);
   int stages = (int)((GEMM_MAX_DYN_SMEM - 1024 - A_BLOCK_BYTES) / stage);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) return CORUN_EINVAL;
@@ -712,8 +766,8 @@ int gemm_plan_create_swiglu_blocks(GemmPlan *p, const void *W, int n_blocks, int
   p->keep_div = Fb / HALF;
   int rc;
   if ((rc = gemm_encode_map(&p->tmW, W, n_blocks * 2 * Fb, K, HALF)) != 0) return rc;
-  if ((rc = gemm_encode_map(&p->tmHi, Xhi, BN, K, BN)) != 0) return rc;
-  if ((rc = gemm_encode_map(&p->tmLo, Xlo, BN, K, BN)) != 0) return rc;
+  if ((rc = gemm_encode_map(&p->tmHi, Xhi, BN, K, gemm_x_box_rows(BN))) != 0) return rc;
+  if ((rc = gemm_encode_map(&p->tmLo, Xlo, BN, K, gemm_x_box_rows(BN))) != 0) return rc;
   // whole tiles only: CTA c takes tiles [c * n_tiles / grid, (c + 1) * n_tiles / grid)
   std::vector<int> tab((size_t)p->grid + 1);
   for (int c = 0; c <= p->grid; ++c) tab[(size_t)c] = (int)((long long)c * p->n_tiles / p->grid) * p->KB;
@@ -818,6 +872,10 @@ cudaError_t gemm_prepare_kernel() {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, false, false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, true, false, false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<false, true, false, true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_streamk_kernel<true, true, false, true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_MAX_DYN_SMEM);
   return e;
 }
 
@@ -833,8 +891,12 @@ cudaError_t gemm_launch(const GemmPlan &p, const CUtensorMap *tmW_override, int 
     return launch_k(kernel, dim3(p.grid), dim3(GEMM_THREADS), p.smem_bytes, st, pdl, tmW_override ? *tmW_override : p.tmW,
                     p.tmHi, p.tmLo, p.direct, p.ws, p.d_cta_start, p.N, p.KB, p.BN, p.R, p.stages, p.tmem_cols, p.idesc,
                     p.row_keep, p.keep_pitch, p.keep_div, p.group_tab, p.tiles_per_group, d_status, trace, p.sw_hi, p.sw_lo,
-                    p.sw_half);
+                    p.sw_half, p.row_blocks);
   };
+  if (!p.group_tab && p.BN > 64 && p.BN <= 128) {   // two stacked blocks of 64 rows
+    if (p.sw_hi) return masked ? go(gemm_streamk_kernel<true, true, false, true, 2>) : go(gemm_streamk_kernel<false, true, false, true, 2>);
+    return masked ? go(gemm_streamk_kernel<true, true, false, false, 2>) : go(gemm_streamk_kernel<false, true, false, false, 2>);
+  }
   if (p.group_tab && p.sw_hi) return go(gemm_streamk_kernel<false, true, true, true>);
   if (p.sw_hi && masked) return stacked ? go(gemm_streamk_kernel<true, true, false, true>) : go(gemm_streamk_kernel<true, false, false, true>);
   if (p.sw_hi) return stacked ? go(gemm_streamk_kernel<false, true, false, true>) : go(gemm_streamk_kernel<false, false, false, true>);

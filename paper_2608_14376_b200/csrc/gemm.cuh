@@ -95,6 +95,10 @@ struct GemmPlan {
   // Gate / up GEMM with SwiGLU in the epilogue (gemm_plan_create_swiglu): the bf16 hi/lo output [BN, N / 2].
   __nv_bfloat16 *sw_hi = nullptr, *sw_lo = nullptr;
   int sw_half = 0;                   // gate rows (= up rows) per tile
+  // 65..128 padded rows (two stacked blocks of 64 rows): device int, not owned, written by an earlier kernel of the
+  // step: bit b set = rows 64 b .. 64 b + 63 hold a request this step; null = both blocks.  An absent block is
+  // neither loaded nor multiplied nor stored.
+  const int *row_blocks = nullptr;
   GemmOut out() const { return GemmOut{direct, ws, d_tile_first, d_tile_cend, N, KB, BN}; }
 };
 

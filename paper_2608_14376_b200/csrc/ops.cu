@@ -741,12 +741,21 @@ __global__ void __cluster_dims__(SMP_CLUSTER, 1, 1) __launch_bounds__(SMP_THREAD
 __global__ void prepare_rows_kernel(const uint8_t *active_mask, const uint64_t *seeds_in, uint64_t *seeds_out,
                                     const int *in_use, const int *ctx_len,
                                     const int *pending, int B, int *row_token, int *row_pos, int *row_active,
-                                    int *row_slot, int *do_sample) {
+                                    int *row_slot, int *do_sample, int *row_blocks) {
   griddep_launch_dependents();
   griddep_wait();
   const int s = blockIdx.x * blockDim.x + threadIdx.x;
+  const int act = (s < B && active_mask[s] != 0 && in_use[s] != 0) ? 1 : 0;
+  // which blocks of 64 rows hold a request this step (up to 128 rows: one CTA of 128 threads sees them all): the
+  // GEMMs of 65..128 padded rows leave blocks without a request out
+  if (row_blocks && B <= 128) {
+    __shared__ int any[4];
+    const unsigned m = __ballot_sync(0xffffffffu, act != 0);
+    if ((threadIdx.x & 31) == 0) any[threadIdx.x >> 5] = m != 0u;
+    __syncthreads();
+    if (threadIdx.x == 0) *row_blocks = ((any[0] | any[1]) ? 1 : 0) | ((any[2] | any[3]) ? 2 : 0);
+  }
   if (s >= B) return;
-  const int act = (active_mask[s] != 0 && in_use[s] != 0) ? 1 : 0;
   seeds_out[s] = seeds_in[s];
   row_active[s] = act;
   row_slot[s] = s;
@@ -860,9 +869,9 @@ cudaError_t launch_sampler(const SampleArgs &a, int R, cudaStream_t st, bool pdl
 cudaError_t launch_prepare_rows(const uint8_t *active_mask, const uint64_t *seeds_in, uint64_t *seeds_out, const int *in_use,
                                 const int *ctx_len, const int *pending,
                                 int B, int *row_token, int *row_pos, int *row_active, int *row_slot, int *do_sample,
-                                cudaStream_t st) {
+                                int *row_blocks, cudaStream_t st) {
   prepare_rows_kernel<<<(B + 127) / 128, 128, 0, st>>>(active_mask, seeds_in, seeds_out, in_use, ctx_len, pending, B, row_token,
-                                                       row_pos, row_active, row_slot, do_sample);
+                                                       row_pos, row_active, row_slot, do_sample, row_blocks);
   return cudaGetLastError();
 }
 

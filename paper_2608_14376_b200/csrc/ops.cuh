@@ -97,7 +97,7 @@ cudaError_t launch_sampler(const SampleArgs &a, int R, cudaStream_t st, bool pdl
 cudaError_t launch_prepare_rows(const uint8_t *active_mask, const uint64_t *seeds_in, uint64_t *seeds_out, const int *in_use,
                                 const int *ctx_len, const int *pending,
                                 int B, int *row_token, int *row_pos, int *row_active, int *row_slot, int *do_sample,
-                                cudaStream_t st);
+                                int *row_blocks, cudaStream_t st);   // row_blocks: see GemmPlan::row_blocks (may be null)
 cudaError_t launch_advance(const int *row_active, const int *sampled, int B, int *ctx_len, int *step, int *pending,
                            int *out_tokens, const int *status_in, int *status_out, cudaStream_t st);
 // debug cache access (fp32 rows of n_kv*hd)
