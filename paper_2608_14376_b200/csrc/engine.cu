@@ -45,7 +45,11 @@ struct Program {
   float *qkv_out = nullptr, *o_out = nullptr, *gu_out = nullptr, *down_out = nullptr, *logits = nullptr, *ws = nullptr;
   bf16 *xn_hi = nullptr, *xn_lo = nullptr, *ao_hi = nullptr, *ao_lo = nullptr, *ff_hi = nullptr, *ff_lo = nullptr;
   int *row_token = nullptr, *row_pos = nullptr, *row_active = nullptr, *row_slot = nullptr, *do_sample = nullptr;
-  int *row_blocks = nullptr;   // decode program: which blocks of 64 rows hold a request this step (GemmPlan::row_blocks)
+  int *row_blocks = nullptr;   // decode program: which blocks of rows hold a request this step (GemmPlan::row_blocks)
+  // decode program: the step's rows are the slots with a request first (prepare_rows); the slot's row, and the
+  // slots' sampling state at the rows' places
+  int *slot_row = nullptr, *row_step = nullptr;
+  float *row_temp = nullptr, *row_top_p = nullptr;
   int *sampled = nullptr, *att_work = nullptr, *att_n_work = nullptr, *att_pool = nullptr;
   GemmPlan p_qkv, p_o, p_gu, p_down, p_lm;
   // Mixture-of-Experts feed-forward layers: p_gu / p_down are then the GEMMs over all experts' gate / up rows
@@ -110,6 +114,8 @@ struct corun_engine {
   // slot state: device
   int *d_in_use = nullptr, *d_ctx = nullptr, *d_step = nullptr, *d_pending = nullptr;
   float *d_temp = nullptr, *d_top_p = nullptr;
+  float *pf_logits = nullptr;            // [B, vocab]: a slot's logits after its prefill (the decode logits are by row)
+  std::vector<int> logits_row;           // per slot: its row of the last decode step it took part in, -1 = pf_logits
   uint64_t *d_seeds = nullptr;
   uint8_t *d_active = nullptr;
   int *d_out_tokens = nullptr, *d_status = nullptr;
@@ -180,6 +186,10 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
   RC(dmalloc(A, &P.do_sample, R));
   RC(dmalloc(A, &P.sampled, R));
   RC(dmalloc(A, &P.row_blocks, 1));
+  RC(dmalloc(A, &P.slot_row, R));
+  RC(dmalloc(A, &P.row_step, R));
+  RC(dmalloc(A, &P.row_temp, R));
+  RC(dmalloc(A, &P.row_top_p, R));
   if (layers) {
     RC(dmalloc(A, &P.h, (size_t)R * H));
     if (!e->mla) {
@@ -441,8 +451,9 @@ int enqueue_decode_body(corun_engine *e, int *launches) {
   int n = 0;
   // mask and seeds are read from the pinned staging buffers by the first kernel, tokens and status are written to
   // them by the last one (zero-copy): a copy node in a graph costs several microseconds, these are 836 bytes
-  CK(launch_prepare_rows(e->h_active, e->h_seeds, e->d_seeds, e->d_in_use, e->d_ctx, e->d_pending, e->B, P.row_token, P.row_pos, P.row_active,
-                         P.row_slot, P.do_sample, P.row_blocks, e->st));
+  CK(launch_prepare_rows(e->h_active, e->h_seeds, e->d_seeds, e->d_in_use, e->d_ctx, e->d_pending, e->d_temp, e->d_top_p, e->d_step, e->B,
+                         P.row_token, P.row_pos, P.row_active, P.row_slot, P.do_sample, P.row_temp, P.row_top_p, P.row_step, P.slot_row,
+                         P.row_blocks, e->st));
   n += 1;
   RC(run_layers(e, P, &n));
   if (!(e->eager && e->stop_after >= 0)) {   // (debug) a truncated layer stack skips the tail too
@@ -451,9 +462,10 @@ int enqueue_decode_body(corun_engine *e, int *launches) {
     CK(launch_resid_norm(P.h, s.hidden, nullptr, rows, &prev, e->final_norm, s.rms_eps, P.xn_hi, P.xn_lo, e->st));
     CK(gemm_launch(P.p_lm, nullptr, e->d_status, e->st, nullptr, true));
     CK(gemm_fixup_launch(P.p_lm, e->st, true));
-    SampleArgs sa{P.logits, s.vocab, P.do_sample, e->d_temp, e->d_top_p, e->d_seeds, e->d_step, nullptr, P.sampled};
+    SampleArgs sa{P.logits, s.vocab, P.do_sample, P.row_temp, P.row_top_p, e->d_seeds, P.row_step, nullptr, P.sampled};   // all by row
     CK(launch_sampler(sa, P.R, e->st, true));
-    CK(launch_advance(P.row_active, P.sampled, e->B, e->d_ctx, e->d_step, e->d_pending, e->h_out_tokens, e->d_status, e->h_status, e->st));
+    CK(launch_advance(P.slot_row, P.row_active, P.sampled, e->B, e->d_ctx, e->d_step, e->d_pending, e->h_out_tokens, e->d_status, e->h_status,
+                      e->st));
     n += 4 + (P.p_lm.n_split_tiles ? 1 : 0);
   }
   if (e->eager && e->stop_after >= 0)            // (debug) no last kernel ran: fetch the status word the plain way
@@ -731,8 +743,9 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
       (rc = dmalloc(A, &e->d_seeds, B)) || (rc = dmalloc(A, &e->d_active, B)) || (rc = dmalloc(A, &e->d_out_tokens, B)) ||
       (rc = dmalloc(A, &e->d_status, 1)) || (rc = dmalloc(A, &e->d_pf_temp, 1)) || (rc = dmalloc(A, &e->d_pf_top_p, 1)) ||
       (rc = dmalloc(A, &e->d_pf_seed, 1)) || (rc = dmalloc(A, &e->d_pf_step, 1)) || (rc = dmalloc(A, &e->d_pf_one, 1)) ||
-      (rc = dmalloc(A, &e->d_pf_tok, 1)))
+      (rc = dmalloc(A, &e->d_pf_tok, 1)) || (rc = dmalloc(A, &e->pf_logits, (size_t)B * s.vocab)))
     return fail(rc);
+  e->logits_row.assign((size_t)B, -1);
   {
     // cos/sin of pos * theta^(-2i/hd), evaluated in fp64 on the host (hd: the rotated width)
     const int rot = mla ? mla->qk_rope : s.head_dim, half = rot / 2;
@@ -849,7 +862,7 @@ struct PfReq {
 };
 
 // Final norm -> LM head (one row) -> sample with R(seed, 0) for the request whose last prompt token is row
-// `row` of the chunk that has just run; the logits go to the slot's row of the decode logits.
+// `row` of the chunk that has just run; the logits go to the slot's place among the prefill logits.
 int prefill_finish_row(corun_engine *e, int row, PfReq &r) {
   const corun_shape &s = e->sh;
   Program &P = e->pre, &L = e->lm1;
@@ -869,8 +882,9 @@ int prefill_finish_row(corun_engine *e, int row, PfReq &r) {
   SampleArgs sa{L.logits, s.vocab, e->d_pf_one, e->d_pf_temp, e->d_pf_top_p, e->d_pf_seed, e->d_pf_step, nullptr,
                 e->d_pf_tok};
   CK(launch_sampler(sa, 1, e->st));
-  CK(cudaMemcpyAsync(e->dec.logits + (size_t)r.slot * s.vocab, L.logits, (size_t)s.vocab * sizeof(float),
+  CK(cudaMemcpyAsync(e->pf_logits + (size_t)r.slot * s.vocab, L.logits, (size_t)s.vocab * sizeof(float),
                      cudaMemcpyDeviceToDevice, e->st));
+  e->logits_row[(size_t)r.slot] = -1;              // corun_get_logits: the prefill's logits until the slot decodes
   CK(cudaMemcpyAsync(&r.first, e->d_pf_tok, sizeof(int), cudaMemcpyDeviceToHost, e->st));
   CK(cudaStreamSynchronize(e->st));   // the one-row buffers and the sampling staging serve the next request
   return CORUN_OK;
@@ -1024,10 +1038,12 @@ int corun_decode_enqueue(corun_engine *e, const uint8_t *active, const uint64_t 
     CK(cudaGraphLaunch(e->graph_exec, e->st));
   }
   e->in_flight = true;
+  int row = 0;                                      // the step's rows: the slots with a request, ascending (prepare_rows)
   for (int s = 0; s < e->B; ++s)
     if (active[s]) {
       e->ctx[s] += 1;
       e->step[s] += 1;
+      e->logits_row[(size_t)s] = row++;
     }
   return CORUN_OK;
 }
@@ -1063,8 +1079,10 @@ int corun_get_logits(corun_engine *e, int32_t slot, float *out) {
   if (!e || !out) return CORUN_EINVAL;
   if (!slot_ok(e, slot) || !e->in_use[slot]) return CORUN_ESLOT;
   RC(sync_stream(e));
-  CK(cudaMemcpyAsync(out, e->dec.logits + (size_t)slot * e->sh.vocab, (size_t)e->sh.vocab * sizeof(float),
-                     cudaMemcpyDeviceToHost, e->st));
+  // the logits of the slot's newest token: its row of the last decode step it took part in, else its prefill's
+  const int row = e->logits_row[(size_t)slot];
+  const float *src = row < 0 ? e->pf_logits + (size_t)slot * e->sh.vocab : e->dec.logits + (size_t)row * e->sh.vocab;
+  CK(cudaMemcpyAsync(out, src, (size_t)e->sh.vocab * sizeof(float), cudaMemcpyDeviceToHost, e->st));
   CK(cudaStreamSynchronize(e->st));
   return CORUN_OK;
 }
@@ -1285,7 +1303,7 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
                               : launch_swiglu(P.p_gu.out(), P.R, s.ffn, P.ff_hi, P.ff_lo, e->st);
                 break;
         case 9: {
-          SampleArgs sa{P.logits, s.vocab, P.do_sample, e->d_temp, e->d_top_p, e->d_seeds, e->d_step, nullptr, P.sampled};
+          SampleArgs sa{P.logits, s.vocab, P.do_sample, P.row_temp, P.row_top_p, e->d_seeds, P.row_step, nullptr, P.sampled};
           ce = launch_sampler(sa, P.R, e->st);
           break;
         }

@@ -736,45 +736,61 @@ __global__ void __cluster_dims__(SMP_CLUSTER, 1, 1) __launch_bounds__(SMP_THREAD
 
 // ---------------------------------------------------------------- decode bookkeeping
 // active_mask / seeds_in are the step's inputs in PINNED HOST memory, read here through their device mapping:
-// 9 bytes per slot cross the bus inside this kernel instead of in two copy nodes in front of it; the seeds
-// go to seeds_out (device) for the sampler.
-__global__ void prepare_rows_kernel(const uint8_t *active_mask, const uint64_t *seeds_in, uint64_t *seeds_out,
-                                    const int *in_use, const int *ctx_len,
-                                    const int *pending, int B, int *row_token, int *row_pos, int *row_active,
-                                    int *row_slot, int *do_sample, int *row_blocks) {
+// 9 bytes per slot cross the bus inside this kernel instead of in two copy nodes in front of it.
+// The rows of the step are the slots in a new order: the slots with a request this step first (ascending slot), the
+// others behind them.  Which row a request lands in depends on its co-tenants; no value of the step depends on the
+// row (that is the invariance the whole path is built for), and with the requests in the first rows the GEMMs can
+// leave out whole blocks of rows that hold none (row_blocks: bit b = block b holds a request; blocks of 64 rows up
+// to 128 padded rows, of 128 rows above).  Per-slot sampling state is copied to the row's place.  One CTA.
+__global__ void __launch_bounds__(256) prepare_rows_kernel(const uint8_t *active_mask, const uint64_t *seeds_in, uint64_t *seeds_out,
+                                                           const int *in_use, const int *ctx_len, const int *pending,
+                                                           const float *temp, const float *top_p, const int *step, int B,
+                                                           int *row_token, int *row_pos, int *row_active, int *row_slot,
+                                                           int *do_sample, float *row_temp, float *row_top_p, int *row_step,
+                                                           int *slot_row, int *row_blocks) {
   griddep_launch_dependents();
   griddep_wait();
-  const int s = blockIdx.x * blockDim.x + threadIdx.x;
+  __shared__ int warp_cnt[8];
+  const int s = threadIdx.x, lane = s & 31, warp = s >> 5;
   const int act = (s < B && active_mask[s] != 0 && in_use[s] != 0) ? 1 : 0;
-  // which blocks of 64 rows hold a request this step (up to 128 rows: one CTA of 128 threads sees them all): the
-  // GEMMs of 65..128 padded rows leave blocks without a request out
-  if (row_blocks && B <= 128) {
-    __shared__ int any[4];
-    const unsigned m = __ballot_sync(0xffffffffu, act != 0);
-    if ((threadIdx.x & 31) == 0) any[threadIdx.x >> 5] = m != 0u;
-    __syncthreads();
-    if (threadIdx.x == 0) *row_blocks = ((any[0] | any[1]) ? 1 : 0) | ((any[2] | any[3]) ? 2 : 0);
+  const unsigned m = __ballot_sync(0xffffffffu, act != 0);
+  if (lane == 0) warp_cnt[warp] = __popc(m);
+  __syncthreads();
+  int before = __popc(m & ((1u << lane) - 1u)), n_act = 0;
+  for (int w = 0; w < 8; ++w) {
+    if (w < warp) before += warp_cnt[w];
+    n_act += warp_cnt[w];
+  }
+  if (s == 0 && row_blocks) {
+    const int blk = B <= 128 ? 64 : 128;
+    *row_blocks = (n_act > 0 ? 1 : 0) | (n_act > blk ? 2 : 0);
   }
   if (s >= B) return;
-  seeds_out[s] = seeds_in[s];
-  row_active[s] = act;
-  row_slot[s] = s;
-  row_pos[s] = act ? ctx_len[s] : 0;
-  row_token[s] = act ? pending[s] : 0;
-  do_sample[s] = act;
+  const int r = act ? before : n_act + (s - before);   // requests first, in slot order; then the other slots
+  slot_row[s] = r;
+  row_slot[r] = s;
+  row_active[r] = act;
+  row_pos[r] = act ? ctx_len[s] : 0;
+  row_token[r] = act ? pending[s] : 0;
+  do_sample[r] = act;
+  seeds_out[r] = seeds_in[s];
+  row_temp[r] = temp[s];
+  row_top_p[r] = top_p[s];
+  row_step[r] = step[s];
 }
 
 // out_tokens / status_out are PINNED HOST memory written through their device mapping (the step's results: 4
 // bytes per slot and the status word), fenced system-wide; the host reads them after synchronising the stream.
-__global__ void advance_kernel(const int *row_active, const int *sampled, int B, int *ctx_len, int *step, int *pending,
-                               int *out_tokens, const int *status_in, int *status_out) {
+__global__ void advance_kernel(const int *slot_row, const int *row_active, const int *sampled, int B, int *ctx_len, int *step,
+                               int *pending, int *out_tokens, const int *status_in, int *status_out) {
   griddep_launch_dependents();
   griddep_wait();
   const int s = blockIdx.x * blockDim.x + threadIdx.x;
   if (s == 0) *status_out = *status_in;
   if (s >= B) { __threadfence_system(); return; }
-  if (row_active[s]) {
-    const int tok = sampled[s];
+  const int r = slot_row[s];
+  if (row_active[r]) {
+    const int tok = sampled[r];
     pending[s] = tok;
     ctx_len[s] += 1;
     step[s] += 1;
@@ -867,18 +883,21 @@ cudaError_t launch_sampler(const SampleArgs &a, int R, cudaStream_t st, bool pdl
 }
 
 cudaError_t launch_prepare_rows(const uint8_t *active_mask, const uint64_t *seeds_in, uint64_t *seeds_out, const int *in_use,
-                                const int *ctx_len, const int *pending,
+                                const int *ctx_len, const int *pending, const float *temp, const float *top_p, const int *step,
                                 int B, int *row_token, int *row_pos, int *row_active, int *row_slot, int *do_sample,
-                                int *row_blocks, cudaStream_t st) {
-  prepare_rows_kernel<<<(B + 127) / 128, 128, 0, st>>>(active_mask, seeds_in, seeds_out, in_use, ctx_len, pending, B, row_token,
-                                                       row_pos, row_active, row_slot, do_sample, row_blocks);
+                                float *row_temp, float *row_top_p, int *row_step, int *slot_row, int *row_blocks,
+                                cudaStream_t st) {
+  if (B > 256) return cudaErrorInvalidValue;
+  prepare_rows_kernel<<<1, 256, 0, st>>>(active_mask, seeds_in, seeds_out, in_use, ctx_len, pending, temp, top_p, step, B,
+                                         row_token, row_pos, row_active, row_slot, do_sample, row_temp, row_top_p, row_step,
+                                         slot_row, row_blocks);
   return cudaGetLastError();
 }
 
-cudaError_t launch_advance(const int *row_active, const int *sampled, int B, int *ctx_len, int *step, int *pending,
-                           int *out_tokens, const int *status_in, int *status_out, cudaStream_t st) {
-  return launch_k(advance_kernel, dim3((B + 127) / 128), dim3(128), 0, st, true, row_active, sampled, B, ctx_len, step,
-                  pending, out_tokens, status_in, status_out);
+cudaError_t launch_advance(const int *slot_row, const int *row_active, const int *sampled, int B, int *ctx_len, int *step,
+                           int *pending, int *out_tokens, const int *status_in, int *status_out, cudaStream_t st) {
+  return launch_k(advance_kernel, dim3((B + 127) / 128), dim3(128), 0, st, true, slot_row, row_active, sampled, B, ctx_len,
+                  step, pending, out_tokens, status_in, status_out);
 }
 
 cudaError_t launch_kv_copy(const KvLayout &kv, int layer, int slot, int pos0, int n, float *k, float *v, int write,

@@ -95,11 +95,12 @@ cudaError_t launch_sampler(const SampleArgs &a, int R, cudaStream_t st, bool pdl
 // The step's inputs (active mask, seeds) and results (tokens, status word) live in pinned host memory and are
 // read / written by these two kernels through its device mapping: no copy nodes around the step.
 cudaError_t launch_prepare_rows(const uint8_t *active_mask, const uint64_t *seeds_in, uint64_t *seeds_out, const int *in_use,
-                                const int *ctx_len, const int *pending,
+                                const int *ctx_len, const int *pending, const float *temp, const float *top_p, const int *step,
                                 int B, int *row_token, int *row_pos, int *row_active, int *row_slot, int *do_sample,
-                                int *row_blocks, cudaStream_t st);   // row_blocks: see GemmPlan::row_blocks (may be null)
-cudaError_t launch_advance(const int *row_active, const int *sampled, int B, int *ctx_len, int *step, int *pending,
-                           int *out_tokens, const int *status_in, int *status_out, cudaStream_t st);
+                                float *row_temp, float *row_top_p, int *row_step, int *slot_row, int *row_blocks,
+                                cudaStream_t st);   // rows = the slots with a request first; row_blocks: see GemmPlan::row_blocks
+cudaError_t launch_advance(const int *slot_row, const int *row_active, const int *sampled, int B, int *ctx_len, int *step,
+                           int *pending, int *out_tokens, const int *status_in, int *status_out, cudaStream_t st);
 // debug cache access (fp32 rows of n_kv*hd)
 cudaError_t launch_kv_copy(const KvLayout &kv, int layer, int slot, int pos0, int n, float *k, float *v, int write,
                            cudaStream_t st);
