@@ -96,7 +96,9 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   // Up to 64 rows: hi and lo share one 128-row A tile (hi in rows 0.., lo in rows 64..), so one MMA
   // per k-slice yields W*hi in accumulator lanes 0-63 and W*lo in lanes 64-127; the epilogue adds them.
   constexpr bool stacked = STACKED;                 // = (BN <= 64), fixed at compile time
-  const uint32_t lo_off = stacked ? (uint32_t)(64 * GEMM_BLOCK_K * 2) : x_bytes;
+  // not stacked, two row blocks: the hi tiles of both blocks (128 rows each, whatever BN is), then the lo tiles
+  const uint32_t x_reg = (!stacked && BN > GEMM_ROW_BLOCK) ? 2u * A_BLOCK_BYTES : x_bytes;
+  const uint32_t lo_off = stacked ? (uint32_t)(64 * GEMM_BLOCK_K * 2) : x_reg;
   const uint32_t w_tile_bytes = SWIGLU ? (uint32_t)(2 * sw_half * GEMM_BLOCK_K * 2) : W_TILE_BYTES;
   // SWIGLU: first gate row of a tile, and the distance to the up rows of the same outputs
   const int sw_fb = (SWIGLU && MASKED) ? N / (2 * keep_pitch) : N / 2;
@@ -108,7 +110,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
     return tile * sw_half;
   };
-  const uint32_t stage_bytes = w_tile_bytes + (stacked ? (uint32_t)NSB * A_BLOCK_BYTES : 2 * x_bytes);
+  const uint32_t stage_bytes = w_tile_bytes + (stacked ? (uint32_t)NSB * A_BLOCK_BYTES : 2 * x_reg);
   uint32_t tx_bytes = w_tile_bytes + 2 * x_bytes;                   // (NSB = 2: set once the blocks are known)
   const int n_rb = NSB == 2 ? 1 : (BN + GEMM_ROW_BLOCK - 1) / GEMM_ROW_BLOCK;   // blocks of 128 activation rows
   // up to 128 rows need 256 TMEM columns: two accumulator buffers fit, so the epilogue of one
@@ -116,16 +118,22 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   int n_acc = (n_rb == 1) ? 2 : 1;
   const uint32_t acc_cols = (uint32_t)n_rb * GEMM_TILE_N;
   // NSB = 2: which blocks exist (read behind the wait for the predecessor), and an accumulator's first column
-  int bmask = (1 << NSB) - 1;
+  // Not STACKED (above 128 padded rows): the blocks are the row blocks of 128 rows (hi and lo boxes of 128 rows each),
+  // left out in the same way; with one block left its two accumulator buffers alternate as for up to 128 rows.
+  constexpr bool DYN_BLOCKS = NSB == 2 || (!STACKED && !GROUPED);
+  int bmask = NSB == 2 ? 3 : (1 << n_rb) - 1;
   auto read_blocks = [&]() {
-    if (NSB == 2) {
-      if (row_blocks) { griddep_wait(); bmask = *reinterpret_cast<const volatile int *>(row_blocks) & 3; }
+    if (DYN_BLOCKS) {
+      const int all = NSB == 2 ? 3 : (1 << n_rb) - 1;
+      if (row_blocks) { griddep_wait(); bmask = *reinterpret_cast<const volatile int *>(row_blocks) & all; }
       if (bmask == 0) bmask = 1;                    // a step without requests: block 0 is computed and ignored
       n_acc = bmask == 3 ? 1 : 2;
-      tx_bytes = w_tile_bytes + (uint32_t)__popc(bmask) * A_BLOCK_BYTES;
+      tx_bytes = w_tile_bytes + (uint32_t)__popc(bmask) * (NSB == 2 ? A_BLOCK_BYTES : 2 * (n_rb == 1 ? x_bytes : A_BLOCK_BYTES));
     }
   };
-  auto acc_col = [&](int acc, int b) { return NSB == 2 ? (uint32_t)(n_acc == 2 ? acc : b) * GEMM_TILE_N : (uint32_t)acc * acc_cols; };
+  auto acc_col = [&](int acc, int b) {
+    return DYN_BLOCKS ? (uint32_t)(n_acc == 2 ? acc : b) * GEMM_TILE_N : (uint32_t)acc * acc_cols + (STACKED ? 0u : (uint32_t)b * GEMM_TILE_N);
+  };
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -181,7 +189,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const int g = k0 + it, tile = g / KB, kb = g - tile * KB;
         look(tile);
         const uint32_t fb = smem_u32(&full_bar[it]);
-        if (NSB == 2) mbar_expect_tx(fb, w_tile_bytes);   // the activations' bytes and the arrival follow behind the wait
+        if (DYN_BLOCKS) mbar_expect_tx(fb, w_tile_bytes);   // the activations' bytes and the arrival follow behind the wait
         else mbar_arrive_expect_tx(fb, tx_bytes);
         if (SWIGLU) {
           tma_load_2d(tiles_base + (uint32_t)it * stage_bytes, &tmW, kb * GEMM_BLOCK_K, sw_gate_row(tile), fb, pol_w);
@@ -203,6 +211,13 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
               tma_load_2d(dst + w_tile_bytes + (uint32_t)b * A_BLOCK_BYTES, &tmHi, kb * GEMM_BLOCK_K, 64 * b, fb, pol_x);
               tma_load_2d(dst + w_tile_bytes + (uint32_t)b * A_BLOCK_BYTES + lo_off, &tmLo, kb * GEMM_BLOCK_K, 64 * b, fb, pol_x);
             }
+        } else if (DYN_BLOCKS && n_rb == 2) {
+#pragma unroll
+          for (int b = 0; b < 2; ++b)
+            if ((bmask >> b) & 1) {
+              tma_load_2d(dst + w_tile_bytes + (uint32_t)b * A_BLOCK_BYTES, &tmHi, kb * GEMM_BLOCK_K, GEMM_ROW_BLOCK * b, fb, pol_x);
+              tma_load_2d(dst + w_tile_bytes + lo_off + (uint32_t)b * A_BLOCK_BYTES, &tmLo, kb * GEMM_BLOCK_K, GEMM_ROW_BLOCK * b, fb, pol_x);
+            }
         } else {
           tma_load_2d(dst + w_tile_bytes, &tmHi, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
           tma_load_2d(dst + w_tile_bytes + lo_off, &tmLo, kb * GEMM_BLOCK_K, GROUPED ? g_id * BN : 0, fb, pol_x);
@@ -213,7 +228,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         look(tile);
         const uint32_t fb = smem_u32(&full_bar[it]);
         const uint32_t dst = tiles_base + (uint32_t)it * stage_bytes;
-        if (NSB == 2) mbar_arrive_expect_tx(fb, tx_bytes - w_tile_bytes);
+        if (DYN_BLOCKS) mbar_arrive_expect_tx(fb, tx_bytes - w_tile_bytes);
         load_x(dst, kb, fb);
       }
       int it = n_pre;
@@ -270,9 +285,10 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             }
           } else {
             for (int rb = 0; rb < n_rb; ++rb) {
+              if (DYN_BLOCKS && !((bmask >> rb) & 1)) continue;
               const uint64_t hi_desc = umma_desc_sw128(w_addr + w_tile_bytes + (uint32_t)rb * A_BLOCK_BYTES);
-              const uint64_t lo_desc = umma_desc_sw128(w_addr + w_tile_bytes + x_bytes + (uint32_t)rb * A_BLOCK_BYTES);
-              const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_cols + (uint32_t)rb * GEMM_TILE_N;
+              const uint64_t lo_desc = umma_desc_sw128(w_addr + w_tile_bytes + lo_off + (uint32_t)rb * A_BLOCK_BYTES);
+              const uint32_t d_tmem = tmem_base + acc_col(acc, rb);
 #pragma unroll
               for (int k = 0; k < GEMM_BLOCK_K / 16; ++k) {
                 // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in 16-byte units
@@ -381,14 +397,14 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
          }
         } else {
           for (int rb = 0; rb < n_rb; ++rb) {
+            if (DYN_BLOCKS && !((bmask >> rb) & 1)) continue;
             const int row_base = rb * GEMM_ROW_BLOCK + lane_base;
             if (row_base >= R) continue;                 // warp-uniform
             const int row = row_base + lane;
             for (int c0 = 0; c0 < HALF; c0 += 8) {
               if (f0 + c0 >= F) break;                   // F % 8 == 0
               uint32_t vg[8], vu[8];
-              const uint32_t ta = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)acc * acc_cols +
-                                  (uint32_t)(rb * GEMM_TILE_N + c0);
+              const uint32_t ta = tmem_base + ((uint32_t)lane_base << 16) + acc_col(acc, rb) + (uint32_t)c0;
               tmem_ld8(ta, vg);
               tmem_ld8(ta + HALF, vu);
               tmem_ld_wait();
@@ -468,6 +484,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
        }
       } else
       for (int rb = 0; rb < n_rb; ++rb) {
+        if (DYN_BLOCKS && !((bmask >> rb) & 1)) continue;
         const int row_base = rb * GEMM_ROW_BLOCK + lane_base;
         const int rows_valid = whole ? R : BN;      // partials keep the padded row count
         if (row_base >= rows_valid) continue;        // warp-uniform: nothing of this warp's lanes is needed
@@ -479,7 +496,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         for (int c0 = 0; c0 < GEMM_TILE_N; c0 += 16) {
           if (whole && n0 + c0 >= N) break;          // columns beyond the matrix (last tile)
           uint32_t v[16];
-          tmem_ld16(tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)acc * acc_cols + (uint32_t)(rb * GEMM_TILE_N + c0), v);
+          tmem_ld16(tmem_base + ((uint32_t)lane_base << 16) + acc_col(acc, rb) + (uint32_t)c0, v);
           tmem_ld_wait();
           if (!row_ok) continue;
           if (vec_ok && (!whole || n0 + c0 + 16 <= N)) {
@@ -582,10 +599,10 @@ int gemm_encode_map(CUtensorMap *m, const void *base, int rows, int K, int box_r
 
 // Activation rows per TMA box and activation bytes per stage: up to 64 padded rows one stacked tile (hi rows 0..,
 // lo rows 64..), 65..128 rows two stacked tiles of 64 rows each (a box of 64 rows per half; the last box reaches
-// past the matrix when BN < 128: those rows arrive as zeros), above that the hi and the lo matrix whole.
-static int gemm_x_box_rows(int BN) { return BN <= 64 ? BN : BN <= 128 ? 64 : BN; }
+// past the matrix when BN < 128: those rows arrive as zeros), above that a hi and a lo box of 128 rows per row block.
+static int gemm_x_box_rows(int BN) { return BN <= 64 ? BN : BN <= 128 ? 64 : GEMM_ROW_BLOCK; }
 static size_t gemm_x_stage_bytes(int BN) {
-  return BN <= 64 ? (size_t)A_BLOCK_BYTES : BN <= 128 ? 2 * (size_t)A_BLOCK_BYTES : 2 * (size_t)BN * GEMM_BLOCK_K * 2;
+  return BN <= 64 ? (size_t)A_BLOCK_BYTES : BN <= 128 ? 2 * (size_t)A_BLOCK_BYTES : 4 * (size_t)A_BLOCK_BYTES;
 }
 
 int gemm_plan_fill(GemmPlan *p, const void *W, int N, int K, const void *Xhi, const void *Xlo, int R, int BN,
