@@ -1,6 +1,7 @@
 // Launchers of the non-GEMM kernels of the decode / prefill row program.
-// A "row" is one query token: in decode row r is slot r, in prefill the rows
-// are consecutive prompt positions of one slot.
+// A "row" is one query token: in decode the rows are the slots in the order prepare_rows gives them (the slots
+// with a request this step first; Rows::slot names a row's slot), in prefill the rows are consecutive prompt
+// positions of one slot.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
