@@ -788,10 +788,13 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
   const bool dec_grouped = e->moe_E > 0 && pad16(B) > 64 && !getenv("CORUN_MOE_DECODE_DENSE");
   if ((rc = program_create(e, e->dec, B, true, true, dec_grouped, true))) return fail(rc);
   // the decode step's first kernel says which blocks of 64 rows hold a request; the GEMMs of 65..128 padded rows leave
-  // the others out (prefill chunks and the one-row program always fill their rows)
+  // the others out (the one-row program has one block)
   for (GemmPlan *pl : {&e->dec.p_qkv, &e->dec.p_o, &e->dec.p_gu, &e->dec.p_down, &e->dec.p_lm, &e->dec.p_gu_d, &e->dec.p_down_d})
     pl->row_blocks = e->dec.row_blocks;
   if ((rc = program_create(e, e->pre, e->chunk, true, false, e->moe_E > 0 && !getenv("CORUN_MOE_PREFILL_DENSE")))) return fail(rc);
+  // a prefill chunk is filled from row 0: the host says which blocks of rows it reaches (prefill_run)
+  for (GemmPlan *pl : {&e->pre.p_qkv, &e->pre.p_o, &e->pre.p_gu, &e->pre.p_down, &e->pre.p_gu_d, &e->pre.p_down_d})
+    pl->row_blocks = e->pre.row_blocks;
   if ((rc = program_create(e, e->lm1, 1, false, true))) return fail(rc);
 
   // the allocations above were cleared and filled through the legacy stream, which the engine's
@@ -923,7 +926,7 @@ int prefill_run(corun_engine *e, PfReq *reqs, int n_req) {
   int unit = 128 / (s.n_q_heads / s.n_kv_heads);    // tokens per attention tile
   if (e->mla) unit = 16;                            // no query tiles there: every row is on its own
   if (unit > CH || CH % unit) unit = CH;
-  int *tok = e->h_rows, *pos = tok + CH, *act = pos + CH, *slt = act + CH;
+  int *tok = e->h_rows, *pos = tok + CH, *act = pos + CH, *slt = act + CH, *blocks = slt + CH;
   std::vector<std::pair<int, int>> fins;           // (request, chunk row of its last prompt token)
   int fill = 0, pad_slot = reqs[0].slot;
   auto run_chunk = [&]() -> int {
@@ -932,6 +935,11 @@ int prefill_run(corun_engine *e, PfReq *reqs, int n_req) {
     CK(cudaMemcpyAsync(P.row_pos, pos, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
     CK(cudaMemcpyAsync(P.row_active, act, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
     CK(cudaMemcpyAsync(P.row_slot, slt, CH * sizeof(int), cudaMemcpyHostToDevice, e->st));
+    // the chunk's rows are filled from row 0: the GEMMs leave out the blocks of rows behind the last one in use
+    // (blocks of 64 rows up to 128 padded rows, of 128 rows above)
+    const int blk = P.BN <= 128 ? 64 : 128;
+    blocks[0] = (fill > 0 ? 1 : 0) | (fill > blk ? 2 : 0);
+    CK(cudaMemcpyAsync(P.row_blocks, blocks, sizeof(int), cudaMemcpyHostToDevice, e->st));
     RC(run_layers(e, P, nullptr));
     for (auto &f : fins) RC(prefill_finish_row(e, f.second, reqs[f.first]));
     CK(cudaStreamSynchronize(e->st));   // the staging arrays are reused by the next chunk
