@@ -225,7 +225,9 @@ void corun_destroy(corun_engine *e);
 
 /* ---- accessors used by tests and reports ---- */
 
-/* Logits row (vocab floats, host) of the slot's latest forward pass. */
+/* Logits row (vocab floats, host) of the slot's latest forward pass: its prefill's until the slot takes part in a
+ * decode step (other slots' steps in between leave them alone), then those of the last decode step it took part in,
+ * readable until the next decode step (whose rows overwrite them). */
 int corun_get_logits(corun_engine *e, int32_t slot, float *out);
 /* Replaces the slot's pending token (teacher forcing). */
 int corun_force_token(corun_engine *e, int32_t slot, int32_t token);

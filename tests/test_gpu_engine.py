@@ -171,6 +171,35 @@ def test_padding_rows_change_nothing_and_report_minus_one(tiny, engine):
     np.testing.assert_array_equal(k0, k1)
 
 
+def test_a_slots_logits_follow_the_slot_whatever_row_it_takes(tiny, engine):
+    """The rows of a decode step are the slots with a request first, so a slot's row changes with its co-tenants:
+    the logits of a slot are its prefill's until it decodes (other slots' steps in between do not touch them), then
+    those of its own row of the last step it took part in."""
+    prompts = synth.make_prompts(tiny.sh.vocab, [20, 33, 27], seed=43)
+    engine.prefill(6, prompts[0], 60)
+    after_prefill = engine.logits(6).tobytes()
+    engine.prefill(2, prompts[1], 60)
+    engine.prefill(0, prompts[2], 60)
+    seeds = np.zeros(B, np.uint64)
+    only = np.zeros(B, np.uint8); only[[0, 2]] = 1          # slot 6 occupied, not active: rows 0 and 1 are slots 0 and 2
+    engine.decode_step(only, seeds)
+    engine.decode_step(only, seeds)
+    assert engine.logits(6).tobytes() == after_prefill
+    a = np.zeros(B, np.uint8); a[6] = 1                       # alone: slot 6 is row 0
+    engine.decode_step(a, seeds)
+    alone = engine.logits(6).tobytes()
+    assert alone != after_prefill
+    # the same step of the same request behind two co-tenants (row 2), on a fresh engine state
+    engine.release(6); engine.release(2); engine.release(0)
+    engine.prefill(6, prompts[0], 60)
+    engine.prefill(2, prompts[1], 60)
+    engine.prefill(0, prompts[2], 60)
+    both = np.zeros(B, np.uint8); both[[0, 2, 6]] = 1
+    out = engine.decode_step(both, seeds)
+    assert engine.logits(6).tobytes() == alone
+    assert all(out[s] >= 0 for s in (0, 2, 6)) and all(out[s] == -1 for s in range(B) if s not in (0, 2, 6))
+
+
 def test_error_paths(tiny, engine):
     from paper_2608_14376_b200 import corun
 

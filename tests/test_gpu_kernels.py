@@ -28,9 +28,11 @@ def _gemm_case(orc, torch, R, N, K, seed):
     return out, ref, Wt, Xt
 
 
-# rows x weight rows x K: single tile, ragged N, several tiles, more k-blocks than CTAs, all 256 rows
+# rows x weight rows x K: single tile, ragged N, several tiles, more k-blocks than CTAs, all 256 rows; 65..128 rows
+# (two stacked blocks of 64 rows, the second one ragged or full), 129..256 rows (two row blocks of 128)
 @pytest.mark.parametrize("R,N,K", [(8, 128, 64), (8, 512, 256), (5, 384, 768), (1, 2048, 256), (40, 200, 128),
-                                   (64, 1536, 256), (64, 4096, 4096), (130, 1024, 1024), (256, 512, 512)])
+                                   (64, 1536, 256), (64, 4096, 4096), (130, 1024, 1024), (256, 512, 512),
+                                   (72, 640, 512), (100, 1024, 1024), (128, 4096, 2048), (200, 768, 1024)])
 def test_gemm_matches_oracle(orc, torch_cuda, R, N, K):
     out, ref, _, _ = _gemm_case(orc, torch_cuda, R, N, K, seed=R + N + K)
     # split activations carry 16 significand bits: error << 1e-4 of the output scale (0.02 * sqrt(K))
@@ -53,6 +55,26 @@ def test_gemm_rows_are_position_invariant(orc, torch_cuda):
     np.testing.assert_array_equal(out_y[0], out[0])
     # repeated runs
     np.testing.assert_array_equal(corun.debug_gemm(Wt, Xt).cpu().numpy(), out)
+
+
+@pytest.mark.parametrize("R", [100, 128, 200])
+def test_gemm_rows_are_position_invariant_across_row_blocks(orc, torch_cuda, R):
+    """Above 64 rows the rows sit in two blocks with an accumulator each: a row's bytes do not depend on the block
+    it is in, nor on what the other block holds."""
+    from paper_2608_14376_b200 import corun
+
+    torch = torch_cuda
+    out, _, Wt, Xt = _gemm_case(orc, torch, R, 1024, 2048, seed=5 + R)
+    perm = torch.randperm(R, generator=torch.Generator().manual_seed(2)).cuda()
+    out_p = corun.debug_gemm(Wt, Xt[perm].contiguous()).cpu().numpy()
+    np.testing.assert_array_equal(out_p, out[perm.cpu().numpy()])
+    Y = Xt.clone()
+    Y[1:] = 1e30
+    np.testing.assert_array_equal(corun.debug_gemm(Wt, Y).cpu().numpy()[0], out[0])
+    # the same rows alone in a smaller matrix of the same row path (R rows -> the first 70 rows of an R-row call)
+    Z = torch.zeros_like(Xt)
+    Z[:70] = Xt[R - 70:]
+    np.testing.assert_array_equal(corun.debug_gemm(Wt, Z).cpu().numpy()[:70], out[R - 70:])
 
 
 def test_variate_matches_oracle(orc, torch_cuda):
