@@ -245,9 +245,9 @@ int program_create(corun_engine *e, Program &P, int R, bool layers, bool lm, boo
     // the plans carry layer 0's weights; the per-layer tensor maps override them at launch
     RC(gemm_plan_create(&P.p_qkv, e->w0_qkv, QKVN, H, P.xn_hi, P.xn_lo, R, P.BN, P.qkv_out, P.ws, e->num_sms));
     RC(gemm_plan_create(&P.p_o, e->w0_o, H, QD, P.ao_hi, P.ao_lo, R, P.BN, P.o_out, P.ws, e->num_sms));
-    // expert layers: the routing weight and the SwiGLU in the epilogue of the GEMM over all experts' gate / up rows
-    // (65..128 rows; up to 64 rows the masked store plus a SwiGLU kernel measured faster: the epilogue would write
-    // zeros for every pair that was not selected through the shared-memory exchange of the stacked path)
+    // expert layers without groups: the routing weight and the SwiGLU in the epilogue of the GEMM over all experts'
+    // gate / up rows (65..128 rows, where the grouped form below does not apply; up to 64 rows the masked store plus a
+    // SwiGLU kernel measured faster: the epilogue would write zeros for every pair that was not selected)
     const bool moe_fused = fuse_swiglu && e->moe_E && P.BN > 64 && P.BN <= 128 &&
                            gemm_swiglu_blocks_half(e->moe_F, e->moe_E + e->moe_S, e->num_sms) > 0;
     if (fuse_swiglu && !e->moe_E && P.BN <= 128)
@@ -787,8 +787,8 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
   // 128 rows and keeps the tensor pipe as busy as the weight stream); up to 64 rows every row through every expert
   const bool dec_grouped = e->moe_E > 0 && pad16(B) > 64 && !getenv("CORUN_MOE_DECODE_DENSE");
   if ((rc = program_create(e, e->dec, B, true, true, dec_grouped, true))) return fail(rc);
-  // the decode step's first kernel says which blocks of 64 rows hold a request; the GEMMs of 65..128 padded rows leave
-  // the others out (the one-row program has one block)
+  // the decode step's first kernel says which blocks of rows hold a request (64 rows each up to 128 padded rows, 128
+  // rows each above); the GEMMs leave the others out (the one-row program has one block)
   for (GemmPlan *pl : {&e->dec.p_qkv, &e->dec.p_o, &e->dec.p_gu, &e->dec.p_down, &e->dec.p_lm, &e->dec.p_gu_d, &e->dec.p_down_d})
     pl->row_blocks = e->dec.row_blocks;
   if ((rc = program_create(e, e->pre, e->chunk, true, false, e->moe_E > 0 && !getenv("CORUN_MOE_PREFILL_DENSE")))) return fail(rc);

@@ -95,9 +95,9 @@ struct GemmPlan {
   // Gate / up GEMM with SwiGLU in the epilogue (gemm_plan_create_swiglu): the bf16 hi/lo output [BN, N / 2].
   __nv_bfloat16 *sw_hi = nullptr, *sw_lo = nullptr;
   int sw_half = 0;                   // gate rows (= up rows) per tile
-  // 65..128 padded rows (two stacked blocks of 64 rows): device int, not owned, written by an earlier kernel of the
-  // step: bit b set = rows 64 b .. 64 b + 63 hold a request this step; null = both blocks.  An absent block is
-  // neither loaded nor multiplied nor stored.
+  // Above 64 padded rows the rows form two blocks (65..128 rows: stacked blocks of 64 rows; above: row blocks of 128
+  // rows).  Device int, not owned, written by an earlier kernel of the step: bit b set = block b holds a request
+  // this step; null = both blocks.  An absent block is neither loaded nor multiplied nor stored.
   const int *row_blocks = nullptr;
   GemmOut out() const { return GemmOut{direct, ws, d_tile_first, d_tile_cend, N, KB, BN}; }
 };

@@ -481,9 +481,10 @@ int corun_moe_create(const corun_moe_shape *shape, const void *router, const voi
     return fail(rc);
   m->router = (const bf16 *)router;
   // the three GEMMs run one after the other and their results are consumed in between: one workspace serves all
-  // from 65 to 128 rows the first GEMM applies the routing weight and the SwiGLU in its epilogue (where a tile
-  // width divides the experts' width); else it stores gate / up sums and a kernel of its own follows (faster up to
-  // 64 rows, where the masked store skips most of the output)
+  // the form without groups: from 65 to 128 rows (used there only where the grouped form below does not apply) the
+  // first GEMM applies the routing weight and the SwiGLU in its epilogue (where a tile width divides the experts'
+  // width); else it stores gate / up sums and a kernel of its own follows (faster up to 64 rows, where the masked
+  // store skips most of the output)
   const bool fused = m->BN > 64 && m->BN <= 128 && gemm_swiglu_blocks_half(F, NB, m->num_sms) > 0;
   if ((rc = fused ? gemm_plan_create_swiglu_blocks(&m->p_gu, gate_up, NB, F, H, m->x_hi, m->x_lo, B, m->BN, m->h_hi, m->h_lo, m->w, m->num_sms)
                   : gemm_plan_create(&m->p_gu, gate_up, (int)N1, H, m->x_hi, m->x_lo, B, m->BN, m->out_gu, m->ws, m->num_sms)) ||
