@@ -455,9 +455,10 @@ attn_split_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 #pragma unroll
       for (int h = 0; h < GROUP; ++h) {
         sc[h] = tok_ok ? (__uint_as_float(sv[h]) + __uint_as_float(sv[8 + h])) * sscale : -CUDART_INF_F;
-        float m = sc[h];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        // the warp's maximum in one instruction, on the order-preserving integer image of the float (exact)
+        const uint32_t u = __float_as_uint(sc[h]);
+        const uint32_t km = __reduce_max_sync(0xffffffffu, (u & 0x80000000u) ? ~u : (u | 0x80000000u));
+        const float m = __uint_as_float((km & 0x80000000u) ? (km ^ 0x80000000u) : ~km);
         if (lane == h) red_s[gi][quad][h] = m;
       }
       asm volatile("bar.sync %0, 128;" ::"r"(1 + gi) : "memory");
