@@ -504,7 +504,8 @@ def run_corun_mla(args, rank, world):
     for l in range(mla_cfg["first_dense"]):               # the dense layers bring no experts
         for k in ("router", "gate_up", "down"):
             e_t[k][l] = None
-    eng = corun.Engine(sh, w_t, B, max_ctx, stream=stream.cuda_stream, moe=e_t, mla=m_t)
+    # cache blocks of 64 tokens: four 16-token pages in a row, which the latent attention fetches with one TMA box
+    eng = corun.Engine(sh, w_t, B, max_ctx, stream=stream.cuda_stream, moe=e_t, mla=m_t, kv_block=int(os.environ.get("CORUN_MLA_KV_BLOCK", "64")))
     for i, (s, c) in enumerate(zip(slots, ctx)):
         eng.adopt(int(s), 0, int(c) + total_steps, pending=1 + i, temperature=T, top_p=P, step=1)
         eng.kv_fill(int(s), int(c), kv_std, seed=100 + i)

@@ -134,6 +134,9 @@ int corun_init_moe(const corun_shape *shape, const corun_weights *weights, const
  * kv_lora_rank 256 or 512; qk_nope a multiple of 64; qk_rope even, a multiple of 8, at most 64;
  * qk_nope + v_head a multiple of 256; n_q_heads * v_head a multiple of 64.  A decode step of B slots and a
  * prefill chunk run the same kernels; a prefill row attends to its request's cache up to its own position.
+ * kv_block may be 16 or 64 here: with 64 a slot's cache grows in blocks of 64 tokens (four pages of 16 tokens that
+ * are neighbours in the pool, which the attention kernel fetches with one TMA box instead of four); kv_pool_blocks,
+ * corun_free_blocks and corun_engine_info then count blocks of 64 tokens.  No value depends on the choice.
  * Errors as corun_init.
  */
 typedef struct {

@@ -184,14 +184,16 @@ class Engine:
     """
 
     def __init__(self, shape, weights: dict, B: int, max_context: int, kv_pool_blocks: int = 0, stream=None, moe: dict = None,
-                 mla: dict = None):
+                 mla: dict = None, kv_block: int = 16):
         """``moe``: Mixture-of-Experts feed-forward layers instead of the dense ones: a dict with n_experts, top_k,
         expert_ffn, n_shared, renormalize and lists of L CUDA bf16 tensors router [E, H], gate_up [(E+S)*2F, H],
         down [H, (E+S)*F] (``weights`` then needs no wgate_up / wdown).
         ``mla``: multi-head latent attention layers (``corun_init_mla``): a dict with kv_lora_rank, qk_nope, qk_rope,
         v_head, first_dense and lists of L CUDA bf16 tensors kv_norm [rank], wkv_b [nh*(nope+v), rank]; wqkv / wo of
         ``weights`` then have the MLA shapes, layers below first_dense are dense (wgate_up / wdown entries; None for
-        the other layers), the others take ``moe`` (its entries below first_dense may be None)."""
+        the other layers), the others take ``moe`` (its entries below first_dense may be None).
+        ``kv_block``: tokens per cache block: 16, or (``mla`` only) 64: the 16-token pages of a slot then come in aligned
+        runs of four and the latent attention fetches a run with one TMA box; ``kv_pool_blocks`` counts these blocks."""
         import torch
 
         self._torch = torch
@@ -239,7 +241,7 @@ class Engine:
             L.corun_init_mla.argtypes = [C.POINTER(Shape), C.POINTER(Weights), C.POINTER(MlaLayers), C.POINTER(MoeLayers), C.c_int32,
                                          C.c_int32, C.c_int32, C.c_int64, C.c_void_p, C.POINTER(C.c_void_p)]
             _check(L.corun_init_mla(C.byref(self._cs), C.byref(cw), C.byref(cl), C.byref(cm) if cm is not None else None, B,
-                                    max_context, 16, kv_pool_blocks, C.c_void_p(stream) if stream else None, C.byref(h)),
+                                    max_context, kv_block, kv_pool_blocks, C.c_void_p(stream) if stream else None, C.byref(h)),
                    "corun_init_mla")
         elif moe:
             L = lib()

@@ -108,6 +108,10 @@ struct corun_engine {
   __half *kv_pool = nullptr;
   size_t layer_stride = 0;
   int *d_block_table = nullptr;
+  // Pages are handed out in aligned runs of kv_run consecutive pool pages (1; 4 for latent caches created with
+  // kv_block = 64: the latent attention kernel then fetches a run with one TMA box).  free_blocks / slot_blocks hold
+  // RUN indices; the block table holds pages (run * kv_run + i).
+  int kv_run = 1;
   std::vector<int> free_blocks;
   std::vector<std::vector<int>> slot_blocks;
   float2 *d_rope = nullptr;
@@ -376,7 +380,7 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
       STAGE(gemm_launch(P.p_uk, &e->tm_uk[l], e->d_status, e->st, nullptr, true));
       STAGE(launch_mla_attention(e->tm_c[l], e->tm_cv[l], P.q_lat, md.rank, (long long)P.RPH * md.rank, P.q_rope, e->d_block_table,
                                  e->max_blocks, nullptr, &rows, P.R, md, 1.0f / sqrtf((float)(md.nope + md.rope)), e->mla_splits,
-                                 P.mla_ml, P.mla_po, nullptr, P.ol_hi, P.ol_lo, P.RPH, e->num_sms, e->d_status, true, e->st));
+                                 P.mla_ml, P.mla_po, nullptr, P.ol_hi, P.ol_lo, P.RPH, e->num_sms, e->d_status, true, e->st, e->kv_run));
       STAGE(gemm_launch(P.p_uv, &e->tm_uv[l], e->d_status, e->st, nullptr, true));
       STAGE(launch_mla_ao_split(P.uv_out, P.R, P.RPH, md, P.ao_hi, P.ao_lo, e->st));
       n += 3 + (&P == &e->dec ? 0 : 1);               // beyond the count below: two grouped GEMMs, the split, and in prefill too a second attention kernel
@@ -487,7 +491,8 @@ int sync_stream(corun_engine *e) {
 }
 
 int reserve_blocks(corun_engine *e, int slot, int reserve_len) {
-  const int need = (reserve_len + KV_BLOCK - 1) / KV_BLOCK;
+  const int run_tokens = KV_BLOCK * e->kv_run;
+  const int need = (reserve_len + run_tokens - 1) / run_tokens;   // runs
   if ((size_t)need > e->free_blocks.size()) return CORUN_ENOSPACE;
   std::vector<int> &mine = e->slot_blocks[slot];
   mine.clear();
@@ -495,7 +500,7 @@ int reserve_blocks(corun_engine *e, int slot, int reserve_len) {
   for (int i = 0; i < need; ++i) {
     mine.push_back(e->free_blocks.back());
     e->free_blocks.pop_back();
-    row[i] = mine.back();
+    for (int j = 0; j < e->kv_run && i * e->kv_run + j < e->max_blocks; ++j) row[i * e->kv_run + j] = mine.back() * e->kv_run + j;
   }
   CK(cudaMemcpyAsync(e->d_block_table + (size_t)slot * e->max_blocks, row.data(), e->max_blocks * sizeof(int),
                      cudaMemcpyHostToDevice, e->st));
@@ -580,7 +585,10 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
   if (group != 1 && group != 2 && group != 4 && group != 8) return CORUN_EINVAL;
   if ((s.n_q_heads * s.head_dim) % 64) return CORUN_EINVAL;
   if (!(s.rms_eps >= 0.f) || !(s.rope_theta > 0.f)) return CORUN_EINVAL;
-  if (B < 1 || B > 256 || max_context < 1 || max_context > 256 * ATT_SPLIT || kv_block != KV_BLOCK || kv_pool_blocks < 0) return CORUN_EINVAL;
+  // kv_block: 16, or (latent caches only) 64: pages of 16 tokens handed out in aligned runs of four
+  if (B < 1 || B > 256 || max_context < 1 || max_context > 256 * ATT_SPLIT || !(kv_block == KV_BLOCK || (mla && kv_block == 4 * KV_BLOCK)) ||
+      kv_pool_blocks < 0)
+    return CORUN_EINVAL;
   if (!w->embed || !w->lm_head || !w->final_norm || !w->attn_norm || !w->wqkv || !w->wo || !w->mlp_norm ||
       (!moe && (!w->wgate_up || !w->wdown)))
     return CORUN_EINVAL;
@@ -604,7 +612,8 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
   e->sh = s;
   e->B = B;
   e->max_ctx = max_context;
-  e->max_blocks = (max_context + KV_BLOCK - 1) / KV_BLOCK;
+  e->kv_run = kv_block / KV_BLOCK;
+  e->max_blocks = (max_context + kv_block - 1) / kv_block * e->kv_run;   // pages of 16 tokens, whole runs
   e->max_splits = (max_context + ATT_SPLIT - 1) / ATT_SPLIT;
   e->num_sms = prop.multiProcessorCount;
   e->st = (cudaStream_t)cuda_stream;
@@ -632,7 +641,7 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
     e->moe_S = moe->n_shared;
     e->moe_renorm = moe->renormalize ? 1 : 0;
   }
-  e->pool_blocks = kv_pool_blocks ? kv_pool_blocks : (int64_t)B * e->max_blocks;
+  e->pool_blocks = kv_pool_blocks ? kv_pool_blocks * e->kv_run : (int64_t)B * e->max_blocks;   // in pages of 16 tokens
   if (!kv_pool_blocks) {
     // default size: a full reservation for every slot, or as many pages as fit beside 6 GiB that are
     // left for the programs' buffers, whichever is less (admission then refuses what does not fit)
@@ -642,8 +651,8 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
                               : (size_t)s.n_layers * 2 * s.n_kv_heads * KV_BLOCK * s.head_dim * sizeof(__half);
     const size_t keep = (size_t)6 << 30;
     const int64_t fit = free_b > keep ? (int64_t)((free_b - keep) / page_b) : 0;
-    if (fit < e->pool_blocks) e->pool_blocks = fit;
-    if (e->pool_blocks < 1) return fail(CORUN_ENOMEM);
+    if (fit < e->pool_blocks) e->pool_blocks = fit / e->kv_run * e->kv_run;
+    if (e->pool_blocks < e->kv_run) return fail(CORUN_ENOMEM);
   }
   e->chunk = 256;
   if (const char *c = getenv("CORUN_ATTN_WHOLE_PAIRS")) e->whole_pairs = atoi(c) != 0;   // ablation only
@@ -715,7 +724,8 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
     e->tm_c.resize(s.n_layers);
     e->tm_cv.resize(s.n_layers);
     for (int l = 0; l < s.n_layers; ++l)
-      if ((rc = mla_encode_maps(&e->tm_c[l], &e->tm_cv[l], e->kv_pool + (size_t)l * e->layer_stride, e->pool_blocks, e->md.rank, e->md.rope)))
+      if ((rc = mla_encode_maps(&e->tm_c[l], &e->tm_cv[l], e->kv_pool + (size_t)l * e->layer_stride, e->pool_blocks, e->md.rank, e->md.rope,
+                                e->kv_run)))
         return fail(rc);
   } else {
     // one layer's pages seen as rows of hd halfs (16 rows per page and head, keys first, then values)
@@ -761,8 +771,9 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
     const int one = 1;
     if (cudaMemcpy(e->d_pf_one, &one, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return fail(CORUN_ECUDA);
   }
-  e->free_blocks.resize((size_t)e->pool_blocks);
-  for (int64_t i = 0; i < e->pool_blocks; ++i) e->free_blocks[(size_t)i] = (int)(e->pool_blocks - 1 - i);
+  const int64_t n_runs = e->pool_blocks / e->kv_run;
+  e->free_blocks.resize((size_t)n_runs);
+  for (int64_t i = 0; i < n_runs; ++i) e->free_blocks[(size_t)i] = (int)(n_runs - 1 - i);
   e->slot_blocks.resize(B);
   e->in_use.assign(B, 0);
   e->ctx.assign(B, 0);
@@ -904,7 +915,7 @@ int prefill_run(corun_engine *e, PfReq *reqs, int n_req);
 int prefill_many(corun_engine *e, PfReq *reqs, int n_req) {
   RC(sync_stream(e));
   size_t need = 0;
-  for (int i = 0; i < n_req; ++i) need += (size_t)(reqs[i].reserve + KV_BLOCK - 1) / KV_BLOCK;
+  for (int i = 0; i < n_req; ++i) need += (size_t)(reqs[i].reserve + KV_BLOCK * e->kv_run - 1) / (KV_BLOCK * e->kv_run);   // runs
   if (need > e->free_blocks.size()) return CORUN_ENOSPACE;
   int rc = CORUN_OK;
   for (int i = 0; i < n_req && rc == CORUN_OK; ++i) rc = reserve_blocks(e, reqs[i].slot, reqs[i].reserve);
@@ -1116,8 +1127,8 @@ int corun_engine_info(corun_engine *e, int32_t *B, int32_t *max_context, int32_t
   if (!e) return CORUN_EINVAL;
   if (B) *B = e->B;
   if (max_context) *max_context = e->max_ctx;
-  if (kv_block) *kv_block = KV_BLOCK;
-  if (pool_blocks) *pool_blocks = e->pool_blocks;
+  if (kv_block) *kv_block = KV_BLOCK * e->kv_run;   // the unit pages are handed out in (corun_free_blocks counts these)
+  if (pool_blocks) *pool_blocks = e->pool_blocks / e->kv_run;
   return CORUN_OK;
 }
 
@@ -1289,7 +1300,7 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
                   ce = launch_mla_attention(e->tm_c[l], e->tm_cv[l], P.q_lat, e->md.rank, (long long)P.RPH * e->md.rank, P.q_rope,
                                             e->d_block_table, e->max_blocks, nullptr, &rows, P.R, e->md,
                                             1.0f / sqrtf((float)(e->md.nope + e->md.rope)), e->mla_splits, P.mla_ml, P.mla_po, nullptr,
-                                            P.ol_hi, P.ol_lo, P.RPH, e->num_sms, e->d_status, true, e->st);
+                                            P.ol_hi, P.ol_lo, P.RPH, e->num_sms, e->d_status, true, e->st, e->kv_run);
                   break;
                 }
                 ce = cudaMemsetAsync(P.att_pool + l, 0, sizeof(int), e->st);   // the launch does not reset its pool counter

@@ -37,7 +37,9 @@ cudaError_t launch_mla_post(const GemmOut &qkv, const Rows &rows, const float2 *
                             __nv_bfloat16 *qn_hi, __nv_bfloat16 *qn_lo, float *q_rope, int *d_status, cudaStream_t st);
 
 // Tensor maps over one layer's latent pages for the attention kernel.
-int mla_encode_maps(CUtensorMap *tmC, CUtensorMap *tmV, const void *pool, long long pool_pages, int rank, int rope);
+// page_run: pool pages per TMA box (1, or 4 where every row's block table holds its pages in aligned runs of four
+// consecutive pool pages: launch_mla_attention takes the same value)
+int mla_encode_maps(CUtensorMap *tmC, CUtensorMap *tmV, const void *pool, long long pool_pages, int rank, int rope, int page_run);
 // Floats of the partial results for R rows of at most max_context cached tokens: (max, sum) pairs, then outputs.
 long long mla_part_ml_floats(int R, int nh, int max_context);
 long long mla_part_o_floats(int R, int nh, int rank, int max_context);
@@ -52,7 +54,7 @@ cudaError_t launch_mla_attention(const CUtensorMap &tmC, const CUtensorMap &tmV,
                                  long long q_head_stride, const float *q_rope, const int *block_table, int max_blocks,
                                  const int *ctx, const Rows *rows, int R, const MlaDims &d, float scale, int max_splits,
                                  float2 *part_ml, float *part_o, float *o_lat, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
-                                 int rows_per_head, int num_sms, int *d_status, bool pdl, cudaStream_t st);
+                                 int rows_per_head, int num_sms, int *d_status, bool pdl, cudaStream_t st, int page_run);
 
 // The value part of the grouped up-projection result uv [nh * rows_per_head][nope + vh] (columns nope.. of every
 // row) -> bf16 hi/lo [R][nh * vh], the o-projection's activations.

@@ -86,7 +86,7 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
                  long long q_rs, long long q_hs, const float *__restrict__ q_rope, const int *__restrict__ block_table, int max_blocks,
                  const int *__restrict__ ctx, const int *__restrict__ row_slot, const int *__restrict__ row_pos,
                  const int *__restrict__ row_active, int B, int n_heads, int d_c, int d_r, float scale_log2e, int max_splits,
-                 float2 *__restrict__ part_ml, float *__restrict__ part_o, int *status) {
+                 float2 *__restrict__ part_ml, float *__restrict__ part_o, int *status, int page_run) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[MP_RING], empty_bar[MP_RING];
   __shared__ __align__(8) uint64_t q_ready_bar, q_free_bar, s_full_bar, s_free_bar, p_ready_bar, o_full_bar, o_free_bar, x_bar;
@@ -220,13 +220,18 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
       const int page = page_ahead, np = np_ahead;      // looked up one item ahead of its use
       page_ahead = pages_of(it + 1, np_ahead);
       if (it < item_hi) {
+        // page_run consecutive pool pages per box (4: the table's pages come in aligned runs of four, so one box of
+        // 64 tokens fetches what four boxes of 16 would: the TMA unit is bound by the number of boxes)
+        const int nbx = (np + page_run - 1) / page_run;
+        const int bpage = __shfl_sync(0xffffffffu, page, (page_run * lane) & 31);
         for (int j = 0; j <= NLB; ++j, ++u) {           // latent blocks, then the rope block
           if (!slot_free(u)) { failed = true; break; }
           const uint32_t bar = smem_u32(&full_bar[u % MP_RING]);
-          if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)(np * MP_BOX));
+          if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)(nbx * page_run * MP_BOX));
           __syncwarp();
-          if (lane < np)
-            tma_load_2d(base + (uint32_t)(u % MP_RING) * MP_SLOT + (uint32_t)lane * MP_BOX, &tmC, j < NLB ? 64 * j : d_c, page * MP_PAGE, bar, pol_keep);
+          if (lane < nbx)
+            tma_load_2d(base + (uint32_t)(u % MP_RING) * MP_SLOT + (uint32_t)(lane * page_run) * MP_BOX, &tmC, j < NLB ? 64 * j : d_c,
+                        bpage * MP_PAGE, bar, pol_keep);
         }
       }
       if (it > item_lo && !failed) {                     // the previous item's latent once more, page-major
@@ -234,10 +239,10 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
         for (int hu = 0; hu < n_half * nu; ++hu, ++u) {
           const int half = hu / nu, uu = hu - half * nu;
           if (!slot_free(u)) { failed = true; break; }
-          const int cnt = min(4, prev_np - 4 * uu);
+          const int cnt = page_run == 4 ? 1 : min(4, prev_np - 4 * uu);   // boxes: a run of four pages is one
           const int pg = __shfl_sync(0xffffffffu, prev_page, (4 * uu + lane) & 31);
           const uint32_t bar = smem_u32(&full_bar[u % MP_RING]);
-          if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)(cnt * BPH * MP_BOX));
+          if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)(cnt * page_run * BPH * MP_BOX));
           __syncwarp();
           if (lane < cnt)
             tma_load_4d(base + (uint32_t)(u % MP_RING) * MP_SLOT + (uint32_t)(lane * BPH) * MP_BOX, &tmV, 0, 0, half * BPH, pg * 2, bar, pol_drop);
@@ -577,19 +582,20 @@ int mla_max_splits(int max_context) { return (max_context + MP_T - 1) / MP_T; }
 long long mla_part_ml_floats(int R, int nh, int max_context) { return ((long long)R * mla_max_splits(max_context) * nh * 2 + 3) / 4 * 4; }
 long long mla_part_o_floats(int R, int nh, int rank, int max_context) { return (long long)R * mla_max_splits(max_context) * nh * rank; }
 
-int mla_encode_maps(CUtensorMap *tmC, CUtensorMap *tmV, const void *pool, long long pool_pages, int rank, int rope) {
-  if (pool_pages < 1 || pool_pages * MP_PAGE >= (1ll << 31)) return CORUN_EINVAL;
+int mla_encode_maps(CUtensorMap *tmC, CUtensorMap *tmV, const void *pool, long long pool_pages, int rank, int rope, int page_run) {
+  if (pool_pages < 1 || pool_pages * MP_PAGE >= (1ll << 31) || (page_run != 1 && page_run != 4)) return CORUN_EINVAL;
   // the pool as rows of rank + rope halfs, fetched in [16 tokens x 64 dims] boxes (the rope box reads past the
   // row's end when rope < 64: those columns arrive as zeros)
-  int rc = tma_encode_2d(tmC, pool, 1, (unsigned long long)pool_pages * MP_PAGE, rank + rope, MP_PAGE, 64);
+  int rc = tma_encode_2d(tmC, pool, 1, (unsigned long long)pool_pages * MP_PAGE, rank + rope, MP_PAGE * page_run, 64);
   if (rc != CORUN_OK) return rc;
   // the latent part once more as [8-token group][token in group][block of 64 dims][64 dims]: one box fetches a page's
   // 16 tokens x (up to) 256 dims as [2 groups][blocks][8 tokens][64 dims], the layout of an MN-major MMA operand
+  // (page_run = 4: boxes of four consecutive pages: [64 tokens x 64 dims] and [8 groups][blocks][8 tokens][64 dims])
   const int bph = rank > 256 ? 4 : rank / 64;
   const unsigned long long row_bytes = (unsigned long long)(rank + rope) * 2;
   const unsigned long long dims[4] = {64, 8, (unsigned long long)(rank / 64), (unsigned long long)pool_pages * 2};
   const unsigned long long strides[3] = {row_bytes, 128, 8 * row_bytes};
-  const unsigned box[4] = {64, 8, (unsigned)bph, 2};
+  const unsigned box[4] = {64, 8, (unsigned)bph, 2u * (unsigned)page_run};
   return tma_encode_fp16_4d(tmV, pool, dims, strides, box);
 }
 
@@ -597,7 +603,7 @@ cudaError_t launch_mla_attention(const CUtensorMap &tmC, const CUtensorMap &tmV,
                                  long long q_head_stride, const float *q_rope, const int *block_table, int max_blocks,
                                  const int *ctx, const Rows *rows, int R, const MlaDims &d, float scale, int max_splits,
                                  float2 *part_ml, float *part_o, float *o_lat, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
-                                 int rows_per_head, int num_sms, int *d_status, bool pdl, cudaStream_t st) {
+                                 int rows_per_head, int num_sms, int *d_status, bool pdl, cudaStream_t st, int page_run) {
   static bool prepared = false;                     // idempotent; a race only repeats it
   if (!prepared) {
     cudaError_t e = cudaFuncSetAttribute(mla_paged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MP_SMEM);
@@ -607,7 +613,7 @@ cudaError_t launch_mla_attention(const CUtensorMap &tmC, const CUtensorMap &tmV,
   const int *row_slot = rows ? rows->slot : nullptr, *row_pos = rows ? rows->pos : nullptr, *row_active = rows ? rows->active : nullptr;
   cudaError_t ce = launch_k(mla_paged_kernel, dim3(num_sms), dim3(MP_THREADS), MP_SMEM, st, pdl, tmC, tmV, q_lat, q_row_stride,
                             q_head_stride, q_rope, block_table, max_blocks, ctx, row_slot, row_pos, row_active, R, d.nh, d.rank, d.rope,
-                            scale * 1.4426950408889634f, max_splits, part_ml, part_o, d_status);
+                            scale * 1.4426950408889634f, max_splits, part_ml, part_o, d_status, page_run);
   if (ce != cudaSuccess) return ce;
   return launch_k(mla_paged_combine_kernel, dim3(R * d.nh), dim3(128), 0, st, true, part_ml, part_o, ctx, row_pos, row_active, R, d.nh,
                   d.rank, max_blocks, max_splits, o_lat, out_hi, out_lo, rows_per_head);
@@ -640,7 +646,7 @@ int corun_mla_attend(const float *q_lat, const float *q_rope, const void *pool, 
   if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (ce != cudaSuccess || sms < 1) { g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
   CUtensorMap tm, tv;
-  int rc = mla_encode_maps(&tm, &tv, pool, pool_pages, d_latent, d_rope);
+  int rc = mla_encode_maps(&tm, &tv, pool, pool_pages, d_latent, d_rope, 1);   // any block table: one page per box
   if (rc != CORUN_OK) return rc;
   const int max_splits = mla_max_splits(max_blocks * MP_PAGE);
   int *status = reinterpret_cast<int *>(ws);
@@ -650,7 +656,7 @@ int corun_mla_attend(const float *q_lat, const float *q_rope, const void *pool, 
   ce = cudaMemsetAsync(status, 0, sizeof(int), st);
   if (ce == cudaSuccess)
     ce = launch_mla_attention(tm, tv, q_lat, (long long)n_heads * d_latent, d_latent, q_rope, block_table, max_blocks, ctx, nullptr, B, dims,
-                              scale, max_splits, part_ml, part_o, o_lat, nullptr, nullptr, 0, sms, status, false, st);
+                              scale, max_splits, part_ml, part_o, o_lat, nullptr, nullptr, 0, sms, status, false, st, 1);
   if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return CORUN_ECUDA; }
   return CORUN_OK;
 }

@@ -35,11 +35,12 @@ def _setup(orc, sh, mla, moe, seed, B=B, max_ctx=MAX_CTX, **kw):
     return model, eng
 
 
-@pytest.mark.parametrize("first_dense,moe", [(1, SMALL_MOE), (3, None)])
-def test_mla_engine_parity_and_invariance(orc, first_dense, moe):
+# kv_block 64: the 16-token pages of a slot in aligned runs of four, fetched by the attention kernel one run per TMA box
+@pytest.mark.parametrize("first_dense,moe,kv_block", [(1, SMALL_MOE, 16), (3, None, 16), (1, SMALL_MOE, 64)])
+def test_mla_engine_parity_and_invariance(orc, first_dense, moe, kv_block):
     sh = SMALL
     mla = dict(SMALL_MLA, first_dense=first_dense)
-    model, eng = _setup(orc, sh, mla, moe, seed=3)
+    model, eng = _setup(orc, sh, mla, moe, seed=3, kv_block=kv_block)
     try:
         lens = [21, 270, 64, 9]                          # one prompt beyond a 256-token attention split and a prefill chunk
         prompts = synth.make_prompts(sh.vocab, lens, seed=31)
