@@ -374,7 +374,7 @@ int run_layers(corun_engine *e, Program &P, int *launches) {
       // cache append and query parts -> q_lat = W_uk^T q_nope per head -> absorbed attention over the row's latent
       // pages (decode rows and prefill rows alike) -> [. | o] = W_kv_b o_lat per head -> the value part, split
       const MlaDims &md = e->md;
-      const MlaCache cache{e->kv_pool + (size_t)l * e->layer_stride, e->d_block_table, e->max_blocks, e->B, (long long)e->pool_blocks};
+      const MlaCache cache{e->kv_pool + (size_t)l * e->layer_stride, e->d_block_table, e->max_blocks, e->B, (long long)e->pool_blocks, e->kv_run};
       STAGE(launch_mla_post(P.p_qkv.out(), rows, e->d_rope, md, e->kv_norm[l], s.rms_eps, cache, P.RPH, P.qn_hi, P.qn_lo, P.q_rope,
                             e->d_status, e->st));
       STAGE(gemm_launch(P.p_uk, &e->tm_uk[l], e->d_status, e->st, nullptr, true));
@@ -647,7 +647,7 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
     // left for the programs' buffers, whichever is less (admission then refuses what does not fit)
     size_t free_b = 0, total_b = 0;
     if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess) return fail(CORUN_ECUDA);
-    const size_t page_b = mla ? (size_t)s.n_layers * KV_BLOCK * (mla->kv_lora_rank + mla->qk_rope) * sizeof(__half)
+    const size_t page_b = mla ? (size_t)s.n_layers * KV_BLOCK * (size_t)mla_token_halfs(mla->kv_lora_rank + mla->qk_rope, e->kv_run) * sizeof(__half)
                               : (size_t)s.n_layers * 2 * s.n_kv_heads * KV_BLOCK * s.head_dim * sizeof(__half);
     const size_t keep = (size_t)6 << 30;
     const int64_t fit = free_b > keep ? (int64_t)((free_b - keep) / page_b) : 0;
@@ -715,7 +715,7 @@ static int engine_create(const corun_shape *shape, const corun_weights *w, const
 
   auto &A = e->allocs;
   int rc;
-  e->layer_stride = mla ? (size_t)e->pool_blocks * KV_BLOCK * (e->md.rank + e->md.rope)
+  e->layer_stride = mla ? (size_t)e->pool_blocks * KV_BLOCK * (size_t)mla_token_halfs(e->md.rank + e->md.rope, e->kv_run)
                         : (size_t)e->pool_blocks * 2 * s.n_kv_heads * KV_BLOCK * s.head_dim;
   // zero-filled: masked positions of a page are multiplied by zero weights, so they must be finite
   if ((rc = dmalloc(A, &e->kv_pool, e->layer_stride * s.n_layers, true))) return fail(rc);
@@ -1148,7 +1148,7 @@ static int latent_io(corun_engine *e, int slot, int layer, int pos0, int n, floa
   const size_t elems = (size_t)n * row;
   float *dk = nullptr;
   if (cudaMalloc(&dk, elems * sizeof(float)) != cudaSuccess) return CORUN_ENOMEM;
-  const MlaCache cache{e->kv_pool + (size_t)layer * e->layer_stride, e->d_block_table, e->max_blocks, e->B, (long long)e->pool_blocks};
+  const MlaCache cache{e->kv_pool + (size_t)layer * e->layer_stride, e->d_block_table, e->max_blocks, e->B, (long long)e->pool_blocks, e->kv_run};
   cudaError_t ce = cudaSuccess;
   if (write) ce = cudaMemcpyAsync(dk, k, elems * sizeof(float), cudaMemcpyHostToDevice, e->st);
   if (ce == cudaSuccess) ce = launch_mla_copy(cache, row, slot, pos0, n, dk, write, e->st);
@@ -1239,7 +1239,7 @@ int corun_debug_kv_fill(corun_engine *e, int32_t slot, int32_t n_ctx, float std,
   RC(sync_stream(e));
   if (e->mla) {
     for (int l = 0; l < e->sh.n_layers; ++l) {
-      const MlaCache cache{e->kv_pool + (size_t)l * e->layer_stride, e->d_block_table, e->max_blocks, e->B, (long long)e->pool_blocks};
+      const MlaCache cache{e->kv_pool + (size_t)l * e->layer_stride, e->d_block_table, e->max_blocks, e->B, (long long)e->pool_blocks, e->kv_run};
       CK(launch_mla_fill(cache, e->md.rank + e->md.rope, l, slot, n_ctx, std, seed, e->st));
     }
   } else {
@@ -1275,7 +1275,7 @@ int corun_debug_time_kernel(corun_engine *e, int32_t kind, int32_t reps, float *
         l = e->first_dense + i % (s.n_layers - e->first_dense);
       GemmOut prev = ffn_out(e, P, l);
       const MlaCache mcache{e->mla ? e->kv_pool + (size_t)l * e->layer_stride : nullptr, e->d_block_table, e->max_blocks, e->B,
-                            (long long)e->pool_blocks};
+                            (long long)e->pool_blocks, e->kv_run};
       switch (kind) {
         // launched as in the step's graph: with programmatic stream serialization
         case 0: ce = gemm_launch(P.p_qkv, &e->tm_qkv[l], e->d_status, e->st, nullptr, true); break;

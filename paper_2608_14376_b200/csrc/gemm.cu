@@ -570,26 +570,31 @@ int tma_encode_2d(CUtensorMap *m, const void *base, int is_fp16, unsigned long l
   return r == CUDA_SUCCESS ? CORUN_OK : CORUN_ECUDA;
 }
 
-int tma_encode_fp16_4d(CUtensorMap *m, const void *base, const unsigned long long dims[4], const unsigned long long strides[3],
-                       const unsigned box[4]) {
+int tma_encode_fp16_nd(CUtensorMap *m, const void *base, int nd, const unsigned long long *dims, const unsigned long long *strides,
+                       const unsigned *box) {
   auto enc = get_encode();
   if (!enc) { g_last_cuda_error = 99999; return CORUN_ECUDA; }
-  if (((uintptr_t)base & 15u) || box[0] * 2 != 128) return CORUN_EINVAL;
-  cuuint64_t d[4], s[3];
-  cuuint32_t b[4], estr[4] = {1, 1, 1, 1};
-  for (int i = 0; i < 4; ++i) {
+  if (nd < 2 || nd > 5 || ((uintptr_t)base & 15u) || box[0] * 2 != 128) return CORUN_EINVAL;
+  cuuint64_t d[5], s[4];
+  cuuint32_t b[5], estr[5] = {1, 1, 1, 1, 1};
+  for (int i = 0; i < nd; ++i) {
     if (dims[i] < 1 || box[i] < 1 || box[i] > 256) return CORUN_EINVAL;
     d[i] = dims[i];
     b[i] = box[i];
   }
-  for (int i = 0; i < 3; ++i) {
+  for (int i = 0; i < nd - 1; ++i) {
     if (strides[i] % 16) return CORUN_EINVAL;
     s[i] = strides[i];
   }
-  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void *>(base), d, s, b, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, (cuuint32_t)nd, const_cast<void *>(base), d, s, b, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) g_last_cuda_error = 100000 + (int)r;
   return r == CUDA_SUCCESS ? CORUN_OK : CORUN_ECUDA;
+}
+
+int tma_encode_fp16_4d(CUtensorMap *m, const void *base, const unsigned long long dims[4], const unsigned long long strides[3],
+                       const unsigned box[4]) {
+  return tma_encode_fp16_nd(m, base, 4, dims, strides, box);
 }
 
 int gemm_encode_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows) {

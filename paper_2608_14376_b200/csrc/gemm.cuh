@@ -168,6 +168,9 @@ int tma_encode_2d(CUtensorMap *m, const void *base, int is_fp16, unsigned long l
 // dimension 0 fastest.
 int tma_encode_fp16_4d(CUtensorMap *m, const void *base, const unsigned long long dims[4], const unsigned long long strides[3],
                        const unsigned box[4]);
+// The same with 2 to 5 dimensions (dims / box: nd values, strides: nd - 1 byte strides of dimensions 1 ..).
+int tma_encode_fp16_nd(CUtensorMap *m, const void *base, int nd, const unsigned long long *dims, const unsigned long long *strides,
+                       const unsigned *box);
 // direct[r, n] = gemm_load(r, n) for every tile that has partials (makes `direct` a plain matrix).
 cudaError_t gemm_fixup_launch(const GemmPlan &p, cudaStream_t st, bool pdl = false);
 

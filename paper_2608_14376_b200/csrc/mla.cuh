@@ -16,12 +16,28 @@ struct MlaDims {
 };
 
 // One layer's latent pages and how a row finds its own.
+// run = 1: the pool is [page][16 tokens][rank + rope] (a token's values contiguous).
+// run = 4: pages come in aligned runs of four (blocks of 64 tokens) and a run is stored BLOCK-MAJOR:
+//          [run][block of 64 dims (the last one zero-padded)][64 tokens][64 dims], so that the attention kernel's
+//          [64 tokens x 64 dims] boxes are 8 KiB of contiguous memory (boxes that take 128 bytes out of every
+//          1152-byte token row stream from HBM at 4.6 TB/s, contiguous ones at 7.0 TB/s).
 struct MlaCache {
-  __half *pool;              // this layer's pages: [page][16 tokens][rank + rope]
+  __half *pool;
   const int *block_table;    // [n_slots][max_blocks]
   int max_blocks, n_slots;
   long long pool_blocks;
+  int run;                   // 1 or 4
 };
+// Halfs per cached token in the pool (run = 4: whole blocks of 64 dims).
+inline long long mla_token_halfs(int row_halfs, int run) { return run == 1 ? row_halfs : (long long)((row_halfs + 63) / 64) * 64; }
+#ifdef __CUDACC__
+// Where value e of the token at offset `off` of page `blk` lives.
+__device__ __forceinline__ __half *mla_cache_at(const MlaCache &c, int row_halfs, int blk, int off, int e) {
+  if (c.run == 1) return c.pool + ((size_t)blk * KV_BLOCK + off) * row_halfs + e;
+  const int nblk = (row_halfs + 63) >> 6, r = blk >> 2, tok = (blk & 3) * KV_BLOCK + off;
+  return c.pool + (((size_t)r * nblk + (e >> 6)) * 64 + tok) * 64 + (e & 63);
+}
+#endif
 
 // Rows of the head-major activation matrices ([head][rows_per_head][K]) for a program of BN padded rows: the
 // grouped GEMMs take blocks of at most 64 rows.

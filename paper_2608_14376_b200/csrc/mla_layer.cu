@@ -60,7 +60,7 @@ mla_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, Mla
     return;
   }
 #endif
-  __half *dst = cache.pool + ((size_t)blk * KV_BLOCK + pos % KV_BLOCK) * (d.rank + d.rope);
+  const int row_halfs = d.rank + d.rope, off = pos % KV_BLOCK;   // the row's cache position: mla_cache_at(.., blk, off, e)
   // the latent's values are requested first and used last: the sums of the GEMM's partials behind every load
   // below overlap instead of queueing behind the block-wide reduction
   float4 x = make_float4(0.f, 0.f, 0.f, 0.f);        // rank <= 4 * threads
@@ -87,8 +87,8 @@ mla_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, Mla
     mla_rotate4(gemm_load4(qkv, r, QD + d.rank + j), gemm_load4(qkv, r, QD + d.rank + j + half), tab + j, ra, rb);
     __half2 oa[2] = {__floats2half2_rn(ra.x, ra.y), __floats2half2_rn(ra.z, ra.w)};
     __half2 ob[2] = {__floats2half2_rn(rb.x, rb.y), __floats2half2_rn(rb.z, rb.w)};
-    *reinterpret_cast<uint2 *>(dst + d.rank + j) = *reinterpret_cast<const uint2 *>(oa);
-    *reinterpret_cast<uint2 *>(dst + d.rank + j + half) = *reinterpret_cast<const uint2 *>(ob);
+    *reinterpret_cast<uint2 *>(mla_cache_at(cache, row_halfs, blk, off, d.rank + j)) = *reinterpret_cast<const uint2 *>(oa);
+    *reinterpret_cast<uint2 *>(mla_cache_at(cache, row_halfs, blk, off, d.rank + j + half)) = *reinterpret_cast<const uint2 *>(ob);
   }
   float ss = 0.f;
   ss = fmaf(x.x, x.x, ss); ss = fmaf(x.y, x.y, ss); ss = fmaf(x.z, x.z, ss); ss = fmaf(x.w, x.w, ss);
@@ -104,7 +104,7 @@ mla_post_kernel(GemmOut qkv, Rows rows, const float2 *__restrict__ rope_tab, Mla
     const __nv_bfloat162 *g2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
     const float2 ga = __bfloat1622float2(g2[0]), gb = __bfloat1622float2(g2[1]);
     __half2 o[2] = {__floats2half2_rn(x.x * inv * ga.x, x.y * inv * ga.y), __floats2half2_rn(x.z * inv * gb.x, x.w * inv * gb.y)};
-    *reinterpret_cast<uint2 *>(dst + 4 * tid) = *reinterpret_cast<const uint2 *>(o);
+    *reinterpret_cast<uint2 *>(mla_cache_at(cache, row_halfs, blk, off, 4 * tid)) = *reinterpret_cast<const uint2 *>(o);
   }
 }
 
@@ -150,9 +150,9 @@ __global__ void mla_fill_kernel(MlaCache cache, int row_halfs, int layer, int sl
   const float u2 = (float)(uint32_t)((h >> 8) & 0xFFFFFFu) * (1.0f / 16777216.0f);
   const float rad = sqrtf(-2.0f * logf(u1)) * std;
   const int blk = cache.block_table[(size_t)slot * cache.max_blocks + t / KV_BLOCK];
-  __half *row = cache.pool + ((size_t)blk * KV_BLOCK + t % KV_BLOCK) * row_halfs;
-  row[2 * e] = __float2half_rn(rad * cospif(2.0f * u2));
-  row[2 * e + 1] = __float2half_rn(rad * sinpif(2.0f * u2));
+  __half *row = mla_cache_at(cache, row_halfs, blk, t % KV_BLOCK, 2 * e);   // a pair never straddles a block of 64 dims
+  row[0] = __float2half_rn(rad * cospif(2.0f * u2));
+  row[1] = __float2half_rn(rad * sinpif(2.0f * u2));
 }
 
 __global__ void mla_copy_kernel(MlaCache cache, int row_halfs, int slot, int pos0, int n, float *buf, int write) {
@@ -160,7 +160,7 @@ __global__ void mla_copy_kernel(MlaCache cache, int row_halfs, int slot, int pos
   if (idx >= (size_t)n * row_halfs) return;
   const int t = pos0 + (int)(idx / row_halfs), e = (int)(idx % row_halfs);
   const int blk = cache.block_table[(size_t)slot * cache.max_blocks + t / KV_BLOCK];
-  __half *p = cache.pool + ((size_t)blk * KV_BLOCK + t % KV_BLOCK) * row_halfs + e;
+  __half *p = mla_cache_at(cache, row_halfs, blk, t % KV_BLOCK, e);
   if (write) *p = __float2half_rn(buf[idx]);
   else buf[idx] = __half2float(*p);
 }

@@ -229,9 +229,13 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
           const uint32_t bar = smem_u32(&full_bar[u % MP_RING]);
           if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)(nbx * page_run * MP_BOX));
           __syncwarp();
-          if (lane < nbx)
-            tma_load_2d(base + (uint32_t)(u % MP_RING) * MP_SLOT + (uint32_t)(lane * page_run) * MP_BOX, &tmC, j < NLB ? 64 * j : d_c,
-                        bpage * MP_PAGE, bar, pol_keep);
+          if (lane < nbx) {
+            const uint32_t dst = base + (uint32_t)(u % MP_RING) * MP_SLOT + (uint32_t)(lane * page_run) * MP_BOX;
+            if (page_run == 4)   // block-major runs: rows of 64 dims, block j of run r = rows ((r * blocks + j) * 64 ..
+              tma_load_2d(dst, &tmC, 0, ((bpage >> 2) * (NLB + 1) + j) * 64, bar, pol_keep);
+            else
+              tma_load_2d(dst, &tmC, j < NLB ? 64 * j : d_c, bpage * MP_PAGE, bar, pol_keep);
+          }
         }
       }
       if (it > item_lo && !failed) {                     // the previous item's latent once more, page-major
@@ -244,8 +248,11 @@ mla_paged_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
           const uint32_t bar = smem_u32(&full_bar[u % MP_RING]);
           if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)(cnt * page_run * BPH * MP_BOX));
           __syncwarp();
-          if (lane < cnt)
-            tma_load_4d(base + (uint32_t)(u % MP_RING) * MP_SLOT + (uint32_t)(lane * BPH) * MP_BOX, &tmV, 0, 0, half * BPH, pg * 2, bar, pol_drop);
+          if (lane < cnt) {
+            const uint32_t dst = base + (uint32_t)(u % MP_RING) * MP_SLOT + (uint32_t)(lane * BPH) * MP_BOX;
+            if (page_run == 4) tma_load_5d(dst, &tmV, 0, 0, half * BPH, 0, pg >> 2, bar, pol_drop);
+            else tma_load_4d(dst, &tmV, 0, 0, half * BPH, pg * 2, bar, pol_drop);
+          }
         }
       }
       prev_page = page;
@@ -584,18 +591,32 @@ long long mla_part_o_floats(int R, int nh, int rank, int max_context) { return (
 
 int mla_encode_maps(CUtensorMap *tmC, CUtensorMap *tmV, const void *pool, long long pool_pages, int rank, int rope, int page_run) {
   if (pool_pages < 1 || pool_pages * MP_PAGE >= (1ll << 31) || (page_run != 1 && page_run != 4)) return CORUN_EINVAL;
+  const int bph = rank > 256 ? 4 : rank / 64;
+  if (page_run == 4) {
+    // block-major runs of 64 tokens: [run][block of 64 dims][64 tokens][64 dims].  Score pass: the pool as rows of 64
+    // halfs, one [64 x 64] box = a block of a run, 8 KiB of contiguous memory.  Output pass: one box fetches a run's
+    // 64 tokens x (up to) 256 dims as [8 groups][blocks][8 tokens][64 dims], the layout of an MN-major MMA operand.
+    if (pool_pages % 4) return CORUN_EINVAL;
+    const unsigned long long runs = (unsigned long long)pool_pages / 4, nblk = (unsigned long long)(rank + rope + 63) / 64;
+    if (runs * nblk * 64 >= (1ull << 31)) return CORUN_EINVAL;
+    const unsigned long long d2[2] = {64, runs * nblk * 64}, s2[1] = {128};
+    const unsigned b2[2] = {64, 64};
+    int rc = tma_encode_fp16_nd(tmC, pool, 2, d2, s2, b2);
+    if (rc != CORUN_OK) return rc;
+    const unsigned long long d5[5] = {64, 8, nblk, 8, runs}, s5[4] = {128, 64 * 128, 8 * 128, nblk * 64 * 128};
+    const unsigned b5[5] = {64, 8, (unsigned)bph, 8, 1};
+    return tma_encode_fp16_nd(tmV, pool, 5, d5, s5, b5);
+  }
   // the pool as rows of rank + rope halfs, fetched in [16 tokens x 64 dims] boxes (the rope box reads past the
   // row's end when rope < 64: those columns arrive as zeros)
-  int rc = tma_encode_2d(tmC, pool, 1, (unsigned long long)pool_pages * MP_PAGE, rank + rope, MP_PAGE * page_run, 64);
+  int rc = tma_encode_2d(tmC, pool, 1, (unsigned long long)pool_pages * MP_PAGE, rank + rope, MP_PAGE, 64);
   if (rc != CORUN_OK) return rc;
   // the latent part once more as [8-token group][token in group][block of 64 dims][64 dims]: one box fetches a page's
   // 16 tokens x (up to) 256 dims as [2 groups][blocks][8 tokens][64 dims], the layout of an MN-major MMA operand
-  // (page_run = 4: boxes of four consecutive pages: [64 tokens x 64 dims] and [8 groups][blocks][8 tokens][64 dims])
-  const int bph = rank > 256 ? 4 : rank / 64;
   const unsigned long long row_bytes = (unsigned long long)(rank + rope) * 2;
   const unsigned long long dims[4] = {64, 8, (unsigned long long)(rank / 64), (unsigned long long)pool_pages * 2};
   const unsigned long long strides[3] = {row_bytes, 128, 8 * row_bytes};
-  const unsigned box[4] = {64, 8, (unsigned)bph, 2u * (unsigned)page_run};
+  const unsigned box[4] = {64, 8, (unsigned)bph, 2};
   return tma_encode_fp16_4d(tmV, pool, dims, strides, box);
 }
 
