@@ -1,6 +1,8 @@
 """The engine with multi-head latent attention layers (a dense first layer, expert layers behind it): prefill and
 teacher-forced decode steps against the C oracle, bitwise invariance to slot, co-tenants and batched prefill, and
 the DeepSeek-V2-Lite layer shape at full width."""
+import os
+
 import numpy as np
 import pytest
 
@@ -112,7 +114,7 @@ def test_mla_engine_with_more_than_64_slots(orc):
     sh, Bw = SMALL, 80
     model, eng = _setup(orc, sh, dict(SMALL_MLA), SMALL_MOE, seed=6, B=Bw, max_ctx=128)
     try:
-        assert eng.decode_launches() == 6 + 13 + 16 * (sh.n_layers - 1)
+        assert eng.decode_launches() == 6 + 13 + (13 if os.environ.get("CORUN_MOE_DECODE_DENSE") else 16) * (sh.n_layers - 1)
         prompts = synth.make_prompts(sh.vocab, [30, 77, 12, 50], seed=6)
         seeds = np.zeros(Bw, np.uint64)
         traces = []
