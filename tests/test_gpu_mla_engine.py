@@ -250,3 +250,33 @@ def test_mla_engine_argument_errors(orc):
     for bad in (dict(kv_lora_rank=128), dict(qk_nope=96), dict(qk_rope=20), dict(v_head=64), dict(first_dense=1)):
         with pytest.raises(corun.CorunError):        # first_dense below the layer count needs expert layers
             corun.Engine(sh, w_t, 4, 64, mla=dict(m_t, **bad))
+
+
+def test_mla_cache_blocks_of_64_tokens_are_accounted_in_blocks(orc):
+    """kv_block = 64: the pool is sized, handed out and counted in blocks of 64 tokens (four 16-token pages in a row);
+    the cache rows read back are the oracle's wherever the block boundaries fall."""
+    sh = SMALL
+    model, eng = _setup(orc, sh, dict(SMALL_MLA), SMALL_MOE, seed=8, B=8, max_ctx=256, kv_block=64, kv_pool_blocks=10)
+    try:
+        assert eng.free_blocks() == 10
+        prompts = synth.make_prompts(sh.vocab, [70, 9, 130], seed=12)
+        eng.prefill(1, prompts[0], 78)                      # 78 tokens reserved: two blocks
+        assert eng.free_blocks() == 8
+        eng.prefill(5, prompts[1], 64)                      # exactly one block
+        assert eng.free_blocks() == 7
+        eng.prefill(2, prompts[2], 200)                     # four blocks
+        assert eng.free_blocks() == 3
+        with pytest.raises(Exception):
+            eng.prefill(3, prompts[0], 64 * 4)              # four more do not fit
+        assert eng.free_blocks() == 3
+        r = orc.Request(model, prompts[2], 1, max_T=256)
+        r.prefill()
+        got = eng.kv_read(2, 1, 0, 130)[0]                  # layer 1, positions 0..129: across three blocks of 64
+        ref = r.cache[0][1, :130]
+        assert got.shape == ref.shape and float(np.abs(got - ref).max()) <= 2e-2
+        eng.release(2)
+        assert eng.free_blocks() == 7
+        eng.release(1); eng.release(5)
+        assert eng.free_blocks() == 10
+    finally:
+        eng.close()
