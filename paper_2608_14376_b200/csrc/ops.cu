@@ -9,6 +9,8 @@
 #include "ptx.cuh"
 
 #include <cooperative_groups.h>
+
+#include <cstdlib>
 #include <math_constants.h>
 
 namespace corun {
@@ -413,7 +415,7 @@ __device__ __noinline__ void smp_tail_full_row(SmpShared &sh, const SampleArgs &
   }
 }
 
-// Sampling S (top-p nucleus + inverse CDF) of one row per cluster of SMP_CLUSTER CTAs, all in integers
+// Sampling S (top-p nucleus + inverse CDF) of one row per cluster of 1..8 CTAs (a launch attribute), all in integers
 // once the weights are formed, so the result does not depend on the order in which threads meet the
 // tokens.  Every CTA takes a contiguous slice of the row; the first CTA of the cluster merges what the
 // slices found (through distributed shared memory) and takes the decisions.  Four passes over the row:
@@ -421,20 +423,21 @@ __device__ __noinline__ void smp_tail_full_row(SmpShared &sh, const SampleArgs &
 // the running weight reaches the cut (the nucleus edge is then found among those few tokens in shared
 // memory); per-warp totals of the nucleus weights in id order, after which one warp walks its range to
 // the drawn token.
-constexpr int SMP_CLUSTER = 6;
+constexpr int SMP_MAX_CLUSTER = 8;   // the cluster size is a launch attribute (launch_sampler): 2..8 CTAs per row
 
-__global__ void __cluster_dims__(SMP_CLUSTER, 1, 1) __launch_bounds__(SMP_THREADS, 2) sampler_kernel(SampleArgs a) {
+__global__ void __launch_bounds__(SMP_THREADS, 2) sampler_kernel(SampleArgs a) {
   namespace cg = cooperative_groups;
   griddep_launch_dependents();
   griddep_wait();
+  cg::cluster_group cluster = cg::this_cluster();
+  const int SMP_CLUSTER = (int)cluster.num_blocks();   // CTAs per row (no value depends on it: integer arithmetic)
   const int r = blockIdx.x / SMP_CLUSTER;
   if (!a.do_sample[r]) return;                     // the same for the whole cluster
-  cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
   __shared__ SmpShared sh;
-  SmpShared *peer[SMP_CLUSTER];
+  SmpShared *peer[SMP_MAX_CLUSTER];
 #pragma unroll
-  for (int k = 0; k < SMP_CLUSTER; ++k) peer[k] = cluster.map_shared_rank(&sh, k);
+  for (int k = 0; k < SMP_MAX_CLUSTER; ++k) peer[k] = cluster.map_shared_rank(&sh, k < SMP_CLUSTER ? k : 0);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int V = a.V;
   const float *lg = a.logits + (size_t)r * V;
@@ -466,7 +469,8 @@ __global__ void __cluster_dims__(SMP_CLUSTER, 1, 1) __launch_bounds__(SMP_THREAD
   cluster.sync();
   bv = peer[0]->loc_val; bi = peer[0]->loc_idx;
 #pragma unroll
-  for (int k = 1; k < SMP_CLUSTER; ++k) {
+  for (int k = 1; k < SMP_MAX_CLUSTER; ++k) {
+    if (k >= SMP_CLUSTER) break;
     const float ov = peer[k]->loc_val;
     const int oi = peer[k]->loc_idx;
     if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
@@ -502,11 +506,13 @@ __global__ void __cluster_dims__(SMP_CLUSTER, 1, 1) __launch_bounds__(SMP_THREAD
   if (rank == 0) {
     unsigned long long total = 0ull;
 #pragma unroll
-    for (int k = 0; k < SMP_CLUSTER; ++k) total += peer[k]->loc_total;
+    for (int k = 0; k < SMP_MAX_CLUSTER; ++k)
+      if (k < SMP_CLUSTER) total += peer[k]->loc_total;
     for (int i = tid; i < SMP_BINS; i += SMP_THREADS) {
       unsigned long long h = sh.hist[i];
 #pragma unroll
-      for (int k = 1; k < SMP_CLUSTER; ++k) h += peer[k]->hist[i];
+      for (int k = 1; k < SMP_MAX_CLUSTER; ++k)
+        if (k < SMP_CLUSTER) h += peer[k]->hist[i];
       sh.hist[i] = h;
     }
     __syncthreads();
@@ -532,10 +538,11 @@ __global__ void __cluster_dims__(SMP_CLUSTER, 1, 1) __launch_bounds__(SMP_THREAD
   if (rank == 0) {
     // gather the other slices' candidates behind this slice's
     unsigned int n_all = sh.n_cand, kmin = sh.kmin, kmax = sh.kmax;
-    unsigned int off[SMP_CLUSTER];
+    unsigned int off[SMP_MAX_CLUSTER];
     off[0] = 0u;
 #pragma unroll
-    for (int k = 1; k < SMP_CLUSTER; ++k) {
+    for (int k = 1; k < SMP_MAX_CLUSTER; ++k) {
+      if (k >= SMP_CLUSTER) break;
       off[k] = n_all;
       n_all += peer[k]->n_cand;
       kmin = min(kmin, peer[k]->kmin);
@@ -546,7 +553,8 @@ __global__ void __cluster_dims__(SMP_CLUSTER, 1, 1) __launch_bounds__(SMP_THREAD
     if (tid == 0) { sh.sel_cnt = n_all; sh.bc_overflow = n_cand > SMP_CAND ? 1 : 0; }   // sel_cnt stands if no refinement is needed
     if (n_cand <= SMP_CAND) {
 #pragma unroll
-      for (int k = 1; k < SMP_CLUSTER; ++k) {
+      for (int k = 1; k < SMP_MAX_CLUSTER; ++k) {
+        if (k >= SMP_CLUSTER) break;
         const int nk = (int)(k + 1 < SMP_CLUSTER ? off[k + 1] : n_all) - (int)off[k];
         for (int c = tid; c < nk; c += SMP_THREADS) {
           sh.cand_x[off[k] + c] = peer[k]->cand_x[c];
@@ -879,7 +887,29 @@ cudaError_t launch_split(const float *x, int R, int K, __nv_bfloat16 *hi, __nv_b
 }
 
 cudaError_t launch_sampler(const SampleArgs &a, int R, cudaStream_t st, bool pdl) {
-  return launch_k(sampler_kernel, dim3(R * SMP_CLUSTER), dim3(SMP_THREADS), 0, st, pdl, a);
+  // CTAs per row: more CTAs shorten a row's passes, fewer keep all rows' clusters resident at once (two CTAs per SM:
+  // 296 in all).  Measured (vocabulary 151 936; 2 / 3 / 4 / 5 / 6 / 7 CTAs per row): 40 sampled rows 90.8 / 70.2 / 85.6 /
+  // 73.1 / 72.1 / 98.1 us, 64 rows 90.5 / 101.2 / 89.0 / 111.8 / 111.6 / 124.3 us, 128 rows 141.0 / 153.9 / 165.2 / 175.5 /
+  // 193.2 / 226.5 us.  The launch shape is fixed in the step's graph, so it follows the padded row count.
+  int nc = R <= 16 ? 6 : R <= 64 ? 3 : 2;
+  if (const char *c = getenv("CORUN_SAMPLER_CLUSTER")) {   // (timing experiments)
+    const int v = atoi(c);
+    if (v >= 1 && v <= SMP_MAX_CLUSTER) nc = v;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(R * nc);
+  cfg.blockDim = dim3(SMP_THREADS);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = nc;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = (pdl && g_use_pdl) ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, sampler_kernel, a);
 }
 
 cudaError_t launch_prepare_rows(const uint8_t *active_mask, const uint64_t *seeds_in, uint64_t *seeds_out, const int *in_use,
