@@ -280,3 +280,47 @@ def test_mla_cache_blocks_of_64_tokens_are_accounted_in_blocks(orc):
         assert eng.free_blocks() == 10
     finally:
         eng.close()
+
+
+@pytest.mark.parametrize("kv_block", [16, 64])
+def test_mla_engine_full_house_changes_no_byte(orc, kv_block):
+    """Three requests alone and among co-tenants in nearly every other slot of an 80-slot engine (rows in both blocks
+    of the 65..128-row GEMMs, two row blocks per head in the grouped up-projections, expert groups of more than one
+    block): the same bytes, and the oracle's values; with 16-token pages and with blocks of 64 tokens."""
+    sh, Bw = SMALL, 80
+    model, eng = _setup(orc, sh, dict(SMALL_MLA), SMALL_MOE, seed=6, B=Bw, max_ctx=128, kv_block=kv_block)
+    try:
+        prompts = synth.make_prompts(sh.vocab, [30, 77, 12], seed=6)
+        tested = [41, 5, 77]
+        others = [s for s in range(Bw) if s not in tested][: Bw - 8]
+        fill = synth.make_prompts(sh.vocab, [9 + (i * 7) % 40 for i in range(len(others))], seed=78)
+        seeds = np.zeros(Bw, np.uint64)
+        traces = []
+        for crowd in (False, True):
+            reqs = [orc.Request(model, p, 1, max_T=128) for p in prompts]
+            for s, p, r in zip(tested, prompts, reqs):
+                r.prefill()
+                eng.prefill(s, p, len(p) + 8)
+            active = np.zeros(Bw, np.uint8); active[tested] = 1
+            if crowd:
+                for s, p in zip(others, fill):
+                    eng.prefill(s, p, len(p) + 8)
+                active[others] = 1
+            worst, trace = 0.0, []
+            for _ in range(3):
+                toks = [int(np.argmax(r.logits)) for r in reqs]
+                for s, t in zip(tested, toks):
+                    eng.force_token(s, t)
+                eng.decode_step(active, seeds)
+                for s, r, t in zip(tested, reqs, toks):
+                    r.decode(force_token=t)
+                    worst = max(worst, float(np.abs(eng.logits(s) - r.logits).max()))
+                trace.append([eng.logits(s).tobytes() for s in tested])
+            assert worst <= TOL, worst
+            traces.append(trace)
+            for s in range(Bw):
+                if active[s]:
+                    eng.release(s)
+        assert traces[0] == traces[1]
+    finally:
+        eng.close()

@@ -141,6 +141,58 @@ def test_moe_engine_with_more_than_64_slots(orc):
         eng.close()
 
 
+@pytest.mark.parametrize("Bw", [96, 200])
+def test_moe_engine_full_house_changes_no_byte(orc, Bw):
+    """The tested requests alone (three rows: one block of rows, a few small expert groups) and among co-tenants in
+    nearly every other slot (rows in every block of 64 / 128 rows, expert groups of several blocks, the tested requests
+    somewhere in the middle of the step's rows): the same bytes, and the oracle's values."""
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2608_14376_b200 import corun
+
+    sh = synth.TINY
+    w_np = synth.make_weights_numpy(sh, seed=4)
+    m_np = synth.make_moe_numpy(sh, 8, 2, 128, 1, False, seed=4)
+    model = orc.Model(orc.Shape(**sh.dict()), w_np, moe=m_np)
+    eng = corun.Engine(sh, synth.weights_numpy_to_torch(w_np, "cuda"), Bw, MAX_CTX, moe=synth.moe_numpy_to_torch(m_np, "cuda"))
+    try:
+        prompts = synth.make_prompts(sh.vocab, [30, 77, 12], seed=6)
+        tested = [Bw // 2 + 1, 5, Bw - 3]
+        others = [s for s in range(Bw) if s not in tested][: Bw - 8]
+        fill = synth.make_prompts(sh.vocab, [9 + (i * 7) % 40 for i in range(len(others))], seed=77)
+        seeds = np.zeros(Bw, np.uint64)
+        traces = []
+        for crowd in (False, True):
+            reqs = [orc.Request(model, p, 1, max_T=MAX_CTX) for p in prompts]
+            for s, p, r in zip(tested, prompts, reqs):
+                r.prefill()
+                eng.prefill(s, p, len(p) + 8)
+            active = np.zeros(Bw, np.uint8); active[tested] = 1
+            if crowd:
+                for s, p in zip(others, fill):
+                    eng.prefill(s, p, len(p) + 8)
+                active[others] = 1
+            worst, trace = 0.0, []
+            for _ in range(3):
+                toks = [int(np.argmax(r.logits)) for r in reqs]
+                for s, t in zip(tested, toks):
+                    eng.force_token(s, t)
+                eng.decode_step(active, seeds)
+                for s, r, t in zip(tested, reqs, toks):
+                    r.decode(force_token=t)
+                    worst = max(worst, float(np.abs(eng.logits(s) - r.logits).max()))
+                trace.append([eng.logits(s).tobytes() for s in tested])
+            assert worst <= TOL, worst
+            traces.append(trace)
+            for s in range(Bw):
+                if active[s]:
+                    eng.release(s)
+        assert traces[0] == traces[1]
+    finally:
+        eng.close()
+
+
 def test_moe_engine_served_together_equals_served_alone(orc):
     """The paper's validation protocol on the MoE decoder: requests served together (sampled, through the host
     scheduler with a pool too small for all of them) produce, bit for bit, the tokens of each served alone."""
